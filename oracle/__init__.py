@@ -1,0 +1,158 @@
+"""ctypes front end of the CPU oracle.  TEST INFRASTRUCTURE ONLY.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this
+package; the CUDA library and its Python binding never do.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from typing import List, Sequence, Tuple
+
+import numpy as np
+
+from .build import build as _build
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        L = C.CDLL(_build())
+        vp, i32, i64, u64, f32, f64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64, C.c_float, C.c_double
+        L.oracle_create.restype = vp
+        L.oracle_create.argtypes = [vp, i32, i32, f64, f32, u64]
+        L.oracle_destroy.argtypes = [vp]
+        L.oracle_step.argtypes = [vp, vp, vp, vp]
+        L.oracle_reset.argtypes = [vp]
+        L.oracle_set_threads.argtypes = [vp, i32]
+        L.oracle_threads_used.argtypes = [vp]
+        L.oracle_threads_used.restype = i32
+        L.oracle_set_leader_override.argtypes = [vp, i32]
+        L.oracle_total.argtypes = [vp]
+        L.oracle_total.restype = i64
+        L.oracle_total_keep.argtypes = [vp]
+        L.oracle_total_keep.restype = i64
+        L.oracle_get_step.argtypes = [vp]
+        L.oracle_get_step.restype = i64
+        L.oracle_get_leader.argtypes = [vp]
+        L.oracle_get_leader.restype = i32
+        L.oracle_get_layout.argtypes = [vp, vp, vp]
+        L.oracle_get_residual.argtypes = [vp, i32, vp]
+        L.oracle_set_residual.argtypes = [vp, i32, vp]
+        L.oracle_get_selection.argtypes = [vp, i32, vp, vp]
+        L.oracle_get_mask.argtypes = [vp, vp]
+        L.oracle_leader.argtypes = [u64, u64, i32]
+        L.oracle_leader.restype = i32
+        L.oracle_mix64.argtypes = [u64]
+        L.oracle_mix64.restype = u64
+        L.oracle_keep_count.argtypes = [i64, f64]
+        L.oracle_keep_count.restype = i64
+        L.oracle_importance_bits.argtypes = [f32, f32, f32]
+        L.oracle_importance_bits.restype = C.c_uint32
+        L.oracle_select.argtypes = [vp, vp, i64, i64, f32, vp]
+        _lib = L
+    return _lib
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def leader(seed: int, t: int, W: int) -> int:
+    return int(lib().oracle_leader(seed, t, W))
+
+
+def mix64(z: int) -> int:
+    return int(lib().oracle_mix64(z))
+
+
+def keep_count(n: int, ratio: float) -> int:
+    return int(lib().oracle_keep_count(n, ratio))
+
+
+def importance_bits(acc: float, w: float, eps: float) -> int:
+    return int(lib().oracle_importance_bits(acc, w, eps))
+
+
+def select(acc: np.ndarray, w: np.ndarray, k: int, eps: float) -> np.ndarray:
+    acc = np.ascontiguousarray(acc, dtype=np.float32)
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    out = np.empty(k, dtype=np.uint32)
+    lib().oracle_select(_p(acc), _p(w), acc.size, k, eps, _p(out))
+    return out
+
+
+class Oracle:
+    """W simulated workers' residuals on the host and the step that updates them."""
+
+    def __init__(self, layer_sizes: Sequence[int], W: int, ratio: float, eps: float, seed: int, threads: int = 0):
+        ls = np.asarray(list(layer_sizes), dtype=np.int64)
+        self._h = lib().oracle_create(_p(ls), len(ls), W, float(ratio), float(eps), int(seed))
+        if not self._h:
+            raise ValueError("oracle_create rejected the arguments")
+        self.L, self.W = len(ls), W
+        self.N = int(lib().oracle_total(self._h))
+        self.K = int(lib().oracle_total_keep(self._h))
+        if threads:
+            lib().oracle_set_threads(self._h, threads)
+
+    def close(self):
+        if self._h:
+            lib().oracle_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
+
+    @property
+    def threads(self) -> int:
+        return int(lib().oracle_threads_used(self._h))
+
+    def layout(self) -> Tuple[List[int], List[int]]:
+        off = np.empty(self.L, dtype=np.int64)
+        k = np.empty(self.L, dtype=np.int64)
+        lib().oracle_get_layout(self._h, _p(off), _p(k))
+        return off.tolist(), k.tolist()
+
+    def set_leader_override(self, leader: int):
+        lib().oracle_set_leader_override(self._h, leader)
+
+    def reset(self):
+        lib().oracle_reset(self._h)
+
+    def step(self, grads: np.ndarray, weights: np.ndarray) -> np.ndarray:
+        assert grads.dtype == np.float32 and grads.flags.c_contiguous and grads.size == self.W * self.N
+        assert weights.dtype == np.float32 and weights.flags.c_contiguous and weights.size == self.N
+        update = np.empty(self.N, dtype=np.float32)
+        lib().oracle_step(self._h, _p(grads), _p(weights), _p(update))
+        return update
+
+    @property
+    def t(self) -> int:
+        return int(lib().oracle_get_step(self._h))
+
+    @property
+    def leader(self) -> int:
+        return int(lib().oracle_get_leader(self._h))
+
+    def residual(self, w: int) -> np.ndarray:
+        out = np.empty(self.N, dtype=np.float32)
+        lib().oracle_get_residual(self._h, w, _p(out))
+        return out
+
+    def set_residual(self, w: int, src: np.ndarray):
+        src = np.ascontiguousarray(src, dtype=np.float32)
+        assert src.size == self.N
+        lib().oracle_set_residual(self._h, w, _p(src))
+
+    def selection(self, w: int) -> Tuple[np.ndarray, np.ndarray]:
+        idx = np.empty(self.K, dtype=np.uint32)
+        val = np.empty(self.K, dtype=np.float32)
+        lib().oracle_get_selection(self._h, w, _p(idx), _p(val))
+        return idx, val
+
+    def mask(self) -> np.ndarray:
+        m = np.empty(self.N, dtype=np.uint8)
+        lib().oracle_get_mask(self._h, _p(m))
+        return m

@@ -1,0 +1,282 @@
+// CPU oracle for the importance-weighted-pruning step.   TEST INFRASTRUCTURE ONLY.
+//
+// A plain, slow, obviously-correct statement of what one data-parallel step of the
+// paper's method computes for W simulated workers, written from the paper's
+// Algorithm 1 and Section 3.2.  It shares no code, header, table or constant with
+// the CUDA library and must never be linked, imported or called by it; only the
+// tests, the smoke check and the benchmark's CPU-baseline leg may use it.
+//
+// Where the selection has a plain definition (the k best elements of a layer under
+// a total order) the oracle is that definition: order the layer by (importance
+// descending, index ascending) with a library partial-ordering routine and keep the
+// first k.  There is no radix select, no histogram, no blocking or fusion here.
+//
+// Arithmetic: IEEE-754 binary32, round to nearest even, one operation at a time
+// (build with -ffp-contract=off, never -ffast-math), denormals kept.
+//
+// Readings of points the paper leaves open (the same readings bind the CUDA path):
+//   * Algorithm 1's first update line is the residual accumulator G += grad, and the
+//     importance is taken on the accumulated value (Section 3.2: the residual is
+//     accumulated locally).
+//   * importance = |G| / (|w| + eps), eps > 0, instead of the unguarded |G / w|.
+//   * the threshold of Algorithm 1 is the k-th largest importance of the worker's
+//     layer, k = ceil(n / ratio) clamped to [1, n]; ties keep the lower index.
+//   * one randomly chosen node per step supplies the index set (Section 3.2:
+//     "randomly choose a node and broadcast its important gradient index").
+//   * the ring all-reduce is a sum in ascending worker order, fp32, without the 1/N
+//     factor (the caller pre-scales gradients as in Eq. 1).
+//
+// Pins: tests/test_oracle_*.py check this file against brute-force full sorts in
+// pure Python, a hand-worked two-step example, closed forms, conservation
+// invariants, numpy/torch library routines for the threshold value, the dense
+// all-reduce special case (ratio = 1) and printed leader test vectors.
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <numeric>
+#include <vector>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+namespace {
+
+struct Oracle {
+  std::vector<int64_t> n;    // layer sizes
+  std::vector<int64_t> off;  // flat offsets
+  std::vector<int64_t> k;    // keep count per layer
+  std::vector<int64_t> koff; // offset of the layer's segment inside a worker's list
+  int64_t N = 0, K = 0;
+  int32_t W = 0;
+  double ratio = 1.0;
+  float eps = 0.f;
+  uint64_t seed = 0;
+  int64_t t = 0;
+  int32_t leader = -1;
+  int32_t leader_override = -1;
+  int threads = 0;
+  std::vector<float> acc;        // [W][N] residuals
+  std::vector<uint32_t> sel_idx; // [W][K] ascending global indices per layer segment
+  std::vector<float> sel_val;    // [W][K] accumulated value at that index (before zeroing)
+};
+
+inline uint32_t bits_of(float x) {
+  uint32_t u;
+  std::memcpy(&u, &x, 4);
+  return u;
+}
+
+// Algorithm 1, mask line: |grad / weight|, guarded with eps.
+inline float importance(float acc, float w, float eps) {
+  float den = std::fabs(w) + eps;
+  return std::fabs(acc) / den;
+}
+
+// keep count: ceil(n / R) in double, clamped to [1, n]
+inline int64_t keep_count(int64_t n, double R) {
+  double q = std::ceil(static_cast<double>(n) / R);
+  int64_t k = static_cast<int64_t>(q);
+  if (k < 1) k = 1;
+  if (k > n) k = n;
+  return k;
+}
+
+inline uint64_t mix64(uint64_t z) {
+  z ^= z >> 30;
+  z *= 0xBF58476D1CE4E5B9ull;
+  z ^= z >> 27;
+  z *= 0x94D049BB133111EBull;
+  z ^= z >> 31;
+  return z;
+}
+
+// the randomly chosen node of step t (0-based)
+inline int32_t leader_of(uint64_t seed, uint64_t t, int32_t W) {
+  uint64_t z = mix64(seed + (t + 1) * 0x9E3779B97F4A7C15ull);
+  uint64_t hi = z >> 32;
+  return static_cast<int32_t>((hi * static_cast<uint64_t>(W)) >> 32);
+}
+
+// Selection of one (worker, layer): indices (local to the layer) of the k elements
+// that come first under (importance descending, index ascending), returned ascending.
+void select_layer(const float* acc, const float* w, int64_t n, int64_t k, float eps,
+                  std::vector<uint32_t>& keys, std::vector<uint32_t>& order) {
+  keys.resize(n);
+  order.resize(n);
+  for (int64_t i = 0; i < n; ++i) keys[i] = bits_of(importance(acc[i], w[i], eps));
+  std::iota(order.begin(), order.end(), 0u);
+  auto before = [&](uint32_t a, uint32_t b) {
+    if (keys[a] != keys[b]) return keys[a] > keys[b];
+    return a < b;
+  };
+  if (k < n) std::nth_element(order.begin(), order.begin() + (k - 1), order.end(), before);
+  order.resize(k);
+  std::sort(order.begin(), order.end());
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t oracle_leader(uint64_t seed, uint64_t t, int32_t W) { return leader_of(seed, t, W); }
+uint64_t oracle_mix64(uint64_t z) { return mix64(z); }
+int64_t oracle_keep_count(int64_t n, double R) { return keep_count(n, R); }
+uint32_t oracle_importance_bits(float acc, float w, float eps) { return bits_of(importance(acc, w, eps)); }
+
+// Stand-alone selection of one layer (used by the brute-force pins).
+void oracle_select(const float* acc, const float* w, int64_t n, int64_t k, float eps, uint32_t* out_idx) {
+  std::vector<uint32_t> keys, order;
+  select_layer(acc, w, n, k, eps, keys, order);
+  std::copy(order.begin(), order.end(), out_idx);
+}
+
+void* oracle_create(const int64_t* layer_sizes, int32_t n_layers, int32_t W, double ratio, float eps,
+                    uint64_t seed) {
+  if (!layer_sizes || n_layers < 1 || W < 1 || !(ratio >= 1.0) || !std::isfinite(ratio) || !(eps > 0.f) ||
+      !std::isfinite(eps))
+    return nullptr;
+  Oracle* o = new Oracle;
+  o->W = W;
+  o->ratio = ratio;
+  o->eps = eps;
+  o->seed = seed;
+  for (int32_t l = 0; l < n_layers; ++l) {
+    if (layer_sizes[l] < 1) {
+      delete o;
+      return nullptr;
+    }
+    o->n.push_back(layer_sizes[l]);
+    o->off.push_back(o->N);
+    o->k.push_back(keep_count(layer_sizes[l], ratio));
+    o->koff.push_back(o->K);
+    o->N += layer_sizes[l];
+    o->K += o->k.back();
+  }
+  if (o->N >= (int64_t(1) << 32)) {
+    delete o;
+    return nullptr;
+  }
+  o->acc.assign(static_cast<size_t>(W) * o->N, 0.0f);
+  o->sel_idx.assign(static_cast<size_t>(W) * o->K, 0u);
+  o->sel_val.assign(static_cast<size_t>(W) * o->K, 0.0f);
+  return o;
+}
+
+void oracle_destroy(void* h) { delete static_cast<Oracle*>(h); }
+
+void oracle_set_threads(void* h, int32_t threads) { static_cast<Oracle*>(h)->threads = threads; }
+int32_t oracle_threads_used(void* h) {
+#ifdef _OPENMP
+  Oracle* o = static_cast<Oracle*>(h);
+  return o->threads > 0 ? o->threads : omp_get_max_threads();
+#else
+  (void)h;
+  return 1;
+#endif
+}
+void oracle_set_leader_override(void* h, int32_t leader) { static_cast<Oracle*>(h)->leader_override = leader; }
+int64_t oracle_total(void* h) { return static_cast<Oracle*>(h)->N; }
+int64_t oracle_total_keep(void* h) { return static_cast<Oracle*>(h)->K; }
+int64_t oracle_get_step(void* h) { return static_cast<Oracle*>(h)->t; }
+int32_t oracle_get_leader(void* h) { return static_cast<Oracle*>(h)->leader; }
+
+void oracle_get_layout(void* h, int64_t* off, int64_t* k) {
+  Oracle* o = static_cast<Oracle*>(h);
+  for (size_t l = 0; l < o->n.size(); ++l) {
+    off[l] = o->off[l];
+    k[l] = o->k[l];
+  }
+}
+
+void oracle_reset(void* h) {
+  Oracle* o = static_cast<Oracle*>(h);
+  std::fill(o->acc.begin(), o->acc.end(), 0.0f);
+  o->t = 0;
+  o->leader = -1;
+}
+
+void oracle_set_residual(void* h, int32_t w, const float* src) {
+  Oracle* o = static_cast<Oracle*>(h);
+  std::memcpy(&o->acc[static_cast<size_t>(w) * o->N], src, sizeof(float) * o->N);
+}
+
+void oracle_get_residual(void* h, int32_t w, float* dst) {
+  Oracle* o = static_cast<Oracle*>(h);
+  std::memcpy(dst, &o->acc[static_cast<size_t>(w) * o->N], sizeof(float) * o->N);
+}
+
+void oracle_get_selection(void* h, int32_t w, uint32_t* idx, float* val) {
+  Oracle* o = static_cast<Oracle*>(h);
+  std::memcpy(idx, &o->sel_idx[static_cast<size_t>(w) * o->K], sizeof(uint32_t) * o->K);
+  std::memcpy(val, &o->sel_val[static_cast<size_t>(w) * o->K], sizeof(float) * o->K);
+}
+
+// one byte per element, 1 where the element is in the index set of the last step
+void oracle_get_mask(void* h, uint8_t* dst) {
+  Oracle* o = static_cast<Oracle*>(h);
+  std::memset(dst, 0, o->N);
+  if (o->leader < 0) return;
+  const uint32_t* S = &o->sel_idx[static_cast<size_t>(o->leader) * o->K];
+  for (int64_t j = 0; j < o->K; ++j) dst[S[j]] = 1;
+}
+
+// One step.  grads[W][N], weights[N], update[N]: host pointers.
+void oracle_step(void* h, const float* grads, const float* weights, float* update) {
+  Oracle* o = static_cast<Oracle*>(h);
+  const int64_t N = o->N, K = o->K;
+  const int32_t W = o->W;
+  const int L = static_cast<int>(o->n.size());
+#ifdef _OPENMP
+  const int nthreads = o->threads > 0 ? o->threads : omp_get_max_threads();
+#endif
+
+  // (a) accumulate the new gradient into the local residual
+#pragma omp parallel for num_threads(nthreads) schedule(static)
+  for (int64_t e = 0; e < static_cast<int64_t>(W) * N; ++e) o->acc[e] = o->acc[e] + grads[e];
+
+  // (b)-(d) per worker and layer: importance, keep the k best, list them in index order
+#pragma omp parallel num_threads(nthreads)
+  {
+    std::vector<uint32_t> keys, order;
+#pragma omp for schedule(dynamic, 1)
+    for (int64_t p = 0; p < static_cast<int64_t>(W) * L; ++p) {
+      // large layers first within a worker does not matter for correctness
+      const int32_t w = static_cast<int32_t>(p / L);
+      const int l = static_cast<int>(p % L);
+      const float* a = &o->acc[static_cast<size_t>(w) * N + o->off[l]];
+      select_layer(a, weights + o->off[l], o->n[l], o->k[l], o->eps, keys, order);
+      uint32_t* li = &o->sel_idx[static_cast<size_t>(w) * K + o->koff[l]];
+      float* lv = &o->sel_val[static_cast<size_t>(w) * K + o->koff[l]];
+      for (int64_t j = 0; j < o->k[l]; ++j) {
+        li[j] = static_cast<uint32_t>(o->off[l] + order[j]);
+        lv[j] = a[order[j]];
+      }
+    }
+  }
+
+  // (e) the randomly chosen node supplies the index set
+  o->leader = o->leader_override >= 0 ? o->leader_override : leader_of(o->seed, static_cast<uint64_t>(o->t), W);
+  const uint32_t* S = &o->sel_idx[static_cast<size_t>(o->leader) * K];
+
+  // (f) sum over workers in ascending order at the shared indices, into a zeroed dense update
+#pragma omp parallel for num_threads(nthreads) schedule(static)
+  for (int64_t i = 0; i < N; ++i) update[i] = 0.0f;
+#pragma omp parallel for num_threads(nthreads) schedule(static)
+  for (int64_t j = 0; j < K; ++j) {
+    const size_t i = S[j];
+    float s = o->acc[i];
+    for (int32_t w = 1; w < W; ++w) s = s + o->acc[static_cast<size_t>(w) * N + i];
+    update[i] = 0.0f + s;
+  }
+
+  // (g) what was sent leaves every worker's residual; the rest stays
+#pragma omp parallel for num_threads(nthreads) schedule(static)
+  for (int64_t j = 0; j < K; ++j) {
+    const size_t i = S[j];
+    for (int32_t w = 0; w < W; ++w) o->acc[static_cast<size_t>(w) * N + i] = 0.0f;
+  }
+  o->t += 1;
+}
+
+}  // extern "C"

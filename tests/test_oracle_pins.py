@@ -1,0 +1,355 @@
+"""Pins of the CPU oracle against things other than itself: hand-worked values,
+closed forms, brute force (full sort) on tiny inputs, invariants, library routines
+and special cases that reduce to a textbook operation.  CPU only."""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from bruteforce import BruteForce, bits, importance
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+F = np.float32
+
+
+def u32(a):
+    return np.asarray(a, dtype=np.float32).view(np.uint32)
+
+
+# ---------------------------------------------------------------- leader, keep count
+
+
+def _leader_rows():
+    rows = []
+    for line in open(os.path.join(GOLD, "leader_vectors.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        head, vals = line.split(":")
+        seed, W = (int(x) for x in head.split())
+        rows.append((seed, W, [int(x) for x in vals.split()]))
+    return rows
+
+
+@pytest.mark.parametrize("seed,W,expect", _leader_rows())
+def test_leader_vectors(seed, W, expect):
+    assert [oracle.leader(seed, t, W) for t in range(len(expect))] == expect
+
+
+def test_mix64_vector():
+    assert oracle.mix64(0x9E3779B97F4A7C15) == 0xE220A8397B1DCDAF
+
+
+def test_leader_range_and_spread():
+    for W in (1, 2, 3, 7, 33):
+        got = [oracle.leader(12345, t, W) for t in range(4000)]
+        assert min(got) >= 0 and max(got) < W
+        counts = np.bincount(got, minlength=W)
+        assert counts.min() > 0.7 * 4000 / W  # every worker gets its turn
+
+
+def test_keep_count_table():
+    n_rows = 0
+    for line in open(os.path.join(GOLD, "keep_counts.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        R, n, k = line.split()
+        assert oracle.keep_count(int(n), float(R)) == int(k), line
+        n_rows += 1
+    assert n_rows > 50
+
+
+def test_keep_count_totals_of_tensor_lists():
+    from paper_1901_01544_b200 import workloads as wl
+
+    a = wl.alexnet_tensors()
+    r = wl.resnet50_tensors()
+    assert len(a) == 16 and sum(t.numel for t in a) == 60965224
+    assert len(r) == 161 and sum(t.numel for t in r) == 25557032
+    assert sum(oracle.keep_count(t.numel, 64.0) for t in a) == 952583
+    assert sum(oracle.keep_count(t.numel, 58.8) for t in r) == 434735
+    assert sum(oracle.keep_count(t.numel, 256.0) for t in a) == 238148
+    f = wl.split_equal(1 << 30, 96)
+    assert f[:64] == [11184811] * 64 and f[64:] == [11184810] * 32
+    assert sum(oracle.keep_count(n, 1000.0) for n in f) == 1073760
+    # N/K reproduces the paper's Table 1 compression ratios by construction
+    assert abs(60965224 / 952583 - 64.0) < 1e-3
+    assert abs(25557032 / 434735 - 58.8) < 2e-2
+
+
+# ---------------------------------------------------------------- importance
+
+
+def test_importance_closed_forms():
+    eps = F(1e-8)
+    assert int(u32(eps)) == 0x322BCC77
+    # |w| + eps rounds back to |w| for these, so importance = |acc| / |w| exactly
+    for a, w, want in [(0.5, 1.0, 0.5), (-0.25, -0.5, 0.5), (0.125, 0.25, 0.5), (-1.0, -0.5, 2.0), (0.0, 1.0, 0.0),
+                       (-0.0, 1.0, 0.0), (3.0, -1.0, 3.0)]:
+        assert oracle.importance_bits(a, w, 1e-8) == int(u32(want)), (a, w)
+    # w = 0: importance = |acc| / eps
+    assert oracle.importance_bits(2.0 ** -20, 0.0, 1e-8) == 0x42BEBC20
+    assert oracle.importance_bits(-(2.0 ** -21), -0.0, 1e-8) == 0x423EBC20
+    # the guard is really added: 0.125 + 1e-8 is not 0.125 in binary32
+    assert oracle.importance_bits(0.125, 0.125, 1e-8) != int(u32(1.0))
+    assert oracle.importance_bits(0.125, 0.125, 1e-8) == int(u32(F(0.125) / (F(0.125) + eps)))
+    # sign of either operand never matters; result is never negative
+    rng = np.random.default_rng(0)
+    for a, w in rng.normal(size=(200, 2)).astype(np.float32):
+        b = oracle.importance_bits(a, w, 1e-8)
+        assert b == oracle.importance_bits(-a, w, 1e-8) == oracle.importance_bits(a, -w, 1e-8)
+        assert b < 0x80000000
+        assert b == bits(importance(a, w, 1e-8))
+    # denormals are kept, not flushed
+    tiny = np.array([1], dtype=np.uint32).view(np.float32)[0]
+    assert oracle.importance_bits(tiny, 1.0, 1e-8) == 1
+
+
+def test_importance_monotone_in_magnitude():
+    w = F(0.3)
+    a = np.sort(np.abs(np.random.default_rng(1).normal(size=500)).astype(np.float32))
+    keys = [oracle.importance_bits(x, w, 1e-8) for x in a]
+    assert all(k0 <= k1 for k0, k1 in zip(keys, keys[1:]))
+
+
+# ---------------------------------------------------------------- selection: brute force
+
+
+def _brute_select(acc, w, k, eps):
+    imp = [bits(importance(a, x, eps)) for a, x in zip(acc, w)]
+    order = sorted(range(len(acc)), key=lambda i: (-imp[i], i))
+    return sorted(order[:k])
+
+
+def _adversarial(n, rng):
+    yield np.zeros(n, np.float32), np.ones(n, np.float32)  # all keys equal (zero)
+    yield np.full(n, 0.5, np.float32), np.full(n, -2.0, np.float32)  # all equal, non-zero
+    yield rng.choice(np.array([0.25, 1.0], np.float32), n), np.ones(n, np.float32)  # two distinct values
+    yield rng.normal(size=n).astype(np.float32), np.zeros(n, np.float32)  # every weight zero
+    a = rng.normal(size=n).astype(np.float32)
+    yield a, a.copy()  # importance ~ 1 everywhere, near-ties
+    yield rng.integers(-3, 4, n).astype(np.float32), rng.integers(-2, 3, n).astype(np.float32)  # many ties, zeros
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 7, 8, 31, 64])
+def test_select_equals_full_sort(n):
+    rng = np.random.default_rng(n)
+    cases = list(_adversarial(n, rng))
+    for _ in range(6):
+        cases.append((rng.normal(size=n).astype(np.float32), (rng.normal(size=n) * (rng.random(n) > 0.2)).astype(np.float32)))
+    for acc, w in cases:
+        for k in sorted({1, max(1, n // 4), max(1, n // 2), n}):
+            got = oracle.select(acc, w, k, 1e-8).tolist()
+            assert got == _brute_select(acc, w, k, F(1e-8)), (n, k)
+
+
+@pytest.mark.parametrize("layers,W,ratio", [([8], 2, 4.0), ([5, 1, 12, 3], 3, 3.0), ([64], 4, 64.0), ([17, 9], 1, 1.0),
+                                            ([6, 6], 5, 2.5)])
+def test_step_equals_bruteforce_model(layers, W, ratio):
+    rng = np.random.default_rng(sum(layers) + W)
+    N = sum(layers)
+    weights = (rng.normal(size=N) * (rng.random(N) > 0.15)).astype(np.float32)
+    orc = oracle.Oracle(layers, W, ratio, 1e-8, seed=3)
+    bf = BruteForce(layers, W, ratio, 1e-8)
+    for t in range(4):
+        # coarse values make ties and exact cancellations frequent
+        grads = (rng.integers(-4, 5, size=(W, N)) / 8.0).astype(np.float32)
+        upd = orc.step(grads, weights)
+        lists, upd_bf = bf.step(grads, weights, orc.leader)
+        assert orc.leader == oracle.leader(3, t, W)
+        assert np.array_equal(u32(upd), u32(upd_bf))
+        for w in range(W):
+            idx, val = orc.selection(w)
+            assert idx.tolist() == [i for i, _ in lists[w]]
+            assert np.array_equal(u32(val), u32(np.array([v for _, v in lists[w]], np.float32)))
+            assert np.array_equal(u32(orc.residual(w)), u32(bf.residual(w)))
+
+
+# ---------------------------------------------------------------- hand-worked example
+
+
+def test_worked_example():
+    g = json.load(open(os.path.join(GOLD, "worked_example.json")))
+    orc = oracle.Oracle(g["layer_sizes"], g["W"], g["ratio"], g["eps"], seed=0)
+    assert orc.layout() == ([0], [2])
+    weights = np.array(g["weights"], np.float32)
+    for st in g["steps"]:
+        orc.set_leader_override(st["leader"])
+        upd = orc.step(np.array(st["grads"], np.float32), weights)
+        assert orc.leader == st["leader"]
+        assert np.array_equal(u32(upd), u32(np.array(st["update"], np.float32)))  # includes +0 for the cancellation
+        for w in range(g["W"]):
+            idx, val = orc.selection(w)
+            assert idx.tolist() == st["lists"][w]
+            assert np.array_equal(u32(val), u32(np.array(st["list_vals"][w], np.float32)))
+            assert np.array_equal(u32(orc.residual(w)), u32(np.array(st["residual"][w], np.float32)))
+        mask = orc.mask()
+        assert mask.tolist() == [1 if i in st["lists"][st["leader"]] else 0 for i in range(8)]
+    assert oracle.importance_bits(2.0 ** -20, 0.0, 1e-8) == int(g["steps"][0]["importance_bits_w0_idx2"], 16)
+    assert oracle.importance_bits(2.0 ** -21, 0.0, 1e-8) == int(g["steps"][1]["importance_bits_w1_idx2"], 16)
+    m = g["mini"]
+    o2 = oracle.Oracle(m["layer_sizes"], m["W"], m["ratio"], m["eps"], seed=0)
+    o2.step(np.array(m["grads"], np.float32), np.array(m["weights"], np.float32))
+    assert o2.selection(0)[0].tolist() == m["list"]
+
+
+# ---------------------------------------------------------------- invariants and library routines
+
+
+def _random_problem(layers, W, seed, zero_frac=0.05):
+    rng = np.random.default_rng(seed)
+    N = sum(layers)
+    weights = (rng.normal(scale=0.05, size=N) * (rng.random(N) > zero_frac)).astype(np.float32)
+    return rng, weights
+
+
+def test_invariants_and_library_threshold():
+    layers, W, R = [5000, 333, 20000, 64, 1], 4, 16.0
+    rng, weights = _random_problem(layers, W, 11)
+    N = sum(layers)
+    orc = oracle.Oracle(layers, W, R, 1e-8, seed=5)
+    off, ks = orc.layout()
+    assert ks == [math.ceil(n / R) for n in layers]
+    acc_model = np.zeros((W, N), np.float32)
+    for t in range(3):
+        grads = rng.normal(scale=1e-3, size=(W, N)).astype(np.float32)
+        acc_model = acc_model + grads  # fp32 elementwise
+        upd = orc.step(grads, weights)
+        S, _ = orc.selection(orc.leader)
+        assert len(S) == orc.K == sum(ks)
+        imp = np.abs(acc_model) / (np.abs(weights) + F(1e-8))  # fp32 arithmetic in numpy
+        assert imp.dtype == np.float32
+        for w in range(W):
+            idx, val = orc.selection(w)
+            assert np.array_equal(u32(val), u32(acc_model[w, idx]))
+            seg = 0
+            for o, n, k in zip(off, layers, ks):
+                loc = idx[seg:seg + k].astype(np.int64) - o
+                seg += k
+                assert np.all(np.diff(loc) > 0) and loc.min() >= 0 and loc.max() < n  # ascending, inside the layer
+                li = imp[w, o:o + n]
+                inside = np.zeros(n, bool)
+                inside[loc] = True
+                # threshold value = k-th largest, by two independent library routines
+                T = li[inside].min()
+                assert T == np.partition(li, n - k)[n - k]
+                assert T == torch.kthvalue(torch.from_numpy(li.copy()), n - k + 1).values.item()
+                if k < n:
+                    assert T >= li[~inside].max()
+                    ties_in = np.flatnonzero(inside & (li == T))
+                    ties_out = np.flatnonzero(~inside & (li == T))
+                    if len(ties_out):
+                        assert ties_in.max() < ties_out.min()  # lower index wins the tie
+                    else:
+                        top = torch.topk(torch.from_numpy(li.copy()), k).indices.numpy()
+                        assert set(top.tolist()) == set(loc.tolist())
+        # shared index set keeps the reduced tensor sparse; everything off S is +0
+        offS = np.ones(N, bool)
+        offS[S] = False
+        assert np.all(u32(upd[offS]) == 0) and np.count_nonzero(upd) <= orc.K
+        # ordered worker sum at S
+        s = acc_model[0, S].copy()
+        for w in range(1, W):
+            s = s + acc_model[w, S]
+        assert np.array_equal(u32(upd[S]), u32(F(0) + s))
+        # what was sent left every residual (+0), the rest is untouched: conservation
+        sent = np.zeros_like(acc_model)
+        sent[:, S] = acc_model[:, S]
+        for w in range(W):
+            r = orc.residual(w)
+            assert np.all(u32(r[S]) == 0)
+            assert np.array_equal(u32(r[offS]), u32(acc_model[w, offS]))
+            assert np.array_equal(r + sent[w], acc_model[w])
+        acc_model[:, S] = 0
+        assert np.array_equal(orc.mask(), (~offS).astype(np.uint8))
+
+
+def test_ratio_one_is_a_dense_allreduce():
+    layers, W = [257, 1000, 3], 5
+    rng, weights = _random_problem(layers, W, 2)
+    N = sum(layers)
+    orc = oracle.Oracle(layers, W, 1.0, 1e-8, seed=0)
+    carry = np.zeros((W, N), np.float32)
+    for t in range(2):
+        grads = rng.normal(size=(W, N)).astype(np.float32)
+        upd = orc.step(grads, weights)
+        tot = grads[0].copy()
+        for w in range(1, W):
+            tot = tot + grads[w]
+        assert np.array_equal(u32(upd), u32(F(0) + tot))
+        for w in range(W):
+            assert np.all(u32(orc.residual(w)) == 0)
+            assert orc.selection(w)[0].tolist() == list(range(N))
+
+
+def test_single_worker_conserves_gradient_mass():
+    layers, W, R = [4096, 100], 1, 8.0
+    rng, weights = _random_problem(layers, W, 4)
+    N = sum(layers)
+    orc = oracle.Oracle(layers, W, R, 1e-8, seed=0)
+    seg_sum = np.zeros(N, np.float32)  # fp32 running sum since the element was last sent
+    total_sent = np.zeros(N, np.float64)
+    total_grad = np.zeros(N, np.float64)
+    for t in range(12):
+        g = rng.normal(scale=1e-2, size=(1, N)).astype(np.float32)
+        seg_sum = seg_sum + g[0]
+        upd = orc.step(g, weights)
+        S = orc.selection(0)[0]
+        assert np.array_equal(u32(upd[S]), u32(F(0) + seg_sum[S]))  # W = 1: update[S] is the residual itself
+        total_sent += upd
+        total_grad += g[0]
+        seg_sum[S] = 0
+        assert np.array_equal(u32(orc.residual(0)), u32(seg_sum))
+    assert np.allclose(total_sent + orc.residual(0), total_grad, rtol=0, atol=1e-6)
+
+
+def test_equal_denominators_reduce_to_magnitude_topk():
+    # batch-norm gammas (all 1) or all-zero weights: ranking by importance = ranking by |residual|
+    n, k = 3000, 100
+    rng = np.random.default_rng(9)
+    acc = rng.normal(size=n).astype(np.float32)
+    for wval in (1.0, 0.0, -0.37):
+        got = oracle.select(acc, np.full(n, wval, np.float32), k, 1e-8)
+        want = torch.topk(torch.from_numpy(np.abs(acc)), k).indices.sort().values.numpy()
+        assert np.array_equal(got, want.astype(np.uint32))
+
+
+def test_zero_weights_dominate():
+    # an element with w = 0 and any non-zero residual outranks every element with |w| >= 1e-3 and |residual| <= 1
+    n = 512
+    rng = np.random.default_rng(3)
+    w = rng.uniform(1e-3, 1.0, n).astype(np.float32)
+    acc = rng.uniform(-1, 1, n).astype(np.float32)
+    zeros = [5, 77, 300]
+    w[zeros] = 0.0
+    acc[zeros] = [1e-4, -2e-4, 3e-4]
+    assert oracle.select(acc, w, 3, 1e-8).tolist() == zeros
+
+
+def test_create_rejects_bad_arguments():
+    ok = dict(layer_sizes=[4, 4], W=2, ratio=2.0, eps=1e-8, seed=0)
+    oracle.Oracle(**ok)
+    for bad in (dict(layer_sizes=[4, 0]), dict(W=0), dict(ratio=0.5), dict(ratio=float("nan")), dict(eps=0.0),
+                dict(eps=-1.0), dict(ratio=float("inf"))):
+        with pytest.raises(ValueError):
+            oracle.Oracle(**{**ok, **bad})
+
+
+def test_reset_and_residual_roundtrip():
+    layers, W = [100, 28], 2
+    rng, weights = _random_problem(layers, W, 6)
+    orc = oracle.Oracle(layers, W, 4.0, 1e-8, seed=1)
+    g = rng.normal(size=(W, 128)).astype(np.float32)
+    u0 = orc.step(g, weights)
+    r = [orc.residual(w) for w in range(W)]
+    orc.reset()
+    assert orc.t == 0 and all(np.all(orc.residual(w) == 0) for w in range(W))
+    u1 = orc.step(g, weights)
+    assert np.array_equal(u32(u0), u32(u1))
+    for w in range(W):
+        orc.set_residual(w, r[w])
+        assert np.array_equal(u32(orc.residual(w)), u32(r[w]))
