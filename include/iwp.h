@@ -1,0 +1,163 @@
+/*
+ * iwp.h - C ABI of the importance-weighted gradient pruning step for data-parallel
+ *         all-reduce (arXiv 1901.01544), for W simulated workers held in one GPU.
+ *
+ * One call of iwp_step() performs, for every worker w and every layer l
+ * (Algorithm 1 of the paper; Section 3.2 "Importance Weighted Pruning"):
+ *   (a) residual accumulation        acc[w][i] += grads[w][i]
+ *   (b) gradient importance          imp = |acc[w][i]| / (|weights[i]| + eps)
+ *   (c) layer-wise selection         the k_l = ceil(n_l / ratio) elements with the largest
+ *                                    importance (ties: lower index first) - Algorithm 1's
+ *                                    "Mask <- |grad / w| > thr" with thr = k_l-th largest
+ *   (d) sparse encoding              ascending (index, value) lists per worker
+ *   (e) index agreement              one seeded-randomly chosen worker ("choose random node")
+ *                                    supplies the index set S every worker gathers at
+ *   (f) reduction                    update[S] = sum over workers in ascending worker order
+ *                                    (the ring all-reduce of the masked gradients), 0 elsewhere
+ *   (g) local accumulation           acc[w][S] = 0 for every w; everything else stays
+ *
+ * All arithmetic is IEEE-754 binary32, round to nearest even, no fused multiply-add,
+ * denormals kept.  Inputs must be finite.  Indices are 32-bit flat element offsets.
+ *
+ * Conventions
+ *   - every function returns an int status (IWP_OK = 0, errors negative); nothing throws,
+ *     aborts or prints; device code never traps or asserts (errors end up in a status word
+ *     read by iwp_sync_status()).
+ *   - pointers named *_dev are DEVICE pointers, *_host are HOST pointers; the caller owns
+ *     every buffer it passes in; the library owns what it allocates in iwp_create().
+ *   - one context = one CUDA device = one stream = one caller thread at a time.
+ *   - the library needs a CUDA device; there is no CPU fallback.
+ */
+#ifndef IWP_H_
+#define IWP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct iwp_ctx iwp_ctx;
+
+enum {
+  IWP_OK = 0,
+  IWP_ERR_INVALID = -1,  /* bad argument (NULL, size, range, alignment of a typed pointer) */
+  IWP_ERR_OOM = -2,      /* device or host allocation failed */
+  IWP_ERR_CUDA = -3,     /* a CUDA runtime call or kernel launch failed */
+  IWP_ERR_INTERNAL = -4, /* a device-side conservation check failed (counts do not add up) */
+  IWP_ERR_TIMEOUT = -5   /* a bounded device-side wait gave up (unused: no kernel here waits) */
+};
+
+/* Human-readable name of a status code; never NULL. */
+const char* iwp_strerror(int status);
+
+/* ---- pure host helpers (no GPU needed) --------------------------------------------- */
+
+/* Keep count of a layer of n elements at compression ratio R (Table 1 of the paper quotes
+ * ratios of 64x and 58.8x): ceil(n / R) in double precision, clamped to [1, n].
+ * Returns 0 for invalid input (n < 1, R < 1 or not finite). */
+int64_t iwp_keep_count(int64_t n, double ratio);
+
+/* The worker that supplies the index set at step t (0-based) - Section 3.2's randomly
+ * chosen node.  The paper names no generator; this one is
+ *   ((mix64(seed + (t + 1) * 0x9E3779B97F4A7C15) >> 32) * W) >> 32
+ * with the splitmix64 finaliser as mix64.  Returns -1 if W < 1. */
+int32_t iwp_leader_at(uint64_t seed, uint64_t t, int32_t W);
+
+/* Sizes the planner derives from a layer list, without touching a GPU.
+ * out[0] = N (total elements)            out[1] = K (total keep count per worker)
+ * out[2] = layers on the one-CTA path    out[3] = layers on the tiled path
+ * out[4] = tiles                          out[5] = chunks
+ * out[6] = device bytes iwp_create() would allocate
+ * out[7] = 1 if 128-bit vector access is possible for library-owned buffers (N % 4 == 0)
+ * Returns IWP_ERR_INVALID under the same rules as iwp_create(). */
+int iwp_plan_sizes(const int64_t* layer_sizes_host, int32_t n_layers, int32_t W, double ratio, int64_t out[8]);
+
+/* ---- life cycle -------------------------------------------------------------------------- */
+
+/* Creates a context on the CURRENT CUDA device.
+ *   layer_sizes_host  n_layers element counts; every tensor is its own selection unit
+ *                     (Algorithm 1 loops over layers j = 0..M); copied, caller keeps ownership
+ *   W                 number of simulated workers (the paper's N nodes), >= 1
+ *   ratio             compression factor R >= 1 (64 keeps 1/64 of each layer), finite
+ *   eps               guard added to |weight| in the importance; > 0 and finite
+ *   seed              seed of the leader draw
+ * Allocates and zeroes the residuals acc[W][N] plus select scratch and the (index, value)
+ * lists.  Errors: IWP_ERR_INVALID (NULL, n_layers < 1, a size < 1, W < 1, bad ratio or eps,
+ * N >= 2^32), IWP_ERR_OOM, IWP_ERR_CUDA; *out is NULL on error. */
+int iwp_create(iwp_ctx** out, const int64_t* layer_sizes_host, int32_t n_layers, int32_t W, double ratio, float eps,
+               uint64_t seed);
+
+/* Synchronises the context's stream and frees everything iwp_create() allocated.
+ * NULL is a no-op returning IWP_OK. */
+int iwp_destroy(iwp_ctx* ctx);
+
+/* Stream all later work of this context is enqueued on (a cudaStream_t passed as void*;
+ * NULL = the legacy default stream, which is also the initial setting). */
+int iwp_set_stream(iwp_ctx* ctx, void* cuda_stream);
+
+/* ---- the step ---------------------------------------------------------------------------- */
+
+/* One pruned all-reduce step, steps (a)-(g) above (Algorithm 1, one iteration of the loop over t
+ * without the optimizer update, which stays with the caller).
+ *   grads_dev    W*N floats, worker-major with stride N, layers concatenated without padding;
+ *                read only
+ *   weights_dev  N floats, one copy shared by all workers (synchronous replicas, Eq. 1); read only
+ *   update_dev   N floats, fully overwritten: +0 outside the index set, the ordered worker sum
+ *                inside; must not alias the other two
+ * Asynchronous: enqueues kernels on the context's stream and returns without synchronising;
+ * the three buffers must stay valid until the stream has run the step.  128-bit accesses are
+ * used when N % 4 == 0 and all three pointers are 16-byte aligned, scalar accesses otherwise.
+ * Advances the step counter.  Errors: IWP_ERR_INVALID (NULL), IWP_ERR_CUDA (launch failure). */
+int iwp_step(iwp_ctx* ctx, const float* grads_dev, const float* weights_dev, float* update_dev);
+
+/* The same step with HOST buffers (pinned memory recommended): copies grads and weights to
+ * library-owned staging buffers (allocated on first use), runs iwp_step(), copies the update
+ * back and synchronises the stream before returning. */
+int iwp_step_host(iwp_ctx* ctx, const float* grads_host, const float* weights_host, float* update_host);
+
+/* Synchronises the stream and returns the device status word: IWP_OK, IWP_ERR_INTERNAL
+ * (a count check failed inside a kernel; results of that step are undefined) or IWP_ERR_CUDA. */
+int iwp_sync_status(iwp_ctx* ctx);
+
+/* ---- state, accessors (none of these is on the timed path) ------------------------------- */
+
+/* off_host[l] = flat offset of layer l, k_host[l] = its keep count; either may be NULL. */
+int iwp_get_layout(iwp_ctx* ctx, int64_t* off_host, int64_t* k_host);
+/* out[0] = N, out[1] = K, out[2] = n_layers, out[3] = W. */
+int iwp_get_sizes(iwp_ctx* ctx, int64_t out[4]);
+int iwp_get_step(iwp_ctx* ctx, int64_t* t_host);
+int iwp_set_step(iwp_ctx* ctx, int64_t t); /* checkpoint / resume; t >= 0 */
+/* Leader used by the last step (-1 before the first). */
+int iwp_get_leader(iwp_ctx* ctx, int32_t* leader_host);
+/* Residual acc[w][0..N) copied to / from a device buffer of N floats (stream-ordered). */
+int iwp_get_residual(iwp_ctx* ctx, int32_t w, float* dst_dev);
+int iwp_set_residual(iwp_ctx* ctx, int32_t w, const float* src_dev);
+/* Worker w's list of the last step: K ascending global indices (layer segments of k_l entries
+ * in layer order) and the accumulated values at those indices as they were BEFORE step (g)
+ * zeroed what was sent.  Device buffers of K entries; either may be NULL. */
+int iwp_get_selection(iwp_ctx* ctx, int32_t w, uint32_t* idx_dev, float* val_dev);
+/* Algorithm 1's encode_uint8(Mask): N bytes on the device, 1 where the element is in the
+ * last step's index set, else 0. */
+int iwp_get_mask(iwp_ctx* ctx, uint8_t* dst_dev);
+/* acc <- 0, step counter <- 0, status word <- 0. */
+int iwp_reset(iwp_ctx* ctx);
+
+/* Options (tests and experiments):
+ *   "leader_override"  >= 0 forces the leader of every following step, -1 = seeded draw
+ *   "force_scalar"     1 = never use 128-bit accesses
+ *   "speculate"        1 (default) = sample-based threshold guess so that large layers are
+ *                      read once; 0 = always the multi-pass exact select.  Both are exact.
+ * Unknown key or out-of-range value: IWP_ERR_INVALID. */
+int iwp_set_option(iwp_ctx* ctx, const char* key, int64_t value);
+
+/* Counters: "launches" (kernels and memsets enqueued since create), "device_bytes",
+ * "spec_pairs" / "spec_failed" ((worker, layer) pairs that tried / fell back from the
+ * single-read path in the last step; reading them synchronises the stream).
+ * Unknown key: IWP_ERR_INVALID. */
+int iwp_get_stat(iwp_ctx* ctx, const char* key, int64_t* value_host);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IWP_H_ */

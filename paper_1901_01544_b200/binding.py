@@ -1,0 +1,231 @@
+"""Thin ctypes binding of the C-ABI library (include/iwp.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.
+torch supplies device memory and the stream.  There is no CPU fallback: if the shared
+library is missing or a CUDA call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence, Tuple
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libiwp.so")
+
+IWP_OK, IWP_ERR_INVALID, IWP_ERR_OOM, IWP_ERR_CUDA, IWP_ERR_INTERNAL, IWP_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+
+EXPORTS = [
+    "iwp_strerror", "iwp_keep_count", "iwp_leader_at", "iwp_plan_sizes", "iwp_create", "iwp_destroy",
+    "iwp_set_stream", "iwp_step", "iwp_step_host", "iwp_sync_status", "iwp_get_layout", "iwp_get_sizes",
+    "iwp_get_step", "iwp_set_step", "iwp_get_leader", "iwp_get_residual", "iwp_set_residual",
+    "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat",
+]
+
+_lib: Optional[C.CDLL] = None
+
+
+class IwpError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {iwp_strerror(status)} ({status})")
+
+
+def lib() -> C.CDLL:
+    """Loads libiwp.so (built in-tree by paper_1901_01544_b200.build); raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_1901_01544_b200.build` (needs nvcc); "
+                "there is no CPU fallback")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, u64, f32, f64, cp = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64, C.c_float, C.c_double, C.c_char_p
+        L.iwp_strerror.restype, L.iwp_strerror.argtypes = cp, [C.c_int]
+        L.iwp_keep_count.restype, L.iwp_keep_count.argtypes = i64, [i64, f64]
+        L.iwp_leader_at.restype, L.iwp_leader_at.argtypes = i32, [u64, u64, i32]
+        L.iwp_plan_sizes.argtypes = [vp, i32, i32, f64, vp]
+        L.iwp_create.argtypes = [C.POINTER(vp), vp, i32, i32, f64, f32, u64]
+        L.iwp_destroy.argtypes = [vp]
+        L.iwp_set_stream.argtypes = [vp, vp]
+        L.iwp_step.argtypes = [vp, vp, vp, vp]
+        L.iwp_step_host.argtypes = [vp, vp, vp, vp]
+        L.iwp_sync_status.argtypes = [vp]
+        L.iwp_get_layout.argtypes = [vp, vp, vp]
+        L.iwp_get_sizes.argtypes = [vp, vp]
+        L.iwp_get_step.argtypes = [vp, vp]
+        L.iwp_set_step.argtypes = [vp, i64]
+        L.iwp_get_leader.argtypes = [vp, vp]
+        L.iwp_get_residual.argtypes = [vp, i32, vp]
+        L.iwp_set_residual.argtypes = [vp, i32, vp]
+        L.iwp_get_selection.argtypes = [vp, i32, vp, vp]
+        L.iwp_get_mask.argtypes = [vp, vp]
+        L.iwp_reset.argtypes = [vp]
+        L.iwp_set_option.argtypes = [vp, cp, i64]
+        L.iwp_get_stat.argtypes = [vp, cp, vp]
+        for name in EXPORTS:
+            getattr(L, name)  # AttributeError if the library does not export a declared symbol
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != IWP_OK:
+        raise IwpError(status, where)
+
+
+# ---- functions with the C names (raw status codes are turned into exceptions) ---------------
+
+
+def iwp_strerror(status: int) -> str:
+    return lib().iwp_strerror(status).decode()
+
+
+def iwp_keep_count(n: int, ratio: float) -> int:
+    return int(lib().iwp_keep_count(n, ratio))
+
+
+def iwp_leader_at(seed: int, t: int, W: int) -> int:
+    return int(lib().iwp_leader_at(seed, t, W))
+
+
+def iwp_plan_sizes(layer_sizes: Sequence[int], W: int, ratio: float) -> dict:
+    arr = (C.c_int64 * len(layer_sizes))(*layer_sizes)
+    out = (C.c_int64 * 8)()
+    _check(lib().iwp_plan_sizes(arr, len(layer_sizes), W, ratio, out), "iwp_plan_sizes")
+    keys = ["N", "K", "small_layers", "tiled_layers", "tiles", "chunks", "device_bytes", "vector_ok"]
+    return dict(zip(keys, [int(v) for v in out]))
+
+
+def iwp_create(layer_sizes: Sequence[int], W: int, ratio: float, eps: float, seed: int) -> C.c_void_p:
+    arr = (C.c_int64 * len(layer_sizes))(*layer_sizes)
+    h = C.c_void_p()
+    _check(lib().iwp_create(C.byref(h), arr, len(layer_sizes), W, ratio, eps, seed), "iwp_create")
+    return h
+
+
+def iwp_destroy(h) -> None:
+    _check(lib().iwp_destroy(h), "iwp_destroy")
+
+
+def iwp_step(h, grads_ptr: int, weights_ptr: int, update_ptr: int) -> None:
+    _check(lib().iwp_step(h, grads_ptr, weights_ptr, update_ptr), "iwp_step")
+
+
+def iwp_step_host(h, grads_ptr: int, weights_ptr: int, update_ptr: int) -> None:
+    _check(lib().iwp_step_host(h, grads_ptr, weights_ptr, update_ptr), "iwp_step_host")
+
+
+# ---- convenience wrapper over torch tensors ----------------------------------------------------
+
+
+class Pruner:
+    """Owns one iwp context; takes torch CUDA tensors (device memory and stream only)."""
+
+    def __init__(self, layer_sizes: Sequence[int], W: int, ratio: float, eps: float = 1e-8, seed: int = 0):
+        import torch
+
+        if not torch.cuda.is_available():
+            raise RuntimeError("iwp needs a CUDA device; there is no CPU fallback")
+        self._torch = torch
+        self._h = iwp_create(list(layer_sizes), W, float(ratio), float(eps), int(seed))
+        out = (C.c_int64 * 4)()
+        _check(lib().iwp_get_sizes(self._h, out), "iwp_get_sizes")
+        self.N, self.K, self.L, self.W = (int(v) for v in out)
+        self.device = torch.device("cuda", torch.cuda.current_device())
+        self.use_current_stream()
+
+    # life cycle
+    def close(self) -> None:
+        if getattr(self, "_h", None):
+            iwp_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def use_current_stream(self) -> None:
+        s = self._torch.cuda.current_stream().cuda_stream
+        _check(lib().iwp_set_stream(self._h, C.c_void_p(s)), "iwp_set_stream")
+
+    # the step
+    def step(self, grads, weights, update=None):
+        t = self._torch
+        assert grads.is_cuda and grads.dtype == t.float32 and grads.is_contiguous() and grads.numel() == self.W * self.N
+        assert weights.is_cuda and weights.dtype == t.float32 and weights.is_contiguous() and weights.numel() == self.N
+        if update is None:
+            update = t.empty(self.N, dtype=t.float32, device=grads.device)
+        assert update.is_cuda and update.dtype == t.float32 and update.is_contiguous() and update.numel() == self.N
+        iwp_step(self._h, grads.data_ptr(), weights.data_ptr(), update.data_ptr())
+        return update
+
+    def step_host(self, grads, weights, update):
+        """Host (ideally pinned) tensors in, host tensor out; copies are inside the call."""
+        t = self._torch
+        for x, n in ((grads, self.W * self.N), (weights, self.N), (update, self.N)):
+            assert (not x.is_cuda) and x.dtype == t.float32 and x.is_contiguous() and x.numel() == n
+        iwp_step_host(self._h, grads.data_ptr(), weights.data_ptr(), update.data_ptr())
+        return update
+
+    def sync_status(self) -> int:
+        return int(lib().iwp_sync_status(self._h))
+
+    def check(self) -> None:
+        _check(self.sync_status(), "iwp_sync_status")
+
+    # state and accessors
+    def layout(self) -> Tuple[List[int], List[int]]:
+        off = (C.c_int64 * self.L)()
+        k = (C.c_int64 * self.L)()
+        _check(lib().iwp_get_layout(self._h, off, k), "iwp_get_layout")
+        return list(off), list(k)
+
+    @property
+    def t(self) -> int:
+        v = C.c_int64()
+        _check(lib().iwp_get_step(self._h, C.byref(v)), "iwp_get_step")
+        return int(v.value)
+
+    def set_step(self, t: int) -> None:
+        _check(lib().iwp_set_step(self._h, t), "iwp_set_step")
+
+    @property
+    def leader(self) -> int:
+        v = C.c_int32()
+        _check(lib().iwp_get_leader(self._h, C.byref(v)), "iwp_get_leader")
+        return int(v.value)
+
+    def residual(self, w: int):
+        out = self._torch.empty(self.N, dtype=self._torch.float32, device=self.device)
+        _check(lib().iwp_get_residual(self._h, w, out.data_ptr()), "iwp_get_residual")
+        return out
+
+    def set_residual(self, w: int, src) -> None:
+        assert src.is_cuda and src.dtype == self._torch.float32 and src.is_contiguous() and src.numel() == self.N
+        _check(lib().iwp_set_residual(self._h, w, src.data_ptr()), "iwp_set_residual")
+
+    def selection(self, w: int):
+        t = self._torch
+        idx = t.empty(self.K, dtype=t.int32, device=self.device)  # uint32 bit patterns
+        val = t.empty(self.K, dtype=t.float32, device=self.device)
+        _check(lib().iwp_get_selection(self._h, w, idx.data_ptr(), val.data_ptr()), "iwp_get_selection")
+        return idx, val
+
+    def mask(self):
+        m = self._torch.empty(self.N, dtype=self._torch.uint8, device=self.device)
+        _check(lib().iwp_get_mask(self._h, m.data_ptr()), "iwp_get_mask")
+        return m
+
+    def reset(self) -> None:
+        _check(lib().iwp_reset(self._h), "iwp_reset")
+
+    def set_option(self, key: str, value: int) -> None:
+        _check(lib().iwp_set_option(self._h, key.encode(), int(value)), f"iwp_set_option({key})")
+
+    def stat(self, key: str) -> int:
+        v = C.c_int64()
+        _check(lib().iwp_get_stat(self._h, key.encode(), C.byref(v)), f"iwp_get_stat({key})")
+        return int(v.value)

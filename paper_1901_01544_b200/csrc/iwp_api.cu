@@ -1,0 +1,489 @@
+// C ABI of the importance-weighted pruning step (see include/iwp.h): argument checks,
+// the host planner, device memory owned by a context, and the launch sequence of a step.
+#include "../../include/iwp.h"
+
+#include <cuda_runtime.h>
+
+#include <cstring>
+#include <new>
+
+#include "iwp_kernels.cuh"
+#include "iwp_plan.hpp"
+
+using namespace iwp;
+
+struct iwp_ctx {
+  Plan plan;
+  float eps = 0.f;
+  double ratio = 1.0;
+  uint64_t seed = 0;
+  int64_t t = 0;
+  int32_t leader = -1;
+  int64_t leader_override = -1;
+  bool force_scalar = false;
+  bool speculate = true;
+  cudaStream_t stream = nullptr;
+  int device = 0;
+  int64_t launches = 0;
+  uint64_t device_bytes = 0;
+  uint32_t n_pairs = 0;  // (tiled layer, worker) pairs
+  // device memory
+  float* acc = nullptr;
+  LayerDesc* d_layers = nullptr;
+  Tile* d_tiles = nullptr;
+  Chunk* d_chunks = nullptr;
+  uint32_t* d_small_ids = nullptr;
+  uint32_t* d_large_ids = nullptr;
+  uint2* d_state = nullptr;
+  uint32_t* d_hist = nullptr;
+  uint2* d_chunk_cnt = nullptr;
+  uint32_t* sel_idx = nullptr;
+  float* sel_val = nullptr;
+  int* d_status = nullptr;
+  // staging for iwp_step_host
+  float* stg_grads = nullptr;
+  float* stg_weights = nullptr;
+  float* stg_update = nullptr;
+};
+
+namespace {
+
+struct Sizes {
+  uint64_t acc, layers, tiles, chunks, small_ids, large_ids, state, hist, chunk_cnt, sel_idx, sel_val, status;
+  uint64_t total() const {
+    return acc + layers + tiles + chunks + small_ids + large_ids + state + hist + chunk_cnt + sel_idx + sel_val +
+           status;
+  }
+};
+
+uint64_t at_least(uint64_t b) { return b ? b : 16; }
+
+Sizes sizes_of(const Plan& p) {
+  Sizes s;
+  const uint64_t W = static_cast<uint64_t>(p.W);
+  const uint64_t pairs = W * p.large_layers.size();
+  s.acc = W * p.N * sizeof(float);
+  s.layers = p.layers.size() * sizeof(LayerDesc);
+  s.tiles = at_least(p.tiles.size() * sizeof(Tile));
+  s.chunks = at_least(p.chunks.size() * sizeof(Chunk));
+  s.small_ids = at_least(p.small_layers.size() * sizeof(uint32_t));
+  s.large_ids = at_least(p.large_layers.size() * sizeof(uint32_t));
+  s.state = at_least(pairs * sizeof(uint2));
+  s.hist = at_least(pairs * NBINS * sizeof(uint32_t));
+  s.chunk_cnt = at_least(W * p.chunks.size() * sizeof(uint2));
+  s.sel_idx = W * p.K * sizeof(uint32_t);
+  s.sel_val = W * p.K * sizeof(float);
+  s.status = sizeof(int);
+  return s;
+}
+
+template <typename T>
+int dev_alloc(T** p, uint64_t bytes) {
+  void* q = nullptr;
+  const cudaError_t e = cudaMalloc(&q, bytes);
+  if (e == cudaErrorMemoryAllocation) {
+    cudaGetLastError();
+    return IWP_ERR_OOM;
+  }
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  *p = static_cast<T*>(q);
+  return IWP_OK;
+}
+
+void free_all(iwp_ctx* c) {
+  cudaFree(c->acc);
+  cudaFree(c->d_layers);
+  cudaFree(c->d_tiles);
+  cudaFree(c->d_chunks);
+  cudaFree(c->d_small_ids);
+  cudaFree(c->d_large_ids);
+  cudaFree(c->d_state);
+  cudaFree(c->d_hist);
+  cudaFree(c->d_chunk_cnt);
+  cudaFree(c->sel_idx);
+  cudaFree(c->sel_val);
+  cudaFree(c->d_status);
+  cudaFree(c->stg_grads);
+  cudaFree(c->stg_weights);
+  cudaFree(c->stg_update);
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+#define IWP_LAUNCH_CHECK(c)                         \
+  do {                                              \
+    (c)->launches += 1;                             \
+    if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA; \
+  } while (0)
+
+template <bool VEC>
+int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update, int32_t leader) {
+  const Plan& p = c->plan;
+  const int W = p.W;
+  const uint64_t N = p.N, K = p.K;
+  cudaStream_t s = c->stream;
+  if (!p.small_layers.empty()) {
+    const size_t dyn = static_cast<size_t>(p.max_small_n) * sizeof(uint32_t);
+    dim3 grid(static_cast<unsigned>(p.small_layers.size()), static_cast<unsigned>(W));
+    k_small<<<grid, THREADS, dyn, s>>>(grads, weights, c->acc, update, c->d_layers, c->d_small_ids, c->sel_idx,
+                                       c->sel_val, c->d_status, c->eps, N, K);
+    IWP_LAUNCH_CHECK(c);
+  }
+  if (!p.large_layers.empty()) {
+    const unsigned n_tiles = static_cast<unsigned>(p.tiles.size());
+    const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
+    dim3 cgrid(n_chunks, static_cast<unsigned>(W));
+    k_accumulate<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, N, W);
+    IWP_LAUNCH_CHECK(c);
+    for (int pass = 0; pass < N_PASSES; ++pass) {
+      k_hist_dense<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_state, c->d_hist,
+                                                  c->eps, N, W, pass);
+      IWP_LAUNCH_CHECK(c);
+      k_find_digit<<<c->n_pairs, THREADS, 0, s>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->d_status, W,
+                                                  pass);
+      IWP_LAUNCH_CHECK(c);
+    }
+    k_count_dense<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_state, c->d_chunk_cnt,
+                                                 c->eps, N, W, n_chunks);
+    IWP_LAUNCH_CHECK(c);
+    k_write_dense<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_state, c->d_chunk_cnt,
+                                                 c->sel_idx, c->sel_val, c->d_status, c->eps, N, K, W, n_chunks);
+    IWP_LAUNCH_CHECK(c);
+  }
+  const unsigned gblocks = static_cast<unsigned>((K + THREADS - 1) / THREADS);
+  k_gather_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->acc, update, N,
+                                                   K, W);
+  IWP_LAUNCH_CHECK(c);
+  return IWP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* iwp_strerror(int status) {
+  switch (status) {
+    case IWP_OK: return "ok";
+    case IWP_ERR_INVALID: return "invalid argument";
+    case IWP_ERR_OOM: return "out of memory";
+    case IWP_ERR_CUDA: return "CUDA runtime error";
+    case IWP_ERR_INTERNAL: return "device-side count check failed";
+    case IWP_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int64_t iwp_keep_count(int64_t n, double ratio) { return keep_count(n, ratio); }
+
+int32_t iwp_leader_at(uint64_t seed, uint64_t t, int32_t W) { return leader_at(seed, t, W); }
+
+int iwp_plan_sizes(const int64_t* layer_sizes, int32_t n_layers, int32_t W, double ratio, int64_t out[8]) {
+  if (!out) return IWP_ERR_INVALID;
+  const Plan p = make_plan(layer_sizes, n_layers, W, ratio, 1.0f);
+  if (!p.valid) return IWP_ERR_INVALID;
+  out[0] = static_cast<int64_t>(p.N);
+  out[1] = static_cast<int64_t>(p.K);
+  out[2] = static_cast<int64_t>(p.small_layers.size());
+  out[3] = static_cast<int64_t>(p.large_layers.size());
+  out[4] = static_cast<int64_t>(p.tiles.size());
+  out[5] = static_cast<int64_t>(p.chunks.size());
+  out[6] = static_cast<int64_t>(sizes_of(p).total());
+  out[7] = (p.N % 4 == 0) ? 1 : 0;
+  return IWP_OK;
+}
+
+int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int32_t W, double ratio, float eps,
+               uint64_t seed) {
+  if (!out) return IWP_ERR_INVALID;
+  *out = nullptr;
+  iwp_ctx* c = new (std::nothrow) iwp_ctx;
+  if (!c) return IWP_ERR_OOM;
+  try {
+    c->plan = make_plan(layer_sizes, n_layers, W, ratio, eps);
+  } catch (...) {
+    delete c;
+    return IWP_ERR_OOM;
+  }
+  if (!c->plan.valid) {
+    delete c;
+    return IWP_ERR_INVALID;
+  }
+  const Plan& p = c->plan;
+  c->eps = eps;
+  c->ratio = ratio;
+  c->seed = seed;
+  c->n_pairs = static_cast<uint32_t>(p.large_layers.size()) * static_cast<uint32_t>(W);
+  if (cudaGetDevice(&c->device) != cudaSuccess) {
+    cudaGetLastError();
+    delete c;
+    return IWP_ERR_CUDA;
+  }
+  const Sizes sz = sizes_of(p);
+  c->device_bytes = sz.total();
+  int rc = IWP_OK;
+  auto A = [&](auto** ptr, uint64_t bytes) {
+    if (rc == IWP_OK) rc = dev_alloc(ptr, bytes);
+  };
+  A(&c->acc, sz.acc);
+  A(&c->d_layers, sz.layers);
+  A(&c->d_tiles, sz.tiles);
+  A(&c->d_chunks, sz.chunks);
+  A(&c->d_small_ids, sz.small_ids);
+  A(&c->d_large_ids, sz.large_ids);
+  A(&c->d_state, sz.state);
+  A(&c->d_hist, sz.hist);
+  A(&c->d_chunk_cnt, sz.chunk_cnt);
+  A(&c->sel_idx, sz.sel_idx);
+  A(&c->sel_val, sz.sel_val);
+  A(&c->d_status, sz.status);
+  if (rc != IWP_OK) {
+    free_all(c);
+    delete c;
+    return rc;
+  }
+  bool ok = true;
+  auto H2D = [&](void* dst, const void* src, size_t bytes) {
+    if (bytes) ok = ok && cudaMemcpy(dst, src, bytes, cudaMemcpyHostToDevice) == cudaSuccess;
+  };
+  H2D(c->d_layers, p.layers.data(), p.layers.size() * sizeof(LayerDesc));
+  H2D(c->d_tiles, p.tiles.data(), p.tiles.size() * sizeof(Tile));
+  H2D(c->d_chunks, p.chunks.data(), p.chunks.size() * sizeof(Chunk));
+  H2D(c->d_small_ids, p.small_layers.data(), p.small_layers.size() * sizeof(uint32_t));
+  H2D(c->d_large_ids, p.large_layers.data(), p.large_layers.size() * sizeof(uint32_t));
+  ok = ok && cudaMemset(c->acc, 0, sz.acc) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_state, 0, sz.state) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_hist, 0, sz.hist) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_chunk_cnt, 0, sz.chunk_cnt) == cudaSuccess;
+  ok = ok && cudaMemset(c->sel_idx, 0, sz.sel_idx) == cudaSuccess;
+  ok = ok && cudaMemset(c->sel_val, 0, sz.sel_val) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_status, 0, sz.status) == cudaSuccess;
+  if (ok && p.max_small_n) {
+    ok = cudaFuncSetAttribute(k_small, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(p.max_small_n * sizeof(uint32_t))) == cudaSuccess;
+  }
+  ok = ok && cudaDeviceSynchronize() == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    free_all(c);
+    delete c;
+    return IWP_ERR_CUDA;
+  }
+  *out = c;
+  return IWP_OK;
+}
+
+int iwp_destroy(iwp_ctx* c) {
+  if (!c) return IWP_OK;
+  cudaStreamSynchronize(c->stream);
+  free_all(c);
+  cudaGetLastError();
+  delete c;
+  return IWP_OK;
+}
+
+int iwp_set_stream(iwp_ctx* c, void* stream) {
+  if (!c) return IWP_ERR_INVALID;
+  c->stream = static_cast<cudaStream_t>(stream);
+  return IWP_OK;
+}
+
+int iwp_step(iwp_ctx* c, const float* grads, const float* weights, float* update) {
+  if (!c || !grads || !weights || !update) return IWP_ERR_INVALID;
+  const int32_t leader = c->leader_override >= 0 ? static_cast<int32_t>(c->leader_override)
+                                                 : leader_at(c->seed, static_cast<uint64_t>(c->t), c->plan.W);
+  const bool vec = !c->force_scalar && (c->plan.N % 4 == 0) && aligned16(grads) && aligned16(weights) &&
+                   aligned16(update) && aligned16(c->acc);
+  const int rc = vec ? run_step<true>(c, grads, weights, update, leader) : run_step<false>(c, grads, weights, update, leader);
+  if (rc != IWP_OK) return rc;
+  c->leader = leader;
+  c->t += 1;
+  return IWP_OK;
+}
+
+int iwp_step_host(iwp_ctx* c, const float* grads, const float* weights, float* update) {
+  if (!c || !grads || !weights || !update) return IWP_ERR_INVALID;
+  const uint64_t N = c->plan.N, W = static_cast<uint64_t>(c->plan.W);
+  if (!c->stg_grads) {
+    int rc = dev_alloc(&c->stg_grads, W * N * sizeof(float));
+    if (rc == IWP_OK) rc = dev_alloc(&c->stg_weights, N * sizeof(float));
+    if (rc == IWP_OK) rc = dev_alloc(&c->stg_update, N * sizeof(float));
+    if (rc != IWP_OK) {
+      cudaFree(c->stg_grads);
+      cudaFree(c->stg_weights);
+      cudaFree(c->stg_update);
+      c->stg_grads = c->stg_weights = c->stg_update = nullptr;
+      return rc;
+    }
+  }
+  cudaStream_t s = c->stream;
+  if (cudaMemcpyAsync(c->stg_grads, grads, W * N * sizeof(float), cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(c->stg_weights, weights, N * sizeof(float), cudaMemcpyHostToDevice, s) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  const int rc = iwp_step(c, c->stg_grads, c->stg_weights, c->stg_update);
+  if (rc != IWP_OK) return rc;
+  if (cudaMemcpyAsync(update, c->stg_update, N * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  return IWP_OK;
+}
+
+int iwp_sync_status(iwp_ctx* c) {
+  if (!c) return IWP_ERR_INVALID;
+  int st = 0;
+  if (cudaMemcpyAsync(&st, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+      cudaStreamSynchronize(c->stream) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  return st;
+}
+
+int iwp_get_layout(iwp_ctx* c, int64_t* off, int64_t* k) {
+  if (!c) return IWP_ERR_INVALID;
+  for (size_t l = 0; l < c->plan.layers.size(); ++l) {
+    if (off) off[l] = c->plan.layers[l].off;
+    if (k) k[l] = c->plan.layers[l].k;
+  }
+  return IWP_OK;
+}
+
+int iwp_get_sizes(iwp_ctx* c, int64_t out[4]) {
+  if (!c || !out) return IWP_ERR_INVALID;
+  out[0] = static_cast<int64_t>(c->plan.N);
+  out[1] = static_cast<int64_t>(c->plan.K);
+  out[2] = static_cast<int64_t>(c->plan.layers.size());
+  out[3] = c->plan.W;
+  return IWP_OK;
+}
+
+int iwp_get_step(iwp_ctx* c, int64_t* t) {
+  if (!c || !t) return IWP_ERR_INVALID;
+  *t = c->t;
+  return IWP_OK;
+}
+
+int iwp_set_step(iwp_ctx* c, int64_t t) {
+  if (!c || t < 0) return IWP_ERR_INVALID;
+  c->t = t;
+  return IWP_OK;
+}
+
+int iwp_get_leader(iwp_ctx* c, int32_t* leader) {
+  if (!c || !leader) return IWP_ERR_INVALID;
+  *leader = c->leader;
+  return IWP_OK;
+}
+
+int iwp_get_residual(iwp_ctx* c, int32_t w, float* dst) {
+  if (!c || !dst || w < 0 || w >= c->plan.W) return IWP_ERR_INVALID;
+  const uint64_t N = c->plan.N;
+  if (cudaMemcpyAsync(dst, c->acc + static_cast<uint64_t>(w) * N, N * sizeof(float), cudaMemcpyDeviceToDevice,
+                      c->stream) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  return IWP_OK;
+}
+
+int iwp_set_residual(iwp_ctx* c, int32_t w, const float* src) {
+  if (!c || !src || w < 0 || w >= c->plan.W) return IWP_ERR_INVALID;
+  const uint64_t N = c->plan.N;
+  if (cudaMemcpyAsync(c->acc + static_cast<uint64_t>(w) * N, src, N * sizeof(float), cudaMemcpyDeviceToDevice,
+                      c->stream) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  return IWP_OK;
+}
+
+int iwp_get_selection(iwp_ctx* c, int32_t w, uint32_t* idx, float* val) {
+  if (!c || w < 0 || w >= c->plan.W) return IWP_ERR_INVALID;
+  const uint64_t K = c->plan.K;
+  bool ok = true;
+  if (idx)
+    ok = ok && cudaMemcpyAsync(idx, c->sel_idx + static_cast<uint64_t>(w) * K, K * sizeof(uint32_t),
+                               cudaMemcpyDeviceToDevice, c->stream) == cudaSuccess;
+  if (val)
+    ok = ok && cudaMemcpyAsync(val, c->sel_val + static_cast<uint64_t>(w) * K, K * sizeof(float),
+                               cudaMemcpyDeviceToDevice, c->stream) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  return IWP_OK;
+}
+
+int iwp_get_mask(iwp_ctx* c, uint8_t* dst) {
+  if (!c || !dst) return IWP_ERR_INVALID;
+  const uint64_t N = c->plan.N, K = c->plan.K;
+  if (cudaMemsetAsync(dst, 0, N, c->stream) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  if (c->leader < 0) return IWP_OK;
+  const unsigned blocks = static_cast<unsigned>((K + THREADS - 1) / THREADS);
+  k_mask_scatter<<<blocks, THREADS, 0, c->stream>>>(c->sel_idx + static_cast<uint64_t>(c->leader) * K, dst, K);
+  if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+  return IWP_OK;
+}
+
+int iwp_reset(iwp_ctx* c) {
+  if (!c) return IWP_ERR_INVALID;
+  const Sizes sz = sizes_of(c->plan);
+  bool ok = cudaMemsetAsync(c->acc, 0, sz.acc, c->stream) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->d_hist, 0, sz.hist, c->stream) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->d_status, 0, sz.status, c->stream) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  c->t = 0;
+  c->leader = -1;
+  return IWP_OK;
+}
+
+int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
+  if (!c || !key) return IWP_ERR_INVALID;
+  if (!std::strcmp(key, "leader_override")) {
+    if (v < -1 || v >= c->plan.W) return IWP_ERR_INVALID;
+    c->leader_override = v;
+    return IWP_OK;
+  }
+  if (!std::strcmp(key, "force_scalar")) {
+    if (v != 0 && v != 1) return IWP_ERR_INVALID;
+    c->force_scalar = v != 0;
+    return IWP_OK;
+  }
+  if (!std::strcmp(key, "speculate")) {
+    if (v != 0 && v != 1) return IWP_ERR_INVALID;
+    c->speculate = v != 0;
+    return IWP_OK;
+  }
+  return IWP_ERR_INVALID;
+}
+
+int iwp_get_stat(iwp_ctx* c, const char* key, int64_t* value) {
+  if (!c || !key || !value) return IWP_ERR_INVALID;
+  if (!std::strcmp(key, "launches")) {
+    *value = c->launches;
+    return IWP_OK;
+  }
+  if (!std::strcmp(key, "device_bytes")) {
+    *value = static_cast<int64_t>(c->device_bytes);
+    return IWP_OK;
+  }
+  if (!std::strcmp(key, "spec_pairs") || !std::strcmp(key, "spec_failed")) {
+    *value = 0;
+    return IWP_OK;
+  }
+  return IWP_ERR_INVALID;
+}
+
+}  // extern "C"

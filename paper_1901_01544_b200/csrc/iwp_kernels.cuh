@@ -1,0 +1,519 @@
+// sm_100a kernels of the importance-weighted pruning step (Algorithm 1 of the paper).
+//
+// Nothing here is a dense contraction, so there are no tensor-core instructions: every
+// kernel is bound by HBM traffic (or, for the small ones, by launch latency).  The work is
+// organised so that the W*N residual/gradient stream is touched as few times as possible
+// and always with coalesced 128-bit accesses.
+//
+// IEEE exactness: the residual add, the eps guard and the division use the explicit
+// round-to-nearest intrinsics, so the results do not depend on compiler contraction or
+// fast-math flags, and denormals are kept.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "iwp_plan.hpp"
+
+namespace iwp {
+
+constexpr int THREADS = 256;
+constexpr int WARPS = THREADS / 32;
+constexpr int STATUS_INTERNAL = -4;
+
+// radix-select digit plan over the 32-bit importance pattern (bit 31 is always 0)
+__host__ __device__ constexpr int pass_shift(int pass) { return pass == 0 ? 21 : (pass == 1 ? 10 : 0); }
+__host__ __device__ constexpr int pass_bins(int pass) { return pass == 2 ? 1024 : 2048; }
+constexpr int N_PASSES = 3;
+
+// ---------------------------------------------------------------------------------------
+// element helpers
+// ---------------------------------------------------------------------------------------
+
+// Algorithm 1, mask line: |grad / w|, with the eps guard; the bit pattern of a non-negative
+// float orders like the float, so the unsigned pattern is the sort key.
+__device__ __forceinline__ uint32_t imp_key(float acc, float w, float eps) {
+  return __float_as_uint(__fdiv_rn(fabsf(acc), __fadd_rn(fabsf(w), eps)));
+}
+
+// A slot is four consecutive floats starting at a multiple of four elements.  [lo, hi) is
+// the valid flat range; a slot fully inside it is moved with one 128-bit access when VEC.
+template <bool VEC>
+__device__ __forceinline__ void load4(const float* __restrict__ p, uint64_t e0, uint64_t lo, uint64_t hi,
+                                      float (&v)[4]) {
+  if (VEC && e0 >= lo && e0 + 4 <= hi) {
+    const float4 t = *reinterpret_cast<const float4*>(p + e0);
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  } else {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint64_t e = e0 + c;
+      v[c] = (e >= lo && e < hi) ? p[e] : 0.0f;
+    }
+  }
+}
+
+// same, for data that is read exactly once (the gradients): streaming / evict-first
+template <bool VEC>
+__device__ __forceinline__ void load4_stream(const float* __restrict__ p, uint64_t e0, uint64_t lo, uint64_t hi,
+                                             float (&v)[4]) {
+  if (VEC && e0 >= lo && e0 + 4 <= hi) {
+    const float4 t = __ldcs(reinterpret_cast<const float4*>(p + e0));
+    v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+  } else {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint64_t e = e0 + c;
+      v[c] = (e >= lo && e < hi) ? __ldcs(p + e) : 0.0f;
+    }
+  }
+}
+
+template <bool VEC>
+__device__ __forceinline__ void store4(float* __restrict__ p, uint64_t e0, uint64_t lo, uint64_t hi,
+                                       const float (&v)[4]) {
+  if (VEC && e0 >= lo && e0 + 4 <= hi) {
+    *reinterpret_cast<float4*>(p + e0) = make_float4(v[0], v[1], v[2], v[3]);
+  } else {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const uint64_t e = e0 + c;
+      if (e >= lo && e < hi) p[e] = v[c];
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// block helpers (THREADS = 256)
+// ---------------------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t x) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, x, d);
+    if (lane >= d) x += y;
+  }
+  return x;
+}
+
+// Exclusive prefix sum over the block in thread order; `total` = block sum.
+// sh_warp: WARPS words of shared memory.  Contains two __syncthreads().
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t x, uint32_t* sh_warp, uint32_t& total) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const uint32_t incl = warp_incl_scan(x);
+  if (lane == 31) sh_warp[wid] = incl;
+  __syncthreads();
+  uint32_t woff = 0, tot = 0;
+#pragma unroll
+  for (int i = 0; i < WARPS; ++i) {
+    const uint32_t v = sh_warp[i];
+    if (i < wid) woff += v;
+    tot += v;
+  }
+  __syncthreads();
+  total = tot;
+  return woff + incl - x;
+}
+
+// Radix-select digit step on a histogram in shared memory: finds the digit d with
+//   count(digit > d) < krem <= count(digit >= d)
+// res[0] = d, res[1] = krem - count(digit > d), res[2] = 1 if found.  sh_scan: THREADS words.
+__device__ __forceinline__ void find_digit(const uint32_t* hist, int nb, uint32_t krem, uint32_t* sh_scan,
+                                           uint32_t* res) {
+  const int tid = threadIdx.x;
+  const int per = nb / THREADS;
+  uint32_t local = 0;
+  for (int b = 0; b < per; ++b) local += hist[tid * per + b];
+  sh_scan[tid] = local;
+  if (tid == 0) res[2] = 0;
+  __syncthreads();
+  for (int d = 1; d < THREADS; d <<= 1) {  // inclusive suffix sum over threads
+    const uint32_t v = (tid + d < THREADS) ? sh_scan[tid + d] : 0u;
+    __syncthreads();
+    sh_scan[tid] += v;
+    __syncthreads();
+  }
+  const uint32_t incl = sh_scan[tid];
+  const uint32_t excl = incl - local;
+  if (excl < krem && krem <= incl) {
+    uint32_t running = excl;
+    for (int b = per - 1; b >= 0; --b) {
+      const uint32_t h = hist[tid * per + b];
+      if (running + h >= krem) {
+        res[0] = static_cast<uint32_t>(tid * per + b);
+        res[1] = krem - running;
+        res[2] = 1;
+        break;
+      }
+      running += h;
+    }
+  }
+  __syncthreads();
+}
+
+// Warp-aggregated increment of a shared-memory histogram: lanes that hit the same bin
+// elect one lane that adds the whole group's count.  Must be called by all 32 lanes.
+__device__ __forceinline__ void hist_add_aggregated(uint32_t* hist, bool valid, uint32_t bin) {
+  const uint32_t tag = valid ? bin : 0xffffffffu;
+  const uint32_t peers = __match_any_sync(0xffffffffu, tag);
+  const int lane = threadIdx.x & 31;
+  if (valid && (__ffs(peers) - 1) == lane) atomicAdd(&hist[bin], static_cast<uint32_t>(__popc(peers)));
+}
+
+// ---------------------------------------------------------------------------------------
+// tiled path, step (a): residual accumulation  acc += grads, and update <- 0
+// grid = tiles; each CTA walks the W workers of one tile.
+// ---------------------------------------------------------------------------------------
+template <bool VEC>
+__global__ void __launch_bounds__(THREADS) k_accumulate(const float* __restrict__ grads, float* __restrict__ acc,
+                                                         float* __restrict__ update, const Tile* __restrict__ tiles,
+                                                         uint64_t N, int W) {
+  const Tile t = tiles[blockIdx.x];
+  const uint64_t lo = t.a, hi = lo + t.len;
+  const uint64_t base = lo & ~static_cast<uint64_t>(TILE - 1);
+  constexpr int SPT = TILE / 4 / THREADS;  // slots per thread
+  uint64_t e0[SPT];
+#pragma unroll
+  for (int s = 0; s < SPT; ++s) e0[s] = base + static_cast<uint64_t>(s * THREADS + threadIdx.x) * 4;
+  const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int s = 0; s < SPT; ++s) store4<VEC>(update, e0[s], lo, hi, zero);
+  for (int w = 0; w < W; ++w) {
+    const float* g = grads + static_cast<uint64_t>(w) * N;
+    float* a = acc + static_cast<uint64_t>(w) * N;
+    float gv[SPT][4], av[SPT][4];
+#pragma unroll
+    for (int s = 0; s < SPT; ++s) {
+      load4_stream<VEC>(g, e0[s], lo, hi, gv[s]);
+      load4<VEC>(a, e0[s], lo, hi, av[s]);
+    }
+#pragma unroll
+    for (int s = 0; s < SPT; ++s) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) av[s][c] = __fadd_rn(av[s][c], gv[s][c]);
+      store4<VEC>(a, e0[s], lo, hi, av[s]);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// tiled path, step (c): exact radix select of the k-th largest key per (worker, layer)
+// ---------------------------------------------------------------------------------------
+
+// One histogram pass over a chunk of the residual: keys that match the prefix found so far
+// are counted by their next digit.  grid = (chunks, W).
+template <bool VEC>
+__global__ void __launch_bounds__(THREADS)
+    k_hist_dense(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
+                 const LayerDesc* __restrict__ layers, const uint2* __restrict__ state, uint32_t* __restrict__ hist,
+                 float eps, uint64_t N, int W, int pass) {
+  __shared__ uint32_t sh[NBINS];
+  const Chunk c = chunks[blockIdx.x];
+  const int w = blockIdx.y;
+  const uint32_t pair = static_cast<uint32_t>(layers[c.layer].large_index) * W + w;
+  const int shift = pass_shift(pass), nb = pass_bins(pass);
+  const int prev_shift = pass == 0 ? 31 : pass_shift(pass - 1);
+  const uint32_t want = pass == 0 ? 0u : (state[pair].x >> prev_shift);
+  for (int b = threadIdx.x; b < nb; b += THREADS) sh[b] = 0;
+  __syncthreads();
+  const uint64_t lo = c.a, hi = lo + c.len;
+  const uint64_t s0 = lo & ~3ull;
+  const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+  const float* a = acc + static_cast<uint64_t>(w) * N;
+  for (uint32_t it = 0; it < n_iter; ++it) {
+    const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+    float av[4], wv[4];
+    load4<VEC>(a, e0, lo, hi, av);
+    load4<VEC>(weights, e0, lo, hi, wv);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint64_t e = e0 + q;
+      const uint32_t key = imp_key(av[q], wv[q], eps);
+      const bool valid = e >= lo && e < hi && (key >> prev_shift) == want;  // pass 0: bit 31 is 0 == want
+      hist_add_aggregated(sh, valid, (key >> shift) & (nb - 1));
+    }
+  }
+  __syncthreads();
+  uint32_t* gh = hist + static_cast<uint64_t>(pair) * NBINS;
+  for (int b = threadIdx.x; b < nb; b += THREADS) {
+    const uint32_t v = sh[b];
+    if (v) atomicAdd(&gh[b], v);
+  }
+}
+
+// Digit decision for every (worker, layer) pair of the tiled path; grid = pairs.
+// Reads the pair's histogram, clears it for the next pass, extends the key prefix.
+// After the last pass state = (threshold key T, number r of T-valued elements to keep).
+__global__ void __launch_bounds__(THREADS)
+    k_find_digit(uint2* __restrict__ state, uint32_t* __restrict__ hist, const LayerDesc* __restrict__ layers,
+                 const uint32_t* __restrict__ large_ids, int* __restrict__ status, int W, int pass) {
+  __shared__ uint32_t sh[NBINS];
+  __shared__ uint32_t sh_scan[THREADS];
+  __shared__ uint32_t res[4];
+  const uint32_t pair = blockIdx.x;
+  const int nb = pass_bins(pass), shift = pass_shift(pass);
+  uint32_t* gh = hist + static_cast<uint64_t>(pair) * NBINS;
+  for (int b = threadIdx.x; b < nb; b += THREADS) {
+    sh[b] = gh[b];
+    gh[b] = 0;
+  }
+  __syncthreads();
+  uint32_t prefix, krem;
+  if (pass == 0) {
+    prefix = 0;
+    krem = layers[large_ids[pair / W]].k;
+  } else {
+    const uint2 s = state[pair];
+    prefix = s.x;
+    krem = s.y;
+  }
+  find_digit(sh, nb, krem, sh_scan, res);
+  if (threadIdx.x == 0) {
+    if (res[2]) {
+      state[pair] = make_uint2(prefix | (res[0] << shift), res[1]);
+    } else {
+      atomicMin(status, STATUS_INTERNAL);
+      state[pair] = make_uint2(0xffffffffu, 0u);  // selects nothing
+    }
+  }
+}
+
+// Per chunk: how many keys are above the threshold and how many equal it.  grid = (chunks, W).
+template <bool VEC>
+__global__ void __launch_bounds__(THREADS)
+    k_count_dense(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
+                  const LayerDesc* __restrict__ layers, const uint2* __restrict__ state, uint2* __restrict__ chunk_cnt,
+                  float eps, uint64_t N, int W, uint32_t n_chunks) {
+  __shared__ uint32_t sh_cnt[2];
+  const Chunk c = chunks[blockIdx.x];
+  const int w = blockIdx.y;
+  const uint32_t pair = static_cast<uint32_t>(layers[c.layer].large_index) * W + w;
+  const uint32_t T = state[pair].x;
+  if (threadIdx.x < 2) sh_cnt[threadIdx.x] = 0;
+  __syncthreads();
+  const uint64_t lo = c.a, hi = lo + c.len;
+  const uint64_t s0 = lo & ~3ull;
+  const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+  const float* a = acc + static_cast<uint64_t>(w) * N;
+  uint32_t gt = 0, eq = 0;
+  for (uint32_t it = 0; it < n_iter; ++it) {
+    const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+    float av[4], wv[4];
+    load4<VEC>(a, e0, lo, hi, av);
+    load4<VEC>(weights, e0, lo, hi, wv);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint64_t e = e0 + q;
+      const bool in = e >= lo && e < hi;
+      const uint32_t key = imp_key(av[q], wv[q], eps);
+      gt += (in && key > T) ? 1u : 0u;
+      eq += (in && key == T) ? 1u : 0u;
+    }
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    gt += __shfl_xor_sync(0xffffffffu, gt, d);
+    eq += __shfl_xor_sync(0xffffffffu, eq, d);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    atomicAdd(&sh_cnt[0], gt);
+    atomicAdd(&sh_cnt[1], eq);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) chunk_cnt[static_cast<uint64_t>(w) * n_chunks + blockIdx.x] = make_uint2(sh_cnt[0], sh_cnt[1]);
+}
+
+// Step (d): stable compaction of the selected elements of a chunk into the worker's list.
+// An element is selected if key > T, or key == T and fewer than r T-valued elements of the
+// layer precede it; its list position is (#greater before it) + min(#equal before it, r).
+// grid = (chunks, W).
+template <bool VEC>
+__global__ void __launch_bounds__(THREADS)
+    k_write_dense(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
+                  const LayerDesc* __restrict__ layers, const uint2* __restrict__ state,
+                  const uint2* __restrict__ chunk_cnt, uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val,
+                  int* __restrict__ status, float eps, uint64_t N, uint64_t K, int W, uint32_t n_chunks) {
+  __shared__ uint32_t sh_warp[WARPS];
+  __shared__ uint32_t sh_base[2];
+  const Chunk c = chunks[blockIdx.x];
+  const int w = blockIdx.y;
+  const LayerDesc L = layers[c.layer];
+  const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
+  const uint2 st = state[pair];
+  const uint32_t T = st.x, r = st.y;
+  // counts of the layer's chunks in front of this one
+  if (threadIdx.x < 2) sh_base[threadIdx.x] = 0;
+  __syncthreads();
+  {
+    const uint2* cc = chunk_cnt + static_cast<uint64_t>(w) * n_chunks;
+    uint32_t g = 0, q = 0;
+    for (uint32_t j = c.first_chunk_of_layer + threadIdx.x; j < blockIdx.x; j += THREADS) {
+      const uint2 v = cc[j];
+      g += v.x;
+      q += v.y;
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      g += __shfl_xor_sync(0xffffffffu, g, d);
+      q += __shfl_xor_sync(0xffffffffu, q, d);
+    }
+    if ((threadIdx.x & 31) == 0 && (g | q)) {
+      atomicAdd(&sh_base[0], g);
+      atomicAdd(&sh_base[1], q);
+    }
+  }
+  __syncthreads();
+  uint32_t run_gt = sh_base[0], run_eq = sh_base[1];
+  const uint64_t lo = c.a, hi = lo + c.len;
+  const uint64_t s0 = lo & ~3ull;
+  const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+  const float* a = acc + static_cast<uint64_t>(w) * N;
+  uint32_t* out_i = sel_idx + static_cast<uint64_t>(w) * K + L.koff;
+  float* out_v = sel_val + static_cast<uint64_t>(w) * K + L.koff;
+  for (uint32_t it = 0; it < n_iter; ++it) {
+    const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+    float av[4], wv[4];
+    load4<VEC>(a, e0, lo, hi, av);
+    load4<VEC>(weights, e0, lo, hi, wv);
+    uint32_t fg = 0, fe = 0;  // per-element flags
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint64_t e = e0 + q;
+      const bool in = e >= lo && e < hi;
+      const uint32_t key = imp_key(av[q], wv[q], eps);
+      fg |= (in && key > T) ? (1u << q) : 0u;
+      fe |= (in && key == T) ? (1u << q) : 0u;
+    }
+    uint32_t total;
+    const uint32_t packed = static_cast<uint32_t>(__popc(fg)) | (static_cast<uint32_t>(__popc(fe)) << 16);
+    const uint32_t ex = block_excl_scan(packed, sh_warp, total);
+    uint32_t g_before = run_gt + (ex & 0xffffu), q_before = run_eq + (ex >> 16);
+    if (fg | fe) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const bool isg = (fg >> q) & 1u, ise = (fe >> q) & 1u;
+        if (isg || (ise && q_before < r)) {
+          const uint32_t pos = g_before + (q_before < r ? q_before : r);
+          if (pos < L.k) {
+            out_i[pos] = static_cast<uint32_t>(e0 + q);
+            out_v[pos] = av[q];
+          } else {
+            atomicMin(status, STATUS_INTERNAL);
+          }
+        }
+        g_before += isg ? 1u : 0u;
+        q_before += ise ? 1u : 0u;
+      }
+    }
+    run_gt += total & 0xffffu;
+    run_eq += total >> 16;
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// one-CTA path: steps (a)-(d) of a whole (worker, layer) pair with n <= SMALL_MAX, keys in
+// shared memory.  grid = (small layers, W); dynamic shared memory = 4 * max n bytes.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(THREADS)
+    k_small(const float* __restrict__ grads, const float* __restrict__ weights, float* __restrict__ acc,
+            float* __restrict__ update, const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ small_ids,
+            uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val, int* __restrict__ status, float eps,
+            uint64_t N, uint64_t K) {
+  extern __shared__ uint32_t keys[];
+  __shared__ uint32_t hist[NBINS];
+  __shared__ uint32_t sh_scan[THREADS];
+  __shared__ uint32_t sh_warp[WARPS];
+  __shared__ uint32_t res[4];
+  const LayerDesc L = layers[small_ids[blockIdx.x]];
+  const int w = blockIdx.y;
+  const int tid = threadIdx.x;
+  const uint32_t n = L.n;
+  float* a = acc + static_cast<uint64_t>(w) * N + L.off;
+  const float* g = grads + static_cast<uint64_t>(w) * N + L.off;
+  const float* wt = weights + L.off;
+  for (uint32_t i = tid; i < n; i += THREADS) {
+    const float v = __fadd_rn(a[i], __ldcs(g + i));
+    a[i] = v;
+    keys[i] = imp_key(v, wt[i], eps);
+    if (w == 0) update[L.off + i] = 0.0f;
+  }
+  __syncthreads();
+  uint32_t prefix = 0, krem = L.k;
+#pragma unroll 1
+  for (int pass = 0; pass < N_PASSES; ++pass) {
+    const int shift = pass_shift(pass), nb = pass_bins(pass);
+    const int prev_shift = pass == 0 ? 31 : pass_shift(pass - 1);
+    const uint32_t want = prefix >> prev_shift;
+    for (int b = tid; b < nb; b += THREADS) hist[b] = 0;
+    __syncthreads();
+    for (uint32_t i = tid; i < n; i += THREADS) {
+      const uint32_t key = keys[i];
+      if ((key >> prev_shift) == want) atomicAdd(&hist[(key >> shift) & (nb - 1)], 1u);
+    }
+    __syncthreads();
+    find_digit(hist, nb, krem, sh_scan, res);
+    if (!res[2]) {
+      if (tid == 0) atomicMin(status, STATUS_INTERNAL);
+      return;
+    }
+    prefix |= res[0] << shift;
+    krem = res[1];
+    __syncthreads();
+  }
+  const uint32_t T = prefix, r = krem;
+  uint32_t* out_i = sel_idx + static_cast<uint64_t>(w) * K + L.koff;
+  float* out_v = sel_val + static_cast<uint64_t>(w) * K + L.koff;
+  uint32_t run_gt = 0, run_eq = 0;
+  for (uint32_t i0 = 0; i0 < n; i0 += THREADS) {
+    const uint32_t i = i0 + tid;
+    const uint32_t key = i < n ? keys[i] : 0u;
+    const bool isg = i < n && key > T, ise = i < n && key == T;
+    uint32_t total;
+    const uint32_t ex = block_excl_scan((isg ? 1u : 0u) | (ise ? 1u << 16 : 0u), sh_warp, total);
+    const uint32_t g_before = run_gt + (ex & 0xffffu), q_before = run_eq + (ex >> 16);
+    if (isg || (ise && q_before < r)) {
+      const uint32_t pos = g_before + (q_before < r ? q_before : r);
+      if (pos < L.k) {
+        out_i[pos] = L.off + i;
+        out_v[pos] = a[i];
+      } else {
+        atomicMin(status, STATUS_INTERNAL);
+      }
+    }
+    run_gt += total & 0xffffu;
+    run_eq += total >> 16;
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// steps (e)-(g): gather every worker's residual at the leader's indices, sum in ascending
+// worker order, scatter into the (already zeroed) dense update, zero what was sent.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(THREADS)
+    k_gather_sum_scatter(const uint32_t* __restrict__ leader_idx, float* __restrict__ acc, float* __restrict__ update,
+                         uint64_t N, uint64_t K, int W) {
+  const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (j >= K) return;
+  const uint64_t i = leader_idx[j];
+  float* p = acc + i;
+  float s = 0.0f;
+  for (int w0 = 0; w0 < W; w0 += 8) {  // loads of a group are independent; the sum keeps worker order
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = (w0 + u < W) ? p[static_cast<uint64_t>(w0 + u) * N] : 0.0f;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
+    }
+  }
+  for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
+  update[i] = __fadd_rn(0.0f, s);
+}
+
+// byte mask of the index set (Algorithm 1's encode_uint8(Mask)); dst is zeroed by the caller
+__global__ void __launch_bounds__(THREADS) k_mask_scatter(const uint32_t* __restrict__ leader_idx, uint8_t* __restrict__ dst, uint64_t K) {
+  const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (j < K) dst[leader_idx[j]] = 1;
+}
+
+}  // namespace iwp

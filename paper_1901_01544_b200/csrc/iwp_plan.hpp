@@ -1,0 +1,149 @@
+// Host-side planner: turns a layer-size list into the tables the kernels walk.
+// Pure C++ (no CUDA): also used by iwp_plan_sizes(), which runs without a GPU.
+//
+// Every tensor is one selection unit (Algorithm 1 loops over layers j = 0..M).  Layers of at
+// most SMALL_MAX elements take the one-CTA path (the whole (worker, layer) problem fits in
+// shared memory); all others are cut into tiles and chunks:
+//   tile   <= TILE consecutive elements of ONE layer, never crossing a multiple of TILE of the
+//          flat element space, so that a tile is at most TILE/4 aligned 128-bit slots;
+//   chunk  <= CHUNK_TILES consecutive tiles of one layer: the unit of work of the select kernels.
+#pragma once
+#include <cmath>
+#include <cstdint>
+#include <vector>
+
+namespace iwp {
+
+constexpr uint32_t TILE = 4096;
+constexpr uint32_t CHUNK_TILES = 16;
+constexpr uint32_t SMALL_MAX = 16384;
+constexpr uint32_t NBINS = 2048;
+
+struct LayerDesc {
+  uint32_t off;         // flat offset of the first element
+  uint32_t n;           // elements
+  uint32_t k;           // keep count
+  uint32_t koff;        // offset of the layer's segment inside a worker's list
+  int32_t large_index;  // index among tiled layers, -1 on the one-CTA path
+  uint32_t first_tile;  // tiled layers: first tile / chunk and their counts
+  uint32_t n_tiles;
+  uint32_t first_chunk;
+  uint32_t n_chunks;
+};
+
+struct Tile {
+  uint32_t a;      // first element (flat)
+  uint32_t len;    // 1..TILE
+  uint32_t layer;  // owning layer
+  uint32_t large_index;
+};
+
+struct Chunk {
+  uint32_t a;           // first element (flat)
+  uint32_t len;         // elements
+  uint32_t layer;       // owning layer
+  uint32_t first_tile;  // first tile of the chunk
+  uint32_t n_tiles;
+  uint32_t first_chunk_of_layer;
+};
+
+inline int64_t keep_count(int64_t n, double ratio) {
+  if (n < 1 || !(ratio >= 1.0) || !std::isfinite(ratio)) return 0;
+  double q = std::ceil(static_cast<double>(n) / ratio);
+  int64_t k = static_cast<int64_t>(q);
+  if (k < 1) k = 1;
+  if (k > n) k = n;
+  return k;
+}
+
+inline uint64_t mix64(uint64_t z) {
+  z ^= z >> 30;
+  z *= 0xBF58476D1CE4E5B9ull;
+  z ^= z >> 27;
+  z *= 0x94D049BB133111EBull;
+  z ^= z >> 31;
+  return z;
+}
+
+inline int32_t leader_at(uint64_t seed, uint64_t t, int32_t W) {
+  if (W < 1) return -1;
+  const uint64_t z = mix64(seed + (t + 1) * 0x9E3779B97F4A7C15ull);
+  return static_cast<int32_t>(((z >> 32) * static_cast<uint64_t>(W)) >> 32);
+}
+
+struct Plan {
+  std::vector<LayerDesc> layers;
+  std::vector<Tile> tiles;
+  std::vector<Chunk> chunks;
+  std::vector<uint32_t> small_layers;  // layer ids on the one-CTA path
+  std::vector<uint32_t> large_layers;  // layer ids on the tiled path
+  uint64_t N = 0, K = 0;
+  uint32_t max_small_n = 0;
+  int32_t W = 0;
+  bool valid = false;
+};
+
+inline Plan make_plan(const int64_t* sizes, int32_t n_layers, int32_t W, double ratio, float eps) {
+  Plan p;
+  if (!sizes || n_layers < 1 || W < 1 || !(ratio >= 1.0) || !std::isfinite(ratio) || !(eps > 0.f) ||
+      !std::isfinite(eps))
+    return p;
+  uint64_t N = 0;
+  for (int32_t l = 0; l < n_layers; ++l) {
+    if (sizes[l] < 1) return p;
+    N += static_cast<uint64_t>(sizes[l]);
+    if (N >= (1ull << 32)) return p;
+  }
+  p.W = W;
+  uint64_t off = 0, koff = 0;
+  for (int32_t l = 0; l < n_layers; ++l) {
+    LayerDesc d{};
+    d.off = static_cast<uint32_t>(off);
+    d.n = static_cast<uint32_t>(sizes[l]);
+    d.k = static_cast<uint32_t>(keep_count(sizes[l], ratio));
+    d.koff = static_cast<uint32_t>(koff);
+    d.large_index = -1;
+    if (d.n <= SMALL_MAX) {
+      p.small_layers.push_back(static_cast<uint32_t>(l));
+      if (d.n > p.max_small_n) p.max_small_n = d.n;
+    } else {
+      d.large_index = static_cast<int32_t>(p.large_layers.size());
+      p.large_layers.push_back(static_cast<uint32_t>(l));
+      d.first_tile = static_cast<uint32_t>(p.tiles.size());
+      d.first_chunk = static_cast<uint32_t>(p.chunks.size());
+      uint64_t a = off;
+      const uint64_t end = off + d.n;
+      while (a < end) {
+        uint64_t b = (a / TILE + 1) * TILE;  // next multiple of TILE
+        if (b > end) b = end;
+        Tile t{static_cast<uint32_t>(a), static_cast<uint32_t>(b - a), static_cast<uint32_t>(l),
+               static_cast<uint32_t>(d.large_index)};
+        p.tiles.push_back(t);
+        a = b;
+      }
+      d.n_tiles = static_cast<uint32_t>(p.tiles.size()) - d.first_tile;
+      for (uint32_t t0 = 0; t0 < d.n_tiles; t0 += CHUNK_TILES) {
+        const uint32_t nt = (d.n_tiles - t0 < CHUNK_TILES) ? d.n_tiles - t0 : CHUNK_TILES;
+        Chunk c{};
+        c.first_tile = d.first_tile + t0;
+        c.n_tiles = nt;
+        c.a = p.tiles[c.first_tile].a;
+        const Tile& last = p.tiles[c.first_tile + nt - 1];
+        c.len = last.a + last.len - c.a;
+        c.layer = static_cast<uint32_t>(l);
+        c.first_chunk_of_layer = d.first_chunk;
+        p.chunks.push_back(c);
+      }
+      d.n_chunks = static_cast<uint32_t>(p.chunks.size()) - d.first_chunk;
+    }
+    p.layers.push_back(d);
+    off += d.n;
+    koff += d.k;
+  }
+  p.N = off;
+  p.K = koff;
+  p.valid = true;
+  return p;
+}
+
+}  // namespace iwp

@@ -1,0 +1,63 @@
+"""Shared helper of the GPU parity tests: runs the CUDA library and the CPU oracle on the
+same seeded inputs and compares every output bit for bit."""
+import numpy as np
+import torch
+
+import oracle
+from paper_1901_01544_b200.binding import Pruner
+
+
+def u32(a: np.ndarray) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+
+
+def assert_bits_equal(got: np.ndarray, want: np.ndarray, what: str):
+    g, w = u32(got), u32(want)
+    if not np.array_equal(g, w):
+        bad = np.flatnonzero(g != w)
+        i = int(bad[0])
+        raise AssertionError(f"{what}: {bad.size} of {g.size} differ; first at {i}: got {got.flat[i]!r} "
+                             f"(0x{int(g.flat[i]):08x}) want {want.flat[i]!r} (0x{int(w.flat[i]):08x})")
+
+
+def compare_state(pr: Pruner, orc: "oracle.Oracle", update_gpu: torch.Tensor, update_cpu: np.ndarray, tag: str,
+                  check_mask: bool = True):
+    assert pr.sync_status() == 0, f"{tag}: device status {pr.sync_status()}"
+    assert pr.leader == orc.leader, f"{tag}: leader {pr.leader} != {orc.leader}"
+    assert_bits_equal(update_gpu.cpu().numpy(), update_cpu, f"{tag}: update")
+    for w in range(pr.W):
+        idx, val = pr.selection(w)
+        oi, ov = orc.selection(w)
+        gi = idx.cpu().numpy().view(np.uint32)
+        if not np.array_equal(gi, oi):
+            bad = np.flatnonzero(gi != oi)
+            raise AssertionError(f"{tag}: worker {w} list indices differ at {bad.size} of {gi.size} positions; "
+                                 f"first at {int(bad[0])}: got {int(gi[bad[0]])} want {int(oi[bad[0]])}")
+        assert_bits_equal(val.cpu().numpy(), ov, f"{tag}: worker {w} list values")
+        assert_bits_equal(pr.residual(w).cpu().numpy(), orc.residual(w), f"{tag}: worker {w} residual")
+    if check_mask:
+        assert np.array_equal(pr.mask().cpu().numpy(), orc.mask()), f"{tag}: mask"
+
+
+def run_parity(layer_sizes, W, ratio, eps, seed, steps, weights: torch.Tensor, grads_fn, options=None,
+               leader_overrides=None, check_mask=True, threads=0):
+    """weights: CUDA tensor [N]; grads_fn(t) -> CUDA tensor [W, N]."""
+    pr = Pruner(layer_sizes, W, ratio, eps, seed)
+    orc = oracle.Oracle(layer_sizes, W, ratio, eps, seed, threads=threads)
+    assert (pr.N, pr.K) == (orc.N, orc.K)
+    assert pr.layout() == orc.layout()
+    for k, v in (options or {}).items():
+        pr.set_option(k, v)
+    w_host = weights.cpu().numpy()
+    update = torch.full((pr.N,), float("nan"), dtype=torch.float32, device="cuda")
+    for t in range(steps):
+        if leader_overrides is not None:
+            pr.set_option("leader_override", leader_overrides[t])
+            orc.set_leader_override(leader_overrides[t])
+        g = grads_fn(t)
+        pr.step(g, weights, update)
+        upd_cpu = orc.step(np.ascontiguousarray(g.cpu().numpy()), w_host)
+        compare_state(pr, orc, update, upd_cpu, f"step {t}", check_mask=check_mask)
+        update.fill_(float("nan"))  # the next step must overwrite every element
+    pr.close()
+    orc.close()

@@ -1,0 +1,125 @@
+"""GPU tests of the API contract: determinism, reset / checkpoint round trip, the host-buffer
+entry point, option and misuse handling.  Nothing here faults, traps or hangs the device."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1901_01544_b200 import binding
+from paper_1901_01544_b200.binding import Pruner
+from parity import assert_bits_equal
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _inputs(W, N, seed):
+    g = torch.Generator(device=DEV)
+    g.manual_seed(seed)
+    weights = torch.randn(N, generator=g, device=DEV) * 0.05
+    grads = [torch.randn((W, N), generator=g, device=DEV) * 1e-3 for _ in range(3)]
+    return weights, grads
+
+
+def test_same_inputs_same_bytes():
+    sizes, W = [70000, 512, 33000], 4
+    N = sum(sizes)
+    weights, grads = _inputs(W, N, 1)
+    outs = []
+    for rep in range(2):
+        pr = Pruner(sizes, W, 32.0, 1e-8, 9)
+        o = []
+        for g in grads:
+            o.append(pr.step(g, weights).clone())
+            o += [pr.residual(w) for w in range(W)] + [pr.selection(w)[0] for w in range(W)]
+        outs.append(o)
+        pr.close()
+    for a, b in zip(*outs):
+        assert torch.equal(a.view(torch.int32), b.view(torch.int32))
+
+
+def test_reset_and_checkpoint_roundtrip():
+    sizes, W = [50000, 100], 3
+    N = sum(sizes)
+    weights, grads = _inputs(W, N, 2)
+    pr = Pruner(sizes, W, 16.0, 1e-8, 5)
+    u0 = pr.step(grads[0], weights).clone()
+    u1 = pr.step(grads[1], weights).clone()
+    saved = [pr.residual(w) for w in range(W)]
+    t_saved = pr.t
+    u2 = pr.step(grads[2], weights).clone()
+    pr.reset()
+    assert pr.t == 0 and pr.leader == -1
+    assert all(int(pr.residual(w).abs().max().item() == 0) for w in range(W))
+    assert torch.equal(pr.step(grads[0], weights), u0) and torch.equal(pr.step(grads[1], weights), u1)
+    # resume from the checkpoint in a fresh context
+    pr2 = Pruner(sizes, W, 16.0, 1e-8, 5)
+    for w in range(W):
+        pr2.set_residual(w, saved[w])
+    pr2.set_step(t_saved)
+    assert torch.equal(pr2.step(grads[2], weights).view(torch.int32), u2.view(torch.int32))
+    assert pr2.leader == binding.iwp_leader_at(5, t_saved, W)
+    pr.close()
+    pr2.close()
+
+
+def test_host_buffer_entry_point_matches_oracle():
+    sizes, W = [40000, 300, 20000], 4
+    N = sum(sizes)
+    weights, grads = _inputs(W, N, 3)
+    pr = Pruner(sizes, W, 64.0, 1e-8, 0)
+    orc = oracle.Oracle(sizes, W, 64.0, 1e-8, 0)
+    wh = weights.cpu().pin_memory()
+    uh = torch.empty(N).pin_memory()
+    for g in grads:
+        gh = g.cpu().pin_memory()
+        pr.step_host(gh, wh, uh)
+        want = orc.step(gh.numpy(), wh.numpy())
+        assert_bits_equal(uh.numpy(), want, "update via host buffers")
+    assert pr.sync_status() == 0
+    pr.close()
+
+
+def test_runs_on_a_side_stream():
+    sizes, W = [60000], 2
+    N = sum(sizes)
+    weights, grads = _inputs(W, N, 4)
+    ref = Pruner(sizes, W, 32.0, 1e-8, 0)
+    want = ref.step(grads[0], weights).clone()
+    ref.close()
+    s = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        pr = Pruner(sizes, W, 32.0, 1e-8, 0)
+        got = pr.step(grads[0], weights)
+        assert pr.sync_status() == 0
+    s.synchronize()
+    assert torch.equal(got, want)
+    pr.close()
+
+
+def test_options_stats_and_misuse():
+    pr = Pruner([5000, 20000], 2, 8.0, 1e-8, 0)
+    L = binding.lib()
+    h = pr._h
+    E = binding.IWP_ERR_INVALID
+    assert L.iwp_set_option(h, b"no_such_option", 1) == E
+    assert L.iwp_set_option(h, b"leader_override", 2) == E and L.iwp_set_option(h, b"leader_override", -2) == E
+    assert L.iwp_set_option(h, b"force_scalar", 7) == E
+    assert L.iwp_set_option(h, b"leader_override", 1) == 0
+    v = C.c_int64()
+    assert L.iwp_get_stat(h, b"nope", C.byref(v)) == E
+    assert L.iwp_get_residual(h, 2, 0) == E and L.iwp_get_residual(h, -1, 0) == E
+    assert L.iwp_get_selection(h, 5, None, None) == E
+    assert L.iwp_set_step(h, -1) == E
+    assert L.iwp_step(h, None, None, None) == E
+    assert pr.t == 0 and pr.stat("launches") == 0
+    weights, grads = _inputs(2, 25000, 6)
+    pr.step(grads[0], weights)
+    assert pr.leader == 1 and pr.t == 1 and pr.stat("launches") > 0 and pr.stat("device_bytes") >= 2 * 25000 * 4
+    assert pr.sync_status() == 0
+    assert pr.layout() == ([0, 5000], [625, 2500])
+    pr.close()
+    pr.close()  # idempotent

@@ -1,0 +1,191 @@
+"""GPU parity: the CUDA library against the CPU oracle, element by element and bit for bit
+(update, residuals, ordered (index, value) lists, leader, byte mask), through the C ABI.
+
+Tolerance: none.  Indices, masks and residuals are integer/bit work; the update is a sum in
+a fixed worker order of IEEE binary32 additions on both sides, so it is compared bit-exactly
+as well (the 1e-6 relative allowance would only apply to an unordered reduction, which
+this library does not use)."""
+import json
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from paper_1901_01544_b200 import workloads as wl
+from parity import assert_bits_equal, run_parity
+
+pytestmark = pytest.mark.gpu
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+DEV = "cuda"
+
+
+def _randn(shape, seed, scale=1.0):
+    g = torch.Generator(device=DEV)
+    g.manual_seed(seed)
+    return torch.randn(shape, generator=g, device=DEV, dtype=torch.float32) * scale
+
+
+def _weights(N, seed, zero_frac=0.05, scale=0.05):
+    w = _randn((N,), seed, scale)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(seed + 1)
+    w[torch.rand(N, generator=g, device=DEV) < zero_frac] = 0.0
+    return w
+
+
+# ------------------------------------------------------------------ hand-worked example
+
+
+def test_worked_example_on_gpu():
+    g = json.load(open(os.path.join(GOLD, "worked_example.json")))
+    from paper_1901_01544_b200.binding import Pruner
+
+    pr = Pruner(g["layer_sizes"], g["W"], g["ratio"], g["eps"], 0)
+    weights = torch.tensor(g["weights"], dtype=torch.float32, device=DEV)
+    for st in g["steps"]:
+        pr.set_option("leader_override", st["leader"])
+        upd = pr.step(torch.tensor(st["grads"], dtype=torch.float32, device=DEV), weights)
+        assert pr.sync_status() == 0 and pr.leader == st["leader"]
+        assert_bits_equal(upd.cpu().numpy(), np.array(st["update"], np.float32), "update")
+        for w in range(g["W"]):
+            idx, val = pr.selection(w)
+            assert idx.cpu().tolist() == st["lists"][w]
+            assert_bits_equal(val.cpu().numpy(), np.array(st["list_vals"][w], np.float32), "list values")
+            assert_bits_equal(pr.residual(w).cpu().numpy(), np.array(st["residual"][w], np.float32), "residual")
+        assert pr.mask().cpu().tolist() == [1 if i in st["lists"][st["leader"]] else 0 for i in range(8)]
+    pr.close()
+
+
+# ------------------------------------------------------------------ tiny and adversarial inputs
+
+CASES = {
+    # name: (layer_sizes, W, ratio)
+    "small_only": ([5, 1, 12, 3, 64, 300], 3, 3.0),
+    "n_less_than_ratio": ([3, 2, 1, 40], 2, 64.0),
+    "single_element": ([1], 4, 64.0),
+    "one_tiled_layer": ([40000], 2, 16.0),
+    "tiled_odd_total_scalar_path": ([20001, 17, 70003], 3, 10.0),
+    "tiled_unaligned_offsets_vector_path": ([16389, 16387, 40000], 2, 7.0),
+    "mixed_many": ([64, 16385, 256, 100000, 9408, 4096, 36864, 1000, 17000], 4, 58.8),
+    "keep_everything": ([50000, 100], 3, 1.0),
+    "one_worker": ([30000, 70], 1, 20.0),
+    "thirty_three_workers": ([17000, 33], 33, 50.0),
+    "chunk_boundaries": ([65536 * 2 + 4096 + 1, 65536], 2, 64.0),
+}
+
+
+@pytest.mark.parametrize("name", sorted(CASES))
+def test_random_values(name):
+    sizes, W, ratio = CASES[name]
+    N = sum(sizes)
+    weights = _weights(N, 100 + N % 97)
+    run_parity(sizes, W, ratio, 1e-8, seed=7, steps=3, weights=weights,
+               grads_fn=lambda t: _randn((W, N), 1000 * t + 3, 1e-3))
+
+
+@pytest.mark.parametrize("name", ["mixed_many", "tiled_unaligned_offsets_vector_path", "one_tiled_layer"])
+def test_many_ties(name):
+    # coarse values: importances collide all the time, exact cancellations to +0 occur
+    sizes, W, ratio = CASES[name]
+    N = sum(sizes)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(5)
+    weights = torch.randint(-2, 3, (N,), generator=g, device=DEV).float() * 0.5
+
+    def grads(t):
+        gg = torch.Generator(device=DEV)
+        gg.manual_seed(50 + t)
+        return torch.randint(-4, 5, (W, N), generator=gg, device=DEV).float() / 8.0
+
+    run_parity(sizes, W, ratio, 1e-8, seed=1, steps=4, weights=weights, grads_fn=grads)
+
+
+@pytest.mark.parametrize("kind", ["all_equal", "all_zero", "two_values", "zero_weights"])
+def test_degenerate_layers(kind):
+    sizes, W, ratio = [100000, 5000, 37], 3, 32.0
+    N = sum(sizes)
+    if kind == "all_equal":
+        weights = torch.full((N,), -0.5, device=DEV)
+        grads = lambda t: torch.full((W, N), 0.25, device=DEV)
+    elif kind == "all_zero":
+        weights = _weights(N, 3)
+        grads = lambda t: torch.zeros((W, N), device=DEV)
+    elif kind == "two_values":
+        weights = torch.ones(N, device=DEV)
+        g = torch.Generator(device=DEV)
+        g.manual_seed(9)
+        pick = torch.rand((W, N), generator=g, device=DEV) < 0.01  # fewer large values than k: ties at the small one
+        grads = lambda t: torch.where(pick, torch.tensor(1.0, device=DEV), torch.tensor(0.25, device=DEV))
+    else:
+        weights = torch.zeros(N, device=DEV)
+        grads = lambda t: _randn((W, N), 77 + t, 1e-3)
+    run_parity(sizes, W, ratio, 1e-8, seed=2, steps=2, weights=weights, grads_fn=grads)
+
+
+def test_forced_scalar_path_and_leader_override():
+    sizes, W, ratio = [40000, 128, 16385], 4, 16.0
+    N = sum(sizes)
+    weights = _weights(N, 11)
+    run_parity(sizes, W, ratio, 1e-8, seed=0, steps=4, weights=weights,
+               grads_fn=lambda t: _randn((W, N), 31 * t + 1, 1e-2), options={"force_scalar": 1},
+               leader_overrides=[3, 0, 2, 2])
+
+
+def test_exact_select_without_speculation():
+    sizes, W, ratio = [300000, 128, 70000], 4, 64.0
+    N = sum(sizes)
+    weights = _weights(N, 13)
+    run_parity(sizes, W, ratio, 1e-8, seed=0, steps=3, weights=weights,
+               grads_fn=lambda t: _randn((W, N), 17 * t + 2, 1e-2), options={"speculate": 0})
+
+
+def test_misaligned_caller_pointers():
+    # caller buffers offset by one float: the library must fall back to scalar accesses
+    sizes, W, ratio = [40000, 24], 2, 16.0
+    N = sum(sizes)
+    import oracle
+    from paper_1901_01544_b200.binding import Pruner
+
+    pr = Pruner(sizes, W, ratio, 1e-8, 4)
+    orc = oracle.Oracle(sizes, W, ratio, 1e-8, 4)
+    wbuf = torch.zeros(N + 1, device=DEV)
+    wbuf[1:] = _weights(N, 5)
+    gbuf = torch.zeros(W * N + 1, device=DEV)
+    ubuf = torch.zeros(N + 1, device=DEV)
+    for t in range(2):
+        gbuf[1:] = _randn((W * N,), 90 + t, 1e-3)
+        pr.step(gbuf[1:], wbuf[1:], ubuf[1:])
+        want = orc.step(gbuf[1:].view(W, N).cpu().numpy().copy(), wbuf[1:].cpu().numpy().copy())
+        assert pr.sync_status() == 0
+        assert_bits_equal(ubuf[1:].cpu().numpy(), want, "update")
+        for w in range(W):
+            assert_bits_equal(pr.residual(w).cpu().numpy(), orc.residual(w), "residual")
+            assert np.array_equal(pr.selection(w)[0].cpu().numpy().view(np.uint32), orc.selection(w)[0])
+    pr.close()
+
+
+# ------------------------------------------------------------------ the five configurations, scaled
+
+
+def _scaled_case(name):
+    if name == "single_layer":
+        return wl.scaled(wl.single_layer(), [1 << 17], name="c1s")
+    if name == "alexnet_w8":
+        b = wl.alexnet_w8()
+        return wl.scaled(b, [max(3, n // 48 + (n % 7)) for n in b.layer_sizes])
+    if name == "resnet50_w8":
+        b = wl.resnet50_w8()
+        return wl.scaled(b, [max(2, n // 16 + (n % 5)) for n in b.layer_sizes], W=4)
+    if name == "alexnet_w32":
+        b = wl.alexnet_w32()
+        return wl.scaled(b, [max(3, n // 192 + (n % 3)) for n in b.layer_sizes], steps=20)
+    b = wl.flat_1g_w4()
+    return wl.scaled(b, wl.split_equal((1 << 22) + 64, 96), steps=4)
+
+
+@pytest.mark.parametrize("name", sorted(wl.CONFIGS))
+def test_scaled_configs(name):
+    c = _scaled_case(name)
+    weights = c.weights(DEV)
+    run_parity(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, c.steps, weights, lambda t: c.grads(t, DEV))
