@@ -1,0 +1,326 @@
+#!/usr/bin/env python
+"""Benchmark of the importance-weighted pruning step (pruned all-reduce steps/s and achieved
+HBM GB/s) on synthetic inputs of the AlexNet-shaped W=8 configuration by default.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+One JSON line is printed by rank 0.  A "step" is one pass of the whole hot path (accumulate,
+importance, layer-wise top-k, compaction, leader gather, ordered worker sum, scatter, zeroing)
+over one batch of W*N synthetic gradients.  The path has no inter-GPU exchange: with --gpus N
+(under torchrun) every rank runs an independent replica of the same configuration.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "pruned_allreduce_steps_per_s"
+UNIT = "steps/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+def step_bytes(W, N, K):
+    """Compulsory bytes of one step: every input read once, every output written once."""
+    return 4 * W * N + 8 * W * N + 4 * N + 4 * N + 16 * W * K + 8 * K
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        try:
+            self.proc.terminate()  # the exact process started above
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        try:
+            rows = [r.strip().split(", ") for r in open(self.path) if r.strip()]
+            os.unlink(self.path)
+        except Exception:
+            return out
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for nme, v in zip(names, r[3:7]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(nme)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def make_workload(name):
+    from paper_1901_01544_b200 import workloads as wl
+
+    return wl.CONFIGS[name]()
+
+
+# ---------------------------------------------------------------------------------- CPU oracle legs
+
+
+def oracle_timing(c, weights_host, grads_host_fn, steps, warmup):
+    """Times the CPU oracle as it stands on the host cores; returns (steps/s, threads, seconds)."""
+    import oracle
+
+    orc = oracle.Oracle(c.layer_sizes, c.W, c.ratio, c.eps, c.seed)
+    for t in range(warmup):
+        orc.step(grads_host_fn(t), weights_host)
+    t0 = time.perf_counter()
+    for t in range(steps):
+        orc.step(grads_host_fn(warmup + t), weights_host)
+    dt = time.perf_counter() - t0
+    threads = orc.threads
+    orc.close()
+    return steps / dt, threads, dt
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the same configuration, metric and unit."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import torch
+
+    c = make_workload(args.config)
+    weights = c.weights("cpu").numpy()
+    n_sets = 2
+    sets = [c.grads(t, "cpu").numpy() for t in range(n_sets)]
+    sps, threads, dt = oracle_timing(c, weights, lambda t: sets[t % n_sets], args.steps, args.warmup)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": sps, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 / sps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": c.name, "W": c.W, "N": c.N, "ratio": c.ratio, "layers": len(c.layer_sizes),
+                   "note": "CPU oracle, every step a full step of the workload"},
+        "cpu_baseline": {"value": sps, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": f"{args.steps} full steps of {c.name} after {args.warmup} warm-up steps"},
+        "e2e": {"value": sps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------- the CUDA arm
+
+
+def run_ours(args):
+    import torch
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the pruning path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    from paper_1901_01544_b200 import build as lib_build
+
+    if rank == 0:
+        lib_build.build()
+    if dist is not None:
+        dist.barrier()
+    from paper_1901_01544_b200.binding import Pruner
+
+    dev = torch.device("cuda", local)
+    c = make_workload(args.config)
+    W, N = c.W, c.N
+    weights = c.weights(dev)
+    grad_bytes = 4 * W * N
+    n_sets = max(2, min(5, int(24e9 // grad_bytes)))  # distinct gradient batches cycled through
+    sets = [c.grads(t, dev) for t in range(n_sets)]
+    update = torch.empty(N, dtype=torch.float32, device=dev)
+    pr = Pruner(c.layer_sizes, W, c.ratio, c.eps, c.seed)
+    K = pr.K
+    if args.speculate is not None:
+        pr.set_option("speculate", args.speculate)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # warm-up (residuals carry over into the timed region, as in training)
+    for t in range(args.warmup):
+        pr.step(sets[t % n_sets], weights, update)
+    pr.check()
+    pr.set_option("time_stages", 1)
+    launches0 = pr.stat("launches")
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(args.steps):
+        pr.step(sets[(args.warmup + t) % n_sets], weights, update)
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    launches = pr.stat("launches") - launches0
+    pr.check()
+    stage_ms = {k: pr.stat(f"time_{k}_ns") / 1e6 / args.steps for k in ("small", "sample", "accumulate", "select",
+                                                                           "compact", "gather")}
+    spec = {"pairs": pr.stat("spec_pairs"), "failed": pr.stat("spec_failed")}
+    pr.set_option("time_stages", 0)
+    if dist is not None:
+        tt = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_total = float(tt.item())
+    ms_per_step = ms_total / args.steps
+    value = world * args.steps / (ms_total / 1e3)
+
+    # end to end through the host-buffer entry point: H2D of grads + weights and D2H of the update inside
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    gh = [sets[i].cpu().pin_memory() for i in range(min(2, n_sets))]
+    wh = weights.cpu().pin_memory()
+    uh = torch.empty(N, dtype=torch.float32).pin_memory()
+    pr.step_host(gh[0], wh, uh)  # allocates the staging buffers
+    barrier()
+    t0 = time.perf_counter()
+    for t in range(e2e_steps):
+        pr.step_host(gh[t % len(gh)], wh, uh)
+    torch.cuda.synchronize()
+    e2e_dt = time.perf_counter() - t0
+    if dist is not None:
+        tt = torch.tensor([e2e_dt], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_dt = float(tt.item())
+    pr.check()
+    e2e_value = world * e2e_steps / e2e_dt
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_peak()
+    B = step_bytes(W, N, K)
+    plan = __import__("paper_1901_01544_b200.binding", fromlist=["x"]).iwp_plan_sizes(c.layer_sizes, W, c.ratio)
+    Nt = sum(n for n in c.layer_sizes if n > 16384)  # elements on the tiled path
+    # algorithmic bytes of one launch of the dominant kernel (fused accumulate + importance + candidate
+    # emission over all tiled layers): grads read, residual read and written, weights read, update zeroed
+    k1_bytes = 12 * W * Nt + 8 * Nt
+    dom = max(stage_ms, key=stage_ms.get)
+    k1_ms = stage_ms["accumulate"]
+    achieved = k1_bytes / (k1_ms * 1e-3) / 1e9 if k1_ms > 0 else 0.0
+    roofline = {
+        "bound": "hbm", "kernel": "k_accumulate (fused accumulate + importance pass over all tiled layers)",
+        "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+        "traffic": None, "algorithmic_bytes_per_launch": k1_bytes, "ms_per_launch": k1_ms,
+        "dominant_stage_by_time": dom,
+    }
+    eff = B / (ms_per_step * 1e-3) / 1e9
+    step_eff = {"compulsory_bytes": B, "effective_gbs": eff, "frac_of_measured_peak": eff / peak,
+                "frac_of_nominal_8tbs": eff / NOMINAL_HBM_GBS}
+
+    # CPU baseline: the oracle as it stands, a bounded sample (a few full steps) on this machine's cores
+    cpu = None
+    if not args.no_cpu_baseline:
+        w_host = wh.numpy()
+        g_host = [g.numpy() for g in gh]
+        sps, threads, dt = oracle_timing(c, w_host, lambda t: g_host[t % len(g_host)], args.cpu_steps, 1)
+        cpu = {"value": sps, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": f"{args.cpu_steps} full steps of {c.name} after 1 warm-up step ({dt:.1f} s of CPU work)"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": c.name, "W": W, "N": N, "K": K, "ratio": c.ratio, "layers": len(c.layer_sizes),
+                   "l2_policy": f"inputs larger than L2: {grad_bytes * 3 / 1e9:.2f} GB streamed per step, "
+                                f"{n_sets} gradient batches cycled",
+                   "multi_gpu": "independent replicas (the path has no inter-GPU exchange)",
+                   "compression_N_over_K": N / K},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * (W * N + N), "d2h_bytes_per_step": 4 * N,
+                "steps": e2e_steps},
+        "gpu_launches": launches,
+        "roofline": roofline,
+        "step_effective": step_eff,
+        "stage_ms": stage_ms,
+        "speculation": spec,
+        "cpu_baseline": cpu,
+        "clocks": clocks,
+        "plan": plan,
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="alexnet_w8")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--speculate", type=int, default=None, choices=[0, 1])
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

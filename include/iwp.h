@@ -148,12 +148,18 @@ int iwp_reset(iwp_ctx* ctx);
  *   "force_scalar"     1 = never use 128-bit accesses
  *   "speculate"        1 (default) = sample-based threshold guess so that large layers are
  *                      read once; 0 = always the multi-pass exact select.  Both are exact.
+ *   "time_stages"      1 = record a CUDA event at every stage boundary of each following step
+ *                      (read the totals with iwp_get_stat); 0 = stop and discard them
  * Unknown key or out-of-range value: IWP_ERR_INVALID. */
 int iwp_set_option(iwp_ctx* ctx, const char* key, int64_t value);
 
 /* Counters: "launches" (kernels and memsets enqueued since create), "device_bytes",
  * "spec_pairs" / "spec_failed" ((worker, layer) pairs that tried / fell back from the
  * single-read path in the last step; reading them synchronises the stream).
+ * With "time_stages" on: "timed_steps" and the summed device time in nanoseconds of each
+ * stage over those steps - "time_small_ns" (one-CTA path), "time_sample_ns" (threshold
+ * guess from a sample), "time_accumulate_ns" (step (a) on the
+ * tiled path), "time_select_ns" (c), "time_compact_ns" (d), "time_gather_ns" ((e)-(g)).
  * Unknown key: IWP_ERR_INVALID. */
 int iwp_get_stat(iwp_ctx* ctx, const char* key, int64_t* value_host);
 

@@ -6,6 +6,7 @@
 
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "iwp_kernels.cuh"
 #include "iwp_plan.hpp"
@@ -37,9 +38,20 @@ struct iwp_ctx {
   uint2* d_state = nullptr;
   uint32_t* d_hist = nullptr;
   uint2* d_chunk_cnt = nullptr;
+  PairInfo* d_info = nullptr;     // threshold guess and candidate totals per pair
+  uint32_t* cand_key = nullptr;   // candidate slots [tile][worker][CAND_CAP]
+  float* cand_val = nullptr;
+  uint16_t* cand_idx = nullptr;
+  uint32_t* cand_cnt = nullptr;   // [tile][worker]
+  bool info_clean = true;         // d_info holds "no guess" everywhere
+  uint32_t max_sample = 0;
+  uint32_t spec_pairs = 0;
   uint32_t* sel_idx = nullptr;
   float* sel_val = nullptr;
   int* d_status = nullptr;
+  // optional per-stage CUDA-event timing (option "time_stages")
+  bool time_stages = false;
+  std::vector<cudaEvent_t> stage_events;  // N_STAGES + 1 events per timed step
   // staging for iwp_step_host
   float* stg_grads = nullptr;
   float* stg_weights = nullptr;
@@ -48,11 +60,33 @@ struct iwp_ctx {
 
 namespace {
 
+// stages of a step, in launch order; an event is recorded at every boundary when timing is on
+enum Stage { ST_SMALL = 0, ST_SAMPLE, ST_ACCUMULATE, ST_SELECT, ST_COMPACT, ST_GATHER, N_STAGES };
+const char* const kStageKeys[N_STAGES] = {"time_small_ns", "time_sample_ns", "time_accumulate_ns", "time_select_ns", "time_compact_ns",
+                                          "time_gather_ns"};
+
+void stage_mark(iwp_ctx* c) {
+  if (!c->time_stages) return;
+  cudaEvent_t e;
+  if (cudaEventCreate(&e) != cudaSuccess) {
+    cudaGetLastError();
+    return;
+  }
+  cudaEventRecord(e, c->stream);
+  c->stage_events.push_back(e);
+}
+
+void stage_clear(iwp_ctx* c) {
+  for (cudaEvent_t e : c->stage_events) cudaEventDestroy(e);
+  c->stage_events.clear();
+}
+
 struct Sizes {
   uint64_t acc, layers, tiles, chunks, small_ids, large_ids, state, hist, chunk_cnt, sel_idx, sel_val, status;
+  uint64_t info, cand_key, cand_val, cand_idx, cand_cnt;
   uint64_t total() const {
     return acc + layers + tiles + chunks + small_ids + large_ids + state + hist + chunk_cnt + sel_idx + sel_val +
-           status;
+           status + info + cand_key + cand_val + cand_idx + cand_cnt;
   }
 };
 
@@ -74,6 +108,14 @@ Sizes sizes_of(const Plan& p) {
   s.sel_idx = W * p.K * sizeof(uint32_t);
   s.sel_val = W * p.K * sizeof(float);
   s.status = sizeof(int);
+  bool any_spec = false;
+  for (uint32_t l : p.large_layers) any_spec = any_spec || p.layers[l].sample != 0;
+  const uint64_t slots = any_spec ? W * p.tiles.size() : 0;
+  s.info = at_least(pairs * sizeof(PairInfo));
+  s.cand_key = at_least(slots * CAND_CAP * sizeof(uint32_t));
+  s.cand_val = at_least(slots * CAND_CAP * sizeof(float));
+  s.cand_idx = at_least(slots * CAND_CAP * sizeof(uint16_t));
+  s.cand_cnt = at_least(slots * sizeof(uint32_t));
   return s;
 }
 
@@ -103,6 +145,11 @@ void free_all(iwp_ctx* c) {
   cudaFree(c->d_state);
   cudaFree(c->d_hist);
   cudaFree(c->d_chunk_cnt);
+  cudaFree(c->d_info);
+  cudaFree(c->cand_key);
+  cudaFree(c->cand_val);
+  cudaFree(c->cand_idx);
+  cudaFree(c->cand_cnt);
   cudaFree(c->sel_idx);
   cudaFree(c->sel_val);
   cudaFree(c->d_status);
@@ -125,6 +172,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   const int W = p.W;
   const uint64_t N = p.N, K = p.K;
   cudaStream_t s = c->stream;
+  stage_mark(c);
   if (!p.small_layers.empty()) {
     const size_t dyn = static_cast<size_t>(p.max_small_n) * sizeof(uint32_t);
     dim3 grid(static_cast<unsigned>(p.small_layers.size()), static_cast<unsigned>(W));
@@ -132,31 +180,68 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
                                        c->sel_val, c->d_status, c->eps, N, K);
     IWP_LAUNCH_CHECK(c);
   }
-  if (!p.large_layers.empty()) {
+  stage_mark(c);
+  const bool tiled = !p.large_layers.empty();
+  const bool spec = tiled && c->speculate && c->spec_pairs > 0;
+  if (tiled && !spec && !c->info_clean) {  // speculation was switched off: forget the old guesses
+    if (cudaMemsetAsync(c->d_info, 0xff, static_cast<size_t>(c->n_pairs) * sizeof(PairInfo), s) != cudaSuccess) {
+      cudaGetLastError();
+      return IWP_ERR_CUDA;
+    }
+    c->launches += 1;
+    c->info_clean = true;
+  }
+  if (spec) {
+    const size_t dyn = static_cast<size_t>(c->max_sample) * sizeof(uint32_t);
+    k_sample<<<c->n_pairs, THREADS, dyn, s>>>(grads, weights, c->acc, c->d_layers, c->d_large_ids, c->d_info, c->eps, N,
+                                             W, static_cast<uint32_t>(c->t));
+    IWP_LAUNCH_CHECK(c);
+    c->info_clean = false;
+  }
+  stage_mark(c);
+  if (tiled) {
     const unsigned n_tiles = static_cast<unsigned>(p.tiles.size());
+    if (spec) {
+      k_accumulate_emit<VEC><<<n_tiles, THREADS, 0, s>>>(grads, weights, c->acc, update, c->d_tiles, c->d_info,
+                                                         c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->eps, N,
+                                                         W);
+    } else {
+      k_accumulate<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, N, W);
+    }
+    IWP_LAUNCH_CHECK(c);
+  }
+  stage_mark(c);
+  if (tiled) {
     const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
     dim3 cgrid(n_chunks, static_cast<unsigned>(W));
-    k_accumulate<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, N, W);
-    IWP_LAUNCH_CHECK(c);
     for (int pass = 0; pass < N_PASSES; ++pass) {
-      k_hist_dense<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_state, c->d_hist,
-                                                  c->eps, N, W, pass);
+      k_hist<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_info, c->cand_key,
+                                            c->cand_cnt, c->d_state, c->d_hist, c->eps, N, W, pass);
       IWP_LAUNCH_CHECK(c);
       k_find_digit<<<c->n_pairs, THREADS, 0, s>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->d_status, W,
                                                   pass);
       IWP_LAUNCH_CHECK(c);
     }
-    k_count_dense<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_state, c->d_chunk_cnt,
-                                                 c->eps, N, W, n_chunks);
+  }
+  stage_mark(c);
+  if (tiled) {
+    const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
+    dim3 cgrid(n_chunks, static_cast<unsigned>(W));
+    k_count<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_info, c->cand_key,
+                                           c->cand_cnt, c->d_state, c->d_chunk_cnt, c->eps, N, W, n_chunks);
     IWP_LAUNCH_CHECK(c);
-    k_write_dense<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_state, c->d_chunk_cnt,
-                                                 c->sel_idx, c->sel_val, c->d_status, c->eps, N, K, W, n_chunks);
+    k_write<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->d_info,
+                                           c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
+                                           c->d_chunk_cnt, c->sel_idx, c->sel_val, c->d_status, c->eps, N, K, W,
+                                           n_chunks);
     IWP_LAUNCH_CHECK(c);
   }
+  stage_mark(c);
   const unsigned gblocks = static_cast<unsigned>((K + THREADS - 1) / THREADS);
   k_gather_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->acc, update, N,
                                                    K, W);
   IWP_LAUNCH_CHECK(c);
+  stage_mark(c);
   return IWP_OK;
 }
 
@@ -236,6 +321,11 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
   A(&c->d_state, sz.state);
   A(&c->d_hist, sz.hist);
   A(&c->d_chunk_cnt, sz.chunk_cnt);
+  A(&c->d_info, sz.info);
+  A(&c->cand_key, sz.cand_key);
+  A(&c->cand_val, sz.cand_val);
+  A(&c->cand_idx, sz.cand_idx);
+  A(&c->cand_cnt, sz.cand_cnt);
   A(&c->sel_idx, sz.sel_idx);
   A(&c->sel_val, sz.sel_val);
   A(&c->d_status, sz.status);
@@ -260,6 +350,16 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
   ok = ok && cudaMemset(c->sel_idx, 0, sz.sel_idx) == cudaSuccess;
   ok = ok && cudaMemset(c->sel_val, 0, sz.sel_val) == cudaSuccess;
   ok = ok && cudaMemset(c->d_status, 0, sz.status) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_info, 0xff, sz.info) == cudaSuccess;  // guess = none, overflow flag set
+  ok = ok && cudaMemset(c->cand_cnt, 0, sz.cand_cnt) == cudaSuccess;
+  for (uint32_t l : p.large_layers) {
+    if (p.layers[l].sample > c->max_sample) c->max_sample = p.layers[l].sample;
+    if (p.layers[l].sample) c->spec_pairs += static_cast<uint32_t>(W);
+  }
+  if (ok && c->max_sample) {
+    ok = cudaFuncSetAttribute(k_sample, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(c->max_sample * sizeof(uint32_t))) == cudaSuccess;
+  }
   if (ok && p.max_small_n) {
     ok = cudaFuncSetAttribute(k_small, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               static_cast<int>(p.max_small_n * sizeof(uint32_t))) == cudaSuccess;
@@ -278,6 +378,7 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
 int iwp_destroy(iwp_ctx* c) {
   if (!c) return IWP_OK;
   cudaStreamSynchronize(c->stream);
+  stage_clear(c);
   free_all(c);
   cudaGetLastError();
   delete c;
@@ -461,6 +562,13 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
     c->force_scalar = v != 0;
     return IWP_OK;
   }
+  if (!std::strcmp(key, "time_stages")) {
+    if (v != 0 && v != 1) return IWP_ERR_INVALID;
+    cudaStreamSynchronize(c->stream);
+    stage_clear(c);
+    c->time_stages = v != 0;
+    return IWP_OK;
+  }
   if (!std::strcmp(key, "speculate")) {
     if (v != 0 && v != 1) return IWP_ERR_INVALID;
     c->speculate = v != 0;
@@ -479,8 +587,51 @@ int iwp_get_stat(iwp_ctx* c, const char* key, int64_t* value) {
     *value = static_cast<int64_t>(c->device_bytes);
     return IWP_OK;
   }
-  if (!std::strcmp(key, "spec_pairs") || !std::strcmp(key, "spec_failed")) {
+  if (!std::strcmp(key, "timed_steps")) {
+    *value = static_cast<int64_t>(c->stage_events.size() / (N_STAGES + 1));
+    return IWP_OK;
+  }
+  for (int st = 0; st < N_STAGES; ++st) {
+    if (std::strcmp(key, kStageKeys[st])) continue;
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) {
+      cudaGetLastError();
+      return IWP_ERR_CUDA;
+    }
+    double ns = 0.0;
+    const size_t steps = c->stage_events.size() / (N_STAGES + 1);
+    for (size_t i = 0; i < steps; ++i) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, c->stage_events[i * (N_STAGES + 1) + st],
+                               c->stage_events[i * (N_STAGES + 1) + st + 1]) != cudaSuccess) {
+        cudaGetLastError();
+        return IWP_ERR_CUDA;
+      }
+      ns += static_cast<double>(ms) * 1e6;
+    }
+    *value = static_cast<int64_t>(ns);
+    return IWP_OK;
+  }
+  if (!std::strcmp(key, "spec_pairs")) {
+    *value = c->speculate ? c->spec_pairs : 0;
+    return IWP_OK;
+  }
+  if (!std::strcmp(key, "spec_failed")) {
     *value = 0;
+    if (!c->speculate || c->spec_pairs == 0 || c->info_clean) return IWP_OK;
+    std::vector<PairInfo> h(c->n_pairs);
+    if (cudaMemcpyAsync(h.data(), c->d_info, h.size() * sizeof(PairInfo), cudaMemcpyDeviceToHost, c->stream) !=
+            cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess) {
+      cudaGetLastError();
+      return IWP_ERR_CUDA;
+    }
+    const int W = c->plan.W;
+    for (uint32_t pr = 0; pr < c->n_pairs; ++pr) {
+      const LayerDesc& L = c->plan.layers[c->plan.large_layers[pr / W]];
+      if (L.sample == 0) continue;
+      const bool cand = h[pr].guess != GUESS_NONE && h[pr].total >= L.k && (h[pr].flags & 1u) == 0u;
+      if (!cand) *value += 1;
+    }
     return IWP_OK;
   }
   return IWP_ERR_INVALID;

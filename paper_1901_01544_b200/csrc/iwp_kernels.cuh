@@ -25,6 +25,20 @@ __host__ __device__ constexpr int pass_shift(int pass) { return pass == 0 ? 21 :
 __host__ __device__ constexpr int pass_bins(int pass) { return pass == 2 ? 1024 : 2048; }
 constexpr int N_PASSES = 3;
 
+// Per (tiled layer, worker) pair: the threshold guess of the single-read path and what the
+// fused accumulate pass found with it.
+struct PairInfo {
+  uint32_t guess;  // candidates are the elements with importance pattern >= guess; GUESS_NONE = none
+  uint32_t total;  // number of such elements in the layer
+  uint32_t flags;  // bit 0: some (tile, worker) slot overflowed
+  uint32_t pad;
+};
+
+// The candidates hold the exact top-k iff there are at least k of them and none was dropped.
+__device__ __forceinline__ bool pair_is_cand(const PairInfo& pi, uint32_t k) {
+  return pi.guess != GUESS_NONE && pi.total >= k && (pi.flags & 1u) == 0u;
+}
+
 // ---------------------------------------------------------------------------------------
 // element helpers
 // ---------------------------------------------------------------------------------------
@@ -33,6 +47,11 @@ constexpr int N_PASSES = 3;
 // float orders like the float, so the unsigned pattern is the sort key.
 __device__ __forceinline__ uint32_t imp_key(float acc, float w, float eps) {
   return __float_as_uint(__fdiv_rn(fabsf(acc), __fadd_rn(fabsf(w), eps)));
+}
+
+__device__ __forceinline__ float imp_den(float w, float eps) { return __fadd_rn(fabsf(w), eps); }
+__device__ __forceinline__ uint32_t imp_key_den(float acc, float den) {
+  return __float_as_uint(__fdiv_rn(fabsf(acc), den));
 }
 
 // A slot is four consecutive floats starting at a multiple of four elements.  [lo, hi) is
@@ -151,6 +170,39 @@ __device__ __forceinline__ void find_digit(const uint32_t* hist, int nb, uint32_
   __syncthreads();
 }
 
+// Exact radix select on keys held in shared memory: the krem-th largest of n keys.
+// On success T = that key and r = how many T-valued keys belong to the top krem.
+// hist: NBINS words, sh_scan: THREADS words, res: 4 words.  Returns false if the counts are
+// inconsistent (krem > n).  All threads of the block must call it.
+__device__ __forceinline__ bool smem_radix_select(const uint32_t* keys, uint32_t n, uint32_t krem, uint32_t* hist,
+                                                  uint32_t* sh_scan, uint32_t* res, uint32_t& T, uint32_t& r) {
+  const int tid = threadIdx.x;
+  uint32_t prefix = 0;
+#pragma unroll 1
+  for (int pass = 0; pass < N_PASSES; ++pass) {
+    const int shift = pass_shift(pass), nb = pass_bins(pass);
+    const int prev_shift = pass == 0 ? 31 : pass_shift(pass - 1);
+    const uint32_t want = prefix >> prev_shift;
+    for (int b = tid; b < nb; b += THREADS) hist[b] = 0;
+    __syncthreads();
+    for (uint32_t i = tid; i < n; i += THREADS) {
+      const uint32_t key = keys[i];
+      if ((key >> prev_shift) == want) atomicAdd(&hist[(key >> shift) & (nb - 1)], 1u);
+    }
+    __syncthreads();
+    find_digit(hist, nb, krem, sh_scan, res);
+    const bool found = res[2] != 0;
+    const uint32_t d = res[0], kr = res[1];
+    __syncthreads();
+    if (!found) return false;
+    prefix |= d << shift;
+    krem = kr;
+  }
+  T = prefix;
+  r = krem;
+  return true;
+}
+
 // Warp-aggregated increment of a shared-memory histogram: lanes that hit the same bin
 // elect one lane that adds the whole group's count.  Must be called by all 32 lanes.
 __device__ __forceinline__ void hist_add_aggregated(uint32_t* hist, bool valid, uint32_t bin) {
@@ -161,8 +213,8 @@ __device__ __forceinline__ void hist_add_aggregated(uint32_t* hist, bool valid, 
 }
 
 // ---------------------------------------------------------------------------------------
-// tiled path, step (a): residual accumulation  acc += grads, and update <- 0
-// grid = tiles; each CTA walks the W workers of one tile.
+// tiled path, step (a) alone: residual accumulation  acc += grads, and update <- 0.
+// Used when speculation is off.  grid = tiles; each CTA walks the W workers of one tile.
 // ---------------------------------------------------------------------------------------
 template <bool VEC>
 __global__ void __launch_bounds__(THREADS) k_accumulate(const float* __restrict__ grads, float* __restrict__ acc,
@@ -197,40 +249,215 @@ __global__ void __launch_bounds__(THREADS) k_accumulate(const float* __restrict_
 }
 
 // ---------------------------------------------------------------------------------------
-// tiled path, step (c): exact radix select of the k-th largest key per (worker, layer)
+// single-read path, threshold guess: one CTA per (tiled layer, worker) pair evaluates the
+// importance the step WILL produce (acc + grad) on a strided, jittered sample of the layer and
+// takes the rho-th largest as the guess.  Only a guess: the select stays exact whatever it is.
+// grid = pairs; dynamic shared memory = 4 * max sample bytes.
 // ---------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t hash32(uint32_t x) {
+  x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
+  return x;
+}
 
-// One histogram pass over a chunk of the residual: keys that match the prefix found so far
-// are counted by their next digit.  grid = (chunks, W).
+__global__ void __launch_bounds__(THREADS)
+    k_sample(const float* __restrict__ grads, const float* __restrict__ weights, const float* __restrict__ acc,
+             const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ large_ids, PairInfo* __restrict__ info,
+             float eps, uint64_t N, int W, uint32_t step) {
+  extern __shared__ uint32_t keys[];
+  __shared__ uint32_t hist[NBINS];
+  __shared__ uint32_t sh_scan[THREADS];
+  __shared__ uint32_t res[4];
+  const uint32_t pair = blockIdx.x;
+  const LayerDesc L = layers[large_ids[pair / W]];
+  const int w = pair % W;
+  const uint32_t s = L.sample;
+  if (s == 0) {
+    if (threadIdx.x == 0) info[pair] = PairInfo{GUESS_NONE, 0u, 0u, 0u};
+    return;
+  }
+  const uint32_t groups = s >> 3;
+  const uint32_t stride = L.n / groups;  // >= 32 because s <= n / 4
+  const float* a = acc + static_cast<uint64_t>(w) * N + L.off;
+  const float* g = grads + static_cast<uint64_t>(w) * N + L.off;
+  const float* wt = weights + L.off;
+  for (uint32_t i = threadIdx.x; i < s; i += THREADS) {
+    const uint32_t grp = i >> 3;
+    const uint32_t jit = hash32(step * 0x9E3779B9u + pair * 0x85EBCA6Bu + grp * 0xC2B2AE35u + 1u) % (stride - 7u);
+    const uint32_t pos = grp * stride + jit + (i & 7u);
+    keys[i] = imp_key(__fadd_rn(a[pos], g[pos]), wt[pos], eps);
+  }
+  __syncthreads();
+  uint32_t T, r;
+  const bool ok = smem_radix_select(keys, s, L.rho, hist, sh_scan, res, T, r);
+  if (threadIdx.x == 0) info[pair] = PairInfo{(ok && T != 0u) ? T : GUESS_NONE, 0u, 0u, 0u};
+}
+
+// ---------------------------------------------------------------------------------------
+// single-read path, steps (a)+(b) fused with candidate emission: acc += grads, update <- 0,
+// importance of every element, and every element whose importance reaches the pair's guess is
+// appended, in index order, to the (tile, worker) candidate slot.  grid = tiles.
+//
+// Thread layout: warp q owns 512 consecutive elements of the tile window; in round s its lanes
+// read one 128-bit slot each of the 128 elements [q*512 + s*128, +128).  Index order is therefore
+// (warp, round, lane, component), which the ranking below follows.
+// ---------------------------------------------------------------------------------------
 template <bool VEC>
 __global__ void __launch_bounds__(THREADS)
-    k_hist_dense(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
-                 const LayerDesc* __restrict__ layers, const uint2* __restrict__ state, uint32_t* __restrict__ hist,
-                 float eps, uint64_t N, int W, int pass) {
+    k_accumulate_emit(const float* __restrict__ grads, const float* __restrict__ weights, float* __restrict__ acc,
+                      float* __restrict__ update, const Tile* __restrict__ tiles, PairInfo* __restrict__ info,
+                      uint32_t* __restrict__ cand_key, float* __restrict__ cand_val, uint16_t* __restrict__ cand_idx,
+                      uint32_t* __restrict__ cand_cnt, float eps, uint64_t N, int W) {
+  __shared__ uint32_t sh_wtot[2][WARPS];
+  constexpr int SPT = TILE / 4 / THREADS;  // rounds (slots per thread) = 4
+  const Tile t = tiles[blockIdx.x];
+  const uint64_t lo = t.a, hi = lo + t.len;
+  const uint64_t base = lo & ~static_cast<uint64_t>(TILE - 1);
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t loc[SPT];  // offset of the slot inside the tile window
+  uint64_t e0[SPT];
+  float den[SPT][4];
+  uint32_t inrange = 0;  // bit (4 s + c): element is inside [lo, hi)
+  const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int s = 0; s < SPT; ++s) {
+    loc[s] = static_cast<uint32_t>(warp * (SPT * 32) + s * 32 + lane) * 4u;
+    e0[s] = base + loc[s];
+    float wv[4];
+    load4<VEC>(weights, e0[s], lo, hi, wv);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      den[s][c] = imp_den(wv[c], eps);
+      const uint64_t e = e0[s] + c;
+      inrange |= (e >= lo && e < hi) ? (1u << (4 * s + c)) : 0u;
+    }
+    store4<VEC>(update, e0[s], lo, hi, zero);
+  }
+  for (int w = 0; w < W; ++w) {
+    const uint32_t pair = t.large_index * W + w;
+    const uint32_t guess = info[pair].guess;
+    const float* g = grads + static_cast<uint64_t>(w) * N;
+    float* a = acc + static_cast<uint64_t>(w) * N;
+    float gv[SPT][4], av[SPT][4];
+#pragma unroll
+    for (int s = 0; s < SPT; ++s) {
+      load4_stream<VEC>(g, e0[s], lo, hi, gv[s]);
+      load4<VEC>(a, e0[s], lo, hi, av[s]);
+    }
+    uint32_t m = 0;  // bit (4 s + c): candidate
+#pragma unroll
+    for (int s = 0; s < SPT; ++s) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        av[s][c] = __fadd_rn(av[s][c], gv[s][c]);
+        m |= (imp_key_den(av[s][c], den[s][c]) >= guess) ? (1u << (4 * s + c)) : 0u;
+      }
+      store4<VEC>(a, e0[s], lo, hi, av[s]);
+    }
+    m &= inrange;
+    // rank inside the warp: per-round counts packed 8 bits each (a warp has at most 128 per round)
+    uint32_t packed = 0;
+#pragma unroll
+    for (int s = 0; s < SPT; ++s) packed |= static_cast<uint32_t>(__popc((m >> (4 * s)) & 0xFu)) << (8 * s);
+    const uint32_t incl = warp_incl_scan(packed);
+    const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
+    const uint32_t excl = incl - packed;
+    uint32_t round_base[SPT];
+    uint32_t warp_total = 0;
+#pragma unroll
+    for (int s = 0; s < SPT; ++s) {
+      round_base[s] = warp_total + ((excl >> (8 * s)) & 0xFFu);
+      warp_total += (tot >> (8 * s)) & 0xFFu;
+    }
+    uint32_t* wt = sh_wtot[w & 1];
+    if (lane == 0) wt[warp] = warp_total;
+    __syncthreads();
+    uint32_t warp_base = 0, block_total = 0;
+#pragma unroll
+    for (int q = 0; q < WARPS; ++q) {
+      const uint32_t v = wt[q];
+      if (q < warp) warp_base += v;
+      block_total += v;
+    }
+    const uint64_t slot = (static_cast<uint64_t>(blockIdx.x) * W + w) * CAND_CAP;
+    if (m) {
+#pragma unroll
+      for (int s = 0; s < SPT; ++s) {
+        uint32_t pos = warp_base + round_base[s];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if ((m >> (4 * s + c)) & 1u) {
+            if (pos < CAND_CAP) {
+              cand_key[slot + pos] = imp_key_den(av[s][c], den[s][c]);
+              cand_val[slot + pos] = av[s][c];
+              cand_idx[slot + pos] = static_cast<uint16_t>(loc[s] + c);
+            }
+            ++pos;
+          }
+        }
+      }
+    }
+    if (threadIdx.x == 0) {
+      cand_cnt[static_cast<uint64_t>(blockIdx.x) * W + w] = block_total;
+      if (block_total) atomicAdd(&info[pair].total, block_total);
+      if (block_total > CAND_CAP) atomicOr(&info[pair].flags, 1u);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// tiled path, step (c): exact radix select of the k-th largest key per (worker, layer).
+// Every kernel below serves both kinds of pair: those whose candidates hold the top-k read the
+// candidate slots, the others read the residual and the weights again (multi-pass exact path).
+// ---------------------------------------------------------------------------------------
+
+// One histogram pass over a chunk: keys that match the prefix found so far are counted by
+// their next digit.  grid = (chunks, W).
+template <bool VEC>
+__global__ void __launch_bounds__(THREADS)
+    k_hist(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
+           const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
+           const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt, const uint2* __restrict__ state,
+           uint32_t* __restrict__ hist, float eps, uint64_t N, int W, int pass) {
   __shared__ uint32_t sh[NBINS];
   const Chunk c = chunks[blockIdx.x];
   const int w = blockIdx.y;
-  const uint32_t pair = static_cast<uint32_t>(layers[c.layer].large_index) * W + w;
+  const LayerDesc L = layers[c.layer];
+  const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
   const int shift = pass_shift(pass), nb = pass_bins(pass);
   const int prev_shift = pass == 0 ? 31 : pass_shift(pass - 1);
   const uint32_t want = pass == 0 ? 0u : (state[pair].x >> prev_shift);
   for (int b = threadIdx.x; b < nb; b += THREADS) sh[b] = 0;
   __syncthreads();
-  const uint64_t lo = c.a, hi = lo + c.len;
-  const uint64_t s0 = lo & ~3ull;
-  const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
-  const float* a = acc + static_cast<uint64_t>(w) * N;
-  for (uint32_t it = 0; it < n_iter; ++it) {
-    const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
-    float av[4], wv[4];
-    load4<VEC>(a, e0, lo, hi, av);
-    load4<VEC>(weights, e0, lo, hi, wv);
+  if (pair_is_cand(info[pair], L.k)) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (uint32_t ti = warp; ti < c.n_tiles; ti += WARPS) {
+      const uint64_t tw = static_cast<uint64_t>(c.first_tile + ti) * W + w;
+      const uint32_t cnt = min(cand_cnt[tw], CAND_CAP);
+      const uint32_t* kp = cand_key + tw * CAND_CAP;
+      for (uint32_t j0 = 0; j0 < cnt; j0 += 32) {
+        const uint32_t j = j0 + lane;
+        const uint32_t key = j < cnt ? kp[j] : 0u;
+        const bool valid = j < cnt && (key >> prev_shift) == want;
+        hist_add_aggregated(sh, valid, (key >> shift) & (nb - 1));
+      }
+    }
+  } else {
+    const uint64_t lo = c.a, hi = lo + c.len;
+    const uint64_t s0 = lo & ~3ull;
+    const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+    const float* a = acc + static_cast<uint64_t>(w) * N;
+    for (uint32_t it = 0; it < n_iter; ++it) {
+      const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+      float av[4], wv[4];
+      load4<VEC>(a, e0, lo, hi, av);
+      load4<VEC>(weights, e0, lo, hi, wv);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const uint64_t e = e0 + q;
-      const uint32_t key = imp_key(av[q], wv[q], eps);
-      const bool valid = e >= lo && e < hi && (key >> prev_shift) == want;  // pass 0: bit 31 is 0 == want
-      hist_add_aggregated(sh, valid, (key >> shift) & (nb - 1));
+      for (int q = 0; q < 4; ++q) {
+        const uint64_t e = e0 + q;
+        const uint32_t key = imp_key(av[q], wv[q], eps);
+        const bool valid = e >= lo && e < hi && (key >> prev_shift) == want;  // pass 0: bit 31 is 0 == want
+        hist_add_aggregated(sh, valid, (key >> shift) & (nb - 1));
+      }
     }
   }
   __syncthreads();
@@ -281,33 +508,49 @@ __global__ void __launch_bounds__(THREADS)
 // Per chunk: how many keys are above the threshold and how many equal it.  grid = (chunks, W).
 template <bool VEC>
 __global__ void __launch_bounds__(THREADS)
-    k_count_dense(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
-                  const LayerDesc* __restrict__ layers, const uint2* __restrict__ state, uint2* __restrict__ chunk_cnt,
-                  float eps, uint64_t N, int W, uint32_t n_chunks) {
+    k_count(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
+            const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
+            const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt, const uint2* __restrict__ state,
+            uint2* __restrict__ chunk_cnt, float eps, uint64_t N, int W, uint32_t n_chunks) {
   __shared__ uint32_t sh_cnt[2];
   const Chunk c = chunks[blockIdx.x];
   const int w = blockIdx.y;
-  const uint32_t pair = static_cast<uint32_t>(layers[c.layer].large_index) * W + w;
+  const LayerDesc L = layers[c.layer];
+  const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
   const uint32_t T = state[pair].x;
   if (threadIdx.x < 2) sh_cnt[threadIdx.x] = 0;
   __syncthreads();
-  const uint64_t lo = c.a, hi = lo + c.len;
-  const uint64_t s0 = lo & ~3ull;
-  const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
-  const float* a = acc + static_cast<uint64_t>(w) * N;
   uint32_t gt = 0, eq = 0;
-  for (uint32_t it = 0; it < n_iter; ++it) {
-    const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
-    float av[4], wv[4];
-    load4<VEC>(a, e0, lo, hi, av);
-    load4<VEC>(weights, e0, lo, hi, wv);
+  if (pair_is_cand(info[pair], L.k)) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (uint32_t ti = warp; ti < c.n_tiles; ti += WARPS) {
+      const uint64_t tw = static_cast<uint64_t>(c.first_tile + ti) * W + w;
+      const uint32_t cnt = min(cand_cnt[tw], CAND_CAP);
+      const uint32_t* kp = cand_key + tw * CAND_CAP;
+      for (uint32_t j = lane; j < cnt; j += 32) {
+        const uint32_t key = kp[j];
+        gt += key > T ? 1u : 0u;
+        eq += key == T ? 1u : 0u;
+      }
+    }
+  } else {
+    const uint64_t lo = c.a, hi = lo + c.len;
+    const uint64_t s0 = lo & ~3ull;
+    const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+    const float* a = acc + static_cast<uint64_t>(w) * N;
+    for (uint32_t it = 0; it < n_iter; ++it) {
+      const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+      float av[4], wv[4];
+      load4<VEC>(a, e0, lo, hi, av);
+      load4<VEC>(weights, e0, lo, hi, wv);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const uint64_t e = e0 + q;
-      const bool in = e >= lo && e < hi;
-      const uint32_t key = imp_key(av[q], wv[q], eps);
-      gt += (in && key > T) ? 1u : 0u;
-      eq += (in && key == T) ? 1u : 0u;
+      for (int q = 0; q < 4; ++q) {
+        const uint64_t e = e0 + q;
+        const bool in = e >= lo && e < hi;
+        const uint32_t key = imp_key(av[q], wv[q], eps);
+        gt += (in && key > T) ? 1u : 0u;
+        eq += (in && key == T) ? 1u : 0u;
+      }
     }
   }
 #pragma unroll
@@ -329,12 +572,16 @@ __global__ void __launch_bounds__(THREADS)
 // grid = (chunks, W).
 template <bool VEC>
 __global__ void __launch_bounds__(THREADS)
-    k_write_dense(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
-                  const LayerDesc* __restrict__ layers, const uint2* __restrict__ state,
-                  const uint2* __restrict__ chunk_cnt, uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val,
-                  int* __restrict__ status, float eps, uint64_t N, uint64_t K, int W, uint32_t n_chunks) {
+    k_write(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
+            const Tile* __restrict__ tiles, const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
+            const uint32_t* __restrict__ cand_key, const float* __restrict__ cand_val,
+            const uint16_t* __restrict__ cand_idx, const uint32_t* __restrict__ cand_cnt,
+            const uint2* __restrict__ state, const uint2* __restrict__ chunk_cnt, uint32_t* __restrict__ sel_idx,
+            float* __restrict__ sel_val, int* __restrict__ status, float eps, uint64_t N, uint64_t K, int W,
+            uint32_t n_chunks) {
   __shared__ uint32_t sh_warp[WARPS];
   __shared__ uint32_t sh_base[2];
+  __shared__ uint32_t sh_pre[CHUNK_TILES + 1];
   const Chunk c = chunks[blockIdx.x];
   const int w = blockIdx.y;
   const LayerDesc L = layers[c.layer];
@@ -364,12 +611,58 @@ __global__ void __launch_bounds__(THREADS)
   }
   __syncthreads();
   uint32_t run_gt = sh_base[0], run_eq = sh_base[1];
+  uint32_t* out_i = sel_idx + static_cast<uint64_t>(w) * K + L.koff;
+  float* out_v = sel_val + static_cast<uint64_t>(w) * K + L.koff;
+
+  if (pair_is_cand(info[pair], L.k)) {
+    // the chunk's candidates, tile after tile, form one index-ordered sequence
+    uint32_t total;
+    {
+      static_assert(CHUNK_TILES <= THREADS, "one thread per tile count");
+      const uint32_t ti = threadIdx.x;
+      const uint32_t cnt = ti < c.n_tiles ? min(cand_cnt[static_cast<uint64_t>(c.first_tile + ti) * W + w], CAND_CAP) : 0u;
+      const uint32_t ex = block_excl_scan(cnt, sh_warp, total);
+      if (ti <= c.n_tiles && ti <= CHUNK_TILES) sh_pre[ti] = ex;  // sh_pre[n_tiles] = total
+      __syncthreads();
+    }
+    for (uint32_t j0 = 0; j0 < total; j0 += THREADS) {
+      const uint32_t j = j0 + threadIdx.x;
+      const bool valid = j < total;
+      uint32_t key = 0, tile = 0;
+      uint64_t slot = 0;
+      if (valid) {
+        uint32_t a = 0, b = c.n_tiles;  // largest tile index with sh_pre[tile] <= j
+        while (b - a > 1) {
+          const uint32_t mid = (a + b) >> 1;
+          if (sh_pre[mid] <= j) a = mid; else b = mid;
+        }
+        tile = c.first_tile + a;
+        slot = (static_cast<uint64_t>(tile) * W + w) * CAND_CAP + (j - sh_pre[a]);
+        key = cand_key[slot];
+      }
+      const bool isg = valid && key > T, ise = valid && key == T;
+      uint32_t tot;
+      const uint32_t ex = block_excl_scan((isg ? 1u : 0u) | (ise ? 1u << 16 : 0u), sh_warp, tot);
+      const uint32_t g_before = run_gt + (ex & 0xffffu), q_before = run_eq + (ex >> 16);
+      if (isg || (ise && q_before < r)) {
+        const uint32_t pos = g_before + (q_before < r ? q_before : r);
+        if (pos < L.k) {
+          out_i[pos] = (tiles[tile].a & ~(TILE - 1u)) + cand_idx[slot];
+          out_v[pos] = cand_val[slot];
+        } else {
+          atomicMin(status, STATUS_INTERNAL);
+        }
+      }
+      run_gt += tot & 0xffffu;
+      run_eq += tot >> 16;
+    }
+    return;
+  }
+
   const uint64_t lo = c.a, hi = lo + c.len;
   const uint64_t s0 = lo & ~3ull;
   const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
   const float* a = acc + static_cast<uint64_t>(w) * N;
-  uint32_t* out_i = sel_idx + static_cast<uint64_t>(w) * K + L.koff;
-  float* out_v = sel_val + static_cast<uint64_t>(w) * K + L.koff;
   for (uint32_t it = 0; it < n_iter; ++it) {
     const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
     float av[4], wv[4];
@@ -438,29 +731,11 @@ __global__ void __launch_bounds__(THREADS)
     if (w == 0) update[L.off + i] = 0.0f;
   }
   __syncthreads();
-  uint32_t prefix = 0, krem = L.k;
-#pragma unroll 1
-  for (int pass = 0; pass < N_PASSES; ++pass) {
-    const int shift = pass_shift(pass), nb = pass_bins(pass);
-    const int prev_shift = pass == 0 ? 31 : pass_shift(pass - 1);
-    const uint32_t want = prefix >> prev_shift;
-    for (int b = tid; b < nb; b += THREADS) hist[b] = 0;
-    __syncthreads();
-    for (uint32_t i = tid; i < n; i += THREADS) {
-      const uint32_t key = keys[i];
-      if ((key >> prev_shift) == want) atomicAdd(&hist[(key >> shift) & (nb - 1)], 1u);
-    }
-    __syncthreads();
-    find_digit(hist, nb, krem, sh_scan, res);
-    if (!res[2]) {
-      if (tid == 0) atomicMin(status, STATUS_INTERNAL);
-      return;
-    }
-    prefix |= res[0] << shift;
-    krem = res[1];
-    __syncthreads();
+  uint32_t T, r;
+  if (!smem_radix_select(keys, n, L.k, hist, sh_scan, res, T, r)) {
+    if (tid == 0) atomicMin(status, STATUS_INTERNAL);
+    return;
   }
-  const uint32_t T = prefix, r = krem;
   uint32_t* out_i = sel_idx + static_cast<uint64_t>(w) * K + L.koff;
   float* out_v = sel_val + static_cast<uint64_t>(w) * K + L.koff;
   uint32_t run_gt = 0, run_eq = 0;

@@ -15,9 +15,13 @@
 namespace iwp {
 
 constexpr uint32_t TILE = 4096;
-constexpr uint32_t CHUNK_TILES = 16;
+constexpr uint32_t CHUNK_TILES = 128;
 constexpr uint32_t SMALL_MAX = 16384;
 constexpr uint32_t NBINS = 2048;
+// single-read path: capacity of a (tile, worker) candidate slot and the sample that sets the guess
+constexpr uint32_t CAND_CAP = 512;
+constexpr uint32_t SAMPLE_MAX = 16384;
+constexpr uint32_t GUESS_NONE = 0xffffffffu;  // no importance pattern reaches this value
 
 struct LayerDesc {
   uint32_t off;         // flat offset of the first element
@@ -29,6 +33,8 @@ struct LayerDesc {
   uint32_t n_tiles;
   uint32_t first_chunk;
   uint32_t n_chunks;
+  uint32_t sample;  // elements sampled for the threshold guess (multiple of 8), 0 = no speculation
+  uint32_t rho;     // the guess is the rho-th largest sampled importance
 };
 
 struct Tile {
@@ -54,6 +60,26 @@ inline int64_t keep_count(int64_t n, double ratio) {
   if (k < 1) k = 1;
   if (k > n) k = n;
   return k;
+}
+
+// Sample size s and rank rho for the threshold guess of a tiled layer.  With p = k/n the number of
+// sampled elements above the true threshold is ~Binomial(s, p); taking the rho-th largest sample with
+// rho = s p + 4.5 sqrt(s p (1-p)) + 2 puts the guess below the true threshold except with probability
+// ~1e-5 (then the exact multi-pass select takes over for that pair).  Speculation is switched off when
+// the expected candidate density rho/s would fill more than a third of a candidate slot.
+inline void sample_plan(uint32_t n, uint32_t k, uint32_t* sample, uint32_t* rho) {
+  *sample = 0;
+  *rho = 0;
+  if (k >= n) return;
+  uint32_t s = (n / 4) & ~7u;
+  if (s > SAMPLE_MAX) s = SAMPLE_MAX;
+  if (s < 64) return;
+  const double p = static_cast<double>(k) / static_cast<double>(n);
+  const double mean = s * p;
+  const double r = std::ceil(mean + 4.5 * std::sqrt(mean * (1.0 - p)) + 2.0);
+  if (r * 24.0 > static_cast<double>(s)) return;
+  *sample = s;
+  *rho = static_cast<uint32_t>(r);
 }
 
 inline uint64_t mix64(uint64_t z) {
@@ -135,6 +161,7 @@ inline Plan make_plan(const int64_t* sizes, int32_t n_layers, int32_t W, double 
         p.chunks.push_back(c);
       }
       d.n_chunks = static_cast<uint32_t>(p.chunks.size()) - d.first_chunk;
+      sample_plan(d.n, d.k, &d.sample, &d.rho);
     }
     p.layers.push_back(d);
     off += d.n;

@@ -123,3 +123,29 @@ def test_options_stats_and_misuse():
     assert pr.layout() == ([0, 5000], [625, 2500])
     pr.close()
     pr.close()  # idempotent
+
+
+def test_single_read_path_is_taken_and_falls_back_when_it_must():
+    sizes, W = [300000, 64, 40000], 4
+    N = sum(sizes)
+    weights, grads = _inputs(W, N, 8)
+    pr = Pruner(sizes, W, 64.0, 1e-8, 0)
+    orc = oracle.Oracle(sizes, W, 64.0, 1e-8, 0)
+    assert pr.stat("spec_pairs") == 2 * W
+    for g in grads:
+        upd = pr.step(g, weights)
+        want = orc.step(g.cpu().numpy(), weights.cpu().numpy())
+        assert pr.stat("spec_failed") == 0  # continuous random values: every pair stays on the single-read path
+        assert_bits_equal(upd.cpu().numpy(), want, "update")
+    # all importances equal: every element reaches the guess, the slots overflow, the exact path takes over
+    pr.reset()
+    orc.reset()
+    g = torch.full((W, N), 0.5, device=DEV)
+    wt = torch.ones(N, device=DEV)
+    upd = pr.step(g, wt)
+    want = orc.step(g.cpu().numpy(), wt.cpu().numpy())
+    assert pr.stat("spec_failed") == 2 * W and pr.sync_status() == 0
+    assert_bits_equal(upd.cpu().numpy(), want, "update after fallback")
+    pr.set_option("speculate", 0)
+    assert pr.stat("spec_pairs") == 0
+    pr.close()
