@@ -97,10 +97,14 @@ class ClockSampler:
         return out
 
 
-def make_workload(name):
+def make_workload(name, layers=None):
     from paper_1901_01544_b200 import workloads as wl
 
-    return wl.CONFIGS[name]()
+    c = wl.CONFIGS[name]()
+    if layers:
+        lo, hi = (int(x) for x in layers.split(":"))
+        c = wl.subset(c, lo, hi)
+    return c
 
 
 # ---------------------------------------------------------------------------------- CPU oracle legs
@@ -129,7 +133,7 @@ def run_reference(args):
         return
     import torch
 
-    c = make_workload(args.config)
+    c = make_workload(args.config, args.layers)
     weights = c.weights("cpu").numpy()
     n_sets = 2
     sets = [c.grads(t, "cpu").numpy() for t in range(n_sets)]
@@ -175,11 +179,13 @@ def run_ours(args):
     from paper_1901_01544_b200.binding import Pruner
 
     dev = torch.device("cuda", local)
-    c = make_workload(args.config)
+    c = make_workload(args.config, args.layers)
     W, N = c.W, c.N
     weights = c.weights(dev)
     grad_bytes = 4 * W * N
     n_sets = max(2, min(5, int(24e9 // grad_bytes)))  # distinct gradient batches cycled through
+    if args.grad_sets:
+        n_sets = args.grad_sets
     sets = [c.grads(t, dev) for t in range(n_sets)]
     update = torch.empty(N, dtype=torch.float32, device=dev)
     pr = Pruner(c.layer_sizes, W, c.ratio, c.eps, c.seed)
@@ -226,22 +232,25 @@ def run_ours(args):
 
     # end to end through the host-buffer entry point: H2D of grads + weights and D2H of the update inside
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    gh = [sets[i].cpu().pin_memory() for i in range(min(2, n_sets))]
-    wh = weights.cpu().pin_memory()
-    uh = torch.empty(N, dtype=torch.float32).pin_memory()
-    pr.step_host(gh[0], wh, uh)  # allocates the staging buffers
-    barrier()
-    t0 = time.perf_counter()
-    for t in range(e2e_steps):
-        pr.step_host(gh[t % len(gh)], wh, uh)
-    torch.cuda.synchronize()
-    e2e_dt = time.perf_counter() - t0
-    if dist is not None:
-        tt = torch.tensor([e2e_dt], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_dt = float(tt.item())
-    pr.check()
-    e2e_value = world * e2e_steps / e2e_dt
+    e2e_value = None
+    gh = wh = None
+    if not args.no_e2e:
+        gh = [sets[i].cpu().pin_memory() for i in range(min(2, n_sets))]
+        wh = weights.cpu().pin_memory()
+        uh = torch.empty(N, dtype=torch.float32).pin_memory()
+        pr.step_host(gh[0], wh, uh)  # allocates the staging buffers
+        barrier()
+        t0 = time.perf_counter()
+        for t in range(e2e_steps):
+            pr.step_host(gh[t % len(gh)], wh, uh)
+        torch.cuda.synchronize()
+        e2e_dt = time.perf_counter() - t0
+        if dist is not None:
+            tt = torch.tensor([e2e_dt], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_dt = float(tt.item())
+        pr.check()
+        e2e_value = world * e2e_steps / e2e_dt
 
     if rank != 0:
         if dist is not None:
@@ -271,8 +280,8 @@ def run_ours(args):
     # CPU baseline: the oracle as it stands, a bounded sample (a few full steps) on this machine's cores
     cpu = None
     if not args.no_cpu_baseline:
-        w_host = wh.numpy()
-        g_host = [g.numpy() for g in gh]
+        w_host = weights.cpu().numpy()
+        g_host = [sets[i].cpu().numpy() for i in range(min(2, n_sets))]
         sps, threads, dt = oracle_timing(c, w_host, lambda t: g_host[t % len(g_host)], args.cpu_steps, 1)
         cpu = {"value": sps, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": f"{args.cpu_steps} full steps of {c.name} after 1 warm-up step ({dt:.1f} s of CPU work)"}
@@ -313,6 +322,9 @@ def main():
     ap.add_argument("--cpu-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--speculate", type=int, default=None, choices=[0, 1])
+    ap.add_argument("--layers", default=None, help="lo:hi - only these layers of the workload (small profiling case)")
+    ap.add_argument("--grad-sets", type=int, default=None, help="distinct gradient batches kept on the device")
+    ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -202,9 +202,10 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   if (tiled) {
     const unsigned n_tiles = static_cast<unsigned>(p.tiles.size());
     if (spec) {
-      k_accumulate_emit<VEC><<<n_tiles, THREADS, 0, s>>>(grads, weights, c->acc, update, c->d_tiles, c->d_info,
-                                                         c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->eps, N,
-                                                         W);
+      const int groups = (W + WARPS - 1) / WARPS;
+      k_accumulate_emit<VEC><<<n_tiles * static_cast<unsigned>(groups), THREADS, 0, s>>>(
+          grads, weights, c->acc, update, c->d_tiles, c->d_info, c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt,
+          c->eps, N, W, groups);
     } else {
       k_accumulate<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, N, W);
     }

@@ -295,112 +295,152 @@ __global__ void __launch_bounds__(THREADS)
 // ---------------------------------------------------------------------------------------
 // single-read path, steps (a)+(b) fused with candidate emission: acc += grads, update <- 0,
 // importance of every element, and every element whose importance reaches the pair's guess is
-// appended, in index order, to the (tile, worker) candidate slot.  grid = tiles.
+// appended, in index order, to the (tile, worker) candidate slot.
 //
-// Thread layout: warp q owns 512 consecutive elements of the tile window; in round s its lanes
-// read one 128-bit slot each of the 128 elements [q*512 + s*128, +128).  Index order is therefore
-// (warp, round, lane, component), which the ranking below follows.
+// One WARP owns one (tile, worker) pair and walks the tile front to back, 512 elements per
+// iteration (four rounds of 32 lanes x one 128-bit slot), so the index order of the candidates
+// is (iteration, round, lane, component) and a running count in a register is all the state:
+// no shared memory, no block barrier, warps never wait for each other.  The eight warps of a
+// CTA take eight workers of the same tile, so the tile's weights are fetched from HBM once and
+// re-read through L1.  grid = tiles * ceil(W / 8).
 // ---------------------------------------------------------------------------------------
+// Conservative multiplier for the cheap candidate pre-test |acc| >= gm * den: with
+// gm = guess * (1 - 2^-20) every element whose correctly rounded quotient |acc| / den reaches the
+// guess passes it (the two roundings of gm * den and the one of the quotient are each below 2^-23
+// relative); the exact quotient is then formed only for the few elements that pass.  The argument
+// needs normal products, so the pre-test is disabled (gm = 0: everything passes) for tiny guesses
+// or a tiny eps.
+__device__ __forceinline__ float pretest_multiplier(uint32_t guess, float eps) {
+  if (guess == GUESS_NONE) return __int_as_float(0x7f800000);  // +inf: nothing passes
+  const float gf = __uint_as_float(guess);
+  const float tiny = 8.673617379884035e-19f;  // 2^-60
+  if (!(gf >= tiny) || !(eps >= tiny)) return 0.0f;
+  return __fmul_rd(gf, 1.0f - 9.5367431640625e-07f);
+}
+
 template <bool VEC>
 __global__ void __launch_bounds__(THREADS)
     k_accumulate_emit(const float* __restrict__ grads, const float* __restrict__ weights, float* __restrict__ acc,
                       float* __restrict__ update, const Tile* __restrict__ tiles, PairInfo* __restrict__ info,
                       uint32_t* __restrict__ cand_key, float* __restrict__ cand_val, uint16_t* __restrict__ cand_idx,
-                      uint32_t* __restrict__ cand_cnt, float eps, uint64_t N, int W) {
-  __shared__ uint32_t sh_wtot[2][WARPS];
-  constexpr int SPT = TILE / 4 / THREADS;  // rounds (slots per thread) = 4
-  const Tile t = tiles[blockIdx.x];
+                      uint32_t* __restrict__ cand_cnt, float eps, uint64_t N, int W, int worker_groups) {
+  constexpr int ROUNDS = 4;                 // 128-bit slots per lane and iteration
+  constexpr int ITER_ELEMS = ROUNDS * 128;  // 512
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t tile_id = blockIdx.x / worker_groups;
+  const int w = static_cast<int>(blockIdx.x % worker_groups) * WARPS + warp;
+  if (w >= W) return;
+  const Tile t = tiles[tile_id];
   const uint64_t lo = t.a, hi = lo + t.len;
   const uint64_t base = lo & ~static_cast<uint64_t>(TILE - 1);
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  uint32_t loc[SPT];  // offset of the slot inside the tile window
-  uint64_t e0[SPT];
-  float den[SPT][4];
-  uint32_t inrange = 0;  // bit (4 s + c): element is inside [lo, hi)
+  const bool full = VEC && t.len == TILE;  // every slot of the window is inside the tile
+  const uint32_t pair = t.large_index * W + w;
+  const uint32_t guess = info[pair].guess;
+  const float gm = pretest_multiplier(guess, eps);
+  const float* g = grads + static_cast<uint64_t>(w) * N;
+  float* a = acc + static_cast<uint64_t>(w) * N;
+  const uint64_t slot = (static_cast<uint64_t>(tile_id) * W + w) * CAND_CAP;
   const float zero[4] = {0.f, 0.f, 0.f, 0.f};
+  uint32_t count = 0;  // candidates of this (tile, worker) so far; the same in every lane
+#pragma unroll 1
+  for (uint32_t it = 0; it < TILE / ITER_ELEMS; ++it) {
+    const uint64_t seg = base + it * ITER_ELEMS;
+    if (seg + ITER_ELEMS <= lo || seg >= hi) continue;  // warp-uniform
+    const uint64_t first = seg + static_cast<uint64_t>(lane) * 4;  // this lane's slot in round 0
+    float gv[ROUNDS][4], av[ROUNDS][4], den[ROUNDS][4];
+    uint32_t inrange = 0xFFFFu;
+    if (full) {
+      const float4* g4 = reinterpret_cast<const float4*>(g + first);
+      const float4* a4 = reinterpret_cast<const float4*>(a + first);
+      const float4* w4 = reinterpret_cast<const float4*>(weights + first);
 #pragma unroll
-  for (int s = 0; s < SPT; ++s) {
-    loc[s] = static_cast<uint32_t>(warp * (SPT * 32) + s * 32 + lane) * 4u;
-    e0[s] = base + loc[s];
-    float wv[4];
-    load4<VEC>(weights, e0[s], lo, hi, wv);
+      for (int s = 0; s < ROUNDS; ++s) {
+        const float4 x = __ldcs(g4 + s * 32), y = a4[s * 32], z = w4[s * 32];
+        gv[s][0] = x.x; gv[s][1] = x.y; gv[s][2] = x.z; gv[s][3] = x.w;
+        av[s][0] = y.x; av[s][1] = y.y; av[s][2] = y.z; av[s][3] = y.w;
+        den[s][0] = z.x; den[s][1] = z.y; den[s][2] = z.z; den[s][3] = z.w;
+      }
+    } else {
+      inrange = 0;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-      den[s][c] = imp_den(wv[c], eps);
-      const uint64_t e = e0[s] + c;
-      inrange |= (e >= lo && e < hi) ? (1u << (4 * s + c)) : 0u;
+      for (int s = 0; s < ROUNDS; ++s) {
+        const uint64_t e0 = first + s * 128;
+        load4_stream<VEC>(g, e0, lo, hi, gv[s]);
+        load4<VEC>(a, e0, lo, hi, av[s]);
+        load4<VEC>(weights, e0, lo, hi, den[s]);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) inrange |= (e0 + c >= lo && e0 + c < hi) ? (1u << (4 * s + c)) : 0u;
+      }
     }
-    store4<VEC>(update, e0[s], lo, hi, zero);
-  }
-  for (int w = 0; w < W; ++w) {
-    const uint32_t pair = t.large_index * W + w;
-    const uint32_t guess = info[pair].guess;
-    const float* g = grads + static_cast<uint64_t>(w) * N;
-    float* a = acc + static_cast<uint64_t>(w) * N;
-    float gv[SPT][4], av[SPT][4];
+    uint32_t m = 0;  // bit (4 s + c): passes the pre-test
 #pragma unroll
-    for (int s = 0; s < SPT; ++s) {
-      load4_stream<VEC>(g, e0[s], lo, hi, gv[s]);
-      load4<VEC>(a, e0[s], lo, hi, av[s]);
-    }
-    uint32_t m = 0;  // bit (4 s + c): candidate
-#pragma unroll
-    for (int s = 0; s < SPT; ++s) {
+    for (int s = 0; s < ROUNDS; ++s) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         av[s][c] = __fadd_rn(av[s][c], gv[s][c]);
-        m |= (imp_key_den(av[s][c], den[s][c]) >= guess) ? (1u << (4 * s + c)) : 0u;
+        den[s][c] = imp_den(den[s][c], eps);
+        m |= (fabsf(av[s][c]) >= __fmul_rn(gm, den[s][c])) ? (1u << (4 * s + c)) : 0u;
       }
-      store4<VEC>(a, e0[s], lo, hi, av[s]);
+    }
+    if (full) {
+      float4* a4 = reinterpret_cast<float4*>(a + first);
+#pragma unroll
+      for (int s = 0; s < ROUNDS; ++s) a4[s * 32] = make_float4(av[s][0], av[s][1], av[s][2], av[s][3]);
+      if (w == 0) {
+        float4* u4 = reinterpret_cast<float4*>(update + first);
+#pragma unroll
+        for (int s = 0; s < ROUNDS; ++s) u4[s * 32] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    } else {
+#pragma unroll
+      for (int s = 0; s < ROUNDS; ++s) {
+        store4<VEC>(a, first + s * 128, lo, hi, av[s]);
+        if (w == 0) store4<VEC>(update, first + s * 128, lo, hi, zero);
+      }
     }
     m &= inrange;
-    // rank inside the warp: per-round counts packed 8 bits each (a warp has at most 128 per round)
-    uint32_t packed = 0;
+    if (__any_sync(0xffffffffu, m != 0u)) {
+      // exact test for the few that passed: Algorithm 1's |grad / w| compared with the guess
 #pragma unroll
-    for (int s = 0; s < SPT; ++s) packed |= static_cast<uint32_t>(__popc((m >> (4 * s)) & 0xFu)) << (8 * s);
-    const uint32_t incl = warp_incl_scan(packed);
-    const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
-    const uint32_t excl = incl - packed;
-    uint32_t round_base[SPT];
-    uint32_t warp_total = 0;
+      for (int s = 0; s < ROUNDS; ++s) {
 #pragma unroll
-    for (int s = 0; s < SPT; ++s) {
-      round_base[s] = warp_total + ((excl >> (8 * s)) & 0xFFu);
-      warp_total += (tot >> (8 * s)) & 0xFFu;
-    }
-    uint32_t* wt = sh_wtot[w & 1];
-    if (lane == 0) wt[warp] = warp_total;
-    __syncthreads();
-    uint32_t warp_base = 0, block_total = 0;
+        for (int c = 0; c < 4; ++c) {
+          const uint32_t bit = 1u << (4 * s + c);
+          if ((m & bit) && imp_key_den(av[s][c], den[s][c]) < guess) m &= ~bit;
+        }
+      }
+      // rank inside the iteration: per-round counts packed 8 bits each (at most 128 per round)
+      uint32_t packed = 0;
 #pragma unroll
-    for (int q = 0; q < WARPS; ++q) {
-      const uint32_t v = wt[q];
-      if (q < warp) warp_base += v;
-      block_total += v;
-    }
-    const uint64_t slot = (static_cast<uint64_t>(blockIdx.x) * W + w) * CAND_CAP;
-    if (m) {
+      for (int s = 0; s < ROUNDS; ++s) packed |= static_cast<uint32_t>(__popc((m >> (4 * s)) & 0xFu)) << (8 * s);
+      const uint32_t incl = warp_incl_scan(packed);
+      const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
+      const uint32_t excl = incl - packed;
+      const uint32_t loc0 = static_cast<uint32_t>(first - base);
+      uint32_t round_base = count;
 #pragma unroll
-      for (int s = 0; s < SPT; ++s) {
-        uint32_t pos = warp_base + round_base[s];
+      for (int s = 0; s < ROUNDS; ++s) {
+        uint32_t pos = round_base + ((excl >> (8 * s)) & 0xFFu);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
           if ((m >> (4 * s + c)) & 1u) {
             if (pos < CAND_CAP) {
               cand_key[slot + pos] = imp_key_den(av[s][c], den[s][c]);
               cand_val[slot + pos] = av[s][c];
-              cand_idx[slot + pos] = static_cast<uint16_t>(loc[s] + c);
+              cand_idx[slot + pos] = static_cast<uint16_t>(loc0 + s * 128 + c);
             }
             ++pos;
           }
         }
+        round_base += (tot >> (8 * s)) & 0xFFu;
       }
+      count = round_base;
     }
-    if (threadIdx.x == 0) {
-      cand_cnt[static_cast<uint64_t>(blockIdx.x) * W + w] = block_total;
-      if (block_total) atomicAdd(&info[pair].total, block_total);
-      if (block_total > CAND_CAP) atomicOr(&info[pair].flags, 1u);
-    }
+  }
+  if (lane == 0) {
+    cand_cnt[static_cast<uint64_t>(tile_id) * W + w] = count;
+    if (count) atomicAdd(&info[pair].total, count);
+    if (count > CAND_CAP) atomicOr(&info[pair].flags, 1u);
   }
 }
 

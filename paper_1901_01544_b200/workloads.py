@@ -324,6 +324,16 @@ def scaled(wl: Workload, layer_sizes: List[int], W: Optional[int] = None, steps:
     )
 
 
+def subset(wl: Workload, lo: int, hi: int, W: Optional[int] = None, name: Optional[str] = None) -> Workload:
+    """Layers lo..hi-1 of a workload with the same value recipe (a smaller case of the same kind,
+    e.g. for a profiler capture that must stay within a few GB)."""
+    ts = wl.tensors[lo:hi] if wl.tensors is not None else None
+    return Workload(
+        name or f"{wl.name}[{lo}:{hi}]", wl.layer_sizes[lo:hi], W or wl.W, wl.ratio, wl.eps, wl.steps, wl.seed,
+        wl.describe + f" (layers {lo}..{hi - 1} only)", wl._weights_fn, wl._grads_fn, ts,
+    )
+
+
 CONFIGS = {
     "single_layer": single_layer,
     "alexnet_w8": alexnet_w8,

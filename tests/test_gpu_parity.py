@@ -101,11 +101,23 @@ def test_many_ties(name):
     run_parity(sizes, W, ratio, 1e-8, seed=1, steps=4, weights=weights, grads_fn=grads)
 
 
-@pytest.mark.parametrize("kind", ["all_equal", "all_zero", "two_values", "zero_weights"])
+@pytest.mark.parametrize("kind", ["all_equal", "all_zero", "two_values", "zero_weights", "tiny_values", "tiny_eps",
+                                  "huge_values"])
 def test_degenerate_layers(kind):
     sizes, W, ratio = [100000, 5000, 37], 3, 32.0
     N = sum(sizes)
-    if kind == "all_equal":
+    eps = 1e-8
+    if kind == "tiny_values":  # importances far below 2^-60, some denormal
+        weights = _weights(N, 3, zero_frac=0.0, scale=1.0) + 0.5
+        grads = lambda t: _randn((W, N), 5 + t, 1e-38)
+    elif kind == "tiny_eps":  # denominators down to 1e-30
+        eps = 1e-30
+        weights = _weights(N, 3, zero_frac=0.3)
+        grads = lambda t: _randn((W, N), 6 + t, 1e-6)
+    elif kind == "huge_values":  # importances up to ~1e37: products in the candidate pre-test overflow
+        weights = _weights(N, 3, zero_frac=0.3)
+        grads = lambda t: _randn((W, N), 7 + t, 1e29)
+    elif kind == "all_equal":
         weights = torch.full((N,), -0.5, device=DEV)
         grads = lambda t: torch.full((W, N), 0.25, device=DEV)
     elif kind == "all_zero":
@@ -120,7 +132,7 @@ def test_degenerate_layers(kind):
     else:
         weights = torch.zeros(N, device=DEV)
         grads = lambda t: _randn((W, N), 77 + t, 1e-3)
-    run_parity(sizes, W, ratio, 1e-8, seed=2, steps=2, weights=weights, grads_fn=grads)
+    run_parity(sizes, W, ratio, eps, seed=2, steps=2, weights=weights, grads_fn=grads)
 
 
 def test_forced_scalar_path_and_leader_override():
