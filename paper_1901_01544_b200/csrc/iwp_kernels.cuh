@@ -28,9 +28,9 @@ constexpr int N_PASSES = 3;
 // Per (tiled layer, worker) pair: the threshold guess of the single-read path and what the
 // fused accumulate pass found with it.
 struct PairInfo {
-  uint32_t guess;  // candidates are the elements with importance pattern >= guess; GUESS_NONE = none
-  uint32_t total;  // number of such elements in the layer
-  uint32_t flags;  // bit 0: some (tile, worker) slot overflowed
+  uint32_t guess;  // candidates include every element with importance pattern >= guess; GUESS_NONE = none
+  uint32_t total;  // number of elements of the layer that reach the guess
+  uint32_t flags;  // bit 0: some (tile, worker) slot or staging queue overflowed
   uint32_t pad;
 };
 
@@ -318,6 +318,14 @@ __device__ __forceinline__ float pretest_multiplier(uint32_t guess, float eps) {
   return __fmul_rd(gf, 1.0f - 9.5367431640625e-07f);
 }
 
+// Elements that pass the pre-test are staged, in index order, in a per-warp queue in shared
+// memory; the lanes then take one queue entry each, form the exact quotient (one division per
+// lane instead of one per element), count how many really reach the guess, and append ALL staged
+// entries to the candidate slot with coalesced stores.  Keeping the few entries that passed the
+// pre-test but fall just short of the guess is harmless: whenever at least k elements of the
+// layer reach the guess, the k best of this superset are the k best of the layer.
+constexpr int EMIT_QUEUE = 128;  // staged entries per warp and iteration; more than this = overflow
+
 template <bool VEC>
 __global__ void __launch_bounds__(THREADS)
     k_accumulate_emit(const float* __restrict__ grads, const float* __restrict__ weights, float* __restrict__ acc,
@@ -326,6 +334,9 @@ __global__ void __launch_bounds__(THREADS)
                       uint32_t* __restrict__ cand_cnt, float eps, uint64_t N, int W, int worker_groups) {
   constexpr int ROUNDS = 4;                 // 128-bit slots per lane and iteration
   constexpr int ITER_ELEMS = ROUNDS * 128;  // 512
+  __shared__ float q_val[WARPS][EMIT_QUEUE];
+  __shared__ float q_den[WARPS][EMIT_QUEUE];
+  __shared__ uint16_t q_loc[WARPS][EMIT_QUEUE];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t tile_id = blockIdx.x / worker_groups;
   const int w = static_cast<int>(blockIdx.x % worker_groups) * WARPS + warp;
@@ -341,7 +352,12 @@ __global__ void __launch_bounds__(THREADS)
   float* a = acc + static_cast<uint64_t>(w) * N;
   const uint64_t slot = (static_cast<uint64_t>(tile_id) * W + w) * CAND_CAP;
   const float zero[4] = {0.f, 0.f, 0.f, 0.f};
-  uint32_t count = 0;  // candidates of this (tile, worker) so far; the same in every lane
+  float* qv = q_val[warp];
+  float* qd = q_den[warp];
+  uint16_t* ql = q_loc[warp];
+  uint32_t count = 0;    // entries appended to the slot so far (the same in every lane)
+  uint32_t reached = 0;  // of those, how many reach the guess exactly
+  bool overflow = false;
 #pragma unroll 1
   for (uint32_t it = 0; it < TILE / ITER_ELEMS; ++it) {
     const uint64_t seg = base + it * ITER_ELEMS;
@@ -400,16 +416,7 @@ __global__ void __launch_bounds__(THREADS)
     }
     m &= inrange;
     if (__any_sync(0xffffffffu, m != 0u)) {
-      // exact test for the few that passed: Algorithm 1's |grad / w| compared with the guess
-#pragma unroll
-      for (int s = 0; s < ROUNDS; ++s) {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const uint32_t bit = 1u << (4 * s + c);
-          if ((m & bit) && imp_key_den(av[s][c], den[s][c]) < guess) m &= ~bit;
-        }
-      }
-      // rank inside the iteration: per-round counts packed 8 bits each (at most 128 per round)
+      // queue position in index order (round, lane, component): per-round counts packed 8 bits each
       uint32_t packed = 0;
 #pragma unroll
       for (int s = 0; s < ROUNDS; ++s) packed |= static_cast<uint32_t>(__popc((m >> (4 * s)) & 0xFu)) << (8 * s);
@@ -417,30 +424,55 @@ __global__ void __launch_bounds__(THREADS)
       const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
       const uint32_t excl = incl - packed;
       const uint32_t loc0 = static_cast<uint32_t>(first - base);
-      uint32_t round_base = count;
+      uint32_t round_base = 0;
+      if (m) {
 #pragma unroll
-      for (int s = 0; s < ROUNDS; ++s) {
-        uint32_t pos = round_base + ((excl >> (8 * s)) & 0xFFu);
+        for (int s = 0; s < ROUNDS; ++s) {
+          uint32_t pos = round_base + ((excl >> (8 * s)) & 0xFFu);
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          if ((m >> (4 * s + c)) & 1u) {
-            if (pos < CAND_CAP) {
-              cand_key[slot + pos] = imp_key_den(av[s][c], den[s][c]);
-              cand_val[slot + pos] = av[s][c];
-              cand_idx[slot + pos] = static_cast<uint16_t>(loc0 + s * 128 + c);
+          for (int c = 0; c < 4; ++c) {
+            if ((m >> (4 * s + c)) & 1u) {
+              if (pos < EMIT_QUEUE) {
+                qv[pos] = av[s][c];
+                qd[pos] = den[s][c];
+                ql[pos] = static_cast<uint16_t>(loc0 + s * 128 + c);
+              }
+              ++pos;
             }
-            ++pos;
+          }
+          round_base += (tot >> (8 * s)) & 0xFFu;
+        }
+      }
+      uint32_t nq = (tot & 0xFFu) + ((tot >> 8) & 0xFFu) + ((tot >> 16) & 0xFFu) + (tot >> 24);
+      if (nq > EMIT_QUEUE) {
+        overflow = true;
+        nq = EMIT_QUEUE;
+      }
+      __syncwarp();
+      for (uint32_t j0 = 0; j0 < nq; j0 += 32) {
+        const uint32_t j = j0 + lane;
+        bool hit = false;
+        if (j < nq) {
+          const float v = qv[j];
+          const uint32_t key = imp_key_den(v, qd[j]);  // Algorithm 1's |grad / w|, exactly rounded
+          hit = key >= guess;
+          const uint32_t pos = count + j;
+          if (pos < CAND_CAP) {
+            cand_key[slot + pos] = key;
+            cand_val[slot + pos] = v;
+            cand_idx[slot + pos] = ql[j];
           }
         }
-        round_base += (tot >> (8 * s)) & 0xFFu;
+        reached += __popc(__ballot_sync(0xffffffffu, hit));
       }
-      count = round_base;
+      count += nq;
+      __syncwarp();
     }
   }
   if (lane == 0) {
     cand_cnt[static_cast<uint64_t>(tile_id) * W + w] = count;
-    if (count) atomicAdd(&info[pair].total, count);
-    if (count > CAND_CAP) atomicOr(&info[pair].flags, 1u);
+    if (reached) atomicAdd(&info[pair].total, reached);
+    if (overflow || count > CAND_CAP) atomicOr(&info[pair].flags, 1u);
   }
 }
 

@@ -1,0 +1,101 @@
+"""GPU parity at the full sizes of the five benchmark configurations, in the launch
+configuration bench.py times (same library, same options, device-resident inputs).
+
+Configurations 1-3 are compared with the oracle on every output of every step.  For the
+W=32 stress case residuals are compared at a subset of steps (lists and updates at every step),
+and for the 2^30-element case the oracle runs on a subset of layers: layers are independent in
+steps (a)-(d) and steps (e)-(g) are element-wise, so a slice of the inputs reproduces exactly
+the slice of the outputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1901_01544_b200 import workloads as wl
+from paper_1901_01544_b200.binding import Pruner
+from parity import assert_bits_equal, run_parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.mark.parametrize("name", ["single_layer", "alexnet_w8", "resnet50_w8"])
+def test_full_size_every_output(name):
+    c = wl.CONFIGS[name]()
+    weights = c.weights(DEV)
+    buf = torch.empty((c.W, c.N), dtype=torch.float32, device=DEV)
+    run_parity(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, c.steps, weights, lambda t: c.grads(t, DEV, out=buf))
+
+
+def test_full_size_w32_stress():
+    c = wl.alexnet_w32()
+    steps = 8  # covers eight leader draws and the step-to-step threshold jumps; 20 steps run scaled elsewhere
+    weights = c.weights(DEV)
+    w_host = weights.cpu().numpy()
+    pr = Pruner(c.layer_sizes, c.W, c.ratio, c.eps, c.seed)
+    orc = oracle.Oracle(c.layer_sizes, c.W, c.ratio, c.eps, c.seed)
+    assert 4 * c.W * c.N > 2 ** 32  # byte offsets into [w][i] buffers do not fit 32 bits
+    g = torch.empty((c.W, c.N), dtype=torch.float32, device=DEV)
+    upd = torch.empty(c.N, dtype=torch.float32, device=DEV)
+    for t in range(steps):
+        c.grads(t, DEV, out=g)
+        pr.step(g, weights, upd)
+        want = orc.step(g.cpu().numpy(), w_host)
+        assert pr.sync_status() == 0 and pr.leader == orc.leader
+        assert_bits_equal(upd.cpu().numpy(), want, f"step {t}: update")
+        for w in range(c.W):
+            gi, gv = pr.selection(w)
+            oi, ov = orc.selection(w)
+            assert np.array_equal(gi.cpu().numpy().view(np.uint32), oi), f"step {t}: worker {w} indices"
+            assert_bits_equal(gv.cpu().numpy(), ov, f"step {t}: worker {w} values")
+        if t in (0, 3, steps - 1):
+            for w in range(c.W):
+                assert_bits_equal(pr.residual(w).cpu().numpy(), orc.residual(w), f"step {t}: worker {w} residual")
+        assert pr.stat("spec_failed") == 0, "the sampled guess must survive the per-step scale jumps"
+    pr.close()
+    orc.close()
+
+
+def test_full_size_flat_2p30_on_layer_subset():
+    c = wl.flat_1g_w4()
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60 * 2 ** 30:
+        pytest.skip("needs about 50 GiB of device memory")
+    steps = 4
+    sub = [0, 1, 63, 64, 95]  # includes layers that start at odd element offsets and both layer sizes
+    off = c.offsets()
+    sizes = [c.layer_sizes[l] for l in sub]
+    assert off[1] % 4 != 0 and c.W * c.N == 2 ** 32
+    weights = c.weights(DEV)
+    pr = Pruner(c.layer_sizes, c.W, c.ratio, c.eps, c.seed)
+    orc = oracle.Oracle(sizes, c.W, c.ratio, c.eps, c.seed)
+    goff, gk = pr.layout()
+    koff = np.concatenate([[0], np.cumsum(gk)]).astype(np.int64)
+    sub_off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    sl = lambda x: torch.cat([x[..., off[l]: off[l] + c.layer_sizes[l]] for l in sub], dim=-1)
+    w_sub = sl(weights).cpu().numpy()
+    g = torch.empty((c.W, c.N), dtype=torch.float32, device=DEV)
+    upd = torch.empty(c.N, dtype=torch.float32, device=DEV)
+    for t in range(steps):
+        c.grads(t, DEV, out=g)
+        pr.step(g, weights, upd)
+        want = orc.step(np.ascontiguousarray(sl(g).cpu().numpy()), w_sub)
+        assert pr.sync_status() == 0 and pr.leader == orc.leader
+        assert pr.stat("spec_failed") == 0
+        assert_bits_equal(sl(upd).cpu().numpy(), want, f"step {t}: update on the layer subset")
+        # everything off the index set is +0, and the set has exactly K members
+        assert int(torch.count_nonzero(upd).item()) <= pr.K
+        assert int(pr.mask().sum().item()) == pr.K
+        for w in range(c.W):
+            gi, gv = pr.selection(w)
+            oi, ov = orc.selection(w)
+            gi = gi.cpu().numpy().view(np.uint32).astype(np.int64)
+            gv = gv.cpu().numpy()
+            for j, l in enumerate(sub):
+                seg = slice(koff[l], koff[l + 1])
+                oseg = slice(j * gk[l], (j + 1) * gk[l])  # every layer keeps the same count here
+                assert np.array_equal(gi[seg] - off[l] + sub_off[j], oi[oseg].astype(np.int64)), (t, w, l)
+                assert_bits_equal(gv[seg], ov[oseg], f"step {t}: worker {w} layer {l} values")
+            assert_bits_equal(sl(pr.residual(w)).cpu().numpy(), orc.residual(w), f"step {t}: worker {w} residual")
+    pr.close()
+    orc.close()
