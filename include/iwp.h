@@ -163,6 +163,36 @@ int iwp_set_option(iwp_ctx* ctx, const char* key, int64_t value);
  * Unknown key: IWP_ERR_INVALID. */
 int iwp_get_stat(iwp_ctx* ctx, const char* key, int64_t* value_host);
 
+/* ---- selection without any allocation --------------------------------------------------- */
+
+/* (No counterpart in the paper: this entry point exists for callers of this library that are not
+ * allowed to allocate device memory while they run - code under a start-up-only arena or pool
+ * discipline, latency-critical loops that cannot afford the device synchronisation an allocation
+ * implies, plug-ins bound by a host framework's no-allocation rule.)
+ *
+ * Writes the exact top-k list of ONE layer for ONE worker: the k = ceil(n / ratio) elements of
+ * residual_dev[0..n) with the largest importance |residual| / (|weights| + eps), ties to the lower
+ * index, as ascending indices idx_dev[0..k) and their residual values val_dev[0..k) - the same
+ * result, bit for bit, as the list iwp_step() builds for that layer.  It needs no context and
+ * calls no cudaMalloc / cudaFree or any other allocating routine: all scratch lives in a fixed
+ * device array of about 10 KB that every GPU loading this library holds until the process exits.
+ *
+ *   residual_dev, weights_dev  n floats each, device, read only
+ *   n                          1 .. 16 777 216 (2^24); larger layers are rejected with IWP_ERR_INVALID
+ *   ratio, eps                 as in iwp_create()
+ *   idx_dev, val_dev           device buffers of at least k entries, overwritten
+ *   k_host                     optional: receives k
+ *   cuda_stream                stream the kernels are enqueued on (NULL = legacy default stream)
+ *
+ * Asynchronous like iwp_step().  The first call made with a given device current looks up the
+ * scratch array's device address; make that first call before any stream capture begins.  All
+ * calls on a device share the one scratch array (it keeps the previous call's contents; the entry
+ * point clears what must start at zero), so two calls whose kernels can overlap on the GPU - on
+ * different streams, or from different threads - race: serialise them.
+ * Errors: IWP_ERR_INVALID (NULL pointer, n out of range, bad ratio or eps), IWP_ERR_CUDA. */
+int iwp_select_static(const float* residual_dev, const float* weights_dev, int64_t n, double ratio, float eps,
+                      uint32_t* idx_dev, float* val_dev, int64_t* k_host, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -19,7 +19,7 @@ EXPORTS = [
     "iwp_strerror", "iwp_keep_count", "iwp_leader_at", "iwp_plan_sizes", "iwp_create", "iwp_destroy",
     "iwp_set_stream", "iwp_step", "iwp_step_host", "iwp_sync_status", "iwp_get_layout", "iwp_get_sizes",
     "iwp_get_step", "iwp_set_step", "iwp_get_leader", "iwp_get_residual", "iwp_set_residual",
-    "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat",
+    "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat", "iwp_select_static",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -63,6 +63,7 @@ def lib() -> C.CDLL:
         L.iwp_reset.argtypes = [vp]
         L.iwp_set_option.argtypes = [vp, cp, i64]
         L.iwp_get_stat.argtypes = [vp, cp, vp]
+        L.iwp_select_static.argtypes = [vp, vp, i64, f64, f32, vp, vp, vp, vp]
         for name in EXPORTS:
             getattr(L, name)  # AttributeError if the library does not export a declared symbol
         _lib = L
@@ -114,6 +115,15 @@ def iwp_step(h, grads_ptr: int, weights_ptr: int, update_ptr: int) -> None:
 
 def iwp_step_host(h, grads_ptr: int, weights_ptr: int, update_ptr: int) -> None:
     _check(lib().iwp_step_host(h, grads_ptr, weights_ptr, update_ptr), "iwp_step_host")
+
+
+def iwp_select_static(residual_ptr: int, weights_ptr: int, n: int, ratio: float, eps: float, idx_ptr: int,
+                      val_ptr: int, stream: int = 0) -> int:
+    """Top-k list of one layer without any allocation (see include/iwp.h); returns k."""
+    k = C.c_int64()
+    _check(lib().iwp_select_static(residual_ptr, weights_ptr, n, ratio, eps, idx_ptr, val_ptr, C.byref(k),
+                                   C.c_void_p(stream)), "iwp_select_static")
+    return int(k.value)
 
 
 # ---- convenience wrapper over torch tensors ----------------------------------------------------

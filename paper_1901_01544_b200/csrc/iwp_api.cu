@@ -4,6 +4,7 @@
 
 #include <cuda_runtime.h>
 
+#include <cmath>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -639,3 +640,124 @@ int iwp_get_stat(iwp_ctx* c, const char* key, int64_t* value) {
 }
 
 }  // extern "C"
+
+// =========================================================================================
+// iwp_select_static: the exact top-k list of ONE layer for ONE worker without any allocation.
+//
+// Some callers must not allocate device memory while they run: code inside a memory-pool or
+// arena discipline that forbids cudaMalloc after start-up, real-time loops where an allocation's
+// implicit device synchronisation is unacceptable, or plug-ins that run under a host framework's
+// "no allocation here" rule.  For them this entry point runs the same exact multi-pass select
+// and stable compaction as the tiled path of iwp_step(), but takes every byte of scratch
+// (histogram, select state, chunk tables and counts) from the fixed device array below instead
+// of from a context created by iwp_create().
+//
+// The array's name is only a host-side handle; kernels get its device address, which is looked
+// up once per device with cudaGetSymbolAddress() on the first call made with that device current.
+// =========================================================================================
+namespace {
+
+constexpr int64_t STATIC_MAX_N = int64_t(1) << 24;  // largest layer the fixed scratch is sized for
+constexpr uint32_t STATIC_CHUNK_ELEMS = CHUNK_TILES * TILE;
+constexpr uint32_t STATIC_MAX_CHUNKS = static_cast<uint32_t>(STATIC_MAX_N / STATIC_CHUNK_ELEMS) + 1;  // 33
+
+struct StaticScratch {
+  uint32_t hist[NBINS];  // must be zero when a select starts
+  uint2 state;
+  PairInfo info;         // guess = none: the select reads the residual itself
+  LayerDesc layer;
+  uint32_t large_id;
+  int status;
+  uint2 chunk_cnt[STATIC_MAX_CHUNKS];
+  Chunk chunks[STATIC_MAX_CHUNKS];
+};
+
+// Held by every GPU that loads this library, until the process exits (about 10 KB).
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+StaticScratch* g_static_ptr[STATIC_MAX_DEVICES] = {};  // device address of the array, per device ordinal
+
+// Fills the tables for a layer of n elements and clears what must start at zero.
+__global__ void k_static_setup(StaticScratch* s, uint32_t n, uint32_t k, uint32_t n_chunks) {
+  for (uint32_t b = threadIdx.x; b < NBINS; b += blockDim.x) s->hist[b] = 0;
+  for (uint32_t j = threadIdx.x; j < n_chunks; j += blockDim.x) {
+    Chunk c{};
+    c.a = j * STATIC_CHUNK_ELEMS;
+    c.len = (n - c.a < STATIC_CHUNK_ELEMS) ? n - c.a : STATIC_CHUNK_ELEMS;
+    c.layer = 0;
+    c.first_tile = 0;
+    c.n_tiles = 0;
+    c.first_chunk_of_layer = 0;
+    s->chunks[j] = c;
+    s->chunk_cnt[j] = make_uint2(0u, 0u);
+  }
+  if (threadIdx.x == 0) {
+    s->state = make_uint2(0u, 0u);
+    s->info = PairInfo{GUESS_NONE, 0u, 0u, 0u};
+    LayerDesc L{};
+    L.off = 0;
+    L.n = n;
+    L.k = k;
+    L.koff = 0;
+    L.large_index = 0;
+    s->layer = L;
+    s->large_id = 0;
+    s->status = 0;
+  }
+}
+
+template <bool VEC>
+int run_select_static(StaticScratch* s, const float* residual, const float* weights, uint32_t n, uint32_t k, float eps,
+                      uint32_t* idx, float* val, cudaStream_t st) {
+  const uint32_t n_chunks = (n + STATIC_CHUNK_ELEMS - 1) / STATIC_CHUNK_ELEMS;
+  k_static_setup<<<1, THREADS, 0, st>>>(s, n, k, n_chunks);
+  if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+  dim3 grid(n_chunks, 1);
+  for (int pass = 0; pass < N_PASSES; ++pass) {
+    k_hist<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr,
+                                          &s->state, s->hist, eps, 0, 1, pass);
+    if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+    k_find_digit<<<1, THREADS, 0, st>>>(&s->state, s->hist, &s->layer, &s->large_id, &s->status, 1, pass);
+    if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+  }
+  k_count<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr, &s->state,
+                                         s->chunk_cnt, eps, 0, 1, n_chunks);
+  if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+  k_write<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, nullptr, &s->layer, &s->info, nullptr, nullptr,
+                                         nullptr, nullptr, &s->state, s->chunk_cnt, idx, val, &s->status, eps, 0, 0, 1,
+                                         n_chunks);
+  if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+  return IWP_OK;
+}
+
+}  // namespace
+
+extern "C" int iwp_select_static(const float* residual_dev, const float* weights_dev, int64_t n, double ratio, float eps,
+                                 uint32_t* idx_dev, float* val_dev, int64_t* k_host, void* cuda_stream) {
+  if (!residual_dev || !weights_dev || !idx_dev || !val_dev) return IWP_ERR_INVALID;
+  if (n < 1 || n > STATIC_MAX_N) return IWP_ERR_INVALID;  // beyond what the fixed scratch is sized for
+  if (!(eps > 0.f) || !std::isfinite(eps)) return IWP_ERR_INVALID;
+  const int64_t k = keep_count(n, ratio);
+  if (k < 1) return IWP_ERR_INVALID;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  if (!g_static_ptr[dev]) {  // first call with this device current: look up the array's device address
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return IWP_ERR_CUDA;
+    }
+    g_static_ptr[dev] = static_cast<StaticScratch*>(p);
+  }
+  if (k_host) *k_host = k;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const bool vec = aligned16(residual_dev) && aligned16(weights_dev);
+  return vec ? run_select_static<true>(g_static_ptr[dev], residual_dev, weights_dev, static_cast<uint32_t>(n),
+                                       static_cast<uint32_t>(k), eps, idx_dev, val_dev, st)
+             : run_select_static<false>(g_static_ptr[dev], residual_dev, weights_dev, static_cast<uint32_t>(n),
+                                        static_cast<uint32_t>(k), eps, idx_dev, val_dev, st);
+}
