@@ -40,6 +40,11 @@ struct iwp_ctx {
   uint32_t* d_hist = nullptr;
   uint2* d_chunk_cnt = nullptr;
   PairInfo* d_info = nullptr;     // threshold guess and candidate totals per pair
+  uint2* d_guess = nullptr;       // read-only (guess, pre-test multiplier) per pair for the streaming pass
+  float* side_val = nullptr;      // every worker's value at the leader's slot positions, laid out like cand_val
+  uint32_t* sel_slot = nullptr;   // [K] slot position of each entry of the leader's list, or REF_NONE
+  uint2* lead_lane = nullptr;     // [segment][32] the leader's staged mask | count << 16, lane prefix
+  uint32_t* lead_tot = nullptr;   // [segment] the leader's per-round totals
   uint32_t* cand_key = nullptr;   // candidate slots [tile][worker][CAND_CAP]
   float* cand_val = nullptr;
   uint16_t* cand_idx = nullptr;
@@ -84,10 +89,11 @@ void stage_clear(iwp_ctx* c) {
 
 struct Sizes {
   uint64_t acc, layers, tiles, chunks, small_ids, large_ids, state, hist, chunk_cnt, sel_idx, sel_val, status;
-  uint64_t info, cand_key, cand_val, cand_idx, cand_cnt;
+  uint64_t info, cand_key, cand_val, cand_idx, cand_cnt, guess, side_val, sel_slot, lead_lane, lead_tot;
   uint64_t total() const {
     return acc + layers + tiles + chunks + small_ids + large_ids + state + hist + chunk_cnt + sel_idx + sel_val +
-           status + info + cand_key + cand_val + cand_idx + cand_cnt;
+           status + info + cand_key + cand_val + cand_idx + cand_cnt + guess + side_val + sel_slot + lead_lane +
+           lead_tot;
   }
 };
 
@@ -117,6 +123,12 @@ Sizes sizes_of(const Plan& p) {
   s.cand_val = at_least(slots * CAND_CAP * sizeof(float));
   s.cand_idx = at_least(slots * CAND_CAP * sizeof(uint16_t));
   s.cand_cnt = at_least(slots * sizeof(uint32_t));
+  const uint64_t segs = any_spec ? p.tiles.size() * SEGS_PER_TILE : 0;
+  s.guess = at_least(pairs * sizeof(uint2));
+  s.side_val = at_least(slots * CAND_CAP * sizeof(float));
+  s.sel_slot = at_least(p.K * sizeof(uint32_t));
+  s.lead_lane = at_least(segs * 32 * sizeof(uint2));
+  s.lead_tot = at_least(segs * sizeof(uint32_t));
   return s;
 }
 
@@ -151,6 +163,11 @@ void free_all(iwp_ctx* c) {
   cudaFree(c->cand_val);
   cudaFree(c->cand_idx);
   cudaFree(c->cand_cnt);
+  cudaFree(c->d_guess);
+  cudaFree(c->side_val);
+  cudaFree(c->sel_slot);
+  cudaFree(c->lead_lane);
+  cudaFree(c->lead_tot);
   cudaFree(c->sel_idx);
   cudaFree(c->sel_val);
   cudaFree(c->d_status);
@@ -178,7 +195,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     const size_t dyn = static_cast<size_t>(p.max_small_n) * sizeof(uint32_t);
     dim3 grid(static_cast<unsigned>(p.small_layers.size()), static_cast<unsigned>(W));
     k_small<<<grid, THREADS, dyn, s>>>(grads, weights, c->acc, update, c->d_layers, c->d_small_ids, c->sel_idx,
-                                       c->sel_val, c->d_status, c->eps, N, K);
+                                       c->sel_val, c->sel_slot, c->d_status, c->eps, N, K, leader);
     IWP_LAUNCH_CHECK(c);
   }
   stage_mark(c);
@@ -194,8 +211,8 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   }
   if (spec) {
     const size_t dyn = static_cast<size_t>(c->max_sample) * sizeof(uint32_t);
-    k_sample<<<c->n_pairs, THREADS, dyn, s>>>(grads, weights, c->acc, c->d_layers, c->d_large_ids, c->d_info, c->eps, N,
-                                             W, static_cast<uint32_t>(c->t));
+    k_sample<<<c->n_pairs, THREADS, dyn, s>>>(grads, weights, c->acc, c->d_layers, c->d_large_ids, c->d_info,
+                                             c->d_guess, c->eps, N, W, static_cast<uint32_t>(c->t));
     IWP_LAUNCH_CHECK(c);
     c->info_clean = false;
   }
@@ -203,10 +220,17 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   if (tiled) {
     const unsigned n_tiles = static_cast<unsigned>(p.tiles.size());
     if (spec) {
-      const int groups = (W + WARPS - 1) / WARPS;
-      k_accumulate_emit<VEC><<<n_tiles * static_cast<unsigned>(groups), THREADS, 0, s>>>(
-          grads, weights, c->acc, update, c->d_tiles, c->d_info, c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt,
-          c->eps, N, W, groups);
+      // the leader's workers first (records where its candidates sit), then everybody else
+      k_stream<VEC, true><<<(n_tiles + WARPS - 1) / WARPS, THREADS, 0, s>>>(
+          grads, weights, c->acc, update, c->d_tiles, c->d_info, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
+          c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->eps, N, W, leader, n_tiles, 1);
+      if (W > 1) {
+        IWP_LAUNCH_CHECK(c);
+        const int groups = (W - 1 + WARPS - 1) / WARPS;
+        k_stream<VEC, false><<<n_tiles * static_cast<unsigned>(groups), THREADS, 0, s>>>(
+            grads, weights, c->acc, update, c->d_tiles, c->d_info, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
+            c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->eps, N, W, leader, n_tiles, groups);
+      }
     } else {
       k_accumulate<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, N, W);
     }
@@ -234,14 +258,19 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     IWP_LAUNCH_CHECK(c);
     k_write<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->d_info,
                                            c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
-                                           c->d_chunk_cnt, c->sel_idx, c->sel_val, c->d_status, c->eps, N, K, W,
-                                           n_chunks);
+                                           c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, c->d_status, c->eps,
+                                           N, K, W, n_chunks, leader);
     IWP_LAUNCH_CHECK(c);
   }
   stage_mark(c);
   const unsigned gblocks = static_cast<unsigned>((K + THREADS - 1) / THREADS);
-  k_gather_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->acc, update, N,
-                                                   K, W);
+  if (spec) {
+    k_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->sel_slot, c->side_val,
+                                              c->cand_val, c->acc, update, N, K, W, leader);
+  } else {
+    k_gather_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->acc, update,
+                                                     N, K, W);
+  }
   IWP_LAUNCH_CHECK(c);
   stage_mark(c);
   return IWP_OK;
@@ -328,6 +357,11 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
   A(&c->cand_val, sz.cand_val);
   A(&c->cand_idx, sz.cand_idx);
   A(&c->cand_cnt, sz.cand_cnt);
+  A(&c->d_guess, sz.guess);
+  A(&c->side_val, sz.side_val);
+  A(&c->sel_slot, sz.sel_slot);
+  A(&c->lead_lane, sz.lead_lane);
+  A(&c->lead_tot, sz.lead_tot);
   A(&c->sel_idx, sz.sel_idx);
   A(&c->sel_val, sz.sel_val);
   A(&c->d_status, sz.status);
@@ -354,6 +388,7 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
   ok = ok && cudaMemset(c->d_status, 0, sz.status) == cudaSuccess;
   ok = ok && cudaMemset(c->d_info, 0xff, sz.info) == cudaSuccess;  // guess = none, overflow flag set
   ok = ok && cudaMemset(c->cand_cnt, 0, sz.cand_cnt) == cudaSuccess;
+  ok = ok && cudaMemset(c->sel_slot, 0xff, sz.sel_slot) == cudaSuccess;
   for (uint32_t l : p.large_layers) {
     if (p.layers[l].sample > c->max_sample) c->max_sample = p.layers[l].sample;
     if (p.layers[l].sample) c->spec_pairs += static_cast<uint32_t>(W);
@@ -725,8 +760,8 @@ int run_select_static(StaticScratch* s, const float* residual, const float* weig
                                          s->chunk_cnt, eps, 0, 1, n_chunks);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   k_write<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, nullptr, &s->layer, &s->info, nullptr, nullptr,
-                                         nullptr, nullptr, &s->state, s->chunk_cnt, idx, val, &s->status, eps, 0, 0, 1,
-                                         n_chunks);
+                                         nullptr, nullptr, &s->state, s->chunk_cnt, idx, val, nullptr, &s->status, eps,
+                                         0, 0, 1, n_chunks, -1);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   return IWP_OK;
 }

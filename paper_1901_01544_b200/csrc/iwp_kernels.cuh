@@ -31,7 +31,7 @@ struct PairInfo {
   uint32_t guess;  // candidates include every element with importance pattern >= guess; GUESS_NONE = none
   uint32_t total;  // number of elements of the layer that reach the guess
   uint32_t flags;  // bit 0: some (tile, worker) slot or staging queue overflowed
-  uint32_t pad;
+  uint32_t gm;     // bit pattern of the pre-test multiplier derived from the guess
 };
 
 // The candidates hold the exact top-k iff there are at least k of them and none was dropped.
@@ -254,6 +254,8 @@ __global__ void __launch_bounds__(THREADS) k_accumulate(const float* __restrict_
 // takes the rho-th largest as the guess.  Only a guess: the select stays exact whatever it is.
 // grid = pairs; dynamic shared memory = 4 * max sample bytes.
 // ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float pretest_multiplier(uint32_t guess, float eps);
+
 __device__ __forceinline__ uint32_t hash32(uint32_t x) {
   x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
   return x;
@@ -262,7 +264,7 @@ __device__ __forceinline__ uint32_t hash32(uint32_t x) {
 __global__ void __launch_bounds__(THREADS)
     k_sample(const float* __restrict__ grads, const float* __restrict__ weights, const float* __restrict__ acc,
              const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ large_ids, PairInfo* __restrict__ info,
-             float eps, uint64_t N, int W, uint32_t step) {
+             uint2* __restrict__ guess_tab, float eps, uint64_t N, int W, uint32_t step) {
   extern __shared__ uint32_t keys[];
   __shared__ uint32_t hist[NBINS];
   __shared__ uint32_t sh_scan[THREADS];
@@ -272,7 +274,11 @@ __global__ void __launch_bounds__(THREADS)
   const int w = pair % W;
   const uint32_t s = L.sample;
   if (s == 0) {
-    if (threadIdx.x == 0) info[pair] = PairInfo{GUESS_NONE, 0u, 0u, 0u};
+    if (threadIdx.x == 0) {
+      const uint32_t gm = __float_as_uint(pretest_multiplier(GUESS_NONE, eps));
+      info[pair] = PairInfo{GUESS_NONE, 0u, 0u, gm};
+      guess_tab[pair] = make_uint2(GUESS_NONE, gm);
+    }
     return;
   }
   const uint32_t groups = s >> 3;
@@ -280,36 +286,66 @@ __global__ void __launch_bounds__(THREADS)
   const float* a = acc + static_cast<uint64_t>(w) * N + L.off;
   const float* g = grads + static_cast<uint64_t>(w) * N + L.off;
   const float* wt = weights + L.off;
-  for (uint32_t i = threadIdx.x; i < s; i += THREADS) {
-    const uint32_t grp = i >> 3;
-    const uint32_t jit = hash32(step * 0x9E3779B9u + pair * 0x85EBCA6Bu + grp * 0xC2B2AE35u + 1u) % (stride - 7u);
-    const uint32_t pos = grp * stride + jit + (i & 7u);
-    keys[i] = imp_key(__fadd_rn(a[pos], g[pos]), wt[pos], eps);
+  // eight samples per thread and trip, all loads issued before any use (memory-level parallelism)
+  for (uint32_t i0 = 0; i0 < s; i0 += THREADS * 8) {
+    float av[8], gv[8], wv[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const uint32_t i = i0 + u * THREADS + threadIdx.x;
+      av[u] = gv[u] = 0.f;
+      wv[u] = 1.f;
+      if (i < s) {
+        const uint32_t grp = i >> 3;
+        const uint32_t jit = hash32(step * 0x9E3779B9u + pair * 0x85EBCA6Bu + grp * 0xC2B2AE35u + 1u) % (stride - 7u);
+        const uint32_t pos = grp * stride + jit + (i & 7u);
+        av[u] = a[pos];
+        gv[u] = g[pos];
+        wv[u] = wt[pos];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const uint32_t i = i0 + u * THREADS + threadIdx.x;
+      if (i < s) keys[i] = imp_key(__fadd_rn(av[u], gv[u]), wv[u], eps);
+    }
   }
   __syncthreads();
   uint32_t T, r;
   const bool ok = smem_radix_select(keys, s, L.rho, hist, sh_scan, res, T, r);
-  if (threadIdx.x == 0) info[pair] = PairInfo{(ok && T != 0u) ? T : GUESS_NONE, 0u, 0u, 0u};
+  if (threadIdx.x == 0) {
+    const uint32_t guess = (ok && T != 0u) ? T : GUESS_NONE;
+    const uint32_t gm = __float_as_uint(pretest_multiplier(guess, eps));
+    info[pair] = PairInfo{guess, 0u, 0u, gm};
+    guess_tab[pair] = make_uint2(guess, gm);  // read-only copy for the streaming pass (no atomics land on it)
+  }
 }
 
 // ---------------------------------------------------------------------------------------
-// single-read path, steps (a)+(b) fused with candidate emission: acc += grads, update <- 0,
-// importance of every element, and every element whose importance reaches the pair's guess is
-// appended, in index order, to the (tile, worker) candidate slot.
+// single-read path: steps (a)+(b) fused with candidate emission and with the gather of step (e).
+//
+// acc += grads, update <- 0, importance of every element; every element whose importance reaches
+// its pair's guess is appended, in index order, to the (tile, worker) candidate slot; and every
+// worker's accumulated value at the positions of the LEADER's candidates is written to a side
+// buffer, so that after the select the reduction reads those few values instead of gathering
+// W * K scattered residuals (each of which costs a 128-byte DRAM fetch).
 //
 // One WARP owns one (tile, worker) pair and walks the tile front to back, 512 elements per
-// iteration (four rounds of 32 lanes x one 128-bit slot), so the index order of the candidates
-// is (iteration, round, lane, component) and a running count in a register is all the state:
-// no shared memory, no block barrier, warps never wait for each other.  The eight warps of a
-// CTA take eight workers of the same tile, so the tile's weights are fetched from HBM once and
-// re-read through L1.  grid = tiles * ceil(W / 8).
+// iteration (four rounds of 32 lanes x one 128-bit slot): candidate order is (iteration, round,
+// lane, component) = index order, a running count in a register is all the state, warps never
+// wait for each other.  The kernel runs twice per step: first for the leader alone (LEADER =
+// true: it also zeroes `update` and records, per segment and lane, its staged mask and ranks),
+// then for all other workers, which read that record to place their values in the side buffer.
+//
+// Cheap pre-test before the exact quotient: with gm = guess * (1 - 2^-20) every element whose
+// correctly rounded quotient |acc| / den reaches the guess passes |acc| >= gm * den (the two
+// roundings of gm * den and the one of the quotient are each below 2^-23 relative).  Elements that
+// pass are staged, in index order, in a per-warp queue in shared memory; the lanes then take one
+// entry each, form the exact quotient (one division per lane, not per element), count how many
+// really reach the guess, and append ALL staged entries with coalesced stores.  Keeping the few
+// entries that fall just short of the guess is harmless: whenever at least k elements of the layer
+// reach the guess, the k best of this superset are the k best of the layer.  The argument needs
+// normal products, so the pre-test is disabled (gm = 0: everything passes) for tiny guesses or eps.
 // ---------------------------------------------------------------------------------------
-// Conservative multiplier for the cheap candidate pre-test |acc| >= gm * den: with
-// gm = guess * (1 - 2^-20) every element whose correctly rounded quotient |acc| / den reaches the
-// guess passes it (the two roundings of gm * den and the one of the quotient are each below 2^-23
-// relative); the exact quotient is then formed only for the few elements that pass.  The argument
-// needs normal products, so the pre-test is disabled (gm = 0: everything passes) for tiny guesses
-// or a tiny eps.
 __device__ __forceinline__ float pretest_multiplier(uint32_t guess, float eps) {
   if (guess == GUESS_NONE) return __int_as_float(0x7f800000);  // +inf: nothing passes
   const float gf = __uint_as_float(guess);
@@ -318,36 +354,52 @@ __device__ __forceinline__ float pretest_multiplier(uint32_t guess, float eps) {
   return __fmul_rd(gf, 1.0f - 9.5367431640625e-07f);
 }
 
-// Elements that pass the pre-test are staged, in index order, in a per-warp queue in shared
-// memory; the lanes then take one queue entry each, form the exact quotient (one division per
-// lane instead of one per element), count how many really reach the guess, and append ALL staged
-// entries to the candidate slot with coalesced stores.  Keeping the few entries that passed the
-// pre-test but fall just short of the guess is harmless: whenever at least k elements of the
-// layer reach the guess, the k best of this superset are the k best of the layer.
 constexpr int EMIT_QUEUE = 128;  // staged entries per warp and iteration; more than this = overflow
 
-template <bool VEC>
+// Position, inside one iteration, of the staged element with mask bit b = 4 * round + component:
+// the staged elements of earlier rounds, of earlier lanes in the same round, and of earlier
+// components of the same lane and round.  `ex` / `tt`: per-round exclusive lane prefix / totals,
+// packed 8 bits per round.
+__device__ __forceinline__ uint32_t staged_position(uint32_t mask, uint32_t ex, uint32_t tt, uint32_t b) {
+  const uint32_t sh = (b >> 2) * 8;
+  const uint32_t rounds_before = ((tt * 0x01010100u) >> sh) & 0xFFu;  // byte r of tt * 0x01010100 = sum of rounds < r
+  return rounds_before + ((ex >> sh) & 0xFFu) + __popc((mask >> (b & ~3u)) & ((1u << (b & 3u)) - 1u));
+}
+
+template <bool VEC, bool LEADER>
 __global__ void __launch_bounds__(THREADS)
-    k_accumulate_emit(const float* __restrict__ grads, const float* __restrict__ weights, float* __restrict__ acc,
-                      float* __restrict__ update, const Tile* __restrict__ tiles, PairInfo* __restrict__ info,
-                      uint32_t* __restrict__ cand_key, float* __restrict__ cand_val, uint16_t* __restrict__ cand_idx,
-                      uint32_t* __restrict__ cand_cnt, float eps, uint64_t N, int W, int worker_groups) {
-  constexpr int ROUNDS = 4;                 // 128-bit slots per lane and iteration
-  constexpr int ITER_ELEMS = ROUNDS * 128;  // 512
+    k_stream(const float* __restrict__ grads, const float* __restrict__ weights, float* __restrict__ acc,
+             float* __restrict__ update, const Tile* __restrict__ tiles, PairInfo* __restrict__ info,
+             const uint2* __restrict__ guess_tab, uint32_t* __restrict__ cand_key, float* __restrict__ cand_val,
+             uint16_t* __restrict__ cand_idx, uint32_t* __restrict__ cand_cnt, float* __restrict__ side_val,
+             uint2* __restrict__ lead_lane, uint32_t* __restrict__ lead_tot, float eps, uint64_t N, int W, int leader,
+             uint32_t n_tiles, int worker_groups) {
+  constexpr int ROUNDS = SEG_ELEMS / 128;  // 128-bit slots per lane and iteration = 4
   __shared__ float q_val[WARPS][EMIT_QUEUE];
   __shared__ float q_den[WARPS][EMIT_QUEUE];
   __shared__ uint16_t q_loc[WARPS][EMIT_QUEUE];
+  __shared__ __align__(16) float r_val[WARPS][SEG_ELEMS];  // results of the iteration, for run-time indexing
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t tile_id = blockIdx.x / worker_groups;
-  const int w = static_cast<int>(blockIdx.x % worker_groups) * WARPS + warp;
-  if (w >= W) return;
+  uint32_t tile_id;
+  int w;
+  if (LEADER) {  // eight tiles of the leader per CTA
+    tile_id = blockIdx.x * WARPS + warp;
+    w = leader;
+    if (tile_id >= n_tiles) return;
+  } else {  // up to eight of the other workers of one tile per CTA: the tile's weights come through L1
+    tile_id = blockIdx.x / worker_groups;
+    const int wi = static_cast<int>(blockIdx.x % worker_groups) * WARPS + warp;
+    if (wi >= W - 1) return;
+    w = wi < leader ? wi : wi + 1;
+  }
   const Tile t = tiles[tile_id];
   const uint64_t lo = t.a, hi = lo + t.len;
   const uint64_t base = lo & ~static_cast<uint64_t>(TILE - 1);
   const bool full = VEC && t.len == TILE;  // every slot of the window is inside the tile
   const uint32_t pair = t.large_index * W + w;
-  const uint32_t guess = info[pair].guess;
-  const float gm = pretest_multiplier(guess, eps);
+  const uint2 pg = guess_tab[pair];
+  const uint32_t guess = pg.x;
+  const float gm = __uint_as_float(pg.y);
   const float* g = grads + static_cast<uint64_t>(w) * N;
   float* a = acc + static_cast<uint64_t>(w) * N;
   const uint64_t slot = (static_cast<uint64_t>(tile_id) * W + w) * CAND_CAP;
@@ -355,23 +407,31 @@ __global__ void __launch_bounds__(THREADS)
   float* qv = q_val[warp];
   float* qd = q_den[warp];
   uint16_t* ql = q_loc[warp];
+  float* res = r_val[warp] + lane * 4;
   uint32_t count = 0;    // entries appended to the slot so far (the same in every lane)
   uint32_t reached = 0;  // of those, how many reach the guess exactly
   bool overflow = false;
 #pragma unroll 1
-  for (uint32_t it = 0; it < TILE / ITER_ELEMS; ++it) {
-    const uint64_t seg = base + it * ITER_ELEMS;
-    if (seg + ITER_ELEMS <= lo || seg >= hi) continue;  // warp-uniform
+  for (uint32_t it = 0; it < SEGS_PER_TILE; ++it) {
+    const uint64_t seg = base + it * SEG_ELEMS;
+    if (seg + SEG_ELEMS <= lo || seg >= hi) continue;  // warp-uniform
     const uint64_t first = seg + static_cast<uint64_t>(lane) * 4;  // this lane's slot in round 0
+    const uint64_t sigma = static_cast<uint64_t>(tile_id) * SEGS_PER_TILE + it;  // global segment id
     float gv[ROUNDS][4], av[ROUNDS][4], den[ROUNDS][4];
     uint32_t inrange = 0xFFFFu;
+    uint2 ll = make_uint2(0u, 0u);
+    uint32_t lt = 0;
+    if (!LEADER) {  // the leader's record for this segment: (mask | count << 16, lane prefix), round totals
+      ll = lead_lane[sigma * 32 + lane];
+      lt = lead_tot[sigma];
+    }
     if (full) {
       const float4* g4 = reinterpret_cast<const float4*>(g + first);
       const float4* a4 = reinterpret_cast<const float4*>(a + first);
       const float4* w4 = reinterpret_cast<const float4*>(weights + first);
 #pragma unroll
       for (int s = 0; s < ROUNDS; ++s) {
-        const float4 x = __ldcs(g4 + s * 32), y = a4[s * 32], z = w4[s * 32];
+        const float4 x = __ldcs(g4 + s * 32), y = __ldcs(a4 + s * 32), z = w4[s * 32];
         gv[s][0] = x.x; gv[s][1] = x.y; gv[s][2] = x.z; gv[s][3] = x.w;
         av[s][0] = y.x; av[s][1] = y.y; av[s][2] = y.z; av[s][3] = y.w;
         den[s][0] = z.x; den[s][1] = z.y; den[s][2] = z.z; den[s][3] = z.w;
@@ -382,7 +442,7 @@ __global__ void __launch_bounds__(THREADS)
       for (int s = 0; s < ROUNDS; ++s) {
         const uint64_t e0 = first + s * 128;
         load4_stream<VEC>(g, e0, lo, hi, gv[s]);
-        load4<VEC>(a, e0, lo, hi, av[s]);
+        load4_stream<VEC>(a, e0, lo, hi, av[s]);
         load4<VEC>(weights, e0, lo, hi, den[s]);
 #pragma unroll
         for (int c = 0; c < 4; ++c) inrange |= (e0 + c >= lo && e0 + c < hi) ? (1u << (4 * s + c)) : 0u;
@@ -398,49 +458,61 @@ __global__ void __launch_bounds__(THREADS)
         m |= (fabsf(av[s][c]) >= __fmul_rn(gm, den[s][c])) ? (1u << (4 * s + c)) : 0u;
       }
     }
+    // results: to HBM, and into shared memory so that the rare-path loops below can pick single
+    // elements by a run-time index without keeping all sixteen in registers
+#pragma unroll
+    for (int s = 0; s < ROUNDS; ++s)
+      *reinterpret_cast<float4*>(res + s * 128) = make_float4(av[s][0], av[s][1], av[s][2], av[s][3]);
     if (full) {
       float4* a4 = reinterpret_cast<float4*>(a + first);
 #pragma unroll
-      for (int s = 0; s < ROUNDS; ++s) a4[s * 32] = make_float4(av[s][0], av[s][1], av[s][2], av[s][3]);
-      if (w == 0) {
+      for (int s = 0; s < ROUNDS; ++s) __stcs(a4 + s * 32, make_float4(av[s][0], av[s][1], av[s][2], av[s][3]));
+      if (LEADER) {
         float4* u4 = reinterpret_cast<float4*>(update + first);
 #pragma unroll
-        for (int s = 0; s < ROUNDS; ++s) u4[s * 32] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s = 0; s < ROUNDS; ++s) __stcs(u4 + s * 32, make_float4(0.f, 0.f, 0.f, 0.f));
       }
     } else {
 #pragma unroll
       for (int s = 0; s < ROUNDS; ++s) {
         store4<VEC>(a, first + s * 128, lo, hi, av[s]);
-        if (w == 0) store4<VEC>(update, first + s * 128, lo, hi, zero);
+        if (LEADER) store4<VEC>(update, first + s * 128, lo, hi, zero);
       }
     }
     m &= inrange;
-    if (__any_sync(0xffffffffu, m != 0u)) {
-      // queue position in index order (round, lane, component): per-round counts packed 8 bits each
+
+    if (!LEADER) {  // this worker's value at every position of the leader's slot (step (e) without a gather)
+      const uint32_t mL = ll.x & 0xFFFFu, countL = ll.x >> 16;
+      for (uint32_t mm = mL; mm; mm &= mm - 1) {
+        const uint32_t b = __ffs(mm) - 1;
+        const uint32_t pos = countL + staged_position(mL, ll.y, lt, b);
+        if (pos < CAND_CAP) side_val[slot + pos] = res[(b >> 2) * 128 + (b & 3u)];
+      }
+    }
+
+    const bool any = __any_sync(0xffffffffu, m != 0u);
+    uint32_t excl = 0, tot = 0;
+    if (any) {  // queue position in index order: per-round counts packed 8 bits each (<= 128 per round)
       uint32_t packed = 0;
 #pragma unroll
       for (int s = 0; s < ROUNDS; ++s) packed |= static_cast<uint32_t>(__popc((m >> (4 * s)) & 0xFu)) << (8 * s);
       const uint32_t incl = warp_incl_scan(packed);
-      const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
-      const uint32_t excl = incl - packed;
-      const uint32_t loc0 = static_cast<uint32_t>(first - base);
-      uint32_t round_base = 0;
-      if (m) {
-#pragma unroll
-        for (int s = 0; s < ROUNDS; ++s) {
-          uint32_t pos = round_base + ((excl >> (8 * s)) & 0xFFu);
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            if ((m >> (4 * s + c)) & 1u) {
-              if (pos < EMIT_QUEUE) {
-                qv[pos] = av[s][c];
-                qd[pos] = den[s][c];
-                ql[pos] = static_cast<uint16_t>(loc0 + s * 128 + c);
-              }
-              ++pos;
-            }
-          }
-          round_base += (tot >> (8 * s)) & 0xFFu;
+      tot = __shfl_sync(0xffffffffu, incl, 31);
+      excl = incl - packed;
+    }
+    if (LEADER) {
+      lead_lane[sigma * 32 + lane] = make_uint2(m | (count << 16), excl);
+      if (lane == 0) lead_tot[sigma] = tot;
+    }
+    if (any) {
+      for (uint32_t mm = m; mm; mm &= mm - 1) {
+        const uint32_t b = __ffs(mm) - 1;
+        const uint32_t pos = staged_position(m, excl, tot, b);
+        if (pos < EMIT_QUEUE) {
+          const uint32_t off = (b >> 2) * 128 + (b & 3u);
+          qv[pos] = res[off];
+          qd[pos] = imp_den(weights[first + off], eps);  // re-read through L1: only staged elements get here
+          ql[pos] = static_cast<uint16_t>(static_cast<uint32_t>(first - base) + off);
         }
       }
       uint32_t nq = (tot & 0xFFu) + ((tot >> 8) & 0xFFu) + ((tot >> 16) & 0xFFu) + (tot >> 24);
@@ -476,6 +548,53 @@ __global__ void __launch_bounds__(THREADS)
   }
 }
 
+// The candidates of (chunk, worker): warp q takes the chunk's tiles 16 q .. 16 q + 15 (consecutive,
+// so that warp order is index order), four tiles at a time; each lane reads entries 4 lane .. 4 lane + 3
+// of a slot with one 128-bit load (a slot rarely holds more than 128 entries; a tail loop covers the
+// rest) and all loads of a batch are issued before any is used.  `f(key)` sees every stored candidate.
+constexpr uint32_t TILES_PER_WARP = CHUNK_TILES / WARPS;
+
+template <typename F>
+__device__ __forceinline__ void for_each_candidate(const Chunk& c, int w, int W, const uint32_t* __restrict__ cand_cnt,
+                                                   const uint32_t* __restrict__ cand_key, F&& f) {
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t t_begin = warp * TILES_PER_WARP;
+  const uint32_t t_end = min(c.n_tiles, t_begin + TILES_PER_WARP);
+  for (uint32_t tb = t_begin; tb < t_end; tb += 4) {
+    uint32_t cnt[4];
+    uint4 k4[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      cnt[q] = (tb + q < t_end) ? min(cand_cnt[static_cast<uint64_t>(c.first_tile + tb + q) * W + w], CAND_CAP) : 0u;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (static_cast<uint64_t>(c.first_tile + tb + q) * W + w) * CAND_CAP);
+      k4[q] = (lane * 4 < cnt[q]) ? kp[lane] : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t j = lane * 4;
+      if (j + 0 < cnt[q]) f(k4[q].x);
+      if (j + 1 < cnt[q]) f(k4[q].y);
+      if (j + 2 < cnt[q]) f(k4[q].z);
+      if (j + 3 < cnt[q]) f(k4[q].w);
+      if (cnt[q] > 128) {
+        const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (static_cast<uint64_t>(c.first_tile + tb + q) * W + w) * CAND_CAP);
+        for (uint32_t j0 = 128; j0 < cnt[q]; j0 += 128) {
+          j = j0 + lane * 4;
+          if (j < cnt[q]) {
+            const uint4 k = kp[j >> 2];
+            f(k.x);
+            if (j + 1 < cnt[q]) f(k.y);
+            if (j + 2 < cnt[q]) f(k.z);
+            if (j + 3 < cnt[q]) f(k.w);
+          }
+        }
+      }
+    }
+  }
+}
+
 // ---------------------------------------------------------------------------------------
 // tiled path, step (c): exact radix select of the k-th largest key per (worker, layer).
 // Every kernel below serves both kinds of pair: those whose candidates hold the top-k read the
@@ -501,18 +620,9 @@ __global__ void __launch_bounds__(THREADS)
   for (int b = threadIdx.x; b < nb; b += THREADS) sh[b] = 0;
   __syncthreads();
   if (pair_is_cand(info[pair], L.k)) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (uint32_t ti = warp; ti < c.n_tiles; ti += WARPS) {
-      const uint64_t tw = static_cast<uint64_t>(c.first_tile + ti) * W + w;
-      const uint32_t cnt = min(cand_cnt[tw], CAND_CAP);
-      const uint32_t* kp = cand_key + tw * CAND_CAP;
-      for (uint32_t j0 = 0; j0 < cnt; j0 += 32) {
-        const uint32_t j = j0 + lane;
-        const uint32_t key = j < cnt ? kp[j] : 0u;
-        const bool valid = j < cnt && (key >> prev_shift) == want;
-        hist_add_aggregated(sh, valid, (key >> shift) & (nb - 1));
-      }
-    }
+    for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
+      if ((key >> prev_shift) == want) atomicAdd(&sh[(key >> shift) & (nb - 1)], 1u);
+    });
   } else {
     const uint64_t lo = c.a, hi = lo + c.len;
     const uint64_t s0 = lo & ~3ull;
@@ -594,17 +704,10 @@ __global__ void __launch_bounds__(THREADS)
   __syncthreads();
   uint32_t gt = 0, eq = 0;
   if (pair_is_cand(info[pair], L.k)) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (uint32_t ti = warp; ti < c.n_tiles; ti += WARPS) {
-      const uint64_t tw = static_cast<uint64_t>(c.first_tile + ti) * W + w;
-      const uint32_t cnt = min(cand_cnt[tw], CAND_CAP);
-      const uint32_t* kp = cand_key + tw * CAND_CAP;
-      for (uint32_t j = lane; j < cnt; j += 32) {
-        const uint32_t key = kp[j];
-        gt += key > T ? 1u : 0u;
-        eq += key == T ? 1u : 0u;
-      }
-    }
+    for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
+      gt += key > T ? 1u : 0u;
+      eq += key == T ? 1u : 0u;
+    });
   } else {
     const uint64_t lo = c.a, hi = lo + c.len;
     const uint64_t s0 = lo & ~3ull;
@@ -649,11 +752,10 @@ __global__ void __launch_bounds__(THREADS)
             const uint32_t* __restrict__ cand_key, const float* __restrict__ cand_val,
             const uint16_t* __restrict__ cand_idx, const uint32_t* __restrict__ cand_cnt,
             const uint2* __restrict__ state, const uint2* __restrict__ chunk_cnt, uint32_t* __restrict__ sel_idx,
-            float* __restrict__ sel_val, int* __restrict__ status, float eps, uint64_t N, uint64_t K, int W,
-            uint32_t n_chunks) {
+            float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot, int* __restrict__ status, float eps,
+            uint64_t N, uint64_t K, int W, uint32_t n_chunks, int leader) {
   __shared__ uint32_t sh_warp[WARPS];
   __shared__ uint32_t sh_base[2];
-  __shared__ uint32_t sh_pre[CHUNK_TILES + 1];
   const Chunk c = chunks[blockIdx.x];
   const int w = blockIdx.y;
   const LayerDesc L = layers[c.layer];
@@ -686,47 +788,78 @@ __global__ void __launch_bounds__(THREADS)
   uint32_t* out_i = sel_idx + static_cast<uint64_t>(w) * K + L.koff;
   float* out_v = sel_val + static_cast<uint64_t>(w) * K + L.koff;
 
+  const bool is_leader = w == leader;
   if (pair_is_cand(info[pair], L.k)) {
-    // the chunk's candidates, tile after tile, form one index-ordered sequence
-    uint32_t total;
-    {
-      static_assert(CHUNK_TILES <= THREADS, "one thread per tile count");
-      const uint32_t ti = threadIdx.x;
-      const uint32_t cnt = ti < c.n_tiles ? min(cand_cnt[static_cast<uint64_t>(c.first_tile + ti) * W + w], CAND_CAP) : 0u;
-      const uint32_t ex = block_excl_scan(cnt, sh_warp, total);
-      if (ti <= c.n_tiles && ti <= CHUNK_TILES) sh_pre[ti] = ex;  // sh_pre[n_tiles] = total
-      __syncthreads();
+    // warp order is index order: count per warp, prefix over the warps, then every warp writes its
+    // tiles front to back, ranking the entries of a slot with one warp scan per 128 entries
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t my_gt = 0, my_eq = 0;
+    for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
+      my_gt += key > T ? 1u : 0u;
+      my_eq += key == T ? 1u : 0u;
+    });
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      my_gt += __shfl_xor_sync(0xffffffffu, my_gt, d);
+      my_eq += __shfl_xor_sync(0xffffffffu, my_eq, d);
     }
-    for (uint32_t j0 = 0; j0 < total; j0 += THREADS) {
-      const uint32_t j = j0 + threadIdx.x;
-      const bool valid = j < total;
-      uint32_t key = 0, tile = 0;
-      uint64_t slot = 0;
-      if (valid) {
-        uint32_t a = 0, b = c.n_tiles;  // largest tile index with sh_pre[tile] <= j
-        while (b - a > 1) {
-          const uint32_t mid = (a + b) >> 1;
-          if (sh_pre[mid] <= j) a = mid; else b = mid;
+    __shared__ uint32_t sh_wg[WARPS], sh_we[WARPS];
+    if (lane == 0) {
+      sh_wg[warp] = my_gt;
+      sh_we[warp] = my_eq;
+    }
+    __syncthreads();
+    uint32_t g_before = run_gt, q_before = run_eq;
+    for (uint32_t q = 0; q < warp; ++q) {
+      g_before += sh_wg[q];
+      q_before += sh_we[q];
+    }
+    if ((my_gt | my_eq) == 0) return;  // nothing of this warp's tiles is selected
+    const uint32_t t_begin = warp * TILES_PER_WARP;
+    const uint32_t t_end = min(c.n_tiles, t_begin + TILES_PER_WARP);
+    for (uint32_t ti = t_begin; ti < t_end; ++ti) {
+      const uint32_t tile = c.first_tile + ti;
+      const uint64_t tw = static_cast<uint64_t>(tile) * W + w;
+      const uint32_t cnt = min(cand_cnt[tw], CAND_CAP);
+      const uint32_t tile_base = tiles[tile].a & ~(TILE - 1u);
+      for (uint32_t j0 = 0; j0 < cnt; j0 += 128) {
+        const uint32_t j = j0 + lane * 4;
+        uint4 k = make_uint4(0u, 0u, 0u, 0u);
+        if (j < cnt) k = reinterpret_cast<const uint4*>(cand_key + tw * CAND_CAP)[j >> 2];
+        const uint32_t kk[4] = {k.x, k.y, k.z, k.w};
+        uint32_t fg = 0, fe = 0;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const bool in = j + u < cnt;
+          fg |= (in && kk[u] > T) ? (1u << u) : 0u;
+          fe |= (in && kk[u] == T) ? (1u << u) : 0u;
         }
-        tile = c.first_tile + a;
-        slot = (static_cast<uint64_t>(tile) * W + w) * CAND_CAP + (j - sh_pre[a]);
-        key = cand_key[slot];
-      }
-      const bool isg = valid && key > T, ise = valid && key == T;
-      uint32_t tot;
-      const uint32_t ex = block_excl_scan((isg ? 1u : 0u) | (ise ? 1u << 16 : 0u), sh_warp, tot);
-      const uint32_t g_before = run_gt + (ex & 0xffffu), q_before = run_eq + (ex >> 16);
-      if (isg || (ise && q_before < r)) {
-        const uint32_t pos = g_before + (q_before < r ? q_before : r);
-        if (pos < L.k) {
-          out_i[pos] = (tiles[tile].a & ~(TILE - 1u)) + cand_idx[slot];
-          out_v[pos] = cand_val[slot];
-        } else {
-          atomicMin(status, STATUS_INTERNAL);
+        const uint32_t packed = static_cast<uint32_t>(__popc(fg)) | (static_cast<uint32_t>(__popc(fe)) << 16);
+        const uint32_t incl = warp_incl_scan(packed);
+        const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
+        uint32_t gb = g_before + ((incl - packed) & 0xffffu), qb = q_before + ((incl - packed) >> 16);
+        if (fg | fe) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const bool isg = (fg >> u) & 1u, ise = (fe >> u) & 1u;
+            if (isg || (ise && qb < r)) {
+              const uint32_t pos = gb + (qb < r ? qb : r);
+              if (pos < L.k) {
+                const uint64_t at = tw * CAND_CAP + j + u;
+                out_i[pos] = tile_base + cand_idx[at];
+                out_v[pos] = cand_val[at];
+                if (is_leader) sel_slot[L.koff + pos] = tile * CAND_CAP + j + u;
+              } else {
+                atomicMin(status, STATUS_INTERNAL);
+              }
+            }
+            gb += isg ? 1u : 0u;
+            qb += ise ? 1u : 0u;
+          }
         }
+        g_before += tot & 0xffffu;
+        q_before += tot >> 16;
       }
-      run_gt += tot & 0xffffu;
-      run_eq += tot >> 16;
     }
     return;
   }
@@ -762,6 +895,7 @@ __global__ void __launch_bounds__(THREADS)
           if (pos < L.k) {
             out_i[pos] = static_cast<uint32_t>(e0 + q);
             out_v[pos] = av[q];
+            if (is_leader) sel_slot[L.koff + pos] = REF_NONE;
           } else {
             atomicMin(status, STATUS_INTERNAL);
           }
@@ -782,8 +916,8 @@ __global__ void __launch_bounds__(THREADS)
 __global__ void __launch_bounds__(THREADS)
     k_small(const float* __restrict__ grads, const float* __restrict__ weights, float* __restrict__ acc,
             float* __restrict__ update, const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ small_ids,
-            uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val, int* __restrict__ status, float eps,
-            uint64_t N, uint64_t K) {
+            uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot,
+            int* __restrict__ status, float eps, uint64_t N, uint64_t K, int leader) {
   extern __shared__ uint32_t keys[];
   __shared__ uint32_t hist[NBINS];
   __shared__ uint32_t sh_scan[THREADS];
@@ -823,6 +957,7 @@ __global__ void __launch_bounds__(THREADS)
       if (pos < L.k) {
         out_i[pos] = L.off + i;
         out_v[pos] = a[i];
+        if (w == leader) sel_slot[L.koff + pos] = REF_NONE;
       } else {
         atomicMin(status, STATUS_INTERNAL);
       }
@@ -851,6 +986,53 @@ __global__ void __launch_bounds__(THREADS)
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
+    }
+  }
+  for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
+  update[i] = __fadd_rn(0.0f, s);
+}
+
+// Steps (e)-(g) on the single-read path.  For a list entry of the leader that came from a candidate
+// slot, every other worker's value at that slot position was written to the side buffer by the
+// streaming pass (the leader's own value is the candidate value): read the W values, sum them in
+// ascending worker order, scatter.  Entries from the one-CTA path or from a pair that fell back to
+// the multi-pass select carry REF_NONE and are gathered from the residuals.  Either way the sent
+// residuals are zeroed.
+__global__ void __launch_bounds__(THREADS)
+    k_sum_scatter(const uint32_t* __restrict__ leader_idx, const uint32_t* __restrict__ sel_slot,
+                  const float* __restrict__ side_val, const float* __restrict__ cand_val, float* __restrict__ acc,
+                  float* __restrict__ update, uint64_t N, uint64_t K, int W, int leader) {
+  const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (j >= K) return;
+  const uint64_t i = leader_idx[j];
+  const uint32_t ref = sel_slot[j];
+  float* p = acc + i;
+  float s = 0.0f;
+  if (ref != REF_NONE) {
+    const uint64_t tile = ref / CAND_CAP, at = ref % CAND_CAP;
+    const uint64_t q0 = tile * W * CAND_CAP + at;
+    for (int w0 = 0; w0 < W; w0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int w = w0 + u;
+        const uint64_t q = q0 + static_cast<uint64_t>(w) * CAND_CAP;
+        v[u] = (w < W) ? (w == leader ? cand_val[q] : side_val[q]) : 0.0f;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
+      }
+    }
+  } else {
+    for (int w0 = 0; w0 < W; w0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = (w0 + u < W) ? p[static_cast<uint64_t>(w0 + u) * N] : 0.0f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
+      }
     }
   }
   for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;

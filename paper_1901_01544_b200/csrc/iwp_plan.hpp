@@ -22,6 +22,9 @@ constexpr uint32_t NBINS = 2048;
 constexpr uint32_t CAND_CAP = 512;
 constexpr uint32_t SAMPLE_MAX = 16384;
 constexpr uint32_t GUESS_NONE = 0xffffffffu;  // no importance pattern reaches this value
+constexpr uint32_t SEG_ELEMS = 512;           // elements a warp handles per iteration of the streaming pass
+constexpr uint32_t SEGS_PER_TILE = TILE / SEG_ELEMS;
+constexpr uint32_t REF_NONE = 0xffffffffu;    // list entry has no side values: gather from the residuals
 
 struct LayerDesc {
   uint32_t off;         // flat offset of the first element
