@@ -45,6 +45,9 @@ struct iwp_ctx {
   uint32_t* sel_slot = nullptr;   // [K] slot position of each entry of the leader's list, or REF_NONE
   uint2* lead_lane = nullptr;     // [segment][32] the leader's staged mask | count << 16, lane prefix
   uint32_t* lead_tot = nullptr;   // [segment] the leader's per-round totals
+  uint32_t* zmask = nullptr;      // residuals sent in the last step and not yet zeroed (lazy step (g))
+  uint64_t zmask_words = 0;
+  bool zero_pending = false;      // zmask may hold marks
   uint32_t* cand_key = nullptr;   // candidate slots [tile][worker][CAND_CAP]
   float* cand_val = nullptr;
   uint16_t* cand_idx = nullptr;
@@ -89,11 +92,11 @@ void stage_clear(iwp_ctx* c) {
 
 struct Sizes {
   uint64_t acc, layers, tiles, chunks, small_ids, large_ids, state, hist, chunk_cnt, sel_idx, sel_val, status;
-  uint64_t info, cand_key, cand_val, cand_idx, cand_cnt, guess, side_val, sel_slot, lead_lane, lead_tot;
+  uint64_t info, cand_key, cand_val, cand_idx, cand_cnt, guess, side_val, sel_slot, lead_lane, lead_tot, zmask;
   uint64_t total() const {
     return acc + layers + tiles + chunks + small_ids + large_ids + state + hist + chunk_cnt + sel_idx + sel_val +
            status + info + cand_key + cand_val + cand_idx + cand_cnt + guess + side_val + sel_slot + lead_lane +
-           lead_tot;
+           lead_tot + zmask;
   }
 };
 
@@ -129,6 +132,7 @@ Sizes sizes_of(const Plan& p) {
   s.sel_slot = at_least(p.K * sizeof(uint32_t));
   s.lead_lane = at_least(segs * 32 * sizeof(uint2));
   s.lead_tot = at_least(segs * sizeof(uint32_t));
+  s.zmask = ((p.N >> 9) + 2) * 16 * sizeof(uint32_t);  // 32 sixteen-bit fields per 512 elements
   return s;
 }
 
@@ -168,6 +172,7 @@ void free_all(iwp_ctx* c) {
   cudaFree(c->sel_slot);
   cudaFree(c->lead_lane);
   cudaFree(c->lead_tot);
+  cudaFree(c->zmask);
   cudaFree(c->sel_idx);
   cudaFree(c->sel_val);
   cudaFree(c->d_status);
@@ -183,6 +188,18 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
     (c)->launches += 1;                             \
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA; \
   } while (0)
+
+// Brings the residuals themselves up to date when the last step left its zeroing to the next
+// streaming pass (see k_sum_scatter) and somebody else is about to look at them.
+int flush_pending_zero(iwp_ctx* c) {
+  if (!c->zero_pending) return IWP_OK;
+  const unsigned blocks = static_cast<unsigned>((c->zmask_words + THREADS - 1) / THREADS);
+  k_flush_zmask<<<blocks, THREADS, 0, c->stream>>>(c->zmask, c->acc, c->zmask_words, c->plan.N, c->plan.W);
+  c->launches += 1;
+  if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+  c->zero_pending = false;
+  return IWP_OK;
+}
 
 template <bool VEC>
 int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update, int32_t leader) {
@@ -201,6 +218,10 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   stage_mark(c);
   const bool tiled = !p.large_layers.empty();
   const bool spec = tiled && c->speculate && c->spec_pairs > 0;
+  if (!spec) {  // the multi-pass path reads the residuals as they are
+    const int rc = flush_pending_zero(c);
+    if (rc != IWP_OK) return rc;
+  }
   if (tiled && !spec && !c->info_clean) {  // speculation was switched off: forget the old guesses
     if (cudaMemsetAsync(c->d_info, 0xff, static_cast<size_t>(c->n_pairs) * sizeof(PairInfo), s) != cudaSuccess) {
       cudaGetLastError();
@@ -211,8 +232,8 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   }
   if (spec) {
     const size_t dyn = static_cast<size_t>(c->max_sample) * sizeof(uint32_t);
-    k_sample<<<c->n_pairs, THREADS, dyn, s>>>(grads, weights, c->acc, c->d_layers, c->d_large_ids, c->d_info,
-                                             c->d_guess, c->eps, N, W, static_cast<uint32_t>(c->t));
+    k_sample<<<c->n_pairs, SAMPLE_THREADS, dyn, s>>>(grads, weights, c->acc, c->d_layers, c->d_large_ids, c->d_info,
+                                             c->d_guess, c->zmask, c->eps, N, W, static_cast<uint32_t>(c->t));
     IWP_LAUNCH_CHECK(c);
     c->info_clean = false;
   }
@@ -223,13 +244,22 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
       // the leader's workers first (records where its candidates sit), then everybody else
       k_stream<VEC, true><<<(n_tiles + WARPS - 1) / WARPS, THREADS, 0, s>>>(
           grads, weights, c->acc, update, c->d_tiles, c->d_info, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
-          c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->eps, N, W, leader, n_tiles, 1);
+          c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, 1);
       if (W > 1) {
         IWP_LAUNCH_CHECK(c);
-        const int groups = (W - 1 + WARPS - 1) / WARPS;
-        k_stream<VEC, false><<<n_tiles * static_cast<unsigned>(groups), THREADS, 0, s>>>(
+        const int wpc = (W - 1 < WARPS) ? W - 1 : WARPS;  // warps (= workers) per CTA
+        const int groups = (W - 1 + wpc - 1) / wpc;
+        k_stream<VEC, false><<<n_tiles * static_cast<unsigned>(groups), wpc * 32, 0, s>>>(
             grads, weights, c->acc, update, c->d_tiles, c->d_info, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
-            c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->eps, N, W, leader, n_tiles, groups);
+            c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, groups);
+      }
+      if (c->zero_pending) {  // every marked residual has now been overwritten: forget the marks
+        IWP_LAUNCH_CHECK(c);
+        if (cudaMemsetAsync(c->zmask, 0, c->zmask_words * sizeof(uint32_t), s) != cudaSuccess) {
+          cudaGetLastError();
+          return IWP_ERR_CUDA;
+        }
+        c->zero_pending = false;
       }
     } else {
       k_accumulate<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, N, W);
@@ -266,7 +296,8 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   const unsigned gblocks = static_cast<unsigned>((K + THREADS - 1) / THREADS);
   if (spec) {
     k_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->sel_slot, c->side_val,
-                                              c->cand_val, c->acc, update, N, K, W, leader);
+                                              c->cand_val, c->acc, update, c->zmask, N, K, W, leader);
+    c->zero_pending = true;
   } else {
     k_gather_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->acc, update,
                                                      N, K, W);
@@ -362,6 +393,7 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
   A(&c->sel_slot, sz.sel_slot);
   A(&c->lead_lane, sz.lead_lane);
   A(&c->lead_tot, sz.lead_tot);
+  A(&c->zmask, sz.zmask);
   A(&c->sel_idx, sz.sel_idx);
   A(&c->sel_val, sz.sel_val);
   A(&c->d_status, sz.status);
@@ -389,6 +421,8 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
   ok = ok && cudaMemset(c->d_info, 0xff, sz.info) == cudaSuccess;  // guess = none, overflow flag set
   ok = ok && cudaMemset(c->cand_cnt, 0, sz.cand_cnt) == cudaSuccess;
   ok = ok && cudaMemset(c->sel_slot, 0xff, sz.sel_slot) == cudaSuccess;
+  ok = ok && cudaMemset(c->zmask, 0, sz.zmask) == cudaSuccess;
+  c->zmask_words = sz.zmask / sizeof(uint32_t);
   for (uint32_t l : p.large_layers) {
     if (p.layers[l].sample > c->max_sample) c->max_sample = p.layers[l].sample;
     if (p.layers[l].sample) c->spec_pairs += static_cast<uint32_t>(W);
@@ -521,6 +555,7 @@ int iwp_get_leader(iwp_ctx* c, int32_t* leader) {
 
 int iwp_get_residual(iwp_ctx* c, int32_t w, float* dst) {
   if (!c || !dst || w < 0 || w >= c->plan.W) return IWP_ERR_INVALID;
+  if (const int rc = flush_pending_zero(c)) return rc;
   const uint64_t N = c->plan.N;
   if (cudaMemcpyAsync(dst, c->acc + static_cast<uint64_t>(w) * N, N * sizeof(float), cudaMemcpyDeviceToDevice,
                       c->stream) != cudaSuccess) {
@@ -532,6 +567,7 @@ int iwp_get_residual(iwp_ctx* c, int32_t w, float* dst) {
 
 int iwp_set_residual(iwp_ctx* c, int32_t w, const float* src) {
   if (!c || !src || w < 0 || w >= c->plan.W) return IWP_ERR_INVALID;
+  if (const int rc = flush_pending_zero(c)) return rc;
   const uint64_t N = c->plan.N;
   if (cudaMemcpyAsync(c->acc + static_cast<uint64_t>(w) * N, src, N * sizeof(float), cudaMemcpyDeviceToDevice,
                       c->stream) != cudaSuccess) {
@@ -576,6 +612,8 @@ int iwp_reset(iwp_ctx* c) {
   if (!c) return IWP_ERR_INVALID;
   const Sizes sz = sizes_of(c->plan);
   bool ok = cudaMemsetAsync(c->acc, 0, sz.acc, c->stream) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->zmask, 0, sz.zmask, c->stream) == cudaSuccess;
+  c->zero_pending = false;
   ok = ok && cudaMemsetAsync(c->d_hist, 0, sz.hist, c->stream) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->d_status, 0, sz.status, c->stream) == cudaSuccess;
   if (!ok) {

@@ -137,17 +137,18 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t x, uint32_t* sh_war
 // Radix-select digit step on a histogram in shared memory: finds the digit d with
 //   count(digit > d) < krem <= count(digit >= d)
 // res[0] = d, res[1] = krem - count(digit > d), res[2] = 1 if found.  sh_scan: THREADS words.
+template <int NT = THREADS>
 __device__ __forceinline__ void find_digit(const uint32_t* hist, int nb, uint32_t krem, uint32_t* sh_scan,
                                            uint32_t* res) {
   const int tid = threadIdx.x;
-  const int per = nb / THREADS;
+  const int per = nb / NT;
   uint32_t local = 0;
   for (int b = 0; b < per; ++b) local += hist[tid * per + b];
   sh_scan[tid] = local;
   if (tid == 0) res[2] = 0;
   __syncthreads();
-  for (int d = 1; d < THREADS; d <<= 1) {  // inclusive suffix sum over threads
-    const uint32_t v = (tid + d < THREADS) ? sh_scan[tid + d] : 0u;
+  for (int d = 1; d < NT; d <<= 1) {  // inclusive suffix sum over threads
+    const uint32_t v = (tid + d < NT) ? sh_scan[tid + d] : 0u;
     __syncthreads();
     sh_scan[tid] += v;
     __syncthreads();
@@ -172,8 +173,9 @@ __device__ __forceinline__ void find_digit(const uint32_t* hist, int nb, uint32_
 
 // Exact radix select on keys held in shared memory: the krem-th largest of n keys.
 // On success T = that key and r = how many T-valued keys belong to the top krem.
-// hist: NBINS words, sh_scan: THREADS words, res: 4 words.  Returns false if the counts are
-// inconsistent (krem > n).  All threads of the block must call it.
+// hist: NBINS words, sh_scan: NT words, res: 4 words.  Returns false if the counts are
+// inconsistent (krem > n).  All NT threads of the block must call it.
+template <int NT = THREADS>
 __device__ __forceinline__ bool smem_radix_select(const uint32_t* keys, uint32_t n, uint32_t krem, uint32_t* hist,
                                                   uint32_t* sh_scan, uint32_t* res, uint32_t& T, uint32_t& r) {
   const int tid = threadIdx.x;
@@ -183,14 +185,14 @@ __device__ __forceinline__ bool smem_radix_select(const uint32_t* keys, uint32_t
     const int shift = pass_shift(pass), nb = pass_bins(pass);
     const int prev_shift = pass == 0 ? 31 : pass_shift(pass - 1);
     const uint32_t want = prefix >> prev_shift;
-    for (int b = tid; b < nb; b += THREADS) hist[b] = 0;
+    for (int b = tid; b < nb; b += NT) hist[b] = 0;
     __syncthreads();
-    for (uint32_t i = tid; i < n; i += THREADS) {
+    for (uint32_t i = tid; i < n; i += NT) {
       const uint32_t key = keys[i];
       if ((key >> prev_shift) == want) atomicAdd(&hist[(key >> shift) & (nb - 1)], 1u);
     }
     __syncthreads();
-    find_digit(hist, nb, krem, sh_scan, res);
+    find_digit<NT>(hist, nb, krem, sh_scan, res);
     const bool found = res[2] != 0;
     const uint32_t d = res[0], kr = res[1];
     __syncthreads();
@@ -256,18 +258,34 @@ __global__ void __launch_bounds__(THREADS) k_accumulate(const float* __restrict_
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ float pretest_multiplier(uint32_t guess, float eps);
 
+// Lazy zeroing of sent residuals (step (g)): instead of scattering W * K four-byte zeros, the
+// reduction marks each sent element in a bit mask and the NEXT streaming pass, which reads every
+// residual anyway, takes a marked residual as +0.  Layout: one 16-bit field per (512-element
+// segment of the flat element space, lane), bit 4 * round + component - exactly the sixteen
+// elements a lane of the streaming pass owns - two fields per 32-bit word.
+__device__ __forceinline__ uint64_t zmask_word(uint64_t i) { return ((i >> 9) * 32 + ((i & 127) >> 2)) >> 1; }
+__device__ __forceinline__ uint32_t zmask_bit(uint64_t i) {
+  return 1u << ((((i & 127) >> 2) & 1) * 16 + ((i >> 7) & 3) * 4 + (i & 3));
+}
+__device__ __forceinline__ bool zmask_test(const uint32_t* __restrict__ zmask, uint64_t i) {
+  return (zmask[zmask_word(i)] & zmask_bit(i)) != 0u;
+}
+
 __device__ __forceinline__ uint32_t hash32(uint32_t x) {
   x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
   return x;
 }
 
-__global__ void __launch_bounds__(THREADS)
+constexpr int SAMPLE_THREADS = 1024;
+
+__global__ void __launch_bounds__(SAMPLE_THREADS)
     k_sample(const float* __restrict__ grads, const float* __restrict__ weights, const float* __restrict__ acc,
              const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ large_ids, PairInfo* __restrict__ info,
-             uint2* __restrict__ guess_tab, float eps, uint64_t N, int W, uint32_t step) {
+             uint2* __restrict__ guess_tab, const uint32_t* __restrict__ zmask, float eps, uint64_t N, int W,
+             uint32_t step) {
   extern __shared__ uint32_t keys[];
   __shared__ uint32_t hist[NBINS];
-  __shared__ uint32_t sh_scan[THREADS];
+  __shared__ uint32_t sh_scan[SAMPLE_THREADS];
   __shared__ uint32_t res[4];
   const uint32_t pair = blockIdx.x;
   const LayerDesc L = layers[large_ids[pair / W]];
@@ -287,31 +305,33 @@ __global__ void __launch_bounds__(THREADS)
   const float* g = grads + static_cast<uint64_t>(w) * N + L.off;
   const float* wt = weights + L.off;
   // eight samples per thread and trip, all loads issued before any use (memory-level parallelism)
-  for (uint32_t i0 = 0; i0 < s; i0 += THREADS * 8) {
+  for (uint32_t i0 = 0; i0 < s; i0 += SAMPLE_THREADS * 8) {
     float av[8], gv[8], wv[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const uint32_t i = i0 + u * THREADS + threadIdx.x;
+      const uint32_t i = i0 + u * SAMPLE_THREADS + threadIdx.x;
       av[u] = gv[u] = 0.f;
       wv[u] = 1.f;
       if (i < s) {
         const uint32_t grp = i >> 3;
         const uint32_t jit = hash32(step * 0x9E3779B9u + pair * 0x85EBCA6Bu + grp * 0xC2B2AE35u + 1u) % (stride - 7u);
         const uint32_t pos = grp * stride + jit + (i & 7u);
-        av[u] = a[pos];
+        const float av_raw = a[pos];
+        const bool sent = zmask_test(zmask, static_cast<uint64_t>(L.off) + pos);  // sent last step: counts as +0
+        av[u] = sent ? 0.0f : av_raw;
         gv[u] = g[pos];
         wv[u] = wt[pos];
       }
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const uint32_t i = i0 + u * THREADS + threadIdx.x;
+      const uint32_t i = i0 + u * SAMPLE_THREADS + threadIdx.x;
       if (i < s) keys[i] = imp_key(__fadd_rn(av[u], gv[u]), wv[u], eps);
     }
   }
   __syncthreads();
   uint32_t T, r;
-  const bool ok = smem_radix_select(keys, s, L.rho, hist, sh_scan, res, T, r);
+  const bool ok = smem_radix_select<SAMPLE_THREADS>(keys, s, L.rho, hist, sh_scan, res, T, r);
   if (threadIdx.x == 0) {
     const uint32_t guess = (ok && T != 0u) ? T : GUESS_NONE;
     const uint32_t gm = __float_as_uint(pretest_multiplier(guess, eps));
@@ -367,13 +387,13 @@ __device__ __forceinline__ uint32_t staged_position(uint32_t mask, uint32_t ex, 
 }
 
 template <bool VEC, bool LEADER>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 3)
     k_stream(const float* __restrict__ grads, const float* __restrict__ weights, float* __restrict__ acc,
              float* __restrict__ update, const Tile* __restrict__ tiles, PairInfo* __restrict__ info,
              const uint2* __restrict__ guess_tab, uint32_t* __restrict__ cand_key, float* __restrict__ cand_val,
              uint16_t* __restrict__ cand_idx, uint32_t* __restrict__ cand_cnt, float* __restrict__ side_val,
-             uint2* __restrict__ lead_lane, uint32_t* __restrict__ lead_tot, float eps, uint64_t N, int W, int leader,
-             uint32_t n_tiles, int worker_groups) {
+             uint2* __restrict__ lead_lane, uint32_t* __restrict__ lead_tot, const uint32_t* __restrict__ zmask,
+             float eps, uint64_t N, int W, int leader, uint32_t n_tiles, int worker_groups) {
   constexpr int ROUNDS = SEG_ELEMS / 128;  // 128-bit slots per lane and iteration = 4
   __shared__ float q_val[WARPS][EMIT_QUEUE];
   __shared__ float q_den[WARPS][EMIT_QUEUE];
@@ -388,7 +408,7 @@ __global__ void __launch_bounds__(THREADS)
     if (tile_id >= n_tiles) return;
   } else {  // up to eight of the other workers of one tile per CTA: the tile's weights come through L1
     tile_id = blockIdx.x / worker_groups;
-    const int wi = static_cast<int>(blockIdx.x % worker_groups) * WARPS + warp;
+    const int wi = static_cast<int>(blockIdx.x % worker_groups) * static_cast<int>(blockDim.x >> 5) + warp;
     if (wi >= W - 1) return;
     w = wi < leader ? wi : wi + 1;
   }
@@ -419,6 +439,8 @@ __global__ void __launch_bounds__(THREADS)
     const uint64_t sigma = static_cast<uint64_t>(tile_id) * SEGS_PER_TILE + it;  // global segment id
     float gv[ROUNDS][4], av[ROUNDS][4], den[ROUNDS][4];
     uint32_t inrange = 0xFFFFu;
+    // residuals sent in the previous step count as +0 (they are overwritten below either way)
+    const uint32_t zm = reinterpret_cast<const uint16_t*>(zmask)[(seg >> 9) * 32 + lane];
     uint2 ll = make_uint2(0u, 0u);
     uint32_t lt = 0;
     if (!LEADER) {  // the leader's record for this segment: (mask | count << 16, lane prefix), round totals
@@ -446,6 +468,13 @@ __global__ void __launch_bounds__(THREADS)
         load4<VEC>(weights, e0, lo, hi, den[s]);
 #pragma unroll
         for (int c = 0; c < 4; ++c) inrange |= (e0 + c >= lo && e0 + c < hi) ? (1u << (4 * s + c)) : 0u;
+      }
+    }
+    if (zm) {
+#pragma unroll
+      for (int s = 0; s < ROUNDS; ++s) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) av[s][c] = ((zm >> (4 * s + c)) & 1u) ? 0.0f : av[s][c];
       }
     }
     uint32_t m = 0;  // bit (4 s + c): passes the pre-test
@@ -817,48 +846,72 @@ __global__ void __launch_bounds__(THREADS)
     if ((my_gt | my_eq) == 0) return;  // nothing of this warp's tiles is selected
     const uint32_t t_begin = warp * TILES_PER_WARP;
     const uint32_t t_end = min(c.n_tiles, t_begin + TILES_PER_WARP);
-    for (uint32_t ti = t_begin; ti < t_end; ++ti) {
-      const uint32_t tile = c.first_tile + ti;
-      const uint64_t tw = static_cast<uint64_t>(tile) * W + w;
-      const uint32_t cnt = min(cand_cnt[tw], CAND_CAP);
-      const uint32_t tile_base = tiles[tile].a & ~(TILE - 1u);
-      for (uint32_t j0 = 0; j0 < cnt; j0 += 128) {
-        const uint32_t j = j0 + lane * 4;
-        uint4 k = make_uint4(0u, 0u, 0u, 0u);
-        if (j < cnt) k = reinterpret_cast<const uint4*>(cand_key + tw * CAND_CAP)[j >> 2];
-        const uint32_t kk[4] = {k.x, k.y, k.z, k.w};
-        uint32_t fg = 0, fe = 0;
+    // ranks the entries [j0, j0 + 128) of one slot with a warp scan and writes the selected ones
+    auto emit = [&](uint32_t tile, uint64_t tw, uint32_t cnt, uint32_t tile_base, uint32_t j0, uint4 k) {
+      const uint32_t j = j0 + lane * 4;
+      const uint32_t kk[4] = {k.x, k.y, k.z, k.w};
+      uint32_t fg = 0, fe = 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const bool in = j + u < cnt;
+        fg |= (in && kk[u] > T) ? (1u << u) : 0u;
+        fe |= (in && kk[u] == T) ? (1u << u) : 0u;
+      }
+      if (!__any_sync(0xffffffffu, (fg | fe) != 0u)) return;
+      const uint32_t packed = static_cast<uint32_t>(__popc(fg)) | (static_cast<uint32_t>(__popc(fe)) << 16);
+      const uint32_t incl = warp_incl_scan(packed);
+      const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
+      uint32_t gb = g_before + ((incl - packed) & 0xffffu), qb = q_before + ((incl - packed) >> 16);
+      if (fg | fe) {
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-          const bool in = j + u < cnt;
-          fg |= (in && kk[u] > T) ? (1u << u) : 0u;
-          fe |= (in && kk[u] == T) ? (1u << u) : 0u;
-        }
-        const uint32_t packed = static_cast<uint32_t>(__popc(fg)) | (static_cast<uint32_t>(__popc(fe)) << 16);
-        const uint32_t incl = warp_incl_scan(packed);
-        const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
-        uint32_t gb = g_before + ((incl - packed) & 0xffffu), qb = q_before + ((incl - packed) >> 16);
-        if (fg | fe) {
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const bool isg = (fg >> u) & 1u, ise = (fe >> u) & 1u;
-            if (isg || (ise && qb < r)) {
-              const uint32_t pos = gb + (qb < r ? qb : r);
-              if (pos < L.k) {
-                const uint64_t at = tw * CAND_CAP + j + u;
-                out_i[pos] = tile_base + cand_idx[at];
-                out_v[pos] = cand_val[at];
-                if (is_leader) sel_slot[L.koff + pos] = tile * CAND_CAP + j + u;
-              } else {
-                atomicMin(status, STATUS_INTERNAL);
-              }
+          const bool isg = (fg >> u) & 1u, ise = (fe >> u) & 1u;
+          if (isg || (ise && qb < r)) {
+            const uint32_t pos = gb + (qb < r ? qb : r);
+            if (pos < L.k) {
+              const uint64_t at = tw * CAND_CAP + j + u;
+              out_i[pos] = tile_base + cand_idx[at];
+              out_v[pos] = cand_val[at];
+              if (is_leader) sel_slot[L.koff + pos] = tile * CAND_CAP + j + u;
+            } else {
+              atomicMin(status, STATUS_INTERNAL);
             }
-            gb += isg ? 1u : 0u;
-            qb += ise ? 1u : 0u;
           }
+          gb += isg ? 1u : 0u;
+          qb += ise ? 1u : 0u;
         }
-        g_before += tot & 0xffffu;
-        q_before += tot >> 16;
+      }
+      g_before += tot & 0xffffu;
+      q_before += tot >> 16;
+    };
+    for (uint32_t tb = t_begin; tb < t_end; tb += 4) {  // four tiles per batch, all their loads first
+      uint32_t cnt[4], tbase[4];
+      uint4 k4[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const bool in = tb + q < t_end;
+        const uint32_t tile = c.first_tile + tb + q;
+        cnt[q] = in ? min(cand_cnt[static_cast<uint64_t>(tile) * W + w], CAND_CAP) : 0u;
+        tbase[q] = in ? (tiles[tile].a & ~(TILE - 1u)) : 0u;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint64_t tw = static_cast<uint64_t>(c.first_tile + tb + q) * W + w;
+        k4[q] = (lane * 4 < cnt[q]) ? reinterpret_cast<const uint4*>(cand_key + tw * CAND_CAP)[lane]
+                                    : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (cnt[q] == 0) continue;
+        const uint32_t tile = c.first_tile + tb + q;
+        const uint64_t tw = static_cast<uint64_t>(tile) * W + w;
+        emit(tile, tw, cnt[q], tbase[q], 0, k4[q]);
+        for (uint32_t j0 = 128; j0 < cnt[q]; j0 += 128) {
+          const uint32_t j = j0 + lane * 4;
+          const uint4 k = (j < cnt[q]) ? reinterpret_cast<const uint4*>(cand_key + tw * CAND_CAP)[j >> 2]
+                                       : make_uint4(0u, 0u, 0u, 0u);
+          emit(tile, tw, cnt[q], tbase[q], j0, k);
+        }
       }
     }
     return;
@@ -1001,12 +1054,12 @@ __global__ void __launch_bounds__(THREADS)
 __global__ void __launch_bounds__(THREADS)
     k_sum_scatter(const uint32_t* __restrict__ leader_idx, const uint32_t* __restrict__ sel_slot,
                   const float* __restrict__ side_val, const float* __restrict__ cand_val, float* __restrict__ acc,
-                  float* __restrict__ update, uint64_t N, uint64_t K, int W, int leader) {
+                  float* __restrict__ update, uint32_t* __restrict__ zmask, uint64_t N, uint64_t K, int W,
+                  int leader) {
   const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
   if (j >= K) return;
   const uint64_t i = leader_idx[j];
   const uint32_t ref = sel_slot[j];
-  float* p = acc + i;
   float s = 0.0f;
   if (ref != REF_NONE) {
     const uint64_t tile = ref / CAND_CAP, at = ref % CAND_CAP;
@@ -1024,7 +1077,9 @@ __global__ void __launch_bounds__(THREADS)
         if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
       }
     }
+    atomicOr(&zmask[zmask_word(i)], zmask_bit(i));  // the next streaming pass zeroes all W residuals
   } else {
+    float* p = acc + i;
     for (int w0 = 0; w0 < W; w0 += 8) {
       float v[8];
 #pragma unroll
@@ -1034,9 +1089,31 @@ __global__ void __launch_bounds__(THREADS)
         if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
       }
     }
+    for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
   }
-  for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
   update[i] = __fadd_rn(0.0f, s);
+}
+
+// Applies a pending zero mask right away (accessors, reset, and the multi-pass path need the
+// residuals themselves up to date).  One thread per mask word; the mask is cleared.
+__global__ void __launch_bounds__(THREADS)
+    k_flush_zmask(uint32_t* __restrict__ zmask, float* __restrict__ acc, uint64_t n_words, uint64_t N, int W) {
+  const uint64_t wd = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (wd >= n_words) return;
+  uint32_t bits = zmask[wd];
+  if (bits == 0u) return;
+  zmask[wd] = 0u;
+  const uint64_t field0 = wd * 2;  // (segment, lane) index of the low half
+  for (; bits; bits &= bits - 1) {
+    const uint32_t b = __ffs(bits) - 1;
+    const uint64_t field = field0 + (b >> 4);
+    const uint64_t seg = field >> 5, lane = field & 31;
+    const uint32_t fb = b & 15u;
+    const uint64_t i = seg * 512 + (fb >> 2) * 128 + lane * 4 + (fb & 3u);
+    if (i < N) {
+      for (int w = 0; w < W; ++w) acc[static_cast<uint64_t>(w) * N + i] = 0.0f;
+    }
+  }
 }
 
 // byte mask of the index set (Algorithm 1's encode_uint8(Mask)); dst is zeroed by the caller

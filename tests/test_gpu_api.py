@@ -149,3 +149,23 @@ def test_single_read_path_is_taken_and_falls_back_when_it_must():
     pr.set_option("speculate", 0)
     assert pr.stat("spec_pairs") == 0
     pr.close()
+
+
+def test_switching_speculation_off_mid_run_keeps_state_exact():
+    sizes, W = [200000, 50], 3
+    N = sum(sizes)
+    weights, grads = _inputs(W, N, 12)
+    pr = Pruner(sizes, W, 64.0, 1e-8, 2)
+    orc = oracle.Oracle(sizes, W, 64.0, 1e-8, 2)
+    for t, g in enumerate(grads + grads):
+        if t == 2:
+            pr.set_option("speculate", 0)  # pending lazy zeroing must be applied before the multi-pass path runs
+        if t == 4:
+            pr.set_option("speculate", 1)
+        upd = pr.step(g, weights)
+        want = orc.step(g.cpu().numpy(), weights.cpu().numpy())
+        assert_bits_equal(upd.cpu().numpy(), want, f"step {t}: update")
+    for w in range(W):
+        assert_bits_equal(pr.residual(w).cpu().numpy(), orc.residual(w), f"worker {w} residual")
+    assert pr.sync_status() == 0
+    pr.close()

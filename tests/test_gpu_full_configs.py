@@ -24,7 +24,10 @@ def test_full_size_every_output(name):
     c = wl.CONFIGS[name]()
     weights = c.weights(DEV)
     buf = torch.empty((c.W, c.N), dtype=torch.float32, device=DEV)
-    run_parity(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, c.steps, weights, lambda t: c.grads(t, DEV, out=buf))
+    # the single-layer case looks at the residuals after every step; the two network-shaped cases only
+    # at steps 2 and 4 (0-based), so that most steps leave their zeroing to the next streaming pass
+    run_parity(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, c.steps, weights, lambda t: c.grads(t, DEV, out=buf),
+               residual_every=1 if name == "single_layer" else 3)
 
 
 def test_full_size_w32_stress():

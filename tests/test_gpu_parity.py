@@ -196,8 +196,29 @@ def _scaled_case(name):
     return wl.scaled(b, wl.split_equal((1 << 22) + 64, 96), steps=4)
 
 
+@pytest.mark.parametrize("residual_every", [1, 1000])
 @pytest.mark.parametrize("name", sorted(wl.CONFIGS))
-def test_scaled_configs(name):
+def test_scaled_configs(name, residual_every):
     c = _scaled_case(name)
     weights = c.weights(DEV)
-    run_parity(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, c.steps, weights, lambda t: c.grads(t, DEV))
+    run_parity(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, c.steps, weights, lambda t: c.grads(t, DEV),
+               residual_every=residual_every)
+
+
+def test_residuals_left_alone_between_steps_with_ties_and_fallbacks():
+    # coarse values: some pairs fall back to the multi-pass select, others stay on the single-read
+    # path; residuals are read only at the end, and the option switch in the middle forces a flush
+    sizes, W, ratio = [70000, 64, 16385, 300000], 4, 64.0
+    N = sum(sizes)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(17)
+    weights = torch.randint(-3, 4, (N,), generator=g, device=DEV).float() * 0.25
+
+    def grads(t):
+        gg = torch.Generator(device=DEV)
+        gg.manual_seed(500 + t)
+        coarse = torch.randint(-4, 5, (W, N), generator=gg, device=DEV).float() / 8.0
+        fine = torch.randn((W, N), generator=gg, device=DEV) * 1e-3
+        return coarse if t % 3 == 2 else fine
+
+    run_parity(sizes, W, ratio, 1e-8, seed=3, steps=7, weights=weights, grads_fn=grads, residual_every=1000)
