@@ -431,21 +431,24 @@ __global__ void __launch_bounds__(THREADS, 3)
   uint32_t count = 0;    // entries appended to the slot so far (the same in every lane)
   uint32_t reached = 0;  // of those, how many reach the guess exactly
   bool overflow = false;
-#pragma unroll 1
-  for (uint32_t it = 0; it < SEGS_PER_TILE; ++it) {
+  // The tile covers the segments it0 .. it1 of its window.  The loads of segment it + 1 are issued
+  // as soon as the arithmetic of segment it is done, so they are in flight while the rare-path work
+  // of segment it (side values, staging, exact quotients) runs out of shared memory.
+  const uint32_t it0 = static_cast<uint32_t>((lo - base) / SEG_ELEMS);
+  const uint32_t it1 = static_cast<uint32_t>((hi - 1 - base) / SEG_ELEMS);
+  float gv[ROUNDS][4], av[ROUNDS][4], den[ROUNDS][4];
+  uint32_t zm_next = 0;
+  uint2 ll_next = make_uint2(0u, 0u);
+  uint32_t lt_next = 0;
+  auto fetch = [&](uint32_t it) {
     const uint64_t seg = base + it * SEG_ELEMS;
-    if (seg + SEG_ELEMS <= lo || seg >= hi) continue;  // warp-uniform
-    const uint64_t first = seg + static_cast<uint64_t>(lane) * 4;  // this lane's slot in round 0
-    const uint64_t sigma = static_cast<uint64_t>(tile_id) * SEGS_PER_TILE + it;  // global segment id
-    float gv[ROUNDS][4], av[ROUNDS][4], den[ROUNDS][4];
-    uint32_t inrange = 0xFFFFu;
-    // residuals sent in the previous step count as +0 (they are overwritten below either way)
-    const uint32_t zm = reinterpret_cast<const uint16_t*>(zmask)[(seg >> 9) * 32 + lane];
-    uint2 ll = make_uint2(0u, 0u);
-    uint32_t lt = 0;
+    const uint64_t first = seg + static_cast<uint64_t>(lane) * 4;
+    // residuals sent in the previous step count as +0 (they are overwritten either way)
+    zm_next = reinterpret_cast<const uint16_t*>(zmask)[(seg >> 9) * 32 + lane];
     if (!LEADER) {  // the leader's record for this segment: (mask | count << 16, lane prefix), round totals
-      ll = lead_lane[sigma * 32 + lane];
-      lt = lead_tot[sigma];
+      const uint64_t sigma = static_cast<uint64_t>(tile_id) * SEGS_PER_TILE + it;
+      ll_next = lead_lane[sigma * 32 + lane];
+      lt_next = lead_tot[sigma];
     }
     if (full) {
       const float4* g4 = reinterpret_cast<const float4*>(g + first);
@@ -459,15 +462,34 @@ __global__ void __launch_bounds__(THREADS, 3)
         den[s][0] = z.x; den[s][1] = z.y; den[s][2] = z.z; den[s][3] = z.w;
       }
     } else {
-      inrange = 0;
 #pragma unroll
       for (int s = 0; s < ROUNDS; ++s) {
         const uint64_t e0 = first + s * 128;
         load4_stream<VEC>(g, e0, lo, hi, gv[s]);
         load4_stream<VEC>(a, e0, lo, hi, av[s]);
         load4<VEC>(weights, e0, lo, hi, den[s]);
+      }
+    }
+  };
+  fetch(it0);
+#pragma unroll 1
+  for (uint32_t it = it0; it <= it1; ++it) {
+    const uint64_t seg = base + it * SEG_ELEMS;
+    const uint64_t first = seg + static_cast<uint64_t>(lane) * 4;  // this lane's slot in round 0
+    const uint64_t sigma = static_cast<uint64_t>(tile_id) * SEGS_PER_TILE + it;  // global segment id
+    const uint32_t zm = zm_next;
+    const uint2 ll = ll_next;
+    const uint32_t lt = lt_next;
+    uint32_t inrange = 0xFFFFu;
+    if (!full) {
+      inrange = 0;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) inrange |= (e0 + c >= lo && e0 + c < hi) ? (1u << (4 * s + c)) : 0u;
+      for (int s = 0; s < ROUNDS; ++s) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const uint64_t e = first + s * 128 + c;
+          inrange |= (e >= lo && e < hi) ? (1u << (4 * s + c)) : 0u;
+        }
       }
     }
     if (zm) {
@@ -509,6 +531,7 @@ __global__ void __launch_bounds__(THREADS, 3)
       }
     }
     m &= inrange;
+    if (it < it1) fetch(it + 1);  // in flight during the rare-path work below
 
     if (!LEADER) {  // this worker's value at every position of the leader's slot (step (e) without a gather)
       const uint32_t mL = ll.x & 0xFFFFu, countL = ll.x >> 16;
