@@ -655,25 +655,42 @@ __device__ __forceinline__ void for_each_candidate(const Chunk& c, int w, int W,
 
 // One histogram pass over a chunk: keys that match the prefix found so far are counted by
 // their next digit.  grid = (chunks, W).
-template <bool VEC>
+//
+// FUSED: the CTA that finishes a pair's pass last (a ticket from an atomic counter tells it; nobody
+// waits for anybody) also takes the digit decision for the pair, so no separate kernel runs between
+// passes.  In the last pass every CTA additionally leaves, per chunk, the number of keys above the
+// prefix and the suffix sums of its low-digit histogram; from those the deciding CTA derives every
+// chunk's (#keys > T, #keys == T), which the compaction needs for its list offsets.
+template <bool VEC, bool FUSED>
 __global__ void __launch_bounds__(THREADS)
     k_hist(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
            const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
-           const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt, const uint2* __restrict__ state,
-           uint32_t* __restrict__ hist, float eps, uint64_t N, int W, int pass) {
+           const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt, uint2* state,
+           uint32_t* __restrict__ hist, uint32_t* __restrict__ done, uint32_t* __restrict__ chunk_sfx,
+           uint2* chunk_cnt, int* __restrict__ status, float eps, uint64_t N, int W, int pass, uint32_t n_chunks) {
   __shared__ uint32_t sh[NBINS];
+  __shared__ uint32_t sh_scan[THREADS];
+  __shared__ uint32_t sh_warp[WARPS];
+  __shared__ uint32_t res[4];
+  __shared__ uint32_t sh_above, sh_last;
   const Chunk c = chunks[blockIdx.x];
   const int w = blockIdx.y;
   const LayerDesc L = layers[c.layer];
   const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
   const int shift = pass_shift(pass), nb = pass_bins(pass);
   const int prev_shift = pass == 0 ? 31 : pass_shift(pass - 1);
-  const uint32_t want = pass == 0 ? 0u : (state[pair].x >> prev_shift);
+  const uint2 st_in = pass == 0 ? make_uint2(0u, L.k) : state[pair];
+  const uint32_t want = pass == 0 ? 0u : (st_in.x >> prev_shift);
+  const bool last_pass = pass == N_PASSES - 1;
   for (int b = threadIdx.x; b < nb; b += THREADS) sh[b] = 0;
+  if (threadIdx.x == 0) sh_above = 0;
   __syncthreads();
+  uint32_t above = 0;  // keys whose higher digits already exceed the prefix (needed in the last pass only)
   if (pair_is_cand(info[pair], L.k)) {
     for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
-      if ((key >> prev_shift) == want) atomicAdd(&sh[(key >> shift) & (nb - 1)], 1u);
+      const uint32_t hi_part = key >> prev_shift;
+      if (hi_part == want) atomicAdd(&sh[(key >> shift) & (nb - 1)], 1u);
+      above += hi_part > want ? 1u : 0u;
     });
   } else {
     const uint64_t lo = c.a, hi = lo + c.len;
@@ -689,16 +706,78 @@ __global__ void __launch_bounds__(THREADS)
       for (int q = 0; q < 4; ++q) {
         const uint64_t e = e0 + q;
         const uint32_t key = imp_key(av[q], wv[q], eps);
-        const bool valid = e >= lo && e < hi && (key >> prev_shift) == want;  // pass 0: bit 31 is 0 == want
+        const bool in = e >= lo && e < hi;
+        const bool valid = in && (key >> prev_shift) == want;  // pass 0: bit 31 is 0 == want
         hist_add_aggregated(sh, valid, (key >> shift) & (nb - 1));
+        above += (in && (key >> prev_shift) > want) ? 1u : 0u;
       }
     }
+  }
+  if (FUSED && last_pass) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) above += __shfl_xor_sync(0xffffffffu, above, d);
+    if ((threadIdx.x & 31) == 0 && above) atomicAdd(&sh_above, above);
   }
   __syncthreads();
   uint32_t* gh = hist + static_cast<uint64_t>(pair) * NBINS;
   for (int b = threadIdx.x; b < nb; b += THREADS) {
     const uint32_t v = sh[b];
     if (v) atomicAdd(&gh[b], v);
+  }
+  if (!FUSED) return;
+
+  if (last_pass) {  // suffix sums S[b] = sum of this chunk's bins >= b, and the count above the prefix
+    static_assert(pass_bins(N_PASSES - 1) == THREADS * 4, "four bins per thread in the last pass");
+    const uint32_t h0 = sh[threadIdx.x * 4], h1 = sh[threadIdx.x * 4 + 1], h2 = sh[threadIdx.x * 4 + 2],
+                   h3 = sh[threadIdx.x * 4 + 3];
+    uint32_t total;
+    const uint32_t before = block_excl_scan(h0 + h1 + h2 + h3, sh_warp, total);
+    const uint32_t s0 = total - before;
+    uint4 sfx = make_uint4(s0, s0 - h0, s0 - h0 - h1, s0 - h0 - h1 - h2);
+    uint32_t* dst = chunk_sfx + (static_cast<uint64_t>(w) * n_chunks + blockIdx.x) * pass_bins(N_PASSES - 1);
+    reinterpret_cast<uint4*>(dst)[threadIdx.x] = sfx;
+    if (threadIdx.x == 0) chunk_cnt[static_cast<uint64_t>(w) * n_chunks + blockIdx.x] = make_uint2(sh_above, 0u);
+  }
+  // ticket: the CTA that arrives last sees every other CTA's contribution
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t ticket = atomicAdd(&done[pair], 1u);
+    sh_last = (ticket == L.n_chunks - 1) ? 1u : 0u;
+  }
+  __syncthreads();
+  if (!sh_last) return;
+  __threadfence();
+  for (int b = threadIdx.x; b < nb; b += THREADS) {
+    sh[b] = __ldcg(&gh[b]);
+    gh[b] = 0;  // ready for the next pass / step
+  }
+  if (threadIdx.x == 0) done[pair] = 0;
+  __syncthreads();
+  find_digit(sh, nb, st_in.y, sh_scan, res);
+  const bool found = res[2] != 0;
+  const uint32_t digit = res[0], krem = res[1];
+  if (threadIdx.x == 0) {
+    if (found) {
+      state[pair] = make_uint2(st_in.x | (digit << shift), krem);
+    } else {
+      atomicMin(status, STATUS_INTERNAL);
+      state[pair] = make_uint2(0xffffffffu, 0u);  // selects nothing
+    }
+  }
+  if (last_pass) {  // per chunk of the pair: (#keys > T, #keys == T)
+    for (uint32_t j = L.first_chunk + threadIdx.x; j < L.first_chunk + L.n_chunks; j += THREADS) {
+      const uint64_t at = static_cast<uint64_t>(w) * n_chunks + j;
+      uint32_t gt = 0, eq = 0;
+      if (found) {
+        const uint32_t* sfx = chunk_sfx + at * pass_bins(N_PASSES - 1);
+        const uint32_t s_d = __ldcg(&sfx[digit]);
+        const uint32_t s_d1 = (digit + 1 < static_cast<uint32_t>(nb)) ? __ldcg(&sfx[digit + 1]) : 0u;
+        gt = __ldcg(reinterpret_cast<const unsigned int*>(&chunk_cnt[at])) + s_d1;
+        eq = s_d - s_d1;
+      }
+      chunk_cnt[at] = make_uint2(gt, eq);
+    }
   }
 }
 
