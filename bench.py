@@ -192,6 +192,9 @@ def run_ours(args):
     K = pr.K
     if args.speculate is not None:
         pr.set_option("speculate", args.speculate)
+    for kv in args.option:
+        k, v = kv.split("=")
+        pr.set_option(k, int(v))
 
     def barrier():
         if dist is not None:
@@ -325,6 +328,7 @@ def main():
     ap.add_argument("--layers", default=None, help="lo:hi - only these layers of the workload (small profiling case)")
     ap.add_argument("--grad-sets", type=int, default=None, help="distinct gradient batches kept on the device")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--option", action="append", default=[], help="key=value passed to iwp_set_option (experiments)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -24,6 +24,7 @@ struct iwp_ctx {
   int64_t leader_override = -1;
   bool force_scalar = false;
   bool speculate = true;
+  bool fused_select = true;
   cudaStream_t stream = nullptr;
   int device = 0;
   int64_t launches = 0;
@@ -276,10 +277,25 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   if (tiled) {
     const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
     dim3 cgrid(n_chunks, static_cast<unsigned>(W));
-    for (int pass = 0; pass < N_PASSES; ++pass) {  // the last CTA of each pair decides the digit (and the counts)
-      k_hist<VEC, true><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_info, c->cand_key,
-                                                  c->cand_cnt, c->d_state, c->d_hist, c->d_done, c->chunk_sfx,
-                                                  c->d_chunk_cnt, c->d_status, c->eps, N, W, pass, n_chunks);
+    for (int pass = 0; pass < N_PASSES; ++pass) {
+      if (c->fused_select) {  // the last CTA of each pair decides the digit (and, in the last pass, the counts)
+        k_hist<VEC, true><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_info, c->cand_key,
+                                                    c->cand_cnt, c->d_state, c->d_hist, c->d_done, c->chunk_sfx,
+                                                    c->d_chunk_cnt, c->d_status, c->eps, N, W, pass, n_chunks);
+        IWP_LAUNCH_CHECK(c);
+      } else {
+        k_hist<VEC, false><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_info, c->cand_key,
+                                                     c->cand_cnt, c->d_state, c->d_hist, c->d_done, c->chunk_sfx,
+                                                     c->d_chunk_cnt, c->d_status, c->eps, N, W, pass, n_chunks);
+        IWP_LAUNCH_CHECK(c);
+        k_find_digit<<<c->n_pairs, THREADS, 0, s>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->d_status,
+                                                    W, pass);
+        IWP_LAUNCH_CHECK(c);
+      }
+    }
+    if (!c->fused_select) {
+      k_count<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_info, c->cand_key,
+                                             c->cand_cnt, c->d_state, c->d_chunk_cnt, c->eps, N, W, n_chunks);
       IWP_LAUNCH_CHECK(c);
     }
   }
@@ -647,6 +663,11 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
     cudaStreamSynchronize(c->stream);
     stage_clear(c);
     c->time_stages = v != 0;
+    return IWP_OK;
+  }
+  if (!std::strcmp(key, "fused_select")) {
+    if (v != 0 && v != 1) return IWP_ERR_INVALID;
+    c->fused_select = v != 0;
     return IWP_OK;
   }
   if (!std::strcmp(key, "speculate")) {

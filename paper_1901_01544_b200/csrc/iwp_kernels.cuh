@@ -376,6 +376,24 @@ __device__ __forceinline__ float pretest_multiplier(uint32_t guess, float eps) {
 
 constexpr int EMIT_QUEUE = 128;  // staged entries per warp and iteration; more than this = overflow
 
+// Candidate entries are re-read several times by the select right after the streaming pass: store
+// them with an L2 evict-last policy so that the 6 GB that stream through L2 meanwhile do not push
+// them out.
+__device__ __forceinline__ uint64_t l2_evict_last_policy() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void st_keep_u32(uint32_t* ptr, uint32_t v, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.u32 [%0], %1, %2;" ::"l"(ptr), "r"(v), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void st_keep_f32(float* ptr, float v, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(ptr), "f"(v), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void st_keep_u16(uint16_t* ptr, uint16_t v, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.u16 [%0], %1, %2;" ::"l"(ptr), "h"(v), "l"(policy) : "memory");
+}
+
 // Position, inside one iteration, of the staged element with mask bit b = 4 * round + component:
 // the staged elements of earlier rounds, of earlier lanes in the same round, and of earlier
 // components of the same lane and round.  `ex` / `tt`: per-round exclusive lane prefix / totals,
@@ -431,6 +449,7 @@ __global__ void __launch_bounds__(THREADS, 3)
   uint32_t count = 0;    // entries appended to the slot so far (the same in every lane)
   uint32_t reached = 0;  // of those, how many reach the guess exactly
   bool overflow = false;
+  const uint64_t keep = l2_evict_last_policy();
   // The tile covers the segments it0 .. it1 of its window.  The loads of segment it + 1 are issued
   // as soon as the arithmetic of segment it is done, so they are in flight while the rare-path work
   // of segment it (side values, staging, exact quotients) runs out of shared memory.
@@ -538,7 +557,7 @@ __global__ void __launch_bounds__(THREADS, 3)
       for (uint32_t mm = mL; mm; mm &= mm - 1) {
         const uint32_t b = __ffs(mm) - 1;
         const uint32_t pos = countL + staged_position(mL, ll.y, lt, b);
-        if (pos < CAND_CAP) side_val[slot + pos] = res[(b >> 2) * 128 + (b & 3u)];
+        if (pos < CAND_CAP) st_keep_f32(side_val + slot + pos, res[(b >> 2) * 128 + (b & 3u)], keep);
       }
     }
 
@@ -582,9 +601,9 @@ __global__ void __launch_bounds__(THREADS, 3)
           hit = key >= guess;
           const uint32_t pos = count + j;
           if (pos < CAND_CAP) {
-            cand_key[slot + pos] = key;
-            cand_val[slot + pos] = v;
-            cand_idx[slot + pos] = ql[j];
+            st_keep_u32(cand_key + slot + pos, key, keep);
+            st_keep_f32(cand_val + slot + pos, v, keep);
+            st_keep_u16(cand_idx + slot + pos, ql[j], keep);
           }
         }
         reached += __popc(__ballot_sync(0xffffffffu, hit));
@@ -594,7 +613,7 @@ __global__ void __launch_bounds__(THREADS, 3)
     }
   }
   if (lane == 0) {
-    cand_cnt[static_cast<uint64_t>(tile_id) * W + w] = count;
+    st_keep_u32(cand_cnt + static_cast<uint64_t>(tile_id) * W + w, count, keep);
     if (reached) atomicAdd(&info[pair].total, reached);
     if (overflow || count > CAND_CAP) atomicOr(&info[pair].flags, 1u);
   }
@@ -611,35 +630,45 @@ __device__ __forceinline__ void for_each_candidate(const Chunk& c, int w, int W,
                                                    const uint32_t* __restrict__ cand_key, F&& f) {
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t t_begin = warp * TILES_PER_WARP;
-  const uint32_t t_end = min(c.n_tiles, t_begin + TILES_PER_WARP);
-  for (uint32_t tb = t_begin; tb < t_end; tb += 4) {
-    uint32_t cnt[4];
-    uint4 k4[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q)
-      cnt[q] = (tb + q < t_end) ? min(cand_cnt[static_cast<uint64_t>(c.first_tile + tb + q) * W + w], CAND_CAP) : 0u;
+  if (t_begin >= c.n_tiles) return;
+  const uint32_t n_mine = min(c.n_tiles - t_begin, TILES_PER_WARP);
+  static_assert(TILES_PER_WARP == 16, "four batches of four tiles; one count per lane");
+  const uint64_t tw0 = static_cast<uint64_t>(c.first_tile + t_begin) * W + w;
+  // all sixteen counts with one load per lane, then the slots in four batches of four, the loads of
+  // batch b + 1 in flight while batch b is consumed
+  const uint32_t my_cnt = lane < n_mine ? min(cand_cnt[tw0 + static_cast<uint64_t>(lane) * W], CAND_CAP) : 0u;
+  uint4 k4[2][4];
+  auto load_batch = [&](int b, uint4 (&dst)[4]) {
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (static_cast<uint64_t>(c.first_tile + tb + q) * W + w) * CAND_CAP);
-      k4[q] = (lane * 4 < cnt[q]) ? kp[lane] : make_uint4(0u, 0u, 0u, 0u);
+      const uint32_t cnt = __shfl_sync(0xffffffffu, my_cnt, b * 4 + q);
+      const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (tw0 + static_cast<uint64_t>(b * 4 + q) * W) * CAND_CAP);
+      dst[q] = (lane * 4 < cnt) ? kp[lane] : make_uint4(0u, 0u, 0u, 0u);
     }
+  };
+  load_batch(0, k4[0]);
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    if (b + 1 < 4) load_batch(b + 1, k4[(b + 1) & 1]);
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
+      const uint32_t cnt = __shfl_sync(0xffffffffu, my_cnt, b * 4 + q);
+      const uint4 k = k4[b & 1][q];
       uint32_t j = lane * 4;
-      if (j + 0 < cnt[q]) f(k4[q].x);
-      if (j + 1 < cnt[q]) f(k4[q].y);
-      if (j + 2 < cnt[q]) f(k4[q].z);
-      if (j + 3 < cnt[q]) f(k4[q].w);
-      if (cnt[q] > 128) {
-        const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (static_cast<uint64_t>(c.first_tile + tb + q) * W + w) * CAND_CAP);
-        for (uint32_t j0 = 128; j0 < cnt[q]; j0 += 128) {
+      if (j + 0 < cnt) f(k.x);
+      if (j + 1 < cnt) f(k.y);
+      if (j + 2 < cnt) f(k.z);
+      if (j + 3 < cnt) f(k.w);
+      if (cnt > 128) {
+        const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (tw0 + static_cast<uint64_t>(b * 4 + q) * W) * CAND_CAP);
+        for (uint32_t j0 = 128; j0 < cnt; j0 += 128) {
           j = j0 + lane * 4;
-          if (j < cnt[q]) {
-            const uint4 k = kp[j >> 2];
-            f(k.x);
-            if (j + 1 < cnt[q]) f(k.y);
-            if (j + 2 < cnt[q]) f(k.z);
-            if (j + 3 < cnt[q]) f(k.w);
+          if (j < cnt) {
+            const uint4 kk = kp[j >> 2];
+            f(kk.x);
+            if (j + 1 < cnt) f(kk.y);
+            if (j + 2 < cnt) f(kk.z);
+            if (j + 3 < cnt) f(kk.w);
           }
         }
       }
@@ -662,7 +691,7 @@ __device__ __forceinline__ void for_each_candidate(const Chunk& c, int w, int W,
 // prefix and the suffix sums of its low-digit histogram; from those the deciding CTA derives every
 // chunk's (#keys > T, #keys == T), which the compaction needs for its list offsets.
 template <bool VEC, bool FUSED>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 5)
     k_hist(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
            const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
            const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt, uint2* state,
@@ -877,7 +906,7 @@ __global__ void __launch_bounds__(THREADS)
 // layer precede it; its list position is (#greater before it) + min(#equal before it, r).
 // grid = (chunks, W).
 template <bool VEC>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 5)
     k_write(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
             const Tile* __restrict__ tiles, const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
             const uint32_t* __restrict__ cand_key, const float* __restrict__ cand_val,
