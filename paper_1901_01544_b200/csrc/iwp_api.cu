@@ -24,8 +24,10 @@ struct iwp_ctx {
   int64_t leader_override = -1;
   bool force_scalar = false;
   bool speculate = true;
-  bool fused_select = true;
+  bool fused_select = false;  // one kernel per pass with a last-CTA decision: fewer launches, measured slower
   cudaStream_t stream = nullptr;
+  cudaStream_t side = nullptr;       // the one-CTA path of small layers runs here, beside the tiled path
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   int device = 0;
   int64_t launches = 0;
   uint64_t device_bytes = 0;
@@ -158,6 +160,12 @@ int dev_alloc(T** p, uint64_t bytes) {
 }
 
 void free_all(iwp_ctx* c) {
+  if (c->side) {
+    cudaStreamSynchronize(c->side);
+    cudaStreamDestroy(c->side);
+  }
+  if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+  if (c->ev_join) cudaEventDestroy(c->ev_join);
   cudaFree(c->acc);
   cudaFree(c->d_layers);
   cudaFree(c->d_tiles);
@@ -215,12 +223,27 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   const uint64_t N = p.N, K = p.K;
   cudaStream_t s = c->stream;
   stage_mark(c);
+  // Small layers touch nothing the tiled path touches until the final reduction, so when both kinds
+  // exist their one-CTA kernel runs on a side stream, forked here and joined before the reduction.
+  const bool fork_small = !p.small_layers.empty() && !p.large_layers.empty() && c->side != nullptr;
   if (!p.small_layers.empty()) {
     const size_t dyn = static_cast<size_t>(p.max_small_n) * sizeof(uint32_t);
     dim3 grid(static_cast<unsigned>(p.small_layers.size()), static_cast<unsigned>(W));
-    k_small<<<grid, THREADS, dyn, s>>>(grads, weights, c->acc, update, c->d_layers, c->d_small_ids, c->sel_idx,
-                                       c->sel_val, c->sel_slot, c->d_status, c->eps, N, K, leader);
+    cudaStream_t ss = s;
+    if (fork_small) {
+      if (cudaEventRecord(c->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess) {
+        cudaGetLastError();
+        return IWP_ERR_CUDA;
+      }
+      ss = c->side;
+    }
+    k_small<<<grid, THREADS, dyn, ss>>>(grads, weights, c->acc, update, c->d_layers, c->d_small_ids, c->sel_idx,
+                                        c->sel_val, c->sel_slot, c->d_status, c->eps, N, K, leader);
     IWP_LAUNCH_CHECK(c);
+    if (fork_small && cudaEventRecord(c->ev_join, c->side) != cudaSuccess) {
+      cudaGetLastError();
+      return IWP_ERR_CUDA;
+    }
   }
   stage_mark(c);
   const bool tiled = !p.large_layers.empty();
@@ -310,6 +333,10 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     IWP_LAUNCH_CHECK(c);
   }
   stage_mark(c);
+  if (fork_small && cudaStreamWaitEvent(s, c->ev_join, 0) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
   const unsigned gblocks = static_cast<unsigned>((K + THREADS - 1) / THREADS);
   if (spec) {
     k_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->sel_slot, c->side_val,
@@ -455,6 +482,9 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
     ok = cudaFuncSetAttribute(k_small, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               static_cast<int>(p.max_small_n * sizeof(uint32_t))) == cudaSuccess;
   }
+  ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaDeviceSynchronize() == cudaSuccess;
   if (!ok) {
     cudaGetLastError();

@@ -438,6 +438,7 @@ __global__ void __launch_bounds__(THREADS, 3)
   const uint2 pg = guess_tab[pair];
   const uint32_t guess = pg.x;
   const float gm = __uint_as_float(pg.y);
+  const float gme = __fmul_rn(gm, eps);
   const float* g = grads + static_cast<uint64_t>(w) * N;
   float* a = acc + static_cast<uint64_t>(w) * N;
   const uint64_t slot = (static_cast<uint64_t>(tile_id) * W + w) * CAND_CAP;
@@ -524,8 +525,9 @@ __global__ void __launch_bounds__(THREADS, 3)
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
         av[s][c] = __fadd_rn(av[s][c], gv[s][c]);
-        den[s][c] = imp_den(den[s][c], eps);
-        m |= (fabsf(av[s][c]) >= __fmul_rn(gm, den[s][c])) ? (1u << (4 * s + c)) : 0u;
+        // gm * (|w| + eps) in one fused operation; its rounding differs from the exact denominator's
+        // by parts in 2^24, far inside the 2^-20 slack of gm (den[][] holds the raw weights here)
+        m |= (fabsf(av[s][c]) >= __fmaf_rn(gm, fabsf(den[s][c]), gme)) ? (1u << (4 * s + c)) : 0u;
       }
     }
     // results: to HBM, and into shared memory so that the rare-path loops below can pick single
@@ -630,45 +632,35 @@ __device__ __forceinline__ void for_each_candidate(const Chunk& c, int w, int W,
                                                    const uint32_t* __restrict__ cand_key, F&& f) {
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t t_begin = warp * TILES_PER_WARP;
-  if (t_begin >= c.n_tiles) return;
-  const uint32_t n_mine = min(c.n_tiles - t_begin, TILES_PER_WARP);
-  static_assert(TILES_PER_WARP == 16, "four batches of four tiles; one count per lane");
-  const uint64_t tw0 = static_cast<uint64_t>(c.first_tile + t_begin) * W + w;
-  // all sixteen counts with one load per lane, then the slots in four batches of four, the loads of
-  // batch b + 1 in flight while batch b is consumed
-  const uint32_t my_cnt = lane < n_mine ? min(cand_cnt[tw0 + static_cast<uint64_t>(lane) * W], CAND_CAP) : 0u;
-  uint4 k4[2][4];
-  auto load_batch = [&](int b, uint4 (&dst)[4]) {
+  const uint32_t t_end = min(c.n_tiles, t_begin + TILES_PER_WARP);
+  for (uint32_t tb = t_begin; tb < t_end; tb += 4) {
+    uint32_t cnt[4];
+    uint4 k4[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      cnt[q] = (tb + q < t_end) ? min(cand_cnt[static_cast<uint64_t>(c.first_tile + tb + q) * W + w], CAND_CAP) : 0u;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const uint32_t cnt = __shfl_sync(0xffffffffu, my_cnt, b * 4 + q);
-      const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (tw0 + static_cast<uint64_t>(b * 4 + q) * W) * CAND_CAP);
-      dst[q] = (lane * 4 < cnt) ? kp[lane] : make_uint4(0u, 0u, 0u, 0u);
+      const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (static_cast<uint64_t>(c.first_tile + tb + q) * W + w) * CAND_CAP);
+      k4[q] = (lane * 4 < cnt[q]) ? kp[lane] : make_uint4(0u, 0u, 0u, 0u);
     }
-  };
-  load_batch(0, k4[0]);
-#pragma unroll
-  for (int b = 0; b < 4; ++b) {
-    if (b + 1 < 4) load_batch(b + 1, k4[(b + 1) & 1]);
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      const uint32_t cnt = __shfl_sync(0xffffffffu, my_cnt, b * 4 + q);
-      const uint4 k = k4[b & 1][q];
       uint32_t j = lane * 4;
-      if (j + 0 < cnt) f(k.x);
-      if (j + 1 < cnt) f(k.y);
-      if (j + 2 < cnt) f(k.z);
-      if (j + 3 < cnt) f(k.w);
-      if (cnt > 128) {
-        const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (tw0 + static_cast<uint64_t>(b * 4 + q) * W) * CAND_CAP);
-        for (uint32_t j0 = 128; j0 < cnt; j0 += 128) {
+      if (j + 0 < cnt[q]) f(k4[q].x);
+      if (j + 1 < cnt[q]) f(k4[q].y);
+      if (j + 2 < cnt[q]) f(k4[q].z);
+      if (j + 3 < cnt[q]) f(k4[q].w);
+      if (cnt[q] > 128) {
+        const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (static_cast<uint64_t>(c.first_tile + tb + q) * W + w) * CAND_CAP);
+        for (uint32_t j0 = 128; j0 < cnt[q]; j0 += 128) {
           j = j0 + lane * 4;
-          if (j < cnt) {
-            const uint4 kk = kp[j >> 2];
-            f(kk.x);
-            if (j + 1 < cnt) f(kk.y);
-            if (j + 2 < cnt) f(kk.z);
-            if (j + 3 < cnt) f(kk.w);
+          if (j < cnt[q]) {
+            const uint4 k = kp[j >> 2];
+            f(k.x);
+            if (j + 1 < cnt[q]) f(k.y);
+            if (j + 2 < cnt[q]) f(k.z);
+            if (j + 3 < cnt[q]) f(k.w);
           }
         }
       }
@@ -691,7 +683,7 @@ __device__ __forceinline__ void for_each_candidate(const Chunk& c, int w, int W,
 // prefix and the suffix sums of its low-digit histogram; from those the deciding CTA derives every
 // chunk's (#keys > T, #keys == T), which the compaction needs for its list offsets.
 template <bool VEC, bool FUSED>
-__global__ void __launch_bounds__(THREADS, 5)
+__global__ void __launch_bounds__(THREADS)
     k_hist(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
            const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
            const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt, uint2* state,
@@ -906,7 +898,7 @@ __global__ void __launch_bounds__(THREADS)
 // layer precede it; its list position is (#greater before it) + min(#equal before it, r).
 // grid = (chunks, W).
 template <bool VEC>
-__global__ void __launch_bounds__(THREADS, 5)
+__global__ void __launch_bounds__(THREADS)
     k_write(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
             const Tile* __restrict__ tiles, const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
             const uint32_t* __restrict__ cand_key, const float* __restrict__ cand_val,
