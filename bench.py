@@ -205,7 +205,7 @@ def run_ours(args):
     for t in range(args.warmup):
         pr.step(sets[t % n_sets], weights, update)
     pr.check()
-    pr.set_option("time_stages", 1)
+    pr.set_option("time_stages", 0 if args.no_stage_times else 1)
     launches0 = pr.stat("launches")
     sampler = ClockSampler(local)
     if rank == 0:
@@ -328,6 +328,7 @@ def main():
     ap.add_argument("--layers", default=None, help="lo:hi - only these layers of the workload (small profiling case)")
     ap.add_argument("--grad-sets", type=int, default=None, help="distinct gradient batches kept on the device")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-stage-times", action="store_true", help="do not record per-stage CUDA events")
     ap.add_argument("--option", action="append", default=[], help="key=value passed to iwp_set_option (experiments)")
     args = ap.parse_args()
     if args.warmup < 3:

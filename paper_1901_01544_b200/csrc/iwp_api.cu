@@ -316,11 +316,6 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
         IWP_LAUNCH_CHECK(c);
       }
     }
-    if (!c->fused_select) {
-      k_count<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_info, c->cand_key,
-                                             c->cand_cnt, c->d_state, c->d_chunk_cnt, c->eps, N, W, n_chunks);
-      IWP_LAUNCH_CHECK(c);
-    }
   }
   stage_mark(c);
   if (tiled) {
@@ -328,8 +323,9 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     dim3 cgrid(n_chunks, static_cast<unsigned>(W));
     k_write<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->d_info,
                                            c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
-                                           c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, c->d_status, c->eps,
-                                           N, K, W, n_chunks, leader);
+                                           c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot,
+                                           c->fused_select ? nullptr : c->chunk_sfx, c->d_status, c->eps, N, K, W,
+                                           n_chunks, leader);
     IWP_LAUNCH_CHECK(c);
   }
   stage_mark(c);
@@ -855,8 +851,8 @@ int run_select_static(StaticScratch* s, const float* residual, const float* weig
                                          s->chunk_cnt, eps, 0, 1, n_chunks);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   k_write<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, nullptr, &s->layer, &s->info, nullptr, nullptr,
-                                         nullptr, nullptr, &s->state, s->chunk_cnt, idx, val, nullptr, &s->status, eps,
-                                         0, 0, 1, n_chunks, -1);
+                                         nullptr, nullptr, &s->state, s->chunk_cnt, idx, val, nullptr, nullptr,
+                                         &s->status, eps, 0, 0, 1, n_chunks, -1);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   return IWP_OK;
 }

@@ -707,7 +707,32 @@ __global__ void __launch_bounds__(THREADS)
   if (threadIdx.x == 0) sh_above = 0;
   __syncthreads();
   uint32_t above = 0;  // keys whose higher digits already exceed the prefix (needed in the last pass only)
-  if (pair_is_cand(info[pair], L.k)) {
+  const PairInfo pi = info[pair];
+  if (pair_is_cand(pi, L.k) && pass == 0) {
+    // Every candidate is at or just above the guess, so almost all of them fall into the guess's own
+    // first-digit bin or the next two: count those in registers (one shared-memory atomic per lane
+    // would serialise on three addresses) and leave only the rest to atomics.
+    const uint32_t g0 = pi.guess >> shift;
+    uint32_t c0 = 0, c1 = 0, c2 = 0;
+    for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
+      const uint32_t d = (key >> shift) - g0;
+      c0 += d == 0u ? 1u : 0u;
+      c1 += d == 1u ? 1u : 0u;
+      c2 += d == 2u ? 1u : 0u;
+      if (d > 2u) atomicAdd(&sh[(key >> shift) & (nb - 1)], 1u);
+    });
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      c0 += __shfl_xor_sync(0xffffffffu, c0, d);
+      c1 += __shfl_xor_sync(0xffffffffu, c1, d);
+      c2 += __shfl_xor_sync(0xffffffffu, c2, d);
+    }
+    if ((threadIdx.x & 31) == 0) {
+      if (c0) atomicAdd(&sh[g0 & (nb - 1)], c0);
+      if (c1) atomicAdd(&sh[(g0 + 1) & (nb - 1)], c1);
+      if (c2) atomicAdd(&sh[(g0 + 2) & (nb - 1)], c2);
+    }
+  } else if (pair_is_cand(pi, L.k)) {
     for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
       const uint32_t hi_part = key >> prev_shift;
       if (hi_part == want) atomicAdd(&sh[(key >> shift) & (nb - 1)], 1u);
@@ -734,7 +759,7 @@ __global__ void __launch_bounds__(THREADS)
       }
     }
   }
-  if (FUSED && last_pass) {
+  if (last_pass && chunk_sfx != nullptr) {
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) above += __shfl_xor_sync(0xffffffffu, above, d);
     if ((threadIdx.x & 31) == 0 && above) atomicAdd(&sh_above, above);
@@ -745,9 +770,7 @@ __global__ void __launch_bounds__(THREADS)
     const uint32_t v = sh[b];
     if (v) atomicAdd(&gh[b], v);
   }
-  if (!FUSED) return;
-
-  if (last_pass) {  // suffix sums S[b] = sum of this chunk's bins >= b, and the count above the prefix
+  if (last_pass && chunk_sfx != nullptr) {  // suffix sums S[b] = sum of this chunk's bins >= b, and the count above the prefix
     static_assert(pass_bins(N_PASSES - 1) == THREADS * 4, "four bins per thread in the last pass");
     const uint32_t h0 = sh[threadIdx.x * 4], h1 = sh[threadIdx.x * 4 + 1], h2 = sh[threadIdx.x * 4 + 2],
                    h3 = sh[threadIdx.x * 4 + 3];
@@ -759,6 +782,7 @@ __global__ void __launch_bounds__(THREADS)
     reinterpret_cast<uint4*>(dst)[threadIdx.x] = sfx;
     if (threadIdx.x == 0) chunk_cnt[static_cast<uint64_t>(w) * n_chunks + blockIdx.x] = make_uint2(sh_above, 0u);
   }
+  if (!FUSED) return;
   // ticket: the CTA that arrives last sees every other CTA's contribution
   __threadfence();
   __syncthreads();
@@ -904,8 +928,8 @@ __global__ void __launch_bounds__(THREADS)
             const uint32_t* __restrict__ cand_key, const float* __restrict__ cand_val,
             const uint16_t* __restrict__ cand_idx, const uint32_t* __restrict__ cand_cnt,
             const uint2* __restrict__ state, const uint2* __restrict__ chunk_cnt, uint32_t* __restrict__ sel_idx,
-            float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot, int* __restrict__ status, float eps,
-            uint64_t N, uint64_t K, int W, uint32_t n_chunks, int leader) {
+            float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot, const uint32_t* __restrict__ chunk_sfx,
+            int* __restrict__ status, float eps, uint64_t N, uint64_t K, int W, uint32_t n_chunks, int leader) {
   __shared__ uint32_t sh_warp[WARPS];
   __shared__ uint32_t sh_base[2];
   const Chunk c = chunks[blockIdx.x];
@@ -922,8 +946,17 @@ __global__ void __launch_bounds__(THREADS)
     uint32_t g = 0, q = 0;
     for (uint32_t j = c.first_chunk_of_layer + threadIdx.x; j < blockIdx.x; j += THREADS) {
       const uint2 v = cc[j];
-      g += v.x;
-      q += v.y;
+      if (chunk_sfx == nullptr) {  // (#keys > T, #keys == T) of the chunk, counted by a kernel of its own
+        g += v.x;
+        q += v.y;
+      } else {  // left by the last histogram pass: keys above the prefix, suffix sums of the low digit
+        constexpr uint32_t LOW_BINS = pass_bins(N_PASSES - 1);
+        const uint32_t d = T & (LOW_BINS - 1);
+        const uint32_t* sfx = chunk_sfx + (static_cast<uint64_t>(w) * n_chunks + j) * LOW_BINS;
+        const uint32_t s_d = sfx[d], s_d1 = (d + 1 < LOW_BINS) ? sfx[d + 1] : 0u;
+        g += v.x + s_d1;
+        q += s_d - s_d1;
+      }
     }
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) {
