@@ -27,7 +27,7 @@ struct iwp_ctx {
   bool fused_select = false;  // one kernel per pass with a last-CTA decision: fewer launches, measured slower
   cudaStream_t stream = nullptr;
   cudaStream_t side = nullptr;       // the one-CTA path of small layers runs here, beside the tiled path
-  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_fork2 = nullptr, ev_join2 = nullptr;
   int device = 0;
   int64_t launches = 0;
   uint64_t device_bytes = 0;
@@ -166,6 +166,8 @@ void free_all(iwp_ctx* c) {
   }
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
+  if (c->ev_fork2) cudaEventDestroy(c->ev_fork2);
+  if (c->ev_join2) cudaEventDestroy(c->ev_join2);
   cudaFree(c->acc);
   cudaFree(c->d_layers);
   cudaFree(c->d_tiles);
@@ -226,6 +228,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   // Small layers touch nothing the tiled path touches until the final reduction, so when both kinds
   // exist their one-CTA kernel runs on a side stream, forked here and joined before the reduction.
   const bool fork_small = !p.small_layers.empty() && !p.large_layers.empty() && c->side != nullptr;
+  bool join_others = false;  // the other workers' lists are still being written on the side stream
   if (!p.small_layers.empty()) {
     const size_t dyn = static_cast<size_t>(p.max_small_n) * sizeof(uint32_t);
     dim3 grid(static_cast<unsigned>(p.small_layers.size()), static_cast<unsigned>(W));
@@ -321,12 +324,39 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   if (tiled) {
     const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
     dim3 cgrid(n_chunks, static_cast<unsigned>(W));
-    k_write<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->d_info,
-                                           c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
-                                           c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot,
-                                           c->fused_select ? nullptr : c->chunk_sfx, c->d_status, c->eps, N, K, W,
-                                           n_chunks, leader);
-    IWP_LAUNCH_CHECK(c);
+    // The reduction needs the leader's list only: write that one here and the other workers' lists on
+    // the side stream, beside the reduction; they are joined at the end of the step.
+    const bool split = spec && W > 1 && c->side != nullptr;
+    const uint32_t* sfx = c->fused_select ? nullptr : c->chunk_sfx;
+    if (split) {
+      if (cudaEventRecord(c->ev_fork2, s) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork2, 0) != cudaSuccess) {
+        cudaGetLastError();
+        return IWP_ERR_CUDA;
+      }
+      dim3 ogrid(n_chunks, static_cast<unsigned>(W - 1));
+      k_write<VEC><<<ogrid, THREADS, 0, c->side>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->d_info,
+                                                   c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
+                                                   c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, sfx,
+                                                   c->d_status, c->eps, N, K, W, n_chunks, leader, 2);
+      IWP_LAUNCH_CHECK(c);
+      if (cudaEventRecord(c->ev_join2, c->side) != cudaSuccess) {
+        cudaGetLastError();
+        return IWP_ERR_CUDA;
+      }
+      dim3 lgrid(n_chunks, 1);
+      k_write<VEC><<<lgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->d_info,
+                                             c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
+                                             c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, sfx, c->d_status,
+                                             c->eps, N, K, W, n_chunks, leader, 1);
+      IWP_LAUNCH_CHECK(c);
+      join_others = true;
+    } else {
+      k_write<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->d_info,
+                                             c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
+                                             c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, sfx, c->d_status,
+                                             c->eps, N, K, W, n_chunks, leader, 0);
+      IWP_LAUNCH_CHECK(c);
+    }
   }
   stage_mark(c);
   if (fork_small && cudaStreamWaitEvent(s, c->ev_join, 0) != cudaSuccess) {
@@ -343,6 +373,10 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
                                                      N, K, W);
   }
   IWP_LAUNCH_CHECK(c);
+  if (join_others && cudaStreamWaitEvent(s, c->ev_join2, 0) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
   stage_mark(c);
   return IWP_OK;
 }
@@ -481,6 +515,8 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
   ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&c->ev_fork2, cudaEventDisableTiming) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&c->ev_join2, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaDeviceSynchronize() == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
@@ -852,7 +888,7 @@ int run_select_static(StaticScratch* s, const float* residual, const float* weig
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   k_write<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, nullptr, &s->layer, &s->info, nullptr, nullptr,
                                          nullptr, nullptr, &s->state, s->chunk_cnt, idx, val, nullptr, nullptr,
-                                         &s->status, eps, 0, 0, 1, n_chunks, -1);
+                                         &s->status, eps, 0, 0, 1, n_chunks, -1, 0);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   return IWP_OK;
 }

@@ -929,11 +929,15 @@ __global__ void __launch_bounds__(THREADS)
             const uint16_t* __restrict__ cand_idx, const uint32_t* __restrict__ cand_cnt,
             const uint2* __restrict__ state, const uint2* __restrict__ chunk_cnt, uint32_t* __restrict__ sel_idx,
             float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot, const uint32_t* __restrict__ chunk_sfx,
-            int* __restrict__ status, float eps, uint64_t N, uint64_t K, int W, uint32_t n_chunks, int leader) {
+            int* __restrict__ status, float eps, uint64_t N, uint64_t K, int W, uint32_t n_chunks, int leader,
+            int which) {
   __shared__ uint32_t sh_warp[WARPS];
   __shared__ uint32_t sh_base[2];
   const Chunk c = chunks[blockIdx.x];
-  const int w = blockIdx.y;
+  // which = 0: blockIdx.y is the worker; 1: only the leader; 2: everybody but the leader
+  const int w = which == 0 ? static_cast<int>(blockIdx.y)
+                           : (which == 1 ? leader : (static_cast<int>(blockIdx.y) < leader ? static_cast<int>(blockIdx.y)
+                                                                                              : static_cast<int>(blockIdx.y) + 1));
   const LayerDesc L = layers[c.layer];
   const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
   const uint2 st = state[pair];
