@@ -333,7 +333,9 @@ __global__ void __launch_bounds__(SAMPLE_THREADS)
   uint32_t T, r;
   const bool ok = smem_radix_select<SAMPLE_THREADS>(keys, s, L.rho, hist, sh_scan, res, T, r);
   if (threadIdx.x == 0) {
-    const uint32_t guess = (ok && T != 0u) ? T : GUESS_NONE;
+    // no speculation on a guess whose first radix digit is zero (importance below 2^-126 * 2^-... ): the
+    // select's shortcuts for candidates assume that key 0 and digit 0 never belong to a candidate
+    const uint32_t guess = (ok && (T >> pass_shift(0)) != 0u) ? T : GUESS_NONE;
     const uint32_t gm = __float_as_uint(pretest_multiplier(guess, eps));
     info[pair] = PairInfo{guess, 0u, 0u, gm};
     guess_tab[pair] = make_uint2(guess, gm);  // read-only copy for the streaming pass (no atomics land on it)
@@ -614,6 +616,13 @@ __global__ void __launch_bounds__(THREADS, 3)
       __syncwarp();
     }
   }
+  // pad the slot to a multiple of four entries with key 0, so that readers can take whole 128-bit
+  // groups without testing every entry (no candidate has key 0: a zero guess is never used)
+  {
+    const uint32_t stored = count < CAND_CAP ? count : CAND_CAP;
+    const uint32_t pad_at = stored + lane;
+    if (pad_at < ((stored + 3u) & ~3u)) st_keep_u32(cand_key + slot + pad_at, 0u, keep);
+  }
   if (lane == 0) {
     st_keep_u32(cand_cnt + static_cast<uint64_t>(tile_id) * W + w, count, keep);
     if (reached) atomicAdd(&info[pair].total, reached);
@@ -624,7 +633,9 @@ __global__ void __launch_bounds__(THREADS, 3)
 // The candidates of (chunk, worker): warp q takes the chunk's tiles 16 q .. 16 q + 15 (consecutive,
 // so that warp order is index order), four tiles at a time; each lane reads entries 4 lane .. 4 lane + 3
 // of a slot with one 128-bit load (a slot rarely holds more than 128 entries; a tail loop covers the
-// rest) and all loads of a batch are issued before any is used.  `f(key)` sees every stored candidate.
+// rest) and all loads of a batch are issued before any is used.  `f(key)` sees every stored candidate,
+// and in addition some keys 0 (padding, slots shorter than 128 entries), which `f` must ignore - every
+// use below does so by construction, because a candidate's key and first digit are never 0.
 constexpr uint32_t TILES_PER_WARP = CHUNK_TILES / WARPS;
 
 template <typename F>
@@ -645,22 +656,21 @@ __device__ __forceinline__ void for_each_candidate(const Chunk& c, int w, int W,
       k4[q] = (lane * 4 < cnt[q]) ? kp[lane] : make_uint4(0u, 0u, 0u, 0u);
     }
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      uint32_t j = lane * 4;
-      if (j + 0 < cnt[q]) f(k4[q].x);
-      if (j + 1 < cnt[q]) f(k4[q].y);
-      if (j + 2 < cnt[q]) f(k4[q].z);
-      if (j + 3 < cnt[q]) f(k4[q].w);
+    for (int q = 0; q < 4; ++q) {  // groups past the count were not loaded (zeros); the last group is zero-padded
+      f(k4[q].x);
+      f(k4[q].y);
+      f(k4[q].z);
+      f(k4[q].w);
       if (cnt[q] > 128) {
         const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (static_cast<uint64_t>(c.first_tile + tb + q) * W + w) * CAND_CAP);
         for (uint32_t j0 = 128; j0 < cnt[q]; j0 += 128) {
-          j = j0 + lane * 4;
+          const uint32_t j = j0 + lane * 4;
           if (j < cnt[q]) {
             const uint4 k = kp[j >> 2];
             f(k.x);
-            if (j + 1 < cnt[q]) f(k.y);
-            if (j + 2 < cnt[q]) f(k.z);
-            if (j + 3 < cnt[q]) f(k.w);
+            f(k.y);
+            f(k.z);
+            f(k.w);
           }
         }
       }
@@ -719,7 +729,7 @@ __global__ void __launch_bounds__(THREADS)
       c0 += d == 0u ? 1u : 0u;
       c1 += d == 1u ? 1u : 0u;
       c2 += d == 2u ? 1u : 0u;
-      if (d > 2u) atomicAdd(&sh[(key >> shift) & (nb - 1)], 1u);
+      if (d > 2u && key != 0u) atomicAdd(&sh[(key >> shift) & (nb - 1)], 1u);
     });
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) {
@@ -1012,26 +1022,34 @@ __global__ void __launch_bounds__(THREADS)
       const uint32_t kk[4] = {k.x, k.y, k.z, k.w};
       uint32_t fg = 0, fe = 0;
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const bool in = j + u < cnt;
-        fg |= (in && kk[u] > T) ? (1u << u) : 0u;
-        fe |= (in && kk[u] == T) ? (1u << u) : 0u;
+      for (int u = 0; u < 4; ++u) {  // padding keys are 0 and T is not: no range test needed
+        fg |= kk[u] > T ? (1u << u) : 0u;
+        fe |= kk[u] == T ? (1u << u) : 0u;
       }
       if (!__any_sync(0xffffffffu, (fg | fe) != 0u)) return;
+      // most entries of a slot are selected: fetch the group's values and indices as vectors now, so
+      // that they arrive while the ranks are computed
+      float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
+      uint2 i2 = make_uint2(0u, 0u);
+      if (fg | fe) {
+        v4 = reinterpret_cast<const float4*>(cand_val + tw * CAND_CAP)[j >> 2];
+        i2 = reinterpret_cast<const uint2*>(cand_idx + tw * CAND_CAP)[j >> 2];
+      }
       const uint32_t packed = static_cast<uint32_t>(__popc(fg)) | (static_cast<uint32_t>(__popc(fe)) << 16);
       const uint32_t incl = warp_incl_scan(packed);
       const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
       uint32_t gb = g_before + ((incl - packed) & 0xffffu), qb = q_before + ((incl - packed) >> 16);
       if (fg | fe) {
+        const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+        const uint32_t ii[4] = {i2.x & 0xffffu, i2.x >> 16, i2.y & 0xffffu, i2.y >> 16};
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const bool isg = (fg >> u) & 1u, ise = (fe >> u) & 1u;
           if (isg || (ise && qb < r)) {
             const uint32_t pos = gb + (qb < r ? qb : r);
             if (pos < L.k) {
-              const uint64_t at = tw * CAND_CAP + j + u;
-              out_i[pos] = tile_base + cand_idx[at];
-              out_v[pos] = cand_val[at];
+              out_i[pos] = tile_base + ii[u];
+              out_v[pos] = vv[u];
               if (is_leader) sel_slot[L.koff + pos] = tile * CAND_CAP + j + u;
             } else {
               atomicMin(status, STATUS_INTERNAL);
