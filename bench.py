@@ -61,7 +61,7 @@ class ClockSampler:
             os.close(fd)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                 "-lms", "50"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -95,6 +95,23 @@ class ClockSampler:
         if sm:
             out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
         return out
+
+
+def max_over_ranks(value: float, dist, device) -> float:
+    """Slowest rank's value (each rank times its own replica on its own device)."""
+    if dist is None:
+        return float(value)
+    import torch
+
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(steps: int, world: int, ms_total_max: float) -> float:
+    """Units all ranks processed divided by the slowest rank's time: every rank runs `steps` steps of
+    its own replica (weak scaling, no data-path collective)."""
+    return world * steps / (ms_total_max / 1e3)
 
 
 def make_workload(name, layers=None):
@@ -205,7 +222,10 @@ def run_ours(args):
     for t in range(args.warmup):
         pr.step(sets[t % n_sets], weights, update)
     pr.check()
-    pr.set_option("time_stages", 0 if args.no_stage_times else 1)
+    # two CUDA events per step, around the streaming stage (the dominant kernel, two launches of k_stream);
+    # the full per-stage breakdown is taken in a separate, shorter pass after the timed region because
+    # seven events per step cost about 1 % of the step
+    pr.set_option("time_stages", 0 if args.no_stage_times else 2)
     launches0 = pr.stat("launches")
     sampler = ClockSampler(local)
     if rank == 0:
@@ -222,16 +242,23 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     launches = pr.stat("launches") - launches0
     pr.check()
-    stage_ms = {k: pr.stat(f"time_{k}_ns") / 1e6 / args.steps for k in ("small", "sample", "accumulate", "select",
-                                                                           "compact", "gather")}
+    k1_ms_live = pr.stat("time_accumulate_ns") / 1e6 / args.steps
     spec = {"pairs": pr.stat("spec_pairs"), "failed": pr.stat("spec_failed")}
+    stage_steps = 0 if args.no_stage_times else max(1, min(args.steps, args.stage_steps))
+    stage_ms = None
+    if stage_steps:
+        pr.set_option("time_stages", 1)
+        for t in range(stage_steps):
+            pr.step(sets[(args.warmup + args.steps + t) % n_sets], weights, update)
+        pr.check()
+        stage_ms = {k: pr.stat(f"time_{k}_ns") / 1e6 / stage_steps for k in ("small", "sample", "accumulate", "select",
+                                                                              "compact", "gather")}
+        stage_ms["note"] = (f"separate pass of {stage_steps} steps with an event at every stage boundary; 'small' runs on a "
+                            "side stream beside the other stages, 'gather' includes waiting for the non-leader lists")
     pr.set_option("time_stages", 0)
-    if dist is not None:
-        tt = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_total = float(tt.item())
+    ms_total = max_over_ranks(ms_total, dist, dev)
     ms_per_step = ms_total / args.steps
-    value = world * args.steps / (ms_total / 1e3)
+    value = whole_job_value(args.steps, world, ms_total)
 
     # end to end through the host-buffer entry point: H2D of grads + weights and D2H of the update inside
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -248,12 +275,9 @@ def run_ours(args):
             pr.step_host(gh[t % len(gh)], wh, uh)
         torch.cuda.synchronize()
         e2e_dt = time.perf_counter() - t0
-        if dist is not None:
-            tt = torch.tensor([e2e_dt], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_dt = float(tt.item())
+        e2e_dt = max_over_ranks(e2e_dt, dist, dev)
         pr.check()
-        e2e_value = world * e2e_steps / e2e_dt
+        e2e_value = whole_job_value(e2e_steps, world, e2e_dt * 1e3)
 
     if rank != 0:
         if dist is not None:
@@ -264,17 +288,20 @@ def run_ours(args):
     B = step_bytes(W, N, K)
     plan = __import__("paper_1901_01544_b200.binding", fromlist=["x"]).iwp_plan_sizes(c.layer_sizes, W, c.ratio)
     Nt = sum(n for n in c.layer_sizes if n > 16384)  # elements on the tiled path
-    # algorithmic bytes of one launch of the dominant kernel (fused accumulate + importance + candidate
-    # emission over all tiled layers): grads read, residual read and written, weights read, update zeroed
+    # The dominant kernel is k_stream (fused accumulate + importance + candidate emission over all tiled
+    # layers).  It is launched twice per step - once for the leader's worker, once for the W-1 others -
+    # and the two launches together move, algorithmically: grads read, residual read and written
+    # (12 bytes per worker and element), weights read and update zeroed once (8 bytes per element).
     k1_bytes = 12 * W * Nt + 8 * Nt
-    dom = max(stage_ms, key=stage_ms.get)
-    k1_ms = stage_ms["accumulate"]
+    k1_ms = k1_ms_live
     achieved = k1_bytes / (k1_ms * 1e-3) / 1e9 if k1_ms > 0 else 0.0
     roofline = {
-        "bound": "hbm", "kernel": "k_accumulate (fused accumulate + importance pass over all tiled layers)",
+        "bound": "hbm",
+        "kernel": "k_stream, both launches of a step (leader, then the other workers), timed together",
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-        "traffic": None, "algorithmic_bytes_per_launch": k1_bytes, "ms_per_launch": k1_ms,
-        "dominant_stage_by_time": dom,
+        "traffic": args.traffic_bytes, "algorithmic_bytes_per_step_of_kernel": k1_bytes, "ms_per_step_of_kernel": k1_ms,
+        "launches_per_step": 2 if W > 1 else 1,
+        "traffic_note": "dram__bytes_read+write of both launches from an ncu capture (profiles/), scaled to this workload",
     }
     eff = B / (ms_per_step * 1e-3) / 1e9
     step_eff = {"compulsory_bytes": B, "effective_gbs": eff, "frac_of_measured_peak": eff / peak,
@@ -317,18 +344,21 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="alexnet_w8")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--cpu-steps", type=int, default=3)
+    ap.add_argument("--cpu-steps", type=int, default=15)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--speculate", type=int, default=None, choices=[0, 1])
     ap.add_argument("--layers", default=None, help="lo:hi - only these layers of the workload (small profiling case)")
     ap.add_argument("--grad-sets", type=int, default=None, help="distinct gradient batches kept on the device")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-stage-times", action="store_true", help="do not record per-stage CUDA events")
+    ap.add_argument("--stage-steps", type=int, default=10, help="steps of the separate per-stage timing pass")
+    ap.add_argument("--traffic-bytes", type=float, default=None,
+                    help="DRAM bytes of the dominant kernel per step from an ncu capture (goes into roofline.traffic)")
     ap.add_argument("--option", action="append", default=[], help="key=value passed to iwp_set_option (experiments)")
     args = ap.parse_args()
     if args.warmup < 3:

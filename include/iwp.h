@@ -149,7 +149,8 @@ int iwp_reset(iwp_ctx* ctx);
  *   "speculate"        1 (default) = sample-based threshold guess so that large layers are
  *                      read once; 0 = always the multi-pass exact select.  Both are exact.
  *   "time_stages"      1 = record a CUDA event at every stage boundary of each following step
- *                      (read the totals with iwp_get_stat); 0 = stop and discard them
+ *                      (read the totals with iwp_get_stat); 2 = only before and after the streaming
+ *                      stage (two events per step); 0 = stop and discard them
  * Unknown key or out-of-range value: IWP_ERR_INVALID. */
 int iwp_set_option(iwp_ctx* ctx, const char* key, int64_t value);
 

@@ -64,7 +64,7 @@ struct iwp_ctx {
   float* sel_val = nullptr;
   int* d_status = nullptr;
   // optional per-stage CUDA-event timing (option "time_stages")
-  bool time_stages = false;
+  int time_stages = 0;  // 0 off, 1 every stage boundary, 2 only around the streaming stage
   std::vector<cudaEvent_t> stage_events;  // N_STAGES + 1 events per timed step
   // staging for iwp_step_host
   float* stg_grads = nullptr;
@@ -79,19 +79,25 @@ enum Stage { ST_SMALL = 0, ST_SAMPLE, ST_ACCUMULATE, ST_SELECT, ST_COMPACT, ST_G
 const char* const kStageKeys[N_STAGES] = {"time_small_ns", "time_sample_ns", "time_accumulate_ns", "time_select_ns", "time_compact_ns",
                                           "time_gather_ns"};
 
-void stage_mark(iwp_ctx* c) {
+// Called at every stage boundary of a step, in order; `boundary` = index of the stage that begins.
+void stage_mark_at(iwp_ctx* c, int boundary) {
   if (!c->time_stages) return;
-  cudaEvent_t e;
-  if (cudaEventCreate(&e) != cudaSuccess) {
-    cudaGetLastError();
-    return;
+  cudaEvent_t e = nullptr;
+  const bool wanted = c->time_stages == 1 || boundary == ST_ACCUMULATE || boundary == ST_ACCUMULATE + 1;
+  if (wanted) {
+    if (cudaEventCreate(&e) != cudaSuccess) {
+      cudaGetLastError();
+      e = nullptr;
+    } else {
+      cudaEventRecord(e, c->stream);
+    }
   }
-  cudaEventRecord(e, c->stream);
-  c->stage_events.push_back(e);
+  c->stage_events.push_back(e);  // a null entry keeps the slots of a step aligned
 }
 
 void stage_clear(iwp_ctx* c) {
-  for (cudaEvent_t e : c->stage_events) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->stage_events)
+    if (e) cudaEventDestroy(e);
   c->stage_events.clear();
 }
 
@@ -224,7 +230,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   const int W = p.W;
   const uint64_t N = p.N, K = p.K;
   cudaStream_t s = c->stream;
-  stage_mark(c);
+  stage_mark_at(c, 0);
   // Small layers touch nothing the tiled path touches until the final reduction, so when both kinds
   // exist their one-CTA kernel runs on a side stream, forked here and joined before the reduction.
   const bool fork_small = !p.small_layers.empty() && !p.large_layers.empty() && c->side != nullptr;
@@ -248,7 +254,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
       return IWP_ERR_CUDA;
     }
   }
-  stage_mark(c);
+  stage_mark_at(c, 1);
   const bool tiled = !p.large_layers.empty();
   const bool spec = tiled && c->speculate && c->spec_pairs > 0;
   if (!spec) {  // the multi-pass path reads the residuals as they are
@@ -270,7 +276,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     IWP_LAUNCH_CHECK(c);
     c->info_clean = false;
   }
-  stage_mark(c);
+  stage_mark_at(c, 2);
   if (tiled) {
     const unsigned n_tiles = static_cast<unsigned>(p.tiles.size());
     if (spec) {
@@ -299,7 +305,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     }
     IWP_LAUNCH_CHECK(c);
   }
-  stage_mark(c);
+  stage_mark_at(c, 3);
   if (tiled) {
     const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
     dim3 cgrid(n_chunks, static_cast<unsigned>(W));
@@ -320,7 +326,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
       }
     }
   }
-  stage_mark(c);
+  stage_mark_at(c, 4);
   if (tiled) {
     const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
     dim3 cgrid(n_chunks, static_cast<unsigned>(W));
@@ -358,7 +364,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
       IWP_LAUNCH_CHECK(c);
     }
   }
-  stage_mark(c);
+  stage_mark_at(c, 5);
   if (fork_small && cudaStreamWaitEvent(s, c->ev_join, 0) != cudaSuccess) {
     cudaGetLastError();
     return IWP_ERR_CUDA;
@@ -377,7 +383,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     cudaGetLastError();
     return IWP_ERR_CUDA;
   }
-  stage_mark(c);
+  stage_mark_at(c, 6);
   return IWP_OK;
 }
 
@@ -721,10 +727,10 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
     return IWP_OK;
   }
   if (!std::strcmp(key, "time_stages")) {
-    if (v != 0 && v != 1) return IWP_ERR_INVALID;
+    if (v < 0 || v > 2) return IWP_ERR_INVALID;
     cudaStreamSynchronize(c->stream);
     stage_clear(c);
-    c->time_stages = v != 0;
+    c->time_stages = static_cast<int>(v);
     return IWP_OK;
   }
   if (!std::strcmp(key, "fused_select")) {
@@ -764,8 +770,9 @@ int iwp_get_stat(iwp_ctx* c, const char* key, int64_t* value) {
     const size_t steps = c->stage_events.size() / (N_STAGES + 1);
     for (size_t i = 0; i < steps; ++i) {
       float ms = 0.f;
-      if (cudaEventElapsedTime(&ms, c->stage_events[i * (N_STAGES + 1) + st],
-                               c->stage_events[i * (N_STAGES + 1) + st + 1]) != cudaSuccess) {
+      cudaEvent_t e0 = c->stage_events[i * (N_STAGES + 1) + st], e1 = c->stage_events[i * (N_STAGES + 1) + st + 1];
+      if (!e0 || !e1) continue;  // this boundary was not recorded in the current timing mode
+      if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) {
         cudaGetLastError();
         return IWP_ERR_CUDA;
       }
