@@ -29,6 +29,7 @@ def lib() -> C.CDLL:
         L.oracle_threads_used.argtypes = [vp]
         L.oracle_threads_used.restype = i32
         L.oracle_set_leader_override.argtypes = [vp, i32]
+        L.oracle_set_momentum.argtypes = [vp, f32]
         L.oracle_total.argtypes = [vp]
         L.oracle_total.restype = i64
         L.oracle_total_keep.argtypes = [vp]
@@ -114,6 +115,9 @@ class Oracle:
         k = np.empty(self.L, dtype=np.int64)
         lib().oracle_get_layout(self._h, _p(off), _p(k))
         return off.tolist(), k.tolist()
+
+    def set_momentum(self, m: float):
+        lib().oracle_set_momentum(self._h, float(m))
 
     def set_leader_override(self, leader: int):
         lib().oracle_set_leader_override(self._h, leader)

@@ -23,6 +23,8 @@
 //     layer, k = ceil(n / ratio) clamped to [1, n]; ties keep the lower index.
 //   * one randomly chosen node per step supplies the index set (Section 3.2:
 //     "randomly choose a node and broadcast its important gradient index").
+//   * Eq. 3's momentum acts on the locally kept residual: G <- m * G + grad (two roundings);
+//     m = 1, the default, is the plain accumulation of Section 3.2.
 //   * the ring all-reduce is a sum in ascending worker order, fp32, without the 1/N
 //     factor (the caller pre-scales gradients as in Eq. 1).
 //
@@ -56,6 +58,7 @@ struct Oracle {
   int32_t leader = -1;
   int32_t leader_override = -1;
   int threads = 0;
+  float momentum = 1.0f;         // Eq. 3: the local residual enters the next step scaled by m
   std::vector<float> acc;        // [W][N] residuals
   std::vector<uint32_t> sel_idx; // [W][K] ascending global indices per layer segment
   std::vector<float> sel_val;    // [W][K] accumulated value at that index (before zeroing)
@@ -175,6 +178,7 @@ int32_t oracle_threads_used(void* h) {
   return 1;
 #endif
 }
+void oracle_set_momentum(void* h, float m) { static_cast<Oracle*>(h)->momentum = m; }
 void oracle_set_leader_override(void* h, int32_t leader) { static_cast<Oracle*>(h)->leader_override = leader; }
 int64_t oracle_total(void* h) { return static_cast<Oracle*>(h)->N; }
 int64_t oracle_total_keep(void* h) { return static_cast<Oracle*>(h)->K; }
@@ -231,9 +235,15 @@ void oracle_step(void* h, const float* grads, const float* weights, float* updat
   const int nthreads = o->threads > 0 ? o->threads : omp_get_max_threads();
 #endif
 
-  // (a) accumulate the new gradient into the local residual
+  // (a) accumulate the new gradient into the local residual; with momentum (Eq. 3,
+  // s_t = sparse(m g_{t-1} + g_t)) what was kept locally is first scaled by m: one rounded
+  // product, then one rounded sum (m = 1 leaves the residual unchanged)
+  const float m = o->momentum;
 #pragma omp parallel for num_threads(nthreads) schedule(static)
-  for (int64_t e = 0; e < static_cast<int64_t>(W) * N; ++e) o->acc[e] = o->acc[e] + grads[e];
+  for (int64_t e = 0; e < static_cast<int64_t>(W) * N; ++e) {
+    const float carried = m * o->acc[e];
+    o->acc[e] = carried + grads[e];
+  }
 
   // (b)-(d) per worker and layer: importance, keep the k best, list them in index order
 #pragma omp parallel num_threads(nthreads)

@@ -18,7 +18,8 @@ def importance(a, w, eps):
 
 
 class BruteForce:
-    def __init__(self, layer_sizes, W, ratio, eps):
+    def __init__(self, layer_sizes, W, ratio, eps, momentum=1.0):
+        self.m = F(momentum)
         self.n = list(layer_sizes)
         self.W, self.ratio, self.eps = W, float(ratio), F(eps)
         self.N = sum(self.n)
@@ -29,7 +30,7 @@ class BruteForce:
         W, N = self.W, self.N
         for w in range(W):
             for i in range(N):
-                self.acc[w][i] = F(self.acc[w][i] + F(grads[w][i]))
+                self.acc[w][i] = F(F(self.m * self.acc[w][i]) + F(grads[w][i]))
         lists = []
         for w in range(W):
             lst, o = [], 0

@@ -353,3 +353,62 @@ def test_reset_and_residual_roundtrip():
     for w in range(W):
         orc.set_residual(w, r[w])
         assert np.array_equal(u32(orc.residual(w)), u32(r[w]))
+
+
+# ---------------------------------------------------------------- momentum on the residual (Eq. 3)
+
+
+def test_momentum_one_is_plain_accumulation_and_bruteforce_agrees():
+    layers, W, ratio = [9, 20, 3], 3, 4.0
+    rng = np.random.default_rng(77)
+    N = sum(layers)
+    weights = (rng.normal(size=N) * (rng.random(N) > 0.1)).astype(np.float32)
+    for m in (1.0, 0.9, 0.5, 0.0):
+        orc = oracle.Oracle(layers, W, ratio, 1e-8, seed=2)
+        orc.set_momentum(m)
+        bf = BruteForce(layers, W, ratio, 1e-8, momentum=m)
+        plain = oracle.Oracle(layers, W, ratio, 1e-8, seed=2)
+        for t in range(4):
+            grads = (rng.integers(-8, 9, size=(W, N)) / 16.0).astype(np.float32)
+            upd = orc.step(grads, weights)
+            lists, upd_bf = bf.step(grads, weights, orc.leader)
+            assert np.array_equal(u32(upd), u32(upd_bf)), (m, t)
+            for w in range(W):
+                assert orc.selection(w)[0].tolist() == [i for i, _ in lists[w]]
+                assert np.array_equal(u32(orc.residual(w)), u32(bf.residual(w)))
+            if m == 1.0:
+                assert np.array_equal(u32(plain.step(grads, weights)), u32(upd))
+
+
+def test_momentum_hand_worked():
+    # one layer of 4, one worker, keep 1 of 4, weights 1: step 0 sends the largest, the rest is carried
+    # scaled by m = 0.5 into step 1:  residual after step 0 = [0, 2, 1, 0.5]; step 1 adds [4, 0, 0, 0]
+    # to 0.5 * residual = [0, 1, 0.5, 0.25]  ->  [4, 1, 0.5, 0.25]: index 0 is sent with value 4.
+    orc = oracle.Oracle([4], 1, 4.0, 1e-8, seed=0)
+    orc.set_momentum(0.5)
+    w = np.ones(4, np.float32)
+    u0 = orc.step(np.array([[8, 2, 1, 0.5]], np.float32), w)
+    assert u0.tolist() == [8, 0, 0, 0] and orc.residual(0).tolist() == [0, 2, 1, 0.5]
+    u1 = orc.step(np.array([[4, 0, 0, 0]], np.float32), w)
+    assert u1.tolist() == [4, 0, 0, 0] and orc.residual(0).tolist() == [0, 1, 0.5, 0.25]
+    # zero momentum forgets everything that was not sent
+    o2 = oracle.Oracle([4], 1, 4.0, 1e-8, seed=0)
+    o2.set_momentum(0.0)
+    o2.step(np.array([[8, 2, 1, 0.5]], np.float32), w)
+    u = o2.step(np.array([[0, 0, 0, 3]], np.float32), w)
+    assert u.tolist() == [0, 0, 0, 3] and o2.residual(0).tolist() == [0, 0, 0, 0]
+
+
+def test_momentum_geometric_carry_closed_form():
+    # an element that is never sent and receives a constant gradient c carries c (1 + m + ... + m^t):
+    # with c = 1 and m = 0.5 every partial sum is exactly representable
+    n = 16
+    orc = oracle.Oracle([n], 1, float(n), 1e-8, seed=0)  # keeps one element per step
+    orc.set_momentum(0.5)
+    w = np.ones(n, np.float32)
+    g = np.ones((1, n), np.float32)
+    g[0, 0] = 100.0  # index 0 always wins, the others are never sent
+    for t in range(10):
+        orc.step(g, w)
+        want = 2.0 - 0.5 ** t
+        assert np.all(orc.residual(0)[1:] == np.float32(want)), t
