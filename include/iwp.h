@@ -96,6 +96,12 @@ int iwp_destroy(iwp_ctx* ctx);
  * NULL = the legacy default stream, which is also the initial setting). */
 int iwp_set_stream(iwp_ctx* ctx, void* cuda_stream);
 
+/* Momentum on the locally kept residual (Eq. 3 of the paper: s_t = sparse(m g_{t-1} + g_t)): step (a)
+ * becomes acc[w][i] = m * acc[w][i] + grads[w][i], one rounded product then one rounded sum.
+ * m = 1 (the default) is the plain accumulation of Section 3.2; m = 0 forgets what was not sent.
+ * Takes effect from the next step.  Errors: IWP_ERR_INVALID (NULL, m negative or not finite). */
+int iwp_set_momentum(iwp_ctx* ctx, float m);
+
 /* ---- the step ---------------------------------------------------------------------------- */
 
 /* One pruned all-reduce step, steps (a)-(g) above (Algorithm 1, one iteration of the loop over t

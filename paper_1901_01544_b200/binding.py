@@ -20,6 +20,7 @@ EXPORTS = [
     "iwp_set_stream", "iwp_step", "iwp_step_host", "iwp_sync_status", "iwp_get_layout", "iwp_get_sizes",
     "iwp_get_step", "iwp_set_step", "iwp_get_leader", "iwp_get_residual", "iwp_set_residual",
     "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat", "iwp_select_static",
+    "iwp_set_momentum",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -48,6 +49,7 @@ def lib() -> C.CDLL:
         L.iwp_create.argtypes = [C.POINTER(vp), vp, i32, i32, f64, f32, u64]
         L.iwp_destroy.argtypes = [vp]
         L.iwp_set_stream.argtypes = [vp, vp]
+        L.iwp_set_momentum.argtypes = [vp, f32]
         L.iwp_step.argtypes = [vp, vp, vp, vp]
         L.iwp_step_host.argtypes = [vp, vp, vp, vp]
         L.iwp_sync_status.argtypes = [vp]
@@ -179,6 +181,9 @@ class Pruner:
             assert (not x.is_cuda) and x.dtype == t.float32 and x.is_contiguous() and x.numel() == n
         iwp_step_host(self._h, grads.data_ptr(), weights.data_ptr(), update.data_ptr())
         return update
+
+    def set_momentum(self, m: float) -> None:
+        _check(lib().iwp_set_momentum(self._h, float(m)), "iwp_set_momentum")
 
     def sync_status(self) -> int:
         return int(lib().iwp_sync_status(self._h))

@@ -17,6 +17,7 @@ using namespace iwp;
 struct iwp_ctx {
   Plan plan;
   float eps = 0.f;
+  float momentum = 1.0f;  // Eq. 3: factor on the locally kept residual before the new gradient is added
   double ratio = 1.0;
   uint64_t seed = 0;
   int64_t t = 0;
@@ -247,7 +248,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
       ss = c->side;
     }
     k_small<<<grid, THREADS, dyn, ss>>>(grads, weights, c->acc, update, c->d_layers, c->d_small_ids, c->sel_idx,
-                                        c->sel_val, c->sel_slot, c->d_status, c->eps, N, K, leader);
+                                        c->sel_val, c->sel_slot, c->d_status, c->eps, N, K, leader, c->momentum);
     IWP_LAUNCH_CHECK(c);
     if (fork_small && cudaEventRecord(c->ev_join, c->side) != cudaSuccess) {
       cudaGetLastError();
@@ -272,7 +273,8 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   if (spec) {
     const size_t dyn = static_cast<size_t>(c->max_sample) * sizeof(uint32_t);
     k_sample<<<c->n_pairs, SAMPLE_THREADS, dyn, s>>>(grads, weights, c->acc, c->d_layers, c->d_large_ids, c->d_info,
-                                             c->d_guess, c->zmask, c->eps, N, W, static_cast<uint32_t>(c->t));
+                                             c->d_guess, c->zmask, c->eps, N, W, static_cast<uint32_t>(c->t),
+                                             c->momentum);
     IWP_LAUNCH_CHECK(c);
     c->info_clean = false;
   }
@@ -283,14 +285,16 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
       // the leader's workers first (records where its candidates sit), then everybody else
       k_stream<VEC, true><<<(n_tiles + WARPS - 1) / WARPS, THREADS, 0, s>>>(
           grads, weights, c->acc, update, c->d_tiles, c->d_info, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
-          c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, 1);
+          c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, 1,
+          c->momentum);
       if (W > 1) {
         IWP_LAUNCH_CHECK(c);
         const int wpc = (W - 1 < WARPS) ? W - 1 : WARPS;  // warps (= workers) per CTA
         const int groups = (W - 1 + wpc - 1) / wpc;
         k_stream<VEC, false><<<n_tiles * static_cast<unsigned>(groups), wpc * 32, 0, s>>>(
             grads, weights, c->acc, update, c->d_tiles, c->d_info, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
-            c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, groups);
+            c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, groups,
+            c->momentum);
       }
       if (c->zero_pending) {  // every marked residual has now been overwritten: forget the marks
         IWP_LAUNCH_CHECK(c);
@@ -301,7 +305,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
         c->zero_pending = false;
       }
     } else {
-      k_accumulate<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, N, W);
+      k_accumulate<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, N, W, c->momentum);
     }
     IWP_LAUNCH_CHECK(c);
   }
@@ -541,6 +545,12 @@ int iwp_destroy(iwp_ctx* c) {
   free_all(c);
   cudaGetLastError();
   delete c;
+  return IWP_OK;
+}
+
+int iwp_set_momentum(iwp_ctx* c, float m) {
+  if (!c || !std::isfinite(m) || m < 0.f) return IWP_ERR_INVALID;
+  c->momentum = m;
   return IWP_OK;
 }
 

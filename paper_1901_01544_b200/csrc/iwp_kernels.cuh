@@ -49,6 +49,10 @@ __device__ __forceinline__ uint32_t imp_key(float acc, float w, float eps) {
   return __float_as_uint(__fdiv_rn(fabsf(acc), __fadd_rn(fabsf(w), eps)));
 }
 
+// Step (a) with Eq. 3's momentum on the locally kept residual: one rounded product, one rounded sum
+// (m = 1 leaves the residual as it is: plain accumulation).
+__device__ __forceinline__ float accumulate(float acc, float g, float m) { return __fadd_rn(__fmul_rn(m, acc), g); }
+
 __device__ __forceinline__ float imp_den(float w, float eps) { return __fadd_rn(fabsf(w), eps); }
 __device__ __forceinline__ uint32_t imp_key_den(float acc, float den) {
   return __float_as_uint(__fdiv_rn(fabsf(acc), den));
@@ -221,7 +225,7 @@ __device__ __forceinline__ void hist_add_aggregated(uint32_t* hist, bool valid, 
 template <bool VEC>
 __global__ void __launch_bounds__(THREADS) k_accumulate(const float* __restrict__ grads, float* __restrict__ acc,
                                                          float* __restrict__ update, const Tile* __restrict__ tiles,
-                                                         uint64_t N, int W) {
+                                                         uint64_t N, int W, float momentum) {
   const Tile t = tiles[blockIdx.x];
   const uint64_t lo = t.a, hi = lo + t.len;
   const uint64_t base = lo & ~static_cast<uint64_t>(TILE - 1);
@@ -244,7 +248,7 @@ __global__ void __launch_bounds__(THREADS) k_accumulate(const float* __restrict_
 #pragma unroll
     for (int s = 0; s < SPT; ++s) {
 #pragma unroll
-      for (int c = 0; c < 4; ++c) av[s][c] = __fadd_rn(av[s][c], gv[s][c]);
+      for (int c = 0; c < 4; ++c) av[s][c] = accumulate(av[s][c], gv[s][c], momentum);
       store4<VEC>(a, e0[s], lo, hi, av[s]);
     }
   }
@@ -282,7 +286,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS)
     k_sample(const float* __restrict__ grads, const float* __restrict__ weights, const float* __restrict__ acc,
              const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ large_ids, PairInfo* __restrict__ info,
              uint2* __restrict__ guess_tab, const uint32_t* __restrict__ zmask, float eps, uint64_t N, int W,
-             uint32_t step) {
+             uint32_t step, float momentum) {
   extern __shared__ uint32_t keys[];
   __shared__ uint32_t hist[NBINS];
   __shared__ uint32_t sh_scan[SAMPLE_THREADS];
@@ -326,7 +330,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS)
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       const uint32_t i = i0 + u * SAMPLE_THREADS + threadIdx.x;
-      if (i < s) keys[i] = imp_key(__fadd_rn(av[u], gv[u]), wv[u], eps);
+      if (i < s) keys[i] = imp_key(accumulate(av[u], gv[u], momentum), wv[u], eps);
     }
   }
   __syncthreads();
@@ -413,7 +417,7 @@ __global__ void __launch_bounds__(THREADS, 3)
              const uint2* __restrict__ guess_tab, uint32_t* __restrict__ cand_key, float* __restrict__ cand_val,
              uint16_t* __restrict__ cand_idx, uint32_t* __restrict__ cand_cnt, float* __restrict__ side_val,
              uint2* __restrict__ lead_lane, uint32_t* __restrict__ lead_tot, const uint32_t* __restrict__ zmask,
-             float eps, uint64_t N, int W, int leader, uint32_t n_tiles, int worker_groups) {
+             float eps, uint64_t N, int W, int leader, uint32_t n_tiles, int worker_groups, float momentum) {
   constexpr int ROUNDS = SEG_ELEMS / 128;  // 128-bit slots per lane and iteration = 4
   __shared__ float q_val[WARPS][EMIT_QUEUE];
   __shared__ float q_den[WARPS][EMIT_QUEUE];
@@ -526,7 +530,7 @@ __global__ void __launch_bounds__(THREADS, 3)
     for (int s = 0; s < ROUNDS; ++s) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        av[s][c] = __fadd_rn(av[s][c], gv[s][c]);
+        av[s][c] = accumulate(av[s][c], gv[s][c], momentum);
         // gm * (|w| + eps) in one fused operation; its rounding differs from the exact denominator's
         // by parts in 2^24, far inside the 2^-20 slack of gm (den[][] holds the raw weights here)
         m |= (fabsf(av[s][c]) >= __fmaf_rn(gm, fabsf(den[s][c]), gme)) ? (1u << (4 * s + c)) : 0u;
@@ -1148,7 +1152,7 @@ __global__ void __launch_bounds__(THREADS)
     k_small(const float* __restrict__ grads, const float* __restrict__ weights, float* __restrict__ acc,
             float* __restrict__ update, const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ small_ids,
             uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot,
-            int* __restrict__ status, float eps, uint64_t N, uint64_t K, int leader) {
+            int* __restrict__ status, float eps, uint64_t N, uint64_t K, int leader, float momentum) {
   extern __shared__ uint32_t keys[];
   __shared__ uint32_t hist[NBINS];
   __shared__ uint32_t sh_scan[THREADS];
@@ -1162,7 +1166,7 @@ __global__ void __launch_bounds__(THREADS)
   const float* g = grads + static_cast<uint64_t>(w) * N + L.off;
   const float* wt = weights + L.off;
   for (uint32_t i = tid; i < n; i += THREADS) {
-    const float v = __fadd_rn(a[i], __ldcs(g + i));
+    const float v = accumulate(a[i], __ldcs(g + i), momentum);
     a[i] = v;
     keys[i] = imp_key(v, wt[i], eps);
     if (w == 0) update[L.off + i] = 0.0f;

@@ -41,7 +41,7 @@ def compare_state(pr: Pruner, orc: "oracle.Oracle", update_gpu: torch.Tensor, up
 
 
 def run_parity(layer_sizes, W, ratio, eps, seed, steps, weights: torch.Tensor, grads_fn, options=None,
-               leader_overrides=None, check_mask=True, threads=0, residual_every=1):
+               leader_overrides=None, check_mask=True, threads=0, residual_every=1, momentum=None):
     """weights: CUDA tensor [N]; grads_fn(t) -> CUDA tensor [W, N].
 
     residual_every: residuals are read back (and compared) only every that many steps and after the
@@ -53,6 +53,9 @@ def run_parity(layer_sizes, W, ratio, eps, seed, steps, weights: torch.Tensor, g
     assert pr.layout() == orc.layout()
     for k, v in (options or {}).items():
         pr.set_option(k, v)
+    if momentum is not None:
+        pr.set_momentum(momentum)
+        orc.set_momentum(momentum)
     w_host = weights.cpu().numpy()
     update = torch.full((pr.N,), float("nan"), dtype=torch.float32, device="cuda")
     for t in range(steps):

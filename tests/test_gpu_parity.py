@@ -222,3 +222,24 @@ def test_residuals_left_alone_between_steps_with_ties_and_fallbacks():
         return coarse if t % 3 == 2 else fine
 
     run_parity(sizes, W, ratio, 1e-8, seed=3, steps=7, weights=weights, grads_fn=grads, residual_every=1000)
+
+
+# ------------------------------------------------------------------ momentum on the residual (Eq. 3)
+
+
+@pytest.mark.parametrize("m", [0.9, 0.5, 0.0])
+@pytest.mark.parametrize("speculate", [1, 0])
+def test_momentum(m, speculate):
+    sizes, W, ratio = [70000, 300, 16385, 64], 4, 64.0
+    N = sum(sizes)
+    weights = _weights(N, 21)
+    run_parity(sizes, W, ratio, 1e-8, seed=5, steps=5, weights=weights,
+               grads_fn=lambda t: _randn((W, N), 400 + t, 1e-3), options={"speculate": speculate}, momentum=m,
+               residual_every=2)
+
+
+def test_momentum_on_a_scaled_network_shape():
+    c = _scaled_case("resnet50_w8")
+    weights = c.weights(DEV)
+    run_parity(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, c.steps, weights, lambda t: c.grads(t, DEV), momentum=0.9,
+               residual_every=1000)
