@@ -25,7 +25,6 @@ struct iwp_ctx {
   int64_t leader_override = -1;
   bool force_scalar = false;
   bool speculate = true;
-  bool fused_select = false;  // one kernel per pass with a last-CTA decision: fewer launches, measured slower
   cudaStream_t stream = nullptr;
   cudaStream_t side = nullptr;       // the one-CTA path of small layers runs here, beside the tiled path
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_fork2 = nullptr, ev_join2 = nullptr;
@@ -49,7 +48,6 @@ struct iwp_ctx {
   uint32_t* sel_slot = nullptr;   // [K] slot position of each entry of the leader's list, or REF_NONE
   uint2* lead_lane = nullptr;     // [segment][32] the leader's staged mask | count << 16, lane prefix
   uint32_t* lead_tot = nullptr;   // [segment] the leader's per-round totals
-  uint32_t* d_done = nullptr;     // per pair: chunks that finished the current histogram pass
   uint32_t* chunk_sfx = nullptr;  // [W][chunk][1024] suffix sums of each chunk's last-pass histogram
   uint32_t* zmask = nullptr;      // residuals sent in the last step and not yet zeroed (lazy step (g))
   uint64_t zmask_words = 0;
@@ -104,11 +102,11 @@ void stage_clear(iwp_ctx* c) {
 
 struct Sizes {
   uint64_t acc, layers, tiles, chunks, small_ids, large_ids, state, hist, chunk_cnt, sel_idx, sel_val, status;
-  uint64_t info, cand_key, cand_val, cand_idx, cand_cnt, guess, side_val, sel_slot, lead_lane, lead_tot, zmask, done, chunk_sfx;
+  uint64_t info, cand_key, cand_val, cand_idx, cand_cnt, guess, side_val, sel_slot, lead_lane, lead_tot, zmask, chunk_sfx;
   uint64_t total() const {
     return acc + layers + tiles + chunks + small_ids + large_ids + state + hist + chunk_cnt + sel_idx + sel_val +
            status + info + cand_key + cand_val + cand_idx + cand_cnt + guess + side_val + sel_slot + lead_lane +
-           lead_tot + zmask + done + chunk_sfx;
+           lead_tot + zmask + chunk_sfx;
   }
 };
 
@@ -145,7 +143,6 @@ Sizes sizes_of(const Plan& p) {
   s.lead_lane = at_least(segs * 32 * sizeof(uint2));
   s.lead_tot = at_least(segs * sizeof(uint32_t));
   s.zmask = ((p.N >> 9) + 2) * 16 * sizeof(uint32_t);  // 32 sixteen-bit fields per 512 elements
-  s.done = at_least(pairs * sizeof(uint32_t));
   s.chunk_sfx = at_least(W * p.chunks.size() * pass_bins(N_PASSES - 1) * sizeof(uint32_t));
   return s;
 }
@@ -195,7 +192,6 @@ void free_all(iwp_ctx* c) {
   cudaFree(c->lead_lane);
   cudaFree(c->lead_tot);
   cudaFree(c->zmask);
-  cudaFree(c->d_done);
   cudaFree(c->chunk_sfx);
   cudaFree(c->sel_idx);
   cudaFree(c->sel_val);
@@ -314,20 +310,13 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
     dim3 cgrid(n_chunks, static_cast<unsigned>(W));
     for (int pass = 0; pass < N_PASSES; ++pass) {
-      if (c->fused_select) {  // the last CTA of each pair decides the digit (and, in the last pass, the counts)
-        k_hist<VEC, true><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_info, c->cand_key,
-                                                    c->cand_cnt, c->d_state, c->d_hist, c->d_done, c->chunk_sfx,
-                                                    c->d_chunk_cnt, c->d_status, c->eps, N, W, pass, n_chunks);
-        IWP_LAUNCH_CHECK(c);
-      } else {
-        k_hist<VEC, false><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_info, c->cand_key,
-                                                     c->cand_cnt, c->d_state, c->d_hist, c->d_done, c->chunk_sfx,
-                                                     c->d_chunk_cnt, c->d_status, c->eps, N, W, pass, n_chunks);
-        IWP_LAUNCH_CHECK(c);
-        k_find_digit<<<c->n_pairs, THREADS, 0, s>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->d_status,
-                                                    W, pass);
-        IWP_LAUNCH_CHECK(c);
-      }
+      k_hist<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_info, c->cand_key,
+                                            c->cand_cnt, c->d_state, c->d_hist, c->chunk_sfx, c->d_chunk_cnt, c->eps, N,
+                                            W, pass, n_chunks);
+      IWP_LAUNCH_CHECK(c);
+      k_find_digit<<<c->n_pairs, THREADS, 0, s>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->d_status, W,
+                                                  pass);
+      IWP_LAUNCH_CHECK(c);
     }
   }
   stage_mark_at(c, 4);
@@ -337,7 +326,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     // The reduction needs the leader's list only: write that one here and the other workers' lists on
     // the side stream, beside the reduction; they are joined at the end of the step.
     const bool split = spec && W > 1 && c->side != nullptr;
-    const uint32_t* sfx = c->fused_select ? nullptr : c->chunk_sfx;
+    const uint32_t* sfx = c->chunk_sfx;
     if (split) {
       if (cudaEventRecord(c->ev_fork2, s) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork2, 0) != cudaSuccess) {
         cudaGetLastError();
@@ -478,7 +467,6 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
   A(&c->lead_lane, sz.lead_lane);
   A(&c->lead_tot, sz.lead_tot);
   A(&c->zmask, sz.zmask);
-  A(&c->d_done, sz.done);
   A(&c->chunk_sfx, sz.chunk_sfx);
   A(&c->sel_idx, sz.sel_idx);
   A(&c->sel_val, sz.sel_val);
@@ -508,7 +496,6 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
   ok = ok && cudaMemset(c->cand_cnt, 0, sz.cand_cnt) == cudaSuccess;
   ok = ok && cudaMemset(c->sel_slot, 0xff, sz.sel_slot) == cudaSuccess;
   ok = ok && cudaMemset(c->zmask, 0, sz.zmask) == cudaSuccess;
-  ok = ok && cudaMemset(c->d_done, 0, sz.done) == cudaSuccess;
   c->zmask_words = sz.zmask / sizeof(uint32_t);
   for (uint32_t l : p.large_layers) {
     if (p.layers[l].sample > c->max_sample) c->max_sample = p.layers[l].sample;
@@ -711,7 +698,6 @@ int iwp_reset(iwp_ctx* c) {
   const Sizes sz = sizes_of(c->plan);
   bool ok = cudaMemsetAsync(c->acc, 0, sz.acc, c->stream) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->zmask, 0, sz.zmask, c->stream) == cudaSuccess;
-  ok = ok && cudaMemsetAsync(c->d_done, 0, sz.done, c->stream) == cudaSuccess;
   c->zero_pending = false;
   ok = ok && cudaMemsetAsync(c->d_hist, 0, sz.hist, c->stream) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->d_status, 0, sz.status, c->stream) == cudaSuccess;
@@ -741,11 +727,6 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
     cudaStreamSynchronize(c->stream);
     stage_clear(c);
     c->time_stages = static_cast<int>(v);
-    return IWP_OK;
-  }
-  if (!std::strcmp(key, "fused_select")) {
-    if (v != 0 && v != 1) return IWP_ERR_INVALID;
-    c->fused_select = v != 0;
     return IWP_OK;
   }
   if (!std::strcmp(key, "speculate")) {
@@ -893,9 +874,8 @@ int run_select_static(StaticScratch* s, const float* residual, const float* weig
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   dim3 grid(n_chunks, 1);
   for (int pass = 0; pass < N_PASSES; ++pass) {
-    k_hist<VEC, false><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr,
-                                                 &s->state, s->hist, nullptr, nullptr, nullptr, &s->status, eps, 0, 1,
-                                                 pass, n_chunks);
+    k_hist<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr, &s->state,
+                                          s->hist, nullptr, nullptr, eps, 0, 1, pass, n_chunks);
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
     k_find_digit<<<1, THREADS, 0, st>>>(&s->state, s->hist, &s->layer, &s->large_id, &s->status, 1, pass);
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;

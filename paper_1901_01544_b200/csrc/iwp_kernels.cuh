@@ -689,25 +689,21 @@ __device__ __forceinline__ void for_each_candidate(const Chunk& c, int w, int W,
 // ---------------------------------------------------------------------------------------
 
 // One histogram pass over a chunk: keys that match the prefix found so far are counted by
-// their next digit.  grid = (chunks, W).
-//
-// FUSED: the CTA that finishes a pair's pass last (a ticket from an atomic counter tells it; nobody
-// waits for anybody) also takes the digit decision for the pair, so no separate kernel runs between
-// passes.  In the last pass every CTA additionally leaves, per chunk, the number of keys above the
-// prefix and the suffix sums of its low-digit histogram; from those the deciding CTA derives every
-// chunk's (#keys > T, #keys == T), which the compaction needs for its list offsets.
-template <bool VEC, bool FUSED>
+// their next digit.  grid = (chunks, W).  In the last pass every CTA additionally leaves, per chunk,
+// the number of keys above the prefix and the suffix sums of its low-digit histogram; with the
+// threshold known, the compaction derives every chunk's (#keys > T, #keys == T) from those without
+// another look at the keys (chunk_sfx == nullptr: skipped, a counting kernel runs instead).
+template <bool VEC>
 __global__ void __launch_bounds__(THREADS)
     k_hist(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
            const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
-           const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt, uint2* state,
-           uint32_t* __restrict__ hist, uint32_t* __restrict__ done, uint32_t* __restrict__ chunk_sfx,
-           uint2* chunk_cnt, int* __restrict__ status, float eps, uint64_t N, int W, int pass, uint32_t n_chunks) {
+           const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt,
+           const uint2* __restrict__ state,
+           uint32_t* __restrict__ hist, uint32_t* __restrict__ chunk_sfx, uint2* __restrict__ chunk_cnt, float eps,
+           uint64_t N, int W, int pass, uint32_t n_chunks) {
   __shared__ uint32_t sh[NBINS];
-  __shared__ uint32_t sh_scan[THREADS];
   __shared__ uint32_t sh_warp[WARPS];
-  __shared__ uint32_t res[4];
-  __shared__ uint32_t sh_above, sh_last;
+  __shared__ uint32_t sh_above;
   const Chunk c = chunks[blockIdx.x];
   const int w = blockIdx.y;
   const LayerDesc L = layers[c.layer];
@@ -795,48 +791,6 @@ __global__ void __launch_bounds__(THREADS)
     uint32_t* dst = chunk_sfx + (static_cast<uint64_t>(w) * n_chunks + blockIdx.x) * pass_bins(N_PASSES - 1);
     reinterpret_cast<uint4*>(dst)[threadIdx.x] = sfx;
     if (threadIdx.x == 0) chunk_cnt[static_cast<uint64_t>(w) * n_chunks + blockIdx.x] = make_uint2(sh_above, 0u);
-  }
-  if (!FUSED) return;
-  // ticket: the CTA that arrives last sees every other CTA's contribution
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const uint32_t ticket = atomicAdd(&done[pair], 1u);
-    sh_last = (ticket == L.n_chunks - 1) ? 1u : 0u;
-  }
-  __syncthreads();
-  if (!sh_last) return;
-  __threadfence();
-  for (int b = threadIdx.x; b < nb; b += THREADS) {
-    sh[b] = __ldcg(&gh[b]);
-    gh[b] = 0;  // ready for the next pass / step
-  }
-  if (threadIdx.x == 0) done[pair] = 0;
-  __syncthreads();
-  find_digit(sh, nb, st_in.y, sh_scan, res);
-  const bool found = res[2] != 0;
-  const uint32_t digit = res[0], krem = res[1];
-  if (threadIdx.x == 0) {
-    if (found) {
-      state[pair] = make_uint2(st_in.x | (digit << shift), krem);
-    } else {
-      atomicMin(status, STATUS_INTERNAL);
-      state[pair] = make_uint2(0xffffffffu, 0u);  // selects nothing
-    }
-  }
-  if (last_pass) {  // per chunk of the pair: (#keys > T, #keys == T)
-    for (uint32_t j = L.first_chunk + threadIdx.x; j < L.first_chunk + L.n_chunks; j += THREADS) {
-      const uint64_t at = static_cast<uint64_t>(w) * n_chunks + j;
-      uint32_t gt = 0, eq = 0;
-      if (found) {
-        const uint32_t* sfx = chunk_sfx + at * pass_bins(N_PASSES - 1);
-        const uint32_t s_d = __ldcg(&sfx[digit]);
-        const uint32_t s_d1 = (digit + 1 < static_cast<uint32_t>(nb)) ? __ldcg(&sfx[digit + 1]) : 0u;
-        gt = __ldcg(reinterpret_cast<const unsigned int*>(&chunk_cnt[at])) + s_d1;
-        eq = s_d - s_d1;
-      }
-      chunk_cnt[at] = make_uint2(gt, eq);
-    }
   }
 }
 
