@@ -30,6 +30,10 @@ def lib() -> C.CDLL:
         L.oracle_threads_used.restype = i32
         L.oracle_set_leader_override.argtypes = [vp, i32]
         L.oracle_set_momentum.argtypes = [vp, f32]
+        L.oracle_set_thresholds.argtypes = [vp, vp]
+        L.oracle_threshold_list_length.argtypes = [vp]
+        L.oracle_threshold_list_length.restype = i64
+        L.oracle_get_threshold_list.argtypes = [vp, vp, vp]
         L.oracle_total.argtypes = [vp]
         L.oracle_total.restype = i64
         L.oracle_total_keep.argtypes = [vp]
@@ -115,6 +119,22 @@ class Oracle:
         k = np.empty(self.L, dtype=np.int64)
         lib().oracle_get_layout(self._h, _p(off), _p(k))
         return off.tolist(), k.tolist()
+
+    def set_thresholds(self, thr):
+        """Per-layer absolute thresholds: Algorithm 1 as printed (None: back to the ratio mode)."""
+        if thr is None:
+            lib().oracle_set_thresholds(self._h, None)
+            return
+        a = np.ascontiguousarray(thr, dtype=np.float32)
+        assert a.size == self.L
+        lib().oracle_set_thresholds(self._h, _p(a))
+
+    def threshold_list(self) -> Tuple[np.ndarray, np.ndarray]:
+        n = int(lib().oracle_threshold_list_length(self._h))
+        idx = np.empty(n, dtype=np.uint32)
+        val = np.empty(n, dtype=np.float32)
+        lib().oracle_get_threshold_list(self._h, _p(idx), _p(val))
+        return idx, val
 
     def set_momentum(self, m: float):
         lib().oracle_set_momentum(self._h, float(m))

@@ -25,6 +25,9 @@
 //     "randomly choose a node and broadcast its important gradient index").
 //   * Eq. 3's momentum acts on the locally kept residual: G <- m * G + grad (two roundings);
 //     m = 1, the default, is the plain accumulation of Section 3.2.
+//   * threshold mode is Algorithm 1 as printed: only the chosen node forms a mask, per layer
+//     Mask = importance > thr[layer] (strict), the index set has whatever size results, and no
+//     other worker makes a selection of its own.
 //   * the ring all-reduce is a sum in ascending worker order, fp32, without the 1/N
 //     factor (the caller pre-scales gradients as in Eq. 1).
 //
@@ -59,6 +62,10 @@ struct Oracle {
   int32_t leader_override = -1;
   int threads = 0;
   float momentum = 1.0f;         // Eq. 3: the local residual enters the next step scaled by m
+  bool threshold_mode = false;   // Algorithm 1 as printed: Mask <- importance > thr on the chosen node
+  std::vector<float> thr;        // per-layer thresholds (threshold mode)
+  std::vector<uint32_t> thr_idx; // the chosen node's index set of the last step (threshold mode)
+  std::vector<float> thr_val;    // its accumulated values at those indices, before zeroing
   std::vector<float> acc;        // [W][N] residuals
   std::vector<uint32_t> sel_idx; // [W][K] ascending global indices per layer segment
   std::vector<float> sel_val;    // [W][K] accumulated value at that index (before zeroing)
@@ -178,6 +185,18 @@ int32_t oracle_threads_used(void* h) {
   return 1;
 #endif
 }
+// Switches to Algorithm 1 as printed, with one absolute threshold per layer (NULL: back to the ratio).
+void oracle_set_thresholds(void* h, const float* thr) {
+  Oracle* o = static_cast<Oracle*>(h);
+  o->threshold_mode = thr != nullptr;
+  if (thr) o->thr.assign(thr, thr + o->n.size());
+}
+int64_t oracle_threshold_list_length(void* h) { return static_cast<int64_t>(static_cast<Oracle*>(h)->thr_idx.size()); }
+void oracle_get_threshold_list(void* h, uint32_t* idx, float* val) {
+  Oracle* o = static_cast<Oracle*>(h);
+  std::copy(o->thr_idx.begin(), o->thr_idx.end(), idx);
+  std::copy(o->thr_val.begin(), o->thr_val.end(), val);
+}
 void oracle_set_momentum(void* h, float m) { static_cast<Oracle*>(h)->momentum = m; }
 void oracle_set_leader_override(void* h, int32_t leader) { static_cast<Oracle*>(h)->leader_override = leader; }
 int64_t oracle_total(void* h) { return static_cast<Oracle*>(h)->N; }
@@ -221,6 +240,10 @@ void oracle_get_mask(void* h, uint8_t* dst) {
   Oracle* o = static_cast<Oracle*>(h);
   std::memset(dst, 0, o->N);
   if (o->leader < 0) return;
+  if (o->threshold_mode) {
+    for (uint32_t i : o->thr_idx) dst[i] = 1;
+    return;
+  }
   const uint32_t* S = &o->sel_idx[static_cast<size_t>(o->leader) * o->K];
   for (int64_t j = 0; j < o->K; ++j) dst[S[j]] = 1;
 }
@@ -245,6 +268,34 @@ void oracle_step(void* h, const float* grads, const float* weights, float* updat
     o->acc[e] = carried + grads[e];
   }
 
+  o->leader = o->leader_override >= 0 ? o->leader_override : leader_of(o->seed, static_cast<uint64_t>(o->t), W);
+  if (o->threshold_mode) {
+    // Algorithm 1 as printed: the chosen node r alone forms Mask_r = |G_r / w| > thr, layer by layer;
+    // every node then splits its accumulated gradient by that mask
+    const float* ar = &o->acc[static_cast<size_t>(o->leader) * N];
+    o->thr_idx.clear();
+    o->thr_val.clear();
+    for (int l = 0; l < L; ++l) {
+      for (int64_t i = o->off[l]; i < o->off[l] + o->n[l]; ++i) {
+        if (importance(ar[i], weights[i], o->eps) > o->thr[l]) {
+          o->thr_idx.push_back(static_cast<uint32_t>(i));
+          o->thr_val.push_back(ar[i]);
+        }
+      }
+    }
+    for (int64_t i = 0; i < N; ++i) update[i] = 0.0f;
+    for (size_t j = 0; j < o->thr_idx.size(); ++j) {
+      const size_t i = o->thr_idx[j];
+      float s = o->acc[i];
+      for (int32_t w = 1; w < W; ++w) s = s + o->acc[static_cast<size_t>(w) * N + i];
+      update[i] = 0.0f + s;
+    }
+    for (size_t j = 0; j < o->thr_idx.size(); ++j)
+      for (int32_t w = 0; w < W; ++w) o->acc[static_cast<size_t>(w) * N + o->thr_idx[j]] = 0.0f;
+    o->t += 1;
+    return;
+  }
+
   // (b)-(d) per worker and layer: importance, keep the k best, list them in index order
 #pragma omp parallel num_threads(nthreads)
   {
@@ -266,7 +317,6 @@ void oracle_step(void* h, const float* grads, const float* weights, float* updat
   }
 
   // (e) the randomly chosen node supplies the index set
-  o->leader = o->leader_override >= 0 ? o->leader_override : leader_of(o->seed, static_cast<uint64_t>(o->t), W);
   const uint32_t* S = &o->sel_idx[static_cast<size_t>(o->leader) * K];
 
   // (f) sum over workers in ascending order at the shared indices, into a zeroed dense update

@@ -412,3 +412,93 @@ def test_momentum_geometric_carry_closed_form():
         orc.step(g, w)
         want = 2.0 - 0.5 ** t
         assert np.all(orc.residual(0)[1:] == np.float32(want)), t
+
+
+# ---------------------------------------------------------------- Algorithm 1 as printed: absolute thresholds
+
+
+def _brute_threshold_step(acc, grads, weights, layers, thr, leader, eps, m=1.0):
+    """Pure-Python statement of one threshold-mode step on lists of numpy float32 scalars."""
+    W, N = len(acc), len(weights)
+    for w in range(W):
+        for i in range(N):
+            acc[w][i] = F(F(F(m) * acc[w][i]) + F(grads[w][i]))
+    S, o = [], 0
+    for n, t in zip(layers, thr):
+        S += [o + i for i in range(n) if importance(acc[leader][o + i], weights[o + i], eps) > F(t)]
+        o += n
+    upd = [F(0)] * N
+    for i in S:
+        s = acc[0][i]
+        for w in range(1, W):
+            s = F(s + acc[w][i])
+        upd[i] = F(F(0) + s)
+    vals = [acc[leader][i] for i in S]
+    for i in S:
+        for w in range(W):
+            acc[w][i] = F(0)
+    return S, vals, np.array(upd, np.float32)
+
+
+def test_threshold_mode_equals_bruteforce():
+    layers, W = [7, 1, 20, 4], 3
+    N = sum(layers)
+    rng = np.random.default_rng(31)
+    weights = (rng.integers(-2, 3, N) * 0.5).astype(np.float32)  # includes zeros
+    thr = [0.5, 0.0, 1.0, 1e9]
+    orc = oracle.Oracle(layers, W, 2.0, 1e-8, seed=4)
+    orc.set_thresholds(thr)
+    acc = [[F(0)] * N for _ in range(W)]
+    for t in range(5):
+        grads = (rng.integers(-4, 5, size=(W, N)) / 4.0).astype(np.float32)  # importances hit the thresholds exactly
+        upd = orc.step(grads, weights)
+        S, vals, upd_bf = _brute_threshold_step(acc, grads, weights, layers, thr, orc.leader, F(1e-8))
+        idx, val = orc.threshold_list()
+        assert idx.tolist() == S and np.array_equal(u32(val), u32(np.array(vals, np.float32)))
+        assert np.array_equal(u32(upd), u32(upd_bf))
+        for w in range(W):
+            assert np.array_equal(u32(orc.residual(w)), u32(np.array(acc[w], np.float32)))
+        assert orc.mask().tolist() == [1 if i in S else 0 for i in range(N)]
+        assert not any(i >= sum(layers[:3]) for i in S)  # the last layer's threshold of 1e9 is never passed
+
+
+def test_threshold_mode_hand_worked_and_strictness():
+    # weights 1, eps negligible: importance = |residual|.  thr = 0.5 is strict: 0.5 itself stays.
+    orc = oracle.Oracle([4], 2, 2.0, 1e-8, seed=0)
+    orc.set_thresholds([0.5])
+    orc.set_leader_override(1)
+    w = np.ones(4, np.float32)
+    g = np.array([[1.0, 0.25, 0.5, -2.0], [0.5, 0.75, -0.5, 0.25]], np.float32)
+    upd = orc.step(g, w)  # node 1's mask: |0.5|>0.5 no, 0.75 yes, |-0.5| no, 0.25 no  ->  S = {1}
+    assert orc.threshold_list()[0].tolist() == [1] and upd.tolist() == [0, 1.0, 0, 0]
+    assert orc.residual(0).tolist() == [1.0, 0, 0.5, -2.0] and orc.residual(1).tolist() == [0.5, 0, -0.5, 0.25]
+    orc.set_leader_override(0)
+    upd = orc.step(np.zeros((2, 4), np.float32), w)  # node 0: 1.0 and |-2| pass  ->  S = {0, 3}
+    assert orc.threshold_list()[0].tolist() == [0, 3] and upd.tolist() == [1.5, 0, 0, -1.75]
+    # thresholds 0 and +inf: everything non-zero / nothing
+    o2 = oracle.Oracle([3, 3], 1, 2.0, 1e-8, seed=0)
+    o2.set_thresholds([0.0, float("inf")])
+    u = o2.step(np.array([[1, 0, -1, 5, 5, 5]], np.float32), np.ones(6, np.float32))
+    assert o2.threshold_list()[0].tolist() == [0, 2] and u.tolist() == [1, 0, -1, 0, 0, 0]
+
+
+def test_threshold_at_the_kplus1_th_importance_reproduces_the_ratio_mode():
+    # with thr = the (k+1)-th largest importance of the chosen node's layer (continuous values, no ties)
+    # the thresholded mask is that node's top-k set, so both modes must give the same update
+    layers, W, R = [4000, 300], 3, 16.0
+    rng, weights = _random_problem(layers, W, 55, zero_frac=0.0)
+    N = sum(layers)
+    grads = rng.normal(scale=1e-3, size=(W, N)).astype(np.float32)
+    ratio = oracle.Oracle(layers, W, R, 1e-8, seed=9)
+    upd_ratio = ratio.step(grads, weights)
+    off, ks = ratio.layout()
+    imp = np.abs(grads[ratio.leader]) / (np.abs(weights) + F(1e-8))
+    thr = [np.sort(imp[o:o + n])[::-1][k] for o, n, k in zip(off, layers, ks)]
+    th = oracle.Oracle(layers, W, R, 1e-8, seed=9)
+    th.set_thresholds(thr)
+    upd_thr = th.step(grads, weights)
+    assert th.leader == ratio.leader
+    assert np.array_equal(th.threshold_list()[0], ratio.selection(ratio.leader)[0])
+    assert np.array_equal(u32(upd_thr), u32(upd_ratio))
+    for w in range(W):
+        assert np.array_equal(u32(th.residual(w)), u32(ratio.residual(w)))
