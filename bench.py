@@ -207,7 +207,14 @@ def run_ours(args):
         n_sets = args.grad_sets
     sets = [c.grads(t, dev) for t in range(n_sets)]
     update = torch.empty(N, dtype=torch.float32, device=dev)
-    pr = Pruner(c.layer_sizes, W, c.ratio, c.eps, c.seed)
+    if args.mode == "threshold":
+        # Algorithm 1 as printed: absolute per-layer thresholds, set near the step-0 top-1/64 point of this
+        # workload's value recipe (weight tensors 0.4; zero-initialised biases rank by |residual| / eps)
+        thr = [0.4 if (c.tensors is None or tn.kind == "weight") else 2.0e4
+               for tn in (c.tensors or [None] * len(c.layer_sizes))]
+        pr = Pruner(c.layer_sizes, W, None, c.eps, c.seed, thresholds=thr)
+    else:
+        pr = Pruner(c.layer_sizes, W, c.ratio, c.eps, c.seed)
     K = pr.K
     if args.speculate is not None:
         pr.set_option("speculate", args.speculate)
@@ -244,6 +251,8 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     launches = pr.stat("launches") - launches0
     pr.check()
+    if args.mode == "threshold":
+        K = pr.list_length()  # size of the last step's index set
     k1_ms_live = pr.stat("time_accumulate_ns") / 1e6 / args.steps
     spec = {"pairs": pr.stat("spec_pairs"), "failed": pr.stat("spec_failed")}
     stage_steps = 0 if args.no_stage_times else max(1, min(args.steps, args.stage_steps))
@@ -313,7 +322,7 @@ def run_ours(args):
 
     # CPU baseline: the oracle as it stands, a bounded sample (a few full steps) on this machine's cores
     cpu = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and args.mode == "ratio":
         w_host = weights.cpu().numpy()
         g_host = [sets[i].cpu().numpy() for i in range(min(2, n_sets))]
         sps, threads, dt = oracle_timing(c, w_host, lambda t: g_host[t % len(g_host)], args.cpu_steps, 1)
@@ -324,7 +333,8 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
-        "config": {"workload": c.name, "W": W, "N": N, "K": K, "ratio": c.ratio, "layers": len(c.layer_sizes),
+        "config": {"workload": c.name, "mode": args.mode, "W": W, "N": N, "K": K,
+                   "ratio": c.ratio if args.mode == "ratio" else None, "layers": len(c.layer_sizes),
                    "l2_policy": f"inputs larger than L2: {grad_bytes * 3 / 1e9:.2f} GB streamed per step, "
                                 f"{n_sets} gradient batches cycled",
                    "multi_gpu": "independent replicas (the path has no inter-GPU exchange)",
@@ -356,6 +366,9 @@ def main():
     ap.add_argument("--cpu-steps", type=int, default=15)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--speculate", type=int, default=None, choices=[0, 1])
+    ap.add_argument("--mode", default="ratio", choices=["ratio", "threshold"],
+                    help="ratio: exact layer-wise top-k at the configured compression (headline); threshold: "
+                         "absolute per-layer thresholds on the chosen node (Algorithm 1 as printed)")
     ap.add_argument("--layers", default=None, help="lo:hi - only these layers of the workload (small profiling case)")
     ap.add_argument("--grad-sets", type=int, default=None, help="distinct gradient batches kept on the device")
     ap.add_argument("--no-e2e", action="store_true")

@@ -45,7 +45,8 @@ enum {
   IWP_ERR_OOM = -2,      /* device or host allocation failed */
   IWP_ERR_CUDA = -3,     /* a CUDA runtime call or kernel launch failed */
   IWP_ERR_INTERNAL = -4, /* a device-side conservation check failed (counts do not add up) */
-  IWP_ERR_TIMEOUT = -5   /* a bounded device-side wait gave up (unused: no kernel here waits) */
+  IWP_ERR_TIMEOUT = -5,  /* a bounded device-side wait gave up (unused: no kernel here waits) */
+  IWP_ERR_CAPACITY = -6  /* threshold mode: the index set did not fit the list (see iwp_create_threshold) */
 };
 
 /* Human-readable name of a status code; never NULL. */
@@ -87,6 +88,28 @@ int iwp_plan_sizes(const int64_t* layer_sizes_host, int32_t n_layers, int32_t W,
  * N >= 2^32), IWP_ERR_OOM, IWP_ERR_CUDA; *out is NULL on error. */
 int iwp_create(iwp_ctx** out, const int64_t* layer_sizes_host, int32_t n_layers, int32_t W, double ratio, float eps,
                uint64_t seed);
+
+/* Absolute-threshold mode: Algorithm 1 of the paper as printed.  Per step, only the chosen node r forms a
+ * mask, layer by layer, Mask_r = |acc_r / w| > thr[layer] (strict, with the eps guard in the denominator);
+ * its index set S has whatever size results; every node then contributes acc[w][S] to the ordered sum,
+ * update[S] = sum, and acc[w][S] = 0.  No other worker makes a selection of its own.  The paper used
+ * thresholds of 0.005 ... 0.1 (Section 4.1).
+ *   max_list   capacity of the index list in entries; 0 or anything above N means N.  If a step's index
+ *              set is longer, IWP_ERR_CAPACITY is raised in the status word and that step's update is
+ *              incomplete.
+ * A context created here takes iwp_set_thresholds() before its first step; iwp_get_selection() is valid for
+ * the last step's leader only and copies max_list entries of which the first iwp_get_list_length() are
+ * meaningful; iwp_get_layout() reports keep counts of 0.  Same errors as iwp_create(). */
+int iwp_create_threshold(iwp_ctx** out, const int64_t* layer_sizes_host, int32_t n_layers, int32_t W, float eps,
+                         uint64_t seed, int64_t max_list);
+
+/* n_layers thresholds (host array, copied), each >= 0; +inf sends nothing from that layer.  Synchronises
+ * the stream.  Errors: IWP_ERR_INVALID (NULL, not a threshold-mode context, negative or NaN value). */
+int iwp_set_thresholds(iwp_ctx* ctx, const float* thr_host);
+
+/* Number of entries of the last step's index set (threshold mode: synchronises the stream and reads
+ * it from the device; ratio mode: K). */
+int iwp_get_list_length(iwp_ctx* ctx, int64_t* len_host);
 
 /* Synchronises the context's stream and frees everything iwp_create() allocated.
  * NULL is a no-op returning IWP_OK. */

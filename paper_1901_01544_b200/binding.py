@@ -14,13 +14,14 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libiwp.so")
 
 IWP_OK, IWP_ERR_INVALID, IWP_ERR_OOM, IWP_ERR_CUDA, IWP_ERR_INTERNAL, IWP_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+IWP_ERR_CAPACITY = -6
 
 EXPORTS = [
     "iwp_strerror", "iwp_keep_count", "iwp_leader_at", "iwp_plan_sizes", "iwp_create", "iwp_destroy",
     "iwp_set_stream", "iwp_step", "iwp_step_host", "iwp_sync_status", "iwp_get_layout", "iwp_get_sizes",
     "iwp_get_step", "iwp_set_step", "iwp_get_leader", "iwp_get_residual", "iwp_set_residual",
     "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat", "iwp_select_static",
-    "iwp_set_momentum",
+    "iwp_set_momentum", "iwp_create_threshold", "iwp_set_thresholds", "iwp_get_list_length",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -47,6 +48,9 @@ def lib() -> C.CDLL:
         L.iwp_leader_at.restype, L.iwp_leader_at.argtypes = i32, [u64, u64, i32]
         L.iwp_plan_sizes.argtypes = [vp, i32, i32, f64, vp]
         L.iwp_create.argtypes = [C.POINTER(vp), vp, i32, i32, f64, f32, u64]
+        L.iwp_create_threshold.argtypes = [C.POINTER(vp), vp, i32, i32, f32, u64, i64]
+        L.iwp_set_thresholds.argtypes = [vp, vp]
+        L.iwp_get_list_length.argtypes = [vp, vp]
         L.iwp_destroy.argtypes = [vp]
         L.iwp_set_stream.argtypes = [vp, vp]
         L.iwp_set_momentum.argtypes = [vp, f32]
@@ -107,6 +111,14 @@ def iwp_create(layer_sizes: Sequence[int], W: int, ratio: float, eps: float, see
     return h
 
 
+def iwp_create_threshold(layer_sizes: Sequence[int], W: int, eps: float, seed: int, max_list: int = 0) -> C.c_void_p:
+    arr = (C.c_int64 * len(layer_sizes))(*layer_sizes)
+    h = C.c_void_p()
+    _check(lib().iwp_create_threshold(C.byref(h), arr, len(layer_sizes), W, eps, seed, max_list),
+           "iwp_create_threshold")
+    return h
+
+
 def iwp_destroy(h) -> None:
     _check(lib().iwp_destroy(h), "iwp_destroy")
 
@@ -134,18 +146,27 @@ def iwp_select_static(residual_ptr: int, weights_ptr: int, n: int, ratio: float,
 class Pruner:
     """Owns one iwp context; takes torch CUDA tensors (device memory and stream only)."""
 
-    def __init__(self, layer_sizes: Sequence[int], W: int, ratio: float, eps: float = 1e-8, seed: int = 0):
+    def __init__(self, layer_sizes: Sequence[int], W: int, ratio: Optional[float], eps: float = 1e-8, seed: int = 0,
+                 thresholds: Optional[Sequence[float]] = None, max_list: int = 0):
+        """ratio mode: `ratio` = compression factor.  Threshold mode (Algorithm 1 as printed): pass
+        ratio=None and per-layer `thresholds`; `max_list` bounds the index list (0 = N entries)."""
         import torch
 
         if not torch.cuda.is_available():
             raise RuntimeError("iwp needs a CUDA device; there is no CPU fallback")
         self._torch = torch
-        self._h = iwp_create(list(layer_sizes), W, float(ratio), float(eps), int(seed))
+        self.threshold_mode = ratio is None
+        if self.threshold_mode:
+            self._h = iwp_create_threshold(list(layer_sizes), W, float(eps), int(seed), int(max_list))
+        else:
+            self._h = iwp_create(list(layer_sizes), W, float(ratio), float(eps), int(seed))
         out = (C.c_int64 * 4)()
         _check(lib().iwp_get_sizes(self._h, out), "iwp_get_sizes")
         self.N, self.K, self.L, self.W = (int(v) for v in out)
         self.device = torch.device("cuda", torch.cuda.current_device())
         self.use_current_stream()
+        if thresholds is not None:
+            self.set_thresholds(thresholds)
 
     # life cycle
     def close(self) -> None:
@@ -181,6 +202,15 @@ class Pruner:
             assert (not x.is_cuda) and x.dtype == t.float32 and x.is_contiguous() and x.numel() == n
         iwp_step_host(self._h, grads.data_ptr(), weights.data_ptr(), update.data_ptr())
         return update
+
+    def set_thresholds(self, thr: Sequence[float]) -> None:
+        arr = (C.c_float * self.L)(*[float(x) for x in thr])
+        _check(lib().iwp_set_thresholds(self._h, arr), "iwp_set_thresholds")
+
+    def list_length(self) -> int:
+        v = C.c_int64()
+        _check(lib().iwp_get_list_length(self._h, C.byref(v)), "iwp_get_list_length")
+        return int(v.value)
 
     def set_momentum(self, m: float) -> None:
         _check(lib().iwp_set_momentum(self._h, float(m)), "iwp_set_momentum")

@@ -49,6 +49,14 @@ struct iwp_ctx {
   uint2* lead_lane = nullptr;     // [segment][32] the leader's staged mask | count << 16, lane prefix
   uint32_t* lead_tot = nullptr;   // [segment] the leader's per-round totals
   uint32_t* chunk_sfx = nullptr;  // [W][chunk][1024] suffix sums of each chunk's last-pass histogram
+  // absolute-threshold mode (Algorithm 1 as printed)
+  bool threshold_mode = false;
+  uint64_t list_cap = 0;          // capacity of the single index list
+  bool thr_set = false;
+  uint32_t* d_thr = nullptr;      // [layer] fp32 patterns of the thresholds
+  uint32_t* d_tcnt = nullptr;     // [chunk] selected elements of the chunk
+  uint32_t* d_toff = nullptr;     // [chunk] list offset of the chunk
+  uint32_t* d_list_len = nullptr; // length of the last step's index list
   uint32_t* zmask = nullptr;      // residuals sent in the last step and not yet zeroed (lazy step (g))
   uint64_t zmask_words = 0;
   bool zero_pending = false;      // zmask may hold marks
@@ -112,10 +120,11 @@ struct Sizes {
 
 uint64_t at_least(uint64_t b) { return b ? b : 16; }
 
-Sizes sizes_of(const Plan& p) {
+Sizes sizes_of(const Plan& p, bool threshold_mode = false, uint64_t list_cap = 0) {
   Sizes s;
   const uint64_t W = static_cast<uint64_t>(p.W);
-  const uint64_t pairs = W * p.large_layers.size();
+  // the threshold mode selects on one worker only and needs none of the per-pair select scratch
+  const uint64_t pairs = threshold_mode ? 0 : W * p.large_layers.size();
   s.acc = W * p.N * sizeof(float);
   s.layers = p.layers.size() * sizeof(LayerDesc);
   s.tiles = at_least(p.tiles.size() * sizeof(Tile));
@@ -124,9 +133,9 @@ Sizes sizes_of(const Plan& p) {
   s.large_ids = at_least(p.large_layers.size() * sizeof(uint32_t));
   s.state = at_least(pairs * sizeof(uint2));
   s.hist = at_least(pairs * NBINS * sizeof(uint32_t));
-  s.chunk_cnt = at_least(W * p.chunks.size() * sizeof(uint2));
-  s.sel_idx = W * p.K * sizeof(uint32_t);
-  s.sel_val = W * p.K * sizeof(float);
+  s.chunk_cnt = at_least((threshold_mode ? 0 : W) * p.chunks.size() * sizeof(uint2));
+  s.sel_idx = threshold_mode ? at_least(list_cap * sizeof(uint32_t)) : W * p.K * sizeof(uint32_t);
+  s.sel_val = threshold_mode ? at_least(list_cap * sizeof(float)) : W * p.K * sizeof(float);
   s.status = sizeof(int);
   bool any_spec = false;
   for (uint32_t l : p.large_layers) any_spec = any_spec || p.layers[l].sample != 0;
@@ -139,11 +148,11 @@ Sizes sizes_of(const Plan& p) {
   const uint64_t segs = any_spec ? p.tiles.size() * SEGS_PER_TILE : 0;
   s.guess = at_least(pairs * sizeof(uint2));
   s.side_val = at_least(slots * CAND_CAP * sizeof(float));
-  s.sel_slot = at_least(p.K * sizeof(uint32_t));
+  s.sel_slot = at_least((threshold_mode ? 0 : p.K) * sizeof(uint32_t));
   s.lead_lane = at_least(segs * 32 * sizeof(uint2));
   s.lead_tot = at_least(segs * sizeof(uint32_t));
   s.zmask = ((p.N >> 9) + 2) * 16 * sizeof(uint32_t);  // 32 sixteen-bit fields per 512 elements
-  s.chunk_sfx = at_least(W * p.chunks.size() * pass_bins(N_PASSES - 1) * sizeof(uint32_t));
+  s.chunk_sfx = at_least((threshold_mode ? 0 : W) * p.chunks.size() * pass_bins(N_PASSES - 1) * sizeof(uint32_t));
   return s;
 }
 
@@ -192,6 +201,10 @@ void free_all(iwp_ctx* c) {
   cudaFree(c->lead_lane);
   cudaFree(c->lead_tot);
   cudaFree(c->zmask);
+  cudaFree(c->d_thr);
+  cudaFree(c->d_tcnt);
+  cudaFree(c->d_toff);
+  cudaFree(c->d_list_len);
   cudaFree(c->chunk_sfx);
   cudaFree(c->sel_idx);
   cudaFree(c->sel_val);
@@ -392,6 +405,7 @@ const char* iwp_strerror(int status) {
     case IWP_ERR_CUDA: return "CUDA runtime error";
     case IWP_ERR_INTERNAL: return "device-side count check failed";
     case IWP_ERR_TIMEOUT: return "device-side wait timed out";
+    case IWP_ERR_CAPACITY: return "index list longer than its capacity";
     default: return "unknown status";
   }
 }
@@ -415,14 +429,22 @@ int iwp_plan_sizes(const int64_t* layer_sizes, int32_t n_layers, int32_t W, doub
   return IWP_OK;
 }
 
-int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int32_t W, double ratio, float eps,
-               uint64_t seed) {
+}  // extern "C"
+
+namespace {
+
+constexpr uint32_t THRESHOLD_CHUNK_TILES = 16;  // 64 Ki elements per CTA of the threshold-mode select
+
+int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int32_t W, double ratio, float eps,
+                  uint64_t seed, bool threshold_mode, int64_t max_list) {
   if (!out) return IWP_ERR_INVALID;
   *out = nullptr;
+  if (threshold_mode && max_list < 0) return IWP_ERR_INVALID;
   iwp_ctx* c = new (std::nothrow) iwp_ctx;
   if (!c) return IWP_ERR_OOM;
   try {
-    c->plan = make_plan(layer_sizes, n_layers, W, ratio, eps);
+    c->plan = make_plan(layer_sizes, n_layers, W, ratio, eps, threshold_mode ? 0u : SMALL_MAX,
+                        threshold_mode ? THRESHOLD_CHUNK_TILES : CHUNK_TILES);
   } catch (...) {
     delete c;
     return IWP_ERR_OOM;
@@ -435,14 +457,19 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
   c->eps = eps;
   c->ratio = ratio;
   c->seed = seed;
+  c->threshold_mode = threshold_mode;
+  c->list_cap = threshold_mode ? ((max_list == 0 || static_cast<uint64_t>(max_list) > p.N) ? p.N : static_cast<uint64_t>(max_list)) : 0;
   c->n_pairs = static_cast<uint32_t>(p.large_layers.size()) * static_cast<uint32_t>(W);
   if (cudaGetDevice(&c->device) != cudaSuccess) {
     cudaGetLastError();
     delete c;
     return IWP_ERR_CUDA;
   }
-  const Sizes sz = sizes_of(p);
-  c->device_bytes = sz.total();
+  const Sizes sz = sizes_of(p, threshold_mode, c->list_cap);
+  const uint64_t thr_bytes = threshold_mode
+                                 ? (p.layers.size() + 2 * p.chunks.size() + 1) * sizeof(uint32_t)
+                                 : 0;
+  c->device_bytes = sz.total() + thr_bytes;
   int rc = IWP_OK;
   auto A = [&](auto** ptr, uint64_t bytes) {
     if (rc == IWP_OK) rc = dev_alloc(ptr, bytes);
@@ -471,12 +498,19 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
   A(&c->sel_idx, sz.sel_idx);
   A(&c->sel_val, sz.sel_val);
   A(&c->d_status, sz.status);
+  if (threshold_mode) {
+    A(&c->d_thr, p.layers.size() * sizeof(uint32_t));
+    A(&c->d_tcnt, at_least(p.chunks.size() * sizeof(uint32_t)));
+    A(&c->d_toff, at_least(p.chunks.size() * sizeof(uint32_t)));
+    A(&c->d_list_len, sizeof(uint32_t));
+  }
   if (rc != IWP_OK) {
     free_all(c);
     delete c;
     return rc;
   }
   bool ok = true;
+  if (threshold_mode) ok = cudaMemset(c->d_list_len, 0, sizeof(uint32_t)) == cudaSuccess;
   auto H2D = [&](void* dst, const void* src, size_t bytes) {
     if (bytes) ok = ok && cudaMemcpy(dst, src, bytes, cudaMemcpyHostToDevice) == cudaSuccess;
   };
@@ -525,6 +559,86 @@ int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int3
   return IWP_OK;
 }
 
+// The threshold-mode step: plain accumulate of every worker, then count / scan / compact on the
+// chosen node's residual alone, then gather, ordered sum, scatter and zeroing at its index set.
+template <bool VEC>
+int run_step_threshold(iwp_ctx* c, const float* grads, const float* weights, float* update, int32_t leader) {
+  const Plan& p = c->plan;
+  const int W = p.W;
+  const uint64_t N = p.N;
+  cudaStream_t s = c->stream;
+  const unsigned n_tiles = static_cast<unsigned>(p.tiles.size());
+  const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
+  const float* acc_leader = c->acc + static_cast<uint64_t>(leader) * N;
+  const uint32_t cap = static_cast<uint32_t>(c->list_cap);
+  stage_mark_at(c, 0);
+  stage_mark_at(c, 1);
+  stage_mark_at(c, 2);
+  k_accumulate<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, N, W, c->momentum);
+  IWP_LAUNCH_CHECK(c);
+  stage_mark_at(c, 3);
+  k_thr_count<VEC><<<n_chunks, THREADS, 0, s>>>(acc_leader, weights, c->d_chunks, c->d_thr, c->d_tcnt, c->eps);
+  IWP_LAUNCH_CHECK(c);
+  k_thr_scan<<<1, 1024, 0, s>>>(c->d_tcnt, c->d_toff, n_chunks, c->d_list_len);
+  IWP_LAUNCH_CHECK(c);
+  stage_mark_at(c, 4);
+  k_thr_write<VEC><<<n_chunks, THREADS, 0, s>>>(acc_leader, weights, c->d_chunks, c->d_thr, c->d_toff, c->sel_idx,
+                                                c->sel_val, cap, c->d_status, c->eps);
+  IWP_LAUNCH_CHECK(c);
+  stage_mark_at(c, 5);
+  k_thr_gather<<<148 * 8, THREADS, 0, s>>>(c->sel_idx, c->d_list_len, cap, c->acc, update, N, W);
+  IWP_LAUNCH_CHECK(c);
+  stage_mark_at(c, 6);
+  return IWP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int iwp_create(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int32_t W, double ratio, float eps,
+               uint64_t seed) {
+  return create_common(out, layer_sizes, n_layers, W, ratio, eps, seed, false, 0);
+}
+
+int iwp_create_threshold(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int32_t W, float eps,
+                         uint64_t seed, int64_t max_list) {
+  return create_common(out, layer_sizes, n_layers, W, 1.0, eps, seed, true, max_list);
+}
+
+int iwp_set_thresholds(iwp_ctx* c, const float* thr) {
+  if (!c || !thr || !c->threshold_mode) return IWP_ERR_INVALID;
+  std::vector<uint32_t> bits(c->plan.layers.size());
+  for (size_t l = 0; l < bits.size(); ++l) {
+    if (!(thr[l] >= 0.0f)) return IWP_ERR_INVALID;  // negative or NaN
+    std::memcpy(&bits[l], &thr[l], sizeof(uint32_t));
+  }
+  // synchronous copy from a temporary: ordered after everything already enqueued on the stream
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess ||
+      cudaMemcpy(c->d_thr, bits.data(), bits.size() * sizeof(uint32_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  c->thr_set = true;
+  return IWP_OK;
+}
+
+int iwp_get_list_length(iwp_ctx* c, int64_t* len) {
+  if (!c || !len) return IWP_ERR_INVALID;
+  if (!c->threshold_mode) {
+    *len = static_cast<int64_t>(c->plan.K);
+    return IWP_OK;
+  }
+  uint32_t v = 0;
+  if (cudaMemcpyAsync(&v, c->d_list_len, sizeof(uint32_t), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+      cudaStreamSynchronize(c->stream) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  *len = static_cast<int64_t>(v);
+  return IWP_OK;
+}
+
 int iwp_destroy(iwp_ctx* c) {
   if (!c) return IWP_OK;
   cudaStreamSynchronize(c->stream);
@@ -553,7 +667,12 @@ int iwp_step(iwp_ctx* c, const float* grads, const float* weights, float* update
                                                  : leader_at(c->seed, static_cast<uint64_t>(c->t), c->plan.W);
   const bool vec = !c->force_scalar && (c->plan.N % 4 == 0) && aligned16(grads) && aligned16(weights) &&
                    aligned16(update) && aligned16(c->acc);
-  const int rc = vec ? run_step<true>(c, grads, weights, update, leader) : run_step<false>(c, grads, weights, update, leader);
+  if (c->threshold_mode && !c->thr_set) return IWP_ERR_INVALID;  // no thresholds given yet
+  const int rc = c->threshold_mode
+                     ? (vec ? run_step_threshold<true>(c, grads, weights, update, leader)
+                            : run_step_threshold<false>(c, grads, weights, update, leader))
+                     : (vec ? run_step<true>(c, grads, weights, update, leader)
+                            : run_step<false>(c, grads, weights, update, leader));
   if (rc != IWP_OK) return rc;
   c->leader = leader;
   c->t += 1;
@@ -606,7 +725,7 @@ int iwp_get_layout(iwp_ctx* c, int64_t* off, int64_t* k) {
   if (!c) return IWP_ERR_INVALID;
   for (size_t l = 0; l < c->plan.layers.size(); ++l) {
     if (off) off[l] = c->plan.layers[l].off;
-    if (k) k[l] = c->plan.layers[l].k;
+    if (k) k[l] = c->threshold_mode ? 0 : c->plan.layers[l].k;  // no fixed keep count under thresholds
   }
   return IWP_OK;
 }
@@ -614,7 +733,7 @@ int iwp_get_layout(iwp_ctx* c, int64_t* off, int64_t* k) {
 int iwp_get_sizes(iwp_ctx* c, int64_t out[4]) {
   if (!c || !out) return IWP_ERR_INVALID;
   out[0] = static_cast<int64_t>(c->plan.N);
-  out[1] = static_cast<int64_t>(c->plan.K);
+  out[1] = static_cast<int64_t>(c->threshold_mode ? c->list_cap : c->plan.K);
   out[2] = static_cast<int64_t>(c->plan.layers.size());
   out[3] = c->plan.W;
   return IWP_OK;
@@ -664,6 +783,21 @@ int iwp_set_residual(iwp_ctx* c, int32_t w, const float* src) {
 
 int iwp_get_selection(iwp_ctx* c, int32_t w, uint32_t* idx, float* val) {
   if (!c || w < 0 || w >= c->plan.W) return IWP_ERR_INVALID;
+  if (c->threshold_mode) {  // one list, the chosen node's; the whole capacity is copied
+    if (w != c->leader) return IWP_ERR_INVALID;
+    bool ok1 = true;
+    if (idx)
+      ok1 = ok1 && cudaMemcpyAsync(idx, c->sel_idx, c->list_cap * sizeof(uint32_t), cudaMemcpyDeviceToDevice,
+                                   c->stream) == cudaSuccess;
+    if (val)
+      ok1 = ok1 && cudaMemcpyAsync(val, c->sel_val, c->list_cap * sizeof(float), cudaMemcpyDeviceToDevice,
+                                   c->stream) == cudaSuccess;
+    if (!ok1) {
+      cudaGetLastError();
+      return IWP_ERR_CUDA;
+    }
+    return IWP_OK;
+  }
   const uint64_t K = c->plan.K;
   bool ok = true;
   if (idx)
@@ -687,6 +821,11 @@ int iwp_get_mask(iwp_ctx* c, uint8_t* dst) {
     return IWP_ERR_CUDA;
   }
   if (c->leader < 0) return IWP_OK;
+  if (c->threshold_mode) {
+    k_thr_mask<<<148 * 8, THREADS, 0, c->stream>>>(c->sel_idx, c->d_list_len, static_cast<uint32_t>(c->list_cap), dst);
+    if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+    return IWP_OK;
+  }
   const unsigned blocks = static_cast<unsigned>((K + THREADS - 1) / THREADS);
   k_mask_scatter<<<blocks, THREADS, 0, c->stream>>>(c->sel_idx + static_cast<uint64_t>(c->leader) * K, dst, K);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
@@ -695,13 +834,17 @@ int iwp_get_mask(iwp_ctx* c, uint8_t* dst) {
 
 int iwp_reset(iwp_ctx* c) {
   if (!c) return IWP_ERR_INVALID;
-  const Sizes sz = sizes_of(c->plan);
+  const Sizes sz = sizes_of(c->plan, c->threshold_mode, c->list_cap);
   bool ok = cudaMemsetAsync(c->acc, 0, sz.acc, c->stream) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->zmask, 0, sz.zmask, c->stream) == cudaSuccess;
   c->zero_pending = false;
   ok = ok && cudaMemsetAsync(c->d_hist, 0, sz.hist, c->stream) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->d_status, 0, sz.status, c->stream) == cudaSuccess;
   if (!ok) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  if (c->threshold_mode && cudaMemsetAsync(c->d_list_len, 0, sizeof(uint32_t), c->stream) != cudaSuccess) {
     cudaGetLastError();
     return IWP_ERR_CUDA;
   }

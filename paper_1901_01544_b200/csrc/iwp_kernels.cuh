@@ -19,6 +19,7 @@ namespace iwp {
 constexpr int THREADS = 256;
 constexpr int WARPS = THREADS / 32;
 constexpr int STATUS_INTERNAL = -4;
+constexpr int STATUS_CAPACITY = -6;
 
 // radix-select digit plan over the 32-bit importance pattern (bit 31 is always 0)
 __host__ __device__ constexpr int pass_shift(int pass) { return pass == 0 ? 21 : (pass == 1 ? 10 : 0); }
@@ -1250,6 +1251,153 @@ __global__ void __launch_bounds__(THREADS)
       for (int w = 0; w < W; ++w) acc[static_cast<uint64_t>(w) * N + i] = 0.0f;
     }
   }
+}
+
+// ---------------------------------------------------------------------------------------
+// Absolute-threshold mode: Algorithm 1 as printed.  Only the chosen node forms a mask, per layer
+// Mask = |G / w| > thr (strict), so after the plain accumulate pass (k_accumulate) the select is
+// two looks at ONE worker's residual: count per chunk, scan, stable compaction; the index set has
+// whatever size results.  thr_bits: the thresholds' fp32 patterns (thr >= 0, so patterns order like
+// values and +inf passes nothing).
+// ---------------------------------------------------------------------------------------
+template <bool VEC>
+__global__ void __launch_bounds__(THREADS)
+    k_thr_count(const float* __restrict__ acc_leader, const float* __restrict__ weights,
+                const Chunk* __restrict__ chunks, const uint32_t* __restrict__ thr_bits,
+                uint32_t* __restrict__ chunk_cnt, float eps) {
+  __shared__ uint32_t sh_cnt;
+  const Chunk c = chunks[blockIdx.x];
+  const uint32_t T = thr_bits[c.layer];
+  if (threadIdx.x == 0) sh_cnt = 0;
+  __syncthreads();
+  const uint64_t lo = c.a, hi = lo + c.len;
+  const uint64_t s0 = lo & ~3ull;
+  const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+  uint32_t cnt = 0;
+  for (uint32_t it = 0; it < n_iter; ++it) {
+    const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+    float av[4], wv[4];
+    load4<VEC>(acc_leader, e0, lo, hi, av);
+    load4<VEC>(weights, e0, lo, hi, wv);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint64_t e = e0 + q;
+      cnt += (e >= lo && e < hi && imp_key(av[q], wv[q], eps) > T) ? 1u : 0u;
+    }
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
+  if ((threadIdx.x & 31) == 0 && cnt) atomicAdd(&sh_cnt, cnt);
+  __syncthreads();
+  if (threadIdx.x == 0) chunk_cnt[blockIdx.x] = sh_cnt;
+}
+
+// Exclusive prefix sum of the chunk counts (chunks are in index order) and the list length.
+// One CTA of 1024 threads walks the chunks 1024 at a time.
+__global__ void __launch_bounds__(1024)
+    k_thr_scan(const uint32_t* __restrict__ chunk_cnt, uint32_t* __restrict__ chunk_off, uint32_t n_chunks,
+               uint32_t* __restrict__ list_len) {
+  __shared__ uint32_t sh_w[32];
+  __shared__ uint32_t sh_run;
+  if (threadIdx.x == 0) sh_run = 0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  for (uint32_t base = 0; base < n_chunks; base += 1024) {
+    const uint32_t j = base + threadIdx.x;
+    const uint32_t v = j < n_chunks ? chunk_cnt[j] : 0u;
+    const uint32_t incl = warp_incl_scan(v);
+    if (lane == 31) sh_w[wid] = incl;
+    __syncthreads();
+    uint32_t woff = 0, tot = 0;
+    for (int i = 0; i < 32; ++i) {
+      const uint32_t x = sh_w[i];
+      if (i < wid) woff += x;
+      tot += x;
+    }
+    const uint32_t run = sh_run;
+    if (j < n_chunks) chunk_off[j] = run + woff + incl - v;
+    __syncthreads();
+    if (threadIdx.x == 0) sh_run = run + tot;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *list_len = sh_run;
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(THREADS)
+    k_thr_write(const float* __restrict__ acc_leader, const float* __restrict__ weights,
+                const Chunk* __restrict__ chunks, const uint32_t* __restrict__ thr_bits,
+                const uint32_t* __restrict__ chunk_off, uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val,
+                uint32_t capacity, int* __restrict__ status, float eps) {
+  __shared__ uint32_t sh_warp[WARPS];
+  const Chunk c = chunks[blockIdx.x];
+  const uint32_t T = thr_bits[c.layer];
+  uint32_t run = chunk_off[blockIdx.x];
+  const uint64_t lo = c.a, hi = lo + c.len;
+  const uint64_t s0 = lo & ~3ull;
+  const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+  for (uint32_t it = 0; it < n_iter; ++it) {
+    const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+    float av[4], wv[4];
+    load4<VEC>(acc_leader, e0, lo, hi, av);
+    load4<VEC>(weights, e0, lo, hi, wv);
+    uint32_t f = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint64_t e = e0 + q;
+      f |= (e >= lo && e < hi && imp_key(av[q], wv[q], eps) > T) ? (1u << q) : 0u;
+    }
+    uint32_t total;
+    uint32_t pos = run + block_excl_scan(static_cast<uint32_t>(__popc(f)), sh_warp, total);
+    if (f) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if ((f >> q) & 1u) {
+          if (pos < capacity) {
+            sel_idx[pos] = static_cast<uint32_t>(e0 + q);
+            sel_val[pos] = av[q];
+          } else {
+            atomicMin(status, STATUS_CAPACITY);
+          }
+          ++pos;
+        }
+      }
+    }
+    run += total;
+  }
+}
+
+// Steps (e)-(g) with a list whose length is only known on the device: grid-stride over its entries.
+__global__ void __launch_bounds__(THREADS)
+    k_thr_gather(const uint32_t* __restrict__ sel_idx, const uint32_t* __restrict__ list_len, uint32_t capacity,
+                 float* __restrict__ acc, float* __restrict__ update, uint64_t N, int W) {
+  const uint32_t len = min(*list_len, capacity);
+  for (uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x; j < len;
+       j += static_cast<uint64_t>(gridDim.x) * THREADS) {
+    const uint64_t i = sel_idx[j];
+    float* p = acc + i;
+    float s = 0.0f;
+    for (int w0 = 0; w0 < W; w0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = (w0 + u < W) ? p[static_cast<uint64_t>(w0 + u) * N] : 0.0f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
+      }
+    }
+    for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
+    update[i] = __fadd_rn(0.0f, s);
+  }
+}
+
+__global__ void __launch_bounds__(THREADS)
+    k_thr_mask(const uint32_t* __restrict__ sel_idx, const uint32_t* __restrict__ list_len, uint32_t capacity,
+               uint8_t* __restrict__ dst) {
+  const uint32_t len = min(*list_len, capacity);
+  for (uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x; j < len;
+       j += static_cast<uint64_t>(gridDim.x) * THREADS)
+    dst[sel_idx[j]] = 1;
 }
 
 // byte mask of the index set (Algorithm 1's encode_uint8(Mask)); dst is zeroed by the caller

@@ -112,7 +112,11 @@ struct Plan {
   bool valid = false;
 };
 
-inline Plan make_plan(const int64_t* sizes, int32_t n_layers, int32_t W, double ratio, float eps) {
+// small_max: layers of at most this many elements take the one-CTA path (0: every layer is tiled, no
+// threshold sampling - the plan of the absolute-threshold mode, which also uses smaller chunks because
+// its select kernels walk one worker only and need the parallelism).
+inline Plan make_plan(const int64_t* sizes, int32_t n_layers, int32_t W, double ratio, float eps,
+                      uint32_t small_max = SMALL_MAX, uint32_t chunk_tiles = CHUNK_TILES) {
   Plan p;
   if (!sizes || n_layers < 1 || W < 1 || !(ratio >= 1.0) || !std::isfinite(ratio) || !(eps > 0.f) ||
       !std::isfinite(eps))
@@ -132,7 +136,7 @@ inline Plan make_plan(const int64_t* sizes, int32_t n_layers, int32_t W, double 
     d.k = static_cast<uint32_t>(keep_count(sizes[l], ratio));
     d.koff = static_cast<uint32_t>(koff);
     d.large_index = -1;
-    if (d.n <= SMALL_MAX) {
+    if (d.n <= small_max) {
       p.small_layers.push_back(static_cast<uint32_t>(l));
       if (d.n > p.max_small_n) p.max_small_n = d.n;
     } else {
@@ -151,8 +155,8 @@ inline Plan make_plan(const int64_t* sizes, int32_t n_layers, int32_t W, double 
         a = b;
       }
       d.n_tiles = static_cast<uint32_t>(p.tiles.size()) - d.first_tile;
-      for (uint32_t t0 = 0; t0 < d.n_tiles; t0 += CHUNK_TILES) {
-        const uint32_t nt = (d.n_tiles - t0 < CHUNK_TILES) ? d.n_tiles - t0 : CHUNK_TILES;
+      for (uint32_t t0 = 0; t0 < d.n_tiles; t0 += chunk_tiles) {
+        const uint32_t nt = (d.n_tiles - t0 < chunk_tiles) ? d.n_tiles - t0 : chunk_tiles;
         Chunk c{};
         c.first_tile = d.first_tile + t0;
         c.n_tiles = nt;
@@ -164,7 +168,7 @@ inline Plan make_plan(const int64_t* sizes, int32_t n_layers, int32_t W, double 
         p.chunks.push_back(c);
       }
       d.n_chunks = static_cast<uint32_t>(p.chunks.size()) - d.first_chunk;
-      sample_plan(d.n, d.k, &d.sample, &d.rho);
+      if (small_max != 0) sample_plan(d.n, d.k, &d.sample, &d.rho);
     }
     p.layers.push_back(d);
     off += d.n;

@@ -1,0 +1,135 @@
+"""GPU parity of the absolute-threshold mode (Algorithm 1 as printed: Mask = importance > thr on the
+chosen node, variable-size index set) against the CPU oracle, bit for bit, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1901_01544_b200 import binding
+from paper_1901_01544_b200 import workloads as wl
+from paper_1901_01544_b200.binding import Pruner
+from parity import assert_bits_equal
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _randn(shape, seed, scale=1.0):
+    g = torch.Generator(device=DEV)
+    g.manual_seed(seed)
+    return torch.randn(shape, generator=g, device=DEV, dtype=torch.float32) * scale
+
+
+def _run(sizes, W, thr, weights, grads_fn, steps, seed=3, momentum=None, max_list=0, force_scalar=False,
+         residual_every=1):
+    N = sum(sizes)
+    pr = Pruner(sizes, W, None, 1e-8, seed, thresholds=thr, max_list=max_list)
+    orc = oracle.Oracle(sizes, W, 2.0, 1e-8, seed)
+    orc.set_thresholds(thr)
+    if momentum is not None:
+        pr.set_momentum(momentum)
+        orc.set_momentum(momentum)
+    if force_scalar:
+        pr.set_option("force_scalar", 1)
+    w_host = weights.cpu().numpy()
+    upd = torch.full((N,), float("nan"), device=DEV)
+    for t in range(steps):
+        g = grads_fn(t)
+        pr.step(g, weights, upd)
+        want = orc.step(np.ascontiguousarray(g.cpu().numpy()), w_host)
+        assert pr.sync_status() == 0 and pr.leader == orc.leader
+        oi, ov = orc.threshold_list()
+        assert pr.list_length() == len(oi), f"step {t}: list length"
+        gi, gv = pr.selection(pr.leader)
+        assert np.array_equal(gi.cpu().numpy().view(np.uint32)[: len(oi)], oi), f"step {t}: indices"
+        assert_bits_equal(gv.cpu().numpy()[: len(oi)], ov, f"step {t}: values")
+        assert_bits_equal(upd.cpu().numpy(), want, f"step {t}: update")
+        assert np.array_equal(pr.mask().cpu().numpy(), orc.mask()), f"step {t}: mask"
+        if (t + 1) % residual_every == 0 or t == steps - 1:
+            for w in range(W):
+                assert_bits_equal(pr.residual(w).cpu().numpy(), orc.residual(w), f"step {t}: worker {w} residual")
+        upd.fill_(float("nan"))
+    pr.close()
+    orc.close()
+
+
+CASES = {
+    "mixed_sizes": ([64, 16385, 256, 100000, 9408, 1, 36864, 1000], 4),
+    "odd_total_scalar_path": ([20001, 17, 70003], 3),
+    "unaligned_offsets": ([16389, 16387, 40000], 2),
+    "many_chunks": ([128 * 4096 * 2 + 4097, 65536], 2),
+    "one_worker": ([30000, 70], 1),
+}
+
+
+@pytest.mark.parametrize("name", sorted(CASES))
+def test_threshold_mode_random_values(name):
+    sizes, W = CASES[name]
+    N = sum(sizes)
+    weights = _randn((N,), 100, 0.05)
+    weights[::53] = 0.0
+    # importance of N(0,1e-3)/N(0,0.05) is heavy tailed; these thresholds keep from ~30 % down to ~0.5 %
+    thr = [[0.02, 0.1, 0.5, 2.0][l % 4] for l in range(len(sizes))]
+    _run(sizes, W, thr, weights, lambda t: _randn((W, N), 7 * t + 1, 1e-3), steps=4)
+
+
+def test_threshold_mode_ties_zero_and_infinite_thresholds():
+    sizes, W = [50000, 300, 20000, 5], 3
+    N = sum(sizes)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(8)
+    weights = torch.randint(-2, 3, (N,), generator=g, device=DEV).float() * 0.5
+
+    def grads(t):
+        gg = torch.Generator(device=DEV)
+        gg.manual_seed(60 + t)
+        return torch.randint(-4, 5, (W, N), generator=gg, device=DEV).float() / 8.0
+
+    # many importances equal a threshold exactly (strict comparison); 0 sends every non-zero residual, inf nothing
+    _run(sizes, W, [0.5, 0.0, 1.0, float("inf")], weights, grads, steps=4)
+
+
+def test_threshold_mode_momentum_and_forced_scalar():
+    sizes, W = [40000, 128, 16385], 4
+    N = sum(sizes)
+    weights = _randn((N,), 5, 0.05)
+    _run(sizes, W, [0.3, 0.05, 1.0], weights, lambda t: _randn((W, N), 31 * t + 2, 1e-3), steps=4, momentum=0.9,
+         force_scalar=True, residual_every=2)
+
+
+def test_threshold_mode_capacity_error_and_argument_checks():
+    sizes, W = [20000], 2
+    weights = torch.ones(20000, device=DEV)
+    pr = Pruner(sizes, W, None, 1e-8, 0, max_list=100)
+    L = binding.lib()
+    E = binding.IWP_ERR_INVALID
+    g = _randn((W, 20000), 1, 1.0)
+    assert L.iwp_step(pr._h, g.data_ptr(), weights.data_ptr(), weights.data_ptr()) == E  # no thresholds yet
+    import ctypes as C
+
+    bad = ((C.c_float * 1)(-1.0), (C.c_float * 1)(float("nan")))
+    for arr in bad:
+        assert L.iwp_set_thresholds(pr._h, arr) == E
+    assert L.iwp_set_thresholds(pr._h, None) == E
+    pr.set_thresholds([0.5])  # about 60 % of 20000 pass: far more than 100 entries
+    pr.step(g, weights)
+    assert pr.sync_status() == binding.IWP_ERR_CAPACITY
+    assert pr.list_length() > 100
+    assert "capacity" in binding.iwp_strerror(binding.IWP_ERR_CAPACITY)
+    pr.close()
+    ratio = Pruner(sizes, W, 4.0)
+    assert L.iwp_set_thresholds(ratio._h, bad[0]) == E  # not a threshold-mode context
+    assert ratio.list_length() == ratio.K
+    ratio.close()
+
+
+def test_threshold_mode_full_size_alexnet_shape():
+    c = wl.alexnet_w8()
+    weights = c.weights(DEV)
+    # thresholds near the step-0 top-1/64 point of the He-normal / N(0, 0.01 std) recipe for weight tensors;
+    # biases are zero-initialised (importance = |residual| / eps), so their thresholds sit at that scale
+    thr = []
+    for tns in c.tensors:
+        thr.append(0.4 if tns.kind == "weight" else 2.0e4)
+    buf = torch.empty((c.W, c.N), dtype=torch.float32, device=DEV)
+    _run(c.layer_sizes, c.W, thr, weights, lambda t: c.grads(t, DEV, out=buf), steps=3, seed=c.seed, residual_every=3)
