@@ -79,12 +79,12 @@ int iwp_plan_sizes(const int64_t* layer_sizes_host, int32_t n_layers, int32_t W,
 /* Creates a context on the CURRENT CUDA device.
  *   layer_sizes_host  n_layers element counts; every tensor is its own selection unit
  *                     (Algorithm 1 loops over layers j = 0..M); copied, caller keeps ownership
- *   W                 number of simulated workers (the paper's N nodes), >= 1
+ *   W                 number of simulated workers (the paper's N nodes), 1 .. 65535
  *   ratio             compression factor R >= 1 (64 keeps 1/64 of each layer), finite
  *   eps               guard added to |weight| in the importance; > 0 and finite
  *   seed              seed of the leader draw
  * Allocates and zeroes the residuals acc[W][N] plus select scratch and the (index, value)
- * lists.  Errors: IWP_ERR_INVALID (NULL, n_layers < 1, a size < 1, W < 1, bad ratio or eps,
+ * lists.  Errors: IWP_ERR_INVALID (NULL, n_layers < 1, a size < 1, W out of range, bad ratio or eps,
  * N >= 2^32), IWP_ERR_OOM, IWP_ERR_CUDA; *out is NULL on error. */
 int iwp_create(iwp_ctx** out, const int64_t* layer_sizes_host, int32_t n_layers, int32_t W, double ratio, float eps,
                uint64_t seed);

@@ -18,6 +18,7 @@ constexpr uint32_t TILE = 4096;
 constexpr uint32_t CHUNK_TILES = 128;
 constexpr uint32_t SMALL_MAX = 16384;
 constexpr uint32_t NBINS = 2048;
+constexpr int32_t MAX_WORKERS = 65535;  // workers index the y dimension of several grids
 // single-read path: capacity of a (tile, worker) candidate slot and the sample that sets the guess
 constexpr uint32_t CAND_CAP = 512;
 constexpr uint32_t SAMPLE_MAX = 16384;
@@ -118,8 +119,8 @@ struct Plan {
 inline Plan make_plan(const int64_t* sizes, int32_t n_layers, int32_t W, double ratio, float eps,
                       uint32_t small_max = SMALL_MAX, uint32_t chunk_tiles = CHUNK_TILES) {
   Plan p;
-  if (!sizes || n_layers < 1 || W < 1 || !(ratio >= 1.0) || !std::isfinite(ratio) || !(eps > 0.f) ||
-      !std::isfinite(eps))
+  if (!sizes || n_layers < 1 || W < 1 || W > MAX_WORKERS || !(ratio >= 1.0) || !std::isfinite(ratio) ||
+      !(eps > 0.f) || !std::isfinite(eps))
     return p;
   uint64_t N = 0;
   for (int32_t l = 0; l < n_layers; ++l) {

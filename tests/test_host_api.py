@@ -81,6 +81,12 @@ def test_invalid_arguments_are_rejected_without_a_gpu(L):
     assert L.iwp_create(C.byref(h), sizes, 0, 2, 2.0, 1e-8, 0) == E
     assert L.iwp_create(C.byref(h), bad, 2, 2, 2.0, 1e-8, 0) == E
     assert L.iwp_create(C.byref(h), sizes, 2, 0, 2.0, 1e-8, 0) == E
+    assert L.iwp_create(C.byref(h), sizes, 2, 65536, 2.0, 1e-8, 0) == E
+    assert L.iwp_create_threshold(C.byref(h), sizes, 2, 0, 1e-8, 0, 0) == E
+    assert L.iwp_create_threshold(C.byref(h), sizes, 2, 2, 1e-8, 0, -1) == E
+    assert L.iwp_create_threshold(None, sizes, 2, 2, 1e-8, 0, 0) == E
+    assert L.iwp_set_thresholds(None, None) == E and L.iwp_get_list_length(None, None) == E
+    assert L.iwp_set_momentum(None, 0.5) == E
     assert L.iwp_create(C.byref(h), sizes, 2, 2, 0.5, 1e-8, 0) == E
     assert L.iwp_create(C.byref(h), sizes, 2, 2, float("inf"), 1e-8, 0) == E
     assert L.iwp_create(C.byref(h), sizes, 2, 2, 2.0, 0.0, 0) == E
