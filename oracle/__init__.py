@@ -31,6 +31,8 @@ def lib() -> C.CDLL:
         L.oracle_set_leader_override.argtypes = [vp, i32]
         L.oracle_set_momentum.argtypes = [vp, f32]
         L.oracle_set_thresholds.argtypes = [vp, vp]
+        L.oracle_set_n_leaders.argtypes = [vp, i32]
+        L.oracle_leaders.argtypes = [u64, u64, i32, i32, vp]
         L.oracle_threshold_list_length.argtypes = [vp]
         L.oracle_threshold_list_length.restype = i64
         L.oracle_get_threshold_list.argtypes = [vp, vp, vp]
@@ -70,6 +72,12 @@ def leader(seed: int, t: int, W: int) -> int:
 
 def mix64(z: int) -> int:
     return int(lib().oracle_mix64(z))
+
+
+def leaders(seed: int, t: int, W: int, n: int) -> List[int]:
+    out = np.empty(n, dtype=np.int32)
+    lib().oracle_leaders(seed, t, W, n, _p(out))
+    return out.tolist()
 
 
 def keep_count(n: int, ratio: float) -> int:
@@ -128,6 +136,11 @@ class Oracle:
         a = np.ascontiguousarray(thr, dtype=np.float32)
         assert a.size == self.L
         lib().oracle_set_thresholds(self._h, _p(a))
+
+    def set_n_leaders(self, n: int):
+        """Threshold mode: OR the masks of n distinct chosen nodes (Algorithm 1's r_1..r_n)."""
+        assert 1 <= n <= self.W
+        lib().oracle_set_n_leaders(self._h, n)
 
     def threshold_list(self) -> Tuple[np.ndarray, np.ndarray]:
         n = int(lib().oracle_threshold_list_length(self._h))

@@ -63,6 +63,8 @@ struct Oracle {
   int threads = 0;
   float momentum = 1.0f;         // Eq. 3: the local residual enters the next step scaled by m
   bool threshold_mode = false;   // Algorithm 1 as printed: Mask <- importance > thr on the chosen node
+  int32_t n_leaders = 1;         // threshold mode: how many chosen nodes' masks are OR-ed
+  std::vector<int32_t> leaders;  // the chosen nodes of the last step, r_1 first
   std::vector<float> thr;        // per-layer thresholds (threshold mode)
   std::vector<uint32_t> thr_idx; // the chosen node's index set of the last step (threshold mode)
   std::vector<float> thr_val;    // its accumulated values at those indices, before zeroing
@@ -106,6 +108,19 @@ inline int32_t leader_of(uint64_t seed, uint64_t t, int32_t W) {
   uint64_t z = mix64(seed + (t + 1) * 0x9E3779B97F4A7C15ull);
   uint64_t hi = z >> 32;
   return static_cast<int32_t>((hi * static_cast<uint64_t>(W)) >> 32);
+}
+
+// the chosen nodes r_1..r_n of step t: n distinct workers drawn without replacement; r_1 is leader_of()
+inline std::vector<int32_t> leaders_of(uint64_t seed, uint64_t t, int32_t W, int32_t n) {
+  std::vector<int32_t> remaining(W), out;
+  std::iota(remaining.begin(), remaining.end(), 0);
+  for (int32_t j = 0; j < n; ++j) {
+    const uint64_t z = mix64(seed + (t + 1) * 0x9E3779B97F4A7C15ull + static_cast<uint64_t>(j) * 0xD1B54A32D192ED03ull);
+    const uint64_t u = ((z >> 32) * static_cast<uint64_t>(W - j)) >> 32;
+    out.push_back(remaining[u]);
+    remaining.erase(remaining.begin() + static_cast<long>(u));
+  }
+  return out;
 }
 
 // Selection of one (worker, layer): indices (local to the layer) of the k elements
@@ -191,6 +206,11 @@ void oracle_set_thresholds(void* h, const float* thr) {
   o->threshold_mode = thr != nullptr;
   if (thr) o->thr.assign(thr, thr + o->n.size());
 }
+void oracle_set_n_leaders(void* h, int32_t n) { static_cast<Oracle*>(h)->n_leaders = n; }
+void oracle_leaders(uint64_t seed, uint64_t t, int32_t W, int32_t n, int32_t* out) {
+  const std::vector<int32_t> v = leaders_of(seed, t, W, n);
+  std::copy(v.begin(), v.end(), out);
+}
 int64_t oracle_threshold_list_length(void* h) { return static_cast<int64_t>(static_cast<Oracle*>(h)->thr_idx.size()); }
 void oracle_get_threshold_list(void* h, uint32_t* idx, float* val) {
   Oracle* o = static_cast<Oracle*>(h);
@@ -272,14 +292,23 @@ void oracle_step(void* h, const float* grads, const float* weights, float* updat
   if (o->threshold_mode) {
     // Algorithm 1 as printed: the chosen node r alone forms Mask_r = |G_r / w| > thr, layer by layer;
     // every node then splits its accumulated gradient by that mask
+    // with n > 1 chosen nodes the masks are OR-ed (Algorithm 1: Mask = OR Mask_{r_i})
+    if (o->leader_override >= 0 || o->n_leaders == 1) {
+      o->leaders.assign(1, o->leader);
+    } else {
+      o->leaders = leaders_of(o->seed, static_cast<uint64_t>(o->t), W, o->n_leaders);
+    }
     const float* ar = &o->acc[static_cast<size_t>(o->leader) * N];
     o->thr_idx.clear();
     o->thr_val.clear();
     for (int l = 0; l < L; ++l) {
       for (int64_t i = o->off[l]; i < o->off[l] + o->n[l]; ++i) {
-        if (importance(ar[i], weights[i], o->eps) > o->thr[l]) {
+        bool in_mask = false;
+        for (int32_t r : o->leaders)
+          in_mask = in_mask || importance(o->acc[static_cast<size_t>(r) * N + i], weights[i], o->eps) > o->thr[l];
+        if (in_mask) {
           o->thr_idx.push_back(static_cast<uint32_t>(i));
-          o->thr_val.push_back(ar[i]);
+          o->thr_val.push_back(ar[i]);  // listed values are r_1's
         }
       }
     }

@@ -502,3 +502,71 @@ def test_threshold_at_the_kplus1_th_importance_reproduces_the_ratio_mode():
     assert np.array_equal(u32(upd_thr), u32(upd_ratio))
     for w in range(W):
         assert np.array_equal(u32(th.residual(w)), u32(ratio.residual(w)))
+
+
+# ---------------------------------------------------------------- several chosen nodes, masks OR-ed
+
+
+def _leader_set_rows():
+    rows = []
+    for line in open(os.path.join(GOLD, "leader_sets.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        head, body = line.split(":")
+        seed, W, n = (int(x) for x in head.split())
+        rows.append((seed, W, n, [[int(x) for x in step.split()] for step in body.split("|")]))
+    return rows
+
+
+@pytest.mark.parametrize("seed,W,n,expect", _leader_set_rows())
+def test_leader_sets(seed, W, n, expect):
+    for t, want in enumerate(expect):
+        got = oracle.leaders(seed, t, W, n)
+        assert got == want
+        assert len(set(got)) == n and got[0] == oracle.leader(seed, t, W)
+
+
+def test_or_of_masks_equals_bruteforce_union():
+    layers, W, n = [30, 6, 50], 5, 3
+    N = sum(layers)
+    rng = np.random.default_rng(5)
+    weights = (rng.integers(-2, 3, N) * 0.5).astype(np.float32)
+    thr = [0.75, 0.25, 1.5]
+    orc = oracle.Oracle(layers, W, 2.0, 1e-8, seed=11)
+    orc.set_thresholds(thr)
+    orc.set_n_leaders(n)
+    acc = np.zeros((W, N), np.float32)
+    for t in range(4):
+        grads = (rng.integers(-4, 5, size=(W, N)) / 4.0).astype(np.float32)
+        acc = acc + grads
+        upd = orc.step(grads, weights)
+        rs = oracle.leaders(11, t, W, n)
+        imp = np.abs(acc) / (np.abs(weights) + F(1e-8))
+        layer_thr = np.repeat(np.array(thr, np.float32), layers)
+        union = np.zeros(N, bool)
+        for r in rs:
+            union |= imp[r] > layer_thr
+        S = np.flatnonzero(union)
+        idx, val = orc.threshold_list()
+        assert idx.tolist() == S.tolist() and orc.leader == rs[0]
+        assert np.array_equal(u32(val), u32(acc[rs[0], S]))
+        s = acc[0, S].copy()
+        for w in range(1, W):
+            s = s + acc[w, S]
+        want = np.zeros(N, np.float32)
+        want[S] = F(0) + s
+        assert np.array_equal(u32(upd), u32(want))
+        acc[:, S] = 0
+        for w in range(W):
+            assert np.array_equal(u32(orc.residual(w)), u32(acc[w]))
+    # a union is never smaller than the first node's own mask
+    one = oracle.Oracle(layers, W, 2.0, 1e-8, seed=11)
+    one.set_thresholds(thr)
+    g = (rng.integers(-4, 5, size=(W, N)) / 4.0).astype(np.float32)
+    many = oracle.Oracle(layers, W, 2.0, 1e-8, seed=11)
+    many.set_thresholds(thr)
+    many.set_n_leaders(W)
+    one.step(g, weights)
+    many.step(g, weights)
+    assert set(one.threshold_list()[0].tolist()) <= set(many.threshold_list()[0].tolist())
