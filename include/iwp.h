@@ -65,6 +65,12 @@ int64_t iwp_keep_count(int64_t n, double ratio);
  * with the splitmix64 finaliser as mix64.  Returns -1 if W < 1. */
 int32_t iwp_leader_at(uint64_t seed, uint64_t t, int32_t W);
 
+/* The n distinct chosen nodes r_1..r_n of step t (Algorithm 1: "choose random node r_1, r_2, ... r_n"), drawn
+ * without replacement: u_j = ((mix64(seed + (t+1)*0x9E3779B97F4A7C15 + j*0xD1B54A32D192ED03) >> 32) * (W-j)) >> 32
+ * picks the u_j-th of the workers not chosen yet; out_host[0] equals iwp_leader_at().  1 <= n <= min(W, 8).
+ * Errors: IWP_ERR_INVALID. */
+int iwp_leaders_at(uint64_t seed, uint64_t t, int32_t W, int32_t n, int32_t* out_host);
+
 /* Sizes the planner derives from a layer list, without touching a GPU.
  * out[0] = N (total elements)            out[1] = K (total keep count per worker)
  * out[2] = layers on the one-CTA path    out[3] = layers on the tiled path
@@ -175,6 +181,9 @@ int iwp_reset(iwp_ctx* ctx);
 /* Options (tests and experiments):
  *   "leader_override"  >= 0 forces the leader of every following step, -1 = seeded draw
  *   "force_scalar"     1 = never use 128-bit accesses
+ *   "n_leaders"        threshold-mode contexts only: 1 .. min(W, 8) chosen nodes per step whose masks are
+ *                      OR-ed (Algorithm 1: Mask = OR Mask_ri); the listed values are r_1's; a forced
+ *                      leader ("leader_override") makes the step a one-node step
  *   "speculate"        1 (default) = sample-based threshold guess so that large layers are
  *                      read once; 0 = always the multi-pass exact select.  Both are exact.
  *   "time_stages"      1 = record a CUDA event at every stage boundary of each following step

@@ -21,7 +21,7 @@ EXPORTS = [
     "iwp_set_stream", "iwp_step", "iwp_step_host", "iwp_sync_status", "iwp_get_layout", "iwp_get_sizes",
     "iwp_get_step", "iwp_set_step", "iwp_get_leader", "iwp_get_residual", "iwp_set_residual",
     "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat", "iwp_select_static",
-    "iwp_set_momentum", "iwp_create_threshold", "iwp_set_thresholds", "iwp_get_list_length",
+    "iwp_set_momentum", "iwp_create_threshold", "iwp_set_thresholds", "iwp_get_list_length", "iwp_leaders_at",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -46,6 +46,7 @@ def lib() -> C.CDLL:
         L.iwp_strerror.restype, L.iwp_strerror.argtypes = cp, [C.c_int]
         L.iwp_keep_count.restype, L.iwp_keep_count.argtypes = i64, [i64, f64]
         L.iwp_leader_at.restype, L.iwp_leader_at.argtypes = i32, [u64, u64, i32]
+        L.iwp_leaders_at.argtypes = [u64, u64, i32, i32, vp]
         L.iwp_plan_sizes.argtypes = [vp, i32, i32, f64, vp]
         L.iwp_create.argtypes = [C.POINTER(vp), vp, i32, i32, f64, f32, u64]
         L.iwp_create_threshold.argtypes = [C.POINTER(vp), vp, i32, i32, f32, u64, i64]
@@ -94,6 +95,12 @@ def iwp_keep_count(n: int, ratio: float) -> int:
 
 def iwp_leader_at(seed: int, t: int, W: int) -> int:
     return int(lib().iwp_leader_at(seed, t, W))
+
+
+def iwp_leaders_at(seed: int, t: int, W: int, n: int) -> List[int]:
+    out = (C.c_int32 * n)()
+    _check(lib().iwp_leaders_at(seed, t, W, n, out), "iwp_leaders_at")
+    return list(out)
 
 
 def iwp_plan_sizes(layer_sizes: Sequence[int], W: int, ratio: float) -> dict:

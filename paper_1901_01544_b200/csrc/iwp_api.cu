@@ -53,6 +53,7 @@ struct iwp_ctx {
   bool threshold_mode = false;
   uint64_t list_cap = 0;          // capacity of the single index list
   bool thr_set = false;
+  int32_t n_leaders = 1;          // chosen nodes whose masks are OR-ed
   uint32_t* d_thr = nullptr;      // [layer] fp32 patterns of the thresholds
   uint32_t* d_tcnt = nullptr;     // [chunk] selected elements of the chunk
   uint32_t* d_toff = nullptr;     // [chunk] list offset of the chunk
@@ -414,6 +415,13 @@ int64_t iwp_keep_count(int64_t n, double ratio) { return keep_count(n, ratio); }
 
 int32_t iwp_leader_at(uint64_t seed, uint64_t t, int32_t W) { return leader_at(seed, t, W); }
 
+int iwp_leaders_at(uint64_t seed, uint64_t t, int32_t W, int32_t n, int32_t* out) {
+  if (!out || W < 1 || n < 1 || n > W || n > MAX_LEADERS) return IWP_ERR_INVALID;
+  const LeaderSet ls = leaders_at(seed, t, W, n);
+  for (int32_t j = 0; j < n; ++j) out[j] = ls.r[j];
+  return IWP_OK;
+}
+
 int iwp_plan_sizes(const int64_t* layer_sizes, int32_t n_layers, int32_t W, double ratio, int64_t out[8]) {
   if (!out) return IWP_ERR_INVALID;
   const Plan p = make_plan(layer_sizes, n_layers, W, ratio, 1.0f);
@@ -569,7 +577,14 @@ int run_step_threshold(iwp_ctx* c, const float* grads, const float* weights, flo
   cudaStream_t s = c->stream;
   const unsigned n_tiles = static_cast<unsigned>(p.tiles.size());
   const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
-  const float* acc_leader = c->acc + static_cast<uint64_t>(leader) * N;
+  // several chosen nodes unless the leader is forced; r_1 is `leader` either way
+  LeaderSet ls{};
+  if (c->n_leaders > 1 && c->leader_override < 0) {
+    ls = leaders_at(c->seed, static_cast<uint64_t>(c->t), W, c->n_leaders);
+  } else {
+    ls.n = 1;
+    ls.r[0] = leader;
+  }
   const uint32_t cap = static_cast<uint32_t>(c->list_cap);
   stage_mark_at(c, 0);
   stage_mark_at(c, 1);
@@ -577,13 +592,13 @@ int run_step_threshold(iwp_ctx* c, const float* grads, const float* weights, flo
   k_accumulate<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, N, W, c->momentum);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 3);
-  k_thr_count<VEC><<<n_chunks, THREADS, 0, s>>>(acc_leader, weights, c->d_chunks, c->d_thr, c->d_tcnt, c->eps);
+  k_thr_count<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_thr, c->d_tcnt, c->eps, N, ls);
   IWP_LAUNCH_CHECK(c);
   k_thr_scan<<<1, 1024, 0, s>>>(c->d_tcnt, c->d_toff, n_chunks, c->d_list_len);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 4);
-  k_thr_write<VEC><<<n_chunks, THREADS, 0, s>>>(acc_leader, weights, c->d_chunks, c->d_thr, c->d_toff, c->sel_idx,
-                                                c->sel_val, cap, c->d_status, c->eps);
+  k_thr_write<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_thr, c->d_toff, c->sel_idx,
+                                                c->sel_val, cap, c->d_status, c->eps, N, ls);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 5);
   k_thr_gather<<<148 * 8, THREADS, 0, s>>>(c->sel_idx, c->d_list_len, cap, c->acc, update, N, W);
@@ -870,6 +885,11 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
     cudaStreamSynchronize(c->stream);
     stage_clear(c);
     c->time_stages = static_cast<int>(v);
+    return IWP_OK;
+  }
+  if (!std::strcmp(key, "n_leaders")) {
+    if (!c->threshold_mode || v < 1 || v > MAX_LEADERS || v > c->plan.W) return IWP_ERR_INVALID;
+    c->n_leaders = static_cast<int32_t>(v);
     return IWP_OK;
   }
   if (!std::strcmp(key, "speculate")) {

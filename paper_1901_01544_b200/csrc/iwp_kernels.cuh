@@ -1256,15 +1256,15 @@ __global__ void __launch_bounds__(THREADS)
 // ---------------------------------------------------------------------------------------
 // Absolute-threshold mode: Algorithm 1 as printed.  Only the chosen node forms a mask, per layer
 // Mask = |G / w| > thr (strict), so after the plain accumulate pass (k_accumulate) the select is
-// two looks at ONE worker's residual: count per chunk, scan, stable compaction; the index set has
-// whatever size results.  thr_bits: the thresholds' fp32 patterns (thr >= 0, so patterns order like
+// two looks at the chosen nodes' residuals (one node, or several whose masks are OR-ed): count per
+// chunk, scan, stable compaction; the index set has whatever size results.  thr_bits: the thresholds' fp32 patterns (thr >= 0, so patterns order like
 // values and +inf passes nothing).
 // ---------------------------------------------------------------------------------------
 template <bool VEC>
 __global__ void __launch_bounds__(THREADS)
-    k_thr_count(const float* __restrict__ acc_leader, const float* __restrict__ weights,
-                const Chunk* __restrict__ chunks, const uint32_t* __restrict__ thr_bits,
-                uint32_t* __restrict__ chunk_cnt, float eps) {
+    k_thr_count(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
+                const uint32_t* __restrict__ thr_bits, uint32_t* __restrict__ chunk_cnt, float eps, uint64_t N,
+                LeaderSet ls) {
   __shared__ uint32_t sh_cnt;
   const Chunk c = chunks[blockIdx.x];
   const uint32_t T = thr_bits[c.layer];
@@ -1276,13 +1276,19 @@ __global__ void __launch_bounds__(THREADS)
   uint32_t cnt = 0;
   for (uint32_t it = 0; it < n_iter; ++it) {
     const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
-    float av[4], wv[4];
-    load4<VEC>(acc_leader, e0, lo, hi, av);
+    float wv[4];
     load4<VEC>(weights, e0, lo, hi, wv);
+    uint32_t f = 0;  // Mask = OR of the chosen nodes' masks
+    for (int j = 0; j < ls.n; ++j) {
+      float av[4];
+      load4<VEC>(acc + static_cast<uint64_t>(ls.r[j]) * N, e0, lo, hi, av);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) f |= (imp_key(av[q], wv[q], eps) > T) ? (1u << q) : 0u;
+    }
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const uint64_t e = e0 + q;
-      cnt += (e >= lo && e < hi && imp_key(av[q], wv[q], eps) > T) ? 1u : 0u;
+      cnt += (e >= lo && e < hi && ((f >> q) & 1u)) ? 1u : 0u;
     }
   }
 #pragma unroll
@@ -1325,10 +1331,10 @@ __global__ void __launch_bounds__(1024)
 
 template <bool VEC>
 __global__ void __launch_bounds__(THREADS)
-    k_thr_write(const float* __restrict__ acc_leader, const float* __restrict__ weights,
-                const Chunk* __restrict__ chunks, const uint32_t* __restrict__ thr_bits,
-                const uint32_t* __restrict__ chunk_off, uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val,
-                uint32_t capacity, int* __restrict__ status, float eps) {
+    k_thr_write(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
+                const uint32_t* __restrict__ thr_bits, const uint32_t* __restrict__ chunk_off,
+                uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val, uint32_t capacity,
+                int* __restrict__ status, float eps, uint64_t N, LeaderSet ls) {
   __shared__ uint32_t sh_warp[WARPS];
   const Chunk c = chunks[blockIdx.x];
   const uint32_t T = thr_bits[c.layer];
@@ -1338,14 +1344,23 @@ __global__ void __launch_bounds__(THREADS)
   const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
   for (uint32_t it = 0; it < n_iter; ++it) {
     const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
-    float av[4], wv[4];
-    load4<VEC>(acc_leader, e0, lo, hi, av);
+    float av[4], wv[4];  // av: r_1's values, the ones listed
+    load4<VEC>(acc + static_cast<uint64_t>(ls.r[0]) * N, e0, lo, hi, av);
     load4<VEC>(weights, e0, lo, hi, wv);
     uint32_t f = 0;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const uint64_t e = e0 + q;
-      f |= (e >= lo && e < hi && imp_key(av[q], wv[q], eps) > T) ? (1u << q) : 0u;
+    for (int q = 0; q < 4; ++q) f |= (imp_key(av[q], wv[q], eps) > T) ? (1u << q) : 0u;
+    for (int j = 1; j < ls.n; ++j) {
+      float bv[4];
+      load4<VEC>(acc + static_cast<uint64_t>(ls.r[j]) * N, e0, lo, hi, bv);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) f |= (imp_key(bv[q], wv[q], eps) > T) ? (1u << q) : 0u;
+    }
+    {
+      uint32_t inside = 0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) inside |= (e0 + q >= lo && e0 + q < hi) ? (1u << q) : 0u;
+      f &= inside;
     }
     uint32_t total;
     uint32_t pos = run + block_excl_scan(static_cast<uint32_t>(__popc(f)), sh_warp, total);

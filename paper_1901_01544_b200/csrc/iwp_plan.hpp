@@ -9,6 +9,7 @@
 //   chunk  <= CHUNK_TILES consecutive tiles of one layer: the unit of work of the select kernels.
 #pragma once
 #include <cmath>
+#include <cstddef>
 #include <cstdint>
 #include <vector>
 
@@ -99,6 +100,27 @@ inline int32_t leader_at(uint64_t seed, uint64_t t, int32_t W) {
   if (W < 1) return -1;
   const uint64_t z = mix64(seed + (t + 1) * 0x9E3779B97F4A7C15ull);
   return static_cast<int32_t>(((z >> 32) * static_cast<uint64_t>(W)) >> 32);
+}
+
+// Chosen nodes r_1..r_n of step t: n distinct workers drawn without replacement; r_1 = leader_at().
+constexpr int MAX_LEADERS = 8;
+struct LeaderSet {
+  int32_t n;
+  int32_t r[MAX_LEADERS];
+};
+
+inline LeaderSet leaders_at(uint64_t seed, uint64_t t, int32_t W, int32_t n) {
+  LeaderSet ls{};
+  ls.n = n;
+  std::vector<int32_t> remaining(static_cast<size_t>(W));
+  for (int32_t w = 0; w < W; ++w) remaining[static_cast<size_t>(w)] = w;
+  for (int32_t j = 0; j < n; ++j) {
+    const uint64_t z = mix64(seed + (t + 1) * 0x9E3779B97F4A7C15ull + static_cast<uint64_t>(j) * 0xD1B54A32D192ED03ull);
+    const uint64_t u = ((z >> 32) * static_cast<uint64_t>(W - j)) >> 32;
+    ls.r[j] = remaining[u];
+    remaining.erase(remaining.begin() + static_cast<std::ptrdiff_t>(u));
+  }
+  return ls;
 }
 
 struct Plan {

@@ -21,7 +21,7 @@ def _randn(shape, seed, scale=1.0):
 
 
 def _run(sizes, W, thr, weights, grads_fn, steps, seed=3, momentum=None, max_list=0, force_scalar=False,
-         residual_every=1):
+         residual_every=1, n_leaders=1):
     N = sum(sizes)
     pr = Pruner(sizes, W, None, 1e-8, seed, thresholds=thr, max_list=max_list)
     orc = oracle.Oracle(sizes, W, 2.0, 1e-8, seed)
@@ -31,6 +31,9 @@ def _run(sizes, W, thr, weights, grads_fn, steps, seed=3, momentum=None, max_lis
         orc.set_momentum(momentum)
     if force_scalar:
         pr.set_option("force_scalar", 1)
+    if n_leaders > 1:
+        pr.set_option("n_leaders", n_leaders)
+        orc.set_n_leaders(n_leaders)
     w_host = weights.cpu().numpy()
     upd = torch.full((N,), float("nan"), device=DEV)
     for t in range(steps):
@@ -133,3 +136,21 @@ def test_threshold_mode_full_size_alexnet_shape():
         thr.append(0.4 if tns.kind == "weight" else 2.0e4)
     buf = torch.empty((c.W, c.N), dtype=torch.float32, device=DEV)
     _run(c.layer_sizes, c.W, thr, weights, lambda t: c.grads(t, DEV, out=buf), steps=3, seed=c.seed, residual_every=3)
+
+
+@pytest.mark.parametrize("n_leaders", [2, 4])
+def test_threshold_mode_several_chosen_nodes(n_leaders):
+    sizes, W = [70000, 300, 16385, 64], 5
+    N = sum(sizes)
+    weights = _randn((N,), 9, 0.05)
+    weights[::31] = 0.0
+    _run(sizes, W, [0.2, 0.05, 1.0, 0.5], weights, lambda t: _randn((W, N), 13 * t + 4, 1e-3), steps=5,
+         n_leaders=n_leaders, residual_every=2)
+    pr = Pruner(sizes, W, None, 1e-8, 0, thresholds=[1.0] * 4)
+    L = binding.lib()
+    assert L.iwp_set_option(pr._h, b"n_leaders", 6) == binding.IWP_ERR_INVALID  # more than W
+    assert L.iwp_set_option(pr._h, b"n_leaders", 0) == binding.IWP_ERR_INVALID
+    pr.close()
+    ratio = Pruner(sizes, W, 4.0)
+    assert L.iwp_set_option(ratio._h, b"n_leaders", 2) == binding.IWP_ERR_INVALID  # ratio-mode context
+    ratio.close()

@@ -54,6 +54,21 @@ def test_leader_matches_vectors(L):
     assert binding.iwp_leader_at(0, 0, 0) == -1
 
 
+def test_leader_sets_match_vectors(L):
+    for line in open(os.path.join(GOLD, "leader_sets.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        head, body = line.split(":")
+        seed, W, n = (int(x) for x in head.split())
+        for t, step in enumerate(body.split("|")):
+            assert binding.iwp_leaders_at(seed, t, W, n) == [int(x) for x in step.split()]
+    out = (C.c_int32 * 9)()
+    E = binding.IWP_ERR_INVALID
+    assert L.iwp_leaders_at(0, 0, 4, 5, out) == E and L.iwp_leaders_at(0, 0, 16, 9, out) == E
+    assert L.iwp_leaders_at(0, 0, 4, 0, out) == E and L.iwp_leaders_at(0, 0, 4, 2, None) == E
+
+
 def test_plan_sizes(L):
     from paper_1901_01544_b200 import workloads as wl
 
