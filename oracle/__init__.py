@@ -32,6 +32,9 @@ def lib() -> C.CDLL:
         L.oracle_set_momentum.argtypes = [vp, f32]
         L.oracle_set_thresholds.argtypes = [vp, vp]
         L.oracle_set_n_leaders.argtypes = [vp, i32]
+        L.oracle_set_random_select.argtypes = [vp, i32]
+        L.oracle_draw24.argtypes = [u64, u64, u64]
+        L.oracle_draw24.restype = C.c_uint32
         L.oracle_leaders.argtypes = [u64, u64, i32, i32, vp]
         L.oracle_threshold_list_length.argtypes = [vp]
         L.oracle_threshold_list_length.restype = i64
@@ -72,6 +75,10 @@ def leader(seed: int, t: int, W: int) -> int:
 
 def mix64(z: int) -> int:
     return int(lib().oracle_mix64(z))
+
+
+def draw24(seed: int, t: int, i: int) -> int:
+    return int(lib().oracle_draw24(seed, t, i))
 
 
 def leaders(seed: int, t: int, W: int, n: int) -> List[int]:
@@ -136,6 +143,10 @@ class Oracle:
         a = np.ascontiguousarray(thr, dtype=np.float32)
         assert a.size == self.L
         lib().oracle_set_thresholds(self._h, _p(a))
+
+    def set_random_select(self, on: bool):
+        """Threshold mode: Section 3.3's P(update) = importance / threshold for elements below the threshold."""
+        lib().oracle_set_random_select(self._h, 1 if on else 0)
 
     def set_n_leaders(self, n: int):
         """Threshold mode: OR the masks of n distinct chosen nodes (Algorithm 1's r_1..r_n)."""

@@ -28,6 +28,9 @@
 //   * threshold mode is Algorithm 1 as printed: only the chosen node forms a mask, per layer
 //     Mask = importance > thr[layer] (strict), the index set has whatever size results, and no
 //     other worker makes a selection of its own.
+//   * Section 3.3's random gradient selection (threshold mode, optional): an element whose importance
+//     does not exceed the threshold is sent iff u < importance / thr, u one 24-bit uniform draw per
+//     element and step, the quotient in fp32.
 //   * the ring all-reduce is a sum in ascending worker order, fp32, without the 1/N
 //     factor (the caller pre-scales gradients as in Eq. 1).
 //
@@ -64,6 +67,7 @@ struct Oracle {
   float momentum = 1.0f;         // Eq. 3: the local residual enters the next step scaled by m
   bool threshold_mode = false;   // Algorithm 1 as printed: Mask <- importance > thr on the chosen node
   int32_t n_leaders = 1;         // threshold mode: how many chosen nodes' masks are OR-ed
+  bool random_select = false;    // Section 3.3: elements below the threshold go with P = importance / thr
   std::vector<int32_t> leaders;  // the chosen nodes of the last step, r_1 first
   std::vector<float> thr;        // per-layer thresholds (threshold mode)
   std::vector<uint32_t> thr_idx; // the chosen node's index set of the last step (threshold mode)
@@ -121,6 +125,11 @@ inline std::vector<int32_t> leaders_of(uint64_t seed, uint64_t t, int32_t W, int
     remaining.erase(remaining.begin() + static_cast<long>(u));
   }
   return out;
+}
+
+// Section 3.3, random gradient selection: the uniform draw of element i at step t, 24 bits
+inline uint32_t draw24(uint64_t seed, uint64_t t, uint64_t i) {
+  return static_cast<uint32_t>(mix64(seed + (t + 1) * 0x9E3779B97F4A7C15ull + (i + 1) * 0xC2B2AE3D27D4EB4Full) >> 40);
 }
 
 // Selection of one (worker, layer): indices (local to the layer) of the k elements
@@ -206,6 +215,8 @@ void oracle_set_thresholds(void* h, const float* thr) {
   o->threshold_mode = thr != nullptr;
   if (thr) o->thr.assign(thr, thr + o->n.size());
 }
+void oracle_set_random_select(void* h, int32_t on) { static_cast<Oracle*>(h)->random_select = on != 0; }
+uint32_t oracle_draw24(uint64_t seed, uint64_t t, uint64_t i) { return draw24(seed, t, i); }
 void oracle_set_n_leaders(void* h, int32_t n) { static_cast<Oracle*>(h)->n_leaders = n; }
 void oracle_leaders(uint64_t seed, uint64_t t, int32_t W, int32_t n, int32_t* out) {
   const std::vector<int32_t> v = leaders_of(seed, t, W, n);
@@ -304,8 +315,17 @@ void oracle_step(void* h, const float* grads, const float* weights, float* updat
     for (int l = 0; l < L; ++l) {
       for (int64_t i = o->off[l]; i < o->off[l] + o->n[l]; ++i) {
         bool in_mask = false;
-        for (int32_t r : o->leaders)
-          in_mask = in_mask || importance(o->acc[static_cast<size_t>(r) * N + i], weights[i], o->eps) > o->thr[l];
+        for (int32_t r : o->leaders) {
+          const float imp = importance(o->acc[static_cast<size_t>(r) * N + i], weights[i], o->eps);
+          bool sel = imp > o->thr[l];
+          if (!sel && o->random_select) {
+            // P(update) = importance / threshold: one draw per element and step, compared in fp32
+            const float u = static_cast<float>(draw24(o->seed, static_cast<uint64_t>(o->t), static_cast<uint64_t>(i))) *
+                            5.9604644775390625e-08f;  // 2^-24
+            sel = u < imp / o->thr[l];
+          }
+          in_mask = in_mask || sel;
+        }
         if (in_mask) {
           o->thr_idx.push_back(static_cast<uint32_t>(i));
           o->thr_val.push_back(ar[i]);  // listed values are r_1's

@@ -570,3 +570,54 @@ def test_or_of_masks_equals_bruteforce_union():
     one.step(g, weights)
     many.step(g, weights)
     assert set(one.threshold_list()[0].tolist()) <= set(many.threshold_list()[0].tolist())
+
+
+# ---------------------------------------------------------------- random sub-threshold selection (Section 3.3)
+
+
+def test_random_select_draw_vectors_and_uniformity():
+    for line in open(os.path.join(GOLD, "random_select_draws.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        seed, t, i, want = (int(x) for x in line.split())
+        assert oracle.draw24(seed, t, i) == want
+    u = np.array([oracle.draw24(3, 2, i) for i in range(20000)]) / 2.0 ** 24
+    assert u.min() >= 0 and u.max() < 1 and abs(u.mean() - 0.5) < 0.01 and abs(u.var() - 1 / 12) < 0.005
+    assert abs(np.corrcoef(u[:-1], u[1:])[0, 1]) < 0.03
+
+
+def test_random_select_equals_bruteforce_and_has_the_right_rate():
+    n, W = 6000, 2
+    rng = np.random.default_rng(21)
+    weights = np.ones(n, np.float32)
+    thr = 1.0
+    orc = oracle.Oracle([n], W, 2.0, 1e-8, seed=13)
+    orc.set_thresholds([thr])
+    orc.set_random_select(True)
+    orc.set_leader_override(0)
+    g = rng.uniform(0.0, 1.0, size=(W, n)).astype(np.float32)  # importance of node 0 = g[0] (weights 1): all below thr
+    g[0, :10] = 0.0          # zero importance is never sent
+    g[0, 10:20] = 2.0        # above the threshold: always sent
+    upd = orc.step(g, weights)
+    S = set(orc.threshold_list()[0].tolist())
+    imp = np.abs(g[0]) / (np.abs(weights) + F(1e-8))
+    want = set()
+    for i in range(n):
+        u = F(oracle.draw24(13, 0, i)) * F(2.0 ** -24)
+        if imp[i] > F(thr) or u < F(imp[i] / F(thr)):
+            want.add(i)
+    assert S == want
+    assert not (S & set(range(10))) and set(range(10, 20)) <= S
+    # P(update) = importance / threshold: bucket the elements by importance and compare frequencies
+    sel = np.zeros(n, bool)
+    sel[list(S)] = True
+    for lo in (0.1, 0.4, 0.7):
+        band = (imp >= lo) & (imp < lo + 0.2) & (np.arange(n) >= 20)
+        assert abs(sel[band].mean() - (lo + 0.1)) < 0.06
+    # switched off: only the ten elements above the threshold go
+    off = oracle.Oracle([n], W, 2.0, 1e-8, seed=13)
+    off.set_thresholds([thr])
+    off.set_leader_override(0)
+    off.step(g, weights)
+    assert off.threshold_list()[0].tolist() == list(range(10, 20))
+    assert np.count_nonzero(upd) >= len(S) - 10
