@@ -184,6 +184,11 @@ int iwp_reset(iwp_ctx* ctx);
  *   "n_leaders"        threshold-mode contexts only: 1 .. min(W, 8) chosen nodes per step whose masks are
  *                      OR-ed (Algorithm 1: Mask = OR Mask_ri); the listed values are r_1's; a forced
  *                      leader ("leader_override") makes the step a one-node step
+ *   "random_select"    threshold-mode contexts only: 1 = Section 3.3's random gradient selection: an
+ *                      element whose importance does not exceed its layer's threshold is still sent iff
+ *                      u < importance / thr (fp32 quotient), u = u24 * 2^-24 with
+ *                      u24 = mix64(seed + (t+1)*0x9E3779B97F4A7C15 + (i+1)*0xC2B2AE3D27D4EB4F) >> 40
+ *                      for element i at step t; 0 (default) = off
  *   "speculate"        1 (default) = sample-based threshold guess so that large layers are
  *                      read once; 0 = always the multi-pass exact select.  Both are exact.
  *   "time_stages"      1 = record a CUDA event at every stage boundary of each following step

@@ -54,6 +54,7 @@ struct iwp_ctx {
   uint64_t list_cap = 0;          // capacity of the single index list
   bool thr_set = false;
   int32_t n_leaders = 1;          // chosen nodes whose masks are OR-ed
+  bool random_select = false;     // Section 3.3: P(update) = importance / threshold below the threshold
   uint32_t* d_thr = nullptr;      // [layer] fp32 patterns of the thresholds
   uint32_t* d_tcnt = nullptr;     // [chunk] selected elements of the chunk
   uint32_t* d_toff = nullptr;     // [chunk] list offset of the chunk
@@ -586,19 +587,20 @@ int run_step_threshold(iwp_ctx* c, const float* grads, const float* weights, flo
     ls.r[0] = leader;
   }
   const uint32_t cap = static_cast<uint32_t>(c->list_cap);
+  const RandomSelect rs{c->random_select ? 1 : 0, c->seed, static_cast<uint64_t>(c->t)};
   stage_mark_at(c, 0);
   stage_mark_at(c, 1);
   stage_mark_at(c, 2);
   k_accumulate<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, N, W, c->momentum);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 3);
-  k_thr_count<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_thr, c->d_tcnt, c->eps, N, ls);
+  k_thr_count<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_thr, c->d_tcnt, c->eps, N, ls, rs);
   IWP_LAUNCH_CHECK(c);
   k_thr_scan<<<1, 1024, 0, s>>>(c->d_tcnt, c->d_toff, n_chunks, c->d_list_len);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 4);
   k_thr_write<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_thr, c->d_toff, c->sel_idx,
-                                                c->sel_val, cap, c->d_status, c->eps, N, ls);
+                                                c->sel_val, cap, c->d_status, c->eps, N, ls, rs);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 5);
   k_thr_gather<<<148 * 8, THREADS, 0, s>>>(c->sel_idx, c->d_list_len, cap, c->acc, update, N, W);
@@ -885,6 +887,11 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
     cudaStreamSynchronize(c->stream);
     stage_clear(c);
     c->time_stages = static_cast<int>(v);
+    return IWP_OK;
+  }
+  if (!std::strcmp(key, "random_select")) {
+    if (!c->threshold_mode || (v != 0 && v != 1)) return IWP_ERR_INVALID;
+    c->random_select = v != 0;
     return IWP_OK;
   }
   if (!std::strcmp(key, "n_leaders")) {

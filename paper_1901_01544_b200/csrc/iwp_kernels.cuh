@@ -1260,11 +1260,29 @@ __global__ void __launch_bounds__(THREADS)
 // chunk, scan, stable compaction; the index set has whatever size results.  thr_bits: the thresholds' fp32 patterns (thr >= 0, so patterns order like
 // values and +inf passes nothing).
 // ---------------------------------------------------------------------------------------
+// Random selection parameters of a step (Section 3.3): off, or the seed and step of the draws.
+struct RandomSelect {
+  int on;
+  uint64_t seed;
+  uint64_t step;
+};
+
+// Mask bit of one element on one chosen node: importance > thr, or - with random selection on - a
+// draw below importance / thr (P(update) = importance / threshold; one draw per element and step).
+__device__ __forceinline__ bool thr_selected(float acc, float w, float eps, uint32_t T, uint64_t e,
+                                             const RandomSelect& rs) {
+  const uint32_t key = imp_key(acc, w, eps);
+  if (key > T) return true;
+  if (!rs.on) return false;
+  const float u = __fmul_rn(static_cast<float>(draw24(rs.seed, rs.step, e)), 5.9604644775390625e-08f);
+  return u < __fdiv_rn(__uint_as_float(key), __uint_as_float(T));
+}
+
 template <bool VEC>
 __global__ void __launch_bounds__(THREADS)
     k_thr_count(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
                 const uint32_t* __restrict__ thr_bits, uint32_t* __restrict__ chunk_cnt, float eps, uint64_t N,
-                LeaderSet ls) {
+                LeaderSet ls, RandomSelect rs) {
   __shared__ uint32_t sh_cnt;
   const Chunk c = chunks[blockIdx.x];
   const uint32_t T = thr_bits[c.layer];
@@ -1283,7 +1301,7 @@ __global__ void __launch_bounds__(THREADS)
       float av[4];
       load4<VEC>(acc + static_cast<uint64_t>(ls.r[j]) * N, e0, lo, hi, av);
 #pragma unroll
-      for (int q = 0; q < 4; ++q) f |= (imp_key(av[q], wv[q], eps) > T) ? (1u << q) : 0u;
+      for (int q = 0; q < 4; ++q) f |= thr_selected(av[q], wv[q], eps, T, e0 + q, rs) ? (1u << q) : 0u;
     }
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
@@ -1334,7 +1352,7 @@ __global__ void __launch_bounds__(THREADS)
     k_thr_write(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
                 const uint32_t* __restrict__ thr_bits, const uint32_t* __restrict__ chunk_off,
                 uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val, uint32_t capacity,
-                int* __restrict__ status, float eps, uint64_t N, LeaderSet ls) {
+                int* __restrict__ status, float eps, uint64_t N, LeaderSet ls, RandomSelect rs) {
   __shared__ uint32_t sh_warp[WARPS];
   const Chunk c = chunks[blockIdx.x];
   const uint32_t T = thr_bits[c.layer];
@@ -1349,12 +1367,12 @@ __global__ void __launch_bounds__(THREADS)
     load4<VEC>(weights, e0, lo, hi, wv);
     uint32_t f = 0;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) f |= (imp_key(av[q], wv[q], eps) > T) ? (1u << q) : 0u;
+    for (int q = 0; q < 4; ++q) f |= thr_selected(av[q], wv[q], eps, T, e0 + q, rs) ? (1u << q) : 0u;
     for (int j = 1; j < ls.n; ++j) {
       float bv[4];
       load4<VEC>(acc + static_cast<uint64_t>(ls.r[j]) * N, e0, lo, hi, bv);
 #pragma unroll
-      for (int q = 0; q < 4; ++q) f |= (imp_key(bv[q], wv[q], eps) > T) ? (1u << q) : 0u;
+      for (int q = 0; q < 4; ++q) f |= thr_selected(bv[q], wv[q], eps, T, e0 + q, rs) ? (1u << q) : 0u;
     }
     {
       uint32_t inside = 0;

@@ -102,6 +102,20 @@ inline int32_t leader_at(uint64_t seed, uint64_t t, int32_t W) {
   return static_cast<int32_t>(((z >> 32) * static_cast<uint64_t>(W)) >> 32);
 }
 
+// Section 3.3, random gradient selection: the 24-bit uniform draw of element i at step t.
+#if defined(__CUDACC__)
+__host__ __device__
+#endif
+inline uint32_t draw24(uint64_t seed, uint64_t t, uint64_t i) {
+  uint64_t z = seed + (t + 1) * 0x9E3779B97F4A7C15ull + (i + 1) * 0xC2B2AE3D27D4EB4Full;
+  z ^= z >> 30;
+  z *= 0xBF58476D1CE4E5B9ull;
+  z ^= z >> 27;
+  z *= 0x94D049BB133111EBull;
+  z ^= z >> 31;
+  return static_cast<uint32_t>(z >> 40);
+}
+
 // Chosen nodes r_1..r_n of step t: n distinct workers drawn without replacement; r_1 = leader_at().
 constexpr int MAX_LEADERS = 8;
 struct LeaderSet {

@@ -21,7 +21,7 @@ def _randn(shape, seed, scale=1.0):
 
 
 def _run(sizes, W, thr, weights, grads_fn, steps, seed=3, momentum=None, max_list=0, force_scalar=False,
-         residual_every=1, n_leaders=1):
+         residual_every=1, n_leaders=1, random_select=False):
     N = sum(sizes)
     pr = Pruner(sizes, W, None, 1e-8, seed, thresholds=thr, max_list=max_list)
     orc = oracle.Oracle(sizes, W, 2.0, 1e-8, seed)
@@ -31,6 +31,9 @@ def _run(sizes, W, thr, weights, grads_fn, steps, seed=3, momentum=None, max_lis
         orc.set_momentum(momentum)
     if force_scalar:
         pr.set_option("force_scalar", 1)
+    if random_select:
+        pr.set_option("random_select", 1)
+        orc.set_random_select(True)
     if n_leaders > 1:
         pr.set_option("n_leaders", n_leaders)
         orc.set_n_leaders(n_leaders)
@@ -154,3 +157,24 @@ def test_threshold_mode_several_chosen_nodes(n_leaders):
     ratio = Pruner(sizes, W, 4.0)
     assert L.iwp_set_option(ratio._h, b"n_leaders", 2) == binding.IWP_ERR_INVALID  # ratio-mode context
     ratio.close()
+
+
+@pytest.mark.parametrize("n_leaders", [1, 3])
+def test_threshold_mode_random_sub_threshold_selection(n_leaders):
+    sizes, W = [90000, 300, 16385], 4
+    N = sum(sizes)
+    weights = _randn((N,), 19, 0.05)
+    weights[::41] = 0.0
+    # high thresholds: most of what is sent is sent by the draw, not by the comparison
+    _run(sizes, W, [5.0, 0.5, 20.0], weights, lambda t: _randn((W, N), 17 * t + 5, 1e-3), steps=5,
+         n_leaders=n_leaders, random_select=True, momentum=0.9, residual_every=2)
+
+
+def test_random_select_with_zero_and_infinite_thresholds():
+    sizes, W = [20000, 20000], 2
+    N = sum(sizes)
+    weights = torch.ones(N, device=DEV)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(3)
+    grads = lambda t: torch.randint(-2, 3, (W, N), generator=g, device=DEV).float()  # many exact zeros
+    _run(sizes, W, [0.0, float("inf")], weights, grads, steps=3, random_select=True)
