@@ -588,10 +588,17 @@ int run_step_threshold(iwp_ctx* c, const float* grads, const float* weights, flo
   }
   const uint32_t cap = static_cast<uint32_t>(c->list_cap);
   const RandomSelect rs{c->random_select ? 1 : 0, c->seed, static_cast<uint64_t>(c->t)};
+  // (1) step (a) for the chosen nodes only; (2) their masks -> index list and a bit per element;
+  // (3) one fused streaming pass over all workers: step (a) for the others, ordered sum, zeroing, update
   stage_mark_at(c, 0);
   stage_mark_at(c, 1);
+  if (cudaMemsetAsync(c->zmask, 0, c->zmask_words * sizeof(uint32_t), s) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  c->launches += 1;
   stage_mark_at(c, 2);
-  k_accumulate<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, N, W, c->momentum);
+  k_thr_accumulate_chosen<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, c->d_tiles, N, c->momentum, ls);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 3);
   k_thr_count<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_thr, c->d_tcnt, c->eps, N, ls, rs);
@@ -600,10 +607,10 @@ int run_step_threshold(iwp_ctx* c, const float* grads, const float* weights, flo
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 4);
   k_thr_write<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_thr, c->d_toff, c->sel_idx,
-                                                c->sel_val, cap, c->d_status, c->eps, N, ls, rs);
+                                                c->sel_val, cap, c->d_status, c->zmask, c->eps, N, ls, rs);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 5);
-  k_thr_gather<<<148 * 8, THREADS, 0, s>>>(c->sel_idx, c->d_list_len, cap, c->acc, update, N, W);
+  k_thr_fused<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, c->zmask, N, W, c->momentum, ls);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 6);
   return IWP_OK;

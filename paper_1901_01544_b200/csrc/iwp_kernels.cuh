@@ -1352,7 +1352,8 @@ __global__ void __launch_bounds__(THREADS)
     k_thr_write(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
                 const uint32_t* __restrict__ thr_bits, const uint32_t* __restrict__ chunk_off,
                 uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val, uint32_t capacity,
-                int* __restrict__ status, float eps, uint64_t N, LeaderSet ls, RandomSelect rs) {
+                int* __restrict__ status, uint32_t* __restrict__ set_bits, float eps, uint64_t N, LeaderSet ls,
+                RandomSelect rs) {
   __shared__ uint32_t sh_warp[WARPS];
   const Chunk c = chunks[blockIdx.x];
   const uint32_t T = thr_bits[c.layer];
@@ -1380,6 +1381,9 @@ __global__ void __launch_bounds__(THREADS)
       for (int q = 0; q < 4; ++q) inside |= (e0 + q >= lo && e0 + q < hi) ? (1u << q) : 0u;
       f &= inside;
     }
+    // the index set as a bit per element (zeroed before the step) for the fused pass over all workers;
+    // a slot's four bits never straddle a word because slots start at multiples of four
+    if (f) atomicOr(&set_bits[e0 >> 5], f << (e0 & 31u));
     uint32_t total;
     uint32_t pos = run + block_excl_scan(static_cast<uint32_t>(__popc(f)), sh_warp, total);
     if (f) {
@@ -1397,6 +1401,107 @@ __global__ void __launch_bounds__(THREADS)
       }
     }
     run += total;
+  }
+}
+
+// Threshold mode, first pass: step (a) for the chosen nodes only (their masks are needed before anybody
+// else's residual is touched).  grid = tiles.
+template <bool VEC>
+__global__ void __launch_bounds__(THREADS)
+    k_thr_accumulate_chosen(const float* __restrict__ grads, float* __restrict__ acc, const Tile* __restrict__ tiles,
+                            uint64_t N, float momentum, LeaderSet ls) {
+  const Tile t = tiles[blockIdx.x];
+  const uint64_t lo = t.a, hi = lo + t.len;
+  const uint64_t base = lo & ~static_cast<uint64_t>(TILE - 1);
+  constexpr int SPT = TILE / 4 / THREADS;
+  for (int j = 0; j < ls.n; ++j) {
+    const float* g = grads + static_cast<uint64_t>(ls.r[j]) * N;
+    float* a = acc + static_cast<uint64_t>(ls.r[j]) * N;
+    float gv[SPT][4], av[SPT][4];
+#pragma unroll
+    for (int s = 0; s < SPT; ++s) {
+      const uint64_t e0 = base + static_cast<uint64_t>(s * THREADS + threadIdx.x) * 4;
+      load4_stream<VEC>(g, e0, lo, hi, gv[s]);
+      load4_stream<VEC>(a, e0, lo, hi, av[s]);
+    }
+#pragma unroll
+    for (int s = 0; s < SPT; ++s) {
+      const uint64_t e0 = base + static_cast<uint64_t>(s * THREADS + threadIdx.x) * 4;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) av[s][c] = accumulate(av[s][c], gv[s][c], momentum);
+      store4<VEC>(a, e0, lo, hi, av[s]);
+    }
+  }
+}
+
+// Threshold mode, last pass: everything that is left of the step in ONE streaming pass over all
+// workers, in ascending worker order per element: step (a) for the workers that are not chosen nodes,
+// and for the elements of the index set (a bit per element, written by k_thr_write) the ordered sum
+// of step (f) and the zeroing of step (g); `update` gets the sum or +0.  No gather: nothing is read
+// at scattered addresses.  grid = tiles.
+template <bool VEC>
+__global__ void __launch_bounds__(THREADS)
+    k_thr_fused(const float* __restrict__ grads, float* __restrict__ acc, float* __restrict__ update,
+                const Tile* __restrict__ tiles, const uint32_t* __restrict__ set_bits, uint64_t N, int W,
+                float momentum, LeaderSet ls) {
+  const Tile t = tiles[blockIdx.x];
+  const uint64_t lo = t.a, hi = lo + t.len;
+  const uint64_t base = lo & ~static_cast<uint64_t>(TILE - 1);
+  constexpr int SPT = 2;                          // slots per thread and trip (keeps the kernel at 4 CTAs per SM)
+  constexpr int TRIPS = TILE / 4 / THREADS / SPT;  // the tile is walked in two halves
+#pragma unroll 1
+  for (int trip = 0; trip < TRIPS; ++trip) {
+    uint64_t e0[SPT];
+    uint32_t in_set[SPT];  // four bits per slot
+    float sum[SPT][4];
+    bool any = false;
+#pragma unroll
+    for (int s = 0; s < SPT; ++s) {
+      e0[s] = base + static_cast<uint64_t>((trip * SPT + s) * THREADS + threadIdx.x) * 4;
+      const bool inside = e0[s] < hi && e0[s] + 4 > lo;
+      any = any || inside;
+      in_set[s] = inside ? (set_bits[e0[s] >> 5] >> (e0[s] & 31u)) & 0xFu : 0u;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) sum[s][c] = 0.0f;
+    }
+    if (!__syncthreads_or(any)) continue;  // this half of the window lies outside a ragged tile
+    for (int w = 0; w < W; ++w) {
+      bool is_chosen = false;
+#pragma unroll
+      for (int j = 0; j < MAX_LEADERS; ++j) is_chosen = is_chosen || (j < ls.n && ls.r[j] == w);
+      const float* g = grads + static_cast<uint64_t>(w) * N;
+      float* a = acc + static_cast<uint64_t>(w) * N;
+      float gv[SPT][4], av[SPT][4];
+#pragma unroll
+      for (int s = 0; s < SPT; ++s) {
+        load4_stream<VEC>(a, e0[s], lo, hi, av[s]);
+        if (is_chosen) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) gv[s][c] = 0.0f;
+        } else {
+          load4_stream<VEC>(g, e0[s], lo, hi, gv[s]);
+        }
+      }
+#pragma unroll
+      for (int s = 0; s < SPT; ++s) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (!is_chosen) av[s][c] = accumulate(av[s][c], gv[s][c], momentum);
+          if ((in_set[s] >> c) & 1u) {
+            sum[s][c] = (w == 0) ? av[s][c] : __fadd_rn(sum[s][c], av[s][c]);
+            av[s][c] = 0.0f;
+          }
+        }
+        if (!is_chosen || in_set[s]) store4<VEC>(a, e0[s], lo, hi, av[s]);
+      }
+    }
+#pragma unroll
+    for (int s = 0; s < SPT; ++s) {
+      float out[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) out[c] = ((in_set[s] >> c) & 1u) ? __fadd_rn(0.0f, sum[s][c]) : 0.0f;
+      store4<VEC>(update, e0[s], lo, hi, out);
+    }
   }
 }
 
