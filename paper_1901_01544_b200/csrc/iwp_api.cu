@@ -73,7 +73,7 @@ struct iwp_ctx {
   float* sel_val = nullptr;
   int* d_status = nullptr;
   // optional per-stage CUDA-event timing (option "time_stages")
-  int time_stages = 0;  // 0 off, 1 every stage boundary, 2 only around the streaming stage
+  int time_stages = 0;  // 0 off, 1 every stage boundary, 2 only around the dominant streaming stage
   std::vector<cudaEvent_t> stage_events;  // N_STAGES + 1 events per timed step
   // staging for iwp_step_host
   float* stg_grads = nullptr;
@@ -92,7 +92,9 @@ const char* const kStageKeys[N_STAGES] = {"time_small_ns", "time_sample_ns", "ti
 void stage_mark_at(iwp_ctx* c, int boundary) {
   if (!c->time_stages) return;
   cudaEvent_t e = nullptr;
-  const bool wanted = c->time_stages == 1 || boundary == ST_ACCUMULATE || boundary == ST_ACCUMULATE + 1;
+  // the dominant stage: the streaming pass of the ratio mode, the fused all-worker pass of the threshold mode
+  const int dominant = c->threshold_mode ? ST_GATHER : ST_ACCUMULATE;
+  const bool wanted = c->time_stages == 1 || boundary == dominant || boundary == dominant + 1;
   if (wanted) {
     if (cudaEventCreate(&e) != cudaSuccess) {
       cudaGetLastError();
@@ -568,8 +570,9 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
   return IWP_OK;
 }
 
-// The threshold-mode step: plain accumulate of every worker, then count / scan / compact on the
-// chosen node's residual alone, then gather, ordered sum, scatter and zeroing at its index set.
+// The threshold-mode step: accumulate the chosen nodes, count / scan / compact their masks into the
+// index list and a bit per element, then one pass over all workers that accumulates the others, sums
+// in worker order and zeroes at the set bits, and writes the dense update.
 template <bool VEC>
 int run_step_threshold(iwp_ctx* c, const float* grads, const float* weights, float* update, int32_t leader) {
   const Plan& p = c->plan;

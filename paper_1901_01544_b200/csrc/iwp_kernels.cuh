@@ -1465,13 +1465,16 @@ __global__ void __launch_bounds__(THREADS)
       for (int c = 0; c < 4; ++c) sum[s][c] = 0.0f;
     }
     if (!__syncthreads_or(any)) continue;  // this half of the window lies outside a ragged tile
-    for (int w = 0; w < W; ++w) {
-      bool is_chosen = false;
+    // the loads of worker w + 1 are issued before worker w's values are combined and stored
+    auto chosen = [&](int w) {
+      bool c = false;
 #pragma unroll
-      for (int j = 0; j < MAX_LEADERS; ++j) is_chosen = is_chosen || (j < ls.n && ls.r[j] == w);
+      for (int j = 0; j < MAX_LEADERS; ++j) c = c || (j < ls.n && ls.r[j] == w);
+      return c;
+    };
+    auto fetch = [&](int w, bool is_chosen, float (&gv)[SPT][4], float (&av)[SPT][4]) {
       const float* g = grads + static_cast<uint64_t>(w) * N;
-      float* a = acc + static_cast<uint64_t>(w) * N;
-      float gv[SPT][4], av[SPT][4];
+      const float* a = acc + static_cast<uint64_t>(w) * N;
 #pragma unroll
       for (int s = 0; s < SPT; ++s) {
         load4_stream<VEC>(a, e0[s], lo, hi, av[s]);
@@ -1482,6 +1485,18 @@ __global__ void __launch_bounds__(THREADS)
           load4_stream<VEC>(g, e0[s], lo, hi, gv[s]);
         }
       }
+    };
+    float gv[SPT][4], av[SPT][4];
+    bool is_chosen = chosen(0);
+    fetch(0, is_chosen, gv, av);
+    for (int w = 0; w < W; ++w) {
+      float gn[SPT][4], an[SPT][4];
+      bool next_chosen = false;
+      if (w + 1 < W) {
+        next_chosen = chosen(w + 1);
+        fetch(w + 1, next_chosen, gn, an);
+      }
+      float* a = acc + static_cast<uint64_t>(w) * N;
 #pragma unroll
       for (int s = 0; s < SPT; ++s) {
 #pragma unroll
@@ -1493,6 +1508,17 @@ __global__ void __launch_bounds__(THREADS)
           }
         }
         if (!is_chosen || in_set[s]) store4<VEC>(a, e0[s], lo, hi, av[s]);
+      }
+      if (w + 1 < W) {
+#pragma unroll
+        for (int s = 0; s < SPT; ++s) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            gv[s][c] = gn[s][c];
+            av[s][c] = an[s][c];
+          }
+        }
+        is_chosen = next_chosen;
       }
     }
 #pragma unroll
