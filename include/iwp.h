@@ -141,8 +141,13 @@ int iwp_set_momentum(iwp_ctx* ctx, float m);
  *   update_dev   N floats, fully overwritten: +0 outside the index set, the ordered worker sum
  *                inside; must not alias the other two
  * Asynchronous: enqueues kernels on the context's stream and returns without synchronising;
- * the three buffers must stay valid until the stream has run the step.  128-bit accesses are
- * used when N % 4 == 0 and all three pointers are 16-byte aligned, scalar accesses otherwise.
+ * the three buffers must stay valid until the stream has run the step, after which the caller may
+ * change or free them.  When the stream has run the step, update_dev and the residuals are final.
+ * The (index, value) lists of workers other than the leader, which nothing in the step consumes,
+ * may still be in the making on streams of the library's own (option "overlap"); they read library
+ * memory only, and every accessor, iwp_sync_status() and the next step order themselves after them.
+ * 128-bit accesses are used when N % 4 == 0 and all three pointers are 16-byte aligned, scalar
+ * accesses otherwise.
  * Advances the step counter.  Errors: IWP_ERR_INVALID (NULL), IWP_ERR_CUDA (launch failure). */
 int iwp_step(iwp_ctx* ctx, const float* grads_dev, const float* weights_dev, float* update_dev);
 
@@ -191,9 +196,15 @@ int iwp_reset(iwp_ctx* ctx);
  *                      for element i at step t; 0 (default) = off
  *   "speculate"        1 (default) = sample-based threshold guess so that large layers are
  *                      read once; 0 = always the multi-pass exact select.  Both are exact.
+ *   "overlap"          1 = the leader's select runs beside the other workers' streaming pass and the
+ *                      other workers' selects beside the reduction and the head of the next step;
+ *                      0 = every kernel of a step in one sequence.  Same results either way; the
+ *                      default is 1 when the tiled layers hold at least 2^25 elements over all
+ *                      workers (below that the extra launches cost more than they hide), else 0.
  *   "time_stages"      1 = record a CUDA event at every stage boundary of each following step
- *                      (read the totals with iwp_get_stat); 2 = only before and after the streaming
- *                      stage (two events per step); 0 = stop and discard them
+ *                      (read the totals with iwp_get_stat; steps run as with "overlap" 0 meanwhile);
+ *                      2 = only before and after the dominant streaming stage (two events per step);
+ *                      0 = stop and discard them
  * Unknown key or out-of-range value: IWP_ERR_INVALID. */
 int iwp_set_option(iwp_ctx* ctx, const char* key, int64_t value);
 

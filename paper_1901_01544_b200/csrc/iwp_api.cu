@@ -28,6 +28,16 @@ struct iwp_ctx {
   cudaStream_t stream = nullptr;
   cudaStream_t side = nullptr;       // the one-CTA path of small layers runs here, beside the tiled path
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_fork2 = nullptr, ev_join2 = nullptr;
+  // Overlapped schedule of the single-read path: the leader's select runs on side_a under the other
+  // workers' streaming pass; the other workers' selects run on side_a (next step's leader) and side_b
+  // (everybody else) beside the reduction and the head of the NEXT step, which waits for them just
+  // before it overwrites what they read.
+  int overlap = 1;  // 0 off, 1 on (the default is chosen by size at create)
+  cudaStream_t side_a = nullptr, side_b = nullptr;
+  cudaEvent_t ev_lead = nullptr, ev_lead_done = nullptr, ev_others = nullptr, ev_a2 = nullptr, ev_b = nullptr;
+  bool pending_a2 = false, pending_b = false;  // deferred selects of the last step not yet joined
+  int32_t predicted_next = -1;                 // the worker whose select pending_a2 covers
+  float* saved_w = nullptr;                    // [N] weights kept for deferred selects that fall back (k_save_weights)
   int device = 0;
   int64_t launches = 0;
   uint64_t device_bytes = 0;
@@ -42,7 +52,8 @@ struct iwp_ctx {
   uint2* d_state = nullptr;
   uint32_t* d_hist = nullptr;
   uint2* d_chunk_cnt = nullptr;
-  PairInfo* d_info = nullptr;     // threshold guess and candidate totals per pair
+  PairInfo* d_info = nullptr;     // threshold guess and candidate totals per pair, two copies used in turn
+  PairInfo* info_cur = nullptr;   // the copy the last step used
   uint2* d_guess = nullptr;       // read-only (guess, pre-test multiplier) per pair for the streaming pass
   float* side_val = nullptr;      // every worker's value at the leader's slot positions, laid out like cand_val
   uint32_t* sel_slot = nullptr;   // [K] slot position of each entry of the leader's list, or REF_NONE
@@ -115,10 +126,11 @@ void stage_clear(iwp_ctx* c) {
 struct Sizes {
   uint64_t acc, layers, tiles, chunks, small_ids, large_ids, state, hist, chunk_cnt, sel_idx, sel_val, status;
   uint64_t info, cand_key, cand_val, cand_idx, cand_cnt, guess, side_val, sel_slot, lead_lane, lead_tot, zmask, chunk_sfx;
+  uint64_t saved_w;
   uint64_t total() const {
     return acc + layers + tiles + chunks + small_ids + large_ids + state + hist + chunk_cnt + sel_idx + sel_val +
            status + info + cand_key + cand_val + cand_idx + cand_cnt + guess + side_val + sel_slot + lead_lane +
-           lead_tot + zmask + chunk_sfx;
+           lead_tot + zmask + chunk_sfx + saved_w;
   }
 };
 
@@ -144,7 +156,7 @@ Sizes sizes_of(const Plan& p, bool threshold_mode = false, uint64_t list_cap = 0
   bool any_spec = false;
   for (uint32_t l : p.large_layers) any_spec = any_spec || p.layers[l].sample != 0;
   const uint64_t slots = any_spec ? W * p.tiles.size() : 0;
-  s.info = at_least(pairs * sizeof(PairInfo));
+  s.info = at_least(2 * pairs * sizeof(PairInfo));
   s.cand_key = at_least(slots * CAND_CAP * sizeof(uint32_t));
   s.cand_val = at_least(slots * CAND_CAP * sizeof(float));
   s.cand_idx = at_least(slots * CAND_CAP * sizeof(uint16_t));
@@ -157,6 +169,7 @@ Sizes sizes_of(const Plan& p, bool threshold_mode = false, uint64_t list_cap = 0
   s.lead_tot = at_least(segs * sizeof(uint32_t));
   s.zmask = ((p.N >> 9) + 2) * 16 * sizeof(uint32_t);  // 32 sixteen-bit fields per 512 elements
   s.chunk_sfx = at_least((threshold_mode ? 0 : W) * p.chunks.size() * pass_bins(N_PASSES - 1) * sizeof(uint32_t));
+  s.saved_w = at_least((any_spec && !threshold_mode && W > 1) ? p.N * sizeof(float) : 0);
   return s;
 }
 
@@ -181,6 +194,14 @@ void free_all(iwp_ctx* c) {
     cudaStreamSynchronize(c->side);
     cudaStreamDestroy(c->side);
   }
+  for (cudaStream_t* q : {&c->side_a, &c->side_b}) {
+    if (*q) {
+      cudaStreamSynchronize(*q);
+      cudaStreamDestroy(*q);
+    }
+  }
+  for (cudaEvent_t e : {c->ev_lead, c->ev_lead_done, c->ev_others, c->ev_a2, c->ev_b})
+    if (e) cudaEventDestroy(e);
   if (c->ev_fork) cudaEventDestroy(c->ev_fork);
   if (c->ev_join) cudaEventDestroy(c->ev_join);
   if (c->ev_fork2) cudaEventDestroy(c->ev_fork2);
@@ -210,6 +231,7 @@ void free_all(iwp_ctx* c) {
   cudaFree(c->d_toff);
   cudaFree(c->d_list_len);
   cudaFree(c->chunk_sfx);
+  cudaFree(c->saved_w);
   cudaFree(c->sel_idx);
   cudaFree(c->sel_val);
   cudaFree(c->d_status);
@@ -226,9 +248,23 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA; \
   } while (0)
 
+// Makes the main stream wait for the selects a previous step left running on the side streams.
+int join_deferred(iwp_ctx* c) {
+  bool ok = true;
+  if (c->pending_a2) ok = cudaStreamWaitEvent(c->stream, c->ev_a2, 0) == cudaSuccess && ok;
+  if (c->pending_b) ok = cudaStreamWaitEvent(c->stream, c->ev_b, 0) == cudaSuccess && ok;
+  c->pending_a2 = c->pending_b = false;
+  if (!ok) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  return IWP_OK;
+}
+
 // Brings the residuals themselves up to date when the last step left its zeroing to the next
 // streaming pass (see k_sum_scatter) and somebody else is about to look at them.
 int flush_pending_zero(iwp_ctx* c) {
+  if (const int rc = join_deferred(c)) return rc;  // a deferred select may still be reading the residuals
   if (!c->zero_pending) return IWP_OK;
   const unsigned blocks = static_cast<unsigned>((c->zmask_words + THREADS - 1) / THREADS);
   k_flush_zmask<<<blocks, THREADS, 0, c->stream>>>(c->zmask, c->acc, c->zmask_words, c->plan.N, c->plan.W);
@@ -238,66 +274,175 @@ int flush_pending_zero(iwp_ctx* c) {
   return IWP_OK;
 }
 
+// Exact select (three histogram passes with their digit decisions) and ordered compaction of the
+// workers `ws` covers, on stream `st`.
+template <bool VEC>
+int select_and_write(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSel ws, int32_t leader, bool use_sfx) {
+  const Plan& p = c->plan;
+  const int W = p.W;
+  const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
+  const unsigned n_sel = static_cast<unsigned>(sel_count(ws, W));
+  if (n_sel == 0) return IWP_OK;
+  dim3 cgrid(n_chunks, n_sel), pgrid(static_cast<unsigned>(p.large_layers.size()), n_sel);
+  uint32_t* sfx = use_sfx ? c->chunk_sfx : nullptr;
+  for (int pass = 0; pass < N_PASSES; ++pass) {
+    k_hist<VEC><<<cgrid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_layers, c->info_cur, c->cand_key,
+                                           c->cand_cnt, c->d_state, c->d_hist, sfx, c->d_chunk_cnt, c->eps, p.N, W,
+                                           pass, n_chunks, ws);
+    IWP_LAUNCH_CHECK(c);
+    k_find_digit<<<pgrid, THREADS, 0, st>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->d_status, W, pass, ws);
+    IWP_LAUNCH_CHECK(c);
+  }
+  k_write<VEC><<<cgrid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur, c->cand_key,
+                                          c->cand_val, c->cand_idx, c->cand_cnt, c->d_state, c->d_chunk_cnt, c->sel_idx,
+                                          c->sel_val, c->sel_slot, sfx, c->d_status, c->eps, p.N, p.K, W, n_chunks,
+                                          leader, ws);
+  IWP_LAUNCH_CHECK(c);
+  return IWP_OK;
+}
+
+int32_t leader_of_step(const iwp_ctx* c, int64_t t) {
+  return c->leader_override >= 0 ? static_cast<int32_t>(c->leader_override)
+                                 : leader_at(c->seed, static_cast<uint64_t>(t), c->plan.W);
+}
+
 template <bool VEC>
 int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update, int32_t leader) {
   const Plan& p = c->plan;
   const int W = p.W;
   const uint64_t N = p.N, K = p.K;
   cudaStream_t s = c->stream;
+  auto cuda_ok = [](cudaError_t e) {
+    if (e == cudaSuccess) return true;
+    cudaGetLastError();
+    return false;
+  };
+  const bool tiled = !p.large_layers.empty();
+  const bool spec = tiled && c->speculate && c->spec_pairs > 0;
+  // the overlapped schedule (not while every stage boundary is being timed)
+  const bool pipe = spec && W > 1 && c->overlap == 1 && c->time_stages != 1 && c->side_a != nullptr && c->side_b != nullptr;
+  if (!pipe) {
+    const int rc = join_deferred(c);
+    if (rc != IWP_OK) return rc;
+  }
   stage_mark_at(c, 0);
   // Small layers touch nothing the tiled path touches until the final reduction, so when both kinds
   // exist their one-CTA kernel runs on a side stream, forked here and joined before the reduction.
-  const bool fork_small = !p.small_layers.empty() && !p.large_layers.empty() && c->side != nullptr;
-  bool join_others = false;  // the other workers' lists are still being written on the side stream
+  const bool fork_small = !p.small_layers.empty() && tiled && c->side != nullptr;
   if (!p.small_layers.empty()) {
     const size_t dyn = static_cast<size_t>(p.max_small_n) * sizeof(uint32_t);
     dim3 grid(static_cast<unsigned>(p.small_layers.size()), static_cast<unsigned>(W));
     cudaStream_t ss = s;
     if (fork_small) {
-      if (cudaEventRecord(c->ev_fork, s) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess) {
-        cudaGetLastError();
+      if (!cuda_ok(cudaEventRecord(c->ev_fork, s)) || !cuda_ok(cudaStreamWaitEvent(c->side, c->ev_fork, 0)))
         return IWP_ERR_CUDA;
-      }
       ss = c->side;
     }
     k_small<<<grid, THREADS, dyn, ss>>>(grads, weights, c->acc, update, c->d_layers, c->d_small_ids, c->sel_idx,
                                         c->sel_val, c->sel_slot, c->d_status, c->eps, N, K, leader, c->momentum);
     IWP_LAUNCH_CHECK(c);
-    if (fork_small && cudaEventRecord(c->ev_join, c->side) != cudaSuccess) {
-      cudaGetLastError();
-      return IWP_ERR_CUDA;
-    }
+    if (fork_small && !cuda_ok(cudaEventRecord(c->ev_join, c->side))) return IWP_ERR_CUDA;
   }
   stage_mark_at(c, 1);
-  const bool tiled = !p.large_layers.empty();
-  const bool spec = tiled && c->speculate && c->spec_pairs > 0;
   if (!spec) {  // the multi-pass path reads the residuals as they are
     const int rc = flush_pending_zero(c);
     if (rc != IWP_OK) return rc;
   }
+  // The per-pair records alternate between two copies, so that a select still running for the last
+  // step keeps reading its own while this step's sampling writes the other.
+  c->info_cur = c->d_info + static_cast<size_t>(c->t & 1) * c->n_pairs;
   if (tiled && !spec && !c->info_clean) {  // speculation was switched off: forget the old guesses
-    if (cudaMemsetAsync(c->d_info, 0xff, static_cast<size_t>(c->n_pairs) * sizeof(PairInfo), s) != cudaSuccess) {
-      cudaGetLastError();
+    if (!cuda_ok(cudaMemsetAsync(c->d_info, 0xff, 2 * static_cast<size_t>(c->n_pairs) * sizeof(PairInfo), s)))
       return IWP_ERR_CUDA;
-    }
     c->launches += 1;
     c->info_clean = true;
   }
   if (spec) {
     const size_t dyn = static_cast<size_t>(c->max_sample) * sizeof(uint32_t);
-    k_sample<<<c->n_pairs, SAMPLE_THREADS, dyn, s>>>(grads, weights, c->acc, c->d_layers, c->d_large_ids, c->d_info,
-                                             c->d_guess, c->zmask, c->eps, N, W, static_cast<uint32_t>(c->t),
-                                             c->momentum);
+    k_sample<<<c->n_pairs, SAMPLE_THREADS, dyn, s>>>(grads, weights, c->acc, c->d_layers, c->d_large_ids, c->info_cur,
+                                                     c->d_guess, c->zmask, c->eps, N, W, static_cast<uint32_t>(c->t),
+                                                     c->momentum);
     IWP_LAUNCH_CHECK(c);
     c->info_clean = false;
   }
-  stage_mark_at(c, 2);
+  const unsigned n_tiles = static_cast<unsigned>(p.tiles.size());
+  const unsigned gblocks = static_cast<unsigned>((K + THREADS - 1) / THREADS);
+  if (!pipe) stage_mark_at(c, 2);
+  if (pipe) {
+    // This step's leader was covered by side_a's deferred select if the last step foresaw it; any
+    // other worker may still be in side_b's.
+    if (c->pending_a2 && !cuda_ok(cudaStreamWaitEvent(s, c->ev_a2, 0))) return IWP_ERR_CUDA;
+    c->pending_a2 = false;
+    if (c->pending_b && leader != c->predicted_next) {
+      if (!cuda_ok(cudaStreamWaitEvent(s, c->ev_b, 0))) return IWP_ERR_CUDA;
+      c->pending_b = false;
+    }
+    stage_mark_at(c, 2);  // after the wait: the streaming stage is timed from where its first kernel may start
+    k_stream<VEC, true><<<(n_tiles + WARPS - 1) / WARPS, THREADS, 0, s>>>(
+        grads, weights, c->acc, update, c->d_tiles, c->info_cur, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
+        c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, 1, c->momentum);
+    IWP_LAUNCH_CHECK(c);
+    // the leader's select and list, under the other workers' streaming pass
+    if (!cuda_ok(cudaEventRecord(c->ev_lead, s)) || !cuda_ok(cudaStreamWaitEvent(c->side_a, c->ev_lead, 0)))
+      return IWP_ERR_CUDA;
+    int rc = select_and_write<VEC>(c, weights, c->side_a, WorkerSel{WorkerSel::ONLY, leader, -1}, leader, true);
+    if (rc != IWP_OK) return rc;
+    if (!cuda_ok(cudaEventRecord(c->ev_lead_done, c->side_a))) return IWP_ERR_CUDA;
+    if (c->pending_b && !cuda_ok(cudaStreamWaitEvent(s, c->ev_b, 0))) return IWP_ERR_CUDA;
+    c->pending_b = false;
+    const int wpc = (W - 1 < WARPS) ? W - 1 : WARPS;  // warps (= workers) per CTA
+    const int groups = (W - 1 + wpc - 1) / wpc;
+    k_stream<VEC, false><<<n_tiles * static_cast<unsigned>(groups), wpc * 32, 0, s>>>(
+        grads, weights, c->acc, update, c->d_tiles, c->info_cur, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
+        c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, groups,
+        c->momentum);
+    IWP_LAUNCH_CHECK(c);
+    if (c->zero_pending) {  // every marked residual has now been overwritten: forget the marks
+      if (!cuda_ok(cudaMemsetAsync(c->zmask, 0, c->zmask_words * sizeof(uint32_t), s))) return IWP_ERR_CUDA;
+      c->launches += 1;
+      c->zero_pending = false;
+    }
+    stage_mark_at(c, 3);
+    stage_mark_at(c, 4);
+    stage_mark_at(c, 5);
+    // The other workers' selects outlive the step: they read the library's copy of the weights
+    // (filled only where a pair fell back), the next step's leader first (its streaming pass comes first).
+    k_save_weights<<<static_cast<unsigned>(p.chunks.size()), THREADS, 0, s>>>(weights, c->saved_w, c->d_chunks, c->d_layers,
+                                                                            c->info_cur, W, leader);
+    IWP_LAUNCH_CHECK(c);
+    if (!cuda_ok(cudaEventRecord(c->ev_others, s))) return IWP_ERR_CUDA;
+    const int32_t next = leader_of_step(c, c->t + 1);
+    if (next != leader) {
+      if (!cuda_ok(cudaStreamWaitEvent(c->side_a, c->ev_others, 0))) return IWP_ERR_CUDA;
+      rc = select_and_write<VEC>(c, c->saved_w, c->side_a, WorkerSel{WorkerSel::ONLY, next, -1}, leader, true);
+      if (rc != IWP_OK) return rc;
+      if (!cuda_ok(cudaEventRecord(c->ev_a2, c->side_a))) return IWP_ERR_CUDA;
+      c->pending_a2 = true;
+    }
+    const WorkerSel rest{WorkerSel::EXCEPT, leader, next};
+    if (sel_count(rest, W) > 0) {
+      if (!cuda_ok(cudaStreamWaitEvent(c->side_b, c->ev_others, 0))) return IWP_ERR_CUDA;
+      rc = select_and_write<VEC>(c, c->saved_w, c->side_b, rest, leader, true);
+      if (rc != IWP_OK) return rc;
+      if (!cuda_ok(cudaEventRecord(c->ev_b, c->side_b))) return IWP_ERR_CUDA;
+      c->pending_b = true;
+    }
+    c->predicted_next = next;
+    // the reduction needs the leader's list and the small layers
+    if (!cuda_ok(cudaStreamWaitEvent(s, c->ev_lead_done, 0))) return IWP_ERR_CUDA;
+    if (fork_small && !cuda_ok(cudaStreamWaitEvent(s, c->ev_join, 0))) return IWP_ERR_CUDA;
+    k_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->sel_slot, c->side_val,
+                                              c->cand_val, c->acc, update, c->zmask, N, K, W, leader);
+    IWP_LAUNCH_CHECK(c);
+    c->zero_pending = true;
+    stage_mark_at(c, 6);
+    return IWP_OK;
+  }
   if (tiled) {
-    const unsigned n_tiles = static_cast<unsigned>(p.tiles.size());
     if (spec) {
-      // the leader's workers first (records where its candidates sit), then everybody else
+      // the leader's worker first (records where its candidates sit), then everybody else
       k_stream<VEC, true><<<(n_tiles + WARPS - 1) / WARPS, THREADS, 0, s>>>(
-          grads, weights, c->acc, update, c->d_tiles, c->d_info, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
+          grads, weights, c->acc, update, c->d_tiles, c->info_cur, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
           c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, 1,
           c->momentum);
       if (W > 1) {
@@ -305,16 +450,13 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
         const int wpc = (W - 1 < WARPS) ? W - 1 : WARPS;  // warps (= workers) per CTA
         const int groups = (W - 1 + wpc - 1) / wpc;
         k_stream<VEC, false><<<n_tiles * static_cast<unsigned>(groups), wpc * 32, 0, s>>>(
-            grads, weights, c->acc, update, c->d_tiles, c->d_info, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
+            grads, weights, c->acc, update, c->d_tiles, c->info_cur, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
             c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, groups,
             c->momentum);
       }
       if (c->zero_pending) {  // every marked residual has now been overwritten: forget the marks
         IWP_LAUNCH_CHECK(c);
-        if (cudaMemsetAsync(c->zmask, 0, c->zmask_words * sizeof(uint32_t), s) != cudaSuccess) {
-          cudaGetLastError();
-          return IWP_ERR_CUDA;
-        }
+        if (!cuda_ok(cudaMemsetAsync(c->zmask, 0, c->zmask_words * sizeof(uint32_t), s))) return IWP_ERR_CUDA;
         c->zero_pending = false;
       }
     } else {
@@ -323,63 +465,49 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     IWP_LAUNCH_CHECK(c);
   }
   stage_mark_at(c, 3);
+  bool join_others = false;  // the other workers' lists are still being written on the side stream
   if (tiled) {
     const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
-    dim3 cgrid(n_chunks, static_cast<unsigned>(W));
+    dim3 cgrid(n_chunks, static_cast<unsigned>(W)), pgrid(static_cast<unsigned>(p.large_layers.size()), static_cast<unsigned>(W));
+    const WorkerSel all{WorkerSel::ALL, 0, -1};
     for (int pass = 0; pass < N_PASSES; ++pass) {
-      k_hist<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->d_info, c->cand_key,
+      k_hist<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->info_cur, c->cand_key,
                                             c->cand_cnt, c->d_state, c->d_hist, c->chunk_sfx, c->d_chunk_cnt, c->eps, N,
-                                            W, pass, n_chunks);
+                                            W, pass, n_chunks, all);
       IWP_LAUNCH_CHECK(c);
-      k_find_digit<<<c->n_pairs, THREADS, 0, s>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->d_status, W,
-                                                  pass);
+      k_find_digit<<<pgrid, THREADS, 0, s>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->d_status, W, pass,
+                                             all);
       IWP_LAUNCH_CHECK(c);
     }
-  }
-  stage_mark_at(c, 4);
-  if (tiled) {
-    const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
-    dim3 cgrid(n_chunks, static_cast<unsigned>(W));
+    stage_mark_at(c, 4);
     // The reduction needs the leader's list only: write that one here and the other workers' lists on
     // the side stream, beside the reduction; they are joined at the end of the step.
     const bool split = spec && W > 1 && c->side != nullptr;
-    const uint32_t* sfx = c->chunk_sfx;
-    if (split) {
-      if (cudaEventRecord(c->ev_fork2, s) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork2, 0) != cudaSuccess) {
-        cudaGetLastError();
-        return IWP_ERR_CUDA;
-      }
-      dim3 ogrid(n_chunks, static_cast<unsigned>(W - 1));
-      k_write<VEC><<<ogrid, THREADS, 0, c->side>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->d_info,
-                                                   c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
-                                                   c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, sfx,
-                                                   c->d_status, c->eps, N, K, W, n_chunks, leader, 2);
-      IWP_LAUNCH_CHECK(c);
-      if (cudaEventRecord(c->ev_join2, c->side) != cudaSuccess) {
-        cudaGetLastError();
-        return IWP_ERR_CUDA;
-      }
-      dim3 lgrid(n_chunks, 1);
-      k_write<VEC><<<lgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->d_info,
+    auto write = [&](cudaStream_t st, WorkerSel ws) {
+      dim3 grid(n_chunks, static_cast<unsigned>(sel_count(ws, W)));
+      k_write<VEC><<<grid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur,
                                              c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
-                                             c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, sfx, c->d_status,
-                                             c->eps, N, K, W, n_chunks, leader, 1);
+                                             c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, c->chunk_sfx,
+                                             c->d_status, c->eps, N, K, W, n_chunks, leader, ws);
+    };
+    if (split) {
+      if (!cuda_ok(cudaEventRecord(c->ev_fork2, s)) || !cuda_ok(cudaStreamWaitEvent(c->side, c->ev_fork2, 0)))
+        return IWP_ERR_CUDA;
+      write(c->side, WorkerSel{WorkerSel::EXCEPT, leader, -1});
+      IWP_LAUNCH_CHECK(c);
+      if (!cuda_ok(cudaEventRecord(c->ev_join2, c->side))) return IWP_ERR_CUDA;
+      write(s, WorkerSel{WorkerSel::ONLY, leader, -1});
       IWP_LAUNCH_CHECK(c);
       join_others = true;
     } else {
-      k_write<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->d_info,
-                                             c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
-                                             c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, sfx, c->d_status,
-                                             c->eps, N, K, W, n_chunks, leader, 0);
+      write(s, all);
       IWP_LAUNCH_CHECK(c);
     }
+  } else {
+    stage_mark_at(c, 4);
   }
   stage_mark_at(c, 5);
-  if (fork_small && cudaStreamWaitEvent(s, c->ev_join, 0) != cudaSuccess) {
-    cudaGetLastError();
-    return IWP_ERR_CUDA;
-  }
-  const unsigned gblocks = static_cast<unsigned>((K + THREADS - 1) / THREADS);
+  if (fork_small && !cuda_ok(cudaStreamWaitEvent(s, c->ev_join, 0))) return IWP_ERR_CUDA;
   if (spec) {
     k_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->sel_slot, c->side_val,
                                               c->cand_val, c->acc, update, c->zmask, N, K, W, leader);
@@ -389,10 +517,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
                                                      N, K, W);
   }
   IWP_LAUNCH_CHECK(c);
-  if (join_others && cudaStreamWaitEvent(s, c->ev_join2, 0) != cudaSuccess) {
-    cudaGetLastError();
-    return IWP_ERR_CUDA;
-  }
+  if (join_others && !cuda_ok(cudaStreamWaitEvent(s, c->ev_join2, 0))) return IWP_ERR_CUDA;
   stage_mark_at(c, 6);
   return IWP_OK;
 }
@@ -506,6 +631,7 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
   A(&c->lead_tot, sz.lead_tot);
   A(&c->zmask, sz.zmask);
   A(&c->chunk_sfx, sz.chunk_sfx);
+  A(&c->saved_w, sz.saved_w);
   A(&c->sel_idx, sz.sel_idx);
   A(&c->sel_val, sz.sel_val);
   A(&c->d_status, sz.status);
@@ -559,6 +685,22 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
   ok = ok && cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&c->ev_fork2, cudaEventDisableTiming) == cudaSuccess;
   ok = ok && cudaEventCreateWithFlags(&c->ev_join2, cudaEventDisableTiming) == cudaSuccess;
+  if (ok && !threshold_mode) {
+    int prio_lo = 0, prio_hi = 0;
+    ok = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi) == cudaSuccess;
+    // The selects are short chains of small dependent kernels: at high priority their CTAs take the
+    // next free slots of a streaming pass running beside them and the chains finish inside their windows.
+    ok = ok && cudaStreamCreateWithPriority(&c->side_a, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithPriority(&c->side_b, cudaStreamNonBlocking, prio_hi) == cudaSuccess;
+    for (cudaEvent_t* e : {&c->ev_lead, &c->ev_lead_done, &c->ev_others, &c->ev_a2, &c->ev_b})
+      ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+  }
+  c->info_cur = c->d_info;
+  {  // the overlapped schedule costs extra launches: it pays once a step streams some hundred megabytes
+    uint64_t tiled = 0;
+    for (uint32_t l : p.large_layers) tiled += p.layers[l].n;
+    c->overlap = (tiled * static_cast<uint64_t>(W) >= (1ull << 25)) ? 1 : 0;
+  }
   ok = ok && cudaDeviceSynchronize() == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
@@ -684,6 +826,11 @@ int iwp_set_momentum(iwp_ctx* c, float m) {
 
 int iwp_set_stream(iwp_ctx* c, void* stream) {
   if (!c) return IWP_ERR_INVALID;
+  // deferred selects were ordered against the old stream: let them finish before the switch
+  if (c->pending_a2) cudaEventSynchronize(c->ev_a2);
+  if (c->pending_b) cudaEventSynchronize(c->ev_b);
+  c->pending_a2 = c->pending_b = false;
+  cudaGetLastError();
   c->stream = static_cast<cudaStream_t>(stream);
   return IWP_OK;
 }
@@ -739,6 +886,7 @@ int iwp_step_host(iwp_ctx* c, const float* grads, const float* weights, float* u
 
 int iwp_sync_status(iwp_ctx* c) {
   if (!c) return IWP_ERR_INVALID;
+  if (const int jrc = join_deferred(c)) return jrc;
   int st = 0;
   if (cudaMemcpyAsync(&st, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
       cudaStreamSynchronize(c->stream) != cudaSuccess) {
@@ -774,6 +922,7 @@ int iwp_get_step(iwp_ctx* c, int64_t* t) {
 
 int iwp_set_step(iwp_ctx* c, int64_t t) {
   if (!c || t < 0) return IWP_ERR_INVALID;
+  if (const int jrc = join_deferred(c)) return jrc;
   c->t = t;
   return IWP_OK;
 }
@@ -798,6 +947,7 @@ int iwp_get_residual(iwp_ctx* c, int32_t w, float* dst) {
 
 int iwp_set_residual(iwp_ctx* c, int32_t w, const float* src) {
   if (!c || !src || w < 0 || w >= c->plan.W) return IWP_ERR_INVALID;
+  if (const int jrc = join_deferred(c)) return jrc;
   if (const int rc = flush_pending_zero(c)) return rc;
   const uint64_t N = c->plan.N;
   if (cudaMemcpyAsync(c->acc + static_cast<uint64_t>(w) * N, src, N * sizeof(float), cudaMemcpyDeviceToDevice,
@@ -810,6 +960,7 @@ int iwp_set_residual(iwp_ctx* c, int32_t w, const float* src) {
 
 int iwp_get_selection(iwp_ctx* c, int32_t w, uint32_t* idx, float* val) {
   if (!c || w < 0 || w >= c->plan.W) return IWP_ERR_INVALID;
+  if (const int jrc = join_deferred(c)) return jrc;
   if (c->threshold_mode) {  // one list, the chosen node's; the whole capacity is copied
     if (w != c->leader) return IWP_ERR_INVALID;
     bool ok1 = true;
@@ -842,6 +993,7 @@ int iwp_get_selection(iwp_ctx* c, int32_t w, uint32_t* idx, float* val) {
 
 int iwp_get_mask(iwp_ctx* c, uint8_t* dst) {
   if (!c || !dst) return IWP_ERR_INVALID;
+  if (const int jrc = join_deferred(c)) return jrc;
   const uint64_t N = c->plan.N, K = c->plan.K;
   if (cudaMemsetAsync(dst, 0, N, c->stream) != cudaSuccess) {
     cudaGetLastError();
@@ -861,6 +1013,7 @@ int iwp_get_mask(iwp_ctx* c, uint8_t* dst) {
 
 int iwp_reset(iwp_ctx* c) {
   if (!c) return IWP_ERR_INVALID;
+  if (const int jrc = join_deferred(c)) return jrc;
   const Sizes sz = sizes_of(c->plan, c->threshold_mode, c->list_cap);
   bool ok = cudaMemsetAsync(c->acc, 0, sz.acc, c->stream) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->zmask, 0, sz.zmask, c->stream) == cudaSuccess;
@@ -882,6 +1035,7 @@ int iwp_reset(iwp_ctx* c) {
 
 int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
   if (!c || !key) return IWP_ERR_INVALID;
+  if (const int jrc = join_deferred(c)) return jrc;
   if (!std::strcmp(key, "leader_override")) {
     if (v < -1 || v >= c->plan.W) return IWP_ERR_INVALID;
     c->leader_override = v;
@@ -909,6 +1063,11 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
     c->n_leaders = static_cast<int32_t>(v);
     return IWP_OK;
   }
+  if (!std::strcmp(key, "overlap")) {
+    if (v != 0 && v != 1) return IWP_ERR_INVALID;
+    c->overlap = static_cast<int>(v);
+    return IWP_OK;
+  }
   if (!std::strcmp(key, "speculate")) {
     if (v != 0 && v != 1) return IWP_ERR_INVALID;
     c->speculate = v != 0;
@@ -919,6 +1078,7 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
 
 int iwp_get_stat(iwp_ctx* c, const char* key, int64_t* value) {
   if (!c || !key || !value) return IWP_ERR_INVALID;
+  if (const int jrc = join_deferred(c)) return jrc;
   if (!std::strcmp(key, "launches")) {
     *value = c->launches;
     return IWP_OK;
@@ -960,7 +1120,7 @@ int iwp_get_stat(iwp_ctx* c, const char* key, int64_t* value) {
     *value = 0;
     if (!c->speculate || c->spec_pairs == 0 || c->info_clean) return IWP_OK;
     std::vector<PairInfo> h(c->n_pairs);
-    if (cudaMemcpyAsync(h.data(), c->d_info, h.size() * sizeof(PairInfo), cudaMemcpyDeviceToHost, c->stream) !=
+    if (cudaMemcpyAsync(h.data(), c->info_cur, h.size() * sizeof(PairInfo), cudaMemcpyDeviceToHost, c->stream) !=
             cudaSuccess ||
         cudaStreamSynchronize(c->stream) != cudaSuccess) {
       cudaGetLastError();
@@ -1053,11 +1213,12 @@ int run_select_static(StaticScratch* s, const float* residual, const float* weig
   k_static_setup<<<1, THREADS, 0, st>>>(s, n, k, n_chunks);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   dim3 grid(n_chunks, 1);
+  const WorkerSel all{WorkerSel::ALL, 0, -1};
   for (int pass = 0; pass < N_PASSES; ++pass) {
     k_hist<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr, &s->state,
-                                          s->hist, nullptr, nullptr, eps, 0, 1, pass, n_chunks);
+                                          s->hist, nullptr, nullptr, eps, 0, 1, pass, n_chunks, all);
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
-    k_find_digit<<<1, THREADS, 0, st>>>(&s->state, s->hist, &s->layer, &s->large_id, &s->status, 1, pass);
+    k_find_digit<<<1, THREADS, 0, st>>>(&s->state, s->hist, &s->layer, &s->large_id, &s->status, 1, pass, all);
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   }
   k_count<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr, &s->state,
@@ -1065,7 +1226,7 @@ int run_select_static(StaticScratch* s, const float* residual, const float* weig
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   k_write<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, nullptr, &s->layer, &s->info, nullptr, nullptr,
                                          nullptr, nullptr, &s->state, s->chunk_cnt, idx, val, nullptr, nullptr,
-                                         &s->status, eps, 0, 0, 1, n_chunks, -1, 0);
+                                         &s->status, eps, 0, 0, 1, n_chunks, -1, all);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   return IWP_OK;
 }

@@ -40,6 +40,28 @@ __device__ __forceinline__ bool pair_is_cand(const PairInfo& pi, uint32_t k) {
   return pi.guess != GUESS_NONE && pi.total >= k && (pi.flags & 1u) == 0u;
 }
 
+// Which workers a launch of the select kernels covers: blockIdx.y runs over the covered workers.
+//   ALL: every worker;  ONLY: worker a, then worker b (b < 0 or b == a: a alone);
+//   EXCEPT: every worker but a and b, ascending.
+struct WorkerSel {
+  int mode, a, b;
+  enum { ALL = 0, ONLY = 1, EXCEPT = 2 };
+};
+__host__ __device__ inline int sel_count(const WorkerSel& ws, int W) {
+  const int named = (ws.b < 0 || ws.b == ws.a) ? 1 : 2;
+  return ws.mode == WorkerSel::ALL ? W : (ws.mode == WorkerSel::ONLY ? named : W - named);
+}
+__device__ __forceinline__ int sel_worker(const WorkerSel& ws, int y) {
+  if (ws.mode == WorkerSel::ALL) return y;
+  if (ws.mode == WorkerSel::ONLY) return y == 0 ? ws.a : ws.b;
+  const int b = ws.b < 0 ? ws.a : ws.b;
+  const int lo = ws.a < b ? ws.a : b, hi = ws.a < b ? b : ws.a;
+  int w = y;
+  if (w >= lo) ++w;
+  if (hi != lo && w >= hi) ++w;
+  return w;
+}
+
 // ---------------------------------------------------------------------------------------
 // element helpers
 // ---------------------------------------------------------------------------------------
@@ -701,12 +723,12 @@ __global__ void __launch_bounds__(THREADS)
            const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt,
            const uint2* __restrict__ state,
            uint32_t* __restrict__ hist, uint32_t* __restrict__ chunk_sfx, uint2* __restrict__ chunk_cnt, float eps,
-           uint64_t N, int W, int pass, uint32_t n_chunks) {
+           uint64_t N, int W, int pass, uint32_t n_chunks, WorkerSel ws) {
   __shared__ uint32_t sh[NBINS];
   __shared__ uint32_t sh_warp[WARPS];
   __shared__ uint32_t sh_above;
   const Chunk c = chunks[blockIdx.x];
-  const int w = blockIdx.y;
+  const int w = sel_worker(ws, static_cast<int>(blockIdx.y));
   const LayerDesc L = layers[c.layer];
   const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
   const int shift = pass_shift(pass), nb = pass_bins(pass);
@@ -795,16 +817,17 @@ __global__ void __launch_bounds__(THREADS)
   }
 }
 
-// Digit decision for every (worker, layer) pair of the tiled path; grid = pairs.
+// Digit decision for (worker, layer) pairs of the tiled path; grid = (tiled layers, covered workers).
 // Reads the pair's histogram, clears it for the next pass, extends the key prefix.
 // After the last pass state = (threshold key T, number r of T-valued elements to keep).
 __global__ void __launch_bounds__(THREADS)
     k_find_digit(uint2* __restrict__ state, uint32_t* __restrict__ hist, const LayerDesc* __restrict__ layers,
-                 const uint32_t* __restrict__ large_ids, int* __restrict__ status, int W, int pass) {
+                 const uint32_t* __restrict__ large_ids, int* __restrict__ status, int W, int pass,
+                 WorkerSel ws) {
   __shared__ uint32_t sh[NBINS];
   __shared__ uint32_t sh_scan[THREADS];
   __shared__ uint32_t res[4];
-  const uint32_t pair = blockIdx.x;
+  const uint32_t pair = blockIdx.x * static_cast<uint32_t>(W) + static_cast<uint32_t>(sel_worker(ws, static_cast<int>(blockIdx.y)));
   const int nb = pass_bins(pass), shift = pass_shift(pass);
   uint32_t* gh = hist + static_cast<uint64_t>(pair) * NBINS;
   for (int b = threadIdx.x; b < nb; b += THREADS) {
@@ -899,14 +922,11 @@ __global__ void __launch_bounds__(THREADS)
             const uint2* __restrict__ state, const uint2* __restrict__ chunk_cnt, uint32_t* __restrict__ sel_idx,
             float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot, const uint32_t* __restrict__ chunk_sfx,
             int* __restrict__ status, float eps, uint64_t N, uint64_t K, int W, uint32_t n_chunks, int leader,
-            int which) {
+            WorkerSel ws) {
   __shared__ uint32_t sh_warp[WARPS];
   __shared__ uint32_t sh_base[2];
   const Chunk c = chunks[blockIdx.x];
-  // which = 0: blockIdx.y is the worker; 1: only the leader; 2: everybody but the leader
-  const int w = which == 0 ? static_cast<int>(blockIdx.y)
-                           : (which == 1 ? leader : (static_cast<int>(blockIdx.y) < leader ? static_cast<int>(blockIdx.y)
-                                                                                              : static_cast<int>(blockIdx.y) + 1));
+  const int w = sel_worker(ws, static_cast<int>(blockIdx.y));
   const LayerDesc L = layers[c.layer];
   const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
   const uint2 st = state[pair];
@@ -1085,7 +1105,7 @@ __global__ void __launch_bounds__(THREADS)
           if (pos < L.k) {
             out_i[pos] = static_cast<uint32_t>(e0 + q);
             out_v[pos] = av[q];
-            if (is_leader) sel_slot[L.koff + pos] = REF_NONE;
+            if (is_leader) sel_slot[L.koff + pos] = REF_LAZY;
           } else {
             atomicMin(status, STATUS_INTERNAL);
           }
@@ -1182,12 +1202,31 @@ __global__ void __launch_bounds__(THREADS)
   update[i] = __fadd_rn(0.0f, s);
 }
 
+// A worker's select that is left running on a side stream past the end of the step may still need
+// the weights if its pair has to fall back to the multi-pass path, and the caller is free to change
+// them once the step's stream work is done.  So the weights of every layer in which a worker other
+// than the leader failed its single-read check are copied here, on the step's own stream; that
+// select then reads the copy.  grid = chunks; nearly always every CTA returns at once.
+__global__ void __launch_bounds__(THREADS)
+    k_save_weights(const float* __restrict__ weights, float* __restrict__ saved, const Chunk* __restrict__ chunks,
+                   const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info, int W, int leader) {
+  const Chunk c = chunks[blockIdx.x];
+  const LayerDesc L = layers[c.layer];
+  bool failed = false;
+  for (int w = threadIdx.x; w < W; w += THREADS)
+    failed = failed || (w != leader && !pair_is_cand(info[static_cast<uint32_t>(L.large_index) * W + w], L.k));
+  if (!__syncthreads_or(failed)) return;
+  for (uint32_t i = threadIdx.x; i < c.len; i += THREADS) saved[c.a + i] = weights[c.a + i];
+}
+
 // Steps (e)-(g) on the single-read path.  For a list entry of the leader that came from a candidate
 // slot, every other worker's value at that slot position was written to the side buffer by the
 // streaming pass (the leader's own value is the candidate value): read the W values, sum them in
-// ascending worker order, scatter.  Entries from the one-CTA path or from a pair that fell back to
-// the multi-pass select carry REF_NONE and are gathered from the residuals.  Either way the sent
-// residuals are zeroed.
+// ascending worker order, scatter, and mark the element for zeroing by the next streaming pass.
+// Entries from the one-CTA path carry REF_NONE: gathered from the residuals, which are zeroed here
+// (no streaming pass visits them).  Entries from a pair that fell back to the multi-pass select
+// carry REF_LAZY: gathered from the residuals and marked like the first kind, because another
+// worker's multi-pass select may still be reading that layer's residuals on a side stream.
 __global__ void __launch_bounds__(THREADS)
     k_sum_scatter(const uint32_t* __restrict__ leader_idx, const uint32_t* __restrict__ sel_slot,
                   const float* __restrict__ side_val, const float* __restrict__ cand_val, float* __restrict__ acc,
@@ -1198,7 +1237,7 @@ __global__ void __launch_bounds__(THREADS)
   const uint64_t i = leader_idx[j];
   const uint32_t ref = sel_slot[j];
   float s = 0.0f;
-  if (ref != REF_NONE) {
+  if (ref < REF_LAZY) {
     const uint64_t tile = ref / CAND_CAP, at = ref % CAND_CAP;
     const uint64_t q0 = tile * W * CAND_CAP + at;
     for (int w0 = 0; w0 < W; w0 += 8) {
@@ -1226,7 +1265,11 @@ __global__ void __launch_bounds__(THREADS)
         if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
       }
     }
-    for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
+    if (ref == REF_LAZY) {
+      atomicOr(&zmask[zmask_word(i)], zmask_bit(i));
+    } else {
+      for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
+    }
   }
   update[i] = __fadd_rn(0.0f, s);
 }

@@ -26,7 +26,8 @@ constexpr uint32_t SAMPLE_MAX = 16384;
 constexpr uint32_t GUESS_NONE = 0xffffffffu;  // no importance pattern reaches this value
 constexpr uint32_t SEG_ELEMS = 512;           // elements a warp handles per iteration of the streaming pass
 constexpr uint32_t SEGS_PER_TILE = TILE / SEG_ELEMS;
-constexpr uint32_t REF_NONE = 0xffffffffu;    // list entry has no side values: gather from the residuals
+constexpr uint32_t REF_NONE = 0xffffffffu;    // list entry has no side values: gather from the residuals, zero them
+constexpr uint32_t REF_LAZY = 0xfffffffeu;    // the same, but leave the zeroing to the next streaming pass
 
 struct LayerDesc {
   uint32_t off;         // flat offset of the first element

@@ -41,8 +41,15 @@ def compare_state(pr: Pruner, orc: "oracle.Oracle", update_gpu: torch.Tensor, up
 
 
 def run_parity(layer_sizes, W, ratio, eps, seed, steps, weights: torch.Tensor, grads_fn, options=None,
-               leader_overrides=None, check_mask=True, threads=0, residual_every=1, momentum=None):
+               leader_overrides=None, check_mask=True, threads=0, residual_every=1, momentum=None, state_every=1,
+               weights_fn=None):
     """weights: CUDA tensor [N]; grads_fn(t) -> CUDA tensor [W, N].
+
+    state_every: lists, mask, residuals and the device status are looked at only every that many steps
+    and after the last one; in between only the update is compared, which asks the library for nothing,
+    so whatever it leaves running past the end of a step keeps running into the next one.
+    weights_fn(t) -> CUDA tensor [N]: if given, `weights` is overwritten in place with it right after
+    step t - 1 was enqueued, as an optimizer would.
 
     residual_every: residuals are read back (and compared) only every that many steps and after the
     last one.  Reading them makes the library bring them up to date first, so runs that look only at
@@ -63,8 +70,16 @@ def run_parity(layer_sizes, W, ratio, eps, seed, steps, weights: torch.Tensor, g
             pr.set_option("leader_override", leader_overrides[t])
             orc.set_leader_override(leader_overrides[t])
         g = grads_fn(t)
+        if weights_fn is not None:
+            weights.copy_(weights_fn(t))
+            w_host = weights.cpu().numpy()
         pr.step(g, weights, update)
         upd_cpu = orc.step(np.ascontiguousarray(g.cpu().numpy()), w_host)
+        if (t + 1) % state_every != 0 and t != steps - 1:
+            assert pr.leader == orc.leader, f"step {t}: leader {pr.leader} != {orc.leader}"
+            assert_bits_equal(update.cpu().numpy(), upd_cpu, f"step {t}: update")
+            update.fill_(float("nan"))
+            continue
         look = (t + 1) % residual_every == 0 or t == steps - 1
         compare_state(pr, orc, update, upd_cpu, f"step {t}", check_mask=check_mask, check_residual=look)
         update.fill_(float("nan"))  # the next step must overwrite every element

@@ -224,6 +224,59 @@ def test_residuals_left_alone_between_steps_with_ties_and_fallbacks():
     run_parity(sizes, W, ratio, 1e-8, seed=3, steps=7, weights=weights, grads_fn=grads, residual_every=1000)
 
 
+# ------------------------------------------------------------------ selects left running past the end of a step
+
+
+@pytest.mark.parametrize("state_every", [2, 3, 1000])
+@pytest.mark.parametrize("overlap", [1, 0])
+def test_steps_back_to_back_with_changing_weights(state_every, overlap):
+    # Nobody asks for lists or residuals between most steps, so the other workers' selects of one step
+    # run beside the head of the next; the weights change right after every step (the library must have
+    # kept what a late fallback still needs), and coarse values make some pairs fall back while others
+    # stay on the single-read path.
+    sizes, W, ratio = [70000, 64, 16385, 300000, 40000], 5, 64.0
+    N = sum(sizes)
+
+    def weights_at(t):
+        g = torch.Generator(device=DEV)
+        g.manual_seed(900 + t)
+        return torch.randint(-3, 4, (N,), generator=g, device=DEV).float() * 0.25
+
+    def grads(t):
+        gg = torch.Generator(device=DEV)
+        gg.manual_seed(700 + t)
+        coarse = torch.randint(-4, 5, (W, N), generator=gg, device=DEV).float() / 8.0
+        fine = torch.randn((W, N), generator=gg, device=DEV) * 1e-3
+        if t % 4 == 1:
+            return coarse
+        if t % 4 == 3:  # only two workers coarse: their pairs fall back, the others' do not
+            fine[1] = coarse[1]
+            fine[3] = coarse[3]
+        return fine
+
+    run_parity(sizes, W, ratio, 1e-8, seed=11, steps=9, weights=weights_at(0).clone(), grads_fn=grads,
+               residual_every=1000, state_every=state_every, weights_fn=weights_at, options={"overlap": overlap})
+
+
+@pytest.mark.parametrize("W", [2, 3])
+def test_back_to_back_steps_with_few_workers(W):
+    # W = 2: the leader and the next step's leader may be all there is
+    sizes, ratio = [50000, 20000], 32.0
+    N = sum(sizes)
+    weights = _weights(N, 3)
+    run_parity(sizes, W, ratio, 1e-8, seed=4, steps=8, weights=weights,
+               grads_fn=lambda t: _randn((W, N), 40 + t), residual_every=1000, state_every=1000)
+
+
+def test_back_to_back_steps_with_leader_overrides():
+    # the leader the library foresaw for the next step is not the one it gets
+    sizes, W, ratio = [50000, 20000, 100], 4, 32.0
+    N = sum(sizes)
+    weights = _weights(N, 5)
+    run_parity(sizes, W, ratio, 1e-8, seed=4, steps=8, weights=weights, grads_fn=lambda t: _randn((W, N), 60 + t),
+               leader_overrides=[0, 3, 3, 1, -1, 2, -1, 0], residual_every=1000, state_every=1000)
+
+
 # ------------------------------------------------------------------ momentum on the residual (Eq. 3)
 
 
