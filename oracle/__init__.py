@@ -33,6 +33,13 @@ def lib() -> C.CDLL:
         L.oracle_set_thresholds.argtypes = [vp, vp]
         L.oracle_set_n_leaders.argtypes = [vp, i32]
         L.oracle_set_random_select.argtypes = [vp, i32]
+        L.oracle_set_layerwise.argtypes = [vp, i32, f64, f64, f64]
+        L.oracle_get_layer_thresholds.argtypes = [vp, vp]
+        L.oracle_get_layer_thresholds.restype = i32
+        L.oracle_exact_sum.argtypes = [vp, i64]
+        L.oracle_exact_sum.restype = f64
+        L.oracle_layerwise_threshold.argtypes = [vp, vp, i64, f32, f64, f64, f64, vp]
+        L.oracle_layerwise_threshold.restype = f32
         L.oracle_draw24.argtypes = [u64, u64, u64]
         L.oracle_draw24.restype = C.c_uint32
         L.oracle_leaders.argtypes = [u64, u64, i32, i32, vp]
@@ -93,6 +100,21 @@ def keep_count(n: int, ratio: float) -> int:
 
 def importance_bits(acc: float, w: float, eps: float) -> int:
     return int(lib().oracle_importance_bits(acc, w, eps))
+
+
+def exact_sum(x: np.ndarray) -> float:
+    """Sum of non-negative finite doubles, exact, rounded once to binary64."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    return float(lib().oracle_exact_sum(_p(x), x.size))
+
+
+def layerwise_threshold(acc: np.ndarray, w: np.ndarray, eps: float, alpha: float, beta: float, c: float):
+    """Eq. 4 for one node and layer -> (thr as np.float32, dict of S1, S2, mean, var, v)."""
+    acc = np.ascontiguousarray(acc, dtype=np.float32)
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    st = np.empty(5, dtype=np.float64)
+    thr = lib().oracle_layerwise_threshold(_p(acc), _p(w), acc.size, eps, alpha, beta, c, _p(st))
+    return np.float32(thr), dict(zip(("S1", "S2", "mean", "var", "v"), st.tolist()))
 
 
 def select(acc: np.ndarray, w: np.ndarray, k: int, eps: float) -> np.ndarray:
@@ -165,6 +187,16 @@ class Oracle:
 
     def set_leader_override(self, leader: int):
         lib().oracle_set_leader_override(self._h, leader)
+
+    def set_layerwise(self, alpha: float, beta: float, c: float, on: bool = True):
+        """Section 3.4: per-layer thresholds from each chosen node's own importance statistics."""
+        lib().oracle_set_layerwise(self._h, int(on), alpha, beta, c)
+
+    def layer_thresholds(self) -> np.ndarray:
+        """[chosen node][layer] thresholds the last step derived (layer-wise mode)."""
+        out = np.empty(self.W * self.L, dtype=np.float32)
+        n = lib().oracle_get_layer_thresholds(self._h, _p(out))
+        return out[: n * self.L].reshape(n, self.L).copy()
 
     def reset(self):
         lib().oracle_reset(self._h)

@@ -31,6 +31,12 @@
 //   * Section 3.3's random gradient selection (threshold mode, optional): an element whose importance
 //     does not exceed the threshold is sent iff u < importance / thr, u one 24-bit uniform draw per
 //     element and step, the quotient in fp32.
+//   * Section 3.4's layer-wise threshold (threshold mode, optional; Eq. 4 with its two branches read as
+//     "v > C" and "otherwise"): per chosen node and layer, thr = alpha + beta v if v > C else alpha - beta v,
+//     v = var / mean of the layer's importances on that node.  So that the value does not depend on a
+//     summation order, S1 = sum imp and S2 = sum imp^2 are the EXACT sums, each rounded once to binary64;
+//     then, one binary64 operation at a time, mean = S1 / n, var = S2 / n - mean * mean (population
+//     variance), v = var / mean (0 if mean = 0), thr rounded to binary32, -0 taken as +0.
 //   * the ring all-reduce is a sum in ascending worker order, fp32, without the 1/N
 //     factor (the caller pre-scales gradients as in Eq. 1).
 //
@@ -70,6 +76,9 @@ struct Oracle {
   bool random_select = false;    // Section 3.3: elements below the threshold go with P = importance / thr
   std::vector<int32_t> leaders;  // the chosen nodes of the last step, r_1 first
   std::vector<float> thr;        // per-layer thresholds (threshold mode)
+  bool layerwise = false;        // Section 3.4: thresholds from each chosen node's per-layer statistics
+  double lw_alpha = 0.0, lw_beta = 0.0, lw_c = 0.0;
+  std::vector<float> lw_thr;     // [chosen node][layer] thresholds of the last step (layer-wise mode)
   std::vector<uint32_t> thr_idx; // the chosen node's index set of the last step (threshold mode)
   std::vector<float> thr_val;    // its accumulated values at those indices, before zeroing
   std::vector<float> acc;        // [W][N] residuals
@@ -125,6 +134,90 @@ inline std::vector<int32_t> leaders_of(uint64_t seed, uint64_t t, int32_t W, int
     remaining.erase(remaining.begin() + static_cast<long>(u));
   }
   return out;
+}
+
+// Exact sum of non-negative finite doubles, rounded once (to nearest, ties to even) at the end.
+// The sum is kept as a wide fixed-point number: base-2^32 digits, digit d weighing 2^(32 d - 1074),
+// so that every binary64 value is an integer number of units of the lowest digit.
+struct ExactSum {
+  static constexpr int DIGITS = 72;
+  uint64_t digit[DIGITS] = {};  // each may run ahead of 2^32 until carries are propagated
+  uint32_t pending = 0;
+
+  void carry() {
+    for (int d = 0; d + 1 < DIGITS; ++d) {
+      digit[d + 1] += digit[d] >> 32;
+      digit[d] &= 0xffffffffull;
+    }
+    pending = 0;
+  }
+  void add(double x) {  // x >= 0, finite
+    if (x == 0.0) return;
+    int e;
+    const double f = std::frexp(x, &e);               // x = f 2^e, 0.5 <= f < 1
+    uint64_t m = static_cast<uint64_t>(std::ldexp(f, 53));  // 53-bit integer, x = m 2^(e - 53)
+    int pos = e - 53 + 1074;                          // weight of m's lowest bit, in units of 2^-1074
+    if (pos < 0) {                                    // subnormal: the low bits of m are zero
+      m >>= -pos;
+      pos = 0;
+    }
+    const unsigned __int128 wide = static_cast<unsigned __int128>(m) << (pos % 32);
+    const int d = pos / 32;
+    digit[d] += static_cast<uint64_t>(wide & 0xffffffffull);
+    digit[d + 1] += static_cast<uint64_t>((wide >> 32) & 0xffffffffull);
+    digit[d + 2] += static_cast<uint64_t>(wide >> 64);
+    if (++pending == (1u << 30)) carry();
+  }
+  bool bit(int b) const { return (digit[b / 32] >> (b % 32)) & 1u; }
+  double rounded() {
+    carry();
+    int top = -1;
+    for (int b = DIGITS * 32 - 1; b >= 0; --b)
+      if (bit(b)) {
+        top = b;
+        break;
+      }
+    if (top < 0) return 0.0;
+    const int low = top >= 52 ? top - 52 : 0;  // lowest bit that fits the 53-bit significand
+    uint64_t m = 0;
+    for (int b = top; b >= low; --b) m = (m << 1) | (bit(b) ? 1u : 0u);
+    if (low > 0) {
+      const bool half = bit(low - 1);
+      bool below = false;
+      for (int b = low - 2; b >= 0 && !below; --b) below = bit(b);
+      if (half && (below || (m & 1u))) m += 1;  // may reach 2^53: still exact as a double
+    }
+    return std::ldexp(static_cast<double>(m), low - 1074);
+  }
+};
+
+// Eq. 4 for one node and layer: threshold from the exact first and second moments of the importances.
+inline float layerwise_threshold(const float* acc, const float* weights, int64_t n, float eps, double alpha, double beta,
+                                 double c, double* stats) {
+  ExactSum s1, s2;
+  for (int64_t i = 0; i < n; ++i) {
+    const double imp = static_cast<double>(importance(acc[i], weights[i], eps));
+    s1.add(imp);
+    s2.add(imp * imp);  // exact: 24-bit significands
+  }
+  const double S1 = s1.rounded(), S2 = s2.rounded();
+  const double nn = static_cast<double>(n);
+  const double mean = S1 / nn;
+  const double msq = mean * mean;
+  const double var = S2 / nn - msq;
+  const double v = mean > 0.0 ? var / mean : 0.0;
+  const double bv = beta * v;
+  const double t = v > c ? alpha + bv : alpha - bv;
+  float thr = static_cast<float>(t);
+  if (thr == 0.0f) thr = 0.0f;  // -0 -> +0
+  if (stats) {
+    stats[0] = S1;
+    stats[1] = S2;
+    stats[2] = mean;
+    stats[3] = var;
+    stats[4] = v;
+  }
+  return thr;
 }
 
 // Section 3.3, random gradient selection: the uniform draw of element i at step t, 24 bits
@@ -214,6 +307,34 @@ void oracle_set_thresholds(void* h, const float* thr) {
   Oracle* o = static_cast<Oracle*>(h);
   o->threshold_mode = thr != nullptr;
   if (thr) o->thr.assign(thr, thr + o->n.size());
+}
+// Section 3.4: thresholds from the chosen nodes' own statistics (switches the threshold mode on as well).
+void oracle_set_layerwise(void* h, int32_t on, double alpha, double beta, double c) {
+  Oracle* o = static_cast<Oracle*>(h);
+  o->layerwise = on != 0;
+  o->lw_alpha = alpha;
+  o->lw_beta = beta;
+  o->lw_c = c;
+  if (on) {
+    o->threshold_mode = true;
+    o->thr.assign(o->n.size(), 0.0f);
+  }
+}
+// [chosen node][layer] thresholds the last step derived; returns how many chosen nodes there were
+int32_t oracle_get_layer_thresholds(void* h, float* out) {
+  Oracle* o = static_cast<Oracle*>(h);
+  std::copy(o->lw_thr.begin(), o->lw_thr.end(), out);
+  return static_cast<int32_t>(o->lw_thr.size() / o->n.size());
+}
+// the pieces of Eq. 4 on their own (tests): exact sum of non-negative doubles; one layer's statistics
+double oracle_exact_sum(const double* x, int64_t n) {
+  ExactSum s;
+  for (int64_t i = 0; i < n; ++i) s.add(x[i]);
+  return s.rounded();
+}
+float oracle_layerwise_threshold(const float* acc, const float* weights, int64_t n, float eps, double alpha, double beta,
+                                 double c, double* stats5) {
+  return layerwise_threshold(acc, weights, n, eps, alpha, beta, c, stats5);
 }
 void oracle_set_random_select(void* h, int32_t on) { static_cast<Oracle*>(h)->random_select = on != 0; }
 uint32_t oracle_draw24(uint64_t seed, uint64_t t, uint64_t i) { return draw24(seed, t, i); }
@@ -312,17 +433,29 @@ void oracle_step(void* h, const float* grads, const float* weights, float* updat
     const float* ar = &o->acc[static_cast<size_t>(o->leader) * N];
     o->thr_idx.clear();
     o->thr_val.clear();
+    const int n_chosen = static_cast<int>(o->leaders.size());
+    if (o->layerwise) {  // Section 3.4: every chosen node derives its own per-layer thresholds
+      o->lw_thr.assign(static_cast<size_t>(n_chosen) * L, 0.0f);
+#pragma omp parallel for num_threads(nthreads) schedule(dynamic, 1)
+      for (int q = 0; q < n_chosen * L; ++q) {
+        const int j = q / L, l = q % L;
+        o->lw_thr[q] = layerwise_threshold(&o->acc[static_cast<size_t>(o->leaders[j]) * N + o->off[l]], weights + o->off[l],
+                                           o->n[l], o->eps, o->lw_alpha, o->lw_beta, o->lw_c, nullptr);
+      }
+    }
     for (int l = 0; l < L; ++l) {
       for (int64_t i = o->off[l]; i < o->off[l] + o->n[l]; ++i) {
         bool in_mask = false;
-        for (int32_t r : o->leaders) {
+        for (int j = 0; j < n_chosen; ++j) {
+          const int32_t r = o->leaders[j];
+          const float thr_l = o->layerwise ? o->lw_thr[static_cast<size_t>(j) * L + l] : o->thr[l];
           const float imp = importance(o->acc[static_cast<size_t>(r) * N + i], weights[i], o->eps);
-          bool sel = imp > o->thr[l];
+          bool sel = imp > thr_l;
           if (!sel && o->random_select) {
             // P(update) = importance / threshold: one draw per element and step, compared in fp32
             const float u = static_cast<float>(draw24(o->seed, static_cast<uint64_t>(o->t), static_cast<uint64_t>(i))) *
                             5.9604644775390625e-08f;  // 2^-24
-            sel = u < imp / o->thr[l];
+            sel = u < imp / thr_l;
           }
           in_mask = in_mask || sel;
         }

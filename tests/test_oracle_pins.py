@@ -621,3 +621,121 @@ def test_random_select_equals_bruteforce_and_has_the_right_rate():
     off.step(g, weights)
     assert off.threshold_list()[0].tolist() == list(range(10, 20))
     assert np.count_nonzero(upd) >= len(S) - 10
+
+
+# ---------------------------------------------------------------- layer-wise threshold (Section 3.4, Eq. 4)
+
+
+def _frac_round(values):
+    """Exact sum by rational arithmetic, rounded once (Fraction -> float is correctly rounded)."""
+    from fractions import Fraction
+
+    return float(sum((Fraction(float(v)) for v in values), Fraction(0)))
+
+
+def _eq4_by_fractions(acc, w, eps, alpha, beta, c):
+    """Eq. 4 written out independently: exact moments by rational arithmetic, the rest in Python floats."""
+    imp = [float(importance(a, b, eps)) for a, b in zip(acc, w)]
+    S1, S2 = _frac_round(imp), _frac_round([x * x for x in imp])  # x * x is exact in binary64 for fp32 x
+    n = float(len(imp))
+    mean = S1 / n
+    var = S2 / n - mean * mean
+    v = var / mean if mean > 0.0 else 0.0
+    t = alpha + beta * v if v > c else alpha - beta * v
+    thr = F(t)
+    return (F(0.0) if thr == 0 else thr), dict(S1=S1, S2=S2, mean=mean, var=var, v=v)
+
+
+def test_exact_sum_equals_fsum_and_fractions():
+    rng = np.random.default_rng(5)
+    for n in (1, 2, 17, 1000, 100000):
+        x = np.abs(rng.standard_normal(n)) * 10.0 ** rng.integers(-40, 40, n)  # 80 decades of magnitude
+        assert oracle.exact_sum(x) == math.fsum(x.tolist())
+    small = np.abs(rng.standard_normal(200)) * 10.0 ** rng.integers(-300, 10, 200)
+    small[:5] = [5e-324, 1e-310, 2.2250738585072014e-308, 0.0, 4.9e-324]  # subnormals, the smallest normal, zero
+    assert oracle.exact_sum(small) == math.fsum(small.tolist()) == _frac_round(small)
+    assert oracle.exact_sum(np.zeros(3)) == 0.0 and oracle.exact_sum(np.zeros(0)) == 0.0
+    # ties go to even, and anything beyond a tie rounds up
+    assert oracle.exact_sum(np.array([2.0**53, 1.0])) == 2.0**53
+    assert oracle.exact_sum(np.array([2.0**53, 1.0, 5e-324])) == 2.0**53 + 2
+    assert oracle.exact_sum(np.array([2.0**53 + 2, 1.0])) == 2.0**53 + 4
+    assert oracle.exact_sum(np.array([1.0, 2.0**-53])) == 1.0 and oracle.exact_sum(np.array([1.0, 2.0**-53, 2.0**-53])) == 1.0 + 2.0**-52
+    # a plain left-to-right sum gets this one wrong: 1e16 + 1 + 1 + ... (1000 ones)
+    x = np.array([1e16] + [1.0] * 1000)
+    assert oracle.exact_sum(x) == 1e16 + 1000 and float(np.cumsum(x)[-1]) != 1e16 + 1000
+
+
+def test_layerwise_threshold_closed_forms():
+    eps = F(2.0**-30)
+    w = np.full(1024, 1.0, np.float32)  # |w| + eps rounds back to 1, so importance = |acc|
+    # a constant layer has no variance: thr = alpha
+    thr, st = oracle.layerwise_threshold(np.full(1024, -0.25, np.float32), w, eps, 0.05, 3.0, 0.5)
+    assert (st["S1"], st["S2"], st["mean"], st["var"], st["v"]) == (256.0, 64.0, 0.25, 0.0, 0.0) and thr == F(0.05)
+    # half 1, half 3: mean 2, var 1, v = 0.5
+    acc = np.where(np.arange(1024) % 2 == 0, 1.0, -3.0).astype(np.float32)
+    thr, st = oracle.layerwise_threshold(acc, w, eps, 0.25, 0.5, 0.25)
+    assert (st["mean"], st["var"], st["v"]) == (2.0, 1.0, 0.5) and thr == F(0.5)  # v > C: alpha + beta v
+    thr, _ = oracle.layerwise_threshold(acc, w, eps, 0.25, 0.5, 0.5)
+    assert thr == F(0.0)  # v == C is not "greater": alpha - beta v = 0
+    thr, _ = oracle.layerwise_threshold(acc, w, eps, 0.25, 1.0, 1.0)
+    assert thr == F(-0.25)  # a negative threshold is kept as it is
+    # nothing accumulated: mean 0, v taken as 0
+    thr, st = oracle.layerwise_threshold(np.zeros(64, np.float32), w[:64], eps, 0.125, 9.0, 0.0)
+    assert st["mean"] == 0.0 and st["v"] == 0.0 and thr == F(0.125)
+    # -0 becomes +0
+    thr, _ = oracle.layerwise_threshold(np.zeros(64, np.float32), w[:64], eps, -0.0, 1.0, 0.0)
+    assert u32([thr])[0] == 0
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_layerwise_threshold_equals_rational_arithmetic(seed):
+    rng = np.random.default_rng(100 + seed)
+    n = [257, 1000, 4096][seed]
+    acc = (rng.standard_normal(n) * 10.0 ** rng.integers(-6, 3, n)).astype(np.float32)
+    w = (rng.standard_normal(n) * 0.05).astype(np.float32)
+    w[rng.random(n) < 0.05] = 0.0  # importances of 1e8 and more beside ones of 1e-6
+    for alpha, beta, c in ((0.01, 1e-9, 1e6), (0.05, 0.001, 1e30), (0.0, 1.0, 0.0)):
+        thr, st = oracle.layerwise_threshold(acc, w, F(1e-8), alpha, beta, c)
+        thr_f, st_f = _eq4_by_fractions(acc, w, F(1e-8), alpha, beta, c)
+        assert st == st_f and u32([thr])[0] == u32([thr_f])[0]
+
+
+def test_layerwise_step_equals_bruteforce_with_two_chosen_nodes():
+    layers, W = [40, 9, 64], 4
+    N, eps = sum(layers), F(1e-8)
+    rng = np.random.default_rng(77)
+    weights = (rng.standard_normal(N) * 0.1).astype(np.float32)
+    alpha, beta, c = 0.5, 0.02, 10.0
+    orc = oracle.Oracle(layers, W, 2.0, eps, seed=9)
+    orc.set_layerwise(alpha, beta, c)
+    orc.set_n_leaders(2)
+    acc = np.zeros((W, N), np.float32)
+    saw_both_branches = set()
+    for t in range(6):
+        grads = (rng.standard_normal((W, N)) * (0.2 if t % 2 else 0.02)).astype(np.float32)
+        upd = orc.step(grads, weights)
+        acc = (acc + grads).astype(np.float32)
+        chosen = oracle.leaders(9, t, W, 2)
+        thr = orc.layer_thresholds()
+        assert thr.shape == (2, len(layers))
+        S, o = set(), 0
+        for l, n in enumerate(layers):
+            for j, r in enumerate(chosen):
+                want, st = _eq4_by_fractions(acc[r, o:o + n], weights[o:o + n], eps, alpha, beta, c)
+                saw_both_branches.add(st["v"] > c)
+                assert u32([thr[j, l]])[0] == u32([want])[0]
+                S |= {o + i for i in range(n) if importance(acc[r, o + i], weights[o + i], eps) > want}
+            o += n
+        idx, val = orc.threshold_list()
+        assert idx.tolist() == sorted(S)
+        want_upd = np.zeros(N, np.float32)
+        for i in S:
+            s = acc[0, i]
+            for w_ in range(1, W):
+                s = F(s + acc[w_, i])
+            want_upd[i] = F(F(0) + s)
+            acc[:, i] = 0
+        assert np.array_equal(u32(upd), u32(want_upd))
+        for w_ in range(W):
+            assert np.array_equal(u32(orc.residual(w_)), u32(acc[w_]))
+    assert saw_both_branches == {True, False}
