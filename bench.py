@@ -213,6 +213,8 @@ def run_ours(args):
         thr = [0.4 if (c.tensors is None or tn.kind == "weight") else 2.0e4
                for tn in (c.tensors or [None] * len(c.layer_sizes))]
         pr = Pruner(c.layer_sizes, W, None, c.eps, c.seed, thresholds=thr)
+        if args.layerwise:  # Section 3.4: thresholds from the chosen node's per-layer var/mean (Eq. 4)
+            pr.set_layerwise(*(float(x) for x in args.layerwise.split(",")))
     else:
         pr = Pruner(c.layer_sizes, W, c.ratio, c.eps, c.seed)
     K = pr.K
@@ -343,7 +345,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
-        "config": {"workload": c.name, "mode": args.mode, "W": W, "N": N, "K": K,
+        "config": {"workload": c.name, "mode": args.mode + ("+layerwise" if args.layerwise else ""), "W": W, "N": N, "K": K,
                    "ratio": c.ratio if args.mode == "ratio" else None, "layers": len(c.layer_sizes),
                    "l2_policy": f"inputs larger than L2: {grad_bytes * 3 / 1e9:.2f} GB streamed per step, "
                                 f"{n_sets} gradient batches cycled",
@@ -379,6 +381,8 @@ def main():
     ap.add_argument("--mode", default="ratio", choices=["ratio", "threshold"],
                     help="ratio: exact layer-wise top-k at the configured compression (headline); threshold: "
                          "absolute per-layer thresholds on the chosen node (Algorithm 1 as printed)")
+    ap.add_argument("--layerwise", default=None,
+                    help="alpha,beta,C - with --mode threshold: layer-wise thresholds alpha +/- beta var/mean (Eq. 4)")
     ap.add_argument("--layers", default=None, help="lo:hi - only these layers of the workload (small profiling case)")
     ap.add_argument("--grad-sets", type=int, default=None, help="distinct gradient batches kept on the device")
     ap.add_argument("--no-e2e", action="store_true")

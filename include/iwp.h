@@ -113,6 +113,22 @@ int iwp_create_threshold(iwp_ctx** out, const int64_t* layer_sizes_host, int32_t
  * the stream.  Errors: IWP_ERR_INVALID (NULL, not a threshold-mode context, negative or NaN value). */
 int iwp_set_thresholds(iwp_ctx* ctx, const float* thr_host);
 
+/* Section 3.4, layer-wise threshold (Eq. 4; its two printed branches carry the same condition and are
+ * read as "v > C" and "otherwise"): with on = 1 every following step of a threshold-mode context derives,
+ * for each chosen node and layer, thr = alpha + beta * v if v > c_split else alpha - beta * v, where
+ * v = var / mean of the layer's importances on that node, and uses it in place of the fixed thresholds
+ * (iwp_set_thresholds() is then not needed).  So that the value depends on no summation order,
+ * S1 = sum imp and S2 = sum imp^2 are exact sums rounded once to binary64; then, one binary64 operation
+ * at a time, mean = S1 / n, var = S2 / n - mean * mean, v = var / mean (0 when mean is 0); thr is rounded
+ * to binary32, -0 taken as +0; a negative thr selects the whole layer.  on = 0 returns to the fixed
+ * thresholds.  Errors: IWP_ERR_INVALID (NULL, not a threshold-mode context, non-finite parameter). */
+int iwp_set_layerwise(iwp_ctx* ctx, int32_t on, double alpha, double beta, double c_split);
+
+/* The thresholds the last layer-wise step derived: n_chosen rows (r_1 first) of one float per layer to
+ * dst_dev (room for 8 rows), the number of rows to *n_chosen_host (0 before the first such step).
+ * Asynchronous on the context's stream.  IWP_ERR_INVALID unless iwp_set_layerwise() is on. */
+int iwp_get_layer_thresholds(iwp_ctx* ctx, float* dst_dev, int32_t* n_chosen_host);
+
 /* Number of entries of the last step's index set (threshold mode: synchronises the stream and reads
  * it from the device; ratio mode: K). */
 int iwp_get_list_length(iwp_ctx* ctx, int64_t* len_host);

@@ -22,6 +22,7 @@ EXPORTS = [
     "iwp_get_step", "iwp_set_step", "iwp_get_leader", "iwp_get_residual", "iwp_set_residual",
     "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat", "iwp_select_static",
     "iwp_set_momentum", "iwp_create_threshold", "iwp_set_thresholds", "iwp_get_list_length", "iwp_leaders_at",
+    "iwp_set_layerwise", "iwp_get_layer_thresholds",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -52,6 +53,8 @@ def lib() -> C.CDLL:
         L.iwp_create_threshold.argtypes = [C.POINTER(vp), vp, i32, i32, f32, u64, i64]
         L.iwp_set_thresholds.argtypes = [vp, vp]
         L.iwp_get_list_length.argtypes = [vp, vp]
+        L.iwp_set_layerwise.argtypes = [vp, i32, f64, f64, f64]
+        L.iwp_get_layer_thresholds.argtypes = [vp, vp, vp]
         L.iwp_destroy.argtypes = [vp]
         L.iwp_set_stream.argtypes = [vp, vp]
         L.iwp_set_momentum.argtypes = [vp, f32]
@@ -213,6 +216,17 @@ class Pruner:
     def set_thresholds(self, thr: Sequence[float]) -> None:
         arr = (C.c_float * self.L)(*[float(x) for x in thr])
         _check(lib().iwp_set_thresholds(self._h, arr), "iwp_set_thresholds")
+
+    def set_layerwise(self, alpha: float, beta: float, c: float, on: bool = True) -> None:
+        """Section 3.4: per-layer thresholds alpha +/- beta * var/mean from each chosen node's importances."""
+        _check(lib().iwp_set_layerwise(self._h, int(on), float(alpha), float(beta), float(c)), "iwp_set_layerwise")
+
+    def layer_thresholds(self):
+        """[chosen node][layer] thresholds of the last layer-wise step (a CUDA float tensor)."""
+        out = self._torch.empty((8, self.L), dtype=self._torch.float32, device=self.device)
+        n = C.c_int32()
+        _check(lib().iwp_get_layer_thresholds(self._h, out.data_ptr(), C.byref(n)), "iwp_get_layer_thresholds")
+        return out[: int(n.value)]
 
     def list_length(self) -> int:
         v = C.c_int64()

@@ -67,6 +67,11 @@ struct iwp_ctx {
   int32_t n_leaders = 1;          // chosen nodes whose masks are OR-ed
   bool random_select = false;     // Section 3.3: P(update) = importance / threshold below the threshold
   uint32_t* d_thr = nullptr;      // [layer] fp32 patterns of the thresholds
+  bool layerwise = false;         // Section 3.4: thresholds from each chosen node's per-layer statistics (Eq. 4)
+  double lw_alpha = 0.0, lw_beta = 0.0, lw_c = 0.0;
+  int32_t lw_chosen = 0;          // chosen nodes of the last layer-wise step
+  uint32_t* d_thr_lw = nullptr;   // [chosen node][layer] fp32 patterns of the derived thresholds
+  unsigned long long* d_bins = nullptr;  // [chosen node][layer][3][256] exact moment sums in the making
   uint32_t* d_tcnt = nullptr;     // [chunk] selected elements of the chunk
   uint32_t* d_toff = nullptr;     // [chunk] list offset of the chunk
   uint32_t* d_list_len = nullptr; // length of the last step's index list
@@ -227,6 +232,8 @@ void free_all(iwp_ctx* c) {
   cudaFree(c->lead_tot);
   cudaFree(c->zmask);
   cudaFree(c->d_thr);
+  cudaFree(c->d_thr_lw);
+  cudaFree(c->d_bins);
   cudaFree(c->d_tcnt);
   cudaFree(c->d_toff);
   cudaFree(c->d_list_len);
@@ -602,8 +609,10 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
     return IWP_ERR_CUDA;
   }
   const Sizes sz = sizes_of(p, threshold_mode, c->list_cap);
+  const uint64_t lw_thr_bytes = MAX_LEADERS * p.layers.size() * sizeof(uint32_t);
+  const uint64_t lw_bin_bytes = MAX_LEADERS * p.layers.size() * 3 * LW_BINS * sizeof(unsigned long long);
   const uint64_t thr_bytes = threshold_mode
-                                 ? (p.layers.size() + 2 * p.chunks.size() + 1) * sizeof(uint32_t)
+                                 ? (p.layers.size() + 2 * p.chunks.size() + 1) * sizeof(uint32_t) + lw_thr_bytes + lw_bin_bytes
                                  : 0;
   c->device_bytes = sz.total() + thr_bytes;
   int rc = IWP_OK;
@@ -640,6 +649,8 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
     A(&c->d_tcnt, at_least(p.chunks.size() * sizeof(uint32_t)));
     A(&c->d_toff, at_least(p.chunks.size() * sizeof(uint32_t)));
     A(&c->d_list_len, sizeof(uint32_t));
+    A(&c->d_thr_lw, lw_thr_bytes);
+    A(&c->d_bins, lw_bin_bytes);
   }
   if (rc != IWP_OK) {
     free_all(c);
@@ -647,7 +658,11 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
     return rc;
   }
   bool ok = true;
-  if (threshold_mode) ok = cudaMemset(c->d_list_len, 0, sizeof(uint32_t)) == cudaSuccess;
+  if (threshold_mode) {
+    ok = cudaMemset(c->d_list_len, 0, sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && cudaMemset(c->d_thr_lw, 0, lw_thr_bytes) == cudaSuccess;
+    ok = ok && cudaMemset(c->d_bins, 0, lw_bin_bytes) == cudaSuccess;  // k_thr_finalize leaves them cleared
+  }
   auto H2D = [&](void* dst, const void* src, size_t bytes) {
     if (bytes) ok = ok && cudaMemcpy(dst, src, bytes, cudaMemcpyHostToDevice) == cudaSuccess;
   };
@@ -746,12 +761,26 @@ int run_step_threshold(iwp_ctx* c, const float* grads, const float* weights, flo
   k_thr_accumulate_chosen<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, c->d_tiles, N, c->momentum, ls);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 3);
-  k_thr_count<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_thr, c->d_tcnt, c->eps, N, ls, rs);
+  const uint32_t n_layers = static_cast<uint32_t>(p.layers.size());
+  const uint32_t* thr = c->d_thr;
+  uint32_t thr_stride = 0;
+  if (c->layerwise) {  // Eq. 4: every chosen node's thresholds from its own exact moments
+    k_thr_stats<VEC><<<dim3(n_chunks, static_cast<unsigned>(ls.n)), THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_bins,
+                                                                                  c->eps, N, n_layers, ls);
+    IWP_LAUNCH_CHECK(c);
+    k_thr_finalize<<<dim3(n_layers, static_cast<unsigned>(ls.n)), THREADS, 0, s>>>(c->d_bins, c->d_layers, c->d_thr_lw, n_layers,
+                                                                                c->lw_alpha, c->lw_beta, c->lw_c);
+    IWP_LAUNCH_CHECK(c);
+    thr = c->d_thr_lw;
+    thr_stride = n_layers;
+    c->lw_chosen = ls.n;
+  }
+  k_thr_count<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, thr, thr_stride, c->d_tcnt, c->eps, N, ls, rs);
   IWP_LAUNCH_CHECK(c);
   k_thr_scan<<<1, 1024, 0, s>>>(c->d_tcnt, c->d_toff, n_chunks, c->d_list_len);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 4);
-  k_thr_write<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_thr, c->d_toff, c->sel_idx,
+  k_thr_write<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, thr, thr_stride, c->d_toff, c->sel_idx,
                                                 c->sel_val, cap, c->d_status, c->zmask, c->eps, N, ls, rs);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 5);
@@ -781,6 +810,7 @@ int iwp_set_thresholds(iwp_ctx* c, const float* thr) {
   for (size_t l = 0; l < bits.size(); ++l) {
     if (!(thr[l] >= 0.0f)) return IWP_ERR_INVALID;  // negative or NaN
     std::memcpy(&bits[l], &thr[l], sizeof(uint32_t));
+    if (thr[l] == 0.0f) bits[l] = 0u;  // -0 is +0
   }
   // synchronous copy from a temporary: ordered after everything already enqueued on the stream
   if (cudaStreamSynchronize(c->stream) != cudaSuccess ||
@@ -789,6 +819,30 @@ int iwp_set_thresholds(iwp_ctx* c, const float* thr) {
     return IWP_ERR_CUDA;
   }
   c->thr_set = true;
+  return IWP_OK;
+}
+
+int iwp_set_layerwise(iwp_ctx* c, int32_t on, double alpha, double beta, double c_split) {
+  if (!c || !c->threshold_mode || (on != 0 && on != 1)) return IWP_ERR_INVALID;
+  if (on && (!std::isfinite(alpha) || !std::isfinite(beta) || !std::isfinite(c_split))) return IWP_ERR_INVALID;
+  c->layerwise = on != 0;
+  if (on) {
+    c->lw_alpha = alpha;
+    c->lw_beta = beta;
+    c->lw_c = c_split;
+  }
+  return IWP_OK;
+}
+
+int iwp_get_layer_thresholds(iwp_ctx* c, float* dst, int32_t* n_chosen) {
+  if (!c || !dst || !n_chosen || !c->threshold_mode || !c->layerwise) return IWP_ERR_INVALID;
+  *n_chosen = c->lw_chosen;
+  if (c->lw_chosen == 0) return IWP_OK;
+  if (cudaMemcpyAsync(dst, c->d_thr_lw, static_cast<size_t>(c->lw_chosen) * c->plan.layers.size() * sizeof(uint32_t),
+                      cudaMemcpyDeviceToDevice, c->stream) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
   return IWP_OK;
 }
 
@@ -841,7 +895,7 @@ int iwp_step(iwp_ctx* c, const float* grads, const float* weights, float* update
                                                  : leader_at(c->seed, static_cast<uint64_t>(c->t), c->plan.W);
   const bool vec = !c->force_scalar && (c->plan.N % 4 == 0) && aligned16(grads) && aligned16(weights) &&
                    aligned16(update) && aligned16(c->acc);
-  if (c->threshold_mode && !c->thr_set) return IWP_ERR_INVALID;  // no thresholds given yet
+  if (c->threshold_mode && !c->thr_set && !c->layerwise) return IWP_ERR_INVALID;  // no thresholds given yet
   const int rc = c->threshold_mode
                      ? (vec ? run_step_threshold<true>(c, grads, weights, update, leader)
                             : run_step_threshold<false>(c, grads, weights, update, leader))

@@ -21,11 +21,16 @@ def _randn(shape, seed, scale=1.0):
 
 
 def _run(sizes, W, thr, weights, grads_fn, steps, seed=3, momentum=None, max_list=0, force_scalar=False,
-         residual_every=1, n_leaders=1, random_select=False):
+         residual_every=1, n_leaders=1, random_select=False, layerwise=None):
+    """thr: fixed per-layer thresholds, or None with layerwise = (alpha, beta, C) of Eq. 4."""
     N = sum(sizes)
     pr = Pruner(sizes, W, None, 1e-8, seed, thresholds=thr, max_list=max_list)
     orc = oracle.Oracle(sizes, W, 2.0, 1e-8, seed)
-    orc.set_thresholds(thr)
+    if layerwise is not None:
+        pr.set_layerwise(*layerwise)
+        orc.set_layerwise(*layerwise)
+    else:
+        orc.set_thresholds(thr)
     if momentum is not None:
         pr.set_momentum(momentum)
         orc.set_momentum(momentum)
@@ -39,11 +44,15 @@ def _run(sizes, W, thr, weights, grads_fn, steps, seed=3, momentum=None, max_lis
         orc.set_n_leaders(n_leaders)
     w_host = weights.cpu().numpy()
     upd = torch.full((N,), float("nan"), device=DEV)
+    seen_thr = []
     for t in range(steps):
         g = grads_fn(t)
         pr.step(g, weights, upd)
         want = orc.step(np.ascontiguousarray(g.cpu().numpy()), w_host)
         assert pr.sync_status() == 0 and pr.leader == orc.leader
+        if layerwise is not None:  # the derived thresholds themselves, bit for bit, one row per chosen node
+            assert_bits_equal(pr.layer_thresholds().cpu().numpy(), orc.layer_thresholds(), f"step {t}: thresholds")
+            seen_thr.append(orc.layer_thresholds())
         oi, ov = orc.threshold_list()
         assert pr.list_length() == len(oi), f"step {t}: list length"
         gi, gv = pr.selection(pr.leader)
@@ -57,6 +66,7 @@ def _run(sizes, W, thr, weights, grads_fn, steps, seed=3, momentum=None, max_lis
         upd.fill_(float("nan"))
     pr.close()
     orc.close()
+    return seen_thr
 
 
 CASES = {
@@ -178,3 +188,80 @@ def test_random_select_with_zero_and_infinite_thresholds():
     g.manual_seed(3)
     grads = lambda t: torch.randint(-2, 3, (W, N), generator=g, device=DEV).float()  # many exact zeros
     _run(sizes, W, [0.0, float("inf")], weights, grads, steps=3, random_select=True)
+
+
+# ------------------------------------------------------------------ layer-wise threshold (Section 3.4, Eq. 4)
+
+
+@pytest.mark.parametrize("name", sorted(CASES))
+def test_layerwise_threshold_random_values(name):
+    sizes, W = CASES[name]
+    N = sum(sizes)
+    weights = _randn((N,), 100, 0.05)
+    weights[::97] = 0.0  # importances of 1e6 and more beside ordinary ones: many exponents in one sum
+    # C in the middle of the values var/mean takes here, so that both branches of Eq. 4 occur
+    _run(sizes, W, None, weights, lambda t: _randn((W, N), 300 + t, 0.01 * (1 + 3 * (t % 2))), steps=4,
+         layerwise=(0.3, 1e-9, 3e7), residual_every=2)
+
+
+@pytest.mark.parametrize("n_leaders", [2, 3])
+def test_layerwise_threshold_several_chosen_nodes_and_random_selection(n_leaders):
+    sizes, W = [64, 16385, 256, 100000, 9408, 1, 36864], 4
+    N = sum(sizes)
+    weights = _randn((N,), 101, 0.05)
+    _run(sizes, W, None, weights, lambda t: _randn((W, N), 400 + t, 0.02), steps=4, n_leaders=n_leaders,
+         layerwise=(0.5, 0.01, 5.0), random_select=(n_leaders == 3), momentum=0.9)
+    # each branch of Eq. 4 on its own: C below every var/mean, then above every one
+    up = _run(sizes, W, None, weights, lambda t: _randn((W, N), 400 + t, 0.02), steps=2, n_leaders=n_leaders,
+              layerwise=(0.5, 1e-6, -1.0))
+    down = _run(sizes, W, None, weights, lambda t: _randn((W, N), 400 + t, 0.02), steps=2, n_leaders=n_leaders,
+                layerwise=(0.5, 1e-6, 1e300))
+    multi = [l for l, n in enumerate(sizes) if n > 1]  # a one-element layer has no variance
+    assert all((thr[:, multi] > 0.5).all() for thr in up) and all((thr[:, multi] < 0.5).all() for thr in down)
+
+
+def test_layerwise_threshold_degenerate_layers():
+    # all-zero gradients (mean 0), a constant layer (variance 0), denormal importances, a negative
+    # threshold (everything goes) and a threshold no importance reaches
+    sizes, W = [4096, 20000, 5000, 70000], 3
+    N = sum(sizes)
+    weights = torch.ones(N, device=DEV)
+    weights[4096 + 20000:4096 + 25000] = 1e30  # importances far below 1e-38 in the third layer
+
+    def grads(t):
+        g = _randn((W, N), 500 + t, 0.25)
+        g[:, :4096] = 0.0
+        g[:, 4096:24096] = 0.5 if t % 2 == 0 else -0.5
+        return g
+
+    _run(sizes, W, None, weights, grads, steps=3, layerwise=(0.2, 1.0, 0.1))
+    _run(sizes, W, None, weights, grads, steps=2, layerwise=(-1.0, 0.0, 0.0))
+    _run(sizes, W, None, weights, grads, steps=2, layerwise=(1e30, 0.0, 0.0))
+
+
+def test_layerwise_argument_checks():
+    pr = Pruner([5000, 300], 2, None, 1e-8, 0)
+    for bad in ((float("nan"), 1.0, 1.0), (0.1, float("inf"), 1.0), (0.1, 1.0, float("nan"))):
+        with pytest.raises(binding.IwpError):
+            pr.set_layerwise(*bad)
+    with pytest.raises(binding.IwpError):
+        pr.layer_thresholds()  # not switched on
+    pr.set_layerwise(0.1, 1.0, 1.0)
+    assert pr.layer_thresholds().shape[0] == 0  # no step yet
+    pr.set_layerwise(0.0, 0.0, 0.0, on=False)
+    g = torch.zeros((2, 5300), device=DEV)
+    with pytest.raises(binding.IwpError):
+        pr.step(g, torch.ones(5300, device=DEV))  # back on fixed thresholds, and none were given
+    pr.close()
+    ratio_ctx = Pruner([5000], 2, 4.0, 1e-8, 0)
+    with pytest.raises(binding.IwpError):
+        ratio_ctx.set_layerwise(0.1, 1.0, 1.0)
+    ratio_ctx.close()
+
+
+def test_layerwise_threshold_full_size_alexnet_shape():
+    c = wl.alexnet_w8()
+    weights = c.weights(DEV)
+    buf = torch.empty((c.W, c.N), dtype=torch.float32, device=DEV)
+    _run(c.layer_sizes, c.W, None, weights, lambda t: c.grads(t, DEV, out=buf), steps=2, seed=c.seed,
+         layerwise=(0.05, 1e-4, 100.0), residual_every=2)
