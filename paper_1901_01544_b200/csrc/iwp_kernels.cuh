@@ -327,7 +327,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS)
     return;
   }
   const uint32_t groups = s >> 3;
-  const uint32_t stride = L.n / groups;  // >= 32 because s <= n / 4
+  const uint32_t stride = L.n / groups;  // >= 128 because s <= n / 16
   const float* a = acc + static_cast<uint64_t>(w) * N + L.off;
   const float* g = grads + static_cast<uint64_t>(w) * N + L.off;
   const float* wt = weights + L.off;

@@ -77,7 +77,7 @@ inline void sample_plan(uint32_t n, uint32_t k, uint32_t* sample, uint32_t* rho)
   *sample = 0;
   *rho = 0;
   if (k >= n) return;
-  uint32_t s = (n / 4) & ~7u;
+  uint32_t s = (n / 16) & ~7u;
   if (s > SAMPLE_MAX) s = SAMPLE_MAX;
   if (s < 64) return;
   const double p = static_cast<double>(k) / static_cast<double>(n);
