@@ -33,6 +33,9 @@ def lib() -> C.CDLL:
         L.oracle_set_thresholds.argtypes = [vp, vp]
         L.oracle_set_n_leaders.argtypes = [vp, i32]
         L.oracle_set_random_select.argtypes = [vp, i32]
+        L.oracle_union_length.argtypes = [vp]
+        L.oracle_union_length.restype = i64
+        L.oracle_get_union.argtypes = [vp, vp]
         L.oracle_set_layerwise.argtypes = [vp, i32, f64, f64, f64]
         L.oracle_get_layer_thresholds.argtypes = [vp, vp]
         L.oracle_get_layer_thresholds.restype = i32
@@ -187,6 +190,12 @@ class Oracle:
 
     def set_leader_override(self, leader: int):
         lib().oracle_set_leader_override(self._h, leader)
+
+    def index_set(self) -> np.ndarray:
+        """Ratio mode: the index set of the last step (union of the chosen nodes' lists), ascending."""
+        out = np.empty(int(lib().oracle_union_length(self._h)), dtype=np.uint32)
+        lib().oracle_get_union(self._h, _p(out))
+        return out
 
     def set_layerwise(self, alpha: float, beta: float, c: float, on: bool = True):
         """Section 3.4: per-layer thresholds from each chosen node's own importance statistics."""

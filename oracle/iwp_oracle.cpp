@@ -22,7 +22,8 @@
 //   * the threshold of Algorithm 1 is the k-th largest importance of the worker's
 //     layer, k = ceil(n / ratio) clamped to [1, n]; ties keep the lower index.
 //   * one randomly chosen node per step supplies the index set (Section 3.2:
-//     "randomly choose a node and broadcast its important gradient index").
+//     "randomly choose a node and broadcast its important gradient index"); optionally several chosen
+//     nodes r_1..r_n, drawn without replacement, whose index sets are OR-ed (Algorithm 1: Mask = OR Mask_ri).
 //   * Eq. 3's momentum acts on the locally kept residual: G <- m * G + grad (two roundings);
 //     m = 1, the default, is the plain accumulation of Section 3.2.
 //   * threshold mode is Algorithm 1 as printed: only the chosen node forms a mask, per layer
@@ -48,6 +49,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <iterator>
 #include <numeric>
 #include <vector>
 #ifdef _OPENMP
@@ -72,7 +74,8 @@ struct Oracle {
   int threads = 0;
   float momentum = 1.0f;         // Eq. 3: the local residual enters the next step scaled by m
   bool threshold_mode = false;   // Algorithm 1 as printed: Mask <- importance > thr on the chosen node
-  int32_t n_leaders = 1;         // threshold mode: how many chosen nodes' masks are OR-ed
+  int32_t n_leaders = 1;         // how many chosen nodes' masks (index sets) are OR-ed
+  std::vector<uint32_t> union_idx; // ratio mode: the index set of the last step, ascending (one node: its list)
   bool random_select = false;    // Section 3.3: elements below the threshold go with P = importance / thr
   std::vector<int32_t> leaders;  // the chosen nodes of the last step, r_1 first
   std::vector<float> thr;        // per-layer thresholds (threshold mode)
@@ -396,8 +399,14 @@ void oracle_get_mask(void* h, uint8_t* dst) {
     for (uint32_t i : o->thr_idx) dst[i] = 1;
     return;
   }
-  const uint32_t* S = &o->sel_idx[static_cast<size_t>(o->leader) * o->K];
-  for (int64_t j = 0; j < o->K; ++j) dst[S[j]] = 1;
+  for (uint32_t i : o->union_idx) dst[i] = 1;
+}
+
+// ratio mode: the index set of the last step (the union of the chosen nodes' lists), ascending
+int64_t oracle_union_length(void* h) { return static_cast<int64_t>(static_cast<Oracle*>(h)->union_idx.size()); }
+void oracle_get_union(void* h, uint32_t* idx) {
+  Oracle* o = static_cast<Oracle*>(h);
+  std::copy(o->union_idx.begin(), o->union_idx.end(), idx);
 }
 
 // One step.  grads[W][N], weights[N], update[N]: host pointers.
@@ -498,14 +507,28 @@ void oracle_step(void* h, const float* grads, const float* weights, float* updat
     }
   }
 
-  // (e) the randomly chosen node supplies the index set
-  const uint32_t* S = &o->sel_idx[static_cast<size_t>(o->leader) * K];
+  // (e) the randomly chosen node supplies the index set; with several chosen nodes (Algorithm 1:
+  // Mask = OR Mask_{r_i}) it is the union of their lists, ascending, each index once
+  if (o->leader_override >= 0 || o->n_leaders == 1) {
+    o->leaders.assign(1, o->leader);
+  } else {
+    o->leaders = leaders_of(o->seed, static_cast<uint64_t>(o->t), W, o->n_leaders);
+  }
+  o->union_idx.clear();
+  for (int32_t r : o->leaders) {
+    const uint32_t* list = &o->sel_idx[static_cast<size_t>(r) * K];
+    std::vector<uint32_t> merged;
+    std::set_union(o->union_idx.begin(), o->union_idx.end(), list, list + K, std::back_inserter(merged));
+    o->union_idx.swap(merged);
+  }
+  const uint32_t* S = o->union_idx.data();
+  const int64_t n_set = static_cast<int64_t>(o->union_idx.size());
 
   // (f) sum over workers in ascending order at the shared indices, into a zeroed dense update
 #pragma omp parallel for num_threads(nthreads) schedule(static)
   for (int64_t i = 0; i < N; ++i) update[i] = 0.0f;
 #pragma omp parallel for num_threads(nthreads) schedule(static)
-  for (int64_t j = 0; j < K; ++j) {
+  for (int64_t j = 0; j < n_set; ++j) {
     const size_t i = S[j];
     float s = o->acc[i];
     for (int32_t w = 1; w < W; ++w) s = s + o->acc[static_cast<size_t>(w) * N + i];
@@ -514,7 +537,7 @@ void oracle_step(void* h, const float* grads, const float* weights, float* updat
 
   // (g) what was sent leaves every worker's residual; the rest stays
 #pragma omp parallel for num_threads(nthreads) schedule(static)
-  for (int64_t j = 0; j < K; ++j) {
+  for (int64_t j = 0; j < n_set; ++j) {
     const size_t i = S[j];
     for (int32_t w = 0; w < W; ++w) o->acc[static_cast<size_t>(w) * N + i] = 0.0f;
   }

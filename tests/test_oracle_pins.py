@@ -739,3 +739,72 @@ def test_layerwise_step_equals_bruteforce_with_two_chosen_nodes():
         for w_ in range(W):
             assert np.array_equal(u32(orc.residual(w_)), u32(acc[w_]))
     assert saw_both_branches == {True, False}
+
+
+# ---------------------------------------------------------------- several chosen nodes in the ratio mode
+
+
+def test_ratio_mode_union_of_chosen_nodes_equals_bruteforce():
+    # every worker's own top-k list comes from the full-sort model; the index set is the union of the
+    # chosen nodes' lists, and sum / zeroing run over that union
+    layers, W, n, ratio, eps = [30, 6, 50], 5, 3, 8.0, F(1e-8)
+    N = sum(layers)
+    rng = np.random.default_rng(21)
+    weights = (rng.integers(-2, 3, N) * 0.5).astype(np.float32)
+    orc = oracle.Oracle(layers, W, ratio, eps, seed=13)
+    orc.set_n_leaders(n)
+    k = [min(m, max(1, math.ceil(m / ratio))) for m in layers]
+    acc = np.zeros((W, N), np.float32)
+    sizes = set()
+    for t in range(5):
+        grads = (rng.integers(-4, 5, size=(W, N)) / 4.0).astype(np.float32)  # coarse: ties everywhere
+        acc = (acc + grads).astype(np.float32)
+        upd = orc.step(grads, weights)
+        lists = []
+        for w in range(W):
+            lst, o = [], 0
+            for m, kk in zip(layers, k):
+                imp = [bits(importance(acc[w, o + i], weights[o + i], eps)) for i in range(m)]
+                ranked = sorted(range(m), key=lambda i: (-imp[i], i))
+                lst += sorted(o + i for i in ranked[:kk])
+                o += m
+            lists.append(lst)
+            assert orc.selection(w)[0].tolist() == lst
+        rs = oracle.leaders(13, t, W, n)
+        assert orc.leader == rs[0]
+        S = sorted(set().union(*(lists[r] for r in rs)))
+        sizes.add(len(S))
+        assert orc.index_set().tolist() == S and sum(k) <= len(S) <= n * sum(k)
+        assert orc.mask().tolist() == [1 if i in set(S) else 0 for i in range(N)]
+        want = np.zeros(N, np.float32)
+        for i in S:
+            s = acc[0, i]
+            for w in range(1, W):
+                s = F(s + acc[w, i])
+            want[i] = F(F(0) + s)
+            acc[:, i] = 0
+        assert np.array_equal(u32(upd), u32(want))
+        for w in range(W):
+            assert np.array_equal(u32(orc.residual(w)), u32(acc[w]))
+    assert any(s > sum(k) for s in sizes)  # the union really grew beyond one node's list
+
+
+def test_ratio_mode_one_chosen_node_is_the_plain_path_and_all_nodes_cover_every_list():
+    layers, W, ratio = [200, 64], 4, 16.0
+    N = sum(layers)
+    rng = np.random.default_rng(3)
+    weights = rng.standard_normal(N).astype(np.float32)
+    a, b, c = (oracle.Oracle(layers, W, ratio, 1e-8, seed=2) for _ in range(3))
+    b.set_n_leaders(1)
+    c.set_n_leaders(W)
+    for t in range(3):
+        g = rng.standard_normal((W, N)).astype(np.float32)
+        ua, ub = a.step(g, weights), b.step(g, weights)
+        assert np.array_equal(u32(ua), u32(ub)) and a.index_set().tolist() == a.selection(a.leader)[0].tolist()
+        c.step(g, weights)
+        every = set()
+        for w in range(W):
+            every |= set(c.selection(w)[0].tolist())
+        assert set(c.index_set().tolist()) == every
+        for w in range(W):  # everything any worker selected has left every residual
+            assert not c.residual(w)[sorted(every)].any()
