@@ -202,9 +202,11 @@ int iwp_reset(iwp_ctx* ctx);
 /* Options (tests and experiments):
  *   "leader_override"  >= 0 forces the leader of every following step, -1 = seeded draw
  *   "force_scalar"     1 = never use 128-bit accesses
- *   "n_leaders"        threshold-mode contexts only: 1 .. min(W, 8) chosen nodes per step whose masks are
- *                      OR-ed (Algorithm 1: Mask = OR Mask_ri); the listed values are r_1's; a forced
- *                      leader ("leader_override") makes the step a one-node step
+ *   "n_leaders"        1 .. min(W, 8) chosen nodes per step, drawn without replacement, whose index sets are
+ *                      OR-ed (Algorithm 1: Mask = OR Mask_ri).  Threshold mode: the masks of the chosen
+ *                      nodes; the listed values are r_1's.  Ratio mode: the union of the chosen nodes' own
+ *                      top-k lists (every worker still lists its own top-k; iwp_get_mask() gives the union).
+ *                      A forced leader ("leader_override") makes the step a one-node step
  *   "random_select"    threshold-mode contexts only: 1 = Section 3.3's random gradient selection: an
  *                      element whose importance does not exceed its layer's threshold is still sent iff
  *                      u < importance / thr (fp32 quotient), u = u24 * 2^-24 with

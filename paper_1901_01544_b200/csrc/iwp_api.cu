@@ -65,6 +65,7 @@ struct iwp_ctx {
   uint64_t list_cap = 0;          // capacity of the single index list
   bool thr_set = false;
   int32_t n_leaders = 1;          // chosen nodes whose masks are OR-ed
+  LeaderSet last_chosen{};        // ratio mode: the chosen nodes of the last step
   bool random_select = false;     // Section 3.3: P(update) = importance / threshold below the threshold
   uint32_t* d_thr = nullptr;      // [layer] fp32 patterns of the thresholds
   bool layerwise = false;         // Section 3.4: thresholds from each chosen node's per-layer statistics (Eq. 4)
@@ -326,10 +327,24 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   };
   const bool tiled = !p.large_layers.empty();
   const bool spec = tiled && c->speculate && c->spec_pairs > 0;
+  // several chosen nodes (their lists are OR-ed) unless the leader is forced; r_1 is `leader` either way
+  LeaderSet ls{};
+  if (c->n_leaders > 1 && c->leader_override < 0) {
+    ls = leaders_at(c->seed, static_cast<uint64_t>(c->t), W, c->n_leaders);
+  } else {
+    ls.n = 1;
+    ls.r[0] = leader;
+  }
+  c->last_chosen = ls;
   // the overlapped schedule (not while every stage boundary is being timed)
-  const bool pipe = spec && W > 1 && c->overlap == 1 && c->time_stages != 1 && c->side_a != nullptr && c->side_b != nullptr;
+  const bool pipe = spec && W > 1 && ls.n == 1 && c->overlap == 1 && c->time_stages != 1 && c->side_a != nullptr &&
+                    c->side_b != nullptr;
   if (!pipe) {
     const int rc = join_deferred(c);
+    if (rc != IWP_OK) return rc;
+  }
+  if (!spec) {  // the multi-pass path reads the residuals as they are (before the small layers' kernel adds to them)
+    const int rc = flush_pending_zero(c);
     if (rc != IWP_OK) return rc;
   }
   stage_mark_at(c, 0);
@@ -351,10 +366,6 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     if (fork_small && !cuda_ok(cudaEventRecord(c->ev_join, c->side))) return IWP_ERR_CUDA;
   }
   stage_mark_at(c, 1);
-  if (!spec) {  // the multi-pass path reads the residuals as they are
-    const int rc = flush_pending_zero(c);
-    if (rc != IWP_OK) return rc;
-  }
   // The per-pair records alternate between two copies, so that a select still running for the last
   // step keeps reading its own while this step's sampling writes the other.
   c->info_cur = c->d_info + static_cast<size_t>(c->t & 1) * c->n_pairs;
@@ -489,7 +500,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     stage_mark_at(c, 4);
     // The reduction needs the leader's list only: write that one here and the other workers' lists on
     // the side stream, beside the reduction; they are joined at the end of the step.
-    const bool split = spec && W > 1 && c->side != nullptr;
+    const bool split = spec && W > 1 && ls.n == 1 && c->side != nullptr;  // (a union needs every chosen node's list here)
     auto write = [&](cudaStream_t st, WorkerSel ws) {
       dim3 grid(n_chunks, static_cast<unsigned>(sel_count(ws, W)));
       k_write<VEC><<<grid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur,
@@ -515,7 +526,14 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   }
   stage_mark_at(c, 5);
   if (fork_small && !cuda_ok(cudaStreamWaitEvent(s, c->ev_join, 0))) return IWP_ERR_CUDA;
-  if (spec) {
+  if (ls.n > 1) {
+    // union of the chosen nodes' lists: the zero mask is all clear here (applied and cleared by the streaming
+    // pass, or flushed at the start of a multi-pass step) and serves to give every element one owner
+    const uint64_t entries = static_cast<uint64_t>(ls.n) * K;
+    k_union_sum_scatter<<<static_cast<unsigned>((entries + THREADS - 1) / THREADS), THREADS, 0, s>>>(
+        c->sel_idx, c->acc, update, c->zmask, N, K, W, ls);
+    c->zero_pending = true;  // the marks are cleared with the next step's
+  } else if (spec) {
     k_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->sel_slot, c->side_val,
                                               c->cand_val, c->acc, update, c->zmask, N, K, W, leader);
     c->zero_pending = true;
@@ -1060,8 +1078,10 @@ int iwp_get_mask(iwp_ctx* c, uint8_t* dst) {
     return IWP_OK;
   }
   const unsigned blocks = static_cast<unsigned>((K + THREADS - 1) / THREADS);
-  k_mask_scatter<<<blocks, THREADS, 0, c->stream>>>(c->sel_idx + static_cast<uint64_t>(c->leader) * K, dst, K);
-  if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+  for (int j = 0; j < c->last_chosen.n; ++j) {  // the index set is the union of the chosen nodes' lists
+    k_mask_scatter<<<blocks, THREADS, 0, c->stream>>>(c->sel_idx + static_cast<uint64_t>(c->last_chosen.r[j]) * K, dst, K);
+    if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+  }
   return IWP_OK;
 }
 
@@ -1113,7 +1133,7 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
     return IWP_OK;
   }
   if (!std::strcmp(key, "n_leaders")) {
-    if (!c->threshold_mode || v < 1 || v > MAX_LEADERS || v > c->plan.W) return IWP_ERR_INVALID;
+    if (v < 1 || v > MAX_LEADERS || v > c->plan.W) return IWP_ERR_INVALID;
     c->n_leaders = static_cast<int32_t>(v);
     return IWP_OK;
   }

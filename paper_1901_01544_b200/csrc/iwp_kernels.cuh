@@ -1202,6 +1202,40 @@ __global__ void __launch_bounds__(THREADS)
   update[i] = __fadd_rn(0.0f, s);
 }
 
+// Steps (e)-(g) with several chosen nodes (Algorithm 1: Mask = OR Mask_ri): the index set is the union
+// of the chosen nodes' lists.  One thread per list entry of every chosen node; the first thread to mark
+// an element in the (all-zero) bit mask owns it - gathers the W residuals, sums them in ascending
+// worker order, scatters the sum and zeroes the residuals - and every later entry with the same element
+// returns at once, so nothing is read after it was zeroed.  The marks stay set (the element is +0 now
+// whether or not the next streaming pass treats it so).
+__global__ void __launch_bounds__(THREADS)
+    k_union_sum_scatter(const uint32_t* __restrict__ sel_idx, float* __restrict__ acc, float* __restrict__ update,
+                        uint32_t* __restrict__ seen, uint64_t N, uint64_t K, int W, LeaderSet ls) {
+  const uint64_t q = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (q >= static_cast<uint64_t>(ls.n) * K) return;
+  const int j = static_cast<int>(q / K);
+  int r = ls.r[0];
+#pragma unroll
+  for (int u = 1; u < MAX_LEADERS; ++u)
+    if (u == j) r = ls.r[u];
+  const uint64_t i = sel_idx[static_cast<uint64_t>(r) * K + q % K];
+  const uint32_t bit = zmask_bit(i);
+  if (atomicOr(&seen[zmask_word(i)], bit) & bit) return;
+  float* p = acc + i;
+  float s = 0.0f;
+  for (int w0 = 0; w0 < W; w0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = (w0 + u < W) ? p[static_cast<uint64_t>(w0 + u) * N] : 0.0f;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
+    }
+  }
+  for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
+  update[i] = __fadd_rn(0.0f, s);
+}
+
 // A worker's select that is left running on a side stream past the end of the step may still need
 // the weights if its pair has to fall back to the multi-pass path, and the caller is free to change
 // them once the step's stream work is done.  So the weights of every layer in which a worker other

@@ -42,7 +42,7 @@ def compare_state(pr: Pruner, orc: "oracle.Oracle", update_gpu: torch.Tensor, up
 
 def run_parity(layer_sizes, W, ratio, eps, seed, steps, weights: torch.Tensor, grads_fn, options=None,
                leader_overrides=None, check_mask=True, threads=0, residual_every=1, momentum=None, state_every=1,
-               weights_fn=None):
+               weights_fn=None, n_leaders=1):
     """weights: CUDA tensor [N]; grads_fn(t) -> CUDA tensor [W, N].
 
     state_every: lists, mask, residuals and the device status are looked at only every that many steps
@@ -63,6 +63,9 @@ def run_parity(layer_sizes, W, ratio, eps, seed, steps, weights: torch.Tensor, g
     if momentum is not None:
         pr.set_momentum(momentum)
         orc.set_momentum(momentum)
+    if n_leaders > 1:  # several chosen nodes: the index set is the union of their lists
+        pr.set_option("n_leaders", n_leaders)
+        orc.set_n_leaders(n_leaders)
     w_host = weights.cpu().numpy()
     update = torch.full((pr.N,), float("nan"), dtype=torch.float32, device="cuda")
     for t in range(steps):

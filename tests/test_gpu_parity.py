@@ -277,6 +277,45 @@ def test_back_to_back_steps_with_leader_overrides():
                leader_overrides=[0, 3, 3, 1, -1, 2, -1, 0], residual_every=1000, state_every=1000)
 
 
+# ------------------------------------------------------------------ several chosen nodes (Mask = OR Mask_ri)
+
+
+@pytest.mark.parametrize("speculate", [1, 0])
+@pytest.mark.parametrize("n_leaders", [2, 4])
+def test_union_of_several_chosen_nodes(n_leaders, speculate):
+    sizes, W, ratio = [70000, 64, 16385, 300000, 9, 40000], 5, 32.0
+    N = sum(sizes)
+    weights = _weights(N, 21)
+    run_parity(sizes, W, ratio, 1e-8, seed=6, steps=5, weights=weights, grads_fn=lambda t: _randn((W, N), 800 + t),
+               n_leaders=n_leaders, options={"speculate": speculate}, residual_every=2)
+
+
+def test_union_with_ties_fallbacks_and_identical_workers():
+    # coarse values (ties, fallbacks) and two workers with the same gradients: their lists coincide, so every
+    # element of the union has two entries competing for it
+    sizes, W, ratio = [70000, 300, 20000], 4, 16.0
+    N = sum(sizes)
+    g0 = torch.Generator(device=DEV)
+    g0.manual_seed(5)
+    weights = torch.randint(-3, 4, (N,), generator=g0, device=DEV).float() * 0.25
+
+    def grads(t):
+        gg = torch.Generator(device=DEV)
+        gg.manual_seed(870 + t)
+        g = torch.randint(-4, 5, (W, N), generator=gg, device=DEV).float() / 8.0 if t % 2 else \
+            torch.randn((W, N), generator=gg, device=DEV) * 1e-3
+        g[2] = g[0]
+        return g
+
+    run_parity(sizes, W, ratio, 1e-8, seed=1, steps=5, weights=weights, grads_fn=grads, n_leaders=4)
+
+
+def test_union_on_a_scaled_network_shape():
+    c = _scaled_case("resnet50_w8")
+    run_parity(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, c.steps, c.weights(DEV), lambda t: c.grads(t, DEV), n_leaders=3,
+               residual_every=1000)
+
+
 # ------------------------------------------------------------------ momentum on the residual (Eq. 3)
 
 
