@@ -165,7 +165,8 @@ def test_threshold_mode_several_chosen_nodes(n_leaders):
     assert L.iwp_set_option(pr._h, b"n_leaders", 0) == binding.IWP_ERR_INVALID
     pr.close()
     ratio = Pruner(sizes, W, 4.0)
-    assert L.iwp_set_option(ratio._h, b"n_leaders", 2) == binding.IWP_ERR_INVALID  # ratio-mode context
+    assert L.iwp_set_option(ratio._h, b"n_leaders", 2) == 0  # the ratio mode takes several chosen nodes too
+    assert L.iwp_set_option(ratio._h, b"n_leaders", 9) == binding.IWP_ERR_INVALID  # more than eight
     ratio.close()
 
 
