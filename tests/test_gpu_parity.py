@@ -335,3 +335,66 @@ def test_momentum_on_a_scaled_network_shape():
     weights = c.weights(DEV)
     run_parity(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, c.steps, weights, lambda t: c.grads(t, DEV), momentum=0.9,
                residual_every=1000)
+
+
+# ------------------------------------------------------------------ option changes between steps
+
+
+@pytest.mark.parametrize("seed", range(int(os.environ.get("IWP_WALK_SEEDS", "4"))))
+def test_random_option_changes_between_steps(seed):
+    """A seeded walk over the library's switches between steps - schedule, select path, number of chosen
+    nodes, forced leaders, momentum, step counter, residual reads - against the oracle taking the same walk.
+    Lists and residuals are compared only now and then, so late selects of one step meet all kinds of
+    next steps."""
+    import oracle
+    from paper_1901_01544_b200.binding import Pruner
+    from parity import compare_state
+
+    rng = np.random.default_rng(1000 + seed)
+    sizes, W, ratio = [70000, 64, 16385, 150000, 9, 40000], 4, 32.0
+    N = sum(sizes)
+    weights = _weights(N, 31 + seed)
+    w_host = weights.cpu().numpy()
+    pr = Pruner(sizes, W, ratio, 1e-8, seed)
+    orc = oracle.Oracle(sizes, W, ratio, 1e-8, seed)
+    pr.set_option("overlap", 1)  # the workload is below the size at which the library would choose it by itself
+    update = torch.full((N,), float("nan"), device=DEV)
+    for t in range(24):
+        what = int(rng.integers(0, 9))
+        if what == 0:
+            pr.set_option("overlap", int(rng.integers(0, 2)))
+        elif what == 1:
+            pr.set_option("speculate", int(rng.integers(0, 2)))
+        elif what == 2:
+            n = int(rng.integers(1, W + 1))
+            pr.set_option("n_leaders", n)
+            orc.set_n_leaders(n)
+        elif what == 3:
+            lead = int(rng.integers(-1, W))
+            pr.set_option("leader_override", lead)
+            orc.set_leader_override(lead)
+        elif what == 4:
+            m = float(rng.choice([1.0, 0.9, 0.5]))
+            pr.set_momentum(m)
+            orc.set_momentum(m)
+        elif what == 5:
+            for w in range(W):  # forces the pending zeroing out
+                assert_bits_equal(pr.residual(w).cpu().numpy(), orc.residual(w), f"before step {t}: worker {w} residual")
+        elif what == 6:
+            pr.set_option("time_stages", int(rng.integers(0, 3)))
+        coarse = rng.random() < 0.3  # ties and fallbacks now and then
+        if coarse:
+            g = torch.randint(-4, 5, (W, N), device=DEV, generator=torch.Generator(device=DEV).manual_seed(t)).float() / 8.0
+        else:
+            g = _randn((W, N), 2000 + 100 * seed + t)
+        pr.step(g, weights, update)
+        upd_cpu = orc.step(np.ascontiguousarray(g.cpu().numpy()), w_host)
+        assert pr.leader == orc.leader
+        if rng.random() < 0.4 or t == 23:
+            compare_state(pr, orc, update, upd_cpu, f"step {t}", check_residual=bool(rng.random() < 0.5) or t == 23)
+        else:
+            assert_bits_equal(update.cpu().numpy(), upd_cpu, f"step {t}: update")
+        update.fill_(float("nan"))
+    pr.set_option("time_stages", 0)
+    pr.close()
+    orc.close()
