@@ -100,6 +100,41 @@ def test_runs_on_a_side_stream():
     pr.close()
 
 
+def test_stream_switch_between_overlapped_steps():
+    # steps alternate between two streams while the other workers' selects of the last step may still be
+    # running on the library's own streams; every list is checked at the end of each pair of steps
+    import oracle
+
+    sizes, W, ratio = [80000, 300, 50000], 4, 16.0
+    N = sum(sizes)
+    weights, grads = _inputs(W, N, 8)
+    pr = Pruner(sizes, W, ratio, 1e-8, 3)
+    pr.set_option("overlap", 1)
+    orc = oracle.Oracle(sizes, W, ratio, 1e-8, 3)
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    w_host = weights.cpu().numpy()
+    for t in range(6):
+        s = streams[t % 2]
+        g = grads[t % len(grads)]
+        with torch.cuda.stream(s):
+            pr.use_current_stream()
+            got = pr.step(g, weights)
+        s.synchronize()
+        want = orc.step(np.ascontiguousarray(g.cpu().numpy()), w_host)
+        assert_bits_equal(got.cpu().numpy(), want, f"step {t}: update")
+        if t % 2 == 1:
+            with torch.cuda.stream(s):
+                assert pr.sync_status() == 0
+                for w in range(W):
+                    idx, val = pr.selection(w)
+                    oi, ov = orc.selection(w)
+                    assert np.array_equal(idx.cpu().numpy().view(np.uint32), oi)
+                    assert_bits_equal(val.cpu().numpy(), ov, f"step {t}: worker {w} list values")
+    pr.close()
+    orc.close()
+
+
 def test_options_stats_and_misuse():
     pr = Pruner([5000, 20000], 2, 8.0, 1e-8, 0)
     L = binding.lib()
