@@ -1331,11 +1331,12 @@ __global__ void __launch_bounds__(THREADS)
 }
 
 // ---------------------------------------------------------------------------------------
-// Absolute-threshold mode: Algorithm 1 as printed.  Only the chosen node forms a mask, per layer
-// Mask = |G / w| > thr (strict), so after the plain accumulate pass (k_accumulate) the select is
-// two looks at the chosen nodes' residuals (one node, or several whose masks are OR-ed): count per
-// chunk, scan, stable compaction; the index set has whatever size results.  thr_bits: the thresholds' fp32 patterns (thr >= 0, so patterns order like
-// values and +inf passes nothing).
+// Absolute-threshold mode: Algorithm 1 as printed.  Only the chosen nodes form masks, per layer
+// Mask = |G / w| > thr (strict; several nodes' masks are OR-ed), and the index set has whatever size
+// results.  A step: step (a) for the chosen nodes (k_thr_accumulate_chosen), two looks at their
+// residuals - count per chunk, scan, stable compaction with one set bit per element - and one
+// streaming pass over all workers that does the rest (k_thr_fused).  thr_bits: the thresholds' fp32
+// patterns; a negative one (the layer-wise rule can produce it) passes everything, +inf nothing.
 // ---------------------------------------------------------------------------------------
 // Random selection parameters of a step (Section 3.3): off, or the seed and step of the draws.
 struct RandomSelect {
@@ -1807,30 +1808,8 @@ __global__ void __launch_bounds__(THREADS)
   }
 }
 
-// Steps (e)-(g) with a list whose length is only known on the device: grid-stride over its entries.
-__global__ void __launch_bounds__(THREADS)
-    k_thr_gather(const uint32_t* __restrict__ sel_idx, const uint32_t* __restrict__ list_len, uint32_t capacity,
-                 float* __restrict__ acc, float* __restrict__ update, uint64_t N, int W) {
-  const uint32_t len = min(*list_len, capacity);
-  for (uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x; j < len;
-       j += static_cast<uint64_t>(gridDim.x) * THREADS) {
-    const uint64_t i = sel_idx[j];
-    float* p = acc + i;
-    float s = 0.0f;
-    for (int w0 = 0; w0 < W; w0 += 8) {
-      float v[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) v[u] = (w0 + u < W) ? p[static_cast<uint64_t>(w0 + u) * N] : 0.0f;
-#pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
-      }
-    }
-    for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
-    update[i] = __fadd_rn(0.0f, s);
-  }
-}
-
+// Byte mask of the index set of a threshold-mode step (accessor): grid-stride over the list, whose length
+// is only known on the device.
 __global__ void __launch_bounds__(THREADS)
     k_thr_mask(const uint32_t* __restrict__ sel_idx, const uint32_t* __restrict__ list_len, uint32_t capacity,
                uint8_t* __restrict__ dst) {
