@@ -177,6 +177,69 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------------- workers spread over GPUs
+
+
+def run_sharded(args):
+    """--shard: the workload's W workers spread over the N ranks (W / N each), the chosen worker's index list
+    broadcast and the gathered values all-gathered over NCCL (ShardedPruner).  Total work is fixed: strong
+    scaling.  Not the default arm; on one GPU it measures the cost of the three-phase protocol itself."""
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the pruning path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world == 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29533")
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    from paper_1901_01544_b200 import build as lib_build
+
+    if rank == 0:
+        lib_build.build()
+    dist.barrier()
+    from paper_1901_01544_b200.binding import ShardedPruner
+
+    c = make_workload(args.config, args.layers)
+    if c.W % world != 0:
+        raise SystemExit(f"--shard needs the workload's {c.W} workers to divide over {world} ranks")
+    Wl, N = c.W // world, c.N
+    weights = c.weights(dev)
+    n_sets = args.grad_sets or 3
+    sets = [c.grads(t, dev)[rank * Wl:(rank + 1) * Wl].contiguous() for t in range(n_sets)]
+    update = torch.empty(N, dtype=torch.float32, device=dev)
+    sp = ShardedPruner(c.layer_sizes, c.W, c.ratio, c.eps, c.seed)
+    for t in range(args.warmup):
+        sp.step(sets[t % n_sets], weights, update)
+    torch.cuda.synchronize()
+    dist.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(args.steps):
+        sp.step(sets[(args.warmup + t) % n_sets], weights, update)
+    e1.record()
+    torch.cuda.synchronize()
+    dist.barrier()
+    ms_total = max_over_ranks(e0.elapsed_time(e1), dist, dev)
+    assert sp.local.sync_status() == 0
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": c.name, "mode": "sharded", "W": c.W, "W_per_gpu": Wl, "N": N, "K": sp.K,
+                       "collectives": "broadcast of K uint32 + all-gather of W x K fp32 per step (NCCL)"},
+            "gpu_launches": sp.local.stat("launches"),
+        }
+        print(json.dumps(line), flush=True)
+    dist.destroy_process_group()
+
+
 # ---------------------------------------------------------------------------------- the CUDA arm
 
 
@@ -390,6 +453,9 @@ def main():
     ap.add_argument("--mode", default="ratio", choices=["ratio", "threshold"],
                     help="ratio: exact layer-wise top-k at the configured compression (headline); threshold: "
                          "absolute per-layer thresholds on the chosen node (Algorithm 1 as printed)")
+    ap.add_argument("--shard", action="store_true",
+                    help="spread the workload's W workers over the ranks (ShardedPruner: NCCL broadcast + all-gather) "
+                         "instead of running independent replicas")
     ap.add_argument("--layerwise", default=None,
                     help="alpha,beta,C - with --mode threshold: layer-wise thresholds alpha +/- beta var/mean (Eq. 4)")
     ap.add_argument("--layers", default=None, help="lo:hi - only these layers of the workload (small profiling case)")
@@ -405,6 +471,8 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.shard:
+        run_sharded(args)
     else:
         run_ours(args)
 

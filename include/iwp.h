@@ -167,6 +167,36 @@ int iwp_set_momentum(iwp_ctx* ctx, float m);
  * Advances the step counter.  Errors: IWP_ERR_INVALID (NULL), IWP_ERR_CUDA (launch failure). */
 int iwp_step(iwp_ctx* ctx, const float* grads_dev, const float* weights_dev, float* update_dev);
 
+/* ---- workers spread over several contexts (one context per GPU) ------------------------------
+ * The paper's deployment is a ring of nodes: the chosen node's index set travels to everybody
+ * (Algorithm 1: AllGather of the encoded mask), then the masked gradients are all-reduced.  With the W
+ * workers of a job split into consecutive groups, one context of W_local workers per group, a step is
+ *   1. iwp_shard_select() on every context: steps (a)-(d) for its own workers;
+ *   2. the caller reads the chosen worker's list from the context that holds it
+ *      (iwp_get_selection(), K indices) and sends it to every context (broadcast);
+ *   3. iwp_shard_gather() on every context: its workers' residuals at those indices (step (e));
+ *   4. the caller concatenates the groups' values in global worker order (all-gather);
+ *   5. iwp_shard_apply() on every context: step (f) over all W workers in ascending order - so every
+ *      context holds the same update, bit for bit the one a single context of W workers computes -
+ *      and step (g) for its own workers.
+ * The transport (steps 2 and 4) is the caller's: the Python binding's ShardedPruner uses
+ * torch.distributed (NCCL).  Ratio-mode contexts only; all three calls are asynchronous on the
+ * context's stream like iwp_step(). */
+
+/* Steps (a)-(d) for this context's W_local workers.  update_dev (N floats) is zero-filled here and
+ * must be the buffer later given to iwp_shard_apply().  Does not advance the step counter. */
+int iwp_shard_select(iwp_ctx* ctx, const float* grads_dev, const float* weights_dev, float* update_dev);
+
+/* vals_dev[w * n + j] = residual of local worker w at idx_dev[j], w < W_local, j < n (the values as they
+ * are after iwp_shard_select()).  idx_dev: n distinct flat indices below N. */
+int iwp_shard_gather(iwp_ctx* ctx, const uint32_t* idx_dev, int64_t n, float* vals_dev);
+
+/* update_dev[idx_dev[j]] = +0 + (((v[0][j] + v[1][j]) + v[2][j]) + ...) over the W_total rows of
+ * vals_all_dev (row w = global worker w, n floats each); the residuals of this context's workers
+ * become +0 at the n indices.  Advances the step counter.  IWP_ERR_INVALID if W_total < W_local. */
+int iwp_shard_apply(iwp_ctx* ctx, const uint32_t* idx_dev, int64_t n, const float* vals_all_dev, int32_t W_total,
+                    float* update_dev);
+
 /* The same step with HOST buffers (pinned memory recommended): copies grads and weights to
  * library-owned staging buffers (allocated on first use), runs iwp_step(), copies the update
  * back and synchronises the stream before returning. */

@@ -22,7 +22,7 @@ EXPORTS = [
     "iwp_get_step", "iwp_set_step", "iwp_get_leader", "iwp_get_residual", "iwp_set_residual",
     "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat", "iwp_select_static",
     "iwp_set_momentum", "iwp_create_threshold", "iwp_set_thresholds", "iwp_get_list_length", "iwp_leaders_at",
-    "iwp_set_layerwise", "iwp_get_layer_thresholds",
+    "iwp_set_layerwise", "iwp_get_layer_thresholds", "iwp_shard_select", "iwp_shard_gather", "iwp_shard_apply",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -60,6 +60,9 @@ def lib() -> C.CDLL:
         L.iwp_set_momentum.argtypes = [vp, f32]
         L.iwp_step.argtypes = [vp, vp, vp, vp]
         L.iwp_step_host.argtypes = [vp, vp, vp, vp]
+        L.iwp_shard_select.argtypes = [vp, vp, vp, vp]
+        L.iwp_shard_gather.argtypes = [vp, vp, i64, vp]
+        L.iwp_shard_apply.argtypes = [vp, vp, i64, vp, i32, vp]
         L.iwp_sync_status.argtypes = [vp]
         L.iwp_get_layout.argtypes = [vp, vp, vp]
         L.iwp_get_sizes.argtypes = [vp, vp]
@@ -195,13 +198,17 @@ class Pruner:
         _check(lib().iwp_set_stream(self._h, C.c_void_p(s)), "iwp_set_stream")
 
     # the step
-    def step(self, grads, weights, update=None):
+    def _check_inputs(self, grads, weights, update) -> None:
         t = self._torch
         assert grads.is_cuda and grads.dtype == t.float32 and grads.is_contiguous() and grads.numel() == self.W * self.N
         assert weights.is_cuda and weights.dtype == t.float32 and weights.is_contiguous() and weights.numel() == self.N
+        assert update.is_cuda and update.dtype == t.float32 and update.is_contiguous() and update.numel() == self.N
+
+    def step(self, grads, weights, update=None):
+        t = self._torch
         if update is None:
             update = t.empty(self.N, dtype=t.float32, device=grads.device)
-        assert update.is_cuda and update.dtype == t.float32 and update.is_contiguous() and update.numel() == self.N
+        self._check_inputs(grads, weights, update)
         iwp_step(self._h, grads.data_ptr(), weights.data_ptr(), update.data_ptr())
         return update
 
@@ -212,6 +219,25 @@ class Pruner:
             assert (not x.is_cuda) and x.dtype == t.float32 and x.is_contiguous() and x.numel() == n
         iwp_step_host(self._h, grads.data_ptr(), weights.data_ptr(), update.data_ptr())
         return update
+
+    # the three phases of a step whose workers are spread over several contexts (see ShardedPruner)
+    def shard_select(self, grads, weights, update) -> None:
+        self._check_inputs(grads, weights, update)
+        _check(lib().iwp_shard_select(self._h, grads.data_ptr(), weights.data_ptr(), update.data_ptr()), "iwp_shard_select")
+
+    def shard_gather(self, idx):
+        t = self._torch
+        assert idx.is_cuda and idx.dtype == t.int32 and idx.is_contiguous()
+        vals = t.empty((self.W, idx.numel()), dtype=t.float32, device=self.device)
+        _check(lib().iwp_shard_gather(self._h, idx.data_ptr(), idx.numel(), vals.data_ptr()), "iwp_shard_gather")
+        return vals
+
+    def shard_apply(self, idx, vals_all, update) -> None:
+        t = self._torch
+        assert vals_all.is_cuda and vals_all.dtype == t.float32 and vals_all.is_contiguous()
+        assert vals_all.dim() == 2 and vals_all.shape[1] == idx.numel()
+        _check(lib().iwp_shard_apply(self._h, idx.data_ptr(), idx.numel(), vals_all.data_ptr(), int(vals_all.shape[0]),
+                                     update.data_ptr()), "iwp_shard_apply")
 
     def set_thresholds(self, thr: Sequence[float]) -> None:
         arr = (C.c_float * self.L)(*[float(x) for x in thr])
@@ -295,3 +321,59 @@ class Pruner:
         v = C.c_int64()
         _check(lib().iwp_get_stat(self._h, key.encode(), C.byref(v)), f"iwp_get_stat({key})")
         return int(v.value)
+
+
+class ShardedPruner:
+    """The W workers of a job spread over the ranks of a torch.distributed group, W / world consecutive
+    workers per rank (rank r holds workers r * W_local .. (r + 1) * W_local - 1), one GPU per rank.
+
+    A step is the ring deployment of the paper in three device phases and two collectives: every rank
+    selects for its own workers; the chosen worker's index list is broadcast from the rank that holds it
+    (Algorithm 1's AllGather of the encoded mask, here the sorted uint32 list); every rank gathers its
+    workers' residuals at those indices; the gathered values are all-gathered (rank order = worker order)
+    and every rank forms the sum over ALL workers in ascending order - bit for bit the update a single
+    context of W workers computes - and zeroes what its own workers sent.  Only argument marshalling and
+    the two collectives happen here; every step of the method runs in the library's kernels.
+
+    `engine`: the per-rank object with shard_select / selection / shard_gather / shard_apply (default: a
+    Pruner on the current CUDA device)."""
+
+    def __init__(self, layer_sizes: Sequence[int], W_total: int, ratio: float, eps: float = 1e-8, seed: int = 0,
+                 group=None, engine=None):
+        import torch
+        import torch.distributed as dist
+
+        self._torch, self._dist, self.group = torch, dist, group
+        self.rank, self.world = dist.get_rank(group), dist.get_world_size(group)
+        if W_total < 1 or W_total % self.world != 0:
+            raise ValueError("the number of workers must be a positive multiple of the group size")
+        self.W_total, self.W_local, self.seed, self.t = W_total, W_total // self.world, int(seed), 0
+        self.leader_override = -1
+        self.leader = -1
+        self.local = engine if engine is not None else Pruner(layer_sizes, self.W_local, ratio, eps, seed)
+        self.N, self.K = self.local.N, self.local.K
+
+    def _global_rank(self, group_rank: int) -> int:
+        return group_rank if self.group is None else self._dist.get_global_rank(self.group, group_rank)
+
+    def step(self, grads_local, weights, update):
+        """grads_local: this rank's [W_local, N] gradients; weights [N]; update [N] (fully overwritten, the
+        same on every rank)."""
+        t, dist = self._torch, self._dist
+        leader = self.leader_override if self.leader_override >= 0 else iwp_leader_at(self.seed, self.t, self.W_total)
+        owner, local_worker = divmod(leader, self.W_local)
+        self.local.shard_select(grads_local, weights, update)
+        if self.rank == owner:
+            idx = self.local.selection(local_worker)[0]
+        else:
+            idx = t.empty(self.K, dtype=t.int32, device=update.device)
+        dist.broadcast(idx, src=self._global_rank(owner), group=self.group)
+        vals_local = self.local.shard_gather(idx)
+        vals_all = t.empty((self.W_total, self.K), dtype=t.float32, device=update.device)
+        dist.all_gather_into_tensor(vals_all, vals_local, group=self.group)
+        self.local.shard_apply(idx, vals_all, update)
+        self.leader, self.t = leader, self.t + 1
+        return update
+
+    def close(self) -> None:
+        self.local.close()

@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 
 #include <cmath>
+#include <algorithm>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -25,6 +26,7 @@ struct iwp_ctx {
   int64_t leader_override = -1;
   bool force_scalar = false;
   bool speculate = true;
+  bool select_only = false;  // iwp_shard_select(): a step stops before the reduction
   cudaStream_t stream = nullptr;
   cudaStream_t side = nullptr;       // the one-CTA path of small layers runs here, beside the tiled path
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_fork2 = nullptr, ev_join2 = nullptr;
@@ -337,8 +339,8 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   }
   c->last_chosen = ls;
   // the overlapped schedule (not while every stage boundary is being timed)
-  const bool pipe = spec && W > 1 && ls.n == 1 && c->overlap == 1 && c->time_stages != 1 && c->side_a != nullptr &&
-                    c->side_b != nullptr;
+  const bool pipe = spec && W > 1 && ls.n == 1 && !c->select_only && c->overlap == 1 && c->time_stages != 1 &&
+                    c->side_a != nullptr && c->side_b != nullptr;
   if (!pipe) {
     const int rc = join_deferred(c);
     if (rc != IWP_OK) return rc;
@@ -500,7 +502,8 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     stage_mark_at(c, 4);
     // The reduction needs the leader's list only: write that one here and the other workers' lists on
     // the side stream, beside the reduction; they are joined at the end of the step.
-    const bool split = spec && W > 1 && ls.n == 1 && c->side != nullptr;  // (a union needs every chosen node's list here)
+    // (a union needs every chosen node's list here, a sharded step every list)
+    const bool split = spec && W > 1 && ls.n == 1 && !c->select_only && c->side != nullptr;
     auto write = [&](cudaStream_t st, WorkerSel ws) {
       dim3 grid(n_chunks, static_cast<unsigned>(sel_count(ws, W)));
       k_write<VEC><<<grid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur,
@@ -526,6 +529,10 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   }
   stage_mark_at(c, 5);
   if (fork_small && !cuda_ok(cudaStreamWaitEvent(s, c->ev_join, 0))) return IWP_ERR_CUDA;
+  if (c->select_only) {  // the reduction is the caller's (iwp_shard_gather / iwp_shard_apply)
+    stage_mark_at(c, 6);
+    return IWP_OK;
+  }
   if (ls.n > 1) {
     // union of the chosen nodes' lists: the zero mask is all clear here (applied and cleared by the streaming
     // pass, or flushed at the start of a multi-pass step) and serves to give every element one owner
@@ -921,6 +928,42 @@ int iwp_step(iwp_ctx* c, const float* grads, const float* weights, float* update
                             : run_step<false>(c, grads, weights, update, leader));
   if (rc != IWP_OK) return rc;
   c->leader = leader;
+  c->t += 1;
+  return IWP_OK;
+}
+
+int iwp_shard_select(iwp_ctx* c, const float* grads, const float* weights, float* update) {
+  if (!c || !grads || !weights || !update || c->threshold_mode) return IWP_ERR_INVALID;
+  const bool vec = !c->force_scalar && (c->plan.N % 4 == 0) && aligned16(grads) && aligned16(weights) &&
+                   aligned16(update) && aligned16(c->acc);
+  c->select_only = true;  // worker 0 plays the leader's part in the streaming pass; nothing is reduced
+  const int rc = vec ? run_step<true>(c, grads, weights, update, 0) : run_step<false>(c, grads, weights, update, 0);
+  c->select_only = false;
+  if (rc != IWP_OK) return rc;
+  c->leader = -1;
+  return IWP_OK;
+}
+
+int iwp_shard_gather(iwp_ctx* c, const uint32_t* idx, int64_t n, float* vals) {
+  if (!c || !idx || !vals || n < 0 || c->threshold_mode) return IWP_ERR_INVALID;
+  if (const int rc = flush_pending_zero(c)) return rc;
+  if (n == 0) return IWP_OK;
+  const uint64_t total = static_cast<uint64_t>(n) * static_cast<uint64_t>(c->plan.W);
+  const unsigned blocks = static_cast<unsigned>(std::min<uint64_t>((total + THREADS - 1) / THREADS, 148ull * 32));
+  k_shard_gather<<<blocks, THREADS, 0, c->stream>>>(idx, c->acc, vals, c->plan.N, static_cast<uint64_t>(n), c->plan.W);
+  IWP_LAUNCH_CHECK(c);
+  return IWP_OK;
+}
+
+int iwp_shard_apply(iwp_ctx* c, const uint32_t* idx, int64_t n, const float* vals_all, int32_t W_total, float* update) {
+  if (!c || !idx || !vals_all || !update || n < 0 || W_total < c->plan.W || c->threshold_mode) return IWP_ERR_INVALID;
+  if (const int rc = flush_pending_zero(c)) return rc;
+  if (n > 0) {
+    const unsigned blocks = static_cast<unsigned>((static_cast<uint64_t>(n) + THREADS - 1) / THREADS);
+    k_shard_apply<<<blocks, THREADS, 0, c->stream>>>(idx, vals_all, c->acc, update, c->plan.N, static_cast<uint64_t>(n),
+                                                    W_total, c->plan.W);
+    IWP_LAUNCH_CHECK(c);
+  }
   c->t += 1;
   return IWP_OK;
 }

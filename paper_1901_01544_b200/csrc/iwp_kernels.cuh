@@ -1236,6 +1236,34 @@ __global__ void __launch_bounds__(THREADS)
   update[i] = __fadd_rn(0.0f, s);
 }
 
+// Workers spread over several contexts (one per GPU): step (e) for this context's workers at an index
+// set that came from elsewhere, vals[w][j] = acc[w][idx[j]]; grid-stride over (worker, entry).
+__global__ void __launch_bounds__(THREADS)
+    k_shard_gather(const uint32_t* __restrict__ idx, const float* __restrict__ acc, float* __restrict__ vals, uint64_t N,
+                   uint64_t n, int W) {
+  const uint64_t total = n * static_cast<uint64_t>(W);
+  for (uint64_t q = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x; q < total;
+       q += static_cast<uint64_t>(gridDim.x) * THREADS) {
+    const uint64_t w = q / n, j = q % n;
+    vals[q] = acc[w * N + idx[j]];
+  }
+}
+
+// ... and steps (f), (g): the values of ALL workers of the job at the index set, in global worker order
+// (vals_all[w][j], w < W_total), are summed in that order into the (already zeroed) update, and this
+// context's own residuals are zeroed there.  One thread per entry.
+__global__ void __launch_bounds__(THREADS)
+    k_shard_apply(const uint32_t* __restrict__ idx, const float* __restrict__ vals_all, float* __restrict__ acc,
+                  float* __restrict__ update, uint64_t N, uint64_t n, int W_total, int W_local) {
+  const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (j >= n) return;
+  const uint64_t i = idx[j];
+  float s = vals_all[j];
+  for (int w = 1; w < W_total; ++w) s = __fadd_rn(s, vals_all[static_cast<uint64_t>(w) * n + j]);
+  update[i] = __fadd_rn(0.0f, s);
+  for (int w = 0; w < W_local; ++w) acc[static_cast<uint64_t>(w) * N + i] = 0.0f;
+}
+
 // A worker's select that is left running on a side stream past the end of the step may still need
 // the weights if its pair has to fall back to the multi-pass path, and the caller is free to change
 // them once the step's stream work is done.  So the weights of every layer in which a worker other

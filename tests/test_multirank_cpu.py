@@ -55,3 +55,105 @@ def test_single_process_needs_no_process_group():
     assert bench.max_over_ranks(12.5, None, torch.device("cpu")) == 12.5
     assert bench.whole_job_value(10, 1, 5.0) == 2000.0
     assert bench.step_bytes(8, 60965224, 952583) == 12 * 8 * 60965224 + 8 * 60965224 + 16 * 8 * 952583 + 8 * 952583
+
+
+# ---------------------------------------------------------------- workers spread over ranks (ShardedPruner)
+
+
+class _NumpyEngine:
+    """Test double for the per-rank CUDA engine: the four calls ShardedPruner makes, on CPU tensors, in plain
+    numpy.  It lets the orchestration (who owns the chosen worker, what is broadcast, in which order the
+    gathered values are summed) run as real gloo ranks; the CUDA engine itself is checked on the GPU."""
+
+    def __init__(self, layer_sizes, W, ratio, eps):
+        import math
+
+        import numpy as np
+
+        self.np = np
+        self.n = list(layer_sizes)
+        self.W, self.N = W, sum(self.n)
+        self.k = [min(n, max(1, math.ceil(n / ratio))) for n in self.n]
+        self.K = sum(self.k)
+        self.eps = np.float32(eps)
+        self.acc = np.zeros((W, self.N), np.float32)
+        self.lists = None
+
+    def shard_select(self, grads, weights, update):
+        np = self.np
+        self.acc = (self.acc + grads.numpy().reshape(self.W, self.N)).astype(np.float32)
+        update.zero_()
+        den = (np.abs(weights.numpy()) + self.eps).astype(np.float32)
+        self.lists = []
+        for w in range(self.W):
+            key = (np.abs(self.acc[w]) / den).astype(np.float32).view(np.uint32).astype(np.int64)
+            out, o = [], 0
+            for n, k in zip(self.n, self.k):
+                order = np.lexsort((np.arange(n), -key[o:o + n]))  # importance descending, index ascending
+                out.append(np.sort(order[:k]) + o)
+                o += n
+            self.lists.append(np.concatenate(out))
+
+    def selection(self, w):
+        idx = self.lists[w]
+        return torch.from_numpy(idx.astype(self.np.int32)), torch.from_numpy(self.acc[w, idx].copy())
+
+    def shard_gather(self, idx):
+        return torch.from_numpy(self.np.ascontiguousarray(self.acc[:, idx.numpy()]))
+
+    def shard_apply(self, idx, vals_all, update):
+        np = self.np
+        v = vals_all.numpy()
+        s = v[0].copy()
+        for w in range(1, v.shape[0]):
+            s = (s + v[w]).astype(np.float32)
+        update[idx.long()] = torch.from_numpy((np.float32(0) + s).astype(np.float32))
+        self.acc[:, idx.numpy()] = 0
+
+    def close(self):
+        pass
+
+
+def _sharded_rank_main(rank: int, world: int, port: int, out):
+    import numpy as np
+
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import oracle
+    from paper_1901_01544_b200.binding import ShardedPruner
+
+    layers, W_total, ratio, eps, seed = [300, 17, 1000], 4, 8.0, 1e-8, 5
+    N, Wl = sum(layers), W_total // world
+    sp = ShardedPruner(layers, W_total, ratio, eps, seed, engine=_NumpyEngine(layers, Wl, ratio, eps))
+    orc = oracle.Oracle(layers, W_total, ratio, eps, seed)  # the whole job on one "node"
+    rng = np.random.default_rng(3)  # the same stream on every rank
+    weights = rng.standard_normal(N).astype(np.float32)
+    ok, owners = True, set()
+    for t in range(6):
+        grads = rng.standard_normal((W_total, N)).astype(np.float32)
+        want = orc.step(grads, weights)
+        upd = torch.full((N,), float("nan"))
+        sp.step(torch.from_numpy(grads[rank * Wl:(rank + 1) * Wl].copy()), torch.from_numpy(weights), upd)
+        ok = ok and sp.leader == orc.leader and np.array_equal(upd.numpy().view(np.uint32), want.view(np.uint32))
+        for w in range(Wl):
+            ok = ok and np.array_equal(sp.local.acc[w].view(np.uint32), orc.residual(rank * Wl + w).view(np.uint32))
+        owners.add(sp.leader // Wl)
+    out.put((rank, bool(ok), sorted(owners)))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_workers_spread_over_two_ranks_equal_one_node():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_sharded_rank_main, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(out.get(timeout=180) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert [g[1] for g in got] == [True, True]
+    assert got[0][2] == [0, 1]  # the chosen worker lived on either rank at some step
