@@ -335,8 +335,9 @@ def run_ours(args):
         pr.check()
         stage_ms = {k: pr.stat(f"time_{k}_ns") / 1e6 / stage_steps for k in ("small", "sample", "accumulate", "select",
                                                                               "compact", "gather")}
-        stage_ms["note"] = (f"separate pass of {stage_steps} steps with an event at every stage boundary; 'small' runs on a "
-                            "side stream beside the other stages, 'gather' includes waiting for the non-leader lists")
+        stage_ms["note"] = (f"separate pass of {stage_steps} steps in the serial schedule (no overlap of the selects with the "
+                            "streaming pass) with an event at every stage boundary; 'small' runs on a side stream beside "
+                            "the other stages, 'gather' includes waiting for the non-leader lists")
     pr.set_option("time_stages", 0)
     ms_total = max_over_ranks(ms_total, dist, dev)
     ms_per_step = ms_total / args.steps
