@@ -75,17 +75,20 @@ CASES = {
 }
 
 
+# overlap: the schedule the library would only pick by itself for larger workloads is forced on as well
+@pytest.mark.parametrize("overlap", [0, 1])
 @pytest.mark.parametrize("name", sorted(CASES))
-def test_random_values(name):
+def test_random_values(name, overlap):
     sizes, W, ratio = CASES[name]
     N = sum(sizes)
     weights = _weights(N, 100 + N % 97)
     run_parity(sizes, W, ratio, 1e-8, seed=7, steps=3, weights=weights,
-               grads_fn=lambda t: _randn((W, N), 1000 * t + 3, 1e-3))
+               grads_fn=lambda t: _randn((W, N), 1000 * t + 3, 1e-3), options={"overlap": overlap})
 
 
+@pytest.mark.parametrize("overlap", [0, 1])
 @pytest.mark.parametrize("name", ["mixed_many", "tiled_unaligned_offsets_vector_path", "one_tiled_layer"])
-def test_many_ties(name):
+def test_many_ties(name, overlap):
     # coarse values: importances collide all the time, exact cancellations to +0 occur
     sizes, W, ratio = CASES[name]
     N = sum(sizes)
@@ -98,12 +101,14 @@ def test_many_ties(name):
         gg.manual_seed(50 + t)
         return torch.randint(-4, 5, (W, N), generator=gg, device=DEV).float() / 8.0
 
-    run_parity(sizes, W, ratio, 1e-8, seed=1, steps=4, weights=weights, grads_fn=grads)
+    run_parity(sizes, W, ratio, 1e-8, seed=1, steps=4, weights=weights, grads_fn=grads, options={"overlap": overlap},
+               state_every=1 + overlap)
 
 
+@pytest.mark.parametrize("overlap", [0, 1])
 @pytest.mark.parametrize("kind", ["all_equal", "all_zero", "two_values", "zero_weights", "tiny_values", "tiny_eps",
                                   "huge_values"])
-def test_degenerate_layers(kind):
+def test_degenerate_layers(kind, overlap):
     sizes, W, ratio = [100000, 5000, 37], 3, 32.0
     N = sum(sizes)
     eps = 1e-8
@@ -132,7 +137,8 @@ def test_degenerate_layers(kind):
     else:
         weights = torch.zeros(N, device=DEV)
         grads = lambda t: _randn((W, N), 77 + t, 1e-3)
-    run_parity(sizes, W, ratio, eps, seed=2, steps=2, weights=weights, grads_fn=grads)
+    run_parity(sizes, W, ratio, eps, seed=2, steps=3, weights=weights, grads_fn=grads, options={"overlap": overlap},
+               state_every=1 + overlap)
 
 
 def test_forced_scalar_path_and_leader_override():
