@@ -1,0 +1,200 @@
+// Steps (e)-(g) of the pruning step: the reduction at the chosen node's index set in its variants (gather,
+// side values, union of several chosen nodes, workers spread over contexts), the zero-mask flush, the copies
+// kept for late selects and the byte mask accessor.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "iwp_device.cuh"
+#include "iwp_stream.cuh"
+
+namespace iwp {
+
+// ---------------------------------------------------------------------------------------
+// steps (e)-(g): gather every worker's residual at the leader's indices, sum in ascending
+// worker order, scatter into the (already zeroed) dense update, zero what was sent.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(THREADS)
+    k_gather_sum_scatter(const uint32_t* __restrict__ leader_idx, float* __restrict__ acc, float* __restrict__ update,
+                         uint64_t N, uint64_t K, int W) {
+  const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (j >= K) return;
+  const uint64_t i = leader_idx[j];
+  float* p = acc + i;
+  float s = 0.0f;
+  for (int w0 = 0; w0 < W; w0 += 8) {  // loads of a group are independent; the sum keeps worker order
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = (w0 + u < W) ? p[static_cast<uint64_t>(w0 + u) * N] : 0.0f;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
+    }
+  }
+  for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
+  update[i] = __fadd_rn(0.0f, s);
+}
+
+// Steps (e)-(g) with several chosen nodes (Algorithm 1: Mask = OR Mask_ri): the index set is the union
+// of the chosen nodes' lists.  One thread per list entry of every chosen node; the first thread to mark
+// an element in the (all-zero) bit mask owns it - gathers the W residuals, sums them in ascending
+// worker order, scatters the sum and zeroes the residuals - and every later entry with the same element
+// returns at once, so nothing is read after it was zeroed.  The marks stay set (the element is +0 now
+// whether or not the next streaming pass treats it so).
+__global__ void __launch_bounds__(THREADS)
+    k_union_sum_scatter(const uint32_t* __restrict__ sel_idx, float* __restrict__ acc, float* __restrict__ update,
+                        uint32_t* __restrict__ seen, uint64_t N, uint64_t K, int W, LeaderSet ls) {
+  const uint64_t q = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (q >= static_cast<uint64_t>(ls.n) * K) return;
+  const int j = static_cast<int>(q / K);
+  int r = ls.r[0];
+#pragma unroll
+  for (int u = 1; u < MAX_LEADERS; ++u)
+    if (u == j) r = ls.r[u];
+  const uint64_t i = sel_idx[static_cast<uint64_t>(r) * K + q % K];
+  const uint32_t bit = zmask_bit(i);
+  if (atomicOr(&seen[zmask_word(i)], bit) & bit) return;
+  float* p = acc + i;
+  float s = 0.0f;
+  for (int w0 = 0; w0 < W; w0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = (w0 + u < W) ? p[static_cast<uint64_t>(w0 + u) * N] : 0.0f;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
+    }
+  }
+  for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
+  update[i] = __fadd_rn(0.0f, s);
+}
+
+// Workers spread over several contexts (one per GPU): step (e) for this context's workers at an index
+// set that came from elsewhere, vals[w][j] = acc[w][idx[j]]; grid-stride over (worker, entry).
+__global__ void __launch_bounds__(THREADS)
+    k_shard_gather(const uint32_t* __restrict__ idx, const float* __restrict__ acc, float* __restrict__ vals, uint64_t N,
+                   uint64_t n, int W) {
+  const uint64_t total = n * static_cast<uint64_t>(W);
+  for (uint64_t q = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x; q < total;
+       q += static_cast<uint64_t>(gridDim.x) * THREADS) {
+    const uint64_t w = q / n, j = q % n;
+    vals[q] = acc[w * N + idx[j]];
+  }
+}
+
+// ... and steps (f), (g): the values of ALL workers of the job at the index set, in global worker order
+// (vals_all[w][j], w < W_total), are summed in that order into the (already zeroed) update, and this
+// context's own residuals are zeroed there.  One thread per entry.
+__global__ void __launch_bounds__(THREADS)
+    k_shard_apply(const uint32_t* __restrict__ idx, const float* __restrict__ vals_all, float* __restrict__ acc,
+                  float* __restrict__ update, uint64_t N, uint64_t n, int W_total, int W_local) {
+  const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (j >= n) return;
+  const uint64_t i = idx[j];
+  float s = vals_all[j];
+  for (int w = 1; w < W_total; ++w) s = __fadd_rn(s, vals_all[static_cast<uint64_t>(w) * n + j]);
+  update[i] = __fadd_rn(0.0f, s);
+  for (int w = 0; w < W_local; ++w) acc[static_cast<uint64_t>(w) * N + i] = 0.0f;
+}
+
+// A worker's select that is left running on a side stream past the end of the step may still need
+// the weights if its pair has to fall back to the multi-pass path, and the caller is free to change
+// them once the step's stream work is done.  So the weights of every layer in which a worker other
+// than the leader failed its single-read check are copied here, on the step's own stream; that
+// select then reads the copy.  grid = chunks; nearly always every CTA returns at once.
+__global__ void __launch_bounds__(THREADS)
+    k_save_weights(const float* __restrict__ weights, float* __restrict__ saved, const Chunk* __restrict__ chunks,
+                   const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info, int W, int leader) {
+  const Chunk c = chunks[blockIdx.x];
+  const LayerDesc L = layers[c.layer];
+  bool failed = false;
+  for (int w = threadIdx.x; w < W; w += THREADS)
+    failed = failed || (w != leader && !pair_is_cand(info[static_cast<uint32_t>(L.large_index) * W + w], L.k));
+  if (!__syncthreads_or(failed)) return;
+  for (uint32_t i = threadIdx.x; i < c.len; i += THREADS) saved[c.a + i] = weights[c.a + i];
+}
+
+// Steps (e)-(g) on the single-read path.  For a list entry of the leader that came from a candidate
+// slot, every other worker's value at that slot position was written to the side buffer by the
+// streaming pass (the leader's own value is the candidate value): read the W values, sum them in
+// ascending worker order, scatter, and mark the element for zeroing by the next streaming pass.
+// Entries from the one-CTA path carry REF_NONE: gathered from the residuals, which are zeroed here
+// (no streaming pass visits them).  Entries from a pair that fell back to the multi-pass select
+// carry REF_LAZY: gathered from the residuals and marked like the first kind, because another
+// worker's multi-pass select may still be reading that layer's residuals on a side stream.
+__global__ void __launch_bounds__(THREADS)
+    k_sum_scatter(const uint32_t* __restrict__ leader_idx, const uint32_t* __restrict__ sel_slot,
+                  const float* __restrict__ side_val, const float* __restrict__ cand_val, float* __restrict__ acc,
+                  float* __restrict__ update, uint32_t* __restrict__ zmask, uint64_t N, uint64_t K, int W,
+                  int leader) {
+  const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (j >= K) return;
+  const uint64_t i = leader_idx[j];
+  const uint32_t ref = sel_slot[j];
+  float s = 0.0f;
+  if (ref < REF_LAZY) {
+    const uint64_t tile = ref / CAND_CAP, at = ref % CAND_CAP;
+    const uint64_t q0 = tile * W * CAND_CAP + at;
+    for (int w0 = 0; w0 < W; w0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int w = w0 + u;
+        const uint64_t q = q0 + static_cast<uint64_t>(w) * CAND_CAP;
+        v[u] = (w < W) ? (w == leader ? cand_val[q] : side_val[q]) : 0.0f;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
+      }
+    }
+    atomicOr(&zmask[zmask_word(i)], zmask_bit(i));  // the next streaming pass zeroes all W residuals
+  } else {
+    float* p = acc + i;
+    for (int w0 = 0; w0 < W; w0 += 8) {
+      float v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) v[u] = (w0 + u < W) ? p[static_cast<uint64_t>(w0 + u) * N] : 0.0f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
+      }
+    }
+    if (ref == REF_LAZY) {
+      atomicOr(&zmask[zmask_word(i)], zmask_bit(i));
+    } else {
+      for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
+    }
+  }
+  update[i] = __fadd_rn(0.0f, s);
+}
+
+// Applies a pending zero mask right away (accessors, reset, and the multi-pass path need the
+// residuals themselves up to date).  One thread per mask word; the mask is cleared.
+__global__ void __launch_bounds__(THREADS)
+    k_flush_zmask(uint32_t* __restrict__ zmask, float* __restrict__ acc, uint64_t n_words, uint64_t N, int W) {
+  const uint64_t wd = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (wd >= n_words) return;
+  uint32_t bits = zmask[wd];
+  if (bits == 0u) return;
+  zmask[wd] = 0u;
+  const uint64_t field0 = wd * 2;  // (segment, lane) index of the low half
+  for (; bits; bits &= bits - 1) {
+    const uint32_t b = __ffs(bits) - 1;
+    const uint64_t field = field0 + (b >> 4);
+    const uint64_t seg = field >> 5, lane = field & 31;
+    const uint32_t fb = b & 15u;
+    const uint64_t i = seg * 512 + (fb >> 2) * 128 + lane * 4 + (fb & 3u);
+    if (i < N) {
+      for (int w = 0; w < W; ++w) acc[static_cast<uint64_t>(w) * N + i] = 0.0f;
+    }
+  }
+}
+
+// byte mask of the index set (Algorithm 1's encode_uint8(Mask)); dst is zeroed by the caller
+__global__ void __launch_bounds__(THREADS) k_mask_scatter(const uint32_t* __restrict__ leader_idx, uint8_t* __restrict__ dst, uint64_t K) {
+  const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (j < K) dst[leader_idx[j]] = 1;
+}
+
+}  // namespace iwp

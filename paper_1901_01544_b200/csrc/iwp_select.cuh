@@ -1,0 +1,532 @@
+// Steps (c)+(d) of the pruning step: exact radix select over the fp32 importance pattern (histogram passes,
+// digit decisions), ordered compaction into the (index, value) lists, and the one-CTA path of small layers.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "iwp_device.cuh"
+#include "iwp_stream.cuh"
+
+namespace iwp {
+
+// The candidates of (chunk, worker): warp q takes the chunk's tiles 16 q .. 16 q + 15 (consecutive,
+// so that warp order is index order), four tiles at a time; each lane reads entries 4 lane .. 4 lane + 3
+// of a slot with one 128-bit load (a slot rarely holds more than 128 entries; a tail loop covers the
+// rest) and all loads of a batch are issued before any is used.  `f(key)` sees every stored candidate,
+// and in addition some keys 0 (padding, slots shorter than 128 entries), which `f` must ignore - every
+// use below does so by construction, because a candidate's key and first digit are never 0.
+constexpr uint32_t TILES_PER_WARP = CHUNK_TILES / WARPS;
+
+template <typename F>
+__device__ __forceinline__ void for_each_candidate(const Chunk& c, int w, int W, const uint32_t* __restrict__ cand_cnt,
+                                                   const uint32_t* __restrict__ cand_key, F&& f) {
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t t_begin = warp * TILES_PER_WARP;
+  const uint32_t t_end = min(c.n_tiles, t_begin + TILES_PER_WARP);
+  for (uint32_t tb = t_begin; tb < t_end; tb += 4) {
+    uint32_t cnt[4];
+    uint4 k4[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      cnt[q] = (tb + q < t_end) ? min(cand_cnt[static_cast<uint64_t>(c.first_tile + tb + q) * W + w], CAND_CAP) : 0u;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (static_cast<uint64_t>(c.first_tile + tb + q) * W + w) * CAND_CAP);
+      k4[q] = (lane * 4 < cnt[q]) ? kp[lane] : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {  // groups past the count were not loaded (zeros); the last group is zero-padded
+      f(k4[q].x);
+      f(k4[q].y);
+      f(k4[q].z);
+      f(k4[q].w);
+      if (cnt[q] > 128) {
+        const uint4* kp = reinterpret_cast<const uint4*>(cand_key + (static_cast<uint64_t>(c.first_tile + tb + q) * W + w) * CAND_CAP);
+        for (uint32_t j0 = 128; j0 < cnt[q]; j0 += 128) {
+          const uint32_t j = j0 + lane * 4;
+          if (j < cnt[q]) {
+            const uint4 k = kp[j >> 2];
+            f(k.x);
+            f(k.y);
+            f(k.z);
+            f(k.w);
+          }
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// tiled path, step (c): exact radix select of the k-th largest key per (worker, layer).
+// Every kernel below serves both kinds of pair: those whose candidates hold the top-k read the
+// candidate slots, the others read the residual and the weights again (multi-pass exact path).
+// ---------------------------------------------------------------------------------------
+
+// One histogram pass over a chunk: keys that match the prefix found so far are counted by
+// their next digit.  grid = (chunks, W).  In the last pass every CTA additionally leaves, per chunk,
+// the number of keys above the prefix and the suffix sums of its low-digit histogram; with the
+// threshold known, the compaction derives every chunk's (#keys > T, #keys == T) from those without
+// another look at the keys (chunk_sfx == nullptr: skipped, a counting kernel runs instead).
+template <bool VEC>
+__global__ void __launch_bounds__(THREADS)
+    k_hist(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
+           const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
+           const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt,
+           const uint2* __restrict__ state,
+           uint32_t* __restrict__ hist, uint32_t* __restrict__ chunk_sfx, uint2* __restrict__ chunk_cnt, float eps,
+           uint64_t N, int W, int pass, uint32_t n_chunks, WorkerSel ws) {
+  __shared__ uint32_t sh[NBINS];
+  __shared__ uint32_t sh_warp[WARPS];
+  __shared__ uint32_t sh_above;
+  const Chunk c = chunks[blockIdx.x];
+  const int w = sel_worker(ws, static_cast<int>(blockIdx.y));
+  const LayerDesc L = layers[c.layer];
+  const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
+  const int shift = pass_shift(pass), nb = pass_bins(pass);
+  const int prev_shift = pass == 0 ? 31 : pass_shift(pass - 1);
+  const uint2 st_in = pass == 0 ? make_uint2(0u, L.k) : state[pair];
+  const uint32_t want = pass == 0 ? 0u : (st_in.x >> prev_shift);
+  const bool last_pass = pass == N_PASSES - 1;
+  for (int b = threadIdx.x; b < nb; b += THREADS) sh[b] = 0;
+  if (threadIdx.x == 0) sh_above = 0;
+  __syncthreads();
+  uint32_t above = 0;  // keys whose higher digits already exceed the prefix (needed in the last pass only)
+  const PairInfo pi = info[pair];
+  if (pair_is_cand(pi, L.k) && pass == 0) {
+    // Every candidate is at or just above the guess, so almost all of them fall into the guess's own
+    // first-digit bin or the next two: count those in registers (one shared-memory atomic per lane
+    // would serialise on three addresses) and leave only the rest to atomics.
+    const uint32_t g0 = pi.guess >> shift;
+    uint32_t c0 = 0, c1 = 0, c2 = 0;
+    for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
+      const uint32_t d = (key >> shift) - g0;
+      c0 += d == 0u ? 1u : 0u;
+      c1 += d == 1u ? 1u : 0u;
+      c2 += d == 2u ? 1u : 0u;
+      if (d > 2u && key != 0u) atomicAdd(&sh[(key >> shift) & (nb - 1)], 1u);
+    });
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      c0 += __shfl_xor_sync(0xffffffffu, c0, d);
+      c1 += __shfl_xor_sync(0xffffffffu, c1, d);
+      c2 += __shfl_xor_sync(0xffffffffu, c2, d);
+    }
+    if ((threadIdx.x & 31) == 0) {
+      if (c0) atomicAdd(&sh[g0 & (nb - 1)], c0);
+      if (c1) atomicAdd(&sh[(g0 + 1) & (nb - 1)], c1);
+      if (c2) atomicAdd(&sh[(g0 + 2) & (nb - 1)], c2);
+    }
+  } else if (pair_is_cand(pi, L.k)) {
+    for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
+      const uint32_t hi_part = key >> prev_shift;
+      if (hi_part == want) atomicAdd(&sh[(key >> shift) & (nb - 1)], 1u);
+      above += hi_part > want ? 1u : 0u;
+    });
+  } else {
+    const uint64_t lo = c.a, hi = lo + c.len;
+    const uint64_t s0 = lo & ~3ull;
+    const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+    const float* a = acc + static_cast<uint64_t>(w) * N;
+    for (uint32_t it = 0; it < n_iter; ++it) {
+      const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+      float av[4], wv[4];
+      load4<VEC>(a, e0, lo, hi, av);
+      load4<VEC>(weights, e0, lo, hi, wv);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint64_t e = e0 + q;
+        const uint32_t key = imp_key(av[q], wv[q], eps);
+        const bool in = e >= lo && e < hi;
+        const bool valid = in && (key >> prev_shift) == want;  // pass 0: bit 31 is 0 == want
+        hist_add_aggregated(sh, valid, (key >> shift) & (nb - 1));
+        above += (in && (key >> prev_shift) > want) ? 1u : 0u;
+      }
+    }
+  }
+  if (last_pass && chunk_sfx != nullptr) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) above += __shfl_xor_sync(0xffffffffu, above, d);
+    if ((threadIdx.x & 31) == 0 && above) atomicAdd(&sh_above, above);
+  }
+  __syncthreads();
+  uint32_t* gh = hist + static_cast<uint64_t>(pair) * NBINS;
+  for (int b = threadIdx.x; b < nb; b += THREADS) {
+    const uint32_t v = sh[b];
+    if (v) atomicAdd(&gh[b], v);
+  }
+  if (last_pass && chunk_sfx != nullptr) {  // suffix sums S[b] = sum of this chunk's bins >= b, and the count above the prefix
+    static_assert(pass_bins(N_PASSES - 1) == THREADS * 4, "four bins per thread in the last pass");
+    const uint32_t h0 = sh[threadIdx.x * 4], h1 = sh[threadIdx.x * 4 + 1], h2 = sh[threadIdx.x * 4 + 2],
+                   h3 = sh[threadIdx.x * 4 + 3];
+    uint32_t total;
+    const uint32_t before = block_excl_scan(h0 + h1 + h2 + h3, sh_warp, total);
+    const uint32_t s0 = total - before;
+    uint4 sfx = make_uint4(s0, s0 - h0, s0 - h0 - h1, s0 - h0 - h1 - h2);
+    uint32_t* dst = chunk_sfx + (static_cast<uint64_t>(w) * n_chunks + blockIdx.x) * pass_bins(N_PASSES - 1);
+    reinterpret_cast<uint4*>(dst)[threadIdx.x] = sfx;
+    if (threadIdx.x == 0) chunk_cnt[static_cast<uint64_t>(w) * n_chunks + blockIdx.x] = make_uint2(sh_above, 0u);
+  }
+}
+
+// Digit decision for (worker, layer) pairs of the tiled path; grid = (tiled layers, covered workers).
+// Reads the pair's histogram, clears it for the next pass, extends the key prefix.
+// After the last pass state = (threshold key T, number r of T-valued elements to keep).
+__global__ void __launch_bounds__(THREADS)
+    k_find_digit(uint2* __restrict__ state, uint32_t* __restrict__ hist, const LayerDesc* __restrict__ layers,
+                 const uint32_t* __restrict__ large_ids, int* __restrict__ status, int W, int pass,
+                 WorkerSel ws) {
+  __shared__ uint32_t sh[NBINS];
+  __shared__ uint32_t sh_scan[THREADS];
+  __shared__ uint32_t res[4];
+  const uint32_t pair = blockIdx.x * static_cast<uint32_t>(W) + static_cast<uint32_t>(sel_worker(ws, static_cast<int>(blockIdx.y)));
+  const int nb = pass_bins(pass), shift = pass_shift(pass);
+  uint32_t* gh = hist + static_cast<uint64_t>(pair) * NBINS;
+  for (int b = threadIdx.x; b < nb; b += THREADS) {
+    sh[b] = gh[b];
+    gh[b] = 0;
+  }
+  __syncthreads();
+  uint32_t prefix, krem;
+  if (pass == 0) {
+    prefix = 0;
+    krem = layers[large_ids[pair / W]].k;
+  } else {
+    const uint2 s = state[pair];
+    prefix = s.x;
+    krem = s.y;
+  }
+  find_digit(sh, nb, krem, sh_scan, res);
+  if (threadIdx.x == 0) {
+    if (res[2]) {
+      state[pair] = make_uint2(prefix | (res[0] << shift), res[1]);
+    } else {
+      atomicMin(status, STATUS_INTERNAL);
+      state[pair] = make_uint2(0xffffffffu, 0u);  // selects nothing
+    }
+  }
+}
+
+// Per chunk: how many keys are above the threshold and how many equal it.  grid = (chunks, W).
+template <bool VEC>
+__global__ void __launch_bounds__(THREADS)
+    k_count(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
+            const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
+            const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt, const uint2* __restrict__ state,
+            uint2* __restrict__ chunk_cnt, float eps, uint64_t N, int W, uint32_t n_chunks) {
+  __shared__ uint32_t sh_cnt[2];
+  const Chunk c = chunks[blockIdx.x];
+  const int w = blockIdx.y;
+  const LayerDesc L = layers[c.layer];
+  const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
+  const uint32_t T = state[pair].x;
+  if (threadIdx.x < 2) sh_cnt[threadIdx.x] = 0;
+  __syncthreads();
+  uint32_t gt = 0, eq = 0;
+  if (pair_is_cand(info[pair], L.k)) {
+    for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
+      gt += key > T ? 1u : 0u;
+      eq += key == T ? 1u : 0u;
+    });
+  } else {
+    const uint64_t lo = c.a, hi = lo + c.len;
+    const uint64_t s0 = lo & ~3ull;
+    const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+    const float* a = acc + static_cast<uint64_t>(w) * N;
+    for (uint32_t it = 0; it < n_iter; ++it) {
+      const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+      float av[4], wv[4];
+      load4<VEC>(a, e0, lo, hi, av);
+      load4<VEC>(weights, e0, lo, hi, wv);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint64_t e = e0 + q;
+        const bool in = e >= lo && e < hi;
+        const uint32_t key = imp_key(av[q], wv[q], eps);
+        gt += (in && key > T) ? 1u : 0u;
+        eq += (in && key == T) ? 1u : 0u;
+      }
+    }
+  }
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    gt += __shfl_xor_sync(0xffffffffu, gt, d);
+    eq += __shfl_xor_sync(0xffffffffu, eq, d);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    atomicAdd(&sh_cnt[0], gt);
+    atomicAdd(&sh_cnt[1], eq);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) chunk_cnt[static_cast<uint64_t>(w) * n_chunks + blockIdx.x] = make_uint2(sh_cnt[0], sh_cnt[1]);
+}
+
+// Step (d): stable compaction of the selected elements of a chunk into the worker's list.
+// An element is selected if key > T, or key == T and fewer than r T-valued elements of the
+// layer precede it; its list position is (#greater before it) + min(#equal before it, r).
+// grid = (chunks, W).
+template <bool VEC>
+__global__ void __launch_bounds__(THREADS)
+    k_write(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
+            const Tile* __restrict__ tiles, const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
+            const uint32_t* __restrict__ cand_key, const float* __restrict__ cand_val,
+            const uint16_t* __restrict__ cand_idx, const uint32_t* __restrict__ cand_cnt,
+            const uint2* __restrict__ state, const uint2* __restrict__ chunk_cnt, uint32_t* __restrict__ sel_idx,
+            float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot, const uint32_t* __restrict__ chunk_sfx,
+            int* __restrict__ status, float eps, uint64_t N, uint64_t K, int W, uint32_t n_chunks, int leader,
+            WorkerSel ws) {
+  __shared__ uint32_t sh_warp[WARPS];
+  __shared__ uint32_t sh_base[2];
+  const Chunk c = chunks[blockIdx.x];
+  const int w = sel_worker(ws, static_cast<int>(blockIdx.y));
+  const LayerDesc L = layers[c.layer];
+  const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
+  const uint2 st = state[pair];
+  const uint32_t T = st.x, r = st.y;
+  // counts of the layer's chunks in front of this one
+  if (threadIdx.x < 2) sh_base[threadIdx.x] = 0;
+  __syncthreads();
+  {
+    const uint2* cc = chunk_cnt + static_cast<uint64_t>(w) * n_chunks;
+    uint32_t g = 0, q = 0;
+    for (uint32_t j = c.first_chunk_of_layer + threadIdx.x; j < blockIdx.x; j += THREADS) {
+      const uint2 v = cc[j];
+      if (chunk_sfx == nullptr) {  // (#keys > T, #keys == T) of the chunk, counted by a kernel of its own
+        g += v.x;
+        q += v.y;
+      } else {  // left by the last histogram pass: keys above the prefix, suffix sums of the low digit
+        constexpr uint32_t LOW_BINS = pass_bins(N_PASSES - 1);
+        const uint32_t d = T & (LOW_BINS - 1);
+        const uint32_t* sfx = chunk_sfx + (static_cast<uint64_t>(w) * n_chunks + j) * LOW_BINS;
+        const uint32_t s_d = sfx[d], s_d1 = (d + 1 < LOW_BINS) ? sfx[d + 1] : 0u;
+        g += v.x + s_d1;
+        q += s_d - s_d1;
+      }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      g += __shfl_xor_sync(0xffffffffu, g, d);
+      q += __shfl_xor_sync(0xffffffffu, q, d);
+    }
+    if ((threadIdx.x & 31) == 0 && (g | q)) {
+      atomicAdd(&sh_base[0], g);
+      atomicAdd(&sh_base[1], q);
+    }
+  }
+  __syncthreads();
+  uint32_t run_gt = sh_base[0], run_eq = sh_base[1];
+  uint32_t* out_i = sel_idx + static_cast<uint64_t>(w) * K + L.koff;
+  float* out_v = sel_val + static_cast<uint64_t>(w) * K + L.koff;
+
+  const bool is_leader = w == leader;
+  if (pair_is_cand(info[pair], L.k)) {
+    // warp order is index order: count per warp, prefix over the warps, then every warp writes its
+    // tiles front to back, ranking the entries of a slot with one warp scan per 128 entries
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t my_gt = 0, my_eq = 0;
+    for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
+      my_gt += key > T ? 1u : 0u;
+      my_eq += key == T ? 1u : 0u;
+    });
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      my_gt += __shfl_xor_sync(0xffffffffu, my_gt, d);
+      my_eq += __shfl_xor_sync(0xffffffffu, my_eq, d);
+    }
+    __shared__ uint32_t sh_wg[WARPS], sh_we[WARPS];
+    if (lane == 0) {
+      sh_wg[warp] = my_gt;
+      sh_we[warp] = my_eq;
+    }
+    __syncthreads();
+    uint32_t g_before = run_gt, q_before = run_eq;
+    for (uint32_t q = 0; q < warp; ++q) {
+      g_before += sh_wg[q];
+      q_before += sh_we[q];
+    }
+    if ((my_gt | my_eq) == 0) return;  // nothing of this warp's tiles is selected
+    const uint32_t t_begin = warp * TILES_PER_WARP;
+    const uint32_t t_end = min(c.n_tiles, t_begin + TILES_PER_WARP);
+    // ranks the entries [j0, j0 + 128) of one slot with a warp scan and writes the selected ones
+    auto emit = [&](uint32_t tile, uint64_t tw, uint32_t cnt, uint32_t tile_base, uint32_t j0, uint4 k) {
+      const uint32_t j = j0 + lane * 4;
+      const uint32_t kk[4] = {k.x, k.y, k.z, k.w};
+      uint32_t fg = 0, fe = 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {  // padding keys are 0 and T is not: no range test needed
+        fg |= kk[u] > T ? (1u << u) : 0u;
+        fe |= kk[u] == T ? (1u << u) : 0u;
+      }
+      if (!__any_sync(0xffffffffu, (fg | fe) != 0u)) return;
+      // most entries of a slot are selected: fetch the group's values and indices as vectors now, so
+      // that they arrive while the ranks are computed
+      float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
+      uint2 i2 = make_uint2(0u, 0u);
+      if (fg | fe) {
+        v4 = reinterpret_cast<const float4*>(cand_val + tw * CAND_CAP)[j >> 2];
+        i2 = reinterpret_cast<const uint2*>(cand_idx + tw * CAND_CAP)[j >> 2];
+      }
+      const uint32_t packed = static_cast<uint32_t>(__popc(fg)) | (static_cast<uint32_t>(__popc(fe)) << 16);
+      const uint32_t incl = warp_incl_scan(packed);
+      const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
+      uint32_t gb = g_before + ((incl - packed) & 0xffffu), qb = q_before + ((incl - packed) >> 16);
+      if (fg | fe) {
+        const float vv[4] = {v4.x, v4.y, v4.z, v4.w};
+        const uint32_t ii[4] = {i2.x & 0xffffu, i2.x >> 16, i2.y & 0xffffu, i2.y >> 16};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const bool isg = (fg >> u) & 1u, ise = (fe >> u) & 1u;
+          if (isg || (ise && qb < r)) {
+            const uint32_t pos = gb + (qb < r ? qb : r);
+            if (pos < L.k) {
+              out_i[pos] = tile_base + ii[u];
+              out_v[pos] = vv[u];
+              if (is_leader) sel_slot[L.koff + pos] = tile * CAND_CAP + j + u;
+            } else {
+              atomicMin(status, STATUS_INTERNAL);
+            }
+          }
+          gb += isg ? 1u : 0u;
+          qb += ise ? 1u : 0u;
+        }
+      }
+      g_before += tot & 0xffffu;
+      q_before += tot >> 16;
+    };
+    for (uint32_t tb = t_begin; tb < t_end; tb += 4) {  // four tiles per batch, all their loads first
+      uint32_t cnt[4], tbase[4];
+      uint4 k4[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const bool in = tb + q < t_end;
+        const uint32_t tile = c.first_tile + tb + q;
+        cnt[q] = in ? min(cand_cnt[static_cast<uint64_t>(tile) * W + w], CAND_CAP) : 0u;
+        tbase[q] = in ? (tiles[tile].a & ~(TILE - 1u)) : 0u;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint64_t tw = static_cast<uint64_t>(c.first_tile + tb + q) * W + w;
+        k4[q] = (lane * 4 < cnt[q]) ? reinterpret_cast<const uint4*>(cand_key + tw * CAND_CAP)[lane]
+                                    : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (cnt[q] == 0) continue;
+        const uint32_t tile = c.first_tile + tb + q;
+        const uint64_t tw = static_cast<uint64_t>(tile) * W + w;
+        emit(tile, tw, cnt[q], tbase[q], 0, k4[q]);
+        for (uint32_t j0 = 128; j0 < cnt[q]; j0 += 128) {
+          const uint32_t j = j0 + lane * 4;
+          const uint4 k = (j < cnt[q]) ? reinterpret_cast<const uint4*>(cand_key + tw * CAND_CAP)[j >> 2]
+                                       : make_uint4(0u, 0u, 0u, 0u);
+          emit(tile, tw, cnt[q], tbase[q], j0, k);
+        }
+      }
+    }
+    return;
+  }
+
+  const uint64_t lo = c.a, hi = lo + c.len;
+  const uint64_t s0 = lo & ~3ull;
+  const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+  const float* a = acc + static_cast<uint64_t>(w) * N;
+  for (uint32_t it = 0; it < n_iter; ++it) {
+    const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+    float av[4], wv[4];
+    load4<VEC>(a, e0, lo, hi, av);
+    load4<VEC>(weights, e0, lo, hi, wv);
+    uint32_t fg = 0, fe = 0;  // per-element flags
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint64_t e = e0 + q;
+      const bool in = e >= lo && e < hi;
+      const uint32_t key = imp_key(av[q], wv[q], eps);
+      fg |= (in && key > T) ? (1u << q) : 0u;
+      fe |= (in && key == T) ? (1u << q) : 0u;
+    }
+    uint32_t total;
+    const uint32_t packed = static_cast<uint32_t>(__popc(fg)) | (static_cast<uint32_t>(__popc(fe)) << 16);
+    const uint32_t ex = block_excl_scan(packed, sh_warp, total);
+    uint32_t g_before = run_gt + (ex & 0xffffu), q_before = run_eq + (ex >> 16);
+    if (fg | fe) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const bool isg = (fg >> q) & 1u, ise = (fe >> q) & 1u;
+        if (isg || (ise && q_before < r)) {
+          const uint32_t pos = g_before + (q_before < r ? q_before : r);
+          if (pos < L.k) {
+            out_i[pos] = static_cast<uint32_t>(e0 + q);
+            out_v[pos] = av[q];
+            if (is_leader) sel_slot[L.koff + pos] = REF_LAZY;
+          } else {
+            atomicMin(status, STATUS_INTERNAL);
+          }
+        }
+        g_before += isg ? 1u : 0u;
+        q_before += ise ? 1u : 0u;
+      }
+    }
+    run_gt += total & 0xffffu;
+    run_eq += total >> 16;
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// one-CTA path: steps (a)-(d) of a whole (worker, layer) pair with n <= SMALL_MAX, keys in
+// shared memory.  grid = (small layers, W); dynamic shared memory = 4 * max n bytes.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(THREADS)
+    k_small(const float* __restrict__ grads, const float* __restrict__ weights, float* __restrict__ acc,
+            float* __restrict__ update, const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ small_ids,
+            uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot,
+            int* __restrict__ status, float eps, uint64_t N, uint64_t K, int leader, float momentum) {
+  extern __shared__ uint32_t keys[];
+  __shared__ uint32_t hist[NBINS];
+  __shared__ uint32_t sh_scan[THREADS];
+  __shared__ uint32_t sh_warp[WARPS];
+  __shared__ uint32_t res[4];
+  const LayerDesc L = layers[small_ids[blockIdx.x]];
+  const int w = blockIdx.y;
+  const int tid = threadIdx.x;
+  const uint32_t n = L.n;
+  float* a = acc + static_cast<uint64_t>(w) * N + L.off;
+  const float* g = grads + static_cast<uint64_t>(w) * N + L.off;
+  const float* wt = weights + L.off;
+  for (uint32_t i = tid; i < n; i += THREADS) {
+    const float v = accumulate(a[i], __ldcs(g + i), momentum);
+    a[i] = v;
+    keys[i] = imp_key(v, wt[i], eps);
+    if (w == 0) update[L.off + i] = 0.0f;
+  }
+  __syncthreads();
+  uint32_t T, r;
+  if (!smem_radix_select(keys, n, L.k, hist, sh_scan, res, T, r)) {
+    if (tid == 0) atomicMin(status, STATUS_INTERNAL);
+    return;
+  }
+  uint32_t* out_i = sel_idx + static_cast<uint64_t>(w) * K + L.koff;
+  float* out_v = sel_val + static_cast<uint64_t>(w) * K + L.koff;
+  uint32_t run_gt = 0, run_eq = 0;
+  for (uint32_t i0 = 0; i0 < n; i0 += THREADS) {
+    const uint32_t i = i0 + tid;
+    const uint32_t key = i < n ? keys[i] : 0u;
+    const bool isg = i < n && key > T, ise = i < n && key == T;
+    uint32_t total;
+    const uint32_t ex = block_excl_scan((isg ? 1u : 0u) | (ise ? 1u << 16 : 0u), sh_warp, total);
+    const uint32_t g_before = run_gt + (ex & 0xffffu), q_before = run_eq + (ex >> 16);
+    if (isg || (ise && q_before < r)) {
+      const uint32_t pos = g_before + (q_before < r ? q_before : r);
+      if (pos < L.k) {
+        out_i[pos] = L.off + i;
+        out_v[pos] = a[i];
+        if (w == leader) sel_slot[L.koff + pos] = REF_NONE;
+      } else {
+        atomicMin(status, STATUS_INTERNAL);
+      }
+    }
+    run_gt += total & 0xffffu;
+    run_eq += total >> 16;
+  }
+}
+
+}  // namespace iwp
