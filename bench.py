@@ -396,7 +396,8 @@ def run_ours(args):
     achieved = k1_bytes / (k1_ms * 1e-3) / 1e9 if k1_ms > 0 else 0.0
     roofline = {
         "bound": "hbm", "kernel": k1_name,
-        "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+        "achieved": achieved if k1_ms > 0 else None, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak if k1_ms > 0 else None, "peak_source": peak_src,
         "traffic": k1_traffic,
         "algorithmic_bytes_per_step_of_kernel": k1_bytes, "ms_per_step_of_kernel": k1_ms,
         "launches_per_step": k1_launches, "traffic_note": k1_note,
