@@ -33,6 +33,9 @@ def lib() -> C.CDLL:
         L.oracle_set_thresholds.argtypes = [vp, vp]
         L.oracle_set_n_leaders.argtypes = [vp, i32]
         L.oracle_set_random_select.argtypes = [vp, i32]
+        L.oracle_set_per_layer_leaders.argtypes = [vp, i32]
+        L.oracle_layer_leader.argtypes = [u64, u64, u64, i32]
+        L.oracle_layer_leader.restype = i32
         L.oracle_union_length.argtypes = [vp]
         L.oracle_union_length.restype = i64
         L.oracle_get_union.argtypes = [vp, vp]
@@ -95,6 +98,10 @@ def leaders(seed: int, t: int, W: int, n: int) -> List[int]:
     out = np.empty(n, dtype=np.int32)
     lib().oracle_leaders(seed, t, W, n, _p(out))
     return out.tolist()
+
+
+def layer_leader(seed: int, t: int, l: int, W: int) -> int:
+    return int(lib().oracle_layer_leader(seed, t, l, W))
 
 
 def keep_count(n: int, ratio: float) -> int:
@@ -190,6 +197,10 @@ class Oracle:
 
     def set_leader_override(self, leader: int):
         lib().oracle_set_leader_override(self._h, leader)
+
+    def set_per_layer_leaders(self, on: bool = True):
+        """Ratio mode: every layer draws its own chosen node each step."""
+        lib().oracle_set_per_layer_leaders(self._h, 1 if on else 0)
 
     def index_set(self) -> np.ndarray:
         """Ratio mode: the index set of the last step (union of the chosen nodes' lists), ascending."""

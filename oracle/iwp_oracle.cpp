@@ -23,7 +23,8 @@
 //     layer, k = ceil(n / ratio) clamped to [1, n]; ties keep the lower index.
 //   * one randomly chosen node per step supplies the index set (Section 3.2:
 //     "randomly choose a node and broadcast its important gradient index"); optionally several chosen
-//     nodes r_1..r_n, drawn without replacement, whose index sets are OR-ed (Algorithm 1: Mask = OR Mask_ri).
+//     nodes r_1..r_n, drawn without replacement, whose index sets are OR-ed (Algorithm 1: Mask = OR Mask_ri),
+//     or one chosen node per LAYER (Algorithm 1 draws the node inside its loop over layers).
 //   * Eq. 3's momentum acts on the locally kept residual: G <- m * G + grad (two roundings);
 //     m = 1, the default, is the plain accumulation of Section 3.2.
 //   * threshold mode is Algorithm 1 as printed: only the chosen node forms a mask, per layer
@@ -75,6 +76,7 @@ struct Oracle {
   float momentum = 1.0f;         // Eq. 3: the local residual enters the next step scaled by m
   bool threshold_mode = false;   // Algorithm 1 as printed: Mask <- importance > thr on the chosen node
   int32_t n_leaders = 1;         // how many chosen nodes' masks (index sets) are OR-ed
+  bool per_layer_leaders = false;  // ratio mode: every layer draws its own chosen node
   std::vector<uint32_t> union_idx; // ratio mode: the index set of the last step, ascending (one node: its list)
   bool random_select = false;    // Section 3.3: elements below the threshold go with P = importance / thr
   std::vector<int32_t> leaders;  // the chosen nodes of the last step, r_1 first
@@ -124,6 +126,12 @@ inline int32_t leader_of(uint64_t seed, uint64_t t, int32_t W) {
   uint64_t z = mix64(seed + (t + 1) * 0x9E3779B97F4A7C15ull);
   uint64_t hi = z >> 32;
   return static_cast<int32_t>((hi * static_cast<uint64_t>(W)) >> 32);
+}
+
+// the chosen node of layer l at step t when every layer draws its own (Algorithm 1 draws inside the layer loop)
+inline int32_t layer_leader_of(uint64_t seed, uint64_t t, uint64_t l, int32_t W) {
+  uint64_t z = mix64(seed + (t + 1) * 0x9E3779B97F4A7C15ull + (l + 1) * 0xA0761D6478BD642Full);
+  return static_cast<int32_t>(((z >> 32) * static_cast<uint64_t>(W)) >> 32);
 }
 
 // the chosen nodes r_1..r_n of step t: n distinct workers drawn without replacement; r_1 is leader_of()
@@ -353,6 +361,8 @@ void oracle_get_threshold_list(void* h, uint32_t* idx, float* val) {
   std::copy(o->thr_val.begin(), o->thr_val.end(), val);
 }
 void oracle_set_momentum(void* h, float m) { static_cast<Oracle*>(h)->momentum = m; }
+void oracle_set_per_layer_leaders(void* h, int32_t on) { static_cast<Oracle*>(h)->per_layer_leaders = on != 0; }
+int32_t oracle_layer_leader(uint64_t seed, uint64_t t, uint64_t l, int32_t W) { return layer_leader_of(seed, t, l, W); }
 void oracle_set_leader_override(void* h, int32_t leader) { static_cast<Oracle*>(h)->leader_override = leader; }
 int64_t oracle_total(void* h) { return static_cast<Oracle*>(h)->N; }
 int64_t oracle_total_keep(void* h) { return static_cast<Oracle*>(h)->K; }
@@ -515,6 +525,15 @@ void oracle_step(void* h, const float* grads, const float* weights, float* updat
     o->leaders = leaders_of(o->seed, static_cast<uint64_t>(o->t), W, o->n_leaders);
   }
   o->union_idx.clear();
+  if (o->per_layer_leaders && o->leader_override < 0 && o->n_leaders == 1) {
+    // every layer takes its own chosen node's segment of that node's list
+    for (int l = 0; l < L; ++l) {
+      const int32_t r = layer_leader_of(o->seed, static_cast<uint64_t>(o->t), static_cast<uint64_t>(l), W);
+      const uint32_t* list = &o->sel_idx[static_cast<size_t>(r) * K + o->koff[l]];
+      o->union_idx.insert(o->union_idx.end(), list, list + o->k[l]);
+    }
+    o->leaders.clear();
+  }
   for (int32_t r : o->leaders) {
     const uint32_t* list = &o->sel_idx[static_cast<size_t>(r) * K];
     std::vector<uint32_t> merged;

@@ -808,3 +808,69 @@ def test_ratio_mode_one_chosen_node_is_the_plain_path_and_all_nodes_cover_every_
         assert set(c.index_set().tolist()) == every
         for w in range(W):  # everything any worker selected has left every residual
             assert not c.residual(w)[sorted(every)].any()
+
+
+# ---------------------------------------------------------------- one chosen node per layer
+
+
+def _layer_leader_rows():
+    rows = []
+    for line in open(os.path.join(GOLD, "layer_leaders.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        head, body = line.split(":")
+        seed, W, L = (int(x) for x in head.split())
+        rows.append((seed, W, L, [[int(x) for x in step.split()] for step in body.split("|")]))
+    return rows
+
+
+@pytest.mark.parametrize("seed,W,L,expect", _layer_leader_rows())
+def test_layer_leader_vectors(seed, W, L, expect):
+    assert [[oracle.layer_leader(seed, t, l, W) for l in range(L)] for t in range(len(expect))] == expect
+
+
+def test_layer_leaders_are_uniform_and_differ_between_layers():
+    W = 8
+    draws = np.array([[oracle.layer_leader(3, t, l, W) for l in range(16)] for t in range(2000)])
+    assert draws.min() == 0 and draws.max() == W - 1
+    counts = np.bincount(draws.ravel(), minlength=W)
+    assert np.all(np.abs(counts - draws.size / W) < 5 * math.sqrt(draws.size / W))  # within five sigma of uniform
+    same = np.mean(draws[:, 0] == draws[:, 1])
+    assert abs(same - 1 / W) < 0.03  # neighbouring layers agree about as often as independent draws would
+
+
+def test_per_layer_leaders_equal_bruteforce():
+    layers, W, ratio, eps = [30, 6, 50, 12], 4, 8.0, F(1e-8)
+    N = sum(layers)
+    rng = np.random.default_rng(41)
+    weights = (rng.integers(-2, 3, N) * 0.5).astype(np.float32)
+    orc = oracle.Oracle(layers, W, ratio, eps, seed=17)
+    orc.set_per_layer_leaders()
+    k = [min(m, max(1, math.ceil(m / ratio))) for m in layers]
+    acc = np.zeros((W, N), np.float32)
+    used = set()
+    for t in range(5):
+        grads = (rng.integers(-4, 5, size=(W, N)) / 4.0).astype(np.float32)
+        acc = (acc + grads).astype(np.float32)
+        upd = orc.step(grads, weights)
+        S, o = [], 0
+        for l, (m, kk) in enumerate(zip(layers, k)):
+            r = oracle.layer_leader(17, t, l, W)
+            used.add(r)
+            imp = [bits(importance(acc[r, o + i], weights[o + i], eps)) for i in range(m)]
+            ranked = sorted(range(m), key=lambda i: (-imp[i], i))
+            S += sorted(o + i for i in ranked[:kk])
+            o += m
+        assert orc.index_set().tolist() == S and len(S) == sum(k)
+        want = np.zeros(N, np.float32)
+        for i in S:
+            s = acc[0, i]
+            for w in range(1, W):
+                s = F(s + acc[w, i])
+            want[i] = F(F(0) + s)
+            acc[:, i] = 0
+        assert np.array_equal(u32(upd), u32(want))
+        for w in range(W):
+            assert np.array_equal(u32(orc.residual(w)), u32(acc[w]))
+    assert len(used) > 1
