@@ -65,6 +65,12 @@ int64_t iwp_keep_count(int64_t n, double ratio);
  * with the splitmix64 finaliser as mix64.  Returns -1 if W < 1. */
 int32_t iwp_leader_at(uint64_t seed, uint64_t t, int32_t W);
 
+/* The chosen node of layer `layer` (0-based) at step t when every layer draws its own (option
+ * "per_layer_leaders"; Algorithm 1 draws the node inside its loop over layers):
+ * ((mix64(seed + (t+1)*0x9E3779B97F4A7C15 + (layer+1)*0xA0761D6478BD642F) >> 32) * W) >> 32.
+ * Host-only helper; -1 for W < 1 or layer < 0. */
+int32_t iwp_layer_leader_at(uint64_t seed, uint64_t t, int32_t layer, int32_t W);
+
 /* The n distinct chosen nodes r_1..r_n of step t (Algorithm 1: "choose random node r_1, r_2, ... r_n"), drawn
  * without replacement: u_j = ((mix64(seed + (t+1)*0x9E3779B97F4A7C15 + j*0xD1B54A32D192ED03) >> 32) * (W-j)) >> 32
  * picks the u_j-th of the workers not chosen yet; out_host[0] equals iwp_leader_at().  1 <= n <= min(W, 8).
@@ -237,6 +243,10 @@ int iwp_reset(iwp_ctx* ctx);
  *                      nodes; the listed values are r_1's.  Ratio mode: the union of the chosen nodes' own
  *                      top-k lists (every worker still lists its own top-k; iwp_get_mask() gives the union).
  *                      A forced leader ("leader_override") makes the step a one-node step
+ *   "per_layer_leaders" ratio-mode contexts only: 1 = every layer draws its own chosen node each step
+ *                      (iwp_layer_leader_at()); the index set is, layer by layer, that node's list segment.
+ *                      Ignored while a leader is forced or several chosen nodes are set.  0 (default) = one
+ *                      node per step for all layers
  *   "random_select"    threshold-mode contexts only: 1 = Section 3.3's random gradient selection: an
  *                      element whose importance does not exceed its layer's threshold is still sent iff
  *                      u < importance / thr (fp32 quotient), u = u24 * 2^-24 with

@@ -23,6 +23,7 @@ EXPORTS = [
     "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat", "iwp_select_static",
     "iwp_set_momentum", "iwp_create_threshold", "iwp_set_thresholds", "iwp_get_list_length", "iwp_leaders_at",
     "iwp_set_layerwise", "iwp_get_layer_thresholds", "iwp_shard_select", "iwp_shard_gather", "iwp_shard_apply",
+    "iwp_layer_leader_at",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -48,6 +49,7 @@ def lib() -> C.CDLL:
         L.iwp_keep_count.restype, L.iwp_keep_count.argtypes = i64, [i64, f64]
         L.iwp_leader_at.restype, L.iwp_leader_at.argtypes = i32, [u64, u64, i32]
         L.iwp_leaders_at.argtypes = [u64, u64, i32, i32, vp]
+        L.iwp_layer_leader_at.restype, L.iwp_layer_leader_at.argtypes = i32, [u64, u64, i32, i32]
         L.iwp_plan_sizes.argtypes = [vp, i32, i32, f64, vp]
         L.iwp_create.argtypes = [C.POINTER(vp), vp, i32, i32, f64, f32, u64]
         L.iwp_create_threshold.argtypes = [C.POINTER(vp), vp, i32, i32, f32, u64, i64]

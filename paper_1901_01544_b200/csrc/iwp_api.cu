@@ -68,6 +68,8 @@ struct iwp_ctx {
   bool thr_set = false;
   int32_t n_leaders = 1;          // chosen nodes whose masks are OR-ed
   LeaderSet last_chosen{};        // ratio mode: the chosen nodes of the last step
+  bool per_layer_leaders = false; // ratio mode: every layer draws its own chosen node
+  bool last_per_layer = false;    // the last step did so
   bool random_select = false;     // Section 3.3: P(update) = importance / threshold below the threshold
   uint32_t* d_thr = nullptr;      // [layer] fp32 patterns of the thresholds
   bool layerwise = false;         // Section 3.4: thresholds from each chosen node's per-layer statistics (Eq. 4)
@@ -338,8 +340,10 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     ls.r[0] = leader;
   }
   c->last_chosen = ls;
+  const bool per_layer = c->per_layer_leaders && c->leader_override < 0 && ls.n == 1 && !c->select_only;
+  c->last_per_layer = per_layer;
   // the overlapped schedule (not while every stage boundary is being timed)
-  const bool pipe = spec && W > 1 && ls.n == 1 && !c->select_only && c->overlap == 1 && c->time_stages != 1 &&
+  const bool pipe = spec && W > 1 && ls.n == 1 && !per_layer && !c->select_only && c->overlap == 1 && c->time_stages != 1 &&
                     c->side_a != nullptr && c->side_b != nullptr;
   if (!pipe) {
     const int rc = join_deferred(c);
@@ -503,7 +507,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     // The reduction needs the leader's list only: write that one here and the other workers' lists on
     // the side stream, beside the reduction; they are joined at the end of the step.
     // (a union needs every chosen node's list here, a sharded step every list)
-    const bool split = spec && W > 1 && ls.n == 1 && !c->select_only && c->side != nullptr;
+    const bool split = spec && W > 1 && ls.n == 1 && !per_layer && !c->select_only && c->side != nullptr;
     auto write = [&](cudaStream_t st, WorkerSel ws) {
       dim3 grid(n_chunks, static_cast<unsigned>(sel_count(ws, W)));
       k_write<VEC><<<grid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur,
@@ -533,7 +537,11 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     stage_mark_at(c, 6);
     return IWP_OK;
   }
-  if (ls.n > 1) {
+  if (per_layer) {
+    k_layer_leader_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx, c->d_layers, static_cast<uint32_t>(p.layers.size()),
+                                                           c->acc, update, nullptr, N, K, W, c->seed,
+                                                           static_cast<uint64_t>(c->t));
+  } else if (ls.n > 1) {
     // union of the chosen nodes' lists: the zero mask is all clear here (applied and cleared by the streaming
     // pass, or flushed at the start of a multi-pass step) and serves to give every element one owner
     const uint64_t entries = static_cast<uint64_t>(ls.n) * K;
@@ -574,6 +582,11 @@ const char* iwp_strerror(int status) {
 int64_t iwp_keep_count(int64_t n, double ratio) { return keep_count(n, ratio); }
 
 int32_t iwp_leader_at(uint64_t seed, uint64_t t, int32_t W) { return leader_at(seed, t, W); }
+
+int32_t iwp_layer_leader_at(uint64_t seed, uint64_t t, int32_t layer, int32_t W) {
+  if (W < 1 || layer < 0) return -1;
+  return layer_leader_at(seed, t, static_cast<uint64_t>(layer), W);
+}
 
 int iwp_leaders_at(uint64_t seed, uint64_t t, int32_t W, int32_t n, int32_t* out) {
   if (!out || W < 1 || n < 1 || n > W || n > MAX_LEADERS) return IWP_ERR_INVALID;
@@ -1121,6 +1134,14 @@ int iwp_get_mask(iwp_ctx* c, uint8_t* dst) {
     return IWP_OK;
   }
   const unsigned blocks = static_cast<unsigned>((K + THREADS - 1) / THREADS);
+  if (c->last_per_layer) {  // every layer's segment from its own chosen node's list
+    k_layer_leader_sum_scatter<<<blocks, THREADS, 0, c->stream>>>(c->sel_idx, c->d_layers,
+                                                                  static_cast<uint32_t>(c->plan.layers.size()), nullptr,
+                                                                  nullptr, dst, N, K, c->plan.W, c->seed,
+                                                                  static_cast<uint64_t>(c->t - 1));
+    if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+    return IWP_OK;
+  }
   for (int j = 0; j < c->last_chosen.n; ++j) {  // the index set is the union of the chosen nodes' lists
     k_mask_scatter<<<blocks, THREADS, 0, c->stream>>>(c->sel_idx + static_cast<uint64_t>(c->last_chosen.r[j]) * K, dst, K);
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
@@ -1178,6 +1199,11 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
   if (!std::strcmp(key, "n_leaders")) {
     if (v < 1 || v > MAX_LEADERS || v > c->plan.W) return IWP_ERR_INVALID;
     c->n_leaders = static_cast<int32_t>(v);
+    return IWP_OK;
+  }
+  if (!std::strcmp(key, "per_layer_leaders")) {
+    if (c->threshold_mode || (v != 0 && v != 1)) return IWP_ERR_INVALID;
+    c->per_layer_leaders = v != 0;
     return IWP_OK;
   }
   if (!std::strcmp(key, "overlap")) {

@@ -103,6 +103,20 @@ inline int32_t leader_at(uint64_t seed, uint64_t t, int32_t W) {
   return static_cast<int32_t>(((z >> 32) * static_cast<uint64_t>(W)) >> 32);
 }
 
+// The chosen node of layer l at step t when every layer draws its own (option "per_layer_leaders").
+#if defined(__CUDACC__)
+__host__ __device__
+#endif
+inline int32_t layer_leader_at(uint64_t seed, uint64_t t, uint64_t l, int32_t W) {
+  uint64_t z = seed + (t + 1) * 0x9E3779B97F4A7C15ull + (l + 1) * 0xA0761D6478BD642Full;
+  z ^= z >> 30;
+  z *= 0xBF58476D1CE4E5B9ull;
+  z ^= z >> 27;
+  z *= 0x94D049BB133111EBull;
+  z ^= z >> 31;
+  return static_cast<int32_t>(((z >> 32) * static_cast<uint64_t>(W)) >> 32);
+}
+
 // Section 3.3, random gradient selection: the 24-bit uniform draw of element i at step t.
 #if defined(__CUDACC__)
 __host__ __device__

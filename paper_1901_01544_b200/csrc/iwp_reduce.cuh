@@ -69,6 +69,43 @@ __global__ void __launch_bounds__(THREADS)
   update[i] = __fadd_rn(0.0f, s);
 }
 
+// Steps (e)-(g) when every layer has its own chosen node (Algorithm 1 draws the node inside its loop over
+// layers): entry j of the index set lies in the list segment of one layer and comes from that layer's
+// node's list.  One thread per entry: find the layer (binary search over the segment offsets), draw its
+// node, then gather, sum in ascending worker order, scatter and zero.  With dst != nullptr the kernel only
+// marks the index set in a byte mask (accessor).
+__global__ void __launch_bounds__(THREADS)
+    k_layer_leader_sum_scatter(const uint32_t* __restrict__ sel_idx, const LayerDesc* __restrict__ layers, uint32_t n_layers,
+                               float* __restrict__ acc, float* __restrict__ update, uint8_t* __restrict__ dst, uint64_t N,
+                               uint64_t K, int W, uint64_t seed, uint64_t step) {
+  const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (j >= K) return;
+  uint32_t lo = 0, hi = n_layers - 1;  // last layer whose segment starts at or before j
+  while (lo < hi) {
+    const uint32_t mid = (lo + hi + 1) >> 1;
+    if (layers[mid].koff <= j) lo = mid; else hi = mid - 1;
+  }
+  const int r = layer_leader_at(seed, step, lo, W);
+  const uint64_t i = sel_idx[static_cast<uint64_t>(r) * K + j];
+  if (dst != nullptr) {
+    dst[i] = 1;
+    return;
+  }
+  float* p = acc + i;
+  float s = 0.0f;
+  for (int w0 = 0; w0 < W; w0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = (w0 + u < W) ? p[static_cast<uint64_t>(w0 + u) * N] : 0.0f;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
+    }
+  }
+  for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
+  update[i] = __fadd_rn(0.0f, s);
+}
+
 // Workers spread over several contexts (one per GPU): step (e) for this context's workers at an index
 // set that came from elsewhere, vals[w][j] = acc[w][idx[j]]; grid-stride over (worker, entry).
 __global__ void __launch_bounds__(THREADS)

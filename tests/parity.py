@@ -42,7 +42,7 @@ def compare_state(pr: Pruner, orc: "oracle.Oracle", update_gpu: torch.Tensor, up
 
 def run_parity(layer_sizes, W, ratio, eps, seed, steps, weights: torch.Tensor, grads_fn, options=None,
                leader_overrides=None, check_mask=True, threads=0, residual_every=1, momentum=None, state_every=1,
-               weights_fn=None, n_leaders=1):
+               weights_fn=None, n_leaders=1, per_layer_leaders=False):
     """weights: CUDA tensor [N]; grads_fn(t) -> CUDA tensor [W, N].
 
     state_every: lists, mask, residuals and the device status are looked at only every that many steps
@@ -66,6 +66,9 @@ def run_parity(layer_sizes, W, ratio, eps, seed, steps, weights: torch.Tensor, g
     if n_leaders > 1:  # several chosen nodes: the index set is the union of their lists
         pr.set_option("n_leaders", n_leaders)
         orc.set_n_leaders(n_leaders)
+    if per_layer_leaders:  # every layer draws its own chosen node
+        pr.set_option("per_layer_leaders", 1)
+        orc.set_per_layer_leaders()
     w_host = weights.cpu().numpy()
     update = torch.full((pr.N,), float("nan"), dtype=torch.float32, device="cuda")
     for t in range(steps):

@@ -322,6 +322,28 @@ def test_union_on_a_scaled_network_shape():
                residual_every=1000)
 
 
+# ------------------------------------------------------------------ one chosen node per layer
+
+
+@pytest.mark.parametrize("speculate", [1, 0])
+def test_one_chosen_node_per_layer(speculate):
+    sizes, W, ratio = [70000, 64, 16385, 300000, 9, 40000, 1], 5, 32.0
+    N = sum(sizes)
+    weights = _weights(N, 23)
+    run_parity(sizes, W, ratio, 1e-8, seed=8, steps=5, weights=weights, grads_fn=lambda t: _randn((W, N), 880 + t),
+               per_layer_leaders=True, options={"speculate": speculate}, residual_every=2)
+
+
+def test_one_chosen_node_per_layer_on_a_scaled_network_shape():
+    from paper_1901_01544_b200 import binding
+
+    c = _scaled_case("resnet50_w8")
+    run_parity(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, c.steps, c.weights(DEV), lambda t: c.grads(t, DEV),
+               per_layer_leaders=True, residual_every=1000)
+    got = [binding.lib().iwp_layer_leader_at(0, t, l, 8) for t in range(2) for l in range(6)]
+    assert got == [2, 6, 1, 3, 7, 2, 7, 7, 5, 2, 7, 5]  # tests/golden/layer_leaders.txt, first row
+
+
 # ------------------------------------------------------------------ momentum on the residual (Eq. 3)
 
 
