@@ -232,6 +232,13 @@ int iwp_get_selection(iwp_ctx* ctx, int32_t w, uint32_t* idx_dev, float* val_dev
 /* Algorithm 1's encode_uint8(Mask): N bytes on the device, 1 where the element is in the
  * last step's index set, else 0. */
 int iwp_get_mask(iwp_ctx* ctx, uint8_t* dst_dev);
+
+/* The other reading of Algorithm 1's encode_uint8(Mask): eight elements per byte.  mask_dev: N bytes as
+ * written by iwp_get_mask(); bits_dev: (N + 7) / 8 bytes, bit i % 8 of byte i / 8 = mask_dev[i] != 0.
+ * Asynchronous on the context's stream; an accessor, not on the timed path (the path itself carries the
+ * sorted index list). */
+int iwp_encode_mask(iwp_ctx* ctx, const uint8_t* mask_dev, uint8_t* bits_dev);
+
 /* acc <- 0, step counter <- 0, status word <- 0. */
 int iwp_reset(iwp_ctx* ctx);
 

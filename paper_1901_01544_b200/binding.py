@@ -23,7 +23,7 @@ EXPORTS = [
     "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat", "iwp_select_static",
     "iwp_set_momentum", "iwp_create_threshold", "iwp_set_thresholds", "iwp_get_list_length", "iwp_leaders_at",
     "iwp_set_layerwise", "iwp_get_layer_thresholds", "iwp_shard_select", "iwp_shard_gather", "iwp_shard_apply",
-    "iwp_layer_leader_at",
+    "iwp_layer_leader_at", "iwp_encode_mask",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -75,6 +75,7 @@ def lib() -> C.CDLL:
         L.iwp_set_residual.argtypes = [vp, i32, vp]
         L.iwp_get_selection.argtypes = [vp, i32, vp, vp]
         L.iwp_get_mask.argtypes = [vp, vp]
+        L.iwp_encode_mask.argtypes = [vp, vp, vp]
         L.iwp_reset.argtypes = [vp]
         L.iwp_set_option.argtypes = [vp, cp, i64]
         L.iwp_get_stat.argtypes = [vp, cp, vp]
@@ -312,6 +313,13 @@ class Pruner:
         m = self._torch.empty(self.N, dtype=self._torch.uint8, device=self.device)
         _check(lib().iwp_get_mask(self._h, m.data_ptr()), "iwp_get_mask")
         return m
+
+    def mask_bits(self):
+        """The index set of the last step at eight elements per byte (bit i % 8 of byte i / 8)."""
+        m = self.mask()
+        bits = self._torch.empty((self.N + 7) // 8, dtype=self._torch.uint8, device=self.device)
+        _check(lib().iwp_encode_mask(self._h, m.data_ptr(), bits.data_ptr()), "iwp_encode_mask")
+        return bits
 
     def reset(self) -> None:
         _check(lib().iwp_reset(self._h), "iwp_reset")

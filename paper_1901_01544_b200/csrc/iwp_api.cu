@@ -1149,6 +1149,14 @@ int iwp_get_mask(iwp_ctx* c, uint8_t* dst) {
   return IWP_OK;
 }
 
+int iwp_encode_mask(iwp_ctx* c, const uint8_t* mask, uint8_t* bits) {
+  if (!c || !mask || !bits) return IWP_ERR_INVALID;
+  const uint64_t N = c->plan.N, n_bytes = (N + 7) / 8;
+  k_pack_mask<<<static_cast<unsigned>((n_bytes + THREADS - 1) / THREADS), THREADS, 0, c->stream>>>(mask, bits, N);
+  if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+  return IWP_OK;
+}
+
 int iwp_reset(iwp_ctx* c) {
   if (!c) return IWP_ERR_INVALID;
   if (const int jrc = join_deferred(c)) return jrc;

@@ -234,4 +234,18 @@ __global__ void __launch_bounds__(THREADS) k_mask_scatter(const uint32_t* __rest
   if (j < K) dst[leader_idx[j]] = 1;
 }
 
+// The byte mask at eight elements per byte (the other reading of encode_uint8(Mask)): bit i % 8 of byte
+// i / 8 is element i's mask value.  One thread per output byte.
+__global__ void __launch_bounds__(THREADS) k_pack_mask(const uint8_t* __restrict__ mask, uint8_t* __restrict__ bits, uint64_t N) {
+  const uint64_t b = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+  if (b * 8 >= N) return;
+  uint32_t v = 0;
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    const uint64_t i = b * 8 + q;
+    if (i < N && mask[i]) v |= 1u << q;
+  }
+  bits[b] = static_cast<uint8_t>(v);
+}
+
 }  // namespace iwp

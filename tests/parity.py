@@ -38,6 +38,7 @@ def compare_state(pr: Pruner, orc: "oracle.Oracle", update_gpu: torch.Tensor, up
             assert_bits_equal(pr.residual(w).cpu().numpy(), orc.residual(w), f"{tag}: worker {w} residual")
     if check_mask:
         assert np.array_equal(pr.mask().cpu().numpy(), orc.mask()), f"{tag}: mask"
+        assert np.array_equal(pr.mask_bits().cpu().numpy(), np.packbits(orc.mask(), bitorder="little")), f"{tag}: packed mask"
 
 
 def run_parity(layer_sizes, W, ratio, eps, seed, steps, weights: torch.Tensor, grads_fn, options=None,
