@@ -289,14 +289,14 @@ int flush_pending_zero(iwp_ctx* c) {
 // Exact select (three histogram passes with their digit decisions) and ordered compaction of the
 // workers `ws` covers, on stream `st`.
 template <bool VEC>
-int select_and_write(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSel ws, int32_t leader, bool use_sfx) {
+int select_and_write(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSel ws, int32_t leader) {
   const Plan& p = c->plan;
   const int W = p.W;
   const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
   const unsigned n_sel = static_cast<unsigned>(sel_count(ws, W));
   if (n_sel == 0) return IWP_OK;
   dim3 cgrid(n_chunks, n_sel), pgrid(static_cast<unsigned>(p.large_layers.size()), n_sel);
-  uint32_t* sfx = use_sfx ? c->chunk_sfx : nullptr;
+  uint32_t* sfx = c->chunk_sfx;
   for (int pass = 0; pass < N_PASSES; ++pass) {
     k_hist<VEC><<<cgrid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_layers, c->info_cur, c->cand_key,
                                            c->cand_cnt, c->d_state, c->d_hist, sfx, c->d_chunk_cnt, c->eps, p.N, W,
@@ -409,7 +409,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     // the leader's select and list, under the other workers' streaming pass
     if (!cuda_ok(cudaEventRecord(c->ev_lead, s)) || !cuda_ok(cudaStreamWaitEvent(c->side_a, c->ev_lead, 0)))
       return IWP_ERR_CUDA;
-    int rc = select_and_write<VEC>(c, weights, c->side_a, WorkerSel{WorkerSel::ONLY, leader, -1}, leader, true);
+    int rc = select_and_write<VEC>(c, weights, c->side_a, WorkerSel{WorkerSel::ONLY, leader, -1}, leader);
     if (rc != IWP_OK) return rc;
     if (!cuda_ok(cudaEventRecord(c->ev_lead_done, c->side_a))) return IWP_ERR_CUDA;
     if (c->pending_b && !cuda_ok(cudaStreamWaitEvent(s, c->ev_b, 0))) return IWP_ERR_CUDA;
@@ -438,7 +438,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     const int32_t next = leader_of_step(c, c->t + 1);
     if (next != leader) {
       if (!cuda_ok(cudaStreamWaitEvent(c->side_a, c->ev_others, 0))) return IWP_ERR_CUDA;
-      rc = select_and_write<VEC>(c, c->saved_w, c->side_a, WorkerSel{WorkerSel::ONLY, next, -1}, leader, true);
+      rc = select_and_write<VEC>(c, c->saved_w, c->side_a, WorkerSel{WorkerSel::ONLY, next, -1}, leader);
       if (rc != IWP_OK) return rc;
       if (!cuda_ok(cudaEventRecord(c->ev_a2, c->side_a))) return IWP_ERR_CUDA;
       c->pending_a2 = true;
@@ -446,7 +446,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     const WorkerSel rest{WorkerSel::EXCEPT, leader, next};
     if (sel_count(rest, W) > 0) {
       if (!cuda_ok(cudaStreamWaitEvent(c->side_b, c->ev_others, 0))) return IWP_ERR_CUDA;
-      rc = select_and_write<VEC>(c, c->saved_w, c->side_b, rest, leader, true);
+      rc = select_and_write<VEC>(c, c->saved_w, c->side_b, rest, leader);
       if (rc != IWP_OK) return rc;
       if (!cuda_ok(cudaEventRecord(c->ev_b, c->side_b))) return IWP_ERR_CUDA;
       c->pending_b = true;
