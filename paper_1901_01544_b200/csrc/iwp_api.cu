@@ -614,7 +614,7 @@ int iwp_plan_sizes(const int64_t* layer_sizes, int32_t n_layers, int32_t W, doub
 
 namespace {
 
-constexpr uint32_t THRESHOLD_CHUNK_TILES = 16;  // 64 Ki elements per CTA of the threshold-mode select
+constexpr uint32_t THRESHOLD_CHUNK_TILES = 8;  // 32 Ki elements per CTA of the threshold-mode passes over the chosen nodes
 
 int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, int32_t W, double ratio, float eps,
                   uint64_t seed, bool threshold_mode, int64_t max_list) {
@@ -796,30 +796,34 @@ int run_step_threshold(iwp_ctx* c, const float* grads, const float* weights, flo
   }
   c->launches += 1;
   stage_mark_at(c, 2);
-  k_thr_accumulate_chosen<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, c->d_tiles, N, c->momentum, ls);
-  IWP_LAUNCH_CHECK(c);
-  stage_mark_at(c, 3);
   const uint32_t n_layers = static_cast<uint32_t>(p.layers.size());
-  const uint32_t* thr = c->d_thr;
-  uint32_t thr_stride = 0;
-  if (c->layerwise) {  // Eq. 4: every chosen node's thresholds from its own exact moments
+  if (c->layerwise) {
+    // Eq. 4 needs the accumulated residuals first: step (a) for the chosen nodes, their exact moments, the
+    // thresholds, and only then the masks
+    k_thr_accumulate_chosen<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, c->d_tiles, N, c->momentum, ls);
+    IWP_LAUNCH_CHECK(c);
+    stage_mark_at(c, 3);
     k_thr_stats<VEC><<<dim3(n_chunks, static_cast<unsigned>(ls.n)), THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_bins,
                                                                                   c->eps, N, n_layers, ls);
     IWP_LAUNCH_CHECK(c);
     k_thr_finalize<<<dim3(n_layers, static_cast<unsigned>(ls.n)), THREADS, 0, s>>>(c->d_bins, c->d_layers, c->d_thr_lw, n_layers,
                                                                                 c->lw_alpha, c->lw_beta, c->lw_c);
     IWP_LAUNCH_CHECK(c);
-    thr = c->d_thr_lw;
-    thr_stride = n_layers;
     c->lw_chosen = ls.n;
+    k_thr_mask_count<VEC, false><<<n_chunks, THREADS, 0, s>>>(grads, c->acc, weights, c->d_chunks, c->d_thr_lw, n_layers,
+                                                              c->zmask, c->d_tcnt, c->eps, N, c->momentum, ls, rs);
+  } else {
+    // fixed thresholds: step (a) for the chosen nodes, their masks and the chunk counts in one pass
+    stage_mark_at(c, 3);
+    k_thr_mask_count<VEC, true><<<n_chunks, THREADS, 0, s>>>(grads, c->acc, weights, c->d_chunks, c->d_thr, 0u, c->zmask,
+                                                             c->d_tcnt, c->eps, N, c->momentum, ls, rs);
   }
-  k_thr_count<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, thr, thr_stride, c->d_tcnt, c->eps, N, ls, rs);
   IWP_LAUNCH_CHECK(c);
   k_thr_scan<<<1, 1024, 0, s>>>(c->d_tcnt, c->d_toff, n_chunks, c->d_list_len);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 4);
-  k_thr_write<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, thr, thr_stride, c->d_toff, c->sel_idx,
-                                                c->sel_val, cap, c->d_status, c->zmask, c->eps, N, ls, rs);
+  k_thr_write<VEC><<<n_chunks, THREADS, 0, s>>>(c->acc + static_cast<uint64_t>(ls.r[0]) * N, c->d_chunks, c->d_toff, c->zmask,
+                                                c->sel_idx, c->sel_val, cap, c->d_status);
   IWP_LAUNCH_CHECK(c);
   stage_mark_at(c, 5);
   k_thr_fused<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, update, c->d_tiles, c->zmask, N, W, c->momentum, ls);

@@ -36,11 +36,15 @@ __device__ __forceinline__ bool thr_selected(float acc, float w, float eps, uint
   return u < __fdiv_rn(__uint_as_float(key), __uint_as_float(T));
 }
 
-template <bool VEC>
+// First look at the chosen nodes' residuals, chunk by chunk: (ACCUMULATE: step (a) for them, acc <- m acc + g,
+// on the way;) the OR of their masks as one bit per element (`set_bits`, zeroed before the step) and the
+// number of set elements of the chunk.  Everything after this pass works from the bits.  grid = chunks.
+template <bool VEC, bool ACCUMULATE>
 __global__ void __launch_bounds__(THREADS)
-    k_thr_count(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
-                const uint32_t* __restrict__ thr_bits, uint32_t thr_stride, uint32_t* __restrict__ chunk_cnt, float eps,
-                uint64_t N, LeaderSet ls, RandomSelect rs) {
+    k_thr_mask_count(const float* __restrict__ grads, float* __restrict__ acc, const float* __restrict__ weights,
+                     const Chunk* __restrict__ chunks, const uint32_t* __restrict__ thr_bits, uint32_t thr_stride,
+                     uint32_t* __restrict__ set_bits, uint32_t* __restrict__ chunk_cnt, float eps, uint64_t N,
+                     float momentum, LeaderSet ls, RandomSelect rs) {
   __shared__ uint32_t sh_cnt;
   const Chunk c = chunks[blockIdx.x];
   // thr_stride = 0: one threshold per layer for every chosen node; = number of layers: node j has its own row
@@ -51,22 +55,35 @@ __global__ void __launch_bounds__(THREADS)
   const uint64_t s0 = lo & ~3ull;
   const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
   uint32_t cnt = 0;
+#pragma unroll 2
   for (uint32_t it = 0; it < n_iter; ++it) {
     const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
     float wv[4];
     load4<VEC>(weights, e0, lo, hi, wv);
     uint32_t f = 0;  // Mask = OR of the chosen nodes' masks
     for (int j = 0; j < ls.n; ++j) {
+      float* a = acc + static_cast<uint64_t>(ls.r[j]) * N;
       float av[4];
-      load4<VEC>(acc + static_cast<uint64_t>(ls.r[j]) * N, e0, lo, hi, av);
+      load4_stream<VEC>(a, e0, lo, hi, av);
+      if (ACCUMULATE) {
+        float gv[4];
+        load4_stream<VEC>(grads + static_cast<uint64_t>(ls.r[j]) * N, e0, lo, hi, gv);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) av[q] = accumulate(av[q], gv[q], momentum);
+        store4<VEC>(a, e0, lo, hi, av);
+      }
 #pragma unroll
       for (int q = 0; q < 4; ++q) f |= thr_selected(av[q], wv[q], eps, T[j * thr_stride], e0 + q, rs) ? (1u << q) : 0u;
     }
+    {
+      uint32_t inside = 0;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const uint64_t e = e0 + q;
-      cnt += (e >= lo && e < hi && ((f >> q) & 1u)) ? 1u : 0u;
+      for (int q = 0; q < 4; ++q) inside |= (e0 + q >= lo && e0 + q < hi) ? (1u << q) : 0u;
+      f &= inside;
     }
+    // a slot's four bits never straddle a word because slots start at multiples of four
+    if (f) atomicOr(&set_bits[e0 >> 5], f << (e0 & 31u));
+    cnt += __popc(f);
   }
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
@@ -106,43 +123,28 @@ __global__ void __launch_bounds__(1024)
   if (threadIdx.x == 0) *list_len = sh_run;
 }
 
+// Second look, from the bits alone: the ordered index list (ascending; offsets from the scan of the chunk
+// counts) with r_1's residuals as the listed values, read only where a bit is set.  grid = chunks.
 template <bool VEC>
 __global__ void __launch_bounds__(THREADS)
-    k_thr_write(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
-                const uint32_t* __restrict__ thr_bits, uint32_t thr_stride, const uint32_t* __restrict__ chunk_off,
-                uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val, uint32_t capacity,
-                int* __restrict__ status, uint32_t* __restrict__ set_bits, float eps, uint64_t N, LeaderSet ls,
-                RandomSelect rs) {
+    k_thr_write(const float* __restrict__ acc_r1, const Chunk* __restrict__ chunks, const uint32_t* __restrict__ chunk_off,
+                const uint32_t* __restrict__ set_bits, uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val,
+                uint32_t capacity, int* __restrict__ status) {
   __shared__ uint32_t sh_warp[WARPS];
   const Chunk c = chunks[blockIdx.x];
-  const uint32_t* T = thr_bits + c.layer;
   uint32_t run = chunk_off[blockIdx.x];
   const uint64_t lo = c.a, hi = lo + c.len;
   const uint64_t s0 = lo & ~3ull;
   const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
   for (uint32_t it = 0; it < n_iter; ++it) {
     const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
-    float av[4], wv[4];  // av: r_1's values, the ones listed
-    load4<VEC>(acc + static_cast<uint64_t>(ls.r[0]) * N, e0, lo, hi, av);
-    load4<VEC>(weights, e0, lo, hi, wv);
-    uint32_t f = 0;
+    // the bits of neighbouring layers in the same word belong to other chunks: keep this chunk's elements only
+    uint32_t f = (e0 < hi) ? (set_bits[e0 >> 5] >> (e0 & 31u)) & 0xFu : 0u;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) f |= thr_selected(av[q], wv[q], eps, T[0], e0 + q, rs) ? (1u << q) : 0u;
-    for (int j = 1; j < ls.n; ++j) {
-      float bv[4];
-      load4<VEC>(acc + static_cast<uint64_t>(ls.r[j]) * N, e0, lo, hi, bv);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) f |= thr_selected(bv[q], wv[q], eps, T[j * thr_stride], e0 + q, rs) ? (1u << q) : 0u;
-    }
-    {
-      uint32_t inside = 0;
-#pragma unroll
-      for (int q = 0; q < 4; ++q) inside |= (e0 + q >= lo && e0 + q < hi) ? (1u << q) : 0u;
-      f &= inside;
-    }
-    // the index set as a bit per element (zeroed before the step) for the fused pass over all workers;
-    // a slot's four bits never straddle a word because slots start at multiples of four
-    if (f) atomicOr(&set_bits[e0 >> 5], f << (e0 & 31u));
+    for (int q = 0; q < 4; ++q)
+      if (e0 + q < lo || e0 + q >= hi) f &= ~(1u << q);
+    float av[4] = {0.f, 0.f, 0.f, 0.f};
+    if (f) load4<VEC>(acc_r1, e0, lo, hi, av);
     uint32_t total;
     uint32_t pos = run + block_excl_scan(static_cast<uint32_t>(__popc(f)), sh_warp, total);
     if (f) {
