@@ -803,8 +803,8 @@ int run_step_threshold(iwp_ctx* c, const float* grads, const float* weights, flo
     k_thr_accumulate_chosen<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, c->d_tiles, N, c->momentum, ls);
     IWP_LAUNCH_CHECK(c);
     stage_mark_at(c, 3);
-    k_thr_stats<VEC><<<dim3(n_chunks, static_cast<unsigned>(ls.n)), THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_bins,
-                                                                                  c->eps, N, n_layers, ls);
+    k_thr_stats<VEC><<<dim3((n_chunks + STATS_GROUP - 1) / STATS_GROUP, static_cast<unsigned>(ls.n)), THREADS, 0, s>>>(
+        c->acc, weights, c->d_chunks, n_chunks, c->d_bins, c->eps, N, n_layers, ls);
     IWP_LAUNCH_CHECK(c);
     k_thr_finalize<<<dim3(n_layers, static_cast<unsigned>(ls.n)), THREADS, 0, s>>>(c->d_bins, c->d_layers, c->d_thr_lw, n_layers,
                                                                                 c->lw_alpha, c->lw_beta, c->lw_c);

@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include "iwp_device.cuh"
+#include "iwp_stream.cuh"
 
 namespace iwp {
 
@@ -25,8 +26,12 @@ struct RandomSelect {
 
 // Mask bit of one element on one chosen node: importance > thr, or - with random selection on - a
 // draw below importance / thr (P(update) = importance / threshold; one draw per element and step).
-__device__ __forceinline__ bool thr_selected(float acc, float w, float eps, uint32_t T, uint64_t e,
+// gm, gme: the multiply pre-test of the streaming pass (pretest_multiplier(T, eps) and its product with eps):
+// an element whose exactly rounded quotient exceeds T passes |acc| >= gm (|w| + eps), so without random
+// selection everything that fails it is out without a division.
+__device__ __forceinline__ bool thr_selected(float acc, float w, float eps, uint32_t T, float gm, float gme, uint64_t e,
                                              const RandomSelect& rs) {
+  if (!rs.on && !(fabsf(acc) >= __fmaf_rn(gm, fabsf(w), gme))) return false;
   const uint32_t key = imp_key(acc, w, eps);
   // importance patterns are non-negative, so as signed integers they order like the values against any
   // threshold pattern: a negative threshold (layer-wise mode can produce one) is below every importance
@@ -49,41 +54,58 @@ __global__ void __launch_bounds__(THREADS)
   const Chunk c = chunks[blockIdx.x];
   // thr_stride = 0: one threshold per layer for every chosen node; = number of layers: node j has its own row
   const uint32_t* T = thr_bits + c.layer;
+  __shared__ float sh_gm[MAX_LEADERS];  // pre-test multiplier of every chosen node's threshold
   if (threadIdx.x == 0) sh_cnt = 0;
+  if (threadIdx.x < ls.n) sh_gm[threadIdx.x] = pretest_multiplier(T[threadIdx.x * thr_stride], eps);
   __syncthreads();
   const uint64_t lo = c.a, hi = lo + c.len;
   const uint64_t s0 = lo & ~3ull;
   const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
   uint32_t cnt = 0;
-#pragma unroll 2
-  for (uint32_t it = 0; it < n_iter; ++it) {
-    const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
-    float wv[4];
-    load4<VEC>(weights, e0, lo, hi, wv);
-    uint32_t f = 0;  // Mask = OR of the chosen nodes' masks
+  constexpr int U = 2;  // slots per thread and trip: the loads of both are issued before either is used
+  for (uint32_t it = 0; it < n_iter; it += U) {
+    uint64_t e0[U];
+    float wv[U][4];
+    uint32_t f[U];  // Mask = OR of the chosen nodes' masks
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      e0[u] = s0 + (static_cast<uint64_t>(it + u) * THREADS + threadIdx.x) * 4;  // beyond the chunk: every access is guarded
+      load4<VEC>(weights, e0[u], lo, hi, wv[u]);
+      f[u] = 0;
+    }
     for (int j = 0; j < ls.n; ++j) {
       float* a = acc + static_cast<uint64_t>(ls.r[j]) * N;
-      float av[4];
-      load4_stream<VEC>(a, e0, lo, hi, av);
-      if (ACCUMULATE) {
-        float gv[4];
-        load4_stream<VEC>(grads + static_cast<uint64_t>(ls.r[j]) * N, e0, lo, hi, gv);
+      const float* g = grads + static_cast<uint64_t>(ls.r[j]) * N;
+      const float gm = sh_gm[j], gme = __fmul_rn(gm, eps);
+      const uint32_t Tj = T[j * thr_stride];
+      float av[U][4], gv[U][4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) av[q] = accumulate(av[q], gv[q], momentum);
-        store4<VEC>(a, e0, lo, hi, av);
+      for (int u = 0; u < U; ++u) {
+        load4_stream<VEC>(a, e0[u], lo, hi, av[u]);
+        if (ACCUMULATE) load4_stream<VEC>(g, e0[u], lo, hi, gv[u]);
       }
 #pragma unroll
-      for (int q = 0; q < 4; ++q) f |= thr_selected(av[q], wv[q], eps, T[j * thr_stride], e0 + q, rs) ? (1u << q) : 0u;
+      for (int u = 0; u < U; ++u) {
+        if (ACCUMULATE) {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) av[u][q] = accumulate(av[u][q], gv[u][q], momentum);
+          store4<VEC>(a, e0[u], lo, hi, av[u]);
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          f[u] |= thr_selected(av[u][q], wv[u][q], eps, Tj, gm, gme, e0[u] + q, rs) ? (1u << q) : 0u;
+      }
     }
-    {
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
       uint32_t inside = 0;
 #pragma unroll
-      for (int q = 0; q < 4; ++q) inside |= (e0 + q >= lo && e0 + q < hi) ? (1u << q) : 0u;
-      f &= inside;
+      for (int q = 0; q < 4; ++q) inside |= (e0[u] + q >= lo && e0[u] + q < hi) ? (1u << q) : 0u;
+      f[u] &= inside;
+      // a slot's four bits never straddle a word because slots start at multiples of four
+      if (f[u]) atomicOr(&set_bits[e0[u] >> 5], f[u] << (e0[u] & 31u));
+      cnt += __popc(f[u]);
     }
-    // a slot's four bits never straddle a word because slots start at multiples of four
-    if (f) atomicOr(&set_bits[e0 >> 5], f << (e0 & 31u));
-    cnt += __popc(f);
   }
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
@@ -185,115 +207,131 @@ constexpr int LW_BINS = 384;  // 255 exponents, plus room for the 32-bit digits 
 // base + 16 k (a bin index step doubles the weight of m and quadruples that of m^2).
 // Slow path, for the few elements outside the window: lanes with the same exponent add their terms
 // with one warp reduction and one shared-memory atomic per term.
+constexpr uint32_t STATS_GROUP = 1;  // chunks per CTA of k_thr_stats (more were measured slower: the pass wants many CTAs)
+
 template <bool VEC>
 __global__ void __launch_bounds__(THREADS)
     k_thr_stats(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
-                unsigned long long* __restrict__ bins, float eps, uint64_t N, uint32_t n_layers, LeaderSet ls) {
+                uint32_t n_chunks, unsigned long long* __restrict__ bins, float eps, uint64_t N, uint32_t n_layers,
+                LeaderSet ls) {
   __shared__ unsigned long long sh[3 * LW_BINS];
-  __shared__ unsigned long long sh_fast[8];  // digits: [0..2] first moment, [3..7] second
-  __shared__ uint32_t sh_exp[2];             // sum and count of the exponents sampled for the window
-  const Chunk c = chunks[blockIdx.x];
+  __shared__ uint32_t sh_exp[2];  // sum and count of the exponents sampled for the window
   const int j = blockIdx.y;
   int r = ls.r[0];
 #pragma unroll
   for (int q = 1; q < MAX_LEADERS; ++q)
     if (q == j) r = ls.r[q];
-  for (int b = threadIdx.x; b < 3 * LW_BINS; b += THREADS) sh[b] = 0ull;
-  if (threadIdx.x < 8) sh_fast[threadIdx.x] = 0ull;
-  if (threadIdx.x < 2) sh_exp[threadIdx.x] = 0u;
-  __syncthreads();
   const float* a = acc + static_cast<uint64_t>(r) * N;
-  const uint64_t lo = c.a, hi = lo + c.len;
-  const uint64_t s0 = lo & ~3ull;
-  const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
   const int lane = threadIdx.x & 31;
-  // widest shift that keeps m << d inside 63 bits summed over this thread's elements (and m^2 << 2d inside 127)
-  const int d_max = min(30, 39 - (32 - __clz(n_iter * 4)));
-  int base = 1;
-  {  // window: average exponent of the first element of every thread, minus 14
-    const uint64_t e = s0 + static_cast<uint64_t>(threadIdx.x) * 4;
-    uint32_t f = 0, cnt = 0;
-    for (int q = 0; q < 4 && cnt == 0; ++q) {
-      if (e + q >= lo && e + q < hi) {
-        const uint32_t key = imp_key(a[e + q], weights[e + q], eps);
-        if (key != 0u && key < 0x7f800000u) {
-          f = max(key >> 23, 1u);
-          cnt = 1;
-        }
+  for (int b = threadIdx.x; b < 3 * LW_BINS; b += THREADS) sh[b] = 0ull;
+  auto flush = [&](uint32_t layer) {  // this CTA's bins of one layer into the global ones; leaves them cleared
+    __syncthreads();
+    unsigned long long* g = bins + (static_cast<uint64_t>(j) * n_layers + layer) * (3 * LW_BINS);
+    for (int b = threadIdx.x; b < 3 * LW_BINS; b += THREADS) {
+      const unsigned long long v = sh[b];
+      if (v) {
+        atomicAdd(&g[b], v);
+        sh[b] = 0ull;
       }
-    }
-    f = __reduce_add_sync(0xffffffffu, f);
-    cnt = __reduce_add_sync(0xffffffffu, cnt);
-    if (lane == 0 && cnt) {
-      atomicAdd(&sh_exp[0], f);
-      atomicAdd(&sh_exp[1], cnt);
     }
     __syncthreads();
-    if (sh_exp[1]) base = max(1, static_cast<int>(sh_exp[0] / sh_exp[1]) - 14);
-  }
-  unsigned long long s1 = 0ull;
-  unsigned __int128 s2 = 0;
-  for (uint32_t it = 0; it < n_iter; ++it) {
-    const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
-    float av[4], wv[4];
-    load4<VEC>(a, e0, lo, hi, av);
-    load4<VEC>(weights, e0, lo, hi, wv);
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const uint64_t e = e0 + q;
-      const uint32_t key = imp_key(av[q], wv[q], eps);
-      // zero adds nothing; a non-finite importance is outside the contract and is left out
-      bool valid = e >= lo && e < hi && key != 0u && key < 0x7f800000u;
-      const uint32_t ex = key >> 23;
-      const uint32_t m = ex ? ((key & 0x7fffffu) | 0x800000u) : key;
-      const unsigned long long m2 = static_cast<unsigned long long>(m) * m;
-      const int d = static_cast<int>(max(ex, 1u)) - base;
-      if (valid && d >= 0 && d <= d_max) {
-        s1 += static_cast<unsigned long long>(m) << d;
-        s2 += static_cast<unsigned __int128>(m2) << (2 * d);
-        valid = false;
-      }
-      unsigned todo = __ballot_sync(0xffffffffu, valid);
-      if (todo == 0u) continue;
-      const uint32_t h = static_cast<uint32_t>(m2 >> 24), l = static_cast<uint32_t>(m2) & 0xffffffu;
-      while (todo) {
-        const int first = __ffs(todo) - 1;
-        const uint32_t ex_first = __shfl_sync(0xffffffffu, ex, first);
-        const bool mine = valid && ex == ex_first;
-        const unsigned grp = __ballot_sync(0xffffffffu, mine);
-        if (mine) {  // 32 terms below 2^24 fit 32 bits
-          const uint32_t sm = __reduce_add_sync(grp, m), shh = __reduce_add_sync(grp, h), sl = __reduce_add_sync(grp, l);
-          if (lane == first) {
-            atomicAdd(&sh[ex_first], static_cast<unsigned long long>(sm));
-            atomicAdd(&sh[LW_BINS + ex_first], static_cast<unsigned long long>(shh));
-            atomicAdd(&sh[2 * LW_BINS + ex_first], static_cast<unsigned long long>(sl));
+  };
+  // a group of consecutive chunks per CTA: the bins are shared by the chunks of a layer and go to global
+  // memory when the layer changes and at the end
+  const uint32_t c_first = blockIdx.x * STATS_GROUP, c_last = min(c_first + STATS_GROUP, n_chunks);
+  uint32_t cur_layer = chunks[c_first].layer;
+  for (uint32_t ci = c_first; ci < c_last; ++ci) {
+    const Chunk c = chunks[ci];
+    if (c.layer != cur_layer) {
+      flush(cur_layer);
+      cur_layer = c.layer;
+    }
+    if (threadIdx.x < 2) sh_exp[threadIdx.x] = 0u;
+    __syncthreads();
+    const uint64_t lo = c.a, hi = lo + c.len;
+    const uint64_t s0 = lo & ~3ull;
+    const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+    // widest shift that keeps m << d inside 63 bits summed over this thread's elements (and m^2 << 2d inside 127)
+    const int d_max = min(30, 39 - (32 - __clz(n_iter * 4)));
+    int base = 1;
+    {  // window: average exponent of the first element of every thread, minus 14
+      const uint64_t e = s0 + static_cast<uint64_t>(threadIdx.x) * 4;
+      uint32_t f = 0, cnt = 0;
+      for (int q = 0; q < 4 && cnt == 0; ++q) {
+        if (e + q >= lo && e + q < hi) {
+          const uint32_t key = imp_key(a[e + q], weights[e + q], eps);
+          if (key != 0u && key < 0x7f800000u) {
+            f = max(key >> 23, 1u);
+            cnt = 1;
           }
         }
-        todo &= ~grp;
+      }
+      f = __reduce_add_sync(0xffffffffu, f);
+      cnt = __reduce_add_sync(0xffffffffu, cnt);
+      if (lane == 0 && cnt) {
+        atomicAdd(&sh_exp[0], f);
+        atomicAdd(&sh_exp[1], cnt);
+      }
+      __syncthreads();
+      if (sh_exp[1]) base = max(1, static_cast<int>(sh_exp[0] / sh_exp[1]) - 14);
+    }
+    unsigned long long s1 = 0ull;
+    unsigned __int128 s2 = 0;
+    for (uint32_t it = 0; it < n_iter; ++it) {
+      const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+      float av[4], wv[4];
+      load4<VEC>(a, e0, lo, hi, av);
+      load4<VEC>(weights, e0, lo, hi, wv);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint64_t e = e0 + q;
+        const uint32_t key = imp_key(av[q], wv[q], eps);
+        // zero adds nothing; a non-finite importance is outside the contract and is left out
+        bool valid = e >= lo && e < hi && key != 0u && key < 0x7f800000u;
+        const uint32_t ex = key >> 23;
+        const uint32_t m = ex ? ((key & 0x7fffffu) | 0x800000u) : key;
+        const unsigned long long m2 = static_cast<unsigned long long>(m) * m;
+        const int d = static_cast<int>(max(ex, 1u)) - base;
+        if (valid && d >= 0 && d <= d_max) {
+          s1 += static_cast<unsigned long long>(m) << d;
+          s2 += static_cast<unsigned __int128>(m2) << (2 * d);
+          valid = false;
+        }
+        unsigned todo = __ballot_sync(0xffffffffu, valid);
+        if (todo == 0u) continue;
+        const uint32_t h = static_cast<uint32_t>(m2 >> 24), l = static_cast<uint32_t>(m2) & 0xffffffu;
+        while (todo) {
+          const int first = __ffs(todo) - 1;
+          const uint32_t ex_first = __shfl_sync(0xffffffffu, ex, first);
+          const bool mine = valid && ex == ex_first;
+          const unsigned grp = __ballot_sync(0xffffffffu, mine);
+          if (mine) {  // 32 terms below 2^24 fit 32 bits
+            const uint32_t sm = __reduce_add_sync(grp, m), shh = __reduce_add_sync(grp, h), sl = __reduce_add_sync(grp, l);
+            if (lane == first) {
+              atomicAdd(&sh[ex_first], static_cast<unsigned long long>(sm));
+              atomicAdd(&sh[LW_BINS + ex_first], static_cast<unsigned long long>(shh));
+              atomicAdd(&sh[2 * LW_BINS + ex_first], static_cast<unsigned long long>(sl));
+            }
+          }
+          todo &= ~grp;
+        }
+      }
+    }
+    // the thread's window sums, digit by digit, into the bins whose weight the digits have: digit k of the
+    // first moment is worth bin base + 32 k, of the second bin base + 16 k (see above)
+    if (s1) {
+      atomicAdd(&sh[base], s1 & 0xffffffffull);
+      atomicAdd(&sh[base + 32], s1 >> 32);
+    }
+    if (s2) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const unsigned long long dg = static_cast<unsigned long long>(s2 >> (32 * k)) & 0xffffffffull;
+        if (dg) atomicAdd(&sh[2 * LW_BINS + base + 16 * k], dg);
       }
     }
   }
-  // the threads' window sums, digit by digit (each digit sum stays far below 2^64)
-  if (s1) {
-    atomicAdd(&sh_fast[0], s1 & 0xffffffffull);
-    atomicAdd(&sh_fast[1], s1 >> 32);
-  }
-  if (s2) {
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const unsigned long long dg = static_cast<unsigned long long>(s2 >> (32 * k)) & 0xffffffffull;
-      if (dg) atomicAdd(&sh_fast[3 + k], dg);
-    }
-  }
-  __syncthreads();
-  unsigned long long* g = bins + (static_cast<uint64_t>(j) * n_layers + c.layer) * (3 * LW_BINS);
-  for (int b = threadIdx.x; b < 3 * LW_BINS; b += THREADS) {
-    const unsigned long long v = sh[b];
-    if (v) atomicAdd(&g[b], v);
-  }
-  if (threadIdx.x < 2 && sh_fast[threadIdx.x]) atomicAdd(&g[base + 32 * threadIdx.x], sh_fast[threadIdx.x]);
-  if (threadIdx.x >= 3 && threadIdx.x < 7 && sh_fast[threadIdx.x])
-    atomicAdd(&g[2 * LW_BINS + base + 16 * (threadIdx.x - 3)], sh_fast[threadIdx.x]);
+  flush(cur_layer);
 }
 
 // The wide integer in base-2^32 digits (64-bit words that may run ahead until the carries are
