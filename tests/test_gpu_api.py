@@ -65,20 +65,29 @@ def test_reset_and_checkpoint_roundtrip():
     pr2.close()
 
 
-def test_host_buffer_entry_point_matches_oracle():
+@pytest.mark.parametrize("overlap", [0, 1])
+def test_host_buffer_entry_point_matches_oracle(overlap):
+    # the host weights change between steps: with the overlapped schedule the other workers' selects of one
+    # step may still run while the next call copies new weights into the staging buffer
     sizes, W = [40000, 300, 20000], 4
     N = sum(sizes)
     weights, grads = _inputs(W, N, 3)
     pr = Pruner(sizes, W, 64.0, 1e-8, 0)
+    pr.set_option("overlap", overlap)
     orc = oracle.Oracle(sizes, W, 64.0, 1e-8, 0)
-    wh = weights.cpu().pin_memory()
     uh = torch.empty(N).pin_memory()
-    for g in grads:
+    for t, g in enumerate(grads + grads):
         gh = g.cpu().pin_memory()
+        wh = (weights * (1.0 + 0.25 * t)).cpu().pin_memory()
         pr.step_host(gh, wh, uh)
         want = orc.step(gh.numpy(), wh.numpy())
         assert_bits_equal(uh.numpy(), want, "update via host buffers")
     assert pr.sync_status() == 0
+    for w in range(W):
+        idx, val = pr.selection(w)
+        oi, ov = orc.selection(w)
+        assert np.array_equal(idx.cpu().numpy().view(np.uint32), oi)
+        assert_bits_equal(val.cpu().numpy(), ov, f"worker {w} list values")
     pr.close()
 
 
