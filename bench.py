@@ -350,12 +350,16 @@ def run_ours(args):
     if not args.no_e2e:
         gh = [sets[i].cpu().pin_memory() for i in range(min(2, n_sets))]
         wh = weights.cpu().pin_memory()
-        uh = torch.empty(N, dtype=torch.float32).pin_memory()
-        pr.step_host(gh[0], wh, uh)  # allocates the staging buffers
+        uh = [torch.empty(N, dtype=torch.float32).pin_memory() for _ in range(2)]
+        # host buffers in, host buffer out, every step; consecutive calls overlap their copies (the inputs of
+        # step t + 1 travel while step t runs and its update travels back), the last update is waited for
+        pr.step_host_async(gh[0], wh, uh[0])  # allocates the staging buffers
+        pr.host_wait()
         barrier()
         t0 = time.perf_counter()
         for t in range(e2e_steps):
-            pr.step_host(gh[t % len(gh)], wh, uh)
+            pr.step_host_async(gh[t % len(gh)], wh, uh[t % 2])
+        pr.host_wait()
         torch.cuda.synchronize()
         e2e_dt = time.perf_counter() - t0
         e2e_dt = max_over_ranks(e2e_dt, dist, dev)

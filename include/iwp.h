@@ -242,6 +242,18 @@ int iwp_encode_mask(iwp_ctx* ctx, const uint8_t* mask_dev, uint8_t* bits_dev);
 /* acc <- 0, step counter <- 0, status word <- 0. */
 int iwp_reset(iwp_ctx* ctx);
 
+/* The same with the copies of consecutive calls overlapped: the call enqueues the host-to-device copies on a
+ * copy stream of the library's own, the step on the context's stream and the copy of the update to
+ * update_host on a second copy stream, and returns without waiting.  Two staging sets are used in turn, so
+ * the inputs of call k + 1 travel while step k runs and while update k travels the other way.  The host
+ * buffers of a call must stay untouched until iwp_host_wait() (pinned memory is needed for the copies to
+ * overlap at all); update_host of call k is valid after iwp_host_wait() or once call k + 2 has returned
+ * and the context's stream has reached it.  Same errors as iwp_step_host(). */
+int iwp_step_host_async(iwp_ctx* ctx, const float* grads_host, const float* weights_host, float* update_host);
+
+/* Blocks until every iwp_step_host_async() call made so far has delivered its update. */
+int iwp_host_wait(iwp_ctx* ctx);
+
 /* Options (tests and experiments):
  *   "leader_override"  >= 0 forces the leader of every following step, -1 = seeded draw
  *   "force_scalar"     1 = never use 128-bit accesses

@@ -23,7 +23,7 @@ EXPORTS = [
     "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat", "iwp_select_static",
     "iwp_set_momentum", "iwp_create_threshold", "iwp_set_thresholds", "iwp_get_list_length", "iwp_leaders_at",
     "iwp_set_layerwise", "iwp_get_layer_thresholds", "iwp_shard_select", "iwp_shard_gather", "iwp_shard_apply",
-    "iwp_layer_leader_at", "iwp_encode_mask",
+    "iwp_layer_leader_at", "iwp_encode_mask", "iwp_step_host_async", "iwp_host_wait",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -62,6 +62,8 @@ def lib() -> C.CDLL:
         L.iwp_set_momentum.argtypes = [vp, f32]
         L.iwp_step.argtypes = [vp, vp, vp, vp]
         L.iwp_step_host.argtypes = [vp, vp, vp, vp]
+        L.iwp_step_host_async.argtypes = [vp, vp, vp, vp]
+        L.iwp_host_wait.argtypes = [vp]
         L.iwp_shard_select.argtypes = [vp, vp, vp, vp]
         L.iwp_shard_gather.argtypes = [vp, vp, i64, vp]
         L.iwp_shard_apply.argtypes = [vp, vp, i64, vp, i32, vp]
@@ -222,6 +224,18 @@ class Pruner:
             assert (not x.is_cuda) and x.dtype == t.float32 and x.is_contiguous() and x.numel() == n
         iwp_step_host(self._h, grads.data_ptr(), weights.data_ptr(), update.data_ptr())
         return update
+
+    def step_host_async(self, grads, weights, update) -> None:
+        """Like step_host, but returns at once; consecutive calls overlap their copies.  Pinned host tensors,
+        untouched until host_wait()."""
+        t = self._torch
+        for x, n in ((grads, self.W * self.N), (weights, self.N), (update, self.N)):
+            assert (not x.is_cuda) and x.dtype == t.float32 and x.is_contiguous() and x.numel() == n and x.is_pinned()
+        _check(lib().iwp_step_host_async(self._h, grads.data_ptr(), weights.data_ptr(), update.data_ptr()),
+               "iwp_step_host_async")
+
+    def host_wait(self) -> None:
+        _check(lib().iwp_host_wait(self._h), "iwp_host_wait")
 
     # the three phases of a step whose workers are spread over several contexts (see ShardedPruner)
     def shard_select(self, grads, weights, update) -> None:

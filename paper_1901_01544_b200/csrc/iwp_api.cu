@@ -100,6 +100,17 @@ struct iwp_ctx {
   float* stg_grads = nullptr;
   float* stg_weights = nullptr;
   float* stg_update = nullptr;
+  // double-buffered staging of iwp_step_host_async: set k & 1 serves call k
+  struct HostPipe {
+    float* grads[2] = {nullptr, nullptr};
+    float* weights[2] = {nullptr, nullptr};
+    float* update[2] = {nullptr, nullptr};
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t in_ready[2] = {nullptr, nullptr};   // the set's inputs have arrived
+    cudaEvent_t step_done[2] = {nullptr, nullptr};  // the step that used the set is through
+    cudaEvent_t out_done[2] = {nullptr, nullptr};   // the set's update has reached the host
+    int64_t calls = 0;
+  } pipe_host;
 };
 
 namespace {
@@ -250,6 +261,21 @@ void free_all(iwp_ctx* c) {
   cudaFree(c->stg_grads);
   cudaFree(c->stg_weights);
   cudaFree(c->stg_update);
+  {
+    iwp_ctx::HostPipe& hp = c->pipe_host;
+    for (cudaStream_t* q : {&hp.h2d, &hp.d2h})
+      if (*q) {
+        cudaStreamSynchronize(*q);
+        cudaStreamDestroy(*q);
+      }
+    for (int k = 0; k < 2; ++k) {
+      cudaFree(hp.grads[k]);
+      cudaFree(hp.weights[k]);
+      cudaFree(hp.update[k]);
+      for (cudaEvent_t e : {hp.in_ready[k], hp.step_done[k], hp.out_done[k]})
+        if (e) cudaEventDestroy(e);
+    }
+  }
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -1010,6 +1036,67 @@ int iwp_step_host(iwp_ctx* c, const float* grads, const float* weights, float* u
   if (rc != IWP_OK) return rc;
   if (cudaMemcpyAsync(update, c->stg_update, N * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
       cudaStreamSynchronize(s) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  return IWP_OK;
+}
+
+int iwp_step_host_async(iwp_ctx* c, const float* grads, const float* weights, float* update) {
+  if (!c || !grads || !weights || !update) return IWP_ERR_INVALID;
+  iwp_ctx::HostPipe& hp = c->pipe_host;
+  const uint64_t N = c->plan.N, W = static_cast<uint64_t>(c->plan.W);
+  if (!hp.h2d) {  // first call: two staging sets, a stream per copy direction, events
+    int rc = IWP_OK;
+    for (int k = 0; k < 2 && rc == IWP_OK; ++k) {
+      rc = dev_alloc(&hp.grads[k], W * N * sizeof(float));
+      if (rc == IWP_OK) rc = dev_alloc(&hp.weights[k], N * sizeof(float));
+      if (rc == IWP_OK) rc = dev_alloc(&hp.update[k], N * sizeof(float));
+    }
+    bool ok = rc == IWP_OK;
+    ok = ok && cudaStreamCreateWithFlags(&hp.h2d, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&hp.d2h, cudaStreamNonBlocking) == cudaSuccess;
+    for (int k = 0; k < 2; ++k)
+      for (cudaEvent_t* e : {&hp.in_ready[k], &hp.step_done[k], &hp.out_done[k]})
+        ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {  // free_all() releases whatever was made
+      cudaGetLastError();
+      return rc != IWP_OK ? rc : IWP_ERR_CUDA;
+    }
+  }
+  const int k = static_cast<int>(hp.calls & 1);
+  bool ok = true;
+  if (hp.calls >= 2) {  // the set's last user: its step has read the inputs, its update has left
+    ok = ok && cudaStreamWaitEvent(hp.h2d, hp.step_done[k], 0) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(c->stream, hp.out_done[k], 0) == cudaSuccess;
+  }
+  ok = ok && cudaMemcpyAsync(hp.grads[k], grads, W * N * sizeof(float), cudaMemcpyHostToDevice, hp.h2d) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(hp.weights[k], weights, N * sizeof(float), cudaMemcpyHostToDevice, hp.h2d) == cudaSuccess;
+  ok = ok && cudaEventRecord(hp.in_ready[k], hp.h2d) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(c->stream, hp.in_ready[k], 0) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  const int rc = iwp_step(c, hp.grads[k], hp.weights[k], hp.update[k]);
+  if (rc != IWP_OK) return rc;
+  ok = cudaEventRecord(hp.step_done[k], c->stream) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(hp.d2h, hp.step_done[k], 0) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(update, hp.update[k], N * sizeof(float), cudaMemcpyDeviceToHost, hp.d2h) == cudaSuccess;
+  ok = ok && cudaEventRecord(hp.out_done[k], hp.d2h) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  hp.calls += 1;
+  return IWP_OK;
+}
+
+int iwp_host_wait(iwp_ctx* c) {
+  if (!c) return IWP_ERR_INVALID;
+  iwp_ctx::HostPipe& hp = c->pipe_host;
+  if (!hp.d2h) return IWP_OK;
+  if (cudaStreamSynchronize(hp.d2h) != cudaSuccess || cudaStreamSynchronize(c->stream) != cudaSuccess) {
     cudaGetLastError();
     return IWP_ERR_CUDA;
   }

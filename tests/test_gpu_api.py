@@ -91,6 +91,31 @@ def test_host_buffer_entry_point_matches_oracle(overlap):
     pr.close()
 
 
+@pytest.mark.parametrize("overlap", [0, 1])
+def test_async_host_entry_point_matches_oracle(overlap):
+    sizes, W = [40000, 300, 20000], 4
+    N = sum(sizes)
+    weights, grads = _inputs(W, N, 5)
+    pr = Pruner(sizes, W, 64.0, 1e-8, 0)
+    pr.set_option("overlap", overlap)
+    orc = oracle.Oracle(sizes, W, 64.0, 1e-8, 0)
+    steps = 7
+    gh = [grads[t % len(grads)].cpu().pin_memory() for t in range(steps)]
+    wh = [(weights * (1.0 + 0.25 * t)).cpu().pin_memory() for t in range(steps)]
+    uh = [torch.full((N,), float("nan")).pin_memory() for _ in range(steps)]
+    for t in range(steps):  # all in flight, two staging sets in turn
+        pr.step_host_async(gh[t], wh[t], uh[t])
+    pr.host_wait()
+    for t in range(steps):
+        want = orc.step(gh[t].numpy(), wh[t].numpy())
+        assert_bits_equal(uh[t].numpy(), want, f"step {t}: update via the asynchronous host entry point")
+    assert pr.sync_status() == 0 and pr.t == steps
+    # the synchronous entry point afterwards, on the same context
+    pr.step_host(gh[0], wh[0], uh[0])
+    assert_bits_equal(uh[0].numpy(), orc.step(gh[0].numpy(), wh[0].numpy()), "synchronous call after asynchronous ones")
+    pr.close()
+
+
 def test_runs_on_a_side_stream():
     sizes, W = [60000], 2
     N = sum(sizes)
