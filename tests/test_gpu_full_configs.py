@@ -30,6 +30,18 @@ def test_full_size_every_output(name):
                residual_every=1 if name == "single_layer" else 3)
 
 
+@pytest.mark.parametrize("name", ["alexnet_w8", "resnet50_w8"])
+def test_full_size_steps_back_to_back(name):
+    # the schedule bench.py times: nobody asks for lists or residuals between steps, so the other workers'
+    # selects of a step run beside the next step's head; the weights change after every step
+    c = wl.CONFIGS[name]()
+    weights = c.weights(DEV)
+    base = weights.clone()
+    buf = torch.empty((c.W, c.N), dtype=torch.float32, device=DEV)
+    run_parity(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, 5, weights, lambda t: c.grads(t, DEV, out=buf),
+               residual_every=1000, state_every=1000, weights_fn=lambda t: base * (1.0 + 0.125 * t))
+
+
 def test_full_size_w32_stress():
     c = wl.alexnet_w32()
     steps = 8  # covers eight leader draws and the step-to-step threshold jumps; 20 steps run scaled elsewhere
