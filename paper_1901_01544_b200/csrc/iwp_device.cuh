@@ -24,7 +24,7 @@ constexpr int N_PASSES = 3;
 struct PairInfo {
   uint32_t guess;  // candidates include every element with importance pattern >= guess; GUESS_NONE = none
   uint32_t total;  // number of elements of the layer that reach the guess
-  uint32_t flags;  // bit 0: some (tile, worker) slot or staging queue overflowed
+  uint32_t flags;  // bit 0: some (tile, worker) slot overflowed
   uint32_t gm;     // bit pattern of the pre-test multiplier derived from the guess
 };
 

@@ -155,13 +155,13 @@ __global__ void __launch_bounds__(SAMPLE_THREADS)
 //
 // Cheap pre-test before the exact quotient: with gm = guess * (1 - 2^-20) every element whose
 // correctly rounded quotient |acc| / den reaches the guess passes |acc| >= gm * den (the two
-// roundings of gm * den and the one of the quotient are each below 2^-23 relative).  Elements that
-// pass are staged, in index order, in a per-warp queue in shared memory; the lanes then take one
-// entry each, form the exact quotient (one division per lane, not per element), count how many
-// really reach the guess, and append ALL staged entries with coalesced stores.  Keeping the few
-// entries that fall just short of the guess is harmless: whenever at least k elements of the layer
-// reach the guess, the k best of this superset are the k best of the layer.  The argument needs
-// normal products, so the pre-test is disabled (gm = 0: everything passes) for tiny guesses or eps.
+// roundings of gm * den and the one of the quotient are each below 2^-23 relative).  Only the
+// elements that pass (about 2 % at a keep ratio of 1/64) get the exact IEEE quotient: each lane
+// handles its own, in index order, and stores key, value and offset at the element's rank in the
+// slot.  Keeping the few entries that fall just short of the guess is harmless: whenever at least k
+// elements of the layer reach the guess, the k best of this superset are the k best of the layer.
+// The argument needs normal products, so the pre-test is disabled (gm = 0: everything passes) for
+// tiny guesses or eps.
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ float pretest_multiplier(uint32_t guess, float eps) {
   if (guess == GUESS_NONE) return __int_as_float(0x7f800000);  // +inf: nothing passes
@@ -171,7 +171,6 @@ __device__ __forceinline__ float pretest_multiplier(uint32_t guess, float eps) {
   return __fmul_rd(gf, 1.0f - 9.5367431640625e-07f);
 }
 
-constexpr int EMIT_QUEUE = 128;  // staged entries per warp and iteration; more than this = overflow
 
 // Candidate entries are re-read several times by the select right after the streaming pass: store
 // them with an L2 evict-last policy so that the 6 GB that stream through L2 meanwhile do not push
@@ -210,9 +209,6 @@ __global__ void __launch_bounds__(THREADS, 3)
              uint2* __restrict__ lead_lane, uint32_t* __restrict__ lead_tot, const uint32_t* __restrict__ zmask,
              float eps, uint64_t N, int W, int leader, uint32_t n_tiles, int worker_groups, float momentum) {
   constexpr int ROUNDS = SEG_ELEMS / 128;  // 128-bit slots per lane and iteration = 4
-  __shared__ float q_val[WARPS][EMIT_QUEUE];
-  __shared__ float q_den[WARPS][EMIT_QUEUE];
-  __shared__ uint16_t q_loc[WARPS][EMIT_QUEUE];
   __shared__ __align__(16) float r_val[WARPS][SEG_ELEMS];  // results of the iteration, for run-time indexing
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t tile_id;
@@ -240,13 +236,9 @@ __global__ void __launch_bounds__(THREADS, 3)
   float* a = acc + static_cast<uint64_t>(w) * N;
   const uint64_t slot = (static_cast<uint64_t>(tile_id) * W + w) * CAND_CAP;
   const float zero[4] = {0.f, 0.f, 0.f, 0.f};
-  float* qv = q_val[warp];
-  float* qd = q_den[warp];
-  uint16_t* ql = q_loc[warp];
   float* res = r_val[warp] + lane * 4;
   uint32_t count = 0;    // entries appended to the slot so far (the same in every lane)
-  uint32_t reached = 0;  // of those, how many reach the guess exactly
-  bool overflow = false;
+  uint32_t reached = 0;  // of those, how many reach the guess exactly (this lane's share until the final reduction)
   const uint64_t keep = l2_evict_last_policy();
   // The tile covers the segments it0 .. it1 of its window.  The loads of segment it + 1 are issued
   // as soon as the arithmetic of segment it is done, so they are in flight while the rare-path work
@@ -375,42 +367,26 @@ __global__ void __launch_bounds__(THREADS, 3)
       if (lane == 0) lead_tot[sigma] = tot;
     }
     if (any) {
+      // every lane takes its own elements that passed the pre-test: exact quotient, then key, value and
+      // offset straight to the slot at the element's rank (the ranks of a warp's elements are consecutive,
+      // so the stores of one trip fall into a few sectors)
       for (uint32_t mm = m; mm; mm &= mm - 1) {
         const uint32_t b = __ffs(mm) - 1;
-        const uint32_t pos = staged_position(m, excl, tot, b);
-        if (pos < EMIT_QUEUE) {
-          const uint32_t off = (b >> 2) * 128 + (b & 3u);
-          qv[pos] = res[off];
-          qd[pos] = imp_den(weights[first + off], eps);  // re-read through L1: only staged elements get here
-          ql[pos] = static_cast<uint16_t>(static_cast<uint32_t>(first - base) + off);
+        const uint32_t pos = count + staged_position(m, excl, tot, b);
+        const uint32_t off = (b >> 2) * 128 + (b & 3u);
+        const float v = res[off];
+        const uint32_t key = imp_key_den(v, imp_den(weights[first + off], eps));  // weight re-read through L1
+        reached += (key >= guess) ? 1u : 0u;
+        if (pos < CAND_CAP) {
+          st_keep_u32(cand_key + slot + pos, key, keep);
+          st_keep_f32(cand_val + slot + pos, v, keep);
+          st_keep_u16(cand_idx + slot + pos, static_cast<uint16_t>(static_cast<uint32_t>(first - base) + off), keep);
         }
       }
-      uint32_t nq = (tot & 0xFFu) + ((tot >> 8) & 0xFFu) + ((tot >> 16) & 0xFFu) + (tot >> 24);
-      if (nq > EMIT_QUEUE) {
-        overflow = true;
-        nq = EMIT_QUEUE;
-      }
-      __syncwarp();
-      for (uint32_t j0 = 0; j0 < nq; j0 += 32) {
-        const uint32_t j = j0 + lane;
-        bool hit = false;
-        if (j < nq) {
-          const float v = qv[j];
-          const uint32_t key = imp_key_den(v, qd[j]);  // Algorithm 1's |grad / w|, exactly rounded
-          hit = key >= guess;
-          const uint32_t pos = count + j;
-          if (pos < CAND_CAP) {
-            st_keep_u32(cand_key + slot + pos, key, keep);
-            st_keep_f32(cand_val + slot + pos, v, keep);
-            st_keep_u16(cand_idx + slot + pos, ql[j], keep);
-          }
-        }
-        reached += __popc(__ballot_sync(0xffffffffu, hit));
-      }
-      count += nq;
-      __syncwarp();
+      count += (tot & 0xFFu) + ((tot >> 8) & 0xFFu) + ((tot >> 16) & 0xFFu) + (tot >> 24);
     }
   }
+  reached = __reduce_add_sync(0xffffffffu, reached);
   // pad the slot to a multiple of four entries with key 0, so that readers can take whole 128-bit
   // groups without testing every entry (no candidate has key 0: a zero guess is never used)
   {
@@ -421,7 +397,7 @@ __global__ void __launch_bounds__(THREADS, 3)
   if (lane == 0) {
     st_keep_u32(cand_cnt + static_cast<uint64_t>(tile_id) * W + w, count, keep);
     if (reached) atomicAdd(&info[pair].total, reached);
-    if (overflow || count > CAND_CAP) atomicOr(&info[pair].flags, 1u);
+    if (count > CAND_CAP) atomicOr(&info[pair].flags, 1u);  // more candidates than the slot holds: exact fallback
   }
 }
 
