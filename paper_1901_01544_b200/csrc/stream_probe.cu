@@ -222,7 +222,8 @@ int main(int argc, char** argv) {
   int sm_count = 148;
   cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, 0);
   std::printf("a += g over 2 x %.2f GB (read 2, write 1), best of 5 timed launches each\n", n * 4 / 1e9);
-  run_walk(b, "plain loads, 4 rounds, 7 warps, 26 KB smem (the library's shape)", k_walk<4, 7, 3>, 7, 26624);
+  run_walk(b, "plain loads, 4 rounds, 7 warps, 16 KB smem (the library's shape)", k_walk<4, 7, 3>, 7, 16384);
+  run_walk(b, "plain loads, 4 rounds, 7 warps, 26 KB smem", k_walk<4, 7, 3>, 7, 26624);
   run_walk(b, "plain loads, 4 rounds, 8 warps, 26 KB smem", k_walk<4, 8, 3>, 8, 26624);
   run_walk(b, "plain loads, 4 rounds, 8 warps, 26 KB smem, 4 CTAs wanted", k_walk<4, 8, 4>, 8, 26624);
   run_walk(b, "plain loads, 8 rounds, 8 warps, 26 KB smem", k_walk<8, 8, 3>, 8, 26624);
