@@ -60,6 +60,7 @@ def _run(sizes, W, thr, weights, grads_fn, steps, seed=3, momentum=None, max_lis
         assert_bits_equal(gv.cpu().numpy()[: len(oi)], ov, f"step {t}: values")
         assert_bits_equal(upd.cpu().numpy(), want, f"step {t}: update")
         assert np.array_equal(pr.mask().cpu().numpy(), orc.mask()), f"step {t}: mask"
+        assert np.array_equal(pr.mask_bits().cpu().numpy(), np.packbits(orc.mask(), bitorder="little")), f"step {t}: packed mask"
         if (t + 1) % residual_every == 0 or t == steps - 1:
             for w in range(W):
                 assert_bits_equal(pr.residual(w).cpu().numpy(), orc.residual(w), f"step {t}: worker {w} residual")

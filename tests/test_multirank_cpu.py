@@ -157,3 +157,32 @@ def test_workers_spread_over_two_ranks_equal_one_node():
         assert p.exitcode == 0
     assert [g[1] for g in got] == [True, True]
     assert got[0][2] == [0, 1]  # the chosen worker lived on either rank at some step
+
+
+def _sharded_bad_split_main(rank: int, world: int, port: int, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_1901_01544_b200.binding import ShardedPruner
+
+    try:
+        ShardedPruner([100], 3, 4.0, engine=_NumpyEngine([100], 1, 4.0, 1e-8))  # three workers over two ranks
+        out.put((rank, "accepted"))
+    except ValueError:
+        out.put((rank, "rejected"))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_sharding_needs_the_workers_to_divide_over_the_ranks():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_sharded_bad_split_main, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert got == [(0, "rejected"), (1, "rejected")]
