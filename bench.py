@@ -406,6 +406,14 @@ def run_ours(args):
         "algorithmic_bytes_per_step_of_kernel": k1_bytes, "ms_per_step_of_kernel": k1_ms,
         "launches_per_step": k1_launches, "traffic_note": k1_note,
     }
+    if stage_ms is not None:
+        # the same kernel with nothing beside it (the serial stage pass): in the timed region the selects of
+        # the overlapped schedule share the GPU with it
+        alone_ms = stage_ms["gather" if args.mode == "threshold" else "accumulate"]
+        if alone_ms > 0:
+            alone = k1_bytes / (alone_ms * 1e-3) / 1e9
+            roofline["alone"] = {"ms_per_step_of_kernel": alone_ms, "achieved": alone, "frac": alone / peak,
+                                 "note": "separate serial pass, no other kernel running beside it"}
     eff = B / (ms_per_step * 1e-3) / 1e9
     step_eff = {"compulsory_bytes": B, "effective_gbs": eff, "frac_of_measured_peak": eff / peak,
                 "frac_of_nominal_8tbs": eff / NOMINAL_HBM_GBS}
