@@ -874,3 +874,66 @@ def test_per_layer_leaders_equal_bruteforce():
         for w in range(W):
             assert np.array_equal(u32(orc.residual(w)), u32(acc[w]))
     assert len(used) > 1
+
+
+# ---------------------------------------------------------------- property tests (hypothesis)
+
+
+def test_selection_properties_on_arbitrary_small_layers():
+    from hypothesis import given, settings
+    from hypothesis import strategies as st
+
+    values = st.sampled_from([0.0, -0.0, 0.25, -0.25, 0.5, 1.0, -2.0, 3.0e-39, 1.0e30])  # ties, zeros, a denormal
+    weights = st.sampled_from([0.0, 0.5, -0.5, 1.0, 2.0])
+
+    @settings(max_examples=200, deadline=None)
+    @given(st.lists(st.tuples(values, weights), min_size=1, max_size=40), st.integers(1, 40))
+    def check(pairs, k):
+        acc = np.array([p[0] for p in pairs], np.float32)
+        w = np.array([p[1] for p in pairs], np.float32)
+        k = min(k, acc.size)
+        got = oracle.select(acc, w, k, 1e-8).tolist()
+        imp = [bits(importance(a, b, F(1e-8))) for a, b in zip(acc, w)]
+        assert got == sorted(got) and len(set(got)) == k  # ascending, distinct, exactly k
+        inside, outside = [imp[i] for i in got], [imp[i] for i in range(acc.size) if i not in got]
+        if outside:
+            t = min(inside)
+            assert t >= max(outside)  # nothing left out beats anything kept
+            # at the threshold value the kept indices are the lowest ones
+            at_t_in = [i for i in got if imp[i] == t]
+            at_t_out = [i for i in range(acc.size) if i not in got and imp[i] == t]
+            assert not at_t_out or max(at_t_in) < min(at_t_out)
+
+    check()
+
+
+def test_step_conserves_every_element_exactly():
+    from hypothesis import given, settings
+    from hypothesis import strategies as st
+
+    @settings(max_examples=40, deadline=None)
+    @given(st.integers(0, 2**31 - 1), st.integers(1, 4), st.sampled_from([1.0, 2.0, 7.0, 64.0]), st.integers(1, 3))
+    def check(seed, W, ratio, n_leaders):
+        rng = np.random.default_rng(seed)
+        layers = [int(x) for x in rng.integers(1, 30, size=3)]
+        N = sum(layers)
+        orc = oracle.Oracle(layers, W, ratio, 1e-8, seed=seed)
+        orc.set_n_leaders(min(n_leaders, W))
+        weights = (rng.integers(-2, 3, N) * 0.5).astype(np.float32)
+        before = np.zeros((W, N), np.float32)
+        for t in range(3):
+            g = (rng.integers(-4, 5, size=(W, N)) / 4.0).astype(np.float32)
+            upd = orc.step(g, weights)
+            mask = orc.mask().astype(bool)
+            after = np.stack([orc.residual(w) for w in range(W)])
+            acc = (before + g).astype(np.float32)
+            assert not after[:, mask].any()  # what was sent has left every residual
+            assert np.array_equal(u32(after[:, ~mask]), u32(acc[:, ~mask]))  # the rest is untouched
+            assert not upd[~mask].any()  # nothing outside the index set
+            s = acc[0].copy()
+            for w in range(1, W):
+                s = (s + acc[w]).astype(np.float32)
+            assert np.array_equal(u32(upd[mask]), u32((F(0) + s)[mask]))  # the ordered sum inside it
+            before = after
+
+    check()
