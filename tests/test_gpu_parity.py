@@ -426,3 +426,31 @@ def test_random_option_changes_between_steps(seed):
     pr.set_option("time_stages", 0)
     pr.close()
     orc.close()
+
+
+# ------------------------------------------------------------------ seeded random shapes
+
+
+@pytest.mark.parametrize("seed", range(int(os.environ.get("IWP_SHAPE_SEEDS", "10"))))
+def test_random_shapes(seed):
+    """Layer lists drawn around the sizes where the code changes behaviour (one-CTA limit, tile and chunk edges,
+    vector alignment), with random worker counts, ratios and schedules."""
+    rng = np.random.default_rng(4000 + seed)
+    edges = [1, 3, 4, 5, 4095, 4096, 4097, 8191, 16383, 16384, 16385, 16388, 65535, 65536, 65537, 128 * 4096, 128 * 4096 + 1]
+    n_layers = int(rng.integers(1, 7))
+    sizes = [int(rng.choice(edges)) if rng.random() < 0.7 else int(rng.integers(1, 200000)) for _ in range(n_layers)]
+    if rng.random() < 0.5 and sum(sizes) % 4:  # half of the cases on the vector path
+        sizes[-1] += 4 - sum(sizes) % 4
+    W = int(rng.integers(1, 10))
+    ratio = float(rng.choice([1.0, 2.0, 7.0, 58.8, 64.0, 1000.0]))
+    N = sum(sizes)
+    weights = _weights(N, 50 + seed)
+    coarse = rng.random() < 0.3
+    def grads(t):
+        if coarse:
+            return torch.randint(-4, 5, (W, N), device=DEV, generator=torch.Generator(device=DEV).manual_seed(seed * 100 + t)).float() / 8.0
+        return _randn((W, N), 7000 + seed * 100 + t, 1e-2)
+    run_parity(sizes, W, ratio, 1e-8, seed=seed, steps=4, weights=weights, grads_fn=grads,
+               options={"overlap": int(rng.integers(0, 2)), "speculate": int(rng.random() < 0.8)},
+               n_leaders=int(rng.integers(1, min(W, 3) + 1)), momentum=float(rng.choice([1.0, 0.9])),
+               state_every=int(rng.choice([1, 2])), residual_every=int(rng.choice([1, 1000])))
