@@ -267,3 +267,28 @@ def test_layerwise_threshold_full_size_alexnet_shape():
     buf = torch.empty((c.W, c.N), dtype=torch.float32, device=DEV)
     _run(c.layer_sizes, c.W, None, weights, lambda t: c.grads(t, DEV, out=buf), steps=2, seed=c.seed,
          layerwise=(0.05, 1e-4, 100.0), residual_every=2)
+
+
+# ------------------------------------------------------------------ seeded random shapes and options
+
+
+@pytest.mark.parametrize("seed", range(int(__import__("os").environ.get("IWP_SHAPE_SEEDS", "8"))))
+def test_threshold_mode_random_shapes(seed):
+    rng = np.random.default_rng(6000 + seed)
+    edges = [1, 3, 4, 5, 4095, 4096, 4097, 16383, 16384, 16385, 32767, 32768, 32769, 65537, 8 * 4096, 8 * 4096 + 1]
+    sizes = [int(rng.choice(edges)) if rng.random() < 0.7 else int(rng.integers(1, 150000)) for _ in range(int(rng.integers(1, 6)))]
+    if rng.random() < 0.5 and sum(sizes) % 4:
+        sizes[-1] += 4 - sum(sizes) % 4
+    W = int(rng.integers(1, 8))
+    N = sum(sizes)
+    weights = _randn((N,), 8000 + seed, 0.05)
+    weights[:: int(rng.integers(7, 100))] = 0.0
+    n_leaders = int(rng.integers(1, min(W, 4) + 1))
+    kw = dict(steps=3, seed=seed, n_leaders=n_leaders, random_select=bool(rng.random() < 0.4),
+              momentum=float(rng.choice([1.0, 0.5])), residual_every=int(rng.choice([1, 1000])))
+    grads = lambda t: _randn((W, N), 9000 + 10 * seed + t, 1e-2)
+    if rng.random() < 0.5:
+        _run(sizes, W, None, weights, grads, layerwise=(float(rng.choice([0.0, 0.3, 2.0])), float(rng.choice([0.0, 1e-6, 0.05])),
+                                                        float(rng.choice([0.0, 5.0, 1e9]))), **kw)
+    else:
+        _run(sizes, W, [float(rng.choice([0.0, 0.05, 0.5, 50.0])) for _ in sizes], weights, grads, **kw)
