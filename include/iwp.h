@@ -271,6 +271,12 @@ int iwp_host_wait(iwp_ctx* ctx);
  *                      u < importance / thr (fp32 quotient), u = u24 * 2^-24 with
  *                      u24 = mix64(seed + (t+1)*0x9E3779B97F4A7C15 + (i+1)*0xC2B2AE3D27D4EB4F) >> 40
  *                      for element i at step t; 0 (default) = off
+ *   "leader_only_select" ratio-mode contexts only: 1 = only the chosen node of a step selects and lists
+ *                      (Algorithm 1 consumes no other worker's index set); update, the chosen node's list,
+ *                      mask and every residual are those of the default; iwp_get_selection() of any other
+ *                      worker then returns unspecified contents.  Ignored with several chosen nodes, with
+ *                      "per_layer_leaders" and in the sharded phases.  0 (default) = every worker lists
+ *                      its own top-k
  *   "speculate"        1 (default) = sample-based threshold guess so that large layers are
  *                      read once; 0 = always the multi-pass exact select.  Both are exact.
  *   "overlap"          1 = the leader's select runs beside the other workers' streaming pass and the
@@ -321,9 +327,18 @@ int iwp_get_stat(iwp_ctx* ctx, const char* key, int64_t* value_host);
  * calls on a device share the one scratch array (it keeps the previous call's contents; the entry
  * point clears what must start at zero), so two calls whose kernels can overlap on the GPU - on
  * different streams, or from different threads - race: serialise them.
- * Errors: IWP_ERR_INVALID (NULL pointer, n out of range, bad ratio or eps), IWP_ERR_CUDA. */
+ * Errors: IWP_ERR_INVALID (NULL pointer, n out of range, bad ratio or eps), IWP_ERR_CUDA.  The return
+ * value covers the arguments and the launches only; the kernels' own count checks (they fail on
+ * non-finite inputs or when two calls raced) are read back with iwp_select_static_status(). */
 int iwp_select_static(const float* residual_dev, const float* weights_dev, int64_t n, double ratio, float eps,
                       uint32_t* idx_dev, float* val_dev, int64_t* k_host, void* cuda_stream);
+
+/* Device status word of the last iwp_select_static() call on the current device: copies it to
+ * *status_host behind everything enqueued on cuda_stream and waits for that stream.  0, or
+ * IWP_ERR_INTERNAL when a count check of the select or the compaction failed (the list is then not to be
+ * trusted).  Allocates nothing.  Errors: IWP_ERR_INVALID (NULL pointer, or no call was made on this
+ * device yet), IWP_ERR_CUDA. */
+int iwp_select_static_status(int32_t* status_host, void* cuda_stream);
 
 #ifdef __cplusplus
 }

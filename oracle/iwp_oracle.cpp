@@ -21,8 +21,7 @@
 //   * importance = |G| / (|w| + eps), eps > 0, instead of the unguarded |G / w|.
 //   * the threshold of Algorithm 1 is the k-th largest importance of the worker's
 //     layer, k = ceil(n / ratio) clamped to [1, n]; ties keep the lower index.
-//   * one randomly chosen node per step supplies the index set (Section 3.2:
-//     "randomly choose a node and broadcast its important gradient index"); optionally several chosen
+//   * one randomly chosen node per step supplies the index set (Section 3.2); optionally several chosen
 //     nodes r_1..r_n, drawn without replacement, whose index sets are OR-ed (Algorithm 1: Mask = OR Mask_ri),
 //     or one chosen node per LAYER (Algorithm 1 draws the node inside its loop over layers).
 //   * Eq. 3's momentum acts on the locally kept residual: G <- m * G + grad (two roundings);

@@ -23,7 +23,7 @@ EXPORTS = [
     "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat", "iwp_select_static",
     "iwp_set_momentum", "iwp_create_threshold", "iwp_set_thresholds", "iwp_get_list_length", "iwp_leaders_at",
     "iwp_set_layerwise", "iwp_get_layer_thresholds", "iwp_shard_select", "iwp_shard_gather", "iwp_shard_apply",
-    "iwp_layer_leader_at", "iwp_encode_mask", "iwp_step_host_async", "iwp_host_wait",
+    "iwp_layer_leader_at", "iwp_encode_mask", "iwp_step_host_async", "iwp_host_wait", "iwp_select_static_status",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -82,6 +82,7 @@ def lib() -> C.CDLL:
         L.iwp_set_option.argtypes = [vp, cp, i64]
         L.iwp_get_stat.argtypes = [vp, cp, vp]
         L.iwp_select_static.argtypes = [vp, vp, i64, f64, f32, vp, vp, vp, vp]
+        L.iwp_select_static_status.argtypes = [vp, vp]
         for name in EXPORTS:
             getattr(L, name)  # AttributeError if the library does not export a declared symbol
         _lib = L
@@ -156,6 +157,13 @@ def iwp_select_static(residual_ptr: int, weights_ptr: int, n: int, ratio: float,
     _check(lib().iwp_select_static(residual_ptr, weights_ptr, n, ratio, eps, idx_ptr, val_ptr, C.byref(k),
                                    C.c_void_p(stream)), "iwp_select_static")
     return int(k.value)
+
+
+def iwp_select_static_status(stream: int = 0) -> int:
+    """Device status word of the last iwp_select_static() call on the current device (waits for `stream`)."""
+    v = C.c_int32()
+    _check(lib().iwp_select_static_status(C.byref(v), C.c_void_p(stream)), "iwp_select_static_status")
+    return int(v.value)
 
 
 # ---- convenience wrapper over torch tensors ----------------------------------------------------

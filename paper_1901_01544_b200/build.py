@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libiwp.so")
 SOURCES = [os.path.join(CSRC, "iwp_api.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("iwp_kernels.cuh", "iwp_device.cuh", "iwp_stream.cuh", "iwp_select.cuh", "iwp_reduce.cuh",
+DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("iwp_device.cuh", "iwp_stream.cuh", "iwp_select.cuh", "iwp_reduce.cuh",
                                             "iwp_threshold.cuh", "iwp_plan.hpp")] + [
     os.path.join(os.path.dirname(HERE), "include", "iwp.h")
 ]
@@ -45,26 +45,5 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
-PROBE = os.path.join(HERE, "stream_probe")
-PROBE_SOURCE = os.path.join(CSRC, "stream_probe.cu")
-
-
-def build_probe(force: bool = False) -> str:
-    """The stand-alone bandwidth probe (csrc/stream_probe.cu): what the streaming pass's shape can reach."""
-    if not force and os.path.exists(PROBE) and os.path.getmtime(PROBE) >= os.path.getmtime(PROBE_SOURCE):
-        return PROBE
-    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", PROBE_SOURCE, "-o", PROBE + ".tmp"]
-    r = subprocess.run(cmd, capture_output=True, text=True)
-    if r.returncode != 0:
-        sys.stderr.write(r.stdout + r.stderr)
-        raise RuntimeError("nvcc failed building stream_probe")
-    os.replace(PROBE + ".tmp", PROBE)
-    return PROBE
-
-
 if __name__ == "__main__":
-    if "--probe" in sys.argv:
-        print(build_probe(force=True))
-    else:
-        print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv))

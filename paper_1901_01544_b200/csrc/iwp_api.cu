@@ -1,5 +1,16 @@
 // C ABI of the importance-weighted pruning step (see include/iwp.h): argument checks,
 // the host planner, device memory owned by a context, and the launch sequence of a step.
+//
+// The sm_100a kernels live in the headers included below, by step of the path (Algorithm 1 of the paper):
+//   iwp_device.cuh     shared device helpers (importance arithmetic, vector loads, scans, radix select)
+//   iwp_stream.cuh     (a)+(b): accumulate, threshold guess from a sample, single-read streaming pass
+//   iwp_select.cuh     (c)+(d): exact radix select, ordered compaction, one-CTA path of small layers
+//   iwp_reduce.cuh     (e)-(g): reduction at the index set, zero mask, sharded phases, mask accessor
+//   iwp_threshold.cuh  absolute-threshold mode, random selection, layer-wise threshold
+// Nothing here is a dense contraction, so there are no tensor-core instructions: every kernel is bound by
+// HBM traffic (or, for the small ones, by launch latency).  The residual add, the eps guard and the division
+// use the explicit round-to-nearest intrinsics, so results do not depend on compiler contraction or fast-math
+// flags, and denormals are kept.
 #include "../../include/iwp.h"
 
 #include <cuda_runtime.h>
@@ -10,8 +21,12 @@
 #include <new>
 #include <vector>
 
-#include "iwp_kernels.cuh"
+#include "iwp_device.cuh"
 #include "iwp_plan.hpp"
+#include "iwp_reduce.cuh"
+#include "iwp_select.cuh"
+#include "iwp_stream.cuh"
+#include "iwp_threshold.cuh"
 
 using namespace iwp;
 
@@ -27,6 +42,7 @@ struct iwp_ctx {
   bool force_scalar = false;
   bool speculate = true;
   bool select_only = false;  // iwp_shard_select(): a step stops before the reduction
+  bool leader_only_select = false;  // option: only the chosen node selects; the other workers' lists are not produced
   cudaStream_t stream = nullptr;
   cudaStream_t side = nullptr;       // the one-CTA path of small layers runs here, beside the tiled path
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr, ev_fork2 = nullptr, ev_join2 = nullptr;
@@ -39,6 +55,7 @@ struct iwp_ctx {
   cudaEvent_t ev_lead = nullptr, ev_lead_done = nullptr, ev_others = nullptr, ev_a2 = nullptr, ev_b = nullptr;
   bool pending_a2 = false, pending_b = false;  // deferred selects of the last step not yet joined
   int32_t predicted_next = -1;                 // the worker whose select pending_a2 covers
+  int32_t last_only = -1;                      // the last step selected for this worker alone (-1: for every worker)
   float* saved_w = nullptr;                    // [N] weights kept for deferred selects that fall back (k_save_weights)
   int device = 0;
   int64_t launches = 0;
@@ -53,6 +70,7 @@ struct iwp_ctx {
   uint32_t* d_large_ids = nullptr;
   uint2* d_state = nullptr;
   uint32_t* d_hist = nullptr;
+  uint32_t* d_reach = nullptr;    // [pair] candidates reaching the guess as the first histogram pass saw them (count check)
   uint2* d_chunk_cnt = nullptr;
   PairInfo* d_info = nullptr;     // threshold guess and candidate totals per pair, two copies used in turn
   PairInfo* info_cur = nullptr;   // the copy the last step used
@@ -145,11 +163,11 @@ void stage_clear(iwp_ctx* c) {
 }
 
 struct Sizes {
-  uint64_t acc, layers, tiles, chunks, small_ids, large_ids, state, hist, chunk_cnt, sel_idx, sel_val, status;
+  uint64_t acc, layers, tiles, chunks, small_ids, large_ids, state, hist, reach, chunk_cnt, sel_idx, sel_val, status;
   uint64_t info, cand_key, cand_val, cand_idx, cand_cnt, guess, side_val, sel_slot, lead_lane, lead_tot, zmask, chunk_sfx;
   uint64_t saved_w;
   uint64_t total() const {
-    return acc + layers + tiles + chunks + small_ids + large_ids + state + hist + chunk_cnt + sel_idx + sel_val +
+    return acc + layers + tiles + chunks + small_ids + large_ids + state + hist + reach + chunk_cnt + sel_idx + sel_val +
            status + info + cand_key + cand_val + cand_idx + cand_cnt + guess + side_val + sel_slot + lead_lane +
            lead_tot + zmask + chunk_sfx + saved_w;
   }
@@ -170,6 +188,7 @@ Sizes sizes_of(const Plan& p, bool threshold_mode = false, uint64_t list_cap = 0
   s.large_ids = at_least(p.large_layers.size() * sizeof(uint32_t));
   s.state = at_least(pairs * sizeof(uint2));
   s.hist = at_least(pairs * NBINS * sizeof(uint32_t));
+  s.reach = at_least(pairs * sizeof(uint32_t));
   s.chunk_cnt = at_least((threshold_mode ? 0 : W) * p.chunks.size() * sizeof(uint2));
   s.sel_idx = threshold_mode ? at_least(list_cap * sizeof(uint32_t)) : W * p.K * sizeof(uint32_t);
   s.sel_val = threshold_mode ? at_least(list_cap * sizeof(float)) : W * p.K * sizeof(float);
@@ -235,6 +254,7 @@ void free_all(iwp_ctx* c) {
   cudaFree(c->d_large_ids);
   cudaFree(c->d_state);
   cudaFree(c->d_hist);
+  cudaFree(c->d_reach);
   cudaFree(c->d_chunk_cnt);
   cudaFree(c->d_info);
   cudaFree(c->cand_key);
@@ -325,10 +345,11 @@ int select_and_write(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSe
   uint32_t* sfx = c->chunk_sfx;
   for (int pass = 0; pass < N_PASSES; ++pass) {
     k_hist<VEC><<<cgrid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_layers, c->info_cur, c->cand_key,
-                                           c->cand_cnt, c->d_state, c->d_hist, sfx, c->d_chunk_cnt, c->eps, p.N, W,
-                                           pass, n_chunks, ws);
+                                           c->cand_cnt, c->d_state, c->d_hist, sfx, c->d_chunk_cnt, c->d_reach, c->eps, p.N,
+                                           W, pass, n_chunks, ws);
     IWP_LAUNCH_CHECK(c);
-    k_find_digit<<<pgrid, THREADS, 0, st>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->d_status, W, pass, ws);
+    k_find_digit<<<pgrid, THREADS, 0, st>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->info_cur, c->d_reach,
+                                            c->d_status, W, pass, ws);
     IWP_LAUNCH_CHECK(c);
   }
   k_write<VEC><<<cgrid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur, c->cand_key,
@@ -368,6 +389,10 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   c->last_chosen = ls;
   const bool per_layer = c->per_layer_leaders && c->leader_override < 0 && ls.n == 1 && !c->select_only;
   c->last_per_layer = per_layer;
+  // only the chosen node's list is consumed by the step: with the option on, nobody else selects
+  const bool only = c->leader_only_select && W > 1 && ls.n == 1 && !per_layer && !c->select_only;
+  const int only_w = only ? leader : -1;
+  c->last_only = only_w;
   // the overlapped schedule (not while every stage boundary is being timed)
   const bool pipe = spec && W > 1 && ls.n == 1 && !per_layer && !c->select_only && c->overlap == 1 && c->time_stages != 1 &&
                     c->side_a != nullptr && c->side_b != nullptr;
@@ -393,7 +418,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
       ss = c->side;
     }
     k_small<<<grid, THREADS, dyn, ss>>>(grads, weights, c->acc, update, c->d_layers, c->d_small_ids, c->sel_idx,
-                                        c->sel_val, c->sel_slot, c->d_status, c->eps, N, K, leader, c->momentum);
+                                        c->sel_val, c->sel_slot, c->d_status, c->eps, N, K, leader, only_w, c->momentum);
     IWP_LAUNCH_CHECK(c);
     if (fork_small && !cuda_ok(cudaEventRecord(c->ev_join, c->side))) return IWP_ERR_CUDA;
   }
@@ -411,7 +436,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     const size_t dyn = static_cast<size_t>(c->max_sample) * sizeof(uint32_t);
     k_sample<<<c->n_pairs, SAMPLE_THREADS, dyn, s>>>(grads, weights, c->acc, c->d_layers, c->d_large_ids, c->info_cur,
                                                      c->d_guess, c->zmask, c->eps, N, W, static_cast<uint32_t>(c->t),
-                                                     c->momentum);
+                                                     only_w, c->momentum);
     IWP_LAUNCH_CHECK(c);
     c->info_clean = false;
   }
@@ -455,13 +480,14 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     stage_mark_at(c, 3);
     stage_mark_at(c, 4);
     stage_mark_at(c, 5);
+    const int32_t next = leader_of_step(c, c->t + 1);
+    if (!only) {
     // The other workers' selects outlive the step: they read the library's copy of the weights
     // (filled only where a pair fell back), the next step's leader first (its streaming pass comes first).
     k_save_weights<<<static_cast<unsigned>(p.chunks.size()), THREADS, 0, s>>>(weights, c->saved_w, c->d_chunks, c->d_layers,
                                                                             c->info_cur, W, leader);
     IWP_LAUNCH_CHECK(c);
     if (!cuda_ok(cudaEventRecord(c->ev_others, s))) return IWP_ERR_CUDA;
-    const int32_t next = leader_of_step(c, c->t + 1);
     if (next != leader) {
       if (!cuda_ok(cudaStreamWaitEvent(c->side_a, c->ev_others, 0))) return IWP_ERR_CUDA;
       rc = select_and_write<VEC>(c, c->saved_w, c->side_a, WorkerSel{WorkerSel::ONLY, next, -1}, leader);
@@ -476,6 +502,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
       if (rc != IWP_OK) return rc;
       if (!cuda_ok(cudaEventRecord(c->ev_b, c->side_b))) return IWP_ERR_CUDA;
       c->pending_b = true;
+    }
     }
     c->predicted_next = next;
     // the reduction needs the leader's list and the small layers
@@ -518,22 +545,23 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
   bool join_others = false;  // the other workers' lists are still being written on the side stream
   if (tiled) {
     const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
-    dim3 cgrid(n_chunks, static_cast<unsigned>(W)), pgrid(static_cast<unsigned>(p.large_layers.size()), static_cast<unsigned>(W));
-    const WorkerSel all{WorkerSel::ALL, 0, -1};
+    const WorkerSel all = only ? WorkerSel{WorkerSel::ONLY, leader, -1} : WorkerSel{WorkerSel::ALL, 0, -1};
+    const unsigned n_sel = static_cast<unsigned>(sel_count(all, W));
+    dim3 cgrid(n_chunks, n_sel), pgrid(static_cast<unsigned>(p.large_layers.size()), n_sel);
     for (int pass = 0; pass < N_PASSES; ++pass) {
       k_hist<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->info_cur, c->cand_key,
-                                            c->cand_cnt, c->d_state, c->d_hist, c->chunk_sfx, c->d_chunk_cnt, c->eps, N,
-                                            W, pass, n_chunks, all);
+                                            c->cand_cnt, c->d_state, c->d_hist, c->chunk_sfx, c->d_chunk_cnt, c->d_reach,
+                                            c->eps, N, W, pass, n_chunks, all);
       IWP_LAUNCH_CHECK(c);
-      k_find_digit<<<pgrid, THREADS, 0, s>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->d_status, W, pass,
-                                             all);
+      k_find_digit<<<pgrid, THREADS, 0, s>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->info_cur, c->d_reach,
+                                             c->d_status, W, pass, all);
       IWP_LAUNCH_CHECK(c);
     }
     stage_mark_at(c, 4);
     // The reduction needs the leader's list only: write that one here and the other workers' lists on
     // the side stream, beside the reduction; they are joined at the end of the step.
     // (a union needs every chosen node's list here, a sharded step every list)
-    const bool split = spec && W > 1 && ls.n == 1 && !per_layer && !c->select_only && c->side != nullptr;
+    const bool split = spec && W > 1 && ls.n == 1 && !per_layer && !c->select_only && !only && c->side != nullptr;
     auto write = [&](cudaStream_t st, WorkerSel ws) {
       dim3 grid(n_chunks, static_cast<unsigned>(sel_count(ws, W)));
       k_write<VEC><<<grid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur,
@@ -691,6 +719,7 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
   A(&c->d_large_ids, sz.large_ids);
   A(&c->d_state, sz.state);
   A(&c->d_hist, sz.hist);
+  A(&c->d_reach, sz.reach);
   A(&c->d_chunk_cnt, sz.chunk_cnt);
   A(&c->d_info, sz.info);
   A(&c->cand_key, sz.cand_key);
@@ -738,6 +767,7 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
   ok = ok && cudaMemset(c->acc, 0, sz.acc) == cudaSuccess;
   ok = ok && cudaMemset(c->d_state, 0, sz.state) == cudaSuccess;
   ok = ok && cudaMemset(c->d_hist, 0, sz.hist) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_reach, 0, sz.reach) == cudaSuccess;
   ok = ok && cudaMemset(c->d_chunk_cnt, 0, sz.chunk_cnt) == cudaSuccess;
   ok = ok && cudaMemset(c->sel_idx, 0, sz.sel_idx) == cudaSuccess;
   ok = ok && cudaMemset(c->sel_val, 0, sz.sel_val) == cudaSuccess;
@@ -1256,6 +1286,7 @@ int iwp_reset(iwp_ctx* c) {
   ok = ok && cudaMemsetAsync(c->zmask, 0, sz.zmask, c->stream) == cudaSuccess;
   c->zero_pending = false;
   ok = ok && cudaMemsetAsync(c->d_hist, 0, sz.hist, c->stream) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(c->d_reach, 0, sz.reach, c->stream) == cudaSuccess;
   ok = ok && cudaMemsetAsync(c->d_status, 0, sz.status, c->stream) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
@@ -1303,6 +1334,11 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
   if (!std::strcmp(key, "per_layer_leaders")) {
     if (c->threshold_mode || (v != 0 && v != 1)) return IWP_ERR_INVALID;
     c->per_layer_leaders = v != 0;
+    return IWP_OK;
+  }
+  if (!std::strcmp(key, "leader_only_select")) {
+    if (c->threshold_mode || (v != 0 && v != 1)) return IWP_ERR_INVALID;
+    c->leader_only_select = v != 0;
     return IWP_OK;
   }
   if (!std::strcmp(key, "overlap")) {
@@ -1372,6 +1408,7 @@ int iwp_get_stat(iwp_ctx* c, const char* key, int64_t* value) {
     for (uint32_t pr = 0; pr < c->n_pairs; ++pr) {
       const LayerDesc& L = c->plan.layers[c->plan.large_layers[pr / W]];
       if (L.sample == 0) continue;
+      if (c->last_only >= 0 && static_cast<int>(pr % W) != c->last_only) continue;  // that worker made no selection
       const bool cand = h[pr].guess != GUESS_NONE && h[pr].total >= L.k && (h[pr].flags & 1u) == 0u;
       if (!cand) *value += 1;
     }
@@ -1458,9 +1495,10 @@ int run_select_static(StaticScratch* s, const float* residual, const float* weig
   const WorkerSel all{WorkerSel::ALL, 0, -1};
   for (int pass = 0; pass < N_PASSES; ++pass) {
     k_hist<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr, &s->state,
-                                          s->hist, nullptr, nullptr, eps, 0, 1, pass, n_chunks, all);
+                                          s->hist, nullptr, nullptr, nullptr, eps, 0, 1, pass, n_chunks, all);
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
-    k_find_digit<<<1, THREADS, 0, st>>>(&s->state, s->hist, &s->layer, &s->large_id, &s->status, 1, pass, all);
+    k_find_digit<<<1, THREADS, 0, st>>>(&s->state, s->hist, &s->layer, &s->large_id, &s->info, nullptr, &s->status, 1, pass,
+                                        all);
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   }
   k_count<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr, &s->state,
@@ -1502,4 +1540,23 @@ extern "C" int iwp_select_static(const float* residual_dev, const float* weights
                                        static_cast<uint32_t>(k), eps, idx_dev, val_dev, st)
              : run_select_static<false>(g_static_ptr[dev], residual_dev, weights_dev, static_cast<uint32_t>(n),
                                         static_cast<uint32_t>(k), eps, idx_dev, val_dev, st);
+}
+
+extern "C" int iwp_select_static_status(int32_t* status_host, void* cuda_stream) {
+  if (!status_host) return IWP_ERR_INVALID;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  if (!g_static_ptr[dev]) return IWP_ERR_INVALID;  // nothing has run on this device yet
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int v = 0;
+  if (cudaMemcpyAsync(&v, &g_static_ptr[dev]->status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  *status_host = v;
+  return IWP_OK;
 }

@@ -74,8 +74,8 @@ __global__ void __launch_bounds__(THREADS)
            const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
            const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt,
            const uint2* __restrict__ state,
-           uint32_t* __restrict__ hist, uint32_t* __restrict__ chunk_sfx, uint2* __restrict__ chunk_cnt, float eps,
-           uint64_t N, int W, int pass, uint32_t n_chunks, WorkerSel ws) {
+           uint32_t* __restrict__ hist, uint32_t* __restrict__ chunk_sfx, uint2* __restrict__ chunk_cnt,
+           uint32_t* __restrict__ reach_seen, float eps, uint64_t N, int W, int pass, uint32_t n_chunks, WorkerSel ws) {
   __shared__ uint32_t sh[NBINS];
   __shared__ uint32_t sh_warp[WARPS];
   __shared__ uint32_t sh_above;
@@ -98,12 +98,15 @@ __global__ void __launch_bounds__(THREADS)
     // first-digit bin or the next two: count those in registers (one shared-memory atomic per lane
     // would serialise on three addresses) and leave only the rest to atomics.
     const uint32_t g0 = pi.guess >> shift;
-    uint32_t c0 = 0, c1 = 0, c2 = 0;
+    // Conservation check: the stored entries that reach the guess are counted again here and must add up
+    // to the number the streaming pass counted when it stored them (k_find_digit compares).
+    uint32_t c0 = 0, c1 = 0, c2 = 0, ge = 0;
     for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
       const uint32_t d = (key >> shift) - g0;
       c0 += d == 0u ? 1u : 0u;
       c1 += d == 1u ? 1u : 0u;
       c2 += d == 2u ? 1u : 0u;
+      ge += key >= pi.guess ? 1u : 0u;
       if (d > 2u && key != 0u) atomicAdd(&sh[(key >> shift) & (nb - 1)], 1u);
     });
 #pragma unroll
@@ -111,11 +114,13 @@ __global__ void __launch_bounds__(THREADS)
       c0 += __shfl_xor_sync(0xffffffffu, c0, d);
       c1 += __shfl_xor_sync(0xffffffffu, c1, d);
       c2 += __shfl_xor_sync(0xffffffffu, c2, d);
+      ge += __shfl_xor_sync(0xffffffffu, ge, d);
     }
     if ((threadIdx.x & 31) == 0) {
       if (c0) atomicAdd(&sh[g0 & (nb - 1)], c0);
       if (c1) atomicAdd(&sh[(g0 + 1) & (nb - 1)], c1);
       if (c2) atomicAdd(&sh[(g0 + 2) & (nb - 1)], c2);
+      if (ge && reach_seen != nullptr) atomicAdd(&reach_seen[pair], ge);
     }
   } else if (pair_is_cand(pi, L.k)) {
     for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
@@ -174,8 +179,8 @@ __global__ void __launch_bounds__(THREADS)
 // After the last pass state = (threshold key T, number r of T-valued elements to keep).
 __global__ void __launch_bounds__(THREADS)
     k_find_digit(uint2* __restrict__ state, uint32_t* __restrict__ hist, const LayerDesc* __restrict__ layers,
-                 const uint32_t* __restrict__ large_ids, int* __restrict__ status, int W, int pass,
-                 WorkerSel ws) {
+                 const uint32_t* __restrict__ large_ids, const PairInfo* __restrict__ info,
+                 uint32_t* __restrict__ reach_seen, int* __restrict__ status, int W, int pass, WorkerSel ws) {
   __shared__ uint32_t sh[NBINS];
   __shared__ uint32_t sh_scan[THREADS];
   __shared__ uint32_t res[4];
@@ -191,6 +196,14 @@ __global__ void __launch_bounds__(THREADS)
   if (pass == 0) {
     prefix = 0;
     krem = layers[large_ids[pair / W]].k;
+    if (threadIdx.x == 0 && reach_seen != nullptr) {
+      // a pair that selects from its candidate slots: what the first histogram pass found in the slots must be
+      // what the streaming pass put there (a lost, overwritten or stale entry shows up as a different count)
+      const PairInfo pi = info[pair];
+      const uint32_t seen = reach_seen[pair];
+      reach_seen[pair] = 0;
+      if (pair_is_cand(pi, krem) && seen != pi.total) atomicMin(status, STATUS_INTERNAL);
+    }
   } else {
     const uint2 s = state[pair];
     prefix = s.x;
@@ -479,7 +492,7 @@ __global__ void __launch_bounds__(THREADS)
     k_small(const float* __restrict__ grads, const float* __restrict__ weights, float* __restrict__ acc,
             float* __restrict__ update, const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ small_ids,
             uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot,
-            int* __restrict__ status, float eps, uint64_t N, uint64_t K, int leader, float momentum) {
+            int* __restrict__ status, float eps, uint64_t N, uint64_t K, int leader, int only_worker, float momentum) {
   extern __shared__ uint32_t keys[];
   __shared__ uint32_t hist[NBINS];
   __shared__ uint32_t sh_scan[THREADS];
@@ -498,6 +511,7 @@ __global__ void __launch_bounds__(THREADS)
     keys[i] = imp_key(v, wt[i], eps);
     if (w == 0) update[L.off + i] = 0.0f;
   }
+  if (only_worker >= 0 && w != only_worker) return;  // only the chosen node selects: steps (a), (b) were this worker's part
   __syncthreads();
   uint32_t T, r;
   if (!smem_radix_select(keys, n, L.k, hist, sh_scan, res, T, r)) {

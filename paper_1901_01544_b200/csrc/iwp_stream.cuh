@@ -77,7 +77,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS)
     k_sample(const float* __restrict__ grads, const float* __restrict__ weights, const float* __restrict__ acc,
              const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ large_ids, PairInfo* __restrict__ info,
              uint2* __restrict__ guess_tab, const uint32_t* __restrict__ zmask, float eps, uint64_t N, int W,
-             uint32_t step, float momentum) {
+             uint32_t step, int only_worker, float momentum) {
   extern __shared__ uint32_t keys[];
   __shared__ uint32_t hist[NBINS];
   __shared__ uint32_t sh_scan[SAMPLE_THREADS];
@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(SAMPLE_THREADS)
   const LayerDesc L = layers[large_ids[pair / W]];
   const int w = pair % W;
   const uint32_t s = L.sample;
-  if (s == 0) {
+  if (s == 0 || (only_worker >= 0 && w != only_worker)) {  // no speculation, or a worker that makes no selection
     if (threadIdx.x == 0) {
       const uint32_t gm = __float_as_uint(pretest_multiplier(GUESS_NONE, eps));
       info[pair] = PairInfo{GUESS_NONE, 0u, 0u, gm};
@@ -193,11 +193,14 @@ __device__ __forceinline__ void st_keep_u16(uint16_t* ptr, uint16_t v, uint64_t 
 // Position, inside one iteration, of the staged element with mask bit b = 4 * round + component:
 // the staged elements of earlier rounds, of earlier lanes in the same round, and of earlier
 // components of the same lane and round.  `ex` / `tt`: per-round exclusive lane prefix / totals,
-// packed 8 bits per round.
+// packed 8 bits per round (a round stages at most 128 elements, so a field never carries).  The
+// sum over the earlier rounds reaches 384 and is therefore taken in a full register: a byte-wise
+// dot product of the totals with a 0/1 selector of the rounds below this one.
 __device__ __forceinline__ uint32_t staged_position(uint32_t mask, uint32_t ex, uint32_t tt, uint32_t b) {
-  const uint32_t sh = (b >> 2) * 8;
-  const uint32_t rounds_before = ((tt * 0x01010100u) >> sh) & 0xFFu;  // byte r of tt * 0x01010100 = sum of rounds < r
-  return rounds_before + ((ex >> sh) & 0xFFu) + __popc((mask >> (b & ~3u)) & ((1u << (b & 3u)) - 1u));
+  const uint32_t round = b >> 2;
+  const uint32_t earlier = 0x00010101u >> (8u * (3u - round));  // byte r is 1 for every round r < round
+  const uint32_t rounds_before = __dp4a(tt, earlier, 0u);
+  return rounds_before + ((ex >> (8u * round)) & 0xFFu) + __popc((mask >> (b & ~3u)) & ((1u << (b & 3u)) - 1u));
 }
 
 template <bool VEC, bool LEADER>

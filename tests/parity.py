@@ -21,11 +21,15 @@ def assert_bits_equal(got: np.ndarray, want: np.ndarray, what: str):
 
 
 def compare_state(pr: Pruner, orc: "oracle.Oracle", update_gpu: torch.Tensor, update_cpu: np.ndarray, tag: str,
-                  check_mask: bool = True, check_residual: bool = True):
+                  check_mask: bool = True, check_residual: bool = True, leader_list_only: bool = False):
     assert pr.sync_status() == 0, f"{tag}: device status {pr.sync_status()}"
     assert pr.leader == orc.leader, f"{tag}: leader {pr.leader} != {orc.leader}"
     assert_bits_equal(update_gpu.cpu().numpy(), update_cpu, f"{tag}: update")
     for w in range(pr.W):
+        if leader_list_only and w != orc.leader:  # option leader_only_select: nobody else makes a list
+            if check_residual:
+                assert_bits_equal(pr.residual(w).cpu().numpy(), orc.residual(w), f"{tag}: worker {w} residual")
+            continue
         idx, val = pr.selection(w)
         oi, ov = orc.selection(w)
         gi = idx.cpu().numpy().view(np.uint32)
@@ -43,7 +47,7 @@ def compare_state(pr: Pruner, orc: "oracle.Oracle", update_gpu: torch.Tensor, up
 
 def run_parity(layer_sizes, W, ratio, eps, seed, steps, weights: torch.Tensor, grads_fn, options=None,
                leader_overrides=None, check_mask=True, threads=0, residual_every=1, momentum=None, state_every=1,
-               weights_fn=None, n_leaders=1, per_layer_leaders=False):
+               weights_fn=None, n_leaders=1, per_layer_leaders=False, leader_list_only=False):
     """weights: CUDA tensor [N]; grads_fn(t) -> CUDA tensor [W, N].
 
     state_every: lists, mask, residuals and the device status are looked at only every that many steps
@@ -88,7 +92,8 @@ def run_parity(layer_sizes, W, ratio, eps, seed, steps, weights: torch.Tensor, g
             update.fill_(float("nan"))
             continue
         look = (t + 1) % residual_every == 0 or t == steps - 1
-        compare_state(pr, orc, update, upd_cpu, f"step {t}", check_mask=check_mask, check_residual=look)
+        compare_state(pr, orc, update, upd_cpu, f"step {t}", check_mask=check_mask, check_residual=look,
+                      leader_list_only=leader_list_only)
         update.fill_(float("nan"))  # the next step must overwrite every element
     pr.close()
     orc.close()

@@ -283,6 +283,47 @@ def test_back_to_back_steps_with_leader_overrides():
                leader_overrides=[0, 3, 3, 1, -1, 2, -1, 0], residual_every=1000, state_every=1000)
 
 
+# ------------------------------------------------------------------ only the chosen node selects (option)
+
+
+@pytest.mark.parametrize("speculate", [1, 0])
+@pytest.mark.parametrize("overlap", [1, 0])
+def test_leader_only_select(overlap, speculate):
+    # Algorithm 1 consumes the chosen node's index set only; with the option on, no other worker makes a list.
+    # Update, chosen node's list, mask and every residual are those of the default path.
+    sizes, W, ratio = [70000, 64, 16385, 300000, 9, 40000], 5, 32.0
+    N = sum(sizes)
+    weights = _weights(N, 27)
+    run_parity(sizes, W, ratio, 1e-8, seed=9, steps=6, weights=weights, grads_fn=lambda t: _randn((W, N), 600 + t),
+               options={"leader_only_select": 1, "overlap": overlap, "speculate": speculate}, residual_every=2,
+               leader_list_only=True)
+
+
+def test_leader_only_select_switched_on_and_off_between_steps():
+    import oracle
+    from paper_1901_01544_b200.binding import Pruner
+    from parity import compare_state
+
+    c = _scaled_case("alexnet_w8")
+    pr = Pruner(c.layer_sizes, c.W, c.ratio, c.eps, c.seed)
+    orc = oracle.Oracle(c.layer_sizes, c.W, c.ratio, c.eps, c.seed)
+    pr.set_option("overlap", 1)
+    weights = c.weights(DEV)
+    w_host = weights.cpu().numpy()
+    update = torch.full((pr.N,), float("nan"), device=DEV)
+    for t in range(8):
+        only = t % 3 != 0
+        pr.set_option("leader_only_select", int(only))
+        g = c.grads(t, DEV)
+        pr.step(g, weights, update)
+        want = orc.step(np.ascontiguousarray(g.cpu().numpy()), w_host)
+        compare_state(pr, orc, update, want, f"step {t}", check_residual=t % 2 == 1, leader_list_only=only)
+        assert pr.stat("spec_failed") == 0
+        update.fill_(float("nan"))
+    pr.close()
+    orc.close()
+
+
 # ------------------------------------------------------------------ several chosen nodes (Mask = OR Mask_ri)
 
 

@@ -90,6 +90,27 @@ def test_threshold_mode_random_values(name):
     _run(sizes, W, thr, weights, lambda t: _randn((W, N), 7 * t + 1, 1e-3), steps=4)
 
 
+@pytest.mark.parametrize("n_leaders", [1, 2])
+def test_threshold_mode_clustered_importances(n_leaders):
+    # runs of consecutive elements far above the threshold (blocks of zero weights, one worker's hot gradients)
+    # at segment, tile and chunk edges of the passes: whole mask words and whole chunks are set
+    sizes, W = [300, 20000, 128 * 4096 + 70000], 4
+    N = sum(sizes)
+    weights = _randn((N,), 100, 0.05)
+    weights = torch.where(weights.abs() < 1e-3, torch.full_like(weights, 1e-3), weights)
+    off = sizes[0] + sizes[1]
+    edge = ((off // 4096) + 128) * 4096
+    for start, length in ((edge - 150, 300), (off + 8192, 513), (N - 280, 280), (100, 150), (4096 - 7, 257)):
+        weights[start:start + length] = 0.0
+
+    def grads(t):
+        g = _randn((W, N), 300 + t, 1e-3)
+        g[(t + 1) % W, off + 3 * 4096 + 500:off + 3 * 4096 + 900] *= 1000.0
+        return g
+
+    _run(sizes, W, [2.0, 1.0, 0.5], weights, grads, steps=4, n_leaders=n_leaders, residual_every=2)
+
+
 def test_threshold_mode_ties_zero_and_infinite_thresholds():
     sizes, W = [50000, 300, 20000, 5], 3
     N = sum(sizes)

@@ -1,6 +1,6 @@
 """The allocation-free entry point iwp_select_static (for callers that may not allocate device
-memory while they run) against the context-based path: same layer, same residual, the list must
-be identical bit for bit.  Two calls in a row share the library's fixed scratch array, so the
+memory while they run) against the CPU oracle's plain top-k definition and against the
+context-based path: same layer, same residual, the list must be identical bit for bit.  Two calls in a row share the library's fixed scratch array, so the
 second call also proves that the first left nothing behind that matters.  Collected last on
 purpose: a run that stops at the first failure has then already run every other test."""
 import ctypes as C
@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_1901_01544_b200 import binding
 from paper_1901_01544_b200.binding import Pruner
 
@@ -37,8 +38,18 @@ def _static_list(residual, weights, ratio, eps):
     stream = torch.cuda.current_stream().cuda_stream
     k = binding.iwp_select_static(residual.data_ptr(), weights.data_ptr(), n, ratio, eps, idx.data_ptr(),
                                   val.data_ptr(), stream)
+    assert binding.iwp_select_static_status(stream) == 0, "a count check of the select failed on the device"
     torch.cuda.synchronize()
     return k, idx, val
+
+
+def _assert_matches_oracle(residual, weights, k, eps, idx, val):
+    """The plain definition: the k best under (importance descending, index ascending), listed by index."""
+    r_host = residual.cpu().numpy()
+    want = oracle.select(r_host, weights.cpu().numpy(), k, eps)
+    got = idx.cpu().numpy().view(np.uint32)
+    assert np.array_equal(got, want), "indices differ from the oracle's top-k"
+    assert np.array_equal(val.cpu().numpy().view(np.uint32), r_host[want].view(np.uint32)), "values differ bit-wise"
 
 
 def test_static_select_matches_context_path_twice_in_a_row():
@@ -52,7 +63,8 @@ def test_static_select_matches_context_path_twice_in_a_row():
         residual[::7] = residual[3]  # repeated values: ties at and around the threshold
         k_ref, idx_ref, val_ref = _reference_list(residual, weights, ratio, 1e-8)
         k, idx, val = _static_list(residual, weights, ratio, 1e-8)
-        assert k == k_ref == binding.iwp_keep_count(n, ratio)
+        assert k == k_ref == binding.iwp_keep_count(n, ratio) == oracle.keep_count(n, ratio)
+        _assert_matches_oracle(residual, weights, k, 1e-8, idx, val)
         assert torch.equal(idx, idx_ref), "indices differ from the context-based path"
         assert torch.equal(val.view(torch.int32), val_ref.view(torch.int32)), "values differ bit-wise"
         assert torch.all(idx[1:] > idx[:-1])
@@ -67,11 +79,13 @@ def test_static_select_unaligned_pointers_and_small_layer():
     k_ref, idx_ref, val_ref = _reference_list(rbuf[1:].clone(), wbuf[1:].clone(), 16.0, 1e-8)
     k, idx, val = _static_list(rbuf[1:], wbuf[1:], 16.0, 1e-8)  # 4-byte aligned only: scalar access path
     assert k == k_ref and torch.equal(idx, idx_ref) and torch.equal(val.view(torch.int32), val_ref.view(torch.int32))
+    _assert_matches_oracle(rbuf[1:], wbuf[1:], k, 1e-8, idx, val)
     # a layer small enough for the context path's one-CTA kernel still gives the same list
     r2, w2 = rbuf[:1000].clone(), wbuf[:1000].clone()
     k_ref, idx_ref, val_ref = _reference_list(r2, w2, 8.0, 1e-8)
     k, idx, val = _static_list(r2, w2, 8.0, 1e-8)
     assert k == k_ref == 125 and torch.equal(idx, idx_ref) and torch.equal(val.view(torch.int32), val_ref.view(torch.int32))
+    _assert_matches_oracle(r2, w2, k, 1e-8, idx, val)
 
 
 def test_static_select_rejects_what_it_cannot_hold():
