@@ -208,6 +208,13 @@ int iwp_shard_apply(iwp_ctx* ctx, const uint32_t* idx_dev, int64_t n, const floa
  * back and synchronises the stream before returning. */
 int iwp_step_host(iwp_ctx* ctx, const float* grads_host, const float* weights_host, float* update_host);
 
+/* Makes the context's stream wait for everything the last step left running on the library's own side
+ * streams (with the overlapped schedule the selects of workers other than the chosen node, whose lists
+ * no step consumes, outlive iwp_step()).  Nothing is synchronised with the host: after this call, work
+ * enqueued on the context's stream - an event record, a copy - is ordered behind ALL of the step's
+ * kernels.  Every accessor does this by itself.  Errors: IWP_ERR_INVALID, IWP_ERR_CUDA. */
+int iwp_join(iwp_ctx* ctx);
+
 /* Synchronises the stream and returns the device status word: IWP_OK, IWP_ERR_INTERNAL
  * (a count check failed inside a kernel; results of that step are undefined) or IWP_ERR_CUDA. */
 int iwp_sync_status(iwp_ctx* ctx);
@@ -288,6 +295,8 @@ int iwp_host_wait(iwp_ctx* ctx);
  *                      (read the totals with iwp_get_stat; steps run as with "overlap" 0 meanwhile);
  *                      2 = only before and after the dominant streaming stage (two events per step);
  *                      0 = stop and discard them
+ *   "reserve_timed_steps" n: creates the CUDA events of the next n timed steps now (in the current
+ *                      "time_stages" mode), so that a timed step only records them
  * Unknown key or out-of-range value: IWP_ERR_INVALID. */
 int iwp_set_option(iwp_ctx* ctx, const char* key, int64_t value);
 

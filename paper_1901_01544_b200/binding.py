@@ -23,7 +23,7 @@ EXPORTS = [
     "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat", "iwp_select_static",
     "iwp_set_momentum", "iwp_create_threshold", "iwp_set_thresholds", "iwp_get_list_length", "iwp_leaders_at",
     "iwp_set_layerwise", "iwp_get_layer_thresholds", "iwp_shard_select", "iwp_shard_gather", "iwp_shard_apply",
-    "iwp_layer_leader_at", "iwp_encode_mask", "iwp_step_host_async", "iwp_host_wait", "iwp_select_static_status",
+    "iwp_layer_leader_at", "iwp_encode_mask", "iwp_step_host_async", "iwp_host_wait", "iwp_select_static_status", "iwp_join",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -68,6 +68,7 @@ def lib() -> C.CDLL:
         L.iwp_shard_gather.argtypes = [vp, vp, i64, vp]
         L.iwp_shard_apply.argtypes = [vp, vp, i64, vp, i32, vp]
         L.iwp_sync_status.argtypes = [vp]
+        L.iwp_join.argtypes = [vp]
         L.iwp_get_layout.argtypes = [vp, vp, vp]
         L.iwp_get_sizes.argtypes = [vp, vp]
         L.iwp_get_step.argtypes = [vp, vp]
@@ -286,6 +287,10 @@ class Pruner:
 
     def set_momentum(self, m: float) -> None:
         _check(lib().iwp_set_momentum(self._h, float(m)), "iwp_set_momentum")
+
+    def join(self) -> None:
+        """Orders the context's stream behind everything the last step left running on side streams."""
+        _check(lib().iwp_join(self._h), "iwp_join")
 
     def sync_status(self) -> int:
         return int(lib().iwp_sync_status(self._h))

@@ -114,6 +114,7 @@ struct iwp_ctx {
   // optional per-stage CUDA-event timing (option "time_stages")
   int time_stages = 0;  // 0 off, 1 every stage boundary, 2 only around the dominant streaming stage
   std::vector<cudaEvent_t> stage_events;  // N_STAGES + 1 events per timed step
+  std::vector<cudaEvent_t> event_pool;    // events made ahead of the timed steps (option "reserve_timed_steps")
   // staging for iwp_step_host
   float* stg_grads = nullptr;
   float* stg_weights = nullptr;
@@ -146,12 +147,14 @@ void stage_mark_at(iwp_ctx* c, int boundary) {
   const int dominant = c->threshold_mode ? ST_GATHER : ST_ACCUMULATE;
   const bool wanted = c->time_stages == 1 || boundary == dominant || boundary == dominant + 1;
   if (wanted) {
-    if (cudaEventCreate(&e) != cudaSuccess) {
+    if (!c->event_pool.empty()) {  // made ahead of time: nothing but the record happens inside a timed step
+      e = c->event_pool.back();
+      c->event_pool.pop_back();
+    } else if (cudaEventCreate(&e) != cudaSuccess) {
       cudaGetLastError();
       e = nullptr;
-    } else {
-      cudaEventRecord(e, c->stream);
     }
+    if (e) cudaEventRecord(e, c->stream);
   }
   c->stage_events.push_back(e);  // a null entry keeps the slots of a step aligned
 }
@@ -160,6 +163,8 @@ void stage_clear(iwp_ctx* c) {
   for (cudaEvent_t e : c->stage_events)
     if (e) cudaEventDestroy(e);
   c->stage_events.clear();
+  for (cudaEvent_t e : c->event_pool) cudaEventDestroy(e);
+  c->event_pool.clear();
 }
 
 struct Sizes {
@@ -1133,6 +1138,11 @@ int iwp_host_wait(iwp_ctx* c) {
   return IWP_OK;
 }
 
+int iwp_join(iwp_ctx* c) {
+  if (!c) return IWP_ERR_INVALID;
+  return join_deferred(c);
+}
+
 int iwp_sync_status(iwp_ctx* c) {
   if (!c) return IWP_ERR_INVALID;
   if (const int jrc = join_deferred(c)) return jrc;
@@ -1319,6 +1329,19 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
     cudaStreamSynchronize(c->stream);
     stage_clear(c);
     c->time_stages = static_cast<int>(v);
+    return IWP_OK;
+  }
+  if (!std::strcmp(key, "reserve_timed_steps")) {
+    if (v < 0 || v > (1 << 20)) return IWP_ERR_INVALID;
+    const size_t per_step = c->time_stages == 1 ? N_STAGES + 1 : 2;
+    for (size_t i = 0; i < static_cast<size_t>(v) * per_step; ++i) {
+      cudaEvent_t e = nullptr;
+      if (cudaEventCreate(&e) != cudaSuccess) {
+        cudaGetLastError();
+        return IWP_ERR_CUDA;
+      }
+      c->event_pool.push_back(e);
+    }
     return IWP_OK;
   }
   if (!std::strcmp(key, "random_select")) {
