@@ -156,24 +156,27 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t x, uint32_t* sh_war
 
 // Radix-select digit step on a histogram in shared memory: finds the digit d with
 //   count(digit > d) < krem <= count(digit >= d)
-// res[0] = d, res[1] = krem - count(digit > d), res[2] = 1 if found.  sh_scan: THREADS words.
+// res[0] = d, res[1] = krem - count(digit > d), res[2] = 1 if found.  sh_scan: NT / 32 words.
+// Suffix sums over the threads' bin groups: by shuffles inside a warp, then over the warps' totals
+// (two block barriers in all).
 template <int NT = THREADS>
 __device__ __forceinline__ void find_digit(const uint32_t* hist, int nb, uint32_t krem, uint32_t* sh_scan,
                                            uint32_t* res) {
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  constexpr int NW = NT / 32;
   const int per = nb / NT;
   uint32_t local = 0;
   for (int b = 0; b < per; ++b) local += hist[tid * per + b];
-  sh_scan[tid] = local;
+  uint32_t incl = local;  // inclusive suffix sum over the lanes of the warp
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t y = __shfl_down_sync(0xffffffffu, incl, d);
+    if (lane + d < 32) incl += y;
+  }
+  if (lane == 0) sh_scan[wid] = incl;
   if (tid == 0) res[2] = 0;
   __syncthreads();
-  for (int d = 1; d < NT; d <<= 1) {  // inclusive suffix sum over threads
-    const uint32_t v = (tid + d < NT) ? sh_scan[tid + d] : 0u;
-    __syncthreads();
-    sh_scan[tid] += v;
-    __syncthreads();
-  }
-  const uint32_t incl = sh_scan[tid];
+  for (int i = wid + 1; i < NW; ++i) incl += sh_scan[i];  // the warps above this one
   const uint32_t excl = incl - local;
   if (excl < krem && krem <= incl) {
     uint32_t running = excl;
