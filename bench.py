@@ -216,10 +216,51 @@ def run_reference(args):
 # ---------------------------------------------------------------------------------- workers spread over GPUs
 
 
+def measure_sharded(c, dist, rank, world, dev, steps, warmup, grad_sets=None, wire="auto"):
+    """The workload's W workers spread over the ranks (W / world each): ShardedPruner - NCCL broadcast of the chosen
+    worker's index set (list or encoded mask, whichever is shorter) and all-gather of the gathered values.  Total
+    work is fixed: strong scaling.  On one GPU it measures the cost of the three-phase protocol itself."""
+    import torch
+
+    from paper_1901_01544_b200.binding import ShardedPruner
+
+    if c.W % world != 0:
+        return {"error": f"the workload's {c.W} workers do not divide over {world} ranks"}
+    Wl, N = c.W // world, c.N
+    weights = c.weights(dev)
+    n_sets = grad_sets or 3
+    sets = [c.grads(t, dev)[rank * Wl:(rank + 1) * Wl].contiguous() for t in range(n_sets)]
+    update = torch.empty(N, dtype=torch.float32, device=dev)
+    sp = ShardedPruner(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, wire=wire)
+    for t in range(warmup):
+        sp.step(sets[t % n_sets], weights, update)
+    launches0 = sp.local.stat("launches")
+    torch.cuda.synchronize()
+    dist.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(steps):
+        sp.step(sets[(warmup + t) % n_sets], weights, update)
+    sp.local.join()
+    e1.record()
+    torch.cuda.synchronize()
+    dist.barrier()
+    ms_total = max_over_ranks(e0.elapsed_time(e1), dist, dev)
+    assert sp.local.sync_status() == 0
+    out = {"value": steps / (ms_total * 1e-3), "unit": UNIT, "ms_per_step": ms_total / steps, "scaling": "strong",
+           "n_gpus": world, "steps": steps, "warmup": warmup, "W": c.W, "W_per_gpu": Wl, "N": N, "K": sp.K,
+           "wire_format": sp.last_wire, "wire_bytes_per_step": sp.wire_bytes, "allgather_bytes_per_step": 4 * c.W * sp.K,
+           "collectives": "broadcast of the index set (sorted uint32 list or one-bit-per-element mask, the shorter) + "
+                          "all-gather of W x K fp32 per step (NCCL)",
+           "gpu_launches": sp.local.stat("launches") - launches0}
+    sp.close()
+    del sets, weights, update, sp
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_sharded(args):
-    """--shard: the workload's W workers spread over the N ranks (W / N each), the chosen worker's index list
-    broadcast and the gathered values all-gathered over NCCL (ShardedPruner).  Total work is fixed: strong
-    scaling.  Not the default arm; on one GPU it measures the cost of the three-phase protocol itself."""
+    """--shard: only the sharded arm (see measure_sharded), one JSON line from rank 0."""
     import torch
     import torch.distributed as dist
 
@@ -239,38 +280,18 @@ def run_sharded(args):
     if rank == 0:
         lib_build.build()
     dist.barrier()
-    from paper_1901_01544_b200.binding import ShardedPruner
-
     c = make_workload(args.config, args.layers)
-    if c.W % world != 0:
-        raise SystemExit(f"--shard needs the workload's {c.W} workers to divide over {world} ranks")
-    Wl, N = c.W // world, c.N
-    weights = c.weights(dev)
-    n_sets = args.grad_sets or 3
-    sets = [c.grads(t, dev)[rank * Wl:(rank + 1) * Wl].contiguous() for t in range(n_sets)]
-    update = torch.empty(N, dtype=torch.float32, device=dev)
-    sp = ShardedPruner(c.layer_sizes, c.W, c.ratio, c.eps, c.seed)
-    for t in range(args.warmup):
-        sp.step(sets[t % n_sets], weights, update)
-    torch.cuda.synchronize()
-    dist.barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for t in range(args.steps):
-        sp.step(sets[(args.warmup + t) % n_sets], weights, update)
-    e1.record()
-    torch.cuda.synchronize()
-    dist.barrier()
-    ms_total = max_over_ranks(e0.elapsed_time(e1), dist, dev)
-    assert sp.local.sync_status() == 0
+    r = measure_sharded(c, dist, rank, world, dev, args.steps, args.warmup, args.grad_sets, args.wire)
+    if "error" in r:
+        raise SystemExit(r["error"])
     if rank == 0:
         line = {
-            "metric": METRIC, "value": args.steps / (ms_total * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "strong",
+            "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": r["ms_per_step"], "higher_is_better": True, "scaling": "strong",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": c.name, "mode": "sharded", "W": c.W, "W_per_gpu": Wl, "N": N, "K": sp.K,
-                       "collectives": "broadcast of K uint32 + all-gather of W x K fp32 per step (NCCL)"},
-            "gpu_launches": sp.local.stat("launches"),
+            "config": {"workload": c.name, "mode": "sharded", "W": c.W, "W_per_gpu": r["W_per_gpu"], "N": c.N, "K": r["K"],
+                       "wire_format": r["wire_format"], "collectives": r["collectives"]},
+            "gpu_launches": r["gpu_launches"],
         }
         print(json.dumps(line), flush=True)
     dist.destroy_process_group()
@@ -471,6 +492,14 @@ def run_ours(args):
         e2e_value = whole_job_value(e2e_steps, world, e2e_dt * 1e3)
         del gh, wh, uh
 
+    # N > 1: the same workload once more with its W workers spread over the ranks (the paper's deployment: the index
+    # set and the gathered values cross NVLink), reported beside the replicas' number
+    sharded = None
+    if dist is not None:
+        pr.close()
+        del sets, weights, update, pr
+        torch.cuda.empty_cache()
+        sharded = measure_sharded(c, dist, rank, world, dev, args.steps, max(3, args.warmup), args.grad_sets, args.wire)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -520,8 +549,8 @@ def run_ours(args):
     # CPU baseline: the oracle as it stands, a bounded sample (a few full steps) on this machine's cores, and on one
     cpu = cpu1 = None
     if not args.no_cpu_baseline and args.mode == "ratio":
-        w_host = weights.cpu().numpy()
-        g_host = [sets[i].cpu().numpy() for i in range(min(2, n_sets))]
+        w_host = c.weights("cpu").numpy() if dist is not None else weights.cpu().numpy()
+        g_host = [(c.grads(i, "cpu") if dist is not None else sets[i].cpu()).numpy() for i in range(min(2, n_sets))]
         sps, threads, dt = oracle_timing(c, w_host, lambda t: g_host[t % len(g_host)], args.cpu_steps, 1)
         cpu = {"value": sps, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": f"{args.cpu_steps} full steps of {c.name} after 1 warm-up step ({dt:.1f} s of CPU work)"}
@@ -548,6 +577,8 @@ def run_ours(args):
         "clocks": clocks,
         "plan": plan,
     }
+    if sharded is not None:
+        line["sharded"] = sharded
 
     # The other configurations and the mode / option variants, each timed like the headline (device-resident
     # inputs, CUDA events around the timed steps), one after the other in this process at N = 1.
@@ -556,6 +587,20 @@ def run_ours(args):
         del sets, weights, update, pr
         torch.cuda.empty_cache()
         table = {}
+        try:  # the three-phase protocol of the sharded deployment on this one GPU (a one-rank NCCL group)
+            import torch.distributed as dist1
+
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29533")
+            dist1.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
+            try:
+                table[f"{args.config}:sharded_protocol_on_one_gpu"] = measure_sharded(
+                    c, dist1, 0, 1, dev, args.extra_steps, max(3, args.warmup), args.grad_sets, args.wire)
+            finally:
+                dist1.destroy_process_group()
+        except Exception as e:
+            table[f"{args.config}:sharded_protocol_on_one_gpu"] = {"error": f"{type(e).__name__}: {e}"}
+            torch.cuda.empty_cache()
         for name in EXTRA_CONFIGS:
             if name == args.config:
                 continue
@@ -597,6 +642,8 @@ def main():
     ap.add_argument("--shard", action="store_true",
                     help="spread the workload's W workers over the ranks (ShardedPruner: NCCL broadcast + all-gather) "
                          "instead of running independent replicas")
+    ap.add_argument("--wire", default="auto", choices=["auto", "list", "mask"],
+                    help="what travels as the index set in the sharded arm (auto = the shorter encoding)")
     ap.add_argument("--layerwise", default=None,
                     help="alpha,beta,C - with --mode threshold: layer-wise thresholds alpha +/- beta var/mean (Eq. 4)")
     ap.add_argument("--layers", default=None, help="lo:hi - only these layers of the workload (small profiling case)")

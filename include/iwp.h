@@ -246,6 +246,25 @@ int iwp_get_mask(iwp_ctx* ctx, uint8_t* dst_dev);
  * sorted index list). */
 int iwp_encode_mask(iwp_ctx* ctx, const uint8_t* mask_dev, uint8_t* bits_dev);
 
+/* ---- wire formats of the index set (workers spread over GPUs) ------------------------------- */
+
+/* Algorithm 1 sends the index set as AllGather(encode_uint8(Mask)) ahead of the all-reduce of the masked
+ * gradients.  Two encodings are offered to whoever moves the bytes: the sorted uint32 index list (4 bytes
+ * per entry - what iwp_get_selection() returns) and the mask at one bit per element, bit i % 8 of byte
+ * i / 8, padded to whole 32-bit words.  The list is the shorter one when the set holds fewer than N / 32
+ * entries (compression above 32), the mask otherwise. */
+
+/* Bytes of the one-bit-per-element mask of an N-element job: 4 * ceil(N / 32).  Pure host function. */
+int64_t iwp_wire_mask_bytes(int64_t N);
+/* idx_dev[0..n) (element indices < N, any order, no duplicates needed) -> bits_dev (iwp_wire_mask_bytes(N)
+ * bytes, 4-byte aligned, fully overwritten; idx_dev may be NULL when n = 0).  Asynchronous on the context's stream.  An index >= N sets the
+ * status word to IWP_ERR_INTERNAL and is skipped. */
+int iwp_wire_pack(iwp_ctx* ctx, const uint32_t* idx_dev, int64_t n, uint8_t* bits_dev);
+/* bits_dev -> the ascending index list in idx_dev[0..cap).  Asynchronous on the context's stream; with
+ * n_host != NULL the call waits for the stream and stores the number of set bits there.  More set bits
+ * than cap: the surplus is dropped and the status word becomes IWP_ERR_CAPACITY. */
+int iwp_wire_unpack(iwp_ctx* ctx, const uint8_t* bits_dev, uint32_t* idx_dev, int64_t cap, int64_t* n_host);
+
 /* acc <- 0, step counter <- 0, status word <- 0. */
 int iwp_reset(iwp_ctx* ctx);
 

@@ -23,7 +23,7 @@ EXPORTS = [
     "iwp_get_selection", "iwp_get_mask", "iwp_reset", "iwp_set_option", "iwp_get_stat", "iwp_select_static",
     "iwp_set_momentum", "iwp_create_threshold", "iwp_set_thresholds", "iwp_get_list_length", "iwp_leaders_at",
     "iwp_set_layerwise", "iwp_get_layer_thresholds", "iwp_shard_select", "iwp_shard_gather", "iwp_shard_apply",
-    "iwp_layer_leader_at", "iwp_encode_mask", "iwp_step_host_async", "iwp_host_wait", "iwp_select_static_status", "iwp_join",
+    "iwp_layer_leader_at", "iwp_encode_mask", "iwp_step_host_async", "iwp_host_wait", "iwp_select_static_status", "iwp_join", "iwp_wire_mask_bytes", "iwp_wire_pack", "iwp_wire_unpack",
 ]
 
 _lib: Optional[C.CDLL] = None
@@ -69,6 +69,9 @@ def lib() -> C.CDLL:
         L.iwp_shard_apply.argtypes = [vp, vp, i64, vp, i32, vp]
         L.iwp_sync_status.argtypes = [vp]
         L.iwp_join.argtypes = [vp]
+        L.iwp_wire_mask_bytes.restype, L.iwp_wire_mask_bytes.argtypes = i64, [i64]
+        L.iwp_wire_pack.argtypes = [vp, vp, i64, vp]
+        L.iwp_wire_unpack.argtypes = [vp, vp, vp, i64, vp]
         L.iwp_get_layout.argtypes = [vp, vp, vp]
         L.iwp_get_sizes.argtypes = [vp, vp]
         L.iwp_get_step.argtypes = [vp, vp]
@@ -158,6 +161,10 @@ def iwp_select_static(residual_ptr: int, weights_ptr: int, n: int, ratio: float,
     _check(lib().iwp_select_static(residual_ptr, weights_ptr, n, ratio, eps, idx_ptr, val_ptr, C.byref(k),
                                    C.c_void_p(stream)), "iwp_select_static")
     return int(k.value)
+
+
+def iwp_wire_mask_bytes(N: int) -> int:
+    return int(lib().iwp_wire_mask_bytes(N))
 
 
 def iwp_select_static_status(stream: int = 0) -> int:
@@ -264,6 +271,23 @@ class Pruner:
         assert vals_all.dim() == 2 and vals_all.shape[1] == idx.numel()
         _check(lib().iwp_shard_apply(self._h, idx.data_ptr(), idx.numel(), vals_all.data_ptr(), int(vals_all.shape[0]),
                                      update.data_ptr()), "iwp_shard_apply")
+
+    # the two wire formats of an index set (see ShardedPruner)
+    def wire_pack(self, idx):
+        """Index list -> mask at one bit per element (uint8 tensor of iwp_wire_mask_bytes(N) bytes)."""
+        t = self._torch
+        assert idx.is_cuda and idx.dtype == t.int32 and idx.is_contiguous()
+        bits = t.empty(iwp_wire_mask_bytes(self.N), dtype=t.uint8, device=self.device)
+        _check(lib().iwp_wire_pack(self._h, idx.data_ptr(), idx.numel(), bits.data_ptr()), "iwp_wire_pack")
+        return bits
+
+    def wire_unpack(self, bits, n: int):
+        """Mask at one bit per element -> ascending index list of n entries (n = the number of set bits)."""
+        t = self._torch
+        assert bits.is_cuda and bits.dtype == t.uint8 and bits.is_contiguous() and bits.numel() == iwp_wire_mask_bytes(self.N)
+        idx = t.empty(n, dtype=t.int32, device=self.device)
+        _check(lib().iwp_wire_unpack(self._h, bits.data_ptr(), idx.data_ptr(), n, None), "iwp_wire_unpack")
+        return idx
 
     def set_thresholds(self, thr: Sequence[float]) -> None:
         arr = (C.c_float * self.L)(*[float(x) for x in thr])
@@ -372,11 +396,16 @@ class ShardedPruner:
     context of W workers computes - and zeroes what its own workers sent.  Only argument marshalling and
     the two collectives happen here; every step of the method runs in the library's kernels.
 
+    What travels in the first collective (`wire`): "list" = the sorted uint32 index list (4 bytes per entry),
+    "mask" = Algorithm 1's encoded mask at one bit per element (N / 8 bytes; packed on the owner and expanded
+    on arrival by the library's kernels), "auto" (default) = whichever is shorter for the step's index set:
+    the list when the set holds fewer than N / 32 entries.  `last_wire` names the last step's choice.
+
     `engine`: the per-rank object with shard_select / selection / shard_gather / shard_apply (default: a
     Pruner on the current CUDA device)."""
 
     def __init__(self, layer_sizes: Sequence[int], W_total: int, ratio: float, eps: float = 1e-8, seed: int = 0,
-                 group=None, engine=None):
+                 group=None, engine=None, wire: str = "auto"):
         import torch
         import torch.distributed as dist
 
@@ -387,6 +416,9 @@ class ShardedPruner:
         self.W_total, self.W_local, self.seed, self.t = W_total, W_total // self.world, int(seed), 0
         self.leader_override = -1
         self.leader = -1
+        if wire not in ("auto", "list", "mask"):
+            raise ValueError("wire must be 'auto', 'list' or 'mask'")
+        self.wire, self.last_wire, self.wire_bytes = wire, None, 0
         self.local = engine if engine is not None else Pruner(layer_sizes, self.W_local, ratio, eps, seed)
         self.N, self.K = self.local.N, self.local.K
 
@@ -400,11 +432,25 @@ class ShardedPruner:
         leader = self.leader_override if self.leader_override >= 0 else iwp_leader_at(self.seed, self.t, self.W_total)
         owner, local_worker = divmod(leader, self.W_local)
         self.local.shard_select(grads_local, weights, update)
-        if self.rank == owner:
-            idx = self.local.selection(local_worker)[0]
+        n = self.K  # ratio mode: every step's index set has K entries, known to every rank
+        mask_bytes = 4 * ((self.N + 31) // 32)
+        use_mask = self.wire == "mask" or (self.wire == "auto" and 4 * n >= mask_bytes)
+        if use_mask:  # the encoded mask travels; every rank but the owner expands it back into the list
+            if self.rank == owner:
+                idx = self.local.selection(local_worker)[0]
+                bits = self.local.wire_pack(idx)
+            else:
+                bits = t.empty(mask_bytes, dtype=t.uint8, device=update.device)
+            dist.broadcast(bits, src=self._global_rank(owner), group=self.group)
+            if self.rank != owner:
+                idx = self.local.wire_unpack(bits, n)
         else:
-            idx = t.empty(self.K, dtype=t.int32, device=update.device)
-        dist.broadcast(idx, src=self._global_rank(owner), group=self.group)
+            if self.rank == owner:
+                idx = self.local.selection(local_worker)[0]
+            else:
+                idx = t.empty(n, dtype=t.int32, device=update.device)
+            dist.broadcast(idx, src=self._global_rank(owner), group=self.group)
+        self.last_wire, self.wire_bytes = ("mask" if use_mask else "list"), (mask_bytes if use_mask else 4 * n)
         vals_local = self.local.shard_gather(idx)
         vals_all = t.empty((self.W_total, self.K), dtype=t.float32, device=update.device)
         dist.all_gather_into_tensor(vals_all, vals_local, group=self.group)

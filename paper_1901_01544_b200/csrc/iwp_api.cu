@@ -7,6 +7,7 @@
 //   iwp_select.cuh     (c)+(d): exact radix select, ordered compaction, one-CTA path of small layers
 //   iwp_reduce.cuh     (e)-(g): reduction at the index set, zero mask, sharded phases, mask accessor
 //   iwp_threshold.cuh  absolute-threshold mode, random selection, layer-wise threshold
+//   iwp_wire.cuh       index list <-> one-bit-per-element mask (the two wire formats of the sharded step)
 // Nothing here is a dense contraction, so there are no tensor-core instructions: every kernel is bound by
 // HBM traffic (or, for the small ones, by launch latency).  The residual add, the eps guard and the division
 // use the explicit round-to-nearest intrinsics, so results do not depend on compiler contraction or fast-math
@@ -27,6 +28,7 @@
 #include "iwp_select.cuh"
 #include "iwp_stream.cuh"
 #include "iwp_threshold.cuh"
+#include "iwp_wire.cuh"
 
 using namespace iwp;
 
@@ -98,6 +100,9 @@ struct iwp_ctx {
   uint32_t* d_tcnt = nullptr;     // [chunk] selected elements of the chunk
   uint32_t* d_toff = nullptr;     // [chunk] list offset of the chunk
   uint32_t* d_list_len = nullptr; // length of the last step's index list
+  uint32_t* d_wire_cnt = nullptr; // [chunk of 32 Ki elements] set bits of a mask being expanded, then their offsets
+  uint32_t* d_wire_off = nullptr;
+  uint32_t* d_wire_len = nullptr; // length of the last expanded list
   uint32_t* zmask = nullptr;      // residuals sent in the last step and not yet zeroed (lazy step (g))
   uint64_t zmask_words = 0;
   bool zero_pending = false;      // zmask may hold marks
@@ -278,6 +283,9 @@ void free_all(iwp_ctx* c) {
   cudaFree(c->d_tcnt);
   cudaFree(c->d_toff);
   cudaFree(c->d_list_len);
+  cudaFree(c->d_wire_cnt);
+  cudaFree(c->d_wire_off);
+  cudaFree(c->d_wire_len);
   cudaFree(c->chunk_sfx);
   cudaFree(c->saved_w);
   cudaFree(c->sel_idx);
@@ -742,6 +750,13 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
   A(&c->sel_idx, sz.sel_idx);
   A(&c->sel_val, sz.sel_val);
   A(&c->d_status, sz.status);
+  {
+    const uint64_t wire_chunks = (((p.N + 31) >> 5) + WIRE_CHUNK_WORDS - 1) / WIRE_CHUNK_WORDS;
+    A(&c->d_wire_cnt, wire_chunks * sizeof(uint32_t));
+    A(&c->d_wire_off, wire_chunks * sizeof(uint32_t));
+    A(&c->d_wire_len, sizeof(uint32_t));
+    c->device_bytes += 2 * wire_chunks * sizeof(uint32_t) + sizeof(uint32_t);
+  }
   if (threshold_mode) {
     A(&c->d_thr, p.layers.size() * sizeof(uint32_t));
     A(&c->d_tcnt, at_least(p.chunks.size() * sizeof(uint32_t)));
@@ -1285,6 +1300,47 @@ int iwp_encode_mask(iwp_ctx* c, const uint8_t* mask, uint8_t* bits) {
   const uint64_t N = c->plan.N, n_bytes = (N + 7) / 8;
   k_pack_mask<<<static_cast<unsigned>((n_bytes + THREADS - 1) / THREADS), THREADS, 0, c->stream>>>(mask, bits, N);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
+  return IWP_OK;
+}
+
+int64_t iwp_wire_mask_bytes(int64_t N) { return N < 0 ? -1 : ((N + 31) / 32) * 4; }
+
+int iwp_wire_pack(iwp_ctx* c, const uint32_t* idx, int64_t n, uint8_t* bits) {
+  if (!c || (!idx && n > 0) || !bits || n < 0 || (reinterpret_cast<uintptr_t>(bits) & 3u)) return IWP_ERR_INVALID;
+  const uint64_t n_words = (c->plan.N + 31) >> 5;
+  if (cudaMemsetAsync(bits, 0, n_words * sizeof(uint32_t), c->stream) != cudaSuccess) {
+    cudaGetLastError();
+    return IWP_ERR_CUDA;
+  }
+  c->launches += 1;
+  if (n == 0) return IWP_OK;
+  k_wire_pack<<<static_cast<unsigned>((static_cast<uint64_t>(n) + THREADS - 1) / THREADS), THREADS, 0, c->stream>>>(
+      idx, static_cast<uint64_t>(n), reinterpret_cast<uint32_t*>(bits), c->plan.N, c->d_status);
+  IWP_LAUNCH_CHECK(c);
+  return IWP_OK;
+}
+
+int iwp_wire_unpack(iwp_ctx* c, const uint8_t* bits, uint32_t* idx, int64_t cap, int64_t* n_host) {
+  if (!c || !bits || (!idx && cap > 0) || cap < 0 || (reinterpret_cast<uintptr_t>(bits) & 3u)) return IWP_ERR_INVALID;
+  const uint64_t n_words = (c->plan.N + 31) >> 5;
+  const unsigned chunks = static_cast<unsigned>((n_words + WIRE_CHUNK_WORDS - 1) / WIRE_CHUNK_WORDS);
+  const uint32_t* words = reinterpret_cast<const uint32_t*>(bits);
+  k_wire_count<<<chunks, THREADS, 0, c->stream>>>(words, n_words, c->d_wire_cnt);
+  IWP_LAUNCH_CHECK(c);
+  k_thr_scan<<<1, 1024, 0, c->stream>>>(c->d_wire_cnt, c->d_wire_off, chunks, c->d_wire_len);
+  IWP_LAUNCH_CHECK(c);
+  k_wire_expand<<<chunks, THREADS, 0, c->stream>>>(words, n_words, c->d_wire_off, idx, static_cast<uint64_t>(cap),
+                                                  c->d_status);
+  IWP_LAUNCH_CHECK(c);
+  if (n_host) {
+    uint32_t v = 0;
+    if (cudaMemcpyAsync(&v, c->d_wire_len, sizeof(uint32_t), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess) {
+      cudaGetLastError();
+      return IWP_ERR_CUDA;
+    }
+    *n_host = static_cast<int64_t>(v);
+  }
   return IWP_OK;
 }
 

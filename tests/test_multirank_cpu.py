@@ -4,6 +4,7 @@ import os
 import socket
 import sys
 
+import pytest
 import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -101,6 +102,18 @@ class _NumpyEngine:
     def shard_gather(self, idx):
         return torch.from_numpy(self.np.ascontiguousarray(self.acc[:, idx.numpy()]))
 
+    def wire_pack(self, idx):
+        np = self.np
+        m = np.zeros(32 * ((self.N + 31) // 32), np.uint8)
+        m[idx.numpy()] = 1
+        return torch.from_numpy(np.packbits(m, bitorder="little"))
+
+    def wire_unpack(self, bits, n):
+        np = self.np
+        idx = np.flatnonzero(np.unpackbits(bits.numpy(), bitorder="little"))
+        assert idx.size == n
+        return torch.from_numpy(idx.astype(np.int32))
+
     def shard_apply(self, idx, vals_all, update):
         np = self.np
         v = vals_all.numpy()
@@ -114,7 +127,7 @@ class _NumpyEngine:
         pass
 
 
-def _sharded_rank_main(rank: int, world: int, port: int, out):
+def _sharded_rank_main(rank: int, world: int, port: int, out, wire="auto", ratio=8.0):
     import numpy as np
 
     sys.path.insert(0, ROOT)
@@ -123,9 +136,9 @@ def _sharded_rank_main(rank: int, world: int, port: int, out):
     import oracle
     from paper_1901_01544_b200.binding import ShardedPruner
 
-    layers, W_total, ratio, eps, seed = [300, 17, 1000], 4, 8.0, 1e-8, 5
+    layers, W_total, eps, seed = [300, 17, 1000], 4, 1e-8, 5
     N, Wl = sum(layers), W_total // world
-    sp = ShardedPruner(layers, W_total, ratio, eps, seed, engine=_NumpyEngine(layers, Wl, ratio, eps))
+    sp = ShardedPruner(layers, W_total, ratio, eps, seed, engine=_NumpyEngine(layers, Wl, ratio, eps), wire=wire)
     orc = oracle.Oracle(layers, W_total, ratio, eps, seed)  # the whole job on one "node"
     rng = np.random.default_rng(3)  # the same stream on every rank
     weights = rng.standard_normal(N).astype(np.float32)
@@ -139,16 +152,20 @@ def _sharded_rank_main(rank: int, world: int, port: int, out):
         for w in range(Wl):
             ok = ok and np.array_equal(sp.local.acc[w].view(np.uint32), orc.residual(rank * Wl + w).view(np.uint32))
         owners.add(sp.leader // Wl)
-    out.put((rank, bool(ok), sorted(owners)))
+    out.put((rank, bool(ok), sorted(owners), sp.last_wire, sp.wire_bytes))
     dist.barrier()
     dist.destroy_process_group()
 
 
-def test_workers_spread_over_two_ranks_equal_one_node():
+# wire, ratio -> what must have travelled: at ratio 8 the mask (N / 8 bytes) is shorter than the list (N / 2
+# bytes), at ratio 64 the list is
+@pytest.mark.parametrize("wire,ratio,expect", [("auto", 8.0, "mask"), ("auto", 64.0, "list"), ("list", 8.0, "list"),
+                                               ("mask", 64.0, "mask")])
+def test_workers_spread_over_two_ranks_equal_one_node(wire, ratio, expect):
     ctx = mp.get_context("spawn")
     out = ctx.Queue()
     port = _free_port()
-    procs = [ctx.Process(target=_sharded_rank_main, args=(r, 2, port, out)) for r in range(2)]
+    procs = [ctx.Process(target=_sharded_rank_main, args=(r, 2, port, out, wire, ratio)) for r in range(2)]
     for p in procs:
         p.start()
     got = sorted(out.get(timeout=180) for _ in procs)
@@ -157,6 +174,9 @@ def test_workers_spread_over_two_ranks_equal_one_node():
         assert p.exitcode == 0
     assert [g[1] for g in got] == [True, True]
     assert got[0][2] == [0, 1]  # the chosen worker lived on either rank at some step
+    assert [g[3] for g in got] == [expect, expect]
+    N, K = 1317, sum(min(n, max(1, -(-n // int(ratio)))) for n in (300, 17, 1000))
+    assert got[0][4] == (4 * ((N + 31) // 32) if expect == "mask" else 4 * K)
 
 
 def _sharded_bad_split_main(rank: int, world: int, port: int, out):
