@@ -11,7 +11,8 @@ import os
 from typing import List, Optional, Sequence, Tuple
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libiwp.so")
+# IWP_LIB_VARIANT=debug loads the build with range and count checks in every kernel (same ABI, slower)
+LIB_PATH = os.path.join(HERE, "libiwp_debug.so" if os.environ.get("IWP_LIB_VARIANT") == "debug" else "libiwp.so")
 
 IWP_OK, IWP_ERR_INVALID, IWP_ERR_OOM, IWP_ERR_CUDA, IWP_ERR_INTERNAL, IWP_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 IWP_ERR_CAPACITY = -6

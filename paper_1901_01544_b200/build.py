@@ -23,27 +23,34 @@ NVCC_FLAGS = [
 ]
 
 
-def stale() -> bool:
-    if not os.path.exists(LIB):
+# The same library with every computed index range-checked and the histogram counts checked for conservation
+# (a failed check sets the status word; nothing traps).  Loaded instead of libiwp.so when IWP_LIB_VARIANT=debug.
+LIB_DEBUG = os.path.join(HERE, "libiwp_debug.so")
+
+
+def stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     return any(os.path.getmtime(d) > t for d in DEPS)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not stale():
-        return LIB
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    lib = LIB_DEBUG if debug else LIB
+    if not force and not stale(lib):
+        return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + SOURCES + ["-o", LIB + ".tmp"]
+    cmd = ([nvcc] + NVCC_FLAGS + (["-DIWP_DEBUG_CHECKS"] if debug else []) + (["-Xptxas", "-v"] if verbose else []) +
+           SOURCES + ["-o", lib + ".tmp"])
     r = subprocess.run(cmd, capture_output=True, text=True)
     if r.returncode != 0:
         sys.stderr.write(r.stdout + r.stderr)
-        raise RuntimeError("nvcc failed building libiwp.so")
+        raise RuntimeError(f"nvcc failed building {os.path.basename(lib)}")
     if verbose:
         sys.stderr.write(r.stdout + r.stderr)
-    os.replace(LIB + ".tmp", LIB)
-    return LIB
+    os.replace(lib + ".tmp", lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose="-v" in sys.argv))
+    print(build(force=True, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -468,7 +468,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     stage_mark_at(c, 2);  // after the wait: the streaming stage is timed from where its first kernel may start
     k_stream<VEC, true><<<(n_tiles + WARPS - 1) / WARPS, THREADS, 0, s>>>(
         grads, weights, c->acc, update, c->d_tiles, c->info_cur, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
-        c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, 1, c->momentum);
+        c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, 1, c->momentum, c->d_status);
     IWP_LAUNCH_CHECK(c);
     // the leader's select and list, under the other workers' streaming pass
     if (!cuda_ok(cudaEventRecord(c->ev_lead, s)) || !cuda_ok(cudaStreamWaitEvent(c->side_a, c->ev_lead, 0)))
@@ -483,7 +483,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     k_stream<VEC, false><<<n_tiles * static_cast<unsigned>(groups), wpc * 32, 0, s>>>(
         grads, weights, c->acc, update, c->d_tiles, c->info_cur, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
         c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, groups,
-        c->momentum);
+        c->momentum, c->d_status);
     IWP_LAUNCH_CHECK(c);
     if (c->zero_pending) {  // every marked residual has now been overwritten: forget the marks
       if (!cuda_ok(cudaMemsetAsync(c->zmask, 0, c->zmask_words * sizeof(uint32_t), s))) return IWP_ERR_CUDA;
@@ -522,7 +522,8 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     if (!cuda_ok(cudaStreamWaitEvent(s, c->ev_lead_done, 0))) return IWP_ERR_CUDA;
     if (fork_small && !cuda_ok(cudaStreamWaitEvent(s, c->ev_join, 0))) return IWP_ERR_CUDA;
     k_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->sel_slot, c->side_val,
-                                              c->cand_val, c->acc, update, c->zmask, N, K, W, leader);
+                                              c->cand_val, c->acc, update, c->zmask, N, K, W, leader,
+                                              static_cast<uint64_t>(p.tiles.size()) * W, c->d_status);
     IWP_LAUNCH_CHECK(c);
     c->zero_pending = true;
     stage_mark_at(c, 6);
@@ -534,7 +535,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
       k_stream<VEC, true><<<(n_tiles + WARPS - 1) / WARPS, THREADS, 0, s>>>(
           grads, weights, c->acc, update, c->d_tiles, c->info_cur, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
           c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, 1,
-          c->momentum);
+          c->momentum, c->d_status);
       if (W > 1) {
         IWP_LAUNCH_CHECK(c);
         const int wpc = (W - 1 < WARPS) ? W - 1 : WARPS;  // warps (= workers) per CTA
@@ -542,7 +543,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
         k_stream<VEC, false><<<n_tiles * static_cast<unsigned>(groups), wpc * 32, 0, s>>>(
             grads, weights, c->acc, update, c->d_tiles, c->info_cur, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
             c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, groups,
-            c->momentum);
+            c->momentum, c->d_status);
       }
       if (c->zero_pending) {  // every marked residual has now been overwritten: forget the marks
         IWP_LAUNCH_CHECK(c);
@@ -617,7 +618,8 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     c->zero_pending = true;  // the marks are cleared with the next step's
   } else if (spec) {
     k_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->sel_slot, c->side_val,
-                                              c->cand_val, c->acc, update, c->zmask, N, K, W, leader);
+                                              c->cand_val, c->acc, update, c->zmask, N, K, W, leader,
+                                              static_cast<uint64_t>(p.tiles.size()) * W, c->d_status);
     c->zero_pending = true;
   } else {
     k_gather_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->acc, update,

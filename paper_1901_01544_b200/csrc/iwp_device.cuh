@@ -14,6 +14,22 @@ constexpr int WARPS = THREADS / 32;
 constexpr int STATUS_INTERNAL = -4;
 constexpr int STATUS_CAPACITY = -6;
 
+// Debug build (-DIWP_DEBUG_CHECKS, `python -m paper_1901_01544_b200.build --debug`): every computed index is
+// range-checked and the histogram counts are checked for conservation; a failed check sets the status word
+// (nothing traps).  In the release build the checks compile to nothing.
+#ifdef IWP_DEBUG_CHECKS
+#define IWP_DBG_CHECK(status, cond)                          \
+  do {                                                       \
+    if (!(cond)) atomicMin((status), STATUS_INTERNAL);       \
+  } while (0)
+constexpr bool DEBUG_CHECKS = true;
+#else
+#define IWP_DBG_CHECK(status, cond) \
+  do {                              \
+  } while (0)
+constexpr bool DEBUG_CHECKS = false;
+#endif
+
 // radix-select digit plan over the 32-bit importance pattern (bit 31 is always 0)
 __host__ __device__ constexpr int pass_shift(int pass) { return pass == 0 ? 21 : (pass == 1 ? 10 : 0); }
 __host__ __device__ constexpr int pass_bins(int pass) { return pass == 2 ? 1024 : 2048; }

@@ -163,11 +163,13 @@ __global__ void __launch_bounds__(THREADS)
     k_sum_scatter(const uint32_t* __restrict__ leader_idx, const uint32_t* __restrict__ sel_slot,
                   const float* __restrict__ side_val, const float* __restrict__ cand_val, float* __restrict__ acc,
                   float* __restrict__ update, uint32_t* __restrict__ zmask, uint64_t N, uint64_t K, int W,
-                  int leader) {
+                  int leader, uint64_t n_slots, int* __restrict__ status) {
   const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
   if (j >= K) return;
   const uint64_t i = leader_idx[j];
   const uint32_t ref = sel_slot[j];
+  // the entry is an element of the job, and it names a position of an existing (tile, worker) slot
+  IWP_DBG_CHECK(status, i < N && (ref >= REF_LAZY || (ref / CAND_CAP) * W + (W - 1) < n_slots));
   float s = 0.0f;
   if (ref < REF_LAZY) {
     const uint64_t tile = ref / CAND_CAP, at = ref % CAND_CAP;

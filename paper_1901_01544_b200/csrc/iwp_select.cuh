@@ -196,6 +196,14 @@ __global__ void __launch_bounds__(THREADS)
   if (pass == 0) {
     prefix = 0;
     krem = layers[large_ids[pair / W]].k;
+    if (DEBUG_CHECKS && info != nullptr && !pair_is_cand(info[pair], krem)) {
+      // multi-pass path: the first histogram pass counted every element of the layer exactly once
+      uint32_t part = 0;
+      for (int b = threadIdx.x; b < nb; b += THREADS) part += sh[b];
+      uint32_t total;
+      block_excl_scan(part, sh_scan, total);
+      if (threadIdx.x == 0) IWP_DBG_CHECK(status, total == layers[large_ids[pair / W]].n);
+    }
     if (threadIdx.x == 0 && reach_seen != nullptr) {
       // a pair that selects from its candidate slots: what the first histogram pass found in the slots must be
       // what the streaming pass put there (a lost, overwritten or stale entry shows up as a different count)
@@ -391,6 +399,8 @@ __global__ void __launch_bounds__(THREADS)
           const bool isg = (fg >> u) & 1u, ise = (fe >> u) & 1u;
           if (isg || (ise && qb < r)) {
             const uint32_t pos = gb + (qb < r ? qb : r);
+            // the listed element lies inside its layer; the slot entry is one of the stored ones
+            IWP_DBG_CHECK(status, tile_base + ii[u] >= L.off && tile_base + ii[u] - L.off < L.n && j + u < cnt);
             if (pos < L.k) {
               out_i[pos] = tile_base + ii[u];
               out_v[pos] = vv[u];

@@ -210,7 +210,8 @@ __global__ void __launch_bounds__(THREADS, 3)
              const uint2* __restrict__ guess_tab, uint32_t* __restrict__ cand_key, float* __restrict__ cand_val,
              uint16_t* __restrict__ cand_idx, uint32_t* __restrict__ cand_cnt, float* __restrict__ side_val,
              uint2* __restrict__ lead_lane, uint32_t* __restrict__ lead_tot, const uint32_t* __restrict__ zmask,
-             float eps, uint64_t N, int W, int leader, uint32_t n_tiles, int worker_groups, float momentum) {
+             float eps, uint64_t N, int W, int leader, uint32_t n_tiles, int worker_groups, float momentum,
+             int* __restrict__ status) {
   constexpr int ROUNDS = SEG_ELEMS / 128;  // 128-bit slots per lane and iteration = 4
   __shared__ __align__(16) float r_val[WARPS][SEG_ELEMS];  // results of the iteration, for run-time indexing
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -242,6 +243,7 @@ __global__ void __launch_bounds__(THREADS, 3)
   float* res = r_val[warp] + lane * 4;
   uint32_t count = 0;    // entries appended to the slot so far (the same in every lane)
   uint32_t reached = 0;  // of those, how many reach the guess exactly (this lane's share until the final reduction)
+  uint32_t dbg_passed = 0;  // debug build: elements of this lane that passed the pre-test (count conservation)
   const uint64_t keep = l2_evict_last_policy();
   // The tile covers the segments it0 .. it1 of its window.  The loads of segment it + 1 are issued
   // as soon as the arithmetic of segment it is done, so they are in flight while the rare-path work
@@ -256,9 +258,11 @@ __global__ void __launch_bounds__(THREADS, 3)
     const uint64_t seg = base + it * SEG_ELEMS;
     const uint64_t first = seg + static_cast<uint64_t>(lane) * 4;
     // residuals sent in the previous step count as +0 (they are overwritten either way)
+    IWP_DBG_CHECK(status, (seg >> 9) < (N >> 9) + 2);  // the segment's zero-mask fields exist
     zm_next = reinterpret_cast<const uint16_t*>(zmask)[(seg >> 9) * 32 + lane];
     if (!LEADER) {  // the leader's record for this segment: (mask | count << 16, lane prefix), round totals
       const uint64_t sigma = static_cast<uint64_t>(tile_id) * SEGS_PER_TILE + it;
+      IWP_DBG_CHECK(status, it < SEGS_PER_TILE && tile_id < n_tiles);
       ll_next = lead_lane[sigma * 32 + lane];
       lt_next = lead_tot[sigma];
     }
@@ -351,6 +355,7 @@ __global__ void __launch_bounds__(THREADS, 3)
       for (uint32_t mm = mL; mm; mm &= mm - 1) {
         const uint32_t b = __ffs(mm) - 1;
         const uint32_t pos = countL + staged_position(mL, ll.y, lt, b);
+        IWP_DBG_CHECK(status, pos < TILE && b < 16u);  // a rank inside the chosen node's tile, a bit of its 16-bit mask
         if (pos < CAND_CAP) st_keep_f32(side_val + slot + pos, res[(b >> 2) * 128 + (b & 3u)], keep);
       }
     }
@@ -377,6 +382,10 @@ __global__ void __launch_bounds__(THREADS, 3)
         const uint32_t b = __ffs(mm) - 1;
         const uint32_t pos = count + staged_position(m, excl, tot, b);
         const uint32_t off = (b >> 2) * 128 + (b & 3u);
+        // ranks inside an iteration stay below the iteration's total, and the element is one of the tile's
+        IWP_DBG_CHECK(status, pos - count < (tot & 0xFFu) + ((tot >> 8) & 0xFFu) + ((tot >> 16) & 0xFFu) + (tot >> 24));
+        IWP_DBG_CHECK(status, first + off >= lo && first + off < hi);
+        if (DEBUG_CHECKS) ++dbg_passed;
         const float v = res[off];
         const uint32_t key = imp_key_den(v, imp_den(weights[first + off], eps));  // weight re-read through L1
         reached += (key >= guess) ? 1u : 0u;
@@ -390,6 +399,10 @@ __global__ void __launch_bounds__(THREADS, 3)
     }
   }
   reached = __reduce_add_sync(0xffffffffu, reached);
+  if (DEBUG_CHECKS) {  // every element that passed the pre-test was given exactly one rank
+    dbg_passed = __reduce_add_sync(0xffffffffu, dbg_passed);
+    IWP_DBG_CHECK(status, dbg_passed == count);
+  }
   // pad the slot to a multiple of four entries with key 0, so that readers can take whole 128-bit
   // groups without testing every entry (no candidate has key 0: a zero guess is never used)
   {
