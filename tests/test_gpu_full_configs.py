@@ -77,7 +77,19 @@ def test_full_size_flat_2p30_on_layer_subset():
     if free < 60 * 2 ** 30:
         pytest.skip("needs about 50 GiB of device memory")
     steps = 4
-    sub = [0, 1, 63, 64, 95]  # includes layers that start at odd element offsets and both layer sizes
+    # The oracle runs on a slice of the layers (layers are independent in steps (a)-(d), and (e)-(g) are element-wise,
+    # so a slice of the inputs reproduces the slice of the outputs exactly): the first 24 layers (2^28 elements) plus
+    # layers that start at odd element offsets and have the other size, if the host has the memory for it
+    # (about 5 GB of residuals, 5 GB of gradients and the selection scratch), else five layers; all 96 layers on a
+    # host with more than 110 GiB free.
+    import psutil
+
+    host_free = psutil.virtual_memory().available
+    if host_free >= 110 * 2 ** 30:  # every layer: 16 GiB of residuals, 16 GiB of gradients, weights, update, scratch
+        sub = list(range(len(c.layer_sizes)))
+    else:
+        sub = (list(range(24)) + [63, 64, 95]) if host_free >= 40 * 2 ** 30 else [0, 1, 63, 64, 95]
+    print(f"host memory available: {host_free / 2 ** 30:.1f} GiB -> oracle on {len(sub)} of {len(c.layer_sizes)} layers")
     off = c.offsets()
     sizes = [c.layer_sizes[l] for l in sub]
     assert off[1] % 4 != 0 and c.W * c.N == 2 ** 32
