@@ -72,6 +72,7 @@ struct iwp_ctx {
   uint32_t* d_large_ids = nullptr;
   uint2* d_state = nullptr;
   uint32_t* d_hist = nullptr;
+  int32_t* d_layer_leader = nullptr;  // [layer] chosen node of each layer (option "per_layer_leaders")
   uint32_t* d_reach = nullptr;    // [pair] candidates reaching the guess as the first histogram pass saw them (count check)
   uint2* d_chunk_cnt = nullptr;
   PairInfo* d_info = nullptr;     // threshold guess and candidate totals per pair, two copies used in turn
@@ -265,6 +266,7 @@ void free_all(iwp_ctx* c) {
   cudaFree(c->d_state);
   cudaFree(c->d_hist);
   cudaFree(c->d_reach);
+  cudaFree(c->d_layer_leader);
   cudaFree(c->d_chunk_cnt);
   cudaFree(c->d_info);
   cudaFree(c->cand_key);
@@ -368,7 +370,7 @@ int select_and_write(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSe
   k_write<VEC><<<cgrid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur, c->cand_key,
                                           c->cand_val, c->cand_idx, c->cand_cnt, c->d_state, c->d_chunk_cnt, c->sel_idx,
                                           c->sel_val, c->sel_slot, sfx, c->d_status, c->eps, p.N, p.K, W, n_chunks,
-                                          leader, ws);
+                                          leader, ws, nullptr);
   IWP_LAUNCH_CHECK(c);
   return IWP_OK;
 }
@@ -417,6 +419,16 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     const int rc = flush_pending_zero(c);
     if (rc != IWP_OK) return rc;
   }
+  // one chosen node per layer: the table the kernels read it from (single-read path; the multi-pass path draws
+  // the nodes inside its reduction kernel)
+  const int32_t* lead_tab = nullptr;
+  if (per_layer && spec) {
+    const unsigned nl = static_cast<unsigned>(p.layers.size());
+    k_layer_leaders<<<(nl + THREADS - 1) / THREADS, THREADS, 0, s>>>(c->d_layer_leader, nl, c->seed,
+                                                                    static_cast<uint64_t>(c->t), W);
+    IWP_LAUNCH_CHECK(c);
+    lead_tab = c->d_layer_leader;
+  }
   stage_mark_at(c, 0);
   // Small layers touch nothing the tiled path touches until the final reduction, so when both kinds
   // exist their one-CTA kernel runs on a side stream, forked here and joined before the reduction.
@@ -431,7 +443,8 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
       ss = c->side;
     }
     k_small<<<grid, THREADS, dyn, ss>>>(grads, weights, c->acc, update, c->d_layers, c->d_small_ids, c->sel_idx,
-                                        c->sel_val, c->sel_slot, c->d_status, c->eps, N, K, leader, only_w, c->momentum);
+                                        c->sel_val, c->sel_slot, c->d_status, c->eps, N, K, leader, only_w, c->momentum,
+                                        lead_tab);
     IWP_LAUNCH_CHECK(c);
     if (fork_small && !cuda_ok(cudaEventRecord(c->ev_join, c->side))) return IWP_ERR_CUDA;
   }
@@ -468,7 +481,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     stage_mark_at(c, 2);  // after the wait: the streaming stage is timed from where its first kernel may start
     k_stream<VEC, true><<<(n_tiles + WARPS - 1) / WARPS, THREADS, 0, s>>>(
         grads, weights, c->acc, update, c->d_tiles, c->info_cur, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
-        c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, 1, c->momentum, c->d_status);
+        c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, 1, c->momentum, c->d_status, lead_tab);
     IWP_LAUNCH_CHECK(c);
     // the leader's select and list, under the other workers' streaming pass
     if (!cuda_ok(cudaEventRecord(c->ev_lead, s)) || !cuda_ok(cudaStreamWaitEvent(c->side_a, c->ev_lead, 0)))
@@ -483,7 +496,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     k_stream<VEC, false><<<n_tiles * static_cast<unsigned>(groups), wpc * 32, 0, s>>>(
         grads, weights, c->acc, update, c->d_tiles, c->info_cur, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
         c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, groups,
-        c->momentum, c->d_status);
+        c->momentum, c->d_status, lead_tab);
     IWP_LAUNCH_CHECK(c);
     if (c->zero_pending) {  // every marked residual has now been overwritten: forget the marks
       if (!cuda_ok(cudaMemsetAsync(c->zmask, 0, c->zmask_words * sizeof(uint32_t), s))) return IWP_ERR_CUDA;
@@ -523,7 +536,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     if (fork_small && !cuda_ok(cudaStreamWaitEvent(s, c->ev_join, 0))) return IWP_ERR_CUDA;
     k_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->sel_slot, c->side_val,
                                               c->cand_val, c->acc, update, c->zmask, N, K, W, leader,
-                                              static_cast<uint64_t>(p.tiles.size()) * W, c->d_status);
+                                              static_cast<uint64_t>(p.tiles.size()) * W, c->d_status, nullptr, 0u, nullptr, 0);
     IWP_LAUNCH_CHECK(c);
     c->zero_pending = true;
     stage_mark_at(c, 6);
@@ -535,7 +548,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
       k_stream<VEC, true><<<(n_tiles + WARPS - 1) / WARPS, THREADS, 0, s>>>(
           grads, weights, c->acc, update, c->d_tiles, c->info_cur, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
           c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, 1,
-          c->momentum, c->d_status);
+          c->momentum, c->d_status, lead_tab);
       if (W > 1) {
         IWP_LAUNCH_CHECK(c);
         const int wpc = (W - 1 < WARPS) ? W - 1 : WARPS;  // warps (= workers) per CTA
@@ -543,7 +556,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
         k_stream<VEC, false><<<n_tiles * static_cast<unsigned>(groups), wpc * 32, 0, s>>>(
             grads, weights, c->acc, update, c->d_tiles, c->info_cur, c->d_guess, c->cand_key, c->cand_val, c->cand_idx,
             c->cand_cnt, c->side_val, c->lead_lane, c->lead_tot, c->zmask, c->eps, N, W, leader, n_tiles, groups,
-            c->momentum, c->d_status);
+            c->momentum, c->d_status, lead_tab);
       }
       if (c->zero_pending) {  // every marked residual has now been overwritten: forget the marks
         IWP_LAUNCH_CHECK(c);
@@ -581,7 +594,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
       k_write<VEC><<<grid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur,
                                              c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
                                              c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, c->chunk_sfx,
-                                             c->d_status, c->eps, N, K, W, n_chunks, leader, ws);
+                                             c->d_status, c->eps, N, K, W, n_chunks, leader, ws, lead_tab);
     };
     if (split) {
       if (!cuda_ok(cudaEventRecord(c->ev_fork2, s)) || !cuda_ok(cudaStreamWaitEvent(c->side, c->ev_fork2, 0)))
@@ -605,21 +618,36 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     stage_mark_at(c, 6);
     return IWP_OK;
   }
-  if (per_layer) {
+  if (per_layer && spec) {
+    // every worker's value at its layer's chosen node's candidate positions came out of the streaming pass
+    k_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx, c->sel_slot, c->side_val, c->cand_val, c->acc, update, c->zmask,
+                                              N, K, W, leader, static_cast<uint64_t>(p.tiles.size()) * W, c->d_status,
+                                              c->d_layers, static_cast<uint32_t>(p.layers.size()), lead_tab, 0);
+    c->zero_pending = true;
+  } else if (per_layer) {
     k_layer_leader_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx, c->d_layers, static_cast<uint32_t>(p.layers.size()),
                                                            c->acc, update, nullptr, N, K, W, c->seed,
                                                            static_cast<uint64_t>(c->t));
   } else if (ls.n > 1) {
     // union of the chosen nodes' lists: the zero mask is all clear here (applied and cleared by the streaming
     // pass, or flushed at the start of a multi-pass step) and serves to give every element one owner
-    const uint64_t entries = static_cast<uint64_t>(ls.n) * K;
+    // r_1 played the chosen node's part in the streaming pass, so its list is reduced from the side values; only
+    // the elements that r_2 .. r_n add to the union are gathered from the residuals
+    const int first_node = spec ? 1 : 0;
+    if (spec) {
+      k_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->sel_slot, c->side_val,
+                                                c->cand_val, c->acc, update, c->zmask, N, K, W, leader,
+                                                static_cast<uint64_t>(p.tiles.size()) * W, c->d_status, nullptr, 0u, nullptr, 1);
+      IWP_LAUNCH_CHECK(c);
+    }
+    const uint64_t entries = static_cast<uint64_t>(ls.n - first_node) * K;
     k_union_sum_scatter<<<static_cast<unsigned>((entries + THREADS - 1) / THREADS), THREADS, 0, s>>>(
-        c->sel_idx, c->acc, update, c->zmask, N, K, W, ls);
+        c->sel_idx, c->acc, update, c->zmask, N, K, W, ls, c->d_layers, static_cast<uint32_t>(p.layers.size()), first_node);
     c->zero_pending = true;  // the marks are cleared with the next step's
   } else if (spec) {
     k_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->sel_slot, c->side_val,
                                               c->cand_val, c->acc, update, c->zmask, N, K, W, leader,
-                                              static_cast<uint64_t>(p.tiles.size()) * W, c->d_status);
+                                              static_cast<uint64_t>(p.tiles.size()) * W, c->d_status, nullptr, 0u, nullptr, 0);
     c->zero_pending = true;
   } else {
     k_gather_sum_scatter<<<gblocks, THREADS, 0, s>>>(c->sel_idx + static_cast<uint64_t>(leader) * K, c->acc, update,
@@ -735,6 +763,7 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
   A(&c->d_state, sz.state);
   A(&c->d_hist, sz.hist);
   A(&c->d_reach, sz.reach);
+  A(&c->d_layer_leader, p.layers.size() * sizeof(int32_t));
   A(&c->d_chunk_cnt, sz.chunk_cnt);
   A(&c->d_info, sz.info);
   A(&c->cand_key, sz.cand_key);
@@ -1587,7 +1616,7 @@ int run_select_static(StaticScratch* s, const float* residual, const float* weig
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   k_write<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, nullptr, &s->layer, &s->info, nullptr, nullptr,
                                          nullptr, nullptr, &s->state, s->chunk_cnt, idx, val, nullptr, nullptr,
-                                         &s->status, eps, 0, 0, 1, n_chunks, -1, all);
+                                         &s->status, eps, 0, 0, 1, n_chunks, -1, all, nullptr);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   return IWP_OK;
 }

@@ -38,13 +38,18 @@ __global__ void __launch_bounds__(THREADS)
 // Steps (e)-(g) with several chosen nodes (Algorithm 1: Mask = OR Mask_ri): the index set is the union
 // of the chosen nodes' lists.  One thread per list entry of every chosen node; the first thread to mark
 // an element in the (all-zero) bit mask owns it - gathers the W residuals, sums them in ascending
-// worker order, scatters the sum and zeroes the residuals - and every later entry with the same element
-// returns at once, so nothing is read after it was zeroed.  The marks stay set (the element is +0 now
-// whether or not the next streaming pass treats it so).
+// worker order and scatters the sum - and every later entry with the same element returns at once.  The
+// marks stay set and are the zeroing: the next streaming pass (or the flush before anything else looks at
+// the residuals) takes a marked residual as +0, which saves W scattered 4-byte stores per element here.
+// Only elements of one-CTA layers, which no streaming pass visits, are zeroed on the spot (their mark is
+// then redundant).
 __global__ void __launch_bounds__(THREADS)
     k_union_sum_scatter(const uint32_t* __restrict__ sel_idx, float* __restrict__ acc, float* __restrict__ update,
-                        uint32_t* __restrict__ seen, uint64_t N, uint64_t K, int W, LeaderSet ls) {
-  const uint64_t q = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
+                        uint32_t* __restrict__ seen, uint64_t N, uint64_t K, int W, LeaderSet ls,
+                        const LayerDesc* __restrict__ layers, uint32_t n_layers, int first_node) {
+  // first_node = 1: r_1's list was already reduced from the side values of the streaming pass (k_sum_scatter,
+  // which marked every element it owns); this launch covers the lists of r_2 .. r_n
+  const uint64_t q = static_cast<uint64_t>(first_node) * K + static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
   if (q >= static_cast<uint64_t>(ls.n) * K) return;
   const int j = static_cast<int>(q / K);
   int r = ls.r[0];
@@ -65,8 +70,15 @@ __global__ void __launch_bounds__(THREADS)
       if (w0 + u < W) s = (w0 + u == 0) ? v[u] : __fadd_rn(s, v[u]);
     }
   }
-  for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
   update[i] = __fadd_rn(0.0f, s);
+  uint32_t lo = 0, hi = n_layers - 1;  // the layer whose list segment holds this entry
+  const uint64_t e = q % K;
+  while (lo < hi) {
+    const uint32_t mid = (lo + hi + 1) >> 1;
+    if (layers[mid].koff <= e) lo = mid; else hi = mid - 1;
+  }
+  if (layers[lo].large_index < 0)
+    for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
 }
 
 // Steps (e)-(g) when every layer has its own chosen node (Algorithm 1 draws the node inside its loop over
@@ -163,9 +175,21 @@ __global__ void __launch_bounds__(THREADS)
     k_sum_scatter(const uint32_t* __restrict__ leader_idx, const uint32_t* __restrict__ sel_slot,
                   const float* __restrict__ side_val, const float* __restrict__ cand_val, float* __restrict__ acc,
                   float* __restrict__ update, uint32_t* __restrict__ zmask, uint64_t N, uint64_t K, int W,
-                  int leader, uint64_t n_slots, int* __restrict__ status) {
+                  int leader, uint64_t n_slots, int* __restrict__ status, const LayerDesc* __restrict__ layers,
+                  uint32_t n_layers, const int32_t* __restrict__ layer_leader, int mark_all) {
   const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
   if (j >= K) return;
+  if (layer_leader != nullptr) {
+    // one chosen node per layer: entry j lies in one layer's list segment and comes from that layer's node's list
+    // (leader_idx is then the base of all W lists)
+    uint32_t lo = 0, hi = n_layers - 1;  // last layer whose segment starts at or before j
+    while (lo < hi) {
+      const uint32_t mid = (lo + hi + 1) >> 1;
+      if (layers[mid].koff <= j) lo = mid; else hi = mid - 1;
+    }
+    leader = layer_leader[lo];
+    leader_idx += static_cast<uint64_t>(leader) * K;
+  }
   const uint64_t i = leader_idx[j];
   const uint32_t ref = sel_slot[j];
   // the entry is an element of the job, and it names a position of an existing (tile, worker) slot
@@ -203,9 +227,17 @@ __global__ void __launch_bounds__(THREADS)
       atomicOr(&zmask[zmask_word(i)], zmask_bit(i));
     } else {
       for (int w = 0; w < W; ++w) p[static_cast<uint64_t>(w) * N] = 0.0f;
+      if (mark_all) atomicOr(&zmask[zmask_word(i)], zmask_bit(i));  // a later launch must see that it is taken
     }
   }
   update[i] = __fadd_rn(0.0f, s);
+}
+
+// Option "per_layer_leaders": the chosen node of every layer for this step, one table entry per layer.
+__global__ void __launch_bounds__(THREADS)
+    k_layer_leaders(int32_t* __restrict__ layer_leader, uint32_t n_layers, uint64_t seed, uint64_t step, int W) {
+  const uint32_t l = blockIdx.x * THREADS + threadIdx.x;
+  if (l < n_layers) layer_leader[l] = layer_leader_at(seed, step, l, W);
 }
 
 // Applies a pending zero mask right away (accessors, reset, and the multi-pass path need the

@@ -295,7 +295,7 @@ __global__ void __launch_bounds__(THREADS)
             const uint2* __restrict__ state, const uint2* __restrict__ chunk_cnt, uint32_t* __restrict__ sel_idx,
             float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot, const uint32_t* __restrict__ chunk_sfx,
             int* __restrict__ status, float eps, uint64_t N, uint64_t K, int W, uint32_t n_chunks, int leader,
-            WorkerSel ws) {
+            WorkerSel ws, const int32_t* __restrict__ layer_leader) {
   __shared__ uint32_t sh_warp[WARPS];
   __shared__ uint32_t sh_base[2];
   const Chunk c = chunks[blockIdx.x];
@@ -339,7 +339,7 @@ __global__ void __launch_bounds__(THREADS)
   uint32_t* out_i = sel_idx + static_cast<uint64_t>(w) * K + L.koff;
   float* out_v = sel_val + static_cast<uint64_t>(w) * K + L.koff;
 
-  const bool is_leader = w == leader;
+  const bool is_leader = w == (layer_leader != nullptr ? layer_leader[c.layer] : leader);
   if (pair_is_cand(info[pair], L.k)) {
     // warp order is index order: count per warp, prefix over the warps, then every warp writes its
     // tiles front to back, ranking the entries of a slot with one warp scan per 128 entries
@@ -502,7 +502,8 @@ __global__ void __launch_bounds__(THREADS)
     k_small(const float* __restrict__ grads, const float* __restrict__ weights, float* __restrict__ acc,
             float* __restrict__ update, const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ small_ids,
             uint32_t* __restrict__ sel_idx, float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot,
-            int* __restrict__ status, float eps, uint64_t N, uint64_t K, int leader, int only_worker, float momentum) {
+            int* __restrict__ status, float eps, uint64_t N, uint64_t K, int leader, int only_worker, float momentum,
+            const int32_t* __restrict__ layer_leader) {
   extern __shared__ uint32_t keys[];
   __shared__ uint32_t hist[NBINS];
   __shared__ uint32_t sh_scan[THREADS];
@@ -511,6 +512,7 @@ __global__ void __launch_bounds__(THREADS)
   const LayerDesc L = layers[small_ids[blockIdx.x]];
   const int w = blockIdx.y;
   const int tid = threadIdx.x;
+  if (layer_leader != nullptr) leader = layer_leader[small_ids[blockIdx.x]];
   const uint32_t n = L.n;
   float* a = acc + static_cast<uint64_t>(w) * N + L.off;
   const float* g = grads + static_cast<uint64_t>(w) * N + L.off;

@@ -211,23 +211,24 @@ __global__ void __launch_bounds__(THREADS, 3)
              uint16_t* __restrict__ cand_idx, uint32_t* __restrict__ cand_cnt, float* __restrict__ side_val,
              uint2* __restrict__ lead_lane, uint32_t* __restrict__ lead_tot, const uint32_t* __restrict__ zmask,
              float eps, uint64_t N, int W, int leader, uint32_t n_tiles, int worker_groups, float momentum,
-             int* __restrict__ status) {
+             int* __restrict__ status, const int32_t* __restrict__ layer_leader) {
   constexpr int ROUNDS = SEG_ELEMS / 128;  // 128-bit slots per lane and iteration = 4
   __shared__ __align__(16) float r_val[WARPS][SEG_ELEMS];  // results of the iteration, for run-time indexing
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t tile_id;
-  int w;
+  int wi = 0;
   if (LEADER) {  // eight tiles of the leader per CTA
     tile_id = blockIdx.x * WARPS + warp;
-    w = leader;
     if (tile_id >= n_tiles) return;
   } else {  // up to eight of the other workers of one tile per CTA: the tile's weights come through L1
     tile_id = blockIdx.x / worker_groups;
-    const int wi = static_cast<int>(blockIdx.x % worker_groups) * static_cast<int>(blockDim.x >> 5) + warp;
+    wi = static_cast<int>(blockIdx.x % worker_groups) * static_cast<int>(blockDim.x >> 5) + warp;
     if (wi >= W - 1) return;
-    w = wi < leader ? wi : wi + 1;
   }
   const Tile t = tiles[tile_id];
+  // the chosen node: one per step, or (option "per_layer_leaders") the one drawn for this tile's layer
+  if (layer_leader != nullptr) leader = layer_leader[t.layer];
+  const int w = LEADER ? leader : (wi < leader ? wi : wi + 1);
   const uint64_t lo = t.a, hi = lo + t.len;
   const uint64_t base = lo & ~static_cast<uint64_t>(TILE - 1);
   const bool full = VEC && t.len == TILE;  // every slot of the window is inside the tile
