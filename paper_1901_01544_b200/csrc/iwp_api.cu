@@ -1084,9 +1084,11 @@ int iwp_shard_apply(iwp_ctx* c, const uint32_t* idx, int64_t n, const float* val
   if (const int rc = flush_pending_zero(c)) return rc;
   if (n > 0) {
     const unsigned blocks = static_cast<unsigned>((static_cast<uint64_t>(n) + THREADS - 1) / THREADS);
-    k_shard_apply<<<blocks, THREADS, 0, c->stream>>>(idx, vals_all, c->acc, update, c->plan.N, static_cast<uint64_t>(n),
-                                                    W_total, c->plan.W);
+    k_shard_apply<<<blocks, THREADS, 0, c->stream>>>(idx, vals_all, c->acc, update, c->zmask, c->d_layers,
+                                                    static_cast<uint32_t>(c->plan.layers.size()), c->plan.N,
+                                                    static_cast<uint64_t>(n), W_total, c->plan.W, c->d_status);
     IWP_LAUNCH_CHECK(c);
+    c->zero_pending = true;  // the marks are the zeroing of the tiled layers' residuals
   }
   c->t += 1;
   return IWP_OK;

@@ -133,17 +133,33 @@ __global__ void __launch_bounds__(THREADS)
 
 // ... and steps (f), (g): the values of ALL workers of the job at the index set, in global worker order
 // (vals_all[w][j], w < W_total), are summed in that order into the (already zeroed) update, and this
-// context's own residuals are zeroed there.  One thread per entry.
+// context's own residuals are zeroed there: by a mark in the zero mask, which the next streaming pass applies
+// while it reads the residuals anyway (instead of W_local scattered 4-byte stores per entry); elements of
+// one-CTA layers, which no streaming pass visits, are zeroed on the spot.  One thread per entry.
 __global__ void __launch_bounds__(THREADS)
     k_shard_apply(const uint32_t* __restrict__ idx, const float* __restrict__ vals_all, float* __restrict__ acc,
-                  float* __restrict__ update, uint64_t N, uint64_t n, int W_total, int W_local) {
+                  float* __restrict__ update, uint32_t* __restrict__ zmask, const LayerDesc* __restrict__ layers,
+                  uint32_t n_layers, uint64_t N, uint64_t n, int W_total, int W_local, int* __restrict__ status) {
   const uint64_t j = static_cast<uint64_t>(blockIdx.x) * THREADS + threadIdx.x;
   if (j >= n) return;
   const uint64_t i = idx[j];
+  if (i >= N) {  // not an element of this job: reported, nothing written
+    atomicMin(status, STATUS_INTERNAL);
+    return;
+  }
   float s = vals_all[j];
   for (int w = 1; w < W_total; ++w) s = __fadd_rn(s, vals_all[static_cast<uint64_t>(w) * n + j]);
   update[i] = __fadd_rn(0.0f, s);
-  for (int w = 0; w < W_local; ++w) acc[static_cast<uint64_t>(w) * N + i] = 0.0f;
+  uint32_t lo = 0, hi = n_layers - 1;  // the layer that holds element i
+  while (lo < hi) {
+    const uint32_t mid = (lo + hi + 1) >> 1;
+    if (layers[mid].off <= i) lo = mid; else hi = mid - 1;
+  }
+  if (layers[lo].large_index < 0) {
+    for (int w = 0; w < W_local; ++w) acc[static_cast<uint64_t>(w) * N + i] = 0.0f;
+  } else {
+    atomicOr(&zmask[zmask_word(i)], zmask_bit(i));
+  }
 }
 
 // A worker's select that is left running on a side stream past the end of the step may still need
