@@ -722,7 +722,7 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
   if (!c) return IWP_ERR_OOM;
   try {
     c->plan = make_plan(layer_sizes, n_layers, W, ratio, eps, threshold_mode ? 0u : SMALL_MAX,
-                        threshold_mode ? THRESHOLD_CHUNK_TILES : CHUNK_TILES);
+                        threshold_mode ? THRESHOLD_CHUNK_TILES : 0u);
   } catch (...) {
     delete c;
     return IWP_ERR_OOM;
@@ -1549,7 +1549,7 @@ namespace {
 
 constexpr int64_t STATIC_MAX_N = int64_t(1) << 24;  // largest layer the fixed scratch is sized for
 constexpr uint32_t STATIC_CHUNK_ELEMS = CHUNK_TILES * TILE;
-constexpr uint32_t STATIC_MAX_CHUNKS = static_cast<uint32_t>(STATIC_MAX_N / STATIC_CHUNK_ELEMS) + 1;  // 33
+constexpr uint32_t STATIC_MAX_CHUNKS = static_cast<uint32_t>(STATIC_MAX_N / STATIC_CHUNK_ELEMS) + 1;
 
 struct StaticScratch {
   uint32_t hist[NBINS];  // must be zero when a select starts

@@ -6,7 +6,8 @@
 // shared memory); all others are cut into tiles and chunks:
 //   tile   <= TILE consecutive elements of ONE layer, never crossing a multiple of TILE of the
 //          flat element space, so that a tile is at most TILE/4 aligned 128-bit slots;
-//   chunk  <= CHUNK_TILES consecutive tiles of one layer: the unit of work of the select kernels.
+//   chunk  <= CHUNK_TILES consecutive tiles of one layer: the unit of work of the select kernels (8 .. 128
+//          tiles, by the size of the job: see chunk_tiles_for).
 #pragma once
 #include <cmath>
 #include <cstddef>
@@ -16,7 +17,8 @@
 namespace iwp {
 
 constexpr uint32_t TILE = 4096;
-constexpr uint32_t CHUNK_TILES = 128;
+constexpr uint32_t CHUNK_TILES = 128;      // largest chunk
+constexpr uint32_t CHUNK_TILES_MIN = 8;
 constexpr uint32_t SMALL_MAX = 16384;
 constexpr uint32_t NBINS = 2048;
 constexpr int32_t MAX_WORKERS = 65535;  // workers index the y dimension of several grids
@@ -58,6 +60,17 @@ struct Chunk {
   uint32_t n_tiles;
   uint32_t first_chunk_of_layer;
 };
+
+// Tiles per chunk for a job of total_tiles tiles and W workers.  A (chunk, worker) is one CTA of the select
+// kernels, which are latency bound: a small job cut into 128-tile chunks would run them on a handful of SMs
+// (one layer of 2^20 elements and four workers: 8 CTAs), while cutting a large job finer only multiplies the
+// per-chunk histogram merges and suffix tables (measured slower).  At least about 256 CTAs per launch where
+// the job has them, 8 to 128 tiles per chunk, a power of two.
+inline uint32_t chunk_tiles_for(uint64_t total_tiles, int32_t W) {
+  uint32_t ct = CHUNK_TILES_MIN;
+  while (ct < CHUNK_TILES && static_cast<uint64_t>(ct) * 2 * 256 <= total_tiles * static_cast<uint64_t>(W)) ct *= 2;
+  return ct;
+}
 
 inline int64_t keep_count(int64_t n, double ratio) {
   if (n < 1 || !(ratio >= 1.0) || !std::isfinite(ratio)) return 0;
@@ -166,9 +179,9 @@ struct Plan {
 
 // small_max: layers of at most this many elements take the one-CTA path (0: every layer is tiled, no
 // threshold sampling - the plan of the absolute-threshold mode, which also uses smaller chunks because
-// its select kernels walk one worker only and need the parallelism).
+// its select kernels walk one worker only and need the parallelism).  chunk_tiles = 0: by layer size.
 inline Plan make_plan(const int64_t* sizes, int32_t n_layers, int32_t W, double ratio, float eps,
-                      uint32_t small_max = SMALL_MAX, uint32_t chunk_tiles = CHUNK_TILES) {
+                      uint32_t small_max = SMALL_MAX, uint32_t chunk_tiles_fixed = 0) {
   Plan p;
   if (!sizes || n_layers < 1 || W < 1 || W > MAX_WORKERS || !(ratio >= 1.0) || !std::isfinite(ratio) ||
       !(eps > 0.f) || !std::isfinite(eps))
@@ -180,6 +193,10 @@ inline Plan make_plan(const int64_t* sizes, int32_t n_layers, int32_t W, double 
     if (N >= (1ull << 32)) return p;
   }
   p.W = W;
+  uint64_t total_tiles = 0;  // of the tiled layers (an upper estimate: ragged layer ends add a tile here and there)
+  for (int32_t l = 0; l < n_layers; ++l)
+    if (static_cast<uint64_t>(sizes[l]) > small_max) total_tiles += (static_cast<uint64_t>(sizes[l]) + TILE - 1) / TILE;
+  const uint32_t chunk_tiles = chunk_tiles_fixed ? chunk_tiles_fixed : chunk_tiles_for(total_tiles, W);
   uint64_t off = 0, koff = 0;
   for (int32_t l = 0; l < n_layers; ++l) {
     LayerDesc d{};

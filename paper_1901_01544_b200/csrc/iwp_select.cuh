@@ -9,20 +9,20 @@
 
 namespace iwp {
 
-// The candidates of (chunk, worker): warp q takes the chunk's tiles 16 q .. 16 q + 15 (consecutive,
+// The candidates of (chunk, worker): warp q takes the q-th eighth of the chunk's tiles (consecutive,
 // so that warp order is index order), four tiles at a time; each lane reads entries 4 lane .. 4 lane + 3
 // of a slot with one 128-bit load (a slot rarely holds more than 128 entries; a tail loop covers the
 // rest) and all loads of a batch are issued before any is used.  `f(key)` sees every stored candidate,
 // and in addition some keys 0 (padding, slots shorter than 128 entries), which `f` must ignore - every
 // use below does so by construction, because a candidate's key and first digit are never 0.
-constexpr uint32_t TILES_PER_WARP = CHUNK_TILES / WARPS;
+__device__ __forceinline__ uint32_t tiles_per_warp(const Chunk& c) { return (c.n_tiles + WARPS - 1) / WARPS; }
 
 template <typename F>
 __device__ __forceinline__ void for_each_candidate(const Chunk& c, int w, int W, const uint32_t* __restrict__ cand_cnt,
                                                    const uint32_t* __restrict__ cand_key, F&& f) {
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t t_begin = warp * TILES_PER_WARP;
-  const uint32_t t_end = min(c.n_tiles, t_begin + TILES_PER_WARP);
+  const uint32_t t_begin = min(c.n_tiles, warp * tiles_per_warp(c));
+  const uint32_t t_end = min(c.n_tiles, t_begin + tiles_per_warp(c));
   for (uint32_t tb = t_begin; tb < t_end; tb += 4) {
     uint32_t cnt[4];
     uint4 k4[4];
@@ -366,8 +366,8 @@ __global__ void __launch_bounds__(THREADS)
       q_before += sh_we[q];
     }
     if ((my_gt | my_eq) == 0) return;  // nothing of this warp's tiles is selected
-    const uint32_t t_begin = warp * TILES_PER_WARP;
-    const uint32_t t_end = min(c.n_tiles, t_begin + TILES_PER_WARP);
+    const uint32_t t_begin = min(c.n_tiles, warp * tiles_per_warp(c));
+    const uint32_t t_end = min(c.n_tiles, t_begin + tiles_per_warp(c));
     // ranks the entries [j0, j0 + 128) of one slot with a warp scan and writes the selected ones
     auto emit = [&](uint32_t tile, uint64_t tw, uint32_t cnt, uint32_t tile_base, uint32_t j0, uint4 k) {
       const uint32_t j = j0 + lane * 4;
