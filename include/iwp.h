@@ -305,6 +305,11 @@ int iwp_host_wait(iwp_ctx* ctx);
  *                      its own top-k
  *   "speculate"        1 (default) = sample-based threshold guess so that large layers are
  *                      read once; 0 = always the multi-pass exact select.  Both are exact.
+ *   "pair_select"      1 = on the single-read path, layers of at most 640 tiles (2.6 M elements) are selected
+ *                      and listed by one kernel launch with one thread-block cluster per (layer, worker)
+ *                      pair; 0 = every tiled layer goes through the chain of histogram, digit and compaction
+ *                      launches; -1 (default) = the library decides at create: the cluster launch for small
+ *                      jobs (at most 64 pairs, no larger layer), where it is faster.  Same results either way.
  *   "overlap"          1 = the leader's select runs beside the other workers' streaming pass and the
  *                      other workers' selects beside the reduction and the head of the next step;
  *                      0 = every kernel of a step in one sequence.  Same results either way; the

@@ -43,6 +43,10 @@ struct iwp_ctx {
   int64_t leader_override = -1;
   bool force_scalar = false;
   bool speculate = true;
+  // option: layers of at most PAIR_MAX_TILES tiles are selected by one cluster launch (k_select_pair) instead of
+  // the chain; -1 = decided by the size of the job at create (see below), 0 = never, 1 = always
+  int pair_select = -1;
+  bool pair_select_auto = false;
   bool select_only = false;  // iwp_shard_select(): a step stops before the reduction
   bool leader_only_select = false;  // option: only the chosen node selects; the other workers' lists are not produced
   cudaStream_t stream = nullptr;
@@ -70,6 +74,9 @@ struct iwp_ctx {
   Chunk* d_chunks = nullptr;
   uint32_t* d_small_ids = nullptr;
   uint32_t* d_large_ids = nullptr;
+  uint32_t* d_pair_ids = nullptr;      // layers the single-read path selects with one CTA per (layer, worker) pair
+  uint32_t* d_chain_large = nullptr;   // the other tiled layers (indices among the tiled layers) ...
+  uint32_t* d_chain_chunks = nullptr;  // ... and their chunks
   uint2* d_state = nullptr;
   uint32_t* d_hist = nullptr;
   int32_t* d_layer_leader = nullptr;  // [layer] chosen node of each layer (option "per_layer_leaders")
@@ -263,6 +270,9 @@ void free_all(iwp_ctx* c) {
   cudaFree(c->d_chunks);
   cudaFree(c->d_small_ids);
   cudaFree(c->d_large_ids);
+  cudaFree(c->d_pair_ids);
+  cudaFree(c->d_chain_large);
+  cudaFree(c->d_chain_chunks);
   cudaFree(c->d_state);
   cudaFree(c->d_hist);
   cudaFree(c->d_reach);
@@ -347,8 +357,41 @@ int flush_pending_zero(iwp_ctx* c) {
   return IWP_OK;
 }
 
-// Exact select (three histogram passes with their digit decisions) and ordered compaction of the
-// workers `ws` covers, on stream `st`.
+// Which tiled layers the chain of histogram / digit / compaction launches covers in a step.
+struct ChainScope {
+  const uint32_t* chunk_ids;  // nullptr: every chunk
+  const uint32_t* large_sel;  // nullptr: every tiled layer
+  unsigned n_chunks, n_large;
+  bool pairs;                 // the layers left out are selected by k_select_pair
+};
+
+// With speculation the layers of at most PAIR_MAX_TILES tiles are selected and listed by one CTA per pair.
+ChainScope chain_scope(const iwp_ctx* c, bool spec) {
+  const Plan& p = c->plan;
+  const bool on = c->pair_select < 0 ? c->pair_select_auto : c->pair_select == 1;
+  if (spec && on && !p.pair_layers.empty())
+    return ChainScope{c->d_chain_chunks, c->d_chain_large, static_cast<unsigned>(p.chain_chunks.size()),
+                      static_cast<unsigned>(p.chain_large.size()), true};
+  return ChainScope{nullptr, nullptr, static_cast<unsigned>(p.chunks.size()), static_cast<unsigned>(p.large_layers.size()), false};
+}
+
+template <bool VEC>
+int launch_pair_select(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSel ws, int32_t leader,
+                       const int32_t* lead_tab) {
+  const Plan& p = c->plan;
+  const unsigned n_sel = static_cast<unsigned>(sel_count(ws, p.W));
+  if (n_sel == 0 || p.pair_layers.empty()) return IWP_OK;
+  k_select_pair<VEC><<<dim3(static_cast<unsigned>(p.pair_layers.size()) * PAIR_CLUSTER, n_sel), THREADS,
+                       PAIR_KEYS_SMEM * sizeof(uint32_t), st>>>(
+      c->acc, weights, c->d_tiles, c->d_layers, c->d_pair_ids, c->info_cur, c->cand_key, c->cand_val, c->cand_idx,
+      c->cand_cnt, c->d_state, c->sel_idx, c->sel_val, c->sel_slot, c->d_status, c->eps, p.N, p.K, p.W, leader, ws, lead_tab);
+  IWP_LAUNCH_CHECK(c);
+  return IWP_OK;
+}
+
+// Exact select and ordered compaction of the workers `ws` covers, on stream `st` (single-read path): one
+// launch for the layers selected per pair, the chain (three histogram passes with their digit decisions, then
+// the compaction) for the others.
 template <bool VEC>
 int select_and_write(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSel ws, int32_t leader) {
   const Plan& p = c->plan;
@@ -356,21 +399,27 @@ int select_and_write(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSe
   const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
   const unsigned n_sel = static_cast<unsigned>(sel_count(ws, W));
   if (n_sel == 0) return IWP_OK;
-  dim3 cgrid(n_chunks, n_sel), pgrid(static_cast<unsigned>(p.large_layers.size()), n_sel);
+  const ChainScope sc = chain_scope(c, true);
+  if (sc.pairs) {
+    const int rc = launch_pair_select<VEC>(c, weights, st, ws, leader, nullptr);
+    if (rc != IWP_OK) return rc;
+  }
+  if (sc.n_chunks == 0) return IWP_OK;
+  dim3 cgrid(sc.n_chunks, n_sel), pgrid(sc.n_large, n_sel);
   uint32_t* sfx = c->chunk_sfx;
   for (int pass = 0; pass < N_PASSES; ++pass) {
     k_hist<VEC><<<cgrid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_layers, c->info_cur, c->cand_key,
                                            c->cand_cnt, c->d_state, c->d_hist, sfx, c->d_chunk_cnt, c->d_reach, c->eps, p.N,
-                                           W, pass, n_chunks, ws);
+                                           W, pass, n_chunks, ws, sc.chunk_ids);
     IWP_LAUNCH_CHECK(c);
     k_find_digit<<<pgrid, THREADS, 0, st>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->info_cur, c->d_reach,
-                                            c->d_status, W, pass, ws);
+                                            c->d_status, W, pass, ws, sc.large_sel);
     IWP_LAUNCH_CHECK(c);
   }
   k_write<VEC><<<cgrid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur, c->cand_key,
                                           c->cand_val, c->cand_idx, c->cand_cnt, c->d_state, c->d_chunk_cnt, c->sel_idx,
                                           c->sel_val, c->sel_slot, sfx, c->d_status, c->eps, p.N, p.K, W, n_chunks,
-                                          leader, ws, nullptr);
+                                          leader, ws, nullptr, sc.chunk_ids);
   IWP_LAUNCH_CHECK(c);
   return IWP_OK;
 }
@@ -574,14 +623,19 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
     const WorkerSel all = only ? WorkerSel{WorkerSel::ONLY, leader, -1} : WorkerSel{WorkerSel::ALL, 0, -1};
     const unsigned n_sel = static_cast<unsigned>(sel_count(all, W));
-    dim3 cgrid(n_chunks, n_sel), pgrid(static_cast<unsigned>(p.large_layers.size()), n_sel);
-    for (int pass = 0; pass < N_PASSES; ++pass) {
+    const ChainScope sc = chain_scope(c, spec);
+    if (sc.pairs) {  // select and list in one launch for the layers small enough for one CTA per pair
+      const int rc = launch_pair_select<VEC>(c, weights, s, all, leader, lead_tab);
+      if (rc != IWP_OK) return rc;
+    }
+    dim3 cgrid(sc.n_chunks, n_sel), pgrid(sc.n_large, n_sel);
+    for (int pass = 0; pass < N_PASSES && sc.n_chunks > 0; ++pass) {
       k_hist<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->info_cur, c->cand_key,
                                             c->cand_cnt, c->d_state, c->d_hist, c->chunk_sfx, c->d_chunk_cnt, c->d_reach,
-                                            c->eps, N, W, pass, n_chunks, all);
+                                            c->eps, N, W, pass, n_chunks, all, sc.chunk_ids);
       IWP_LAUNCH_CHECK(c);
       k_find_digit<<<pgrid, THREADS, 0, s>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->info_cur, c->d_reach,
-                                             c->d_status, W, pass, all);
+                                             c->d_status, W, pass, all, sc.large_sel);
       IWP_LAUNCH_CHECK(c);
     }
     stage_mark_at(c, 4);
@@ -590,11 +644,12 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     // (a union needs every chosen node's list here, a sharded step every list)
     const bool split = spec && W > 1 && ls.n == 1 && !per_layer && !c->select_only && !only && c->side != nullptr;
     auto write = [&](cudaStream_t st, WorkerSel ws) {
-      dim3 grid(n_chunks, static_cast<unsigned>(sel_count(ws, W)));
+      if (sc.n_chunks == 0) return;
+      dim3 grid(sc.n_chunks, static_cast<unsigned>(sel_count(ws, W)));
       k_write<VEC><<<grid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur,
                                              c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
                                              c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, c->chunk_sfx,
-                                             c->d_status, c->eps, N, K, W, n_chunks, leader, ws, lead_tab);
+                                             c->d_status, c->eps, N, K, W, n_chunks, leader, ws, lead_tab, sc.chunk_ids);
     };
     if (split) {
       if (!cuda_ok(cudaEventRecord(c->ev_fork2, s)) || !cuda_ok(cudaStreamWaitEvent(c->side, c->ev_fork2, 0)))
@@ -760,6 +815,9 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
   A(&c->d_chunks, sz.chunks);
   A(&c->d_small_ids, sz.small_ids);
   A(&c->d_large_ids, sz.large_ids);
+  A(&c->d_pair_ids, at_least(p.pair_layers.size() * sizeof(uint32_t)));
+  A(&c->d_chain_large, at_least(p.chain_large.size() * sizeof(uint32_t)));
+  A(&c->d_chain_chunks, at_least(p.chain_chunks.size() * sizeof(uint32_t)));
   A(&c->d_state, sz.state);
   A(&c->d_hist, sz.hist);
   A(&c->d_reach, sz.reach);
@@ -815,6 +873,9 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
   H2D(c->d_chunks, p.chunks.data(), p.chunks.size() * sizeof(Chunk));
   H2D(c->d_small_ids, p.small_layers.data(), p.small_layers.size() * sizeof(uint32_t));
   H2D(c->d_large_ids, p.large_layers.data(), p.large_layers.size() * sizeof(uint32_t));
+  H2D(c->d_pair_ids, p.pair_layers.data(), p.pair_layers.size() * sizeof(uint32_t));
+  H2D(c->d_chain_large, p.chain_large.data(), p.chain_large.size() * sizeof(uint32_t));
+  H2D(c->d_chain_chunks, p.chain_chunks.data(), p.chain_chunks.size() * sizeof(uint32_t));
   ok = ok && cudaMemset(c->acc, 0, sz.acc) == cudaSuccess;
   ok = ok && cudaMemset(c->d_state, 0, sz.state) == cudaSuccess;
   ok = ok && cudaMemset(c->d_hist, 0, sz.hist) == cudaSuccess;
@@ -836,6 +897,11 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
     ok = cudaFuncSetAttribute(k_sample, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               static_cast<int>(c->max_sample * sizeof(uint32_t))) == cudaSuccess;
   }
+  if (ok && !p.pair_layers.empty()) {
+    const int dyn = static_cast<int>(PAIR_KEYS_SMEM * sizeof(uint32_t));
+    ok = cudaFuncSetAttribute(k_select_pair<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) == cudaSuccess;
+    ok = ok && cudaFuncSetAttribute(k_select_pair<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, dyn) == cudaSuccess;
+  }
   if (ok && p.max_small_n) {
     ok = cudaFuncSetAttribute(k_small, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               static_cast<int>(p.max_small_n * sizeof(uint32_t))) == cudaSuccess;
@@ -856,6 +922,13 @@ int create_common(iwp_ctx** out, const int64_t* layer_sizes, int32_t n_layers, i
       ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
   }
   c->info_cur = c->d_info;
+  // One cluster per (layer, worker) pair costs about 25 us whatever the pair's size (nine cluster barriers, three
+  // histogram merges through distributed shared memory) and holds eight CTA slots meanwhile.  With a few pairs
+  // that beats the seven dependent launches of the chain (one layer of 2^20 elements, four workers: select and
+  // compaction 0.045 -> 0.027 ms); with hundreds of pairs the clusters queue up in waves while every launch of
+  // the chain covers all pairs at once (161-tensor network shape, 368 pairs: 0.15 -> 0.30 ms).  So: by default
+  // only for jobs of at most 64 pairs that have no layer left for the chain.
+  c->pair_select_auto = !threshold_mode && p.chain_large.empty() && p.pair_layers.size() * static_cast<size_t>(W) <= 64;
   {  // the overlapped schedule costs extra launches: it pays once a step streams some hundred megabytes
     uint64_t tiled = 0;
     for (uint32_t l : p.large_layers) tiled += p.layers[l].n;
@@ -1458,6 +1531,11 @@ int iwp_set_option(iwp_ctx* c, const char* key, int64_t v) {
     c->overlap = static_cast<int>(v);
     return IWP_OK;
   }
+  if (!std::strcmp(key, "pair_select")) {
+    if (v < -1 || v > 1) return IWP_ERR_INVALID;
+    c->pair_select = static_cast<int>(v);
+    return IWP_OK;
+  }
   if (!std::strcmp(key, "speculate")) {
     if (v != 0 && v != 1) return IWP_ERR_INVALID;
     c->speculate = v != 0;
@@ -1607,10 +1685,10 @@ int run_select_static(StaticScratch* s, const float* residual, const float* weig
   const WorkerSel all{WorkerSel::ALL, 0, -1};
   for (int pass = 0; pass < N_PASSES; ++pass) {
     k_hist<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr, &s->state,
-                                          s->hist, nullptr, nullptr, nullptr, eps, 0, 1, pass, n_chunks, all);
+                                          s->hist, nullptr, nullptr, nullptr, eps, 0, 1, pass, n_chunks, all, nullptr);
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
     k_find_digit<<<1, THREADS, 0, st>>>(&s->state, s->hist, &s->layer, &s->large_id, &s->info, nullptr, &s->status, 1, pass,
-                                        all);
+                                        all, nullptr);
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   }
   k_count<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr, &s->state,
@@ -1618,7 +1696,7 @@ int run_select_static(StaticScratch* s, const float* residual, const float* weig
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   k_write<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, nullptr, &s->layer, &s->info, nullptr, nullptr,
                                          nullptr, nullptr, &s->state, s->chunk_cnt, idx, val, nullptr, nullptr,
-                                         &s->status, eps, 0, 0, 1, n_chunks, -1, all, nullptr);
+                                         &s->status, eps, 0, 0, 1, n_chunks, -1, all, nullptr, nullptr);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   return IWP_OK;
 }

@@ -151,8 +151,9 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t x) {
   return x;
 }
 
-// Exclusive prefix sum over the block in thread order; `total` = block sum.
-// sh_warp: WARPS words of shared memory.  Contains two __syncthreads().
+// Exclusive prefix sum over the block (NW warps) in thread order; `total` = block sum.
+// sh_warp: NW words of shared memory.  Contains two __syncthreads().
+template <int NW = WARPS>
 __device__ __forceinline__ uint32_t block_excl_scan(uint32_t x, uint32_t* sh_warp, uint32_t& total) {
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const uint32_t incl = warp_incl_scan(x);
@@ -160,7 +161,7 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t x, uint32_t* sh_war
   __syncthreads();
   uint32_t woff = 0, tot = 0;
 #pragma unroll
-  for (int i = 0; i < WARPS; ++i) {
+  for (int i = 0; i < NW; ++i) {
     const uint32_t v = sh_warp[i];
     if (i < wid) woff += v;
     tot += v;

@@ -28,6 +28,9 @@ constexpr uint32_t SAMPLE_MAX = 16384;
 constexpr uint32_t GUESS_NONE = 0xffffffffu;  // no importance pattern reaches this value
 constexpr uint32_t SEG_ELEMS = 512;           // elements a warp handles per iteration of the streaming pass
 constexpr uint32_t SEGS_PER_TILE = TILE / SEG_ELEMS;
+// single-read path, one-launch select: a (layer, worker) pair of at most this many tiles is selected and listed
+// by one CTA from its candidate slots; larger layers take the multi-launch chain
+constexpr uint32_t PAIR_MAX_TILES = 640;
 constexpr uint32_t REF_NONE = 0xffffffffu;    // list entry has no side values: gather from the residuals, zero them
 constexpr uint32_t REF_LAZY = 0xfffffffeu;    // the same, but leave the zeroing to the next streaming pass
 
@@ -171,6 +174,11 @@ struct Plan {
   std::vector<Chunk> chunks;
   std::vector<uint32_t> small_layers;  // layer ids on the one-CTA path
   std::vector<uint32_t> large_layers;  // layer ids on the tiled path
+  // tiled layers by how the single-read path selects: one CTA per (layer, worker) pair, or the chain of
+  // histogram / digit / compaction launches over chunks
+  std::vector<uint32_t> pair_layers;   // layer ids
+  std::vector<uint32_t> chain_large;   // indices among the tiled layers
+  std::vector<uint32_t> chain_chunks;  // chunk ids
   uint64_t N = 0, K = 0;
   uint32_t max_small_n = 0;
   int32_t W = 0;
@@ -238,6 +246,12 @@ inline Plan make_plan(const int64_t* sizes, int32_t n_layers, int32_t W, double 
       }
       d.n_chunks = static_cast<uint32_t>(p.chunks.size()) - d.first_chunk;
       if (small_max != 0) sample_plan(d.n, d.k, &d.sample, &d.rho);
+      if (d.sample != 0 && d.n_tiles <= PAIR_MAX_TILES) {
+        p.pair_layers.push_back(static_cast<uint32_t>(l));
+      } else {
+        p.chain_large.push_back(static_cast<uint32_t>(d.large_index));
+        for (uint32_t q = 0; q < d.n_chunks; ++q) p.chain_chunks.push_back(d.first_chunk + q);
+      }
     }
     p.layers.push_back(d);
     off += d.n;

@@ -1,6 +1,7 @@
 // Steps (c)+(d) of the pruning step: exact radix select over the fp32 importance pattern (histogram passes,
 // digit decisions), ordered compaction into the (index, value) lists, and the one-CTA path of small layers.
 #pragma once
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -75,11 +76,14 @@ __global__ void __launch_bounds__(THREADS)
            const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt,
            const uint2* __restrict__ state,
            uint32_t* __restrict__ hist, uint32_t* __restrict__ chunk_sfx, uint2* __restrict__ chunk_cnt,
-           uint32_t* __restrict__ reach_seen, float eps, uint64_t N, int W, int pass, uint32_t n_chunks, WorkerSel ws) {
+           uint32_t* __restrict__ reach_seen, float eps, uint64_t N, int W, int pass, uint32_t n_chunks, WorkerSel ws,
+           const uint32_t* __restrict__ chunk_ids) {
   __shared__ uint32_t sh[NBINS];
   __shared__ uint32_t sh_warp[WARPS];
   __shared__ uint32_t sh_above;
-  const Chunk c = chunks[blockIdx.x];
+  // the chunks this launch covers: all of them, or (chunk_ids) those of the layers the chain selects
+  const uint32_t ci = chunk_ids != nullptr ? chunk_ids[blockIdx.x] : blockIdx.x;
+  const Chunk c = chunks[ci];
   const int w = sel_worker(ws, static_cast<int>(blockIdx.y));
   const LayerDesc L = layers[c.layer];
   const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
@@ -168,9 +172,9 @@ __global__ void __launch_bounds__(THREADS)
     const uint32_t before = block_excl_scan(h0 + h1 + h2 + h3, sh_warp, total);
     const uint32_t s0 = total - before;
     uint4 sfx = make_uint4(s0, s0 - h0, s0 - h0 - h1, s0 - h0 - h1 - h2);
-    uint32_t* dst = chunk_sfx + (static_cast<uint64_t>(w) * n_chunks + blockIdx.x) * pass_bins(N_PASSES - 1);
+    uint32_t* dst = chunk_sfx + (static_cast<uint64_t>(w) * n_chunks + ci) * pass_bins(N_PASSES - 1);
     reinterpret_cast<uint4*>(dst)[threadIdx.x] = sfx;
-    if (threadIdx.x == 0) chunk_cnt[static_cast<uint64_t>(w) * n_chunks + blockIdx.x] = make_uint2(sh_above, 0u);
+    if (threadIdx.x == 0) chunk_cnt[static_cast<uint64_t>(w) * n_chunks + ci] = make_uint2(sh_above, 0u);
   }
 }
 
@@ -180,11 +184,14 @@ __global__ void __launch_bounds__(THREADS)
 __global__ void __launch_bounds__(THREADS)
     k_find_digit(uint2* __restrict__ state, uint32_t* __restrict__ hist, const LayerDesc* __restrict__ layers,
                  const uint32_t* __restrict__ large_ids, const PairInfo* __restrict__ info,
-                 uint32_t* __restrict__ reach_seen, int* __restrict__ status, int W, int pass, WorkerSel ws) {
+                 uint32_t* __restrict__ reach_seen, int* __restrict__ status, int W, int pass, WorkerSel ws,
+                 const uint32_t* __restrict__ large_sel) {
   __shared__ uint32_t sh[NBINS];
   __shared__ uint32_t sh_scan[THREADS];
   __shared__ uint32_t res[4];
-  const uint32_t pair = blockIdx.x * static_cast<uint32_t>(W) + static_cast<uint32_t>(sel_worker(ws, static_cast<int>(blockIdx.y)));
+  // the tiled layers this launch covers: all of them, or (large_sel) those the chain selects
+  const uint32_t li = large_sel != nullptr ? large_sel[blockIdx.x] : blockIdx.x;
+  const uint32_t pair = li * static_cast<uint32_t>(W) + static_cast<uint32_t>(sel_worker(ws, static_cast<int>(blockIdx.y)));
   const int nb = pass_bins(pass), shift = pass_shift(pass);
   uint32_t* gh = hist + static_cast<uint64_t>(pair) * NBINS;
   for (int b = threadIdx.x; b < nb; b += THREADS) {
@@ -295,10 +302,11 @@ __global__ void __launch_bounds__(THREADS)
             const uint2* __restrict__ state, const uint2* __restrict__ chunk_cnt, uint32_t* __restrict__ sel_idx,
             float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot, const uint32_t* __restrict__ chunk_sfx,
             int* __restrict__ status, float eps, uint64_t N, uint64_t K, int W, uint32_t n_chunks, int leader,
-            WorkerSel ws, const int32_t* __restrict__ layer_leader) {
+            WorkerSel ws, const int32_t* __restrict__ layer_leader, const uint32_t* __restrict__ chunk_ids) {
   __shared__ uint32_t sh_warp[WARPS];
   __shared__ uint32_t sh_base[2];
-  const Chunk c = chunks[blockIdx.x];
+  const uint32_t ci = chunk_ids != nullptr ? chunk_ids[blockIdx.x] : blockIdx.x;
+  const Chunk c = chunks[ci];
   const int w = sel_worker(ws, static_cast<int>(blockIdx.y));
   const LayerDesc L = layers[c.layer];
   const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
@@ -310,7 +318,7 @@ __global__ void __launch_bounds__(THREADS)
   {
     const uint2* cc = chunk_cnt + static_cast<uint64_t>(w) * n_chunks;
     uint32_t g = 0, q = 0;
-    for (uint32_t j = c.first_chunk_of_layer + threadIdx.x; j < blockIdx.x; j += THREADS) {
+    for (uint32_t j = c.first_chunk_of_layer + threadIdx.x; j < ci; j += THREADS) {
       const uint2 v = cc[j];
       if (chunk_sfx == nullptr) {  // (#keys > T, #keys == T) of the chunk, counted by a kernel of its own
         g += v.x;
@@ -552,6 +560,404 @@ __global__ void __launch_bounds__(THREADS)
     }
     run_gt += total & 0xffffu;
     run_eq += total >> 16;
+  }
+}
+
+}  // namespace iwp
+
+namespace iwp {
+
+// ---------------------------------------------------------------------------------------
+// single-read path, steps (c)+(d) in ONE launch for layers of at most PAIR_MAX_TILES tiles: a thread-block
+// CLUSTER of PAIR_CLUSTER CTAs per (layer, worker) pair.  Each CTA takes a contiguous share of the pair's tiles,
+// copies their candidate keys into shared memory, and the cluster runs the three digit passes of the exact radix
+// select on them - local shared-memory histograms, merged through distributed shared memory - and writes the
+// ordered list, every CTA its own part at an offset taken from the other CTAs' counts.  It replaces seven
+// dependent launches (three histogram passes with their digit decisions, then the compaction) whose CTAs mostly
+// wait on each other.  CTAs of a cluster meet only at cluster.sync(), a hardware barrier: nothing spins.
+// A pair whose guess failed (fewer than k elements reached it, or a slot overflowed) is selected by the same
+// cluster from the residuals and weights themselves: exact, slower, and rare.
+// grid = (pair layers * PAIR_CLUSTER, covered workers); THREADS threads; dynamic shared memory =
+// 4 * PAIR_KEYS_SMEM bytes.
+// ---------------------------------------------------------------------------------------
+constexpr int PAIR_CLUSTER = 8;
+constexpr uint32_t PAIR_KEYS_SMEM = 16384;  // candidate keys a CTA keeps in shared memory (the rest is re-read)
+constexpr uint32_t PAIR_CTA_TILES = (PAIR_MAX_TILES + PAIR_CLUSTER - 1) / PAIR_CLUSTER;
+
+// Merges the CTAs' local histograms and leaves the sum in every CTA's `hist`.  CTA r adds up bins
+// [r * THREADS, (r + 1) * THREADS) of all CTAs into CTA 0's `merged`; after the barrier everybody copies it.
+// Contains two cluster barriers and one block barrier.
+__device__ __forceinline__ void cluster_merge_hist(cooperative_groups::cluster_group& cluster, uint32_t* hist,
+                                                   uint32_t* merged, int nb) {
+  static_assert(NBINS == PAIR_CLUSTER * THREADS, "one bin per thread and CTA of the cluster");
+  const unsigned cr = cluster.block_rank();
+  cluster.sync();  // every local histogram is complete
+  const int b = static_cast<int>(cr) * THREADS + static_cast<int>(threadIdx.x);
+  if (b < nb) {
+    uint32_t sum = 0;
+#pragma unroll
+    for (int q = 0; q < PAIR_CLUSTER; ++q) sum += cluster.map_shared_rank(hist, q)[b];
+    cluster.map_shared_rank(merged, 0)[b] = sum;
+  }
+  cluster.sync();  // the merged histogram is complete, nobody reads a local one any more
+  const uint32_t* src = cluster.map_shared_rank(merged, 0);
+  for (int q = threadIdx.x; q < nb; q += THREADS) hist[q] = src[q];
+  __syncthreads();
+}
+
+template <bool VEC>
+__global__ void __cluster_dims__(PAIR_CLUSTER, 1, 1) __launch_bounds__(THREADS)
+    k_select_pair(const float* __restrict__ acc, const float* __restrict__ weights, const Tile* __restrict__ tiles,
+                  const LayerDesc* __restrict__ layers, const uint32_t* __restrict__ pair_layer_ids,
+                  const PairInfo* __restrict__ info, const uint32_t* __restrict__ cand_key,
+                  const float* __restrict__ cand_val, const uint16_t* __restrict__ cand_idx,
+                  const uint32_t* __restrict__ cand_cnt, uint2* __restrict__ state, uint32_t* __restrict__ sel_idx,
+                  float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot, int* __restrict__ status, float eps,
+                  uint64_t N, uint64_t K, int W, int leader, WorkerSel ws, const int32_t* __restrict__ layer_leader) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  const unsigned cr = cluster.block_rank();
+  extern __shared__ uint32_t keys[];  // this CTA's first PAIR_KEYS_SMEM candidate keys, in slot order
+  __shared__ uint32_t hist[NBINS];
+  __shared__ uint32_t merged[NBINS];                // CTA 0's copy is the cluster's
+  __shared__ uint32_t x_cnt[PAIR_CLUSTER][2];       // CTA 0's copy: every CTA's (#keys > T, #keys == T)
+  __shared__ uint32_t x_reach;                      // CTA 0's copy: stored entries that reach the guess
+  __shared__ uint32_t sh_scan[WARPS];
+  __shared__ uint32_t res[4];
+  __shared__ uint32_t tile_off[PAIR_CTA_TILES + 1];  // exclusive prefix of this CTA's tiles' stored candidate counts
+  __shared__ uint32_t sh_wg[WARPS], sh_we[WARPS];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t layer_id = pair_layer_ids[blockIdx.x / PAIR_CLUSTER];
+  const LayerDesc L = layers[layer_id];
+  const int w = sel_worker(ws, static_cast<int>(blockIdx.y));
+  const uint32_t pair = static_cast<uint32_t>(L.large_index) * W + w;
+  const PairInfo pi = info[pair];
+  const bool is_leader = w == (layer_leader != nullptr ? layer_leader[layer_id] : leader);
+  const bool cand = pair_is_cand(pi, L.k);
+  uint32_t* out_i = sel_idx + static_cast<uint64_t>(w) * K + L.koff;
+  float* out_v = sel_val + static_cast<uint64_t>(w) * K + L.koff;
+  if (tid == 0) x_reach = 0;
+  cluster.sync();  // every CTA of the cluster runs and has cleared what others add to
+
+  // this CTA's share: tiles [t0, t1) of the pair, or (guess failed) elements [lo, hi) of the layer
+  const uint32_t per = (L.n_tiles + PAIR_CLUSTER - 1) / PAIR_CLUSTER;
+  const uint32_t t0 = min(L.n_tiles, cr * per), t1 = min(L.n_tiles, t0 + per), nt = t1 - t0;
+  const uint64_t share = ((static_cast<uint64_t>(L.n) + PAIR_CLUSTER - 1) / PAIR_CLUSTER + 3) & ~3ull;
+  const uint64_t lo = min(static_cast<uint64_t>(L.off) + L.n, L.off + cr * share), hi = min(static_cast<uint64_t>(L.off) + L.n, lo + share);
+  const uint64_t s0 = lo & ~3ull;
+  const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+  const float* a = acc + static_cast<uint64_t>(w) * N;
+  auto slot_of = [&](uint32_t t) { return (static_cast<uint64_t>(L.first_tile + t0 + t) * W + w) * CAND_CAP; };
+  uint32_t total = 0;  // stored candidates of this CTA's tiles
+
+  if (cand) {
+    for (uint32_t t = tid; t < nt; t += THREADS)
+      tile_off[t + 1] = min(cand_cnt[static_cast<uint64_t>(L.first_tile + t0 + t) * W + w], CAND_CAP);
+    if (tid == 0) tile_off[0] = 0;
+    __syncthreads();
+    if (warp == 0) {  // inclusive scan in place, 32 tiles at a time
+      uint32_t run = 0;
+      for (uint32_t b = 0; b < nt; b += 32) {
+        const uint32_t t = b + lane;
+        const uint32_t v = t < nt ? tile_off[t + 1] : 0u;
+        const uint32_t incl = warp_incl_scan(v);
+        if (t < nt) tile_off[t + 1] = run + incl;
+        run += __shfl_sync(0xffffffffu, incl, 31);
+      }
+    }
+    __syncthreads();
+    total = tile_off[nt];
+    // keys into shared memory, four tiles per warp and trip with all loads issued first
+    for (uint32_t tb = warp * 4; tb < nt; tb += WARPS * 4) {
+      uint4 k4[4];
+      uint32_t cnt[4], p0[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint32_t t = tb + q;
+        p0[q] = t < nt ? tile_off[t] : 0u;
+        cnt[q] = t < nt ? tile_off[t + 1] - p0[q] : 0u;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q)  // slots are zero-padded to groups of four entries
+        k4[q] = (static_cast<uint32_t>(lane) * 4 < cnt[q]) ? reinterpret_cast<const uint4*>(cand_key + slot_of(tb + q))[lane]
+                                                           : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint32_t kk[4] = {k4[q].x, k4[q].y, k4[q].z, k4[q].w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const uint32_t j = lane * 4 + u;
+          if (j < cnt[q] && p0[q] + j < PAIR_KEYS_SMEM) keys[p0[q] + j] = kk[u];
+        }
+        for (uint32_t j = 128 + lane; j < cnt[q]; j += 32)  // the rare slot with more than 128 entries
+          if (p0[q] + j < PAIR_KEYS_SMEM) keys[p0[q] + j] = cand_key[slot_of(tb + q) + j];
+      }
+    }
+    __syncthreads();
+  }
+  // f(key) over this CTA's keys: the cached ones flat out of shared memory, the rest (a CTA whose tiles hold more
+  // than PAIR_KEYS_SMEM candidates) tile by tile through the L2; or, guess failed, over its share of the layer
+  auto for_each_key = [&](auto&& f) {
+    if (cand) {
+      const uint32_t cached = min(total, PAIR_KEYS_SMEM);
+      for (uint32_t p = tid; p < cached; p += THREADS) f(keys[p]);
+      if (total > PAIR_KEYS_SMEM) {
+        for (uint32_t t = warp; t < nt; t += WARPS) {
+          if (tile_off[t + 1] <= PAIR_KEYS_SMEM) continue;
+          const uint32_t first = tile_off[t] >= PAIR_KEYS_SMEM ? 0u : PAIR_KEYS_SMEM - tile_off[t];
+          const uint32_t cnt = tile_off[t + 1] - tile_off[t];
+          for (uint32_t j = first + lane; j < cnt; j += 32) f(cand_key[slot_of(t) + j]);
+        }
+      }
+    } else {
+      for (uint32_t it = 0; it < n_iter; ++it) {
+        const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + tid) * 4;
+        float av[4], wv[4];
+        load4<VEC>(a, e0, lo, hi, av);
+        load4<VEC>(weights, e0, lo, hi, wv);
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          if (e0 + q >= lo && e0 + q < hi) f(imp_key(av[q], wv[q], eps));
+      }
+    }
+  };
+
+  // three digit passes
+  uint32_t prefix = 0, krem = L.k;
+#pragma unroll 1
+  for (int pass = 0; pass < N_PASSES; ++pass) {
+    const int shift = pass_shift(pass), nb = pass_bins(pass);
+    const int prev_shift = pass == 0 ? 31 : pass_shift(pass - 1);
+    const uint32_t want = prefix >> prev_shift;
+    for (int b = tid; b < NBINS; b += THREADS) hist[b] = 0;
+    __syncthreads();
+    uint32_t ge = 0;
+    for_each_key([&](uint32_t key) {
+      if ((key >> prev_shift) == want) atomicAdd(&hist[(key >> shift) & (nb - 1)], 1u);  // pass 0: bit 31 is 0 == want
+      ge += key >= pi.guess ? 1u : 0u;
+    });
+    if (pass == 0 && cand) {  // the stored entries that reach the guess, re-counted (conservation check)
+      ge = __reduce_add_sync(0xffffffffu, ge);
+      if (lane == 0 && ge) atomicAdd(cluster.map_shared_rank(&x_reach, 0), ge);
+    }
+    __syncthreads();
+    cluster_merge_hist(cluster, hist, merged, nb);
+    if (pass == 0 && cand && cr == 0 && tid == 0 && x_reach != pi.total) atomicMin(status, STATUS_INTERNAL);
+    find_digit(hist, nb, krem, sh_scan, res);
+    const bool found = res[2] != 0;
+    const uint32_t d = res[0], kr = res[1];
+    __syncthreads();
+    if (!found) {  // the same in every CTA of the cluster
+      if (cr == 0 && tid == 0) {
+        atomicMin(status, STATUS_INTERNAL);
+        state[pair] = make_uint2(0xffffffffu, 0u);
+      }
+      cluster.sync();  // nobody leaves while its shared memory may still be read
+      return;
+    }
+    prefix |= d << shift;
+    krem = kr;
+  }
+  const uint32_t T = prefix, r = krem;
+  if (cr == 0 && tid == 0) state[pair] = make_uint2(T, r);
+
+  // list offset of this CTA's part: the counts of the CTAs in front of it
+  {
+    uint32_t gt = 0, eq = 0;
+    for_each_key([&](uint32_t key) {
+      gt += key > T ? 1u : 0u;
+      eq += key == T ? 1u : 0u;
+    });
+    gt = __reduce_add_sync(0xffffffffu, gt);
+    eq = __reduce_add_sync(0xffffffffu, eq);
+    if (lane == 0) {
+      sh_wg[warp] = gt;
+      sh_we[warp] = eq;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      uint32_t g = 0, e = 0;
+      for (int q = 0; q < WARPS; ++q) {
+        g += sh_wg[q];
+        e += sh_we[q];
+      }
+      uint32_t* dst = cluster.map_shared_rank(&x_cnt[0][0], 0);
+      dst[2 * cr] = g;
+      dst[2 * cr + 1] = e;
+    }
+  }
+  cluster.sync();
+  uint32_t run_gt = 0, run_eq = 0;
+  {
+    const uint32_t* src = cluster.map_shared_rank(&x_cnt[0][0], 0);
+    for (unsigned q = 0; q < cr; ++q) {
+      run_gt += src[2 * q];
+      run_eq += src[2 * q + 1];
+    }
+  }
+  cluster.sync();  // the last remote read is done: from here on every CTA is on its own
+
+  if (!cand) {  // ordered compaction of this CTA's share of the layer
+    for (uint32_t it = 0; it < n_iter; ++it) {
+      const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + tid) * 4;
+      float av[4], wv[4];
+      load4<VEC>(a, e0, lo, hi, av);
+      load4<VEC>(weights, e0, lo, hi, wv);
+      uint32_t fg = 0, fe = 0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint64_t e = e0 + q;
+        const bool in = e >= lo && e < hi;
+        const uint32_t key = imp_key(av[q], wv[q], eps);
+        fg |= (in && key > T) ? (1u << q) : 0u;
+        fe |= (in && key == T) ? (1u << q) : 0u;
+      }
+      uint32_t tot;
+      const uint32_t packed = static_cast<uint32_t>(__popc(fg)) | (static_cast<uint32_t>(__popc(fe)) << 16);
+      const uint32_t ex = block_excl_scan(packed, sh_scan, tot);
+      uint32_t g_before = run_gt + (ex & 0xffffu), q_before = run_eq + (ex >> 16);
+      if (fg | fe) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const bool isg = (fg >> q) & 1u, ise = (fe >> q) & 1u;
+          if (isg || (ise && q_before < r)) {
+            const uint32_t pos = g_before + (q_before < r ? q_before : r);
+            if (pos < L.k) {
+              out_i[pos] = static_cast<uint32_t>(e0 + q);
+              out_v[pos] = av[q];
+              if (is_leader) sel_slot[L.koff + pos] = REF_LAZY;
+            } else {
+              atomicMin(status, STATUS_INTERNAL);
+            }
+          }
+          g_before += isg ? 1u : 0u;
+          q_before += ise ? 1u : 0u;
+        }
+      }
+      run_gt += tot & 0xffffu;
+      run_eq += tot >> 16;
+    }
+    return;
+  }
+
+  // ordered compaction from the slots: batches of WARPS * 4 consecutive tiles, warp q the q-th group of four, so
+  // that warp order is index order.  Each lane takes four consecutive entries of a slot; keys, values and offsets
+  // of the warp's four tiles are all requested before any is used; ranks come from one warp scan per 128 entries.
+  for (uint32_t tb0 = 0; tb0 < nt; tb0 += WARPS * 4) {
+    const uint32_t t_begin = min(nt, tb0 + warp * 4), t_end = min(nt, t_begin + 4);
+    uint32_t cnt[4];
+    uint4 k4[4];
+    float4 v4[4];
+    uint2 i2[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) cnt[q] = (t_begin + q < t_end) ? tile_off[t_begin + q + 1] - tile_off[t_begin + q] : 0u;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {  // slots are zero-padded to groups of four entries; entries past the count are masked
+      const bool has = static_cast<uint32_t>(lane) * 4 < cnt[q];
+      const uint64_t slot = slot_of(t_begin + q);
+      k4[q] = has ? reinterpret_cast<const uint4*>(cand_key + slot)[lane] : make_uint4(0u, 0u, 0u, 0u);
+      v4[q] = has ? reinterpret_cast<const float4*>(cand_val + slot)[lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+      i2[q] = has ? reinterpret_cast<const uint2*>(cand_idx + slot)[lane] : make_uint2(0u, 0u);
+    }
+    // flags of a lane's four entries of one group of 128
+    auto flags = [&](uint32_t cnt_t, uint32_t j0, uint4 k, uint32_t& fg, uint32_t& fe) {
+      const uint32_t j = j0 + lane * 4;
+      const uint32_t kk[4] = {k.x, k.y, k.z, k.w};
+      fg = fe = 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const bool in = j + u < cnt_t;
+        fg |= (in && kk[u] > T) ? (1u << u) : 0u;
+        fe |= (in && kk[u] == T) ? (1u << u) : 0u;
+      }
+    };
+    auto group = [&](uint32_t t, uint32_t g) {  // group g of 128 entries of tile t, beyond the preloaded first one
+      const uint64_t slot = slot_of(t);
+      return reinterpret_cast<const uint4*>(cand_key + slot)[g * 32 + lane];
+    };
+    uint32_t my_gt = 0, my_eq = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t fg, fe;
+      flags(cnt[q], 0, k4[q], fg, fe);
+      my_gt += __popc(fg);
+      my_eq += __popc(fe);
+      for (uint32_t j0 = 128; j0 < cnt[q]; j0 += 128) {  // the rare slot with more than 128 entries
+        flags(cnt[q], j0, (j0 + lane * 4 < cnt[q]) ? group(t_begin + q, j0 >> 7) : make_uint4(0u, 0u, 0u, 0u), fg, fe);
+        my_gt += __popc(fg);
+        my_eq += __popc(fe);
+      }
+    }
+    my_gt = __reduce_add_sync(0xffffffffu, my_gt);
+    my_eq = __reduce_add_sync(0xffffffffu, my_eq);
+    __syncthreads();  // the previous batch has read the per-warp counts
+    if (lane == 0) {
+      sh_wg[warp] = my_gt;
+      sh_we[warp] = my_eq;
+    }
+    __syncthreads();
+    uint32_t g_before = run_gt, q_before = run_eq, tot_g = 0, tot_e = 0;
+#pragma unroll
+    for (int q = 0; q < WARPS; ++q) {
+      const uint32_t g = sh_wg[q], e = sh_we[q];
+      if (q < warp) {
+        g_before += g;
+        q_before += e;
+      }
+      tot_g += g;
+      tot_e += e;
+    }
+    run_gt += tot_g;
+    run_eq += tot_e;
+    if ((my_gt | my_eq) == 0) continue;  // nothing of this warp's tiles is selected
+    auto emit = [&](uint32_t t, uint32_t cnt_t, uint32_t j0, uint4 k, float4 vals, uint2 offs) {
+      const uint32_t j = j0 + lane * 4;
+      const uint32_t tile = L.first_tile + t0 + t;
+      const uint32_t tile_base = tiles[tile].a & ~(TILE - 1u);
+      uint32_t fg, fe;
+      flags(cnt_t, j0, k, fg, fe);
+      const uint32_t packed = static_cast<uint32_t>(__popc(fg)) | (static_cast<uint32_t>(__popc(fe)) << 16);
+      const uint32_t incl = warp_incl_scan(packed);
+      const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
+      uint32_t gb = g_before + ((incl - packed) & 0xffffu), qb = q_before + ((incl - packed) >> 16);
+      if (fg | fe) {
+        const float vv[4] = {vals.x, vals.y, vals.z, vals.w};
+        const uint32_t ii[4] = {offs.x & 0xffffu, offs.x >> 16, offs.y & 0xffffu, offs.y >> 16};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const bool isg = (fg >> u) & 1u, ise = (fe >> u) & 1u;
+          if (isg || (ise && qb < r)) {
+            const uint32_t pos = gb + (qb < r ? qb : r);
+            IWP_DBG_CHECK(status, tile_base + ii[u] >= L.off && tile_base + ii[u] - L.off < L.n);
+            if (pos < L.k) {
+              out_i[pos] = tile_base + ii[u];
+              out_v[pos] = vv[u];
+              if (is_leader) sel_slot[L.koff + pos] = tile * CAND_CAP + j + u;
+            } else {
+              atomicMin(status, STATUS_INTERNAL);
+            }
+          }
+          gb += isg ? 1u : 0u;
+          qb += ise ? 1u : 0u;
+        }
+      }
+      g_before += tot & 0xffffu;
+      q_before += tot >> 16;
+    };
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (cnt[q] == 0) continue;
+      const uint32_t t = t_begin + q;
+      emit(t, cnt[q], 0, k4[q], v4[q], i2[q]);
+      for (uint32_t j0 = 128; j0 < cnt[q]; j0 += 128) {
+        const bool has = j0 + lane * 4 < cnt[q];
+        const uint64_t slot = slot_of(t);
+        const uint32_t g = (j0 >> 2) + lane;
+        emit(t, cnt[q], j0, has ? reinterpret_cast<const uint4*>(cand_key + slot)[g] : make_uint4(0u, 0u, 0u, 0u),
+             has ? reinterpret_cast<const float4*>(cand_val + slot)[g] : make_float4(0.f, 0.f, 0.f, 0.f),
+             has ? reinterpret_cast<const uint2*>(cand_idx + slot)[g] : make_uint2(0u, 0u));
+      }
+    }
   }
 }
 

@@ -34,12 +34,15 @@ def _dense_weights(N, seed, scale=0.05):
 
 
 def _run_checked(sizes, W, ratio, weights, grads_fn, steps, overlap, leaders=None, expect_single_read=True, seed=7,
-                 state_every=1, residual_every=1):
+                 state_every=1, residual_every=1, pair_select=None):
     """run_parity plus the proof that the case stayed on the single-read path (no pair fell back)."""
     pr = Pruner(sizes, W, ratio, 1e-8, seed)
     orc = oracle.Oracle(sizes, W, ratio, 1e-8, seed)
     pr.set_option("overlap", overlap)
     pr.set_option("speculate", 1)
+    # the two ways the single-read path selects from the candidate slots: the chain of launches (0) and the
+    # one-launch cluster kernel (1); by default the one the overlap parameter does not pick is used too
+    pr.set_option("pair_select", overlap if pair_select is None else pair_select)
     w_host = weights.cpu().numpy()
     update = torch.full((pr.N,), float("nan"), device=DEV)
     failed = 0

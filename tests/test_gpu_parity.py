@@ -150,6 +150,28 @@ def test_forced_scalar_path_and_leader_override():
                leader_overrides=[3, 0, 2, 2])
 
 
+@pytest.mark.parametrize("overlap", [0, 1])
+def test_select_chain_for_every_layer(overlap):
+    # the one-launch select per (layer, worker) pair switched off: every tiled layer goes through the chain
+    sizes, W, ratio = [300000, 128, 70000, 16385], 4, 64.0
+    N = sum(sizes)
+    weights = _weights(N, 13)
+    run_parity(sizes, W, ratio, 1e-8, seed=0, steps=3, weights=weights,
+               grads_fn=lambda t: _randn((W, N), 17 * t + 2, 1e-2), options={"pair_select": 0, "overlap": overlap})
+
+
+def test_pair_select_next_to_the_chain_and_beyond_its_key_cache():
+    # one layer above the limit of the one-launch select (641 tiles: chain), one of 600 tiles whose candidates
+    # exceed what the kernel keeps in shared memory (the rest is re-read), and small ones
+    sizes, W, ratio = [641 * 4096 - 100, 600 * 4096, 20000, 64], 3, 32.0
+    N = sum(sizes)
+    weights = _weights(N, 15, zero_frac=0.0)
+    for overlap in (0, 1):
+        run_parity(sizes, W, ratio, 1e-8, seed=2, steps=3, weights=weights,
+                   grads_fn=lambda t: _randn((W, N), 19 * t + 5, 1e-2), options={"overlap": overlap, "pair_select": 1},
+                   residual_every=3)
+
+
 def test_exact_select_without_speculation():
     sizes, W, ratio = [300000, 128, 70000], 4, 64.0
     N = sum(sizes)
@@ -451,6 +473,8 @@ def test_random_option_changes_between_steps(seed):
                 assert_bits_equal(pr.residual(w).cpu().numpy(), orc.residual(w), f"before step {t}: worker {w} residual")
         elif what == 6:
             pr.set_option("time_stages", int(rng.integers(0, 3)))
+        elif what == 7:
+            pr.set_option("pair_select", int(rng.integers(-1, 2)))
         coarse = rng.random() < 0.3  # ties and fallbacks now and then
         if coarse:
             g = torch.randint(-4, 5, (W, N), device=DEV, generator=torch.Generator(device=DEV).manual_seed(t)).float() / 8.0
@@ -492,6 +516,7 @@ def test_random_shapes(seed):
             return torch.randint(-4, 5, (W, N), device=DEV, generator=torch.Generator(device=DEV).manual_seed(seed * 100 + t)).float() / 8.0
         return _randn((W, N), 7000 + seed * 100 + t, 1e-2)
     run_parity(sizes, W, ratio, 1e-8, seed=seed, steps=4, weights=weights, grads_fn=grads,
-               options={"overlap": int(rng.integers(0, 2)), "speculate": int(rng.random() < 0.8)},
+               options={"overlap": int(rng.integers(0, 2)), "speculate": int(rng.random() < 0.8),
+                        "pair_select": int(rng.random() < 0.7)},
                n_leaders=int(rng.integers(1, min(W, 3) + 1)), momentum=float(rng.choice([1.0, 0.9])),
                state_every=int(rng.choice([1, 2])), residual_every=int(rng.choice([1, 1000])))
