@@ -525,11 +525,32 @@ __global__ void __launch_bounds__(THREADS)
   float* a = acc + static_cast<uint64_t>(w) * N + L.off;
   const float* g = grads + static_cast<uint64_t>(w) * N + L.off;
   const float* wt = weights + L.off;
-  for (uint32_t i = tid; i < n; i += THREADS) {
-    const float v = accumulate(a[i], __ldcs(g + i), momentum);
-    a[i] = v;
-    keys[i] = imp_key(v, wt[i], eps);
-    if (w == 0) update[L.off + i] = 0.0f;
+  // step (a)+(b): four elements per thread and trip, all loads issued before any is used (one CTA walks the
+  // whole layer, so memory-level parallelism has to come from here)
+  constexpr int U = 4;
+  for (uint32_t i0 = 0; i0 < n; i0 += THREADS * U) {
+    float av[U], gv[U], wv[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const uint32_t i = i0 + u * THREADS + tid;
+      av[u] = gv[u] = 0.f;
+      wv[u] = 1.f;
+      if (i < n) {
+        av[u] = a[i];
+        gv[u] = __ldcs(g + i);
+        wv[u] = wt[i];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const uint32_t i = i0 + u * THREADS + tid;
+      if (i < n) {
+        const float v = accumulate(av[u], gv[u], momentum);
+        a[i] = v;
+        keys[i] = imp_key(v, wv[u], eps);
+        if (w == 0) update[L.off + i] = 0.0f;
+      }
+    }
   }
   if (only_worker >= 0 && w != only_worker) return;  // only the chosen node selects: steps (a), (b) were this worker's part
   __syncthreads();
@@ -540,16 +561,40 @@ __global__ void __launch_bounds__(THREADS)
   }
   uint32_t* out_i = sel_idx + static_cast<uint64_t>(w) * K + L.koff;
   float* out_v = sel_val + static_cast<uint64_t>(w) * K + L.koff;
-  uint32_t run_gt = 0, run_eq = 0;
-  for (uint32_t i0 = 0; i0 < n; i0 += THREADS) {
-    const uint32_t i = i0 + tid;
-    const uint32_t key = i < n ? keys[i] : 0u;
-    const bool isg = i < n && key > T, ise = i < n && key == T;
-    uint32_t total;
-    const uint32_t ex = block_excl_scan((isg ? 1u : 0u) | (ise ? 1u << 16 : 0u), sh_warp, total);
-    const uint32_t g_before = run_gt + (ex & 0xffffu), q_before = run_eq + (ex >> 16);
-    if (isg || (ise && q_before < r)) {
-      const uint32_t pos = g_before + (q_before < r ? q_before : r);
+  // ordered compaction: warp q owns the q-th contiguous stretch of the layer (a multiple of 32 elements), counts
+  // its keys above / at the threshold, and after one prefix over the warps ranks them 32 at a time by ballots
+  const int lane = tid & 31, warp = tid >> 5;
+  const uint32_t per_warp = (((n + WARPS - 1) / WARPS) + 31u) & ~31u;
+  const uint32_t wb = min(n, warp * per_warp), we = min(n, wb + per_warp);
+  uint32_t my_gt = 0, my_eq = 0;
+  for (uint32_t i = wb + lane; i < we; i += 32) {
+    const uint32_t key = keys[i];
+    my_gt += key > T ? 1u : 0u;
+    my_eq += key == T ? 1u : 0u;
+  }
+  my_gt = __reduce_add_sync(0xffffffffu, my_gt);
+  my_eq = __reduce_add_sync(0xffffffffu, my_eq);
+  __shared__ uint32_t sh_we[WARPS];
+  if (lane == 0) {
+    sh_warp[warp] = my_gt;
+    sh_we[warp] = my_eq;
+  }
+  __syncthreads();
+  uint32_t g_before = 0, q_before = 0;
+  for (int q = 0; q < warp; ++q) {
+    g_before += sh_warp[q];
+    q_before += sh_we[q];
+  }
+  if ((my_gt | my_eq) == 0) return;
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  for (uint32_t i0 = wb; i0 < we; i0 += 32) {
+    const uint32_t i = i0 + lane;
+    const uint32_t key = i < we ? keys[i] : 0u;
+    const bool isg = i < we && key > T, ise = i < we && key == T;
+    const uint32_t bg = __ballot_sync(0xffffffffu, isg), be = __ballot_sync(0xffffffffu, ise);
+    const uint32_t gb = g_before + __popc(bg & lt_mask), qb = q_before + __popc(be & lt_mask);
+    if (isg || (ise && qb < r)) {
+      const uint32_t pos = gb + (qb < r ? qb : r);
       if (pos < L.k) {
         out_i[pos] = L.off + i;
         out_v[pos] = a[i];
@@ -558,8 +603,8 @@ __global__ void __launch_bounds__(THREADS)
         atomicMin(status, STATUS_INTERNAL);
       }
     }
-    run_gt += total & 0xffffu;
-    run_eq += total >> 16;
+    g_before += __popc(bg);
+    q_before += __popc(be);
   }
 }
 
