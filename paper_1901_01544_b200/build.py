@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libiwp.so")
 SOURCES = [os.path.join(CSRC, "iwp_api.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("iwp_device.cuh", "iwp_stream.cuh", "iwp_select.cuh", "iwp_reduce.cuh",
+DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("iwp_device.cuh", "iwp_stream.cuh", "iwp_sample.cuh", "iwp_select.cuh", "iwp_reduce.cuh",
                                             "iwp_threshold.cuh", "iwp_wire.cuh", "iwp_plan.hpp")] + [
     os.path.join(os.path.dirname(HERE), "include", "iwp.h")
 ]

@@ -3,7 +3,8 @@
 //
 // The sm_100a kernels live in the headers included below, by step of the path (Algorithm 1 of the paper):
 //   iwp_device.cuh     shared device helpers (importance arithmetic, vector loads, scans, radix select)
-//   iwp_stream.cuh     (a)+(b): accumulate, threshold guess from a sample, single-read streaming pass
+//   iwp_sample.cuh     threshold guess of the single-read path from a sample of every (layer, worker) pair
+//   iwp_stream.cuh     (a)+(b): accumulate, single-read streaming pass (importance, candidates, side values)
 //   iwp_select.cuh     (c)+(d): exact radix select, ordered compaction, one-CTA path of small layers
 //   iwp_reduce.cuh     (e)-(g): reduction at the index set, zero mask, sharded phases, mask accessor
 //   iwp_threshold.cuh  absolute-threshold mode, random selection, layer-wise threshold
@@ -25,6 +26,7 @@
 #include "iwp_device.cuh"
 #include "iwp_plan.hpp"
 #include "iwp_reduce.cuh"
+#include "iwp_sample.cuh"
 #include "iwp_select.cuh"
 #include "iwp_stream.cuh"
 #include "iwp_threshold.cuh"

@@ -245,6 +245,31 @@ __device__ __forceinline__ bool smem_radix_select(const uint32_t* keys, uint32_t
   return true;
 }
 
+// Lazy zeroing of sent residuals (step (g)): instead of scattering W * K four-byte zeros, the
+// reduction marks each sent element in a bit mask and the NEXT streaming pass, which reads every
+// residual anyway, takes a marked residual as +0.  Layout: one 16-bit field per (512-element
+// segment of the flat element space, lane), bit 4 * round + component - exactly the sixteen
+// elements a lane of the streaming pass owns - two fields per 32-bit word.
+__device__ __forceinline__ uint64_t zmask_word(uint64_t i) { return ((i >> 9) * 32 + ((i & 127) >> 2)) >> 1; }
+__device__ __forceinline__ uint32_t zmask_bit(uint64_t i) {
+  return 1u << ((((i & 127) >> 2) & 1) * 16 + ((i >> 7) & 3) * 4 + (i & 3));
+}
+__device__ __forceinline__ bool zmask_test(const uint32_t* __restrict__ zmask, uint64_t i) {
+  return (zmask[zmask_word(i)] & zmask_bit(i)) != 0u;
+}
+
+// Pre-test multiplier of the single-read path: with gm = guess * (1 - 2^-20) every element whose correctly
+// rounded quotient |acc| / den reaches the guess passes |acc| >= gm * den (the two roundings of gm * den and the
+// one of the quotient are each below 2^-23 relative).  The argument needs normal products, so the pre-test is
+// disabled (gm = 0: everything passes) for tiny guesses or eps; +inf = no guess, nothing passes.
+__device__ __forceinline__ float pretest_multiplier(uint32_t guess, float eps) {
+  if (guess == GUESS_NONE) return __int_as_float(0x7f800000);  // +inf: nothing passes
+  const float gf = __uint_as_float(guess);
+  const float tiny = 8.673617379884035e-19f;  // 2^-60
+  if (!(gf >= tiny) || !(eps >= tiny)) return 0.0f;
+  return __fmul_rd(gf, 1.0f - 9.5367431640625e-07f);
+}
+
 // Warp-aggregated increment of a shared-memory histogram: lanes that hit the same bin
 // elect one lane that adds the whole group's count.  Must be called by all 32 lanes.
 __device__ __forceinline__ void hist_add_aggregated(uint32_t* hist, bool valid, uint32_t bin) {
