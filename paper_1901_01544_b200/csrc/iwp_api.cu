@@ -34,6 +34,11 @@
 
 using namespace iwp;
 
+// Warps per CTA of the select kernels of one chain: histogram + digit kernels, compaction kernel.
+struct ChainWidth {
+  int hist, write;
+};
+
 struct iwp_ctx {
   Plan plan;
   float eps = 0.f;
@@ -62,6 +67,13 @@ struct iwp_ctx {
   cudaStream_t side_a = nullptr, side_b = nullptr;
   cudaEvent_t ev_lead = nullptr, ev_lead_done = nullptr, ev_others = nullptr, ev_a2 = nullptr, ev_b = nullptr;
   bool pending_a2 = false, pending_b = false;  // deferred selects of the last step not yet joined
+  // The three select chains of the overlapped schedule.  Histogram and digit kernels with four warps per CTA (64
+  // registers a thread) fit into the registers the streaming pass leaves free on an SM, so they take no CTA slot
+  // from it, but take longer; the chain of the next step's chosen node is waited for by that step's first launch
+  // and keeps eight warps; the compaction always does (with four it takes twice as long and the next step waits).
+  // Measured, ms per step on the AlexNet shape W=8 / the ResNet-50 shape: all eight 1.294 / 0.700; this choice
+  // 1.293 / 0.678; four everywhere in the histogram kernels 1.306 / 0.673.
+  ChainWidth cw_lead{4, 8}, cw_next{8, 8}, cw_rest{4, 8};
   int32_t predicted_next = -1;                 // the worker whose select pending_a2 covers
   int32_t last_only = -1;                      // the last step selected for this worker alone (-1: for every worker)
   float* saved_w = nullptr;                    // [N] weights kept for deferred selects that fall back (k_save_weights)
@@ -148,6 +160,8 @@ struct iwp_ctx {
 };
 
 namespace {
+
+constexpr int WRITE_WARPS = 8;  // warps per CTA of the select kernels in the serial schedule
 
 // stages of a step, in launch order; an event is recorded at every boundary when timing is on
 enum Stage { ST_SMALL = 0, ST_SAMPLE, ST_ACCUMULATE, ST_SELECT, ST_COMPACT, ST_GATHER, N_STAGES };
@@ -391,11 +405,8 @@ int launch_pair_select(iwp_ctx* c, const float* weights, cudaStream_t st, Worker
   return IWP_OK;
 }
 
-// Exact select and ordered compaction of the workers `ws` covers, on stream `st` (single-read path): one
-// launch for the layers selected per pair, the chain (three histogram passes with their digit decisions, then
-// the compaction) for the others.
-template <bool VEC>
-int select_and_write(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSel ws, int32_t leader) {
+template <bool VEC, int HW, int WW>
+int select_and_write_w(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSel ws, int32_t leader) {
   const Plan& p = c->plan;
   const int W = p.W;
   const unsigned n_chunks = static_cast<unsigned>(p.chunks.size());
@@ -410,20 +421,33 @@ int select_and_write(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSe
   dim3 cgrid(sc.n_chunks, n_sel), pgrid(sc.n_large, n_sel);
   uint32_t* sfx = c->chunk_sfx;
   for (int pass = 0; pass < N_PASSES; ++pass) {
-    k_hist<VEC><<<cgrid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_layers, c->info_cur, c->cand_key,
-                                           c->cand_cnt, c->d_state, c->d_hist, sfx, c->d_chunk_cnt, c->d_reach, c->eps, p.N,
-                                           W, pass, n_chunks, ws, sc.chunk_ids);
+    k_hist<VEC, HW><<<cgrid, HW * 32, 0, st>>>(c->acc, weights, c->d_chunks, c->d_layers, c->info_cur, c->cand_key,
+                                               c->cand_cnt, c->d_state, c->d_hist, sfx, c->d_chunk_cnt, c->d_reach, c->eps,
+                                               p.N, W, pass, n_chunks, ws, sc.chunk_ids);
     IWP_LAUNCH_CHECK(c);
-    k_find_digit<<<pgrid, THREADS, 0, st>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->info_cur, c->d_reach,
-                                            c->d_status, W, pass, ws, sc.large_sel);
+    k_find_digit<HW><<<pgrid, HW * 32, 0, st>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->info_cur, c->d_reach,
+                                                c->d_status, W, pass, ws, sc.large_sel);
     IWP_LAUNCH_CHECK(c);
   }
-  k_write<VEC><<<cgrid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur, c->cand_key,
-                                          c->cand_val, c->cand_idx, c->cand_cnt, c->d_state, c->d_chunk_cnt, c->sel_idx,
-                                          c->sel_val, c->sel_slot, sfx, c->d_status, c->eps, p.N, p.K, W, n_chunks,
-                                          leader, ws, nullptr, sc.chunk_ids);
+  k_write<VEC, WW><<<cgrid, WW * 32, 0, st>>>(
+      c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur, c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt,
+      c->d_state, c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, sfx, c->d_status, c->eps, p.N, p.K, W, n_chunks, leader,
+      ws, nullptr, sc.chunk_ids);
   IWP_LAUNCH_CHECK(c);
   return IWP_OK;
+}
+
+// Exact select and ordered compaction of the workers `ws` covers, on stream `st` (single-read path): one
+// launch for the layers selected per pair, the chain (three histogram passes with their digit decisions, then
+// the compaction) for the others.
+template <bool VEC>
+int select_and_write(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSel ws, int32_t leader, ChainWidth cw) {
+  if (cw.hist == 4) {
+    return cw.write == 4 ? select_and_write_w<VEC, 4, 4>(c, weights, st, ws, leader)
+                         : select_and_write_w<VEC, 4, 8>(c, weights, st, ws, leader);
+  }
+  return cw.write == 4 ? select_and_write_w<VEC, 8, 4>(c, weights, st, ws, leader)
+                       : select_and_write_w<VEC, 8, 8>(c, weights, st, ws, leader);
 }
 
 int32_t leader_of_step(const iwp_ctx* c, int64_t t) {
@@ -537,7 +561,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     // the leader's select and list, under the other workers' streaming pass
     if (!cuda_ok(cudaEventRecord(c->ev_lead, s)) || !cuda_ok(cudaStreamWaitEvent(c->side_a, c->ev_lead, 0)))
       return IWP_ERR_CUDA;
-    int rc = select_and_write<VEC>(c, weights, c->side_a, WorkerSel{WorkerSel::ONLY, leader, -1}, leader);
+    int rc = select_and_write<VEC>(c, weights, c->side_a, WorkerSel{WorkerSel::ONLY, leader, -1}, leader, c->cw_lead);
     if (rc != IWP_OK) return rc;
     if (!cuda_ok(cudaEventRecord(c->ev_lead_done, c->side_a))) return IWP_ERR_CUDA;
     if (c->pending_b && !cuda_ok(cudaStreamWaitEvent(s, c->ev_b, 0))) return IWP_ERR_CUDA;
@@ -567,7 +591,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     if (!cuda_ok(cudaEventRecord(c->ev_others, s))) return IWP_ERR_CUDA;
     if (next != leader) {
       if (!cuda_ok(cudaStreamWaitEvent(c->side_a, c->ev_others, 0))) return IWP_ERR_CUDA;
-      rc = select_and_write<VEC>(c, c->saved_w, c->side_a, WorkerSel{WorkerSel::ONLY, next, -1}, leader);
+      rc = select_and_write<VEC>(c, c->saved_w, c->side_a, WorkerSel{WorkerSel::ONLY, next, -1}, leader, c->cw_next);
       if (rc != IWP_OK) return rc;
       if (!cuda_ok(cudaEventRecord(c->ev_a2, c->side_a))) return IWP_ERR_CUDA;
       c->pending_a2 = true;
@@ -575,7 +599,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     const WorkerSel rest{WorkerSel::EXCEPT, leader, next};
     if (sel_count(rest, W) > 0) {
       if (!cuda_ok(cudaStreamWaitEvent(c->side_b, c->ev_others, 0))) return IWP_ERR_CUDA;
-      rc = select_and_write<VEC>(c, c->saved_w, c->side_b, rest, leader);
+      rc = select_and_write<VEC>(c, c->saved_w, c->side_b, rest, leader, c->cw_rest);
       if (rc != IWP_OK) return rc;
       if (!cuda_ok(cudaEventRecord(c->ev_b, c->side_b))) return IWP_ERR_CUDA;
       c->pending_b = true;
@@ -632,11 +656,11 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     }
     dim3 cgrid(sc.n_chunks, n_sel), pgrid(sc.n_large, n_sel);
     for (int pass = 0; pass < N_PASSES && sc.n_chunks > 0; ++pass) {
-      k_hist<VEC><<<cgrid, THREADS, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->info_cur, c->cand_key,
+      k_hist<VEC, WRITE_WARPS><<<cgrid, WRITE_WARPS * 32, 0, s>>>(c->acc, weights, c->d_chunks, c->d_layers, c->info_cur, c->cand_key,
                                             c->cand_cnt, c->d_state, c->d_hist, c->chunk_sfx, c->d_chunk_cnt, c->d_reach,
                                             c->eps, N, W, pass, n_chunks, all, sc.chunk_ids);
       IWP_LAUNCH_CHECK(c);
-      k_find_digit<<<pgrid, THREADS, 0, s>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->info_cur, c->d_reach,
+      k_find_digit<WRITE_WARPS><<<pgrid, WRITE_WARPS * 32, 0, s>>>(c->d_state, c->d_hist, c->d_layers, c->d_large_ids, c->info_cur, c->d_reach,
                                              c->d_status, W, pass, all, sc.large_sel);
       IWP_LAUNCH_CHECK(c);
     }
@@ -648,7 +672,7 @@ int run_step(iwp_ctx* c, const float* grads, const float* weights, float* update
     auto write = [&](cudaStream_t st, WorkerSel ws) {
       if (sc.n_chunks == 0) return;
       dim3 grid(sc.n_chunks, static_cast<unsigned>(sel_count(ws, W)));
-      k_write<VEC><<<grid, THREADS, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur,
+      k_write<VEC, WRITE_WARPS><<<grid, WRITE_WARPS * 32, 0, st>>>(c->acc, weights, c->d_chunks, c->d_tiles, c->d_layers, c->info_cur,
                                              c->cand_key, c->cand_val, c->cand_idx, c->cand_cnt, c->d_state,
                                              c->d_chunk_cnt, c->sel_idx, c->sel_val, c->sel_slot, c->chunk_sfx,
                                              c->d_status, c->eps, N, K, W, n_chunks, leader, ws, lead_tab, sc.chunk_ids);
@@ -1686,17 +1710,17 @@ int run_select_static(StaticScratch* s, const float* residual, const float* weig
   dim3 grid(n_chunks, 1);
   const WorkerSel all{WorkerSel::ALL, 0, -1};
   for (int pass = 0; pass < N_PASSES; ++pass) {
-    k_hist<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr, &s->state,
+    k_hist<VEC, SEL_WARPS><<<grid, SEL_THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr, &s->state,
                                           s->hist, nullptr, nullptr, nullptr, eps, 0, 1, pass, n_chunks, all, nullptr);
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
-    k_find_digit<<<1, THREADS, 0, st>>>(&s->state, s->hist, &s->layer, &s->large_id, &s->info, nullptr, &s->status, 1, pass,
+    k_find_digit<SEL_WARPS><<<1, SEL_THREADS, 0, st>>>(&s->state, s->hist, &s->layer, &s->large_id, &s->info, nullptr, &s->status, 1, pass,
                                         all, nullptr);
     if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
   }
-  k_count<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr, &s->state,
+  k_count<VEC><<<grid, SEL_THREADS, 0, st>>>(residual, weights, s->chunks, &s->layer, &s->info, nullptr, nullptr, &s->state,
                                          s->chunk_cnt, eps, 0, 1, n_chunks);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;
-  k_write<VEC><<<grid, THREADS, 0, st>>>(residual, weights, s->chunks, nullptr, &s->layer, &s->info, nullptr, nullptr,
+  k_write<VEC, SEL_WARPS><<<grid, SEL_THREADS, 0, st>>>(residual, weights, s->chunks, nullptr, &s->layer, &s->info, nullptr, nullptr,
                                          nullptr, nullptr, &s->state, s->chunk_cnt, idx, val, nullptr, nullptr,
                                          &s->status, eps, 0, 0, 1, n_chunks, -1, all, nullptr, nullptr);
   if (cudaGetLastError() != cudaSuccess) return IWP_ERR_CUDA;

@@ -10,20 +10,28 @@
 
 namespace iwp {
 
+// CTA size of the select kernels (histogram passes, digit decisions, compaction).  Four warps of at most 64
+// registers: such a CTA fits into the registers three CTAs of the streaming pass leave free on an SM (7 warps x
+// 80 registers each in the other workers' launch: 53 760 of 65 536), so a select that runs beside the streaming
+// pass takes no CTA slot away from it.
+constexpr int SEL_THREADS = 128;
+constexpr int SEL_WARPS = SEL_THREADS / 32;
+
 // The candidates of (chunk, worker): warp q takes the q-th eighth of the chunk's tiles (consecutive,
 // so that warp order is index order), four tiles at a time; each lane reads entries 4 lane .. 4 lane + 3
 // of a slot with one 128-bit load (a slot rarely holds more than 128 entries; a tail loop covers the
 // rest) and all loads of a batch are issued before any is used.  `f(key)` sees every stored candidate,
 // and in addition some keys 0 (padding, slots shorter than 128 entries), which `f` must ignore - every
 // use below does so by construction, because a candidate's key and first digit are never 0.
-__device__ __forceinline__ uint32_t tiles_per_warp(const Chunk& c) { return (c.n_tiles + WARPS - 1) / WARPS; }
+template <int NW>
+__device__ __forceinline__ uint32_t tiles_per_warp(const Chunk& c) { return (c.n_tiles + NW - 1) / NW; }
 
-template <typename F>
+template <int NW = SEL_WARPS, typename F>
 __device__ __forceinline__ void for_each_candidate(const Chunk& c, int w, int W, const uint32_t* __restrict__ cand_cnt,
                                                    const uint32_t* __restrict__ cand_key, F&& f) {
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t t_begin = min(c.n_tiles, warp * tiles_per_warp(c));
-  const uint32_t t_end = min(c.n_tiles, t_begin + tiles_per_warp(c));
+  const uint32_t t_begin = min(c.n_tiles, warp * tiles_per_warp<NW>(c));
+  const uint32_t t_end = min(c.n_tiles, t_begin + tiles_per_warp<NW>(c));
   for (uint32_t tb = t_begin; tb < t_end; tb += 4) {
     uint32_t cnt[4];
     uint4 k4[4];
@@ -69,8 +77,8 @@ __device__ __forceinline__ void for_each_candidate(const Chunk& c, int w, int W,
 // the number of keys above the prefix and the suffix sums of its low-digit histogram; with the
 // threshold known, the compaction derives every chunk's (#keys > T, #keys == T) from those without
 // another look at the keys (chunk_sfx == nullptr: skipped, a counting kernel runs instead).
-template <bool VEC>
-__global__ void __launch_bounds__(THREADS)
+template <bool VEC, int NW>
+__global__ void __launch_bounds__(NW * 32, 512 / (NW * 32) * 2)
     k_hist(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
            const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
            const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt,
@@ -79,7 +87,7 @@ __global__ void __launch_bounds__(THREADS)
            uint32_t* __restrict__ reach_seen, float eps, uint64_t N, int W, int pass, uint32_t n_chunks, WorkerSel ws,
            const uint32_t* __restrict__ chunk_ids) {
   __shared__ uint32_t sh[NBINS];
-  __shared__ uint32_t sh_warp[WARPS];
+  __shared__ uint32_t sh_warp[NW];
   __shared__ uint32_t sh_above;
   // the chunks this launch covers: all of them, or (chunk_ids) those of the layers the chain selects
   const uint32_t ci = chunk_ids != nullptr ? chunk_ids[blockIdx.x] : blockIdx.x;
@@ -92,7 +100,7 @@ __global__ void __launch_bounds__(THREADS)
   const uint2 st_in = pass == 0 ? make_uint2(0u, L.k) : state[pair];
   const uint32_t want = pass == 0 ? 0u : (st_in.x >> prev_shift);
   const bool last_pass = pass == N_PASSES - 1;
-  for (int b = threadIdx.x; b < nb; b += THREADS) sh[b] = 0;
+  for (int b = threadIdx.x; b < nb; b += (NW * 32)) sh[b] = 0;
   if (threadIdx.x == 0) sh_above = 0;
   __syncthreads();
   uint32_t above = 0;  // keys whose higher digits already exceed the prefix (needed in the last pass only)
@@ -105,7 +113,7 @@ __global__ void __launch_bounds__(THREADS)
     // Conservation check: the stored entries that reach the guess are counted again here and must add up
     // to the number the streaming pass counted when it stored them (k_find_digit compares).
     uint32_t c0 = 0, c1 = 0, c2 = 0, ge = 0;
-    for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
+    for_each_candidate<NW>(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
       const uint32_t d = (key >> shift) - g0;
       c0 += d == 0u ? 1u : 0u;
       c1 += d == 1u ? 1u : 0u;
@@ -127,7 +135,7 @@ __global__ void __launch_bounds__(THREADS)
       if (ge && reach_seen != nullptr) atomicAdd(&reach_seen[pair], ge);
     }
   } else if (pair_is_cand(pi, L.k)) {
-    for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
+    for_each_candidate<NW>(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
       const uint32_t hi_part = key >> prev_shift;
       if (hi_part == want) atomicAdd(&sh[(key >> shift) & (nb - 1)], 1u);
       above += hi_part > want ? 1u : 0u;
@@ -135,10 +143,10 @@ __global__ void __launch_bounds__(THREADS)
   } else {
     const uint64_t lo = c.a, hi = lo + c.len;
     const uint64_t s0 = lo & ~3ull;
-    const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+    const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + (NW * 32) * 4 - 1) / ((NW * 32) * 4));
     const float* a = acc + static_cast<uint64_t>(w) * N;
     for (uint32_t it = 0; it < n_iter; ++it) {
-      const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+      const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * (NW * 32) + threadIdx.x) * 4;
       float av[4], wv[4];
       load4<VEC>(a, e0, lo, hi, av);
       load4<VEC>(weights, e0, lo, hi, wv);
@@ -160,20 +168,29 @@ __global__ void __launch_bounds__(THREADS)
   }
   __syncthreads();
   uint32_t* gh = hist + static_cast<uint64_t>(pair) * NBINS;
-  for (int b = threadIdx.x; b < nb; b += THREADS) {
+  for (int b = threadIdx.x; b < nb; b += (NW * 32)) {
     const uint32_t v = sh[b];
     if (v) atomicAdd(&gh[b], v);
   }
   if (last_pass && chunk_sfx != nullptr) {  // suffix sums S[b] = sum of this chunk's bins >= b, and the count above the prefix
-    static_assert(pass_bins(N_PASSES - 1) == THREADS * 4, "four bins per thread in the last pass");
-    const uint32_t h0 = sh[threadIdx.x * 4], h1 = sh[threadIdx.x * 4 + 1], h2 = sh[threadIdx.x * 4 + 2],
-                   h3 = sh[threadIdx.x * 4 + 3];
+    constexpr int BPT = pass_bins(N_PASSES - 1) / (NW * 32);  // bins per thread in the last pass
+    static_assert(BPT % 4 == 0 && BPT * (NW * 32) == pass_bins(N_PASSES - 1), "whole 128-bit groups of bins per thread");
+    uint32_t h[BPT], mine = 0;
+#pragma unroll
+    for (int q = 0; q < BPT; ++q) {
+      h[q] = sh[threadIdx.x * BPT + q];
+      mine += h[q];
+    }
     uint32_t total;
-    const uint32_t before = block_excl_scan(h0 + h1 + h2 + h3, sh_warp, total);
-    const uint32_t s0 = total - before;
-    uint4 sfx = make_uint4(s0, s0 - h0, s0 - h0 - h1, s0 - h0 - h1 - h2);
+    const uint32_t before = block_excl_scan<NW>(mine, sh_warp, total);
+    uint32_t run = total - before;  // sum of the bins >= this thread's first one
     uint32_t* dst = chunk_sfx + (static_cast<uint64_t>(w) * n_chunks + ci) * pass_bins(N_PASSES - 1);
-    reinterpret_cast<uint4*>(dst)[threadIdx.x] = sfx;
+#pragma unroll
+    for (int q = 0; q < BPT; q += 4) {
+      const uint4 sfx = make_uint4(run, run - h[q], run - h[q] - h[q + 1], run - h[q] - h[q + 1] - h[q + 2]);
+      reinterpret_cast<uint4*>(dst)[(threadIdx.x * BPT + q) >> 2] = sfx;
+      run -= h[q] + h[q + 1] + h[q + 2] + h[q + 3];
+    }
     if (threadIdx.x == 0) chunk_cnt[static_cast<uint64_t>(w) * n_chunks + ci] = make_uint2(sh_above, 0u);
   }
 }
@@ -181,20 +198,21 @@ __global__ void __launch_bounds__(THREADS)
 // Digit decision for (worker, layer) pairs of the tiled path; grid = (tiled layers, covered workers).
 // Reads the pair's histogram, clears it for the next pass, extends the key prefix.
 // After the last pass state = (threshold key T, number r of T-valued elements to keep).
-__global__ void __launch_bounds__(THREADS)
+template <int NW>
+__global__ void __launch_bounds__(NW * 32, 512 / (NW * 32) * 2)
     k_find_digit(uint2* __restrict__ state, uint32_t* __restrict__ hist, const LayerDesc* __restrict__ layers,
                  const uint32_t* __restrict__ large_ids, const PairInfo* __restrict__ info,
                  uint32_t* __restrict__ reach_seen, int* __restrict__ status, int W, int pass, WorkerSel ws,
                  const uint32_t* __restrict__ large_sel) {
   __shared__ uint32_t sh[NBINS];
-  __shared__ uint32_t sh_scan[THREADS];
+  __shared__ uint32_t sh_scan[(NW * 32)];
   __shared__ uint32_t res[4];
   // the tiled layers this launch covers: all of them, or (large_sel) those the chain selects
   const uint32_t li = large_sel != nullptr ? large_sel[blockIdx.x] : blockIdx.x;
   const uint32_t pair = li * static_cast<uint32_t>(W) + static_cast<uint32_t>(sel_worker(ws, static_cast<int>(blockIdx.y)));
   const int nb = pass_bins(pass), shift = pass_shift(pass);
   uint32_t* gh = hist + static_cast<uint64_t>(pair) * NBINS;
-  for (int b = threadIdx.x; b < nb; b += THREADS) {
+  for (int b = threadIdx.x; b < nb; b += (NW * 32)) {
     sh[b] = gh[b];
     gh[b] = 0;
   }
@@ -206,9 +224,9 @@ __global__ void __launch_bounds__(THREADS)
     if (DEBUG_CHECKS && info != nullptr && !pair_is_cand(info[pair], krem)) {
       // multi-pass path: the first histogram pass counted every element of the layer exactly once
       uint32_t part = 0;
-      for (int b = threadIdx.x; b < nb; b += THREADS) part += sh[b];
+      for (int b = threadIdx.x; b < nb; b += (NW * 32)) part += sh[b];
       uint32_t total;
-      block_excl_scan(part, sh_scan, total);
+      block_excl_scan<NW>(part, sh_scan, total);
       if (threadIdx.x == 0) IWP_DBG_CHECK(status, total == layers[large_ids[pair / W]].n);
     }
     if (threadIdx.x == 0 && reach_seen != nullptr) {
@@ -224,7 +242,7 @@ __global__ void __launch_bounds__(THREADS)
     prefix = s.x;
     krem = s.y;
   }
-  find_digit(sh, nb, krem, sh_scan, res);
+  find_digit<(NW * 32)>(sh, nb, krem, sh_scan, res);
   if (threadIdx.x == 0) {
     if (res[2]) {
       state[pair] = make_uint2(prefix | (res[0] << shift), res[1]);
@@ -237,7 +255,7 @@ __global__ void __launch_bounds__(THREADS)
 
 // Per chunk: how many keys are above the threshold and how many equal it.  grid = (chunks, W).
 template <bool VEC>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(SEL_THREADS, 8)
     k_count(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
             const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
             const uint32_t* __restrict__ cand_key, const uint32_t* __restrict__ cand_cnt, const uint2* __restrict__ state,
@@ -259,10 +277,10 @@ __global__ void __launch_bounds__(THREADS)
   } else {
     const uint64_t lo = c.a, hi = lo + c.len;
     const uint64_t s0 = lo & ~3ull;
-    const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+    const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + SEL_THREADS * 4 - 1) / (SEL_THREADS * 4));
     const float* a = acc + static_cast<uint64_t>(w) * N;
     for (uint32_t it = 0; it < n_iter; ++it) {
-      const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+      const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * SEL_THREADS + threadIdx.x) * 4;
       float av[4], wv[4];
       load4<VEC>(a, e0, lo, hi, av);
       load4<VEC>(weights, e0, lo, hi, wv);
@@ -293,8 +311,9 @@ __global__ void __launch_bounds__(THREADS)
 // An element is selected if key > T, or key == T and fewer than r T-valued elements of the
 // layer precede it; its list position is (#greater before it) + min(#equal before it, r).
 // grid = (chunks, W).
-template <bool VEC>
-__global__ void __launch_bounds__(THREADS)
+// NW warps per CTA (4: fits beside the streaming pass; 8: half the latency).
+template <bool VEC, int NW>
+__global__ void __launch_bounds__(NW * 32, 512 / (NW * 32) * 2)
     k_write(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
             const Tile* __restrict__ tiles, const LayerDesc* __restrict__ layers, const PairInfo* __restrict__ info,
             const uint32_t* __restrict__ cand_key, const float* __restrict__ cand_val,
@@ -303,7 +322,7 @@ __global__ void __launch_bounds__(THREADS)
             float* __restrict__ sel_val, uint32_t* __restrict__ sel_slot, const uint32_t* __restrict__ chunk_sfx,
             int* __restrict__ status, float eps, uint64_t N, uint64_t K, int W, uint32_t n_chunks, int leader,
             WorkerSel ws, const int32_t* __restrict__ layer_leader, const uint32_t* __restrict__ chunk_ids) {
-  __shared__ uint32_t sh_warp[WARPS];
+  __shared__ uint32_t sh_warp[NW];
   __shared__ uint32_t sh_base[2];
   const uint32_t ci = chunk_ids != nullptr ? chunk_ids[blockIdx.x] : blockIdx.x;
   const Chunk c = chunks[ci];
@@ -318,7 +337,7 @@ __global__ void __launch_bounds__(THREADS)
   {
     const uint2* cc = chunk_cnt + static_cast<uint64_t>(w) * n_chunks;
     uint32_t g = 0, q = 0;
-    for (uint32_t j = c.first_chunk_of_layer + threadIdx.x; j < ci; j += THREADS) {
+    for (uint32_t j = c.first_chunk_of_layer + threadIdx.x; j < ci; j += (NW * 32)) {
       const uint2 v = cc[j];
       if (chunk_sfx == nullptr) {  // (#keys > T, #keys == T) of the chunk, counted by a kernel of its own
         g += v.x;
@@ -353,7 +372,7 @@ __global__ void __launch_bounds__(THREADS)
     // tiles front to back, ranking the entries of a slot with one warp scan per 128 entries
     const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t my_gt = 0, my_eq = 0;
-    for_each_candidate(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
+    for_each_candidate<NW>(c, w, W, cand_cnt, cand_key, [&](uint32_t key) {
       my_gt += key > T ? 1u : 0u;
       my_eq += key == T ? 1u : 0u;
     });
@@ -362,7 +381,7 @@ __global__ void __launch_bounds__(THREADS)
       my_gt += __shfl_xor_sync(0xffffffffu, my_gt, d);
       my_eq += __shfl_xor_sync(0xffffffffu, my_eq, d);
     }
-    __shared__ uint32_t sh_wg[WARPS], sh_we[WARPS];
+    __shared__ uint32_t sh_wg[NW], sh_we[NW];
     if (lane == 0) {
       sh_wg[warp] = my_gt;
       sh_we[warp] = my_eq;
@@ -374,8 +393,8 @@ __global__ void __launch_bounds__(THREADS)
       q_before += sh_we[q];
     }
     if ((my_gt | my_eq) == 0) return;  // nothing of this warp's tiles is selected
-    const uint32_t t_begin = min(c.n_tiles, warp * tiles_per_warp(c));
-    const uint32_t t_end = min(c.n_tiles, t_begin + tiles_per_warp(c));
+    const uint32_t t_begin = min(c.n_tiles, warp * tiles_per_warp<NW>(c));
+    const uint32_t t_end = min(c.n_tiles, t_begin + tiles_per_warp<NW>(c));
     // ranks the entries [j0, j0 + 128) of one slot with a warp scan and writes the selected ones
     auto emit = [&](uint32_t tile, uint64_t tw, uint32_t cnt, uint32_t tile_base, uint32_t j0, uint4 k) {
       const uint32_t j = j0 + lane * 4;
@@ -459,10 +478,10 @@ __global__ void __launch_bounds__(THREADS)
 
   const uint64_t lo = c.a, hi = lo + c.len;
   const uint64_t s0 = lo & ~3ull;
-  const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + THREADS * 4 - 1) / (THREADS * 4));
+  const uint32_t n_iter = static_cast<uint32_t>((hi - s0 + (NW * 32) * 4 - 1) / ((NW * 32) * 4));
   const float* a = acc + static_cast<uint64_t>(w) * N;
   for (uint32_t it = 0; it < n_iter; ++it) {
-    const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * THREADS + threadIdx.x) * 4;
+    const uint64_t e0 = s0 + (static_cast<uint64_t>(it) * (NW * 32) + threadIdx.x) * 4;
     float av[4], wv[4];
     load4<VEC>(a, e0, lo, hi, av);
     load4<VEC>(weights, e0, lo, hi, wv);
@@ -477,7 +496,7 @@ __global__ void __launch_bounds__(THREADS)
     }
     uint32_t total;
     const uint32_t packed = static_cast<uint32_t>(__popc(fg)) | (static_cast<uint32_t>(__popc(fe)) << 16);
-    const uint32_t ex = block_excl_scan(packed, sh_warp, total);
+    const uint32_t ex = block_excl_scan<NW>(packed, sh_warp, total);
     uint32_t g_before = run_gt + (ex & 0xffffu), q_before = run_eq + (ex >> 16);
     if (fg | fe) {
 #pragma unroll
