@@ -1004,13 +1004,11 @@ int run_step_threshold(iwp_ctx* c, const float* grads, const float* weights, flo
   stage_mark_at(c, 2);
   const uint32_t n_layers = static_cast<uint32_t>(p.layers.size());
   if (c->layerwise) {
-    // Eq. 4 needs the accumulated residuals first: step (a) for the chosen nodes, their exact moments, the
-    // thresholds, and only then the masks
-    k_thr_accumulate_chosen<VEC><<<n_tiles, THREADS, 0, s>>>(grads, c->acc, c->d_tiles, N, c->momentum, ls);
-    IWP_LAUNCH_CHECK(c);
+    // Eq. 4 needs the accumulated residuals first: step (a) for the chosen nodes and their exact moments in one
+    // pass, the thresholds, and only then the masks
     stage_mark_at(c, 3);
-    k_thr_stats<VEC><<<dim3((n_chunks + STATS_GROUP - 1) / STATS_GROUP, static_cast<unsigned>(ls.n)), THREADS, 0, s>>>(
-        c->acc, weights, c->d_chunks, n_chunks, c->d_bins, c->eps, N, n_layers, ls);
+    k_thr_stats<VEC, true><<<dim3((n_chunks + STATS_GROUP - 1) / STATS_GROUP, static_cast<unsigned>(ls.n)), THREADS, 0, s>>>(
+        c->acc, grads, weights, c->d_chunks, n_chunks, c->d_bins, c->eps, N, n_layers, c->momentum, ls);
     IWP_LAUNCH_CHECK(c);
     k_thr_finalize<<<dim3(n_layers, static_cast<unsigned>(ls.n)), THREADS, 0, s>>>(c->d_bins, c->d_layers, c->d_thr_lw, n_layers,
                                                                                 c->lw_alpha, c->lw_beta, c->lw_c);

@@ -12,7 +12,8 @@ namespace iwp {
 // ---------------------------------------------------------------------------------------
 // Absolute-threshold mode: Algorithm 1 as printed.  Only the chosen nodes form masks, per layer
 // Mask = |G / w| > thr (strict; several nodes' masks are OR-ed), and the index set has whatever size
-// results.  A step: step (a) for the chosen nodes (k_thr_accumulate_chosen), two looks at their
+// results.  A step: step (a) for the chosen nodes (inside k_thr_mask_count, or k_thr_stats with layer-wise
+// thresholds), two looks at their
 // residuals - count per chunk, scan, stable compaction with one set bit per element - and one
 // streaming pass over all workers that does the rest (k_thr_fused).  thr_bits: the thresholds' fp32
 // patterns; a negative one (the layer-wise rule can produce it) passes everything, +inf nothing.
@@ -209,11 +210,13 @@ constexpr int LW_BINS = 384;  // 255 exponents, plus room for the 32-bit digits 
 // with one warp reduction and one shared-memory atomic per term.
 constexpr uint32_t STATS_GROUP = 1;  // chunks per CTA of k_thr_stats (more were measured slower: the pass wants many CTAs)
 
-template <bool VEC>
+// ACCUM: the pass is also step (a) for the chosen nodes (it reads their gradients and writes their residuals back),
+// which saves the separate accumulate pass over them.
+template <bool VEC, bool ACCUM>
 __global__ void __launch_bounds__(THREADS)
-    k_thr_stats(const float* __restrict__ acc, const float* __restrict__ weights, const Chunk* __restrict__ chunks,
-                uint32_t n_chunks, unsigned long long* __restrict__ bins, float eps, uint64_t N, uint32_t n_layers,
-                LeaderSet ls) {
+    k_thr_stats(float* __restrict__ acc, const float* __restrict__ grads, const float* __restrict__ weights,
+                const Chunk* __restrict__ chunks, uint32_t n_chunks, unsigned long long* __restrict__ bins, float eps,
+                uint64_t N, uint32_t n_layers, float momentum, LeaderSet ls) {
   __shared__ unsigned long long sh[3 * LW_BINS];
   __shared__ uint32_t sh_exp[2];  // sum and count of the exponents sampled for the window
   const int j = blockIdx.y;
@@ -221,7 +224,8 @@ __global__ void __launch_bounds__(THREADS)
 #pragma unroll
   for (int q = 1; q < MAX_LEADERS; ++q)
     if (q == j) r = ls.r[q];
-  const float* a = acc + static_cast<uint64_t>(r) * N;
+  float* a = acc + static_cast<uint64_t>(r) * N;
+  const float* g = grads + static_cast<uint64_t>(r) * N;
   const int lane = threadIdx.x & 31;
   for (int b = threadIdx.x; b < 3 * LW_BINS; b += THREADS) sh[b] = 0ull;
   auto flush = [&](uint32_t layer) {  // this CTA's bins of one layer into the global ones; leaves them cleared
@@ -259,7 +263,8 @@ __global__ void __launch_bounds__(THREADS)
       uint32_t f = 0, cnt = 0;
       for (int q = 0; q < 4 && cnt == 0; ++q) {
         if (e + q >= lo && e + q < hi) {
-          const uint32_t key = imp_key(a[e + q], weights[e + q], eps);
+          const float v = ACCUM ? accumulate(a[e + q], g[e + q], momentum) : a[e + q];  // (not stored yet: read only)
+          const uint32_t key = imp_key(v, weights[e + q], eps);
           if (key != 0u && key < 0x7f800000u) {
             f = max(key >> 23, 1u);
             cnt = 1;
@@ -282,6 +287,13 @@ __global__ void __launch_bounds__(THREADS)
       float av[4], wv[4];
       load4<VEC>(a, e0, lo, hi, av);
       load4<VEC>(weights, e0, lo, hi, wv);
+      if (ACCUM) {
+        float gv[4];
+        load4_stream<VEC>(g, e0, lo, hi, gv);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) av[q] = accumulate(av[q], gv[q], momentum);
+        store4<VEC>(a, e0, lo, hi, av);
+      }
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const uint64_t e = e0 + q;
@@ -399,35 +411,6 @@ __global__ void __launch_bounds__(THREADS)
   thr_bits[j * n_layers + layer] = __float_as_uint(thr);
 }
 
-// Threshold mode, first pass: step (a) for the chosen nodes only (their masks are needed before anybody
-// else's residual is touched).  grid = tiles.
-template <bool VEC>
-__global__ void __launch_bounds__(THREADS)
-    k_thr_accumulate_chosen(const float* __restrict__ grads, float* __restrict__ acc, const Tile* __restrict__ tiles,
-                            uint64_t N, float momentum, LeaderSet ls) {
-  const Tile t = tiles[blockIdx.x];
-  const uint64_t lo = t.a, hi = lo + t.len;
-  const uint64_t base = lo & ~static_cast<uint64_t>(TILE - 1);
-  constexpr int SPT = TILE / 4 / THREADS;
-  for (int j = 0; j < ls.n; ++j) {
-    const float* g = grads + static_cast<uint64_t>(ls.r[j]) * N;
-    float* a = acc + static_cast<uint64_t>(ls.r[j]) * N;
-    float gv[SPT][4], av[SPT][4];
-#pragma unroll
-    for (int s = 0; s < SPT; ++s) {
-      const uint64_t e0 = base + static_cast<uint64_t>(s * THREADS + threadIdx.x) * 4;
-      load4_stream<VEC>(g, e0, lo, hi, gv[s]);
-      load4_stream<VEC>(a, e0, lo, hi, av[s]);
-    }
-#pragma unroll
-    for (int s = 0; s < SPT; ++s) {
-      const uint64_t e0 = base + static_cast<uint64_t>(s * THREADS + threadIdx.x) * 4;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) av[s][c] = accumulate(av[s][c], gv[s][c], momentum);
-      store4<VEC>(a, e0, lo, hi, av[s]);
-    }
-  }
-}
 
 // Threshold mode, last pass: everything that is left of the step in ONE streaming pass over all
 // workers, in ascending worker order per element: step (a) for the workers that are not chosen nodes,
