@@ -70,10 +70,11 @@ struct iwp_ctx {
   // The three select chains of the overlapped schedule.  Histogram and digit kernels with four warps per CTA (64
   // registers a thread) fit into the registers the streaming pass leaves free on an SM, so they take no CTA slot
   // from it, but take longer; the chain of the next step's chosen node is waited for by that step's first launch
-  // and keeps eight warps; the compaction always does (with four it takes twice as long and the next step waits).
-  // Measured, ms per step on the AlexNet shape W=8 / the ResNet-50 shape: all eight 1.294 / 0.700; this choice
-  // 1.293 / 0.678; four everywhere in the histogram kernels 1.306 / 0.673.
-  ChainWidth cw_lead{4, 8}, cw_next{8, 8}, cw_rest{4, 8};
+  // and keeps eight warps there and runs its compaction with sixteen warps per CTA (half the latency again); the other compactions keep eight
+  // (with four they take twice as long and the next step waits).  Measured, ms per step on the AlexNet shape
+  // W=8 / the ResNet-50 shape: eight warps everywhere 1.294 / 0.700; this choice 1.288 / 0.668; four everywhere in
+  // the histogram kernels 1.306 / 0.673; sixteen in every compaction 1.292 / 0.673.
+  ChainWidth cw_lead{4, 8}, cw_next{8, 16}, cw_rest{4, 8};
   int32_t predicted_next = -1;                 // the worker whose select pending_a2 covers
   int32_t last_only = -1;                      // the last step selected for this worker alone (-1: for every worker)
   float* saved_w = nullptr;                    // [N] weights kept for deferred selects that fall back (k_save_weights)
@@ -442,12 +443,16 @@ int select_and_write_w(iwp_ctx* c, const float* weights, cudaStream_t st, Worker
 // the compaction) for the others.
 template <bool VEC>
 int select_and_write(iwp_ctx* c, const float* weights, cudaStream_t st, WorkerSel ws, int32_t leader, ChainWidth cw) {
-  if (cw.hist == 4) {
-    return cw.write == 4 ? select_and_write_w<VEC, 4, 4>(c, weights, st, ws, leader)
-                         : select_and_write_w<VEC, 4, 8>(c, weights, st, ws, leader);
+  if (cw.hist == 16) {
+    return cw.write == 16 ? select_and_write_w<VEC, 16, 16>(c, weights, st, ws, leader)
+                          : select_and_write_w<VEC, 16, 8>(c, weights, st, ws, leader);
   }
-  return cw.write == 4 ? select_and_write_w<VEC, 8, 4>(c, weights, st, ws, leader)
-                       : select_and_write_w<VEC, 8, 8>(c, weights, st, ws, leader);
+  if (cw.hist == 4) {
+    return cw.write == 16 ? select_and_write_w<VEC, 4, 16>(c, weights, st, ws, leader)
+                          : select_and_write_w<VEC, 4, 8>(c, weights, st, ws, leader);
+  }
+  return cw.write == 16 ? select_and_write_w<VEC, 8, 16>(c, weights, st, ws, leader)
+                        : select_and_write_w<VEC, 8, 8>(c, weights, st, ws, leader);
 }
 
 int32_t leader_of_step(const iwp_ctx* c, int64_t t) {

@@ -174,7 +174,7 @@ __global__ void __launch_bounds__(NW * 32, 512 / (NW * 32) * 2)
   }
   if (last_pass && chunk_sfx != nullptr) {  // suffix sums S[b] = sum of this chunk's bins >= b, and the count above the prefix
     constexpr int BPT = pass_bins(N_PASSES - 1) / (NW * 32);  // bins per thread in the last pass
-    static_assert(BPT % 4 == 0 && BPT * (NW * 32) == pass_bins(N_PASSES - 1), "whole 128-bit groups of bins per thread");
+    static_assert(BPT >= 2 && BPT * (NW * 32) == pass_bins(N_PASSES - 1), "a whole number of bins per thread");
     uint32_t h[BPT], mine = 0;
 #pragma unroll
     for (int q = 0; q < BPT; ++q) {
@@ -185,11 +185,19 @@ __global__ void __launch_bounds__(NW * 32, 512 / (NW * 32) * 2)
     const uint32_t before = block_excl_scan<NW>(mine, sh_warp, total);
     uint32_t run = total - before;  // sum of the bins >= this thread's first one
     uint32_t* dst = chunk_sfx + (static_cast<uint64_t>(w) * n_chunks + ci) * pass_bins(N_PASSES - 1);
+    if constexpr (BPT % 4 == 0) {
 #pragma unroll
-    for (int q = 0; q < BPT; q += 4) {
-      const uint4 sfx = make_uint4(run, run - h[q], run - h[q] - h[q + 1], run - h[q] - h[q + 1] - h[q + 2]);
-      reinterpret_cast<uint4*>(dst)[(threadIdx.x * BPT + q) >> 2] = sfx;
-      run -= h[q] + h[q + 1] + h[q + 2] + h[q + 3];
+      for (int q = 0; q < BPT; q += 4) {
+        const uint4 sfx = make_uint4(run, run - h[q], run - h[q] - h[q + 1], run - h[q] - h[q + 1] - h[q + 2]);
+        reinterpret_cast<uint4*>(dst)[(threadIdx.x * BPT + q) >> 2] = sfx;
+        run -= h[q] + h[q + 1] + h[q + 2] + h[q + 3];
+      }
+    } else {
+#pragma unroll
+      for (int q = 0; q < BPT; q += 2) {
+        reinterpret_cast<uint2*>(dst)[(threadIdx.x * BPT + q) >> 1] = make_uint2(run, run - h[q]);
+        run -= h[q] + h[q + 1];
+      }
     }
     if (threadIdx.x == 0) chunk_cnt[static_cast<uint64_t>(w) * n_chunks + ci] = make_uint2(sh_above, 0u);
   }
