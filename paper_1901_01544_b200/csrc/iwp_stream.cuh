@@ -121,9 +121,7 @@ __global__ void __launch_bounds__(THREADS, 3)
     tile_id = blockIdx.x * WARPS + warp;
     if (tile_id >= n_tiles) return;
   } else {  // up to eight of the other workers of one tile per CTA: the tile's weights come through L1
-    // back to front: the chosen node's launch went front to back, so the weights and the record of the last tiles it
-    // touched are still in the L2 when this launch starts with them
-    tile_id = n_tiles - 1 - blockIdx.x / worker_groups;
+    tile_id = blockIdx.x / worker_groups;
     wi = static_cast<int>(blockIdx.x % worker_groups) * static_cast<int>(blockDim.x >> 5) + warp;
     if (wi >= W - 1) return;
   }
