@@ -194,6 +194,46 @@ def test_options_stats_and_misuse():
     pr.close()  # idempotent
 
 
+def test_newer_options_join_and_wire_argument_checks():
+    sizes, W = [70000, 300], 3
+    N = sum(sizes)
+    pr = Pruner(sizes, W, 32.0, 1e-8, 0)
+    L = binding.lib()
+    h = pr._h
+    E = binding.IWP_ERR_INVALID
+    for key, bad in ((b"pair_select", 2), (b"pair_select", -2), (b"leader_only_select", 2), (b"reserve_timed_steps", -1),
+                     (b"overlap", 2)):
+        assert L.iwp_set_option(h, key, bad) == E
+    for key, ok in ((b"pair_select", -1), (b"pair_select", 1), (b"leader_only_select", 0), (b"reserve_timed_steps", 4)):
+        assert L.iwp_set_option(h, key, ok) == 0
+    assert L.iwp_join(None) == E and L.iwp_join(h) == 0
+    weights, grads = _inputs(W, N, 12)
+    pr.set_option("overlap", 1)
+    upd = pr.step(grads[0], weights)
+    pr.join()  # work enqueued now is behind every kernel of the step, the late selects included
+    done = torch.cuda.Event()
+    done.record()
+    done.synchronize()
+    assert pr.sync_status() == 0 and int(torch.count_nonzero(upd).item()) <= pr.K
+    # wire formats: NULL pointers, negative sizes, a mask buffer that is not 4-byte aligned
+    idx = pr.selection(pr.leader)[0]
+    bits = torch.zeros(binding.iwp_wire_mask_bytes(N) + 4, dtype=torch.uint8, device=DEV)
+    assert L.iwp_wire_pack(h, idx.data_ptr(), -1, bits.data_ptr()) == E
+    assert L.iwp_wire_pack(h, None, 5, bits.data_ptr()) == E
+    assert L.iwp_wire_pack(h, idx.data_ptr(), idx.numel(), bits.data_ptr() + 1) == E
+    assert L.iwp_wire_unpack(h, bits.data_ptr() + 2, idx.data_ptr(), idx.numel(), None) == E
+    assert L.iwp_wire_unpack(h, bits.data_ptr(), None, 5, None) == E
+    assert L.iwp_wire_pack(h, idx.data_ptr(), idx.numel(), bits.data_ptr()) == 0
+    n = C.c_int64(-1)
+    out = torch.empty_like(idx)
+    assert L.iwp_wire_unpack(h, bits.data_ptr(), out.data_ptr(), out.numel(), C.byref(n)) == 0
+    assert n.value == idx.numel() and torch.equal(out, idx)  # the list is ascending already
+    thr = Pruner(sizes, W, None, 1e-8, 0, thresholds=[1.0, 1.0])
+    assert L.iwp_set_option(thr._h, b"leader_only_select", 1) == E  # ratio-mode contexts only
+    thr.close()
+    pr.close()
+
+
 def test_single_read_path_is_taken_and_falls_back_when_it_must():
     sizes, W = [300000, 64, 40000], 4
     N = sum(sizes)
