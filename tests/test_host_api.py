@@ -82,8 +82,19 @@ def test_plan_sizes(L):
     assert (f["N"], f["K"]) == (1 << 30, 1073760) and f["tiled_layers"] == 96
     assert f["tiles"] >= (1 << 30) // 4096 and f["tiles"] <= (1 << 30) // 4096 + 96
     assert f["device_bytes"] >= 4 * 4 * (1 << 30)
+    # chunk size by job size: 128-tile chunks for the large jobs, 8-tile chunks for one small layer
+    assert a["tiles"] == 14889 and a["chunks"] == 121
+    one = binding.iwp_plan_sizes(wl.single_layer().layer_sizes, 4, 64.0)
+    assert (one["tiles"], one["chunks"]) == (256, 32)
+    assert f["chunks"] == 96 * 22  # 2731 tiles per layer in chunks of 128
     odd = binding.iwp_plan_sizes([5, 17, 40001], 3, 2.0)
     assert odd["N"] == 40023 and odd["vector_ok"] == 0 and odd["small_layers"] == 2 and odd["tiled_layers"] == 1
+
+
+def test_wire_mask_bytes_is_a_host_function(L):
+    assert binding.iwp_wire_mask_bytes(0) == 0 and binding.iwp_wire_mask_bytes(1) == 4
+    assert binding.iwp_wire_mask_bytes(32) == 4 and binding.iwp_wire_mask_bytes(33) == 8
+    assert binding.iwp_wire_mask_bytes(60965224) == 4 * ((60965224 + 31) // 32) and binding.iwp_wire_mask_bytes(-1) == -1
 
 
 def test_invalid_arguments_are_rejected_without_a_gpu(L):
