@@ -233,6 +233,18 @@ def test_scaled_configs(name, residual_every):
                residual_every=residual_every)
 
 
+@pytest.mark.parametrize("overlap", [1, 0])
+def test_long_run_into_the_steady_state(overlap):
+    # 150 steps over five cycled gradient batches, as the bench runs them: residuals pile up, the chosen node's set
+    # is zeroed on every worker step after step, thresholds settle.  The update is compared after every step, lists
+    # and residuals now and then and at the end.
+    c = _scaled_case("alexnet_w8")
+    weights = c.weights(DEV)
+    sets = [c.grads(t, DEV) for t in range(5)]
+    run_parity(c.layer_sizes, c.W, c.ratio, c.eps, c.seed, 150, weights, lambda t: sets[t % 5],
+               options={"overlap": overlap}, state_every=37, residual_every=74)
+
+
 def test_residuals_left_alone_between_steps_with_ties_and_fallbacks():
     # coarse values: some pairs fall back to the multi-pass select, others stay on the single-read
     # path; residuals are read only at the end, and the option switch in the middle forces a flush
