@@ -141,6 +141,21 @@ def test_one_tile_full_of_candidates_spread_over_its_segments(overlap):
     _run_checked([n], W, ratio, weights, lambda t: _randn((W, n), 51 + t, 1e-3), steps=3, overlap=overlap)
 
 
+@pytest.mark.parametrize("pair_select", [1, 0])
+def test_many_dense_tiles_in_a_row(pair_select):
+    # 640 tiles; the first eighty hold about 460 candidates each (380 zero weights at random places + the usual 2 %):
+    # 37 k candidate keys in the share of ONE CTA of the cluster select, more than the 16 k it keeps in shared memory
+    # (the rest is re-read from the slots), and slots of more than 128 entries in every one of those tiles for the chain
+    n, W, ratio = 640 * TILE, 2, 64.0
+    weights = _dense_weights(n, 23)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(7)
+    for tile in range(80):
+        pick = torch.randperm(TILE, generator=g, device=DEV)[:380] + tile * TILE
+        weights[pick] = 0.0
+    _run_checked([n], W, ratio, weights, lambda t: _randn((W, n), 71 + t, 1e-3), steps=2, overlap=0, pair_select=pair_select)
+
+
 def test_clustered_runs_with_ties_inside_the_run():
     # the run's importances are all equal (same residual, zero weight): the threshold falls inside the run when the
     # run is longer than k, and the lower indices must win

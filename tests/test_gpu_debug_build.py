@@ -23,7 +23,7 @@ def test_parity_cases_on_the_checked_build():
     assert which.returncode == 0 and which.stdout.strip().endswith("libiwp_debug.so"), which.stdout + which.stderr
     cases = ("test_random_values or test_many_ties or test_degenerate_layers or test_forced_scalar or test_exact_select "
              "or test_misaligned or test_random_shapes or test_zero_weight_block or test_run_lengths or "
-             "test_hot_gradient_run or test_union_of_several or test_leader_only_select")
+             "test_hot_gradient_run or test_many_dense or test_union_of_several or test_leader_only_select")
     r = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "tests/test_gpu_clustered.py", "-q", "-x",
                         "-m", "gpu", "-k", cases, "-p", "no:cacheprovider"], cwd=ROOT, env=env, capture_output=True, text=True)
     assert r.returncode == 0, r.stdout[-4000:] + r.stderr[-2000:]
